@@ -1,0 +1,401 @@
+"""Pins of the fp64 oracle against things other than itself.
+
+The paper prints no worked attention example, so the pins are mathematics: brute force on tiny
+inputs, closed forms, invariants that hold for any input, central finite differences, an
+independent library routine (torch float64 scaled_dot_product_attention + autograd), and the
+identity that merging the partials of any chunking reproduces unchunked attention.
+"""
+import numpy as np
+import pytest
+
+import hydra_workloads as hw
+import oracle
+
+DQK, DV = hw.D_QK, hw.D_V
+
+
+def rand_bits(rng, shape, scale=1.0):
+    return hw.f32_to_bf16_bits((scale * rng.standard_normal(shape)).astype(np.float32))
+
+
+def make(rng, lengths, h, scale=1.0):
+    T = int(sum(lengths))
+    return dict(q=rand_bits(rng, (T, h, DQK), scale), k=rand_bits(rng, (T, h, DQK), scale),
+                v=rand_bits(rng, (T, h, DV)), do=rand_bits(rng, (T, h, DV)), cu=hw.cu_seqlens(lengths))
+
+
+SCALE = np.float32(1.0 / np.sqrt(np.float32(DQK)))
+
+
+def full(x, causal=True):
+    out, lse = oracle.attn_fwd(x["q"], x["k"], x["v"], x["cu"], causal, SCALE)
+    dq, dk, dv = oracle.attn_bwd(x["q"], x["k"], x["v"], x["do"], x["cu"], causal, SCALE, out, lse)
+    return out, lse, dq, dk, dv
+
+
+# ---------------------------------------------------------------------------------------------
+# brute force: exp(s) / sum exp(s), no max subtraction, plain numpy, written independently
+# ---------------------------------------------------------------------------------------------
+def brute_force(x, causal=True):
+    q, k, v, g = (hw.bf16_bits_to_f64(x[n]) for n in ("q", "k", "v", "do"))
+    cu = x["cu"]
+    T, h, _ = q.shape
+    out = np.zeros((T, h, DV)); lse = np.zeros((h, T))
+    dq = np.zeros_like(q); dk = np.zeros_like(k); dv = np.zeros_like(v)
+    sc = float(SCALE)
+    for b in range(len(cu) - 1):
+        lo, hi = int(cu[b]), int(cu[b + 1])
+        L = hi - lo
+        if L == 0:
+            continue
+        mask = np.tril(np.ones((L, L))) if causal else np.ones((L, L))
+        for a in range(h):
+            S = sc * q[lo:hi, a] @ k[lo:hi, a].T
+            E = np.exp(S) * mask
+            Z = E.sum(1, keepdims=True)
+            P = E / Z
+            O = P @ v[lo:hi, a]
+            out[lo:hi, a] = O
+            lse[a, lo:hi] = np.log(Z[:, 0])
+            G = g[lo:hi, a]
+            dP = G @ v[lo:hi, a].T
+            D = (G * O).sum(1, keepdims=True)
+            dS = P * (dP - D)
+            dq[lo:hi, a] = sc * dS @ k[lo:hi, a]
+            dk[lo:hi, a] = sc * dS.T @ q[lo:hi, a]
+            dv[lo:hi, a] = P.T @ G
+    return out, lse, dq, dk, dv
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_brute_force_tiny(causal):
+    rng = np.random.default_rng(1)
+    x = make(rng, [1, 5, 17, 64, 0, 3], 2)
+    got = full(x, causal)
+    ref = brute_force(x, causal)
+    for g, r, name in zip(got, ref, ("out", "lse", "dq", "dk", "dv")):
+        np.testing.assert_allclose(g, r, rtol=1e-10, atol=1e-12, err_msg=name)
+
+
+# ---------------------------------------------------------------------------------------------
+# closed forms
+# ---------------------------------------------------------------------------------------------
+def test_length_one_sequences():
+    rng = np.random.default_rng(2)
+    x = make(rng, [1, 1, 1], 3)
+    out, lse, dq, dk, dv = full(x)
+    q, k, v, g = (hw.bf16_bits_to_f64(x[n]) for n in ("q", "k", "v", "do"))
+    np.testing.assert_allclose(out, v, rtol=0, atol=1e-15)
+    np.testing.assert_allclose(lse.T, float(SCALE) * (q * k).sum(-1), rtol=1e-14)
+    np.testing.assert_allclose(dv, g, rtol=0, atol=1e-15)
+    assert np.abs(dq).max() < 1e-14 and np.abs(dk).max() < 1e-14
+
+
+def test_zero_queries_give_prefix_means():
+    rng = np.random.default_rng(3)
+    L, h = 40, 2
+    x = make(rng, [L], h)
+    x["q"][:] = 0
+    out, lse, dq, dk, dv = full(x)
+    v, g = hw.bf16_bits_to_f64(x["v"]), hw.bf16_bits_to_f64(x["do"])
+    n = np.arange(1, L + 1, dtype=np.float64)
+    np.testing.assert_allclose(out, np.cumsum(v, 0) / n[:, None, None], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(lse, np.broadcast_to(np.log(n), (h, L)), rtol=1e-13)
+    # dV_j = sum_{i>=j} dO_i / (i+1)
+    want = np.cumsum((g / n[:, None, None])[::-1], 0)[::-1]
+    np.testing.assert_allclose(dv, want, rtol=1e-12, atol=1e-14)
+    assert np.abs(dk).max() < 1e-14       # q = 0  =>  dK = scale * dS^T q = 0
+
+
+def test_constant_keys():
+    rng = np.random.default_rng(4)
+    L, h = 33, 2
+    x = make(rng, [L], h)
+    x["k"][:] = x["k"][0:1]
+    out, lse, dq, dk, dv = full(x)
+    q, k, v = (hw.bf16_bits_to_f64(x[n]) for n in ("q", "k", "v"))
+    n = np.arange(1, L + 1, dtype=np.float64)
+    np.testing.assert_allclose(out, np.cumsum(v, 0) / n[:, None, None], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(lse.T, float(SCALE) * (q * k).sum(-1) + np.log(n)[:, None], rtol=1e-12)
+    assert np.abs(dq).max() < 1e-13       # sum_j dS_ij = 0 and all k_j equal
+
+
+def test_constant_values():
+    rng = np.random.default_rng(5)
+    L, h = 29, 2
+    x = make(rng, [L], h)
+    x["v"][:] = x["v"][0:1, 0:1]
+    out, lse, dq, dk, dv = full(x)
+    v, g = hw.bf16_bits_to_f64(x["v"]), hw.bf16_bits_to_f64(x["do"])
+    np.testing.assert_allclose(out, v, rtol=1e-13, atol=1e-14)
+    assert np.abs(dq).max() < 1e-13 and np.abs(dk).max() < 1e-13
+    for a in range(h):
+        want = np.zeros((L, DV))
+        for i in range(L):
+            p = oracle.p_row(x["q"], x["k"], x["cu"], 0, a, i, True, SCALE)
+            want[: i + 1] += p[:, None] * g[i, a][None, :]
+        np.testing.assert_allclose(dv[:, a], want, rtol=1e-11, atol=1e-13)
+
+
+def test_key_shift_invariance():
+    """k_j -> k_j + c leaves P, O and all gradients unchanged and moves LSE_i by scale <q_i, c>."""
+    rng = np.random.default_rng(6)
+    L, h = 24, 2
+    # small integers are exact in bf16 and stay exact after the shift
+    def ints(shape, lo, hi):
+        return hw.f32_to_bf16_bits(rng.integers(lo, hi, size=shape).astype(np.float32))
+    x = dict(q=ints((L, h, DQK), -2, 3), k=ints((L, h, DQK), -2, 3), v=rand_bits(rng, (L, h, DV)),
+             do=rand_bits(rng, (L, h, DV)), cu=hw.cu_seqlens([L]))
+    c = rng.integers(-2, 3, size=(1, h, DQK)).astype(np.float32)
+    y = dict(x)
+    y["k"] = hw.f32_to_bf16_bits(hw.bf16_bits_to_f32(x["k"]) + c)
+    a, b = full(x), full(y)
+    for i in (0, 2, 3, 4):
+        np.testing.assert_allclose(a[i], b[i], rtol=1e-9, atol=1e-11)
+    shift = float(SCALE) * (hw.bf16_bits_to_f64(x["q"]) * c.astype(np.float64)).sum(-1)
+    np.testing.assert_allclose(b[1] - a[1], shift.T, rtol=1e-10, atol=1e-11)
+
+
+def test_peaked_limit_selects_one_key():
+    rng = np.random.default_rng(7)
+    L, h = 16, 1
+    x = make(rng, [L], h)
+    # distinct keys of equal norm: signed permutation-like patterns scaled to norm 8
+    k = np.zeros((L, h, DQK), dtype=np.float32)
+    for j in range(L):
+        k[j, 0, j * 4:(j * 4 + 4)] = 4.0
+    x["k"] = hw.f32_to_bf16_bits(k)
+    pi = np.array([rng.integers(0, i + 1) for i in range(L)])
+    beta = 64.0
+    x["q"] = hw.f32_to_bf16_bits(beta * k[pi])
+    out, lse = oracle.attn_fwd(x["q"], x["k"], x["v"], x["cu"], True, SCALE)
+    v = hw.bf16_bits_to_f64(x["v"])
+    np.testing.assert_allclose(out[:, 0], v[pi, 0], rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse[0], float(SCALE) * beta * 64.0, rtol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------
+# invariants for arbitrary inputs
+# ---------------------------------------------------------------------------------------------
+def test_probability_rows_sum_to_one():
+    rng = np.random.default_rng(8)
+    x = make(rng, [50, 21], 2)
+    for seq, i in ((0, 0), (0, 17), (0, 49), (1, 20)):
+        for a in range(2):
+            p = oracle.p_row(x["q"], x["k"], x["cu"], seq, a, i, True, SCALE)
+            assert len(p) == i + 1
+            assert abs(p.sum() - 1.0) < 1e-13
+            assert (p > 0).all()
+
+
+def test_gradient_invariants():
+    rng = np.random.default_rng(9)
+    lengths = [37, 64, 5]
+    x = make(rng, lengths, 3)
+    out, lse, dq, dk, dv = full(x)
+    q, k, g = (hw.bf16_bits_to_f64(x[n]) for n in ("q", "k", "do"))
+    cu = x["cu"]
+    for b in range(len(lengths)):
+        s = slice(int(cu[b]), int(cu[b + 1]))
+        # softmax is shift invariant along keys  =>  sum_j dK_j = scale * sum_i (sum_j dS_ij) q_i = 0
+        assert np.abs(dk[s].sum(0)).max() < 1e-12
+        # rows of P sum to one  =>  sum_j dV_j = sum_i dO_i
+        np.testing.assert_allclose(dv[s].sum(0), g[s].sum(0), rtol=1e-12, atol=1e-12)
+        # scores depend on q, k only through <q_i, k_j>
+        np.testing.assert_allclose((q[s] * dq[s]).sum((0, 2)), (k[s] * dk[s]).sum((0, 2)),
+                                   rtol=1e-10, atol=1e-12)
+
+
+def test_packing_and_head_independence():
+    rng = np.random.default_rng(10)
+    lengths = [9, 30, 14]
+    x = make(rng, lengths, 3)
+    ref = full(x)
+    cu = x["cu"]
+    s = slice(int(cu[1]), int(cu[2]))
+    alone = {n: x[n][s] for n in ("q", "k", "v", "do")}
+    alone["cu"] = hw.cu_seqlens([30])
+    got = full(alone)
+    for name, r, g_ in zip(("out", "lse", "dq", "dk", "dv"), ref, got):
+        r_slice = r[:, s] if name == "lse" else r[s]
+        assert np.array_equal(r_slice, g_), name
+    perm = [2, 0, 1]
+    y = {n: x[n][:, perm] for n in ("q", "k", "v", "do")}
+    y["cu"] = cu
+    got = full(y)
+    assert np.array_equal(got[0], ref[0][:, perm]) and np.array_equal(got[1], ref[1][perm])
+    assert np.array_equal(got[3], ref[3][:, perm])
+
+
+# ---------------------------------------------------------------------------------------------
+# finite differences (float64 inputs)
+# ---------------------------------------------------------------------------------------------
+def test_finite_differences():
+    rng = np.random.default_rng(11)
+    lengths = [33, 6]
+    T, h = sum(lengths), 1
+    cu = hw.cu_seqlens(lengths)
+    t = {n: rng.standard_normal((T, h, DQK if n in "qk" else DV)) for n in ("q", "k", "v", "do")}
+
+    def loss(tt):
+        with oracle.f64_inputs():
+            out, _ = oracle.attn_fwd(tt["q"], tt["k"], tt["v"], cu, True, SCALE)
+        return float((out * tt["do"]).sum())
+
+    with oracle.f64_inputs():
+        out, lse = oracle.attn_fwd(t["q"], t["k"], t["v"], cu, True, SCALE)
+        grads = dict(zip(("q", "k", "v"),
+                         oracle.attn_bwd(t["q"], t["k"], t["v"], t["do"], cu, True, SCALE, out, lse)))
+    eps = 1e-5
+    for name in ("q", "k", "v"):
+        g = grads[name]
+        idx = [tuple(rng.integers(0, s) for s in g.shape) for _ in range(24)]
+        idx += [(0, 0, 0), (T - 1, 0, 0), (32, 0, 5), (33, 0, 7)]
+        scale_ref = np.abs(g).max()
+        for ix in idx:
+            plus = {k_: v_.copy() for k_, v_ in t.items()}
+            minus = {k_: v_.copy() for k_, v_ in t.items()}
+            plus[name][ix] += eps
+            minus[name][ix] -= eps
+            fd = (loss(plus) - loss(minus)) / (2 * eps)
+            assert abs(fd - g[ix]) <= 1e-6 * scale_ref + 1e-9, (name, ix, fd, g[ix])
+
+
+# ---------------------------------------------------------------------------------------------
+# independent library routine
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("causal", [True, False])
+def test_against_torch_float64_sdpa(causal):
+    torch = pytest.importorskip("torch")
+    import torch.nn.functional as F
+    rng = np.random.default_rng(12)
+    lengths = [48, 7, 130]
+    h = 2
+    x = make(rng, lengths, h)
+    out, lse, dq, dk, dv = full(x, causal)
+    cu = x["cu"]
+    for b in range(len(lengths)):
+        s = slice(int(cu[b]), int(cu[b + 1]))
+        tq, tk, tv = (torch.tensor(hw.bf16_bits_to_f64(x[n][s]).transpose(1, 0, 2).copy(),
+                                   requires_grad=True) for n in ("q", "k", "v"))
+        tg = torch.tensor(hw.bf16_bits_to_f64(x["do"][s]).transpose(1, 0, 2).copy())
+        o = F.scaled_dot_product_attention(tq[None], tk[None], tv[None], is_causal=causal,
+                                           scale=float(SCALE))[0]
+        (o * tg).sum().backward()
+        np.testing.assert_allclose(out[s], o.detach().numpy().transpose(1, 0, 2), rtol=1e-10, atol=1e-12)
+        for mine, theirs in ((dq, tq), (dk, tk), (dv, tv)):
+            np.testing.assert_allclose(mine[s], theirs.grad.numpy().transpose(1, 0, 2),
+                                       rtol=1e-9, atol=1e-11)
+        sc = float(SCALE) * tq.detach() @ tk.detach().transpose(1, 2)
+        if causal:
+            L = lengths[b]
+            sc = sc.masked_fill(~torch.tril(torch.ones(L, L, dtype=torch.bool)), float("-inf"))
+        np.testing.assert_allclose(lse[:, s], torch.logsumexp(sc, -1).numpy(), rtol=1e-12, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------
+# partials and merge
+# ---------------------------------------------------------------------------------------------
+def _merged(x, pairs):
+    """Merge the oracle partials of `pairs` group by group into [T,h,dv] / [h,T]."""
+    T, h, _ = x["q"].shape
+    out = np.zeros((T, h, DV)); lse = np.full((h, T), -np.inf)
+    groups = {}
+    for p in pairs:
+        groups.setdefault(p["group"], []).append(p)
+    for plist in groups.values():
+        parts = [oracle.attn_partial(x["q"], x["k"], x["v"], x["cu"], p, True, SCALE) for p in plist]
+        o, l = oracle.lse_merge([a for a, _ in parts], [b for _, b in parts])
+        t0 = int(x["cu"][plist[0]["seq"]]) + plist[0]["q_start"]
+        out[t0:t0 + plist[0]["q_len"]] = o
+        lse[:, t0:t0 + plist[0]["q_len"]] = l
+    return out, lse
+
+
+@pytest.mark.parametrize("cp_r", [1, 2, 4])
+def test_merge_of_zigzag_partials_is_unchunked_attention(cp_r):
+    rng = np.random.default_rng(13)
+    lengths = [300, 37, 5, 64]
+    x = make(rng, lengths, 2)
+    pairs = oracle.causal_pairs(x["cu"], cp_r)
+    out, lse = oracle.attn_fwd(x["q"], x["k"], x["v"], x["cu"], True, SCALE)
+    mo, ml = _merged(x, pairs)
+    np.testing.assert_allclose(mo, out, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(ml, lse, rtol=1e-12, atol=1e-12)
+    # backward over the same pairs with the merged LSE and D equals the unchunked backward
+    d = oracle.bwd_prep(x["do"], out)
+    got = oracle.attn_bwd_pairs(x["q"], x["k"], x["v"], x["do"], x["cu"], pairs, True, SCALE, lse, d)
+    ref = oracle.attn_bwd(x["q"], x["k"], x["v"], x["do"], x["cu"], True, SCALE, out, lse)
+    for g_, r in zip(got, ref):
+        np.testing.assert_allclose(g_, r, rtol=1e-10, atol=1e-12)
+
+
+def test_merge_of_unequal_hand_made_chunks():
+    rng = np.random.default_rng(14)
+    L = 90
+    x = make(rng, [L], 2)
+    edges = [0, 1, 30, 31, 77, 90]
+    pairs = []
+    for qc in range(len(edges) - 1):
+        for kc in range(qc + 1):
+            pairs.append(dict(seq=0, q_start=edges[qc], q_len=edges[qc + 1] - edges[qc],
+                              k_start=edges[kc], k_len=edges[kc + 1] - edges[kc], group=qc))
+    out, lse = oracle.attn_fwd(x["q"], x["k"], x["v"], x["cu"], True, SCALE)
+    mo, ml = _merged(x, pairs)
+    np.testing.assert_allclose(mo, out, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(ml, lse, rtol=1e-12, atol=1e-12)
+
+
+def test_merge_identities():
+    rng = np.random.default_rng(15)
+    rows, h = 11, 3
+    o = [rng.standard_normal((rows, h, DV)) for _ in range(3)]
+    l = [rng.standard_normal((h, rows)) * 3 for _ in range(3)]
+    # one partial merges to itself
+    mo, ml = oracle.lse_merge(o[:1], l[:1])
+    assert np.array_equal(mo, o[0]) and np.array_equal(ml, l[0])
+    # (anything, -inf) is the identity element
+    dead = np.full((h, rows), -np.inf)
+    mo, ml = oracle.lse_merge([o[0], o[1]], [l[0], dead])
+    np.testing.assert_allclose(mo, o[0], rtol=1e-15); np.testing.assert_allclose(ml, l[0], rtol=1e-15)
+    # all -inf: O = 0, LSE = -inf, no NaN
+    mo, ml = oracle.lse_merge([o[0], o[1]], [dead, dead])
+    assert np.array_equal(mo, np.zeros_like(mo)) and np.isneginf(ml).all()
+    # commutative, associative, and equal to the direct weights formula
+    a, la = oracle.lse_merge(o, l)
+    b, lb = oracle.lse_merge(o[::-1], l[::-1])
+    np.testing.assert_allclose(a, b, rtol=1e-13, atol=1e-15); np.testing.assert_allclose(la, lb, rtol=1e-14)
+    c01, l01 = oracle.lse_merge(o[:2], l[:2])
+    c, lc = oracle.lse_merge([c01, o[2]], [l01, l[2]])
+    np.testing.assert_allclose(a, c, rtol=1e-12, atol=1e-14); np.testing.assert_allclose(la, lc, rtol=1e-13)
+    w = np.exp(np.stack(l))                     # direct formula, no max subtraction
+    want = (w.transpose(0, 2, 1)[..., None] * np.stack(o)).sum(0) / w.sum(0).T[..., None]
+    np.testing.assert_allclose(a, want, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(la, np.log(w.sum(0)), rtol=1e-13)
+
+
+def test_partial_with_no_admissible_key():
+    rng = np.random.default_rng(16)
+    x = make(rng, [20], 1)
+    p = dict(seq=0, q_start=0, q_len=5, k_start=10, k_len=10, group=0)   # keys all in the future
+    o, l = oracle.attn_partial(x["q"], x["k"], x["v"], x["cu"], p, True, SCALE)
+    assert np.array_equal(o, np.zeros_like(o)) and np.isneginf(l).all()
+
+
+# ---------------------------------------------------------------------------------------------
+# sampled rows / keys agree with the full computation
+# ---------------------------------------------------------------------------------------------
+def test_sampled_rows_and_keys_match_full():
+    rng = np.random.default_rng(17)
+    lengths = [70, 45]
+    x = make(rng, lengths, 2)
+    out, lse, dq, dk, dv = full(x)
+    tok = np.array([0, 1, 69, 70, 100, 114]); head = np.array([0, 1, 1, 0, 1, 0])
+    o, l, d, q_ = oracle.sample_rows(x["q"], x["k"], x["v"], x["do"], x["cu"], True, SCALE, tok, head)
+    np.testing.assert_allclose(o, out[tok, head], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(l, lse[head, tok], rtol=1e-13)
+    np.testing.assert_allclose(q_, dq[tok, head], rtol=1e-10, atol=1e-13)
+    np.testing.assert_allclose(d, (hw.bf16_bits_to_f64(x["do"]) * out).sum(-1)[tok, head], rtol=1e-12)
+    kk, vv = oracle.sample_keys(x["q"], x["k"], x["v"], x["do"], x["cu"], True, SCALE, tok, head)
+    np.testing.assert_allclose(kk, dk[tok, head], rtol=1e-10, atol=1e-13)
+    np.testing.assert_allclose(vv, dv[tok, head], rtol=1e-10, atol=1e-13)
