@@ -1,0 +1,185 @@
+/*
+ * hydra_attn.h - C ABI of the B200 (sm_100a) attention library.
+ *
+ * The library computes the per-GPU work that HyDra's context-parallel engine schedules: causal
+ * softmax attention, forward and backward, over variable-length packed sequences with one K/V head
+ * per query head (MLA with materialised K/V; d_qk = 192, d_v = 128), cut into the (q-chunk,
+ * kv-chunk) pairs of an outer ring, each pair emitting a partial (O, LSE), plus the log-sum-exp
+ * merge of the partials.
+ *
+ * Conventions that hold for every entry point
+ *   - "device" pointers are CUDA device memory of the current device, 16-byte aligned, contiguous;
+ *     "host" pointers are ordinary host memory, read during the call and free to reuse on return.
+ *   - Tensors: q, k, dq, dk [T, h, 192] bf16; v, out, dout, dv, o_part [rows, h, 128] bf16;
+ *     lse [h, T] fp32, lse_part [h, part_rows] fp32 (natural logarithm, softmax scale included).
+ *     T = cu_seqlens[n_seqs]; sequence b owns tokens [cu_seqlens[b], cu_seqlens[b+1]).
+ *   - Every call returns a status (HYDRA_OK = 0). Work is enqueued on `cuda_stream` (a
+ *     cudaStream_t passed as void*; NULL = the legacy default stream); results are valid once the
+ *     stream has been synchronised. No call synchronises the device except hydra_poll_status and,
+ *     the first time a given (cu_seqlens, pairs, h) combination is seen, the internal cudaMalloc of
+ *     its cached work lists (freed by hydra_shutdown).
+ *   - The caller owns all tensors and the workspace; the library keeps no caller pointer.
+ *   - Inputs must be finite: a tile that straddles the end of a sequence reads (and masks) the
+ *     rows of its neighbour, and 0 * NaN is NaN.
+ *   - Only compute capability 10.0 is supported; there is no fallback path.
+ */
+#ifndef HYDRA_ATTN_H
+#define HYDRA_ATTN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+#if defined(__GNUC__)
+#pragma GCC visibility push(default)
+#endif
+
+#define HYDRA_D_QK 192
+#define HYDRA_D_V 128
+
+enum {
+    HYDRA_OK = 0,
+    HYDRA_ERR_INVALID_ARG = 1,         /* null/misaligned pointer, bad cu_seqlens, bad pair      */
+    HYDRA_ERR_UNSUPPORTED = 2,         /* shape outside the compiled configuration               */
+    HYDRA_ERR_WORKSPACE_TOO_SMALL = 3,
+    HYDRA_ERR_CUDA = 4,                /* a CUDA runtime/driver call failed                      */
+    HYDRA_ERR_DEVICE_TIMEOUT = 5,      /* a bounded device-side wait gave up                     */
+    HYDRA_ERR_NOT_SM100 = 6            /* current device is not compute capability 10.x          */
+};
+
+enum { HYDRA_WS_FWD = 0, HYDRA_WS_MERGE = 1, HYDRA_WS_BWD = 2 };
+
+/*
+ * One (q-chunk, kv-chunk) pair of one sequence: the unit of work of a ring step (Section 5.2: the
+ * outer ring circulates K/V blocks and pipelines them with attention).  Offsets are local to the
+ * sequence. With causal != 0 a key at position k_start+j is visible to the query at position
+ * q_start+i iff k_start+j <= q_start+i (absolute positions; not "bottom-right aligned").
+ */
+typedef struct hydra_pair_t {
+    int32_t seq;       /* index into cu_seqlens                                                    */
+    int32_t q_start;   /* q rows  [q_start, q_start + q_len) of the sequence                       */
+    int32_t q_len;
+    int32_t k_start;   /* kv rows [k_start, k_start + k_len) of the sequence                       */
+    int32_t k_len;
+    int32_t part_row;  /* first row of this pair's partial in o_part / lse_part;                   */
+                       /* -1: the pair is alone in its group and writes out / lse directly         */
+    int32_t group;     /* merge group (the q chunk): pairs with equal ids share q_start/q_len and  */
+                       /* are merged; ids are non-decreasing along the array                       */
+    int32_t flags;     /* must be 0                                                                */
+} hydra_pair_t;
+
+/*
+ * Eq. (usp), Section 5.2: a context-parallel degree P over h heads is run as an inner Ulysses
+ * group cp_u = min(P, h) inside an outer ring cp_r = P / cp_u. The kernel of one rank then sees
+ * H / cp_u heads and sequences cut into 2 * cp_r zigzag chunks.
+ * Returns HYDRA_ERR_INVALID_ARG if degree or heads < 1 or cp_u does not divide degree.
+ */
+int32_t hydra_usp_factor(int32_t degree, int32_t heads, int32_t* cp_u, int32_t* cp_r);
+
+/*
+ * Chunk cutting and causal pair enumeration (host only, integers).
+ * Sequence b is cut into n_c = 2*cp_r[b] contiguous chunks with boundaries floor(c*L/n_c)
+ * (cp_r[b] == 0: not cut, one chunk); ring rank r owns chunks r and n_c-1-r; every pair
+ * (q chunk, kv chunk) with kv chunk <= q chunk and both non-empty is emitted, q chunks in order.
+ * Groups with one pair get part_row = -1, the others consecutive rows of the partial buffers.
+ *   cu_seqlens_host [n_seqs+1] host; cp_r_host [n_seqs] host, or NULL to use cp_r_all everywhere.
+ *   pairs_out       host array of capacity max_pairs (may be NULL with max_pairs = 0 to count).
+ *   n_pairs_out     number of pairs (always written); part_rows_out rows needed in o_part/lse_part.
+ *   rank_out, step_out  optional host arrays [max_pairs]: owner rank of the q chunk and ring step
+ *                   (rank(q chunk) - rank(kv chunk)) mod cp_r at which the K/V block visits.
+ * Returns HYDRA_ERR_INVALID_ARG on bad input, HYDRA_ERR_WORKSPACE_TOO_SMALL if max_pairs is too
+ * small (counts are still written).
+ */
+int32_t hydra_zigzag_pairs(const int32_t* cu_seqlens_host, int32_t n_seqs, const int32_t* cp_r_host,
+                           int32_t cp_r_all, hydra_pair_t* pairs_out, int32_t max_pairs,
+                           int32_t* n_pairs_out, int64_t* part_rows_out, int32_t* rank_out,
+                           int32_t* step_out);
+
+/*
+ * Bytes of device workspace the call `which` (HYDRA_WS_*) needs for this problem. pairs == NULL
+ * with n_pairs == 0 means one whole-sequence pair per sequence. Returns 0 on invalid input.
+ */
+size_t hydra_workspace_bytes(int32_t which, const int32_t* cu_seqlens_host, int32_t n_seqs,
+                             int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs);
+
+/*
+ * Forward attention of every listed pair (the attention kernel of Section 3.5, restricted to one
+ * ring step's blocks as in Section 5.2).  For pair p, head a and q row i:
+ *   s_j = softmax_scale * <q_i, k_j> over the visible keys j of the pair,
+ *   LSE = ln sum_j exp(s_j),  O = sum_j exp(s_j - LSE) v_j   (no visible key: O = 0, LSE = -inf).
+ * Pairs with part_row >= 0 write rows [part_row, part_row+q_len) of o_part / lse_part, pairs with
+ * part_row == -1 write their rows of out / lse.
+ *   q, k, v device bf16; cu_seqlens_host, pairs host; out, lse, o_part, lse_part device (the
+ *   partial buffers may be NULL when no pair uses them; out/lse likewise). part_rows = rows of the
+ *   partial buffers. workspace device, >= hydra_workspace_bytes(HYDRA_WS_FWD, ...).
+ * bf16 operands, fp32 accumulation. Rows not covered by any pair are left untouched.
+ */
+int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_t* cu_seqlens_host,
+                       int32_t n_seqs, int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs,
+                       int32_t causal, float softmax_scale, void* out, float* lse, void* o_part,
+                       float* lse_part, int64_t part_rows, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream);
+
+/*
+ * Log-sum-exp merge of the partials of every group with two or more pairs (the combination step
+ * of ring attention, Section 5.2):  LSE = ln sum_p exp(LSE_p),  O = sum_p exp(LSE_p - LSE) O_p,
+ * all n partials at once in fp32 with one rounding to bf16; a partial with LSE_p = -inf has weight
+ * zero; all -inf gives O = 0, LSE = -inf. Writes the group's rows of out / lse.
+ *   o_part, lse_part device (as written by hydra_attn_fwd); out, lse device.
+ */
+int32_t hydra_lse_merge(const void* o_part, const float* lse_part, int64_t part_rows,
+                        const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
+                        const hydra_pair_t* pairs, int32_t n_pairs, void* out, float* lse,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward of the listed pairs, given the MERGED out and lse and the upstream gradient dout:
+ *   D_i = <dout_i, out_i>;  P_ij = exp(s_ij - LSE_i);  dS_ij = P_ij (<dout_i, v_j> - D_i);
+ *   dq_i = scale sum_j dS_ij k_j;  dk_j = scale sum_i dS_ij q_i;  dv_j = sum_i P_ij dout_i,
+ * summed over all listed pairs that contain (i, j). The sums are accumulated on chip in fp32 and
+ * written once as bf16, so results are deterministic. Rows of dq covered by no q chunk and rows of
+ * dk/dv covered by no kv chunk are left untouched.
+ * Requirement: any two pairs of a sequence have q ranges that are identical or disjoint, and kv
+ * ranges that are identical or disjoint (true for chunk pairs); otherwise HYDRA_ERR_INVALID_ARG.
+ *   q, k, v, out, dout device bf16; lse device fp32; dq, dk, dv device bf16.
+ */
+int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* out,
+                       const float* lse, const void* dout, const int32_t* cu_seqlens_host,
+                       int32_t n_seqs, int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs,
+                       int32_t causal, float softmax_scale, void* dq, void* dk, void* dv,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Human-readable name of a status code (static storage). */
+const char* hydra_status_string(int32_t status);
+
+/*
+ * Synchronises `cuda_stream` and reports what the kernels of the last call that used `workspace`
+ * left in its status word: *device_status is HYDRA_OK or HYDRA_ERR_DEVICE_TIMEOUT, *detail the
+ * index of the work item that gave up (or -1). Returns HYDRA_ERR_CUDA if the stream is in error.
+ */
+int32_t hydra_poll_status(void* workspace, void* cuda_stream, int32_t* device_status,
+                          int64_t* detail);
+
+/* Kernel launches issued by this process so far (all entry points), for launch accounting. */
+int64_t hydra_launch_count(void);
+
+/*
+ * Debug knob: upper bound, in nanoseconds, of any single device-side wait (default 2e9). Waits that
+ * exceed it make the kernel record HYDRA_ERR_DEVICE_TIMEOUT and return.
+ */
+void hydra_set_wait_limit_ns(uint64_t ns);
+
+int32_t hydra_version(void);
+
+/* Frees the cached work lists (device and pinned host memory). Safe to call at any time. */
+void hydra_shutdown(void);
+
+#if defined(__GNUC__)
+#pragma GCC visibility pop
+#endif
+#ifdef __cplusplus
+}
+#endif
+#endif /* HYDRA_ATTN_H */

@@ -1,0 +1,249 @@
+"""ctypes binding of libhydra_attn.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels; there is no Python or CPU fallback.
+If the shared library is missing it is built with nvcc; if that fails, importing raises.
+Tensors are torch CUDA tensors (used for device memory and streams only) or raw device pointers.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Iterable, Optional, Sequence, Tuple
+
+import numpy as np
+
+from . import build as _build
+
+D_QK = 192
+D_V = 128
+
+HYDRA_OK = 0
+HYDRA_ERR_INVALID_ARG = 1
+HYDRA_ERR_UNSUPPORTED = 2
+HYDRA_ERR_WORKSPACE_TOO_SMALL = 3
+HYDRA_ERR_CUDA = 4
+HYDRA_ERR_DEVICE_TIMEOUT = 5
+HYDRA_ERR_NOT_SM100 = 6
+HYDRA_WS_FWD, HYDRA_WS_MERGE, HYDRA_WS_BWD = 0, 1, 2
+
+
+class hydra_pair_t(ctypes.Structure):
+    _fields_ = [("seq", ctypes.c_int32), ("q_start", ctypes.c_int32), ("q_len", ctypes.c_int32),
+                ("k_start", ctypes.c_int32), ("k_len", ctypes.c_int32), ("part_row", ctypes.c_int32),
+                ("group", ctypes.c_int32), ("flags", ctypes.c_int32)]
+
+
+PAIR_DTYPE = np.dtype([("seq", "<i4"), ("q_start", "<i4"), ("q_len", "<i4"), ("k_start", "<i4"),
+                       ("k_len", "<i4"), ("part_row", "<i4"), ("group", "<i4"), ("flags", "<i4")])
+
+
+class HydraError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {hydra_status_string(status)} ({status})")
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.build(force=bool(os.environ.get("HYDRA_REBUILD")))   # no-op when up to date
+    lib = ctypes.CDLL(path)
+    i32, i64, vp, f32 = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_float
+    sz = ctypes.c_size_t
+    lib.hydra_version.restype = i32
+    lib.hydra_status_string.restype = ctypes.c_char_p
+    lib.hydra_status_string.argtypes = [i32]
+    lib.hydra_launch_count.restype = i64
+    lib.hydra_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
+    lib.hydra_set_wait_limit_ns.restype = None
+    lib.hydra_shutdown.restype = None
+    lib.hydra_usp_factor.restype = i32
+    lib.hydra_usp_factor.argtypes = [i32, i32, vp, vp]
+    lib.hydra_zigzag_pairs.restype = i32
+    lib.hydra_zigzag_pairs.argtypes = [vp, i32, vp, i32, vp, i32, vp, vp, vp, vp]
+    lib.hydra_workspace_bytes.restype = sz
+    lib.hydra_workspace_bytes.argtypes = [i32, vp, i32, i32, vp, i32]
+    lib.hydra_attn_fwd.restype = i32
+    lib.hydra_attn_fwd.argtypes = [vp, vp, vp, vp, i32, i32, vp, i32, i32, f32, vp, vp, vp, vp, i64,
+                                   vp, sz, vp]
+    lib.hydra_lse_merge.restype = i32
+    lib.hydra_lse_merge.argtypes = [vp, vp, i64, vp, i32, i32, vp, i32, vp, vp, vp, sz, vp]
+    lib.hydra_attn_bwd.restype = i32
+    lib.hydra_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, i32, i32, f32, vp, vp, vp,
+                                   vp, sz, vp]
+    lib.hydra_poll_status.restype = i32
+    lib.hydra_poll_status.argtypes = [vp, vp, vp, vp]
+    return lib
+
+
+_lib = _load()
+LIBRARY_PATH = _build.OUT
+EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_set_wait_limit_ns",
+           "hydra_shutdown", "hydra_usp_factor", "hydra_zigzag_pairs", "hydra_workspace_bytes",
+           "hydra_attn_fwd", "hydra_lse_merge", "hydra_attn_bwd", "hydra_poll_status")
+
+
+# ------------------------------------------------------------------------------------------------
+# marshalling helpers
+# ------------------------------------------------------------------------------------------------
+def _ptr(x) -> Optional[int]:
+    """Device pointer of a torch tensor, or the integer / None passed through."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if not x.is_cuda or not x.is_contiguous():
+        raise ValueError("tensors must be contiguous CUDA tensors")
+    return x.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _cu(cu_seqlens) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
+
+
+def as_pairs(pairs) -> Optional[np.ndarray]:
+    """Accepts None, a structured array of PAIR_DTYPE, or an iterable of dicts / tuples."""
+    if pairs is None:
+        return None
+    if isinstance(pairs, np.ndarray) and pairs.dtype == PAIR_DTYPE:
+        return np.ascontiguousarray(pairs)
+    out = np.zeros(len(pairs), dtype=PAIR_DTYPE)
+    for i, p in enumerate(pairs):
+        if isinstance(p, dict):
+            for name in ("seq", "q_start", "q_len", "k_start", "k_len", "group"):
+                out[i][name] = p[name]
+            out[i]["part_row"] = p.get("part_row", -1)
+            out[i]["flags"] = p.get("flags", 0)
+        else:
+            out[i] = tuple(p)
+    return out
+
+
+def _pairs_arg(pairs) -> Tuple[Optional[int], int, Optional[np.ndarray]]:
+    arr = as_pairs(pairs)
+    if arr is None:
+        return None, 0, None
+    return arr.ctypes.data, len(arr), arr
+
+
+def _check(status: int, where: str) -> None:
+    if status != HYDRA_OK:
+        raise HydraError(status, where)
+
+
+# ------------------------------------------------------------------------------------------------
+# the C ABI, one Python function per entry point
+# ------------------------------------------------------------------------------------------------
+def hydra_version() -> int:
+    return int(_lib.hydra_version())
+
+
+def hydra_status_string(status: int) -> str:
+    return _lib.hydra_status_string(int(status)).decode()
+
+
+def hydra_launch_count() -> int:
+    return int(_lib.hydra_launch_count())
+
+
+def hydra_set_wait_limit_ns(ns: int) -> None:
+    _lib.hydra_set_wait_limit_ns(int(ns))
+
+
+def hydra_shutdown() -> None:
+    _lib.hydra_shutdown()
+
+
+def hydra_usp_factor(degree: int, heads: int) -> Tuple[int, int]:
+    u, r = ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(_lib.hydra_usp_factor(degree, heads, ctypes.addressof(u), ctypes.addressof(r)),
+           "hydra_usp_factor")
+    return u.value, r.value
+
+
+def hydra_zigzag_pairs(cu_seqlens, cp_r):
+    """Returns (pairs structured array, part_rows, rank array, step array)."""
+    cu = _cu(cu_seqlens)
+    n = len(cu) - 1
+    per_seq = None if isinstance(cp_r, (int, np.integer)) else np.ascontiguousarray(cp_r, dtype=np.int32)
+    all_r = int(cp_r) if per_seq is None else 0
+    n_pairs, part_rows = ctypes.c_int32(0), ctypes.c_int64(0)
+    s = _lib.hydra_zigzag_pairs(cu.ctypes.data, n, None if per_seq is None else per_seq.ctypes.data, all_r,
+                                None, 0, ctypes.addressof(n_pairs), ctypes.addressof(part_rows), None, None)
+    if s not in (HYDRA_OK, HYDRA_ERR_WORKSPACE_TOO_SMALL):
+        raise HydraError(s, "hydra_zigzag_pairs")
+    pairs = np.zeros(n_pairs.value, dtype=PAIR_DTYPE)
+    rank = np.zeros(n_pairs.value, dtype=np.int32)
+    step = np.zeros(n_pairs.value, dtype=np.int32)
+    if n_pairs.value:
+        _check(_lib.hydra_zigzag_pairs(cu.ctypes.data, n, None if per_seq is None else per_seq.ctypes.data,
+                                       all_r, pairs.ctypes.data, len(pairs), ctypes.addressof(n_pairs),
+                                       ctypes.addressof(part_rows), rank.ctypes.data, step.ctypes.data),
+               "hydra_zigzag_pairs")
+    return pairs, int(part_rows.value), rank, step
+
+
+def hydra_workspace_bytes(which: int, cu_seqlens, n_heads: int, pairs=None) -> int:
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    return int(_lib.hydra_workspace_bytes(which, cu.ctypes.data, len(cu) - 1, n_heads, pp, npairs))
+
+
+def hydra_attn_fwd(q, k, v, cu_seqlens, n_heads: int, pairs, causal: bool, softmax_scale: float, out, lse,
+                   o_part, lse_part, part_rows: int, workspace, workspace_bytes: Optional[int] = None,
+                   stream=None, check: bool = True) -> int:
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = _lib.hydra_attn_fwd(_ptr(q), _ptr(k), _ptr(v), cu.ctypes.data, len(cu) - 1, n_heads, pp, npairs,
+                            int(bool(causal)), ctypes.c_float(float(softmax_scale)), _ptr(out), _ptr(lse),
+                            _ptr(o_part), _ptr(lse_part), int(part_rows), _ptr(workspace),
+                            int(workspace_bytes), _stream(stream))
+    if check:
+        _check(s, "hydra_attn_fwd")
+    return s
+
+
+def hydra_lse_merge(o_part, lse_part, part_rows: int, cu_seqlens, n_heads: int, pairs, out, lse, workspace,
+                    workspace_bytes: Optional[int] = None, stream=None, check: bool = True) -> int:
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = _lib.hydra_lse_merge(_ptr(o_part), _ptr(lse_part), int(part_rows), cu.ctypes.data, len(cu) - 1,
+                             n_heads, pp, npairs, _ptr(out), _ptr(lse), _ptr(workspace),
+                             int(workspace_bytes), _stream(stream))
+    if check:
+        _check(s, "hydra_lse_merge")
+    return s
+
+
+def hydra_attn_bwd(q, k, v, out, lse, dout, cu_seqlens, n_heads: int, pairs, causal: bool,
+                   softmax_scale: float, dq, dk, dv, workspace, workspace_bytes: Optional[int] = None,
+                   stream=None, check: bool = True) -> int:
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = _lib.hydra_attn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout), cu.ctypes.data,
+                            len(cu) - 1, n_heads, pp, npairs, int(bool(causal)),
+                            ctypes.c_float(float(softmax_scale)), _ptr(dq), _ptr(dk), _ptr(dv),
+                            _ptr(workspace), int(workspace_bytes), _stream(stream))
+    if check:
+        _check(s, "hydra_attn_bwd")
+    return s
+
+
+def hydra_poll_status(workspace, stream=None) -> Tuple[int, int]:
+    st, detail = ctypes.c_int32(0), ctypes.c_int64(-1)
+    _check(_lib.hydra_poll_status(_ptr(workspace), _stream(stream), ctypes.addressof(st),
+                                  ctypes.addressof(detail)), "hydra_poll_status")
+    return st.value, detail.value

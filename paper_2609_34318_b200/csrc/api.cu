@@ -1,0 +1,698 @@
+// Host side of the C ABI: argument validation, chunk cutting (zigzag pairs), work-list planning
+// with a small cache, tensor-map encoding and kernel launches.
+#include <algorithm>
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <memory>
+#include <mutex>
+#include <vector>
+
+#include "hydra_internal.h"
+
+namespace hydra {
+namespace {
+
+std::atomic<int64_t> g_launches{0};
+std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};
+
+constexpr size_t kStatusBytes = 256;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---------------------------------------------------------------------------------------------
+// validated problem description
+// ---------------------------------------------------------------------------------------------
+struct Problem {
+    std::vector<int32_t> cu;
+    std::vector<hydra_pair_t> pairs;
+    int32_t n_seqs = 0, h = 0;
+    int64_t T = 0;
+};
+
+int32_t make_problem(const int32_t* cu, int32_t n_seqs, int32_t h, const hydra_pair_t* pairs,
+                     int32_t n_pairs, Problem& out)
+{
+    if (n_seqs < 0 || h < 1 || h > 65535 || (n_seqs > 0 && cu == nullptr)) return HYDRA_ERR_INVALID_ARG;
+    if ((pairs == nullptr) != (n_pairs == 0) || n_pairs < 0) return HYDRA_ERR_INVALID_ARG;
+    out.n_seqs = n_seqs;
+    out.h = h;
+    out.cu.assign(1, 0);
+    if (n_seqs > 0) {
+        out.cu.assign(cu, cu + n_seqs + 1);
+        if (out.cu[0] != 0) return HYDRA_ERR_INVALID_ARG;
+        for (int b = 0; b < n_seqs; ++b)
+            if (out.cu[b + 1] < out.cu[b]) return HYDRA_ERR_INVALID_ARG;
+    }
+    out.T = out.cu[n_seqs];
+    if (out.T > (int64_t{1} << 30)) return HYDRA_ERR_UNSUPPORTED;
+    out.pairs.clear();
+    if (pairs == nullptr) {
+        for (int b = 0; b < n_seqs; ++b) {
+            const int32_t len = out.cu[b + 1] - out.cu[b];
+            if (len == 0) continue;
+            out.pairs.push_back(hydra_pair_t{b, 0, len, 0, len, -1, b, 0});
+        }
+        return HYDRA_OK;
+    }
+    for (int i = 0; i < n_pairs; ++i) {
+        const hydra_pair_t& p = pairs[i];
+        if (p.seq < 0 || p.seq >= n_seqs || p.flags != 0) return HYDRA_ERR_INVALID_ARG;
+        const int64_t len = out.cu[p.seq + 1] - out.cu[p.seq];
+        if (p.q_start < 0 || p.q_len < 0 || int64_t{p.q_start} + p.q_len > len) return HYDRA_ERR_INVALID_ARG;
+        if (p.k_start < 0 || p.k_len < 0 || int64_t{p.k_start} + p.k_len > len) return HYDRA_ERR_INVALID_ARG;
+        if (p.part_row < -1) return HYDRA_ERR_INVALID_ARG;
+        if (i > 0) {
+            const hydra_pair_t& o = pairs[i - 1];
+            if (p.group < o.group) return HYDRA_ERR_INVALID_ARG;
+            if (p.group == o.group &&
+                (p.seq != o.seq || p.q_start != o.q_start || p.q_len != o.q_len ||
+                 (p.part_row < 0) != (o.part_row < 0)))
+                return HYDRA_ERR_INVALID_ARG;
+            if (p.group == o.group && p.part_row < 0) return HYDRA_ERR_INVALID_ARG;  // two direct writers
+        }
+        out.pairs.push_back(p);
+    }
+    return HYDRA_OK;
+}
+
+// partial rows must lie inside the buffers and must not overlap
+int32_t check_part_rows(const Problem& pb, int64_t part_rows)
+{
+    std::vector<std::pair<int64_t, int64_t>> iv;
+    for (const auto& p : pb.pairs)
+        if (p.part_row >= 0 && p.q_len > 0) {
+            if (int64_t{p.part_row} + p.q_len > part_rows) return HYDRA_ERR_INVALID_ARG;
+            iv.emplace_back(p.part_row, int64_t{p.part_row} + p.q_len);
+        }
+    std::sort(iv.begin(), iv.end());
+    for (size_t i = 1; i < iv.size(); ++i)
+        if (iv[i].first < iv[i - 1].second) return HYDRA_ERR_INVALID_ARG;
+    return HYDRA_OK;
+}
+
+// ranges of one kind (q or kv) inside one sequence must be identical or disjoint
+struct Range { int32_t seq, start, len; };
+inline bool range_less(const Range& a, const Range& b)
+{
+    if (a.seq != b.seq) return a.seq < b.seq;
+    if (a.start != b.start) return a.start < b.start;
+    return a.len < b.len;
+}
+int32_t check_identical_or_disjoint(std::vector<Range> r)
+{
+    std::sort(r.begin(), r.end(), range_less);
+    for (size_t i = 1; i < r.size(); ++i) {
+        const Range &a = r[i - 1], &b = r[i];
+        if (a.seq != b.seq) continue;
+        if (a.start == b.start && a.len == b.len) continue;
+        if (b.start < a.start + a.len) return HYDRA_ERR_INVALID_ARG;
+    }
+    return HYDRA_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// plans: device-resident work lists, cached by content
+// ---------------------------------------------------------------------------------------------
+struct DeviceBlob {
+    void* ptr = nullptr;
+    ~DeviceBlob() { if (ptr) cudaFree(ptr); }
+    cudaError_t upload(const std::vector<uint8_t>& bytes)
+    {
+        cudaError_t e = cudaMalloc(&ptr, std::max<size_t>(bytes.size(), 16));
+        if (e != cudaSuccess) { ptr = nullptr; return e; }
+        if (!bytes.empty()) e = cudaMemcpy(ptr, bytes.data(), bytes.size(), cudaMemcpyHostToDevice);
+        return e;
+    }
+};
+
+template <class T>
+size_t append(std::vector<uint8_t>& blob, const std::vector<T>& v)
+{
+    const size_t off = align_up(blob.size(), 16);
+    blob.resize(off + v.size() * sizeof(T));
+    if (!v.empty()) std::memcpy(blob.data() + off, v.data(), v.size() * sizeof(T));
+    return off;
+}
+
+struct Plan {
+    std::vector<uint8_t> key;
+    int kind = 0, device = 0;
+    DeviceBlob blob;
+    size_t off_pairs = 0, off_items = 0, off_lists = 0, off_groups = 0, off_items2 = 0, off_lists2 = 0;
+    int32_t n_items = 0, n_items2 = 0;
+};
+
+std::mutex g_plan_mutex;
+std::vector<std::unique_ptr<Plan>> g_plans;
+constexpr size_t kMaxPlans = 32;
+
+std::vector<uint8_t> make_key(int kind, int device, const Problem& pb, int causal)
+{
+    std::vector<uint8_t> key;
+    auto put = [&](const void* p, size_t n) {
+        const uint8_t* b = static_cast<const uint8_t*>(p);
+        key.insert(key.end(), b, b + n);
+    };
+    const int32_t head[5] = {kind, device, pb.h, causal, pb.n_seqs};
+    put(head, sizeof head);
+    put(pb.cu.data(), pb.cu.size() * sizeof(int32_t));
+    put(pb.pairs.data(), pb.pairs.size() * sizeof(hydra_pair_t));
+    return key;
+}
+
+std::vector<PairDev> device_pairs(const Problem& pb)
+{
+    std::vector<PairDev> v;
+    v.reserve(pb.pairs.size());
+    for (const auto& p : pb.pairs) {
+        PairDev d;
+        d.q_tok0 = pb.cu[p.seq] + p.q_start;
+        d.q_len = p.q_len;
+        d.k_tok0 = pb.cu[p.seq] + p.k_start;
+        d.k_len = p.k_len;
+        d.off = p.q_start - p.k_start;
+        d.to_part = p.part_row >= 0;
+        d.out_row0 = d.to_part ? p.part_row : d.q_tok0;
+        d.pad = 0;
+        v.push_back(d);
+    }
+    return v;
+}
+
+inline int32_t kv_tiles(const hydra_pair_t& p, int32_t q0, int causal)
+{
+    const int32_t last_row = std::min(q0 + TILE, p.q_len) - 1;
+    int64_t n_keys = p.k_len;
+    if (causal) n_keys = std::min<int64_t>(n_keys, int64_t{last_row} + (p.q_start - p.k_start) + 1);
+    return n_keys > 0 ? static_cast<int32_t>((n_keys + TILE - 1) / TILE) : 0;
+}
+
+// Order: blocks of items that share their operands (same pair/chunk and head) stay together so
+// that CTAs running at the same time hit the same K/V (or Q/dO) tiles in L2; blocks go
+// longest-first, and inside a block items go longest-first too (the quadratic load model of
+// Sections 3.2 / 5.1: cost ~ number of inner tiles).
+struct Keyed { int64_t block_cost; int32_t block; int32_t cost; int32_t idx; };
+template <class Item>
+void order_items(std::vector<Item>& items, const std::vector<int32_t>& block_of,
+                 const std::vector<int32_t>& cost)
+{
+    int32_t n_blocks = 0;
+    for (int32_t b : block_of) n_blocks = std::max(n_blocks, b + 1);
+    std::vector<int64_t> block_cost(n_blocks, 0);
+    for (size_t i = 0; i < items.size(); ++i) block_cost[block_of[i]] += cost[i];
+    std::vector<Keyed> k(items.size());
+    for (size_t i = 0; i < items.size(); ++i)
+        k[i] = Keyed{block_cost[block_of[i]], block_of[i], cost[i], static_cast<int32_t>(i)};
+    std::sort(k.begin(), k.end(), [](const Keyed& a, const Keyed& b) {
+        if (a.block_cost != b.block_cost) return a.block_cost > b.block_cost;
+        if (a.block != b.block) return a.block < b.block;
+        if (a.cost != b.cost) return a.cost > b.cost;
+        return a.idx < b.idx;
+    });
+    std::vector<Item> sorted(items.size());
+    for (size_t i = 0; i < items.size(); ++i) sorted[i] = items[k[i].idx];
+    items.swap(sorted);
+}
+
+void build_fwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& blob)
+{
+    std::vector<FwdItem> items;
+    std::vector<int32_t> block_of, cost;
+    for (size_t pi = 0; pi < pb.pairs.size(); ++pi) {
+        const auto& p = pb.pairs[pi];
+        for (int32_t q0 = 0; q0 < p.q_len; q0 += TILE) {
+            const int32_t n = kv_tiles(p, q0, causal);
+            for (int32_t a = 0; a < pb.h; ++a) {
+                items.push_back(FwdItem{static_cast<int32_t>(pi), a, q0, n});
+                block_of.push_back(static_cast<int32_t>(pi) * pb.h + a);
+                cost.push_back(n);
+            }
+        }
+    }
+    order_items(items, block_of, cost);
+    plan.off_pairs = append(blob, device_pairs(pb));
+    plan.off_items = append(blob, items);
+    plan.n_items = static_cast<int32_t>(items.size());
+}
+
+void build_merge(const Problem& pb, Plan& plan, std::vector<uint8_t>& blob)
+{
+    std::vector<MergeGroup> groups;
+    std::vector<int32_t> lists;
+    std::vector<MergeItem> items;
+    size_t i = 0;
+    while (i < pb.pairs.size()) {
+        size_t j = i;
+        while (j < pb.pairs.size() && pb.pairs[j].group == pb.pairs[i].group) ++j;
+        const auto& p = pb.pairs[i];
+        if (p.part_row >= 0 && p.q_len > 0) {
+            MergeGroup g;
+            g.out_tok0 = pb.cu[p.seq] + p.q_start;
+            g.rows = p.q_len;
+            g.list_off = static_cast<int32_t>(lists.size());
+            g.n_parts = static_cast<int32_t>(j - i);
+            for (size_t t = i; t < j; ++t) lists.push_back(pb.pairs[t].part_row);
+            for (int32_t r = 0; r < g.rows; r += MERGE_ROWS)
+                items.push_back(MergeItem{static_cast<int32_t>(groups.size()), r});
+            groups.push_back(g);
+        }
+        i = j;
+    }
+    plan.off_groups = append(blob, groups);
+    plan.off_lists = append(blob, lists);
+    plan.off_items = append(blob, items);
+    plan.n_items = static_cast<int32_t>(items.size());
+}
+
+// Backward lists: pairs grouped by q chunk (dQ kernel) and by kv chunk (dK/dV kernel).
+void build_bwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& blob)
+{
+    const int32_t n = static_cast<int32_t>(pb.pairs.size());
+    auto group_by = [&](bool by_q, std::vector<int32_t>& lists, std::vector<GroupItem>& items) {
+        std::vector<int32_t> order(n);
+        for (int32_t i = 0; i < n; ++i) order[i] = i;
+        auto key = [&](int32_t i) {
+            const auto& p = pb.pairs[i];
+            return Range{p.seq, by_q ? p.q_start : p.k_start, by_q ? p.q_len : p.k_len};
+        };
+        std::stable_sort(order.begin(), order.end(),
+                         [&](int32_t a, int32_t b) { return range_less(key(a), key(b)); });
+        std::vector<int32_t> block_of, cost;
+        int32_t block = 0;
+        int32_t i = 0;
+        while (i < n) {
+            int32_t j = i;
+            const Range r = key(order[i]);
+            while (j < n) {
+                const Range s = key(order[j]);
+                if (s.seq != r.seq || s.start != r.start || s.len != r.len) break;
+                ++j;
+            }
+            // a chunk with no rows, or whose pairs are all empty on the other side, has no work
+            const int32_t list_off = static_cast<int32_t>(lists.size());
+            for (int32_t t = i; t < j; ++t) {
+                const auto& p = pb.pairs[order[t]];
+                if ((by_q ? p.k_len : p.q_len) > 0) lists.push_back(order[t]);
+            }
+            const int32_t list_len = static_cast<int32_t>(lists.size()) - list_off;
+            if (r.len > 0 && list_len > 0) {
+                for (int32_t r0 = 0; r0 < r.len; r0 += TILE) {
+                    int32_t c = 0;
+                    for (int32_t t = 0; t < list_len; ++t) {
+                        const auto& p = pb.pairs[lists[list_off + t]];
+                        if (by_q) {
+                            c += kv_tiles(p, r0, causal);
+                        } else {
+                            const int32_t n_sub = (p.q_len + SUB - 1) / SUB;
+                            int32_t first = 0;
+                            if (causal) {
+                                const int32_t i_min = r0 - (p.q_start - p.k_start);
+                                first = i_min > 0 ? i_min / SUB : 0;
+                            }
+                            c += std::max(0, n_sub - first);
+                        }
+                    }
+                    for (int32_t a = 0; a < pb.h; ++a) {
+                        items.push_back(GroupItem{list_off, list_len, a, r0});
+                        block_of.push_back(block * pb.h + a);
+                        cost.push_back(c);
+                    }
+                }
+                ++block;
+            }
+            i = j;
+        }
+        order_items(items, block_of, cost);
+    };
+    std::vector<int32_t> lists_q, lists_k;
+    std::vector<GroupItem> items_q, items_k;
+    group_by(true, lists_q, items_q);
+    group_by(false, lists_k, items_k);
+    plan.off_pairs = append(blob, device_pairs(pb));
+    plan.off_lists = append(blob, lists_q);
+    plan.off_items = append(blob, items_q);
+    plan.off_lists2 = append(blob, lists_k);
+    plan.off_items2 = append(blob, items_k);
+    plan.n_items = static_cast<int32_t>(items_q.size());
+    plan.n_items2 = static_cast<int32_t>(items_k.size());
+}
+
+// Returns a cached plan or builds it (cudaMalloc + synchronous upload the first time only).
+int32_t get_plan(int kind, const Problem& pb, int causal, const Plan** out)
+{
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess) return HYDRA_ERR_CUDA;
+    std::vector<uint8_t> key = make_key(kind, device, pb, causal);
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    for (size_t i = 0; i < g_plans.size(); ++i)
+        if (g_plans[i]->key == key) {
+            if (i + 1 != g_plans.size()) std::rotate(g_plans.begin() + i, g_plans.begin() + i + 1, g_plans.end());
+            *out = g_plans.back().get();
+            return HYDRA_OK;
+        }
+    auto plan = std::make_unique<Plan>();
+    plan->kind = kind;
+    plan->device = device;
+    std::vector<uint8_t> blob;
+    if (kind == HYDRA_WS_FWD) build_fwd(pb, causal, *plan, blob);
+    else if (kind == HYDRA_WS_MERGE) build_merge(pb, *plan, blob);
+    else build_bwd(pb, causal, *plan, blob);
+    if (plan->blob.upload(blob) != cudaSuccess) return HYDRA_ERR_CUDA;
+    plan->key.swap(key);
+    if (g_plans.size() >= kMaxPlans) {
+        // evicting frees device memory a kernel in flight may still read: drain first
+        cudaDeviceSynchronize();
+        g_plans.erase(g_plans.begin());
+    }
+    g_plans.push_back(std::move(plan));
+    *out = g_plans.back().get();
+    return HYDRA_OK;
+}
+
+template <class T>
+const T* at(const Plan& p, size_t off) { return reinterpret_cast<const T*>(static_cast<const uint8_t*>(p.blob.ptr) + off); }
+
+// ---------------------------------------------------------------------------------------------
+// device properties and tensor maps
+// ---------------------------------------------------------------------------------------------
+struct DeviceInfo { int major = 0, sms = 0; bool known = false; };
+int32_t device_info(int* sms)
+{
+    static DeviceInfo info[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HYDRA_ERR_CUDA;
+    if (!info[dev].known) {
+        if (cudaDeviceGetAttribute(&info[dev].major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&info[dev].sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return HYDRA_ERR_CUDA;
+        info[dev].known = true;
+    }
+    if (info[dev].major != 10) return HYDRA_ERR_NOT_SM100;
+    *sms = info[dev].sms;
+    return HYDRA_OK;
+}
+
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                              CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                              CUtensorMapFloatOOBfill);
+EncodeFn encode_fn()
+{
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess)
+            fn = reinterpret_cast<EncodeFn>(p);
+    }
+    return fn;
+}
+
+// [T, h, d] bf16 seen as (d, h, T); a box is 64 elements x 1 head x `rows` tokens, written to
+// shared memory as `rows` 128-byte rows with the 128-byte swizzle. Tokens past T read as zero.
+int32_t make_map(CUtensorMap* map, const void* base, int64_t T, int32_t h, int32_t d, int32_t rows)
+{
+    EncodeFn enc = encode_fn();
+    if (!enc) return HYDRA_ERR_CUDA;
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(h),
+                                static_cast<cuuint64_t>(std::max<int64_t>(T, 1))};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2, static_cast<cuuint64_t>(d) * 2 * h};
+    const cuuint32_t box[3] = {64, 1, static_cast<cuuint32_t>(rows)};
+    const cuuint32_t es[3] = {1, 1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides,
+                           box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? HYDRA_OK : HYDRA_ERR_CUDA;
+}
+
+int32_t reset_status(void* workspace, cudaStream_t s)
+{
+    return cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), s) == cudaSuccess ? HYDRA_OK : HYDRA_ERR_CUDA;
+}
+
+}  // namespace
+}  // namespace hydra
+
+using namespace hydra;
+
+// =============================================================================================
+// C ABI
+// =============================================================================================
+extern "C" {
+
+int32_t hydra_version(void) { return 1; }
+
+const char* hydra_status_string(int32_t s)
+{
+    switch (s) {
+        case HYDRA_OK: return "HYDRA_OK";
+        case HYDRA_ERR_INVALID_ARG: return "HYDRA_ERR_INVALID_ARG";
+        case HYDRA_ERR_UNSUPPORTED: return "HYDRA_ERR_UNSUPPORTED";
+        case HYDRA_ERR_WORKSPACE_TOO_SMALL: return "HYDRA_ERR_WORKSPACE_TOO_SMALL";
+        case HYDRA_ERR_CUDA: return "HYDRA_ERR_CUDA";
+        case HYDRA_ERR_DEVICE_TIMEOUT: return "HYDRA_ERR_DEVICE_TIMEOUT";
+        case HYDRA_ERR_NOT_SM100: return "HYDRA_ERR_NOT_SM100";
+        default: return "HYDRA_ERR_UNKNOWN";
+    }
+}
+
+int64_t hydra_launch_count(void) { return g_launches.load(); }
+
+void hydra_set_wait_limit_ns(uint64_t ns) { g_wait_limit_ns.store(ns ? ns : 1); }
+
+void hydra_shutdown(void)
+{
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    if (!g_plans.empty()) cudaDeviceSynchronize();
+    g_plans.clear();
+}
+
+int32_t hydra_usp_factor(int32_t degree, int32_t heads, int32_t* cp_u, int32_t* cp_r)
+{
+    if (degree < 1 || heads < 1 || !cp_u || !cp_r) return HYDRA_ERR_INVALID_ARG;
+    const int32_t u = degree < heads ? degree : heads;
+    if (degree % u != 0) return HYDRA_ERR_INVALID_ARG;
+    *cp_u = u;
+    *cp_r = degree / u;
+    return HYDRA_OK;
+}
+
+int32_t hydra_zigzag_pairs(const int32_t* cu, int32_t n_seqs, const int32_t* cp_r_host, int32_t cp_r_all,
+                           hydra_pair_t* pairs_out, int32_t max_pairs, int32_t* n_pairs_out,
+                           int64_t* part_rows_out, int32_t* rank_out, int32_t* step_out)
+{
+    if (n_seqs < 0 || (n_seqs > 0 && !cu) || !n_pairs_out || !part_rows_out || max_pairs < 0 ||
+        (max_pairs > 0 && !pairs_out))
+        return HYDRA_ERR_INVALID_ARG;
+    if (n_seqs > 0 && cu[0] != 0) return HYDRA_ERR_INVALID_ARG;
+    int64_t n_pairs = 0, part_rows = 0;
+    int32_t group = 0;
+    for (int32_t b = 0; b < n_seqs; ++b) {
+        const int64_t len = int64_t{cu[b + 1]} - cu[b];
+        const int32_t ring = cp_r_host ? cp_r_host[b] : cp_r_all;
+        if (len < 0 || ring < 0 || ring > 4096) return HYDRA_ERR_INVALID_ARG;
+        const int32_t n_c = ring == 0 ? 1 : 2 * ring;
+        auto edge = [&](int32_t c) { return static_cast<int32_t>(c * len / n_c); };
+        auto owner = [&](int32_t c) { return ring == 0 ? 0 : (c < ring ? c : n_c - 1 - c); };
+        for (int32_t qc = 0; qc < n_c; ++qc) {
+            const int32_t qs = edge(qc), ql = edge(qc + 1) - qs;
+            if (ql == 0) continue;
+            int32_t in_group = 0;
+            for (int32_t kc = 0; kc <= qc; ++kc)
+                if (edge(kc + 1) - edge(kc) > 0) ++in_group;
+            for (int32_t kc = 0; kc <= qc; ++kc) {
+                const int32_t ks = edge(kc), kl = edge(kc + 1) - ks;
+                if (kl == 0) continue;
+                if (n_pairs < max_pairs) {
+                    hydra_pair_t& p = pairs_out[n_pairs];
+                    p.seq = b; p.q_start = qs; p.q_len = ql; p.k_start = ks; p.k_len = kl;
+                    p.group = group; p.flags = 0;
+                    p.part_row = in_group > 1 ? static_cast<int32_t>(part_rows) : -1;
+                    if (rank_out) rank_out[n_pairs] = owner(qc);
+                    if (step_out) {
+                        const int32_t m = ring > 0 ? ring : 1;
+                        step_out[n_pairs] = ((owner(qc) - owner(kc)) % m + m) % m;
+                    }
+                }
+                if (in_group > 1) part_rows += ql;
+                ++n_pairs;
+            }
+            ++group;
+        }
+    }
+    if (n_pairs > INT32_MAX || part_rows > INT32_MAX) return HYDRA_ERR_UNSUPPORTED;
+    *n_pairs_out = static_cast<int32_t>(n_pairs);
+    *part_rows_out = part_rows;
+    return n_pairs > max_pairs ? HYDRA_ERR_WORKSPACE_TOO_SMALL : HYDRA_OK;
+}
+
+size_t hydra_workspace_bytes(int32_t which, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                             const hydra_pair_t* pairs, int32_t n_pairs)
+{
+    Problem pb;
+    if (make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb) != HYDRA_OK) return 0;
+    switch (which) {
+        case HYDRA_WS_FWD:
+        case HYDRA_WS_MERGE: return kStatusBytes;
+        case HYDRA_WS_BWD: return kStatusBytes + align_up(static_cast<size_t>(pb.T) * n_heads * sizeof(float), 256);
+        default: return 0;
+    }
+}
+
+int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_t* cu, int32_t n_seqs,
+                       int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal,
+                       float softmax_scale, void* out, float* lse, void* o_part, float* lse_part,
+                       int64_t part_rows, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    int sms = 0;
+    if (int32_t s = device_info(&sms)) return s;
+    Problem pb;
+    if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
+    if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return HYDRA_ERR_INVALID_ARG;
+    if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
+    if (workspace_bytes < kStatusBytes) return HYDRA_ERR_WORKSPACE_TOO_SMALL;
+    bool any_part = false, any_direct = false;
+    for (const auto& p : pb.pairs) (p.part_row >= 0 ? any_part : any_direct) = true;
+    if (pb.T > 0 && (!q || !k || !v || !aligned16(q) || !aligned16(k) || !aligned16(v))) return HYDRA_ERR_INVALID_ARG;
+    if (any_direct && (!out || !lse || !aligned16(out) || !aligned16(lse))) return HYDRA_ERR_INVALID_ARG;
+    if (any_part && (!o_part || !lse_part || !aligned16(o_part) || !aligned16(lse_part) || part_rows <= 0))
+        return HYDRA_ERR_INVALID_ARG;
+    if (int32_t s = check_part_rows(pb, part_rows)) return s;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (pb.pairs.empty()) return HYDRA_OK;
+
+    const Plan* plan = nullptr;
+    if (int32_t s = get_plan(HYDRA_WS_FWD, pb, causal != 0, &plan)) return s;
+    if (plan->n_items == 0) return HYDRA_OK;
+    CUtensorMap mq, mk, mv;
+    if (make_map(&mq, q, pb.T, n_heads, D_QK, TILE) || make_map(&mk, k, pb.T, n_heads, D_QK, TILE) ||
+        make_map(&mv, v, pb.T, n_heads, D_V, TILE))
+        return HYDRA_ERR_CUDA;
+    if (int32_t s = reset_status(workspace, stream)) return s;
+    FwdParams fp{};
+    fp.pairs = at<PairDev>(*plan, plan->off_pairs);
+    fp.items = at<FwdItem>(*plan, plan->off_items);
+    fp.n_items = plan->n_items;
+    fp.out = out; fp.lse = lse; fp.o_part = o_part; fp.lse_part = lse_part;
+    fp.T = pb.T; fp.part_rows = part_rows; fp.h = n_heads; fp.causal = causal != 0;
+    fp.scale_log2 = softmax_scale * 1.4426950408889634f;
+    fp.status = static_cast<StatusBlock*>(workspace);
+    fp.wait_limit_ns = g_wait_limit_ns.load();
+    const int grid = std::min(plan->n_items, sms);
+    if (launch_fwd(mq, mk, mv, fp, grid, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    g_launches += 1;
+    return HYDRA_OK;
+}
+
+int32_t hydra_lse_merge(const void* o_part, const float* lse_part, int64_t part_rows, const int32_t* cu,
+                        int32_t n_seqs, int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs,
+                        void* out, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    int sms = 0;
+    if (int32_t s = device_info(&sms)) return s;
+    Problem pb;
+    if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
+    if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
+    if (workspace_bytes < kStatusBytes) return HYDRA_ERR_WORKSPACE_TOO_SMALL;
+    bool any_part = false;
+    for (const auto& p : pb.pairs) any_part |= (p.part_row >= 0 && p.q_len > 0);
+    if (!any_part) return HYDRA_OK;
+    if (!o_part || !lse_part || !out || !lse || !aligned16(o_part) || !aligned16(lse_part) ||
+        !aligned16(out) || !aligned16(lse) || part_rows <= 0)
+        return HYDRA_ERR_INVALID_ARG;
+    if (int32_t s = check_part_rows(pb, part_rows)) return s;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const Plan* plan = nullptr;
+    if (int32_t s = get_plan(HYDRA_WS_MERGE, pb, 0, &plan)) return s;
+    MergeParams mp{};
+    mp.groups = at<MergeGroup>(*plan, plan->off_groups);
+    mp.lists = at<int32_t>(*plan, plan->off_lists);
+    mp.items = at<MergeItem>(*plan, plan->off_items);
+    mp.n_items = plan->n_items;
+    mp.o_part = o_part; mp.lse_part = lse_part; mp.out = out; mp.lse = lse;
+    mp.T = pb.T; mp.part_rows = part_rows; mp.h = n_heads;
+    if (launch_merge(mp, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    g_launches += 1;
+    return HYDRA_OK;
+}
+
+int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                       const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                       const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
+                       void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream)
+{
+    int sms = 0;
+    if (int32_t s = device_info(&sms)) return s;
+    Problem pb;
+    if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
+    if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return HYDRA_ERR_INVALID_ARG;
+    if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
+    const size_t need = kStatusBytes + align_up(static_cast<size_t>(pb.T) * n_heads * sizeof(float), 256);
+    if (workspace_bytes < need) return HYDRA_ERR_WORKSPACE_TOO_SMALL;
+    if (pb.T == 0 || pb.pairs.empty()) return HYDRA_OK;
+    const void* ptrs[] = {q, k, v, out, lse, dout, dq, dk, dv};
+    for (const void* p : ptrs)
+        if (!p || !aligned16(p)) return HYDRA_ERR_INVALID_ARG;
+    {
+        std::vector<Range> rq, rk;
+        for (const auto& p : pb.pairs) {
+            if (p.q_len > 0) rq.push_back(Range{p.seq, p.q_start, p.q_len});
+            if (p.k_len > 0) rk.push_back(Range{p.seq, p.k_start, p.k_len});
+        }
+        if (check_identical_or_disjoint(rq) || check_identical_or_disjoint(rk)) return HYDRA_ERR_INVALID_ARG;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const Plan* plan = nullptr;
+    if (int32_t s = get_plan(HYDRA_WS_BWD, pb, causal != 0, &plan)) return s;
+
+    float* dsum = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kStatusBytes);
+    CUtensorMap mq, mk, mv, mdo, mq_sub, mdo_sub;
+    if (make_map(&mq, q, pb.T, n_heads, D_QK, TILE) || make_map(&mk, k, pb.T, n_heads, D_QK, TILE) ||
+        make_map(&mv, v, pb.T, n_heads, D_V, TILE) || make_map(&mdo, dout, pb.T, n_heads, D_V, TILE) ||
+        make_map(&mq_sub, q, pb.T, n_heads, D_QK, SUB) || make_map(&mdo_sub, dout, pb.T, n_heads, D_V, SUB))
+        return HYDRA_ERR_CUDA;
+    if (int32_t s = reset_status(workspace, stream)) return s;
+    if (launch_bwd_prep(dout, out, dsum, pb.T, n_heads, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    g_launches += 1;
+
+    BwdParams bp{};
+    bp.pairs = at<PairDev>(*plan, plan->off_pairs);
+    bp.lse = lse; bp.dsum = dsum; bp.dq = dq; bp.dk = dk; bp.dv = dv;
+    bp.T = pb.T; bp.h = n_heads; bp.causal = causal != 0;
+    bp.scale = softmax_scale; bp.scale_log2 = softmax_scale * 1.4426950408889634f;
+    bp.status = static_cast<StatusBlock*>(workspace);
+    bp.wait_limit_ns = g_wait_limit_ns.load();
+    if (plan->n_items2 > 0) {
+        bp.lists = at<int32_t>(*plan, plan->off_lists2);
+        bp.items = at<GroupItem>(*plan, plan->off_items2);
+        bp.n_items = plan->n_items2;
+        if (launch_bwd_dkv(mq_sub, mk, mv, mdo_sub, bp, std::min(plan->n_items2, sms), stream) != cudaSuccess)
+            return HYDRA_ERR_CUDA;
+        g_launches += 1;
+    }
+    if (plan->n_items > 0) {
+        bp.lists = at<int32_t>(*plan, plan->off_lists);
+        bp.items = at<GroupItem>(*plan, plan->off_items);
+        bp.n_items = plan->n_items;
+        if (launch_bwd_dq(mq, mk, mv, mdo, bp, std::min(plan->n_items, sms), stream) != cudaSuccess)
+            return HYDRA_ERR_CUDA;
+        g_launches += 1;
+    }
+    return HYDRA_OK;
+}
+
+int32_t hydra_poll_status(void* workspace, void* cuda_stream, int32_t* device_status, int64_t* detail)
+{
+    if (!workspace || !device_status) return HYDRA_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return HYDRA_ERR_CUDA;
+    StatusBlock sb;
+    if (cudaMemcpy(&sb, workspace, sizeof sb, cudaMemcpyDeviceToHost) != cudaSuccess) return HYDRA_ERR_CUDA;
+    *device_status = sb.status;
+    if (detail) *detail = sb.status ? sb.detail : -1;
+    return HYDRA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,115 @@
+// Internal declarations shared by the host API and the kernel translation units.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/hydra_attn.h"
+
+namespace hydra {
+
+constexpr int D_QK = HYDRA_D_QK;
+constexpr int D_V = HYDRA_D_V;
+constexpr int TILE = 128;       // rows of a q tile and of a kv tile
+constexpr int SUB = 64;         // rows of a q sub-tile in the key-side backward kernel
+
+// One (q-chunk, kv-chunk) pair with absolute token offsets, as the kernels see it.
+struct PairDev {
+    int32_t q_tok0;    // token index of the pair's first q row
+    int32_t q_len;
+    int32_t k_tok0;    // token index of the pair's first kv row
+    int32_t k_len;
+    int32_t off;       // q_start - k_start: key j is visible to q row i iff j <= i + off (causal)
+    int32_t out_row0;  // first output row: part_row (partial buffers) or q_tok0 (out / lse)
+    int32_t to_part;   // 1: partial buffers, 0: out / lse
+    int32_t pad;
+};
+
+// Forward work item: one 128-row q tile of one pair and head.
+struct FwdItem {
+    int32_t pair;
+    int32_t head;
+    int32_t q0;        // first q row of the tile, relative to the pair
+    int32_t n_kv;      // kv tiles to visit (after causal clipping); 0: the rows see no key
+};
+
+// Backward work item: one tile of one chunk and head, visiting every pair that shares the chunk.
+struct GroupItem {
+    int32_t list_off;  // first entry of the chunk's pair list
+    int32_t list_len;
+    int32_t head;
+    int32_t r0;        // first row of the tile, relative to the chunk
+};
+
+// Merge: one q chunk with two or more partials.
+struct MergeGroup {
+    int32_t out_tok0;  // first token of the chunk in out / lse
+    int32_t rows;
+    int32_t list_off;  // first entry of the chunk's part_row list
+    int32_t n_parts;
+};
+struct MergeItem {
+    int32_t group;
+    int32_t row0;      // first row of the block, relative to the chunk
+};
+constexpr int MERGE_ROWS = 8;   // rows of a merge block
+
+struct StatusBlock {            // lives at the start of the workspace
+    int32_t status;
+    int32_t pad;
+    int64_t detail;
+};
+
+struct FwdParams {
+    const PairDev* pairs;
+    const FwdItem* items;
+    int32_t n_items;
+    void* out; float* lse; void* o_part; float* lse_part;
+    int64_t T; int64_t part_rows;
+    int32_t h; int32_t causal;
+    float scale_log2;           // softmax_scale * log2(e)
+    StatusBlock* status;
+    uint64_t wait_limit_ns;
+};
+
+struct BwdParams {
+    const PairDev* pairs;
+    const int32_t* lists;       // pair indices, grouped by chunk
+    const GroupItem* items;
+    int32_t n_items;
+    const float* lse; const float* dsum;   // [h, T]
+    void* dq; void* dk; void* dv;
+    int64_t T;
+    int32_t h; int32_t causal;
+    float scale; float scale_log2;
+    StatusBlock* status;
+    uint64_t wait_limit_ns;
+};
+
+struct MergeParams {
+    const MergeGroup* groups;
+    const int32_t* lists;       // part_row of every partial, grouped by chunk
+    const MergeItem* items;
+    int32_t n_items;
+    const void* o_part; const float* lse_part;
+    void* out; float* lse;
+    int64_t T; int64_t part_rows;
+    int32_t h;
+};
+
+size_t fwd_smem_bytes();
+size_t bwd_dq_smem_bytes();
+size_t bwd_dkv_smem_bytes();
+
+cudaError_t launch_fwd(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                       const FwdParams& p, int grid, cudaStream_t stream);
+cudaError_t launch_bwd_dq(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                          const CUtensorMap& mdo, const BwdParams& p, int grid, cudaStream_t stream);
+cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, const CUtensorMap& mv,
+                           const CUtensorMap& mdo_sub, const BwdParams& p, int grid,
+                           cudaStream_t stream);
+cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
+cudaError_t launch_bwd_prep(const void* dout, const void* out, float* dsum, int64_t T, int32_t h,
+                            cudaStream_t stream);
+
+}  // namespace hydra

@@ -1,0 +1,91 @@
+"""Helpers of the GPU parity tests: run a problem through the C ABI and through the oracle."""
+from __future__ import annotations
+
+import numpy as np
+
+import hydra_workloads as hw
+import oracle
+
+TOL_REL = 2e-2      # max |gpu - ref| <= TOL_REL * max |ref| on O, dQ, dK, dV
+TOL_LSE = 1e-3      # absolute, on LSE
+
+
+def pairs_for(cu, cp_r):
+    """(library pairs, part_rows, oracle pairs) for a uniform outer-ring degree (0 = not cut)."""
+    import paper_2609_34318_b200 as P
+    lib_pairs, part_rows, _, _ = P.hydra_zigzag_pairs(cu, cp_r)
+    return lib_pairs, part_rows, oracle.causal_pairs(cu, cp_r)
+
+
+def run_gpu(x, cu, h, pairs=None, part_rows=0, causal=True, scale=None, backward=True, poison=True):
+    """x: dict of uint16 bit arrays q, k, v, do. Returns dict of float64 numpy results."""
+    import torch
+    from paper_2609_34318_b200.runner import AttnStep, bits_to_tensor
+    step = AttnStep(cu, h, pairs, part_rows, causal, scale)
+    if poison:
+        for t in (step.out, step.lse, step.dq, step.dk, step.dv, step.o_part, step.lse_part):
+            t.fill_(float("nan"))
+    q, k, v, do = (bits_to_tensor(x[n]) for n in ("q", "k", "v", "do"))
+    step.forward(q, k, v)
+    res = {}
+    if backward:
+        step.backward(q, k, v, do)
+    status, detail = step.poll()
+    assert status == 0, f"device status {status} (item {detail})"
+    torch.cuda.synchronize()
+    T = int(cu[-1])
+    res["out"] = step.out[:T].float().cpu().numpy().astype(np.float64)
+    res["lse"] = step.lse[:, :T].cpu().numpy().astype(np.float64)
+    if backward:
+        res["dq"] = step.dq[:T].float().cpu().numpy().astype(np.float64)
+        res["dk"] = step.dk[:T].float().cpu().numpy().astype(np.float64)
+        res["dv"] = step.dv[:T].float().cpu().numpy().astype(np.float64)
+    res["_step"] = step
+    return res
+
+
+def run_oracle(x, cu, causal=True, scale=None, pairs=None, backward=True):
+    """Unchunked oracle forward; backward over `pairs` (oracle pair dicts) or unchunked."""
+    scale = np.float32(1.0 / np.sqrt(np.float32(hw.D_QK))) if scale is None else np.float32(scale)
+    out, lse = oracle.attn_fwd(x["q"], x["k"], x["v"], cu, causal, scale)
+    res = dict(out=out, lse=lse)
+    if backward:
+        if pairs is None:
+            dq, dk, dv = oracle.attn_bwd(x["q"], x["k"], x["v"], x["do"], cu, causal, scale, out, lse)
+        else:
+            d = oracle.bwd_prep(x["do"], out)
+            dq, dk, dv = oracle.attn_bwd_pairs(x["q"], x["k"], x["v"], x["do"], cu, pairs, causal, scale,
+                                               lse, d)
+        res.update(dq=dq, dk=dk, dv=dv)
+    return res
+
+
+def check(got, ref, names=("out", "lse", "dq", "dk", "dv"), tol_rel=TOL_REL, tol_lse=TOL_LSE, label=""):
+    report = {}
+    for n in names:
+        if n not in ref:
+            continue
+        g, r = got[n], ref[n]
+        assert g.shape == r.shape, (n, g.shape, r.shape)
+        assert np.isfinite(g[np.isfinite(r)]).all(), f"{label}{n}: non-finite values (unwritten rows?)"
+        if n == "lse":
+            fin = np.isfinite(r)
+            err = np.abs(g[fin] - r[fin]).max() if fin.any() else 0.0
+            assert np.array_equal(np.isneginf(g), np.isneginf(r)), f"{label}lse: -inf pattern differs"
+            report[n] = err
+            assert err <= tol_lse, f"{label}lse: max abs err {err:.3e} > {tol_lse}"
+        else:
+            err = np.abs(g - r).max()
+            ref_max = np.abs(r).max()
+            report[n] = err / max(ref_max, 1e-30)
+            assert err <= tol_rel * ref_max + 1e-30, \
+                f"{label}{n}: max abs err {err:.3e} > {tol_rel} * max|ref| = {tol_rel * ref_max:.3e}"
+    return report
+
+
+def row_rel_err(got, ref):
+    """Per-row relative L2 error (rows = all leading axes), max over rows with a non-zero reference."""
+    g = got.reshape(-1, got.shape[-1]); r = ref.reshape(-1, ref.shape[-1])
+    nr = np.linalg.norm(r, axis=1)
+    ok = nr > 0
+    return float((np.linalg.norm(g - r, axis=1)[ok] / nr[ok]).max()) if ok.any() else 0.0
