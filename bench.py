@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the attention hot path (forward of every chunk pair, LSE merge, backward).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step = one pass of the whole path over one synthetic microbatch: hydra_attn_fwd,
+hydra_lse_merge (when the workload is chunked) and hydra_attn_bwd (D-prep, dK/dV kernel, dQ kernel).
+The metric is causal-pair TFLOP/s: fwd = 2 * sum_pairs * h * (192 + 128), bwd counted as 2.5 x fwd.
+Prints ONE JSON line (rank 0). With N > 1 (launched by torch.distributed.run) every rank processes
+its own microbatch of the same shape: weak scaling, no data-path collective.
+`--impl reference` times the fp64 CPU oracle, as it stands, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import hydra_workloads as hw  # noqa: E402
+
+METRIC = "attention fwd+bwd TFLOP/s (causal pairs)"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# algorithmic FLOPs per causal (i, j) pair and head of each tensor-core kernel
+FLOPS_PER_PAIR = {"fwd": 2.0 * (192 + 128),                  # S = QK^T and O = PV
+                  "bwd_dkv": 2.0 * (192 + 128 + 128 + 192),  # S, dP, dV, dK: each needed once
+                  "bwd_dq": 2.0 * 192}                       # dQ = dS K (its S, dP are recomputation)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# --------------------------------------------------------------------------------------------------
+# clocks during the timed region (read-only NVML queries)
+# --------------------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap"}
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        while self.ok and not self._halt.is_set():
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.dev, self.nv.NVML_CLOCK_SM))
+                bits = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev) \
+                    if hasattr(self.nv, "nvmlDeviceGetCurrentClocksEventReasons") \
+                    else self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.dev)
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                break
+            self._halt.wait(0.01)
+
+    def stop(self):
+        self._halt.set()
+        self.join(timeout=2)
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------------------------------
+# reference arm: the oracle on the host cores, bounded sample
+# --------------------------------------------------------------------------------------------------
+def oracle_sample(w, budget_s: float):
+    """Leading sequences of the workload, one head, sized so one fwd+bwd takes about `budget_s`."""
+    import oracle
+    probe = hw.Workload("probe", [768], 1)
+    x = probe.tensors([0])
+    t0 = time.perf_counter()
+    out, lse = oracle.attn_fwd(x["q"], x["k"], x["v"], probe.cu(), True, probe.scale)
+    oracle.attn_bwd(x["q"], x["k"], x["v"], x["do"], probe.cu(), True, probe.scale, out, lse)
+    rate = probe.causal_pairs_total / max(time.perf_counter() - t0, 1e-6)      # pairs*head / s
+    lengths, pairs = [], 0
+    for length in w.lengths:
+        cost = length * (length + 1) // 2
+        if lengths and (pairs + cost) / rate > budget_s:
+            break
+        if not lengths and cost / rate > budget_s:          # even the first sequence is too long
+            length = max(64, int((2.0 * budget_s * rate) ** 0.5))
+            cost = length * (length + 1) // 2
+        lengths.append(length)
+        pairs += cost
+    return hw.Workload(w.name + "_sample", lengths, 1, cp_r=w.cp_r)
+
+
+def oracle_step(sample):
+    import oracle
+    x = sample.tensors([0])
+    cu = sample.cu()
+    t0 = time.perf_counter()
+    out, lse = oracle.attn_fwd(x["q"], x["k"], x["v"], cu, True, sample.scale)
+    if sample.cp_r:
+        pairs = oracle.causal_pairs(cu, sample.cp_r)
+        d = oracle.bwd_prep(x["do"], out)
+        oracle.attn_bwd_pairs(x["q"], x["k"], x["v"], x["do"], cu, pairs, True, sample.scale, lse, d)
+    else:
+        oracle.attn_bwd(x["q"], x["k"], x["v"], x["do"], cu, True, sample.scale, out, lse)
+    return time.perf_counter() - t0
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    budget = min(15.0, 150.0 / max(args.steps + args.warmup, 1))
+    sample = oracle_sample(w, budget)
+    for _ in range(args.warmup):
+        oracle_step(sample)
+    times = [oracle_step(sample) for _ in range(args.steps)]
+    total = sum(times)
+    flops = 3.5 * sample.flops_fwd() * args.steps
+    value = flops / total / 1e12
+    desc = f"first {len(sample.lengths)} sequence(s) ({sample.total} tokens), 1 head of {w.name}, fwd+bwd"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": w.name, "sample": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.n_threads(), "kind": "oracle",
+                             "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------------
+def device_inputs(w, torch, seed_shift: int):
+    from paper_2609_34318_b200.runner import bits_to_tensor
+    T, h = w.total, w.n_heads
+    t = {}
+    for n in ("q", "k", "v", "do"):
+        d = hw.D_V if n in ("v", "do") else hw.D_QK
+        t[n] = torch.empty((T, h, d), dtype=torch.bfloat16, device="cuda")
+        for a in range(h):
+            t[n][:, a, :] = bits_to_tensor(hw.tensor_bits(n, T, [a], seed=hw.SEED + seed_shift))[:, 0, :]
+    return t
+
+
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.runner import AttnStep
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    cu = w.cu()
+    pairs, part_rows = (None, 0)
+    if w.cp_r:
+        pairs, part_rows, _, _ = P.hydra_zigzag_pairs(cu, w.cp_r)
+    t = device_inputs(w, torch, rank)
+    step = AttnStep(cu, w.n_heads, pairs, part_rows, True, float(w.scale))
+    stream = torch.cuda.current_stream()
+
+    def one_step():
+        step.forward(t["q"], t["k"], t["v"])
+        step.backward(t["q"], t["k"], t["v"], t["do"])
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    status, detail = step.poll()
+    if status != 0:
+        raise RuntimeError(f"device status {status} at item {detail}")
+
+    # ---- timed region: K steps, CUDA events on the launching stream, per-kernel events inside ----
+    sampler = ClockSampler(local)
+    P.hydra_profile_enable(True)
+    P.hydra_profile_collect()
+    launches0 = P.hydra_launch_count()
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        one_step()
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    total_ms = e0.elapsed_time(e1)
+    launches = P.hydra_launch_count() - launches0
+    kernel_ms, kernel_n = P.hydra_profile_collect()
+    P.hydra_profile_enable(False)
+    if world > 1:
+        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    status, detail = step.poll()
+    if status != 0:
+        raise RuntimeError(f"device status {status} at item {detail}")
+
+    flops_step = 3.5 * w.flops_fwd()
+    value = world * flops_step * args.steps / (total_ms * 1e-3) / 1e12
+
+    # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region ----
+    e2e = None
+    if not args.no_e2e:
+        host = {n: v.cpu().pin_memory() for n, v in t.items()}
+        T, h = w.total, w.n_heads
+        ho = {"out": torch.empty((T, h, hw.D_V), dtype=torch.bfloat16).pin_memory(),
+              "lse": torch.empty((h, T), dtype=torch.float32).pin_memory(),
+              "dq": torch.empty((T, h, hw.D_QK), dtype=torch.bfloat16).pin_memory(),
+              "dk": torch.empty((T, h, hw.D_QK), dtype=torch.bfloat16).pin_memory(),
+              "dv": torch.empty((T, h, hw.D_V), dtype=torch.bfloat16).pin_memory()}
+        del step
+        torch.cuda.empty_cache()
+        arena = torch.empty(P.hydra_host_step_arena_bytes(cu, h, pairs) + 256, dtype=torch.uint8, device="cuda")
+        off = (-arena.data_ptr()) % 256
+        arena_ptr, arena_bytes = arena.data_ptr() + off, arena.numel() - off
+
+        def host_step():
+            P.hydra_attn_fwd_bwd_host(host["q"], host["k"], host["v"], host["do"], cu, h, pairs, True,
+                                      float(w.scale), ho["out"], ho["lse"], ho["dq"], ho["dk"], ho["dv"],
+                                      arena_ptr, arena_bytes)
+
+        e_steps = max(1, min(args.steps, 5))
+        host_step()
+        barrier()
+        e0.record(stream)
+        for _ in range(e_steps):
+            host_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        if world > 1:
+            tt = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_ms = float(tt.item())
+        h2d = sum(v.numel() * v.element_size() for v in host.values())
+        d2h = sum(v.numel() * v.element_size() for v in ho.values())
+        e2e = {"value": world * flops_step * e_steps / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e_steps,
+               "ms_per_step": e2e_ms / e_steps}
+        assert torch.isfinite(ho["dq"].float()).all()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel ----
+    peaks, peak_kind = measured_peaks()
+    dominant = max(kernel_ms, key=lambda k: kernel_ms[k])
+    per_launch_ms = kernel_ms[dominant] / max(kernel_n[dominant], 1)
+    if dominant in FLOPS_PER_PAIR:
+        work = FLOPS_PER_PAIR[dominant] * w.causal_pairs_total * w.n_heads
+        sustained = total_ms > 2000.0
+        peak = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"]
+        roof = {"kernel": dominant, "bound": "tensor", "achieved": work / (per_launch_ms * 1e-3) / 1e12,
+                "peak": peak, "unit": "TFLOP/s",
+                "peak_kind": f"{peak_kind} {'sustained' if sustained else 'burst'} bf16"}
+    else:
+        th = w.total * w.n_heads
+        work = th * 516.0 if dominant == "bwd_prep" else 0.0
+        if dominant == "merge":
+            work = sum((int(n) + 1) * 260.0 * rows * w.n_heads for n, rows in merge_groups(pairs))
+        roof = {"kernel": dominant, "bound": "hbm", "achieved": work / (per_launch_ms * 1e-3) / 1e9,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "peak_kind": f"{peak_kind} copy"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = recorded_traffic(dominant, w.name)
+    roof["ms_per_launch"] = per_launch_ms
+
+    # ---- CPU baseline: the oracle on a bounded sample, rank 0, N = 1 only ----
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        import oracle
+        sample = oracle_sample(w, 12.0)
+        sec = oracle_step(sample)
+        cpu = {"value": 3.5 * sample.flops_fwd() / sec / 1e12, "unit": UNIT, "cores": oracle.n_threads(),
+               "kind": "oracle", "seconds": sec,
+               "sample": f"first {len(sample.lengths)} sequence(s) ({sample.total} tokens), 1 head of "
+                         f"{w.name}, fwd+bwd"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "tokens": w.total, "heads": w.n_heads, "sequences": len(w.lengths),
+                       "d_qk": hw.D_QK, "d_v": hw.D_V, "pairs": 0 if pairs is None else int(len(pairs)),
+                       "causal_pairs": w.causal_pairs_total, "note": w.note,
+                       "l2": "inputs larger than L2 (no flush between iterations)"},
+            "frac_of_bf16_peak": value / world / peaks["bf16_tflops"],
+            "kernel_ms_per_step": {k: v / args.steps for k, v in kernel_ms.items()},
+            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clocks}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def merge_groups(pairs):
+    """(number of partials, rows) of every merged q chunk."""
+    if pairs is None:
+        return []
+    out, i = [], 0
+    while i < len(pairs):
+        j = i
+        while j < len(pairs) and pairs[j]["group"] == pairs[i]["group"]:
+            j += 1
+        if pairs[i]["part_row"] >= 0:
+            out.append((j - i, int(pairs[i]["q_len"])))
+        i = j
+    return out
+
+
+def recorded_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch from the ncu capture summarised under profiles/ (None if not captured)."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        table = json.load(f)
+    return table.get(f"{kernel}:{workload}")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="packed32k", choices=list(hw.WORKLOADS))
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    w = hw.workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -117,8 +117,8 @@ class Workload:
     name: str
     lengths: List[int]
     n_heads: int
-    cp_r: int = 0                 # outer-ring degree used to cut every sequence (0 = not cut)
-    split_two: bool = False       # cut every sequence in two chunks (floor(L/2), rest)
+    cp_r: int = 0                 # outer-ring degree used to cut every sequence (0 = not cut);
+                                  # 1 cuts a sequence in two chunks (floor(L/2), rest)
     causal: bool = True
     note: str = ""
     extra: Dict[str, object] = field(default_factory=dict)
@@ -167,7 +167,7 @@ def workload(name: str) -> Workload:
         return Workload("short64k", lengths_uniform(), 32,
                         note="64K tokens of sequences with lengths uniform in [64, 512]")
     if name == "short64k_split":
-        return Workload("short64k_split", lengths_uniform(), 32, split_two=True,
+        return Workload("short64k_split", lengths_uniform(), 32, cp_r=1,
                         note="many-short with every sequence cut in two chunks and merged")
     raise KeyError(name)
 

@@ -151,6 +151,34 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
                        int32_t causal, float softmax_scale, void* dq, void* dk, void* dv,
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * The whole step (forward of every pair, merge, backward; Sections 3.5 and 5.2 as above) with HOST
+ * buffers: copies q, k, v, dout to the device, runs hydra_attn_fwd, hydra_lse_merge (if any pair has
+ * partial rows) and hydra_attn_bwd, and copies out, lse, dq, dk, dv back, all enqueued on
+ * `cuda_stream`. Host buffers have the tensor layouts above; pinned memory makes the copies
+ * asynchronous. `device_arena` is device memory, 256-byte aligned, of at least
+ * hydra_host_step_arena_bytes(...) bytes, owned by the caller; the library carves every device
+ * tensor, the partial buffers and the workspace out of it and allocates nothing itself.
+ * Host outputs are valid once the stream has been synchronised.
+ */
+size_t hydra_host_step_arena_bytes(const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
+                                   const hydra_pair_t* pairs, int32_t n_pairs);
+int32_t hydra_attn_fwd_bwd_host(const void* q_host, const void* k_host, const void* v_host,
+                                const void* dout_host, const int32_t* cu_seqlens_host, int32_t n_seqs,
+                                int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs,
+                                int32_t causal, float softmax_scale, void* out_host, float* lse_host,
+                                void* dq_host, void* dk_host, void* dv_host, void* device_arena,
+                                size_t arena_bytes, void* cuda_stream);
+
+/*
+ * Per-kernel timing (measurement aid, not part of the method). While enabled, every kernel launch
+ * is bracketed by CUDA events on its stream. hydra_profile_collect waits for the recorded events,
+ * adds their durations into ms_out[5] and their counts into launches_out[5] (index: 0 forward,
+ * 1 merge, 2 backward prep, 3 backward dK/dV, 4 backward dQ) and forgets them.
+ */
+void hydra_profile_enable(int32_t on);
+int32_t hydra_profile_collect(double* ms_out, int64_t* launches_out);
+
 /* Human-readable name of a status code (static storage). */
 const char* hydra_status_string(int32_t status);
 

@@ -356,22 +356,50 @@ ORACLE_API void oracle_sample_rows(const uint16_t *q, const uint16_t *k, const u
         const int64_t nk = admissible(i, 0, L, causal);
         double *qi = gather_head(q, t, 1, h, a, dqk);
         double *gi = gather_head(dout, t, 1, h, a, dv);
-        double *K = gather_head(k, t0, nk, h, a, dqk);
-        double *V = gather_head(v, t0, nk, h, a, dv);
+        /* keys and values are gathered in blocks so that a late row of a long sequence does not
+         * need a private copy of the whole sequence */
+        enum { BLK = 1024 };
         double *sbuf = (double *)malloc(sizeof(double) * (size_t)(nk > 0 ? nk : 1));
         double *orow = o + s * dv;
-        const double l = row_forward(qi, K, V, 0, nk, dqk, dv, scale, sbuf, orow);
-        lse[s] = l;
+        double *dqrow = dq + s * dqk;
+        for (int e = 0; e < dv; ++e) orow[e] = 0.0;
+        for (int e = 0; e < dqk; ++e) dqrow[e] = 0.0;
+        double m = -INFINITY, l = 0.0;
+        for (int64_t j0 = 0; j0 < nk; j0 += BLK) {
+            const int64_t nb = (nk - j0 < BLK) ? nk - j0 : BLK;
+            double *K = gather_head(k, t0 + j0, nb, h, a, dqk);
+            for (int64_t j = 0; j < nb; ++j) {
+                sbuf[j0 + j] = scale * dot(qi, K + j * dqk, dqk);
+                if (sbuf[j0 + j] > m) m = sbuf[j0 + j];
+            }
+            free(K);
+        }
+        for (int64_t j = 0; j < nk; ++j) l += exp(sbuf[j] - m);
+        const double lse_i = (nk > 0) ? m + log(l) : -INFINITY;
+        for (int64_t j0 = 0; j0 < nk; j0 += BLK) {
+            const int64_t nb = (nk - j0 < BLK) ? nk - j0 : BLK;
+            double *V = gather_head(v, t0 + j0, nb, h, a, dv);
+            for (int64_t j = 0; j < nb; ++j) {
+                const double p = exp(sbuf[j0 + j] - lse_i);
+                for (int e = 0; e < dv; ++e) orow[e] += p * V[j * dv + e];
+            }
+            free(V);
+        }
+        lse[s] = lse_i;
         const double D = dot(gi, orow, dv);
         dsum[s] = D;
-        double *dqrow = dq + s * dqk;
-        for (int e = 0; e < dqk; ++e) dqrow[e] = 0.0;
-        for (int64_t j = 0; j < nk; ++j) {
-            const double p = exp(scale * dot(qi, K + j * dqk, dqk) - l);
-            const double ds = p * (dot(gi, V + j * dv, dv) - D);
-            for (int e = 0; e < dqk; ++e) dqrow[e] += scale * ds * K[j * dqk + e];
+        for (int64_t j0 = 0; j0 < nk; j0 += BLK) {
+            const int64_t nb = (nk - j0 < BLK) ? nk - j0 : BLK;
+            double *K = gather_head(k, t0 + j0, nb, h, a, dqk);
+            double *V = gather_head(v, t0 + j0, nb, h, a, dv);
+            for (int64_t j = 0; j < nb; ++j) {
+                const double p = exp(sbuf[j0 + j] - lse_i);
+                const double ds = p * (dot(gi, V + j * dv, dv) - D);
+                for (int e = 0; e < dqk; ++e) dqrow[e] += scale * ds * K[j * dqk + e];
+            }
+            free(K); free(V);
         }
-        free(qi); free(gi); free(K); free(V); free(sbuf);
+        free(qi); free(gi); free(sbuf);
     }
 }
 

@@ -71,6 +71,15 @@ def _load() -> ctypes.CDLL:
                                    vp, sz, vp]
     lib.hydra_poll_status.restype = i32
     lib.hydra_poll_status.argtypes = [vp, vp, vp, vp]
+    lib.hydra_profile_enable.restype = None
+    lib.hydra_profile_enable.argtypes = [i32]
+    lib.hydra_profile_collect.restype = i32
+    lib.hydra_profile_collect.argtypes = [vp, vp]
+    lib.hydra_host_step_arena_bytes.restype = sz
+    lib.hydra_host_step_arena_bytes.argtypes = [vp, i32, i32, vp, i32]
+    lib.hydra_attn_fwd_bwd_host.restype = i32
+    lib.hydra_attn_fwd_bwd_host.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, i32, i32, f32, vp, vp, vp, vp,
+                                            vp, vp, sz, vp]
     return lib
 
 
@@ -78,7 +87,10 @@ _lib = _load()
 LIBRARY_PATH = _build.OUT
 EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_set_wait_limit_ns",
            "hydra_shutdown", "hydra_usp_factor", "hydra_zigzag_pairs", "hydra_workspace_bytes",
-           "hydra_attn_fwd", "hydra_lse_merge", "hydra_attn_bwd", "hydra_poll_status")
+           "hydra_attn_fwd", "hydra_lse_merge", "hydra_attn_bwd", "hydra_poll_status",
+           "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
+           "hydra_attn_fwd_bwd_host")
+KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq")
 
 
 # ------------------------------------------------------------------------------------------------
@@ -247,3 +259,52 @@ def hydra_poll_status(workspace, stream=None) -> Tuple[int, int]:
     _check(_lib.hydra_poll_status(_ptr(workspace), _stream(stream), ctypes.addressof(st),
                                   ctypes.addressof(detail)), "hydra_poll_status")
     return st.value, detail.value
+
+
+def hydra_profile_enable(on: bool) -> None:
+    _lib.hydra_profile_enable(int(bool(on)))
+
+
+def hydra_profile_collect():
+    """Returns ({kind: total ms}, {kind: launches}) since the last collect."""
+    ms = (ctypes.c_double * 5)()
+    n = (ctypes.c_int64 * 5)()
+    _check(_lib.hydra_profile_collect(ctypes.addressof(ms), ctypes.addressof(n)), "hydra_profile_collect")
+    return dict(zip(KERNEL_KINDS, list(ms))), dict(zip(KERNEL_KINDS, list(n)))
+
+
+def hydra_host_step_arena_bytes(cu_seqlens, n_heads: int, pairs=None) -> int:
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    return int(_lib.hydra_host_step_arena_bytes(cu.ctypes.data, len(cu) - 1, n_heads, pp, npairs))
+
+
+def _host_ptr(x) -> int:
+    """Address of a host buffer: a CPU torch tensor (ideally pinned) or a numpy array."""
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        if not x.flags["C_CONTIGUOUS"]:
+            raise ValueError("host arrays must be contiguous")
+        return x.ctypes.data
+    if x.is_cuda or not x.is_contiguous():
+        raise ValueError("host buffers must be contiguous CPU tensors")
+    return x.data_ptr()
+
+
+def hydra_attn_fwd_bwd_host(q_host, k_host, v_host, dout_host, cu_seqlens, n_heads: int, pairs, causal: bool,
+                            softmax_scale: float, out_host, lse_host, dq_host, dk_host, dv_host, device_arena,
+                            arena_bytes: Optional[int] = None, stream=None, check: bool = True) -> int:
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    if arena_bytes is None:
+        arena_bytes = device_arena.numel() * device_arena.element_size()
+    s = _lib.hydra_attn_fwd_bwd_host(_host_ptr(q_host), _host_ptr(k_host), _host_ptr(v_host),
+                                     _host_ptr(dout_host), cu.ctypes.data, len(cu) - 1, n_heads, pp, npairs,
+                                     int(bool(causal)), ctypes.c_float(float(softmax_scale)),
+                                     _host_ptr(out_host), _host_ptr(lse_host), _host_ptr(dq_host),
+                                     _host_ptr(dk_host), _host_ptr(dv_host), _ptr(device_arena),
+                                     int(arena_bytes), _stream(stream))
+    if check:
+        _check(s, "hydra_attn_fwd_bwd_host")
+    return s

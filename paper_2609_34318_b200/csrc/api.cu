@@ -18,6 +18,43 @@ std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};
 
 constexpr size_t kStatusBytes = 256;
 
+// ---------------------------------------------------------------------------------------------
+// optional per-kernel timing with CUDA events on the launching stream
+// ---------------------------------------------------------------------------------------------
+enum KernelKind { K_FWD = 0, K_MERGE, K_PREP, K_DKV, K_DQ, K_COUNT };
+struct ProfRecord { int kind; cudaEvent_t start, stop; };
+std::mutex g_prof_mutex;
+bool g_prof_on = false;
+std::vector<ProfRecord> g_prof_records;
+std::vector<cudaEvent_t> g_prof_pool;
+
+struct ScopedKernelTimer {
+    cudaStream_t stream;
+    ProfRecord rec{};
+    bool active = false;
+    ScopedKernelTimer(int kind, cudaStream_t s) : stream(s)
+    {
+        std::lock_guard<std::mutex> lock(g_prof_mutex);
+        if (!g_prof_on) return;
+        auto get = [&]() {
+            cudaEvent_t e = nullptr;
+            if (!g_prof_pool.empty()) { e = g_prof_pool.back(); g_prof_pool.pop_back(); }
+            else cudaEventCreate(&e);
+            return e;
+        };
+        rec.kind = kind; rec.start = get(); rec.stop = get();
+        active = rec.start && rec.stop;
+        if (active) cudaEventRecord(rec.start, stream);
+    }
+    ~ScopedKernelTimer()
+    {
+        if (!active) return;
+        cudaEventRecord(rec.stop, stream);
+        std::lock_guard<std::mutex> lock(g_prof_mutex);
+        g_prof_records.push_back(rec);
+    }
+};
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -546,8 +583,6 @@ int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_
                        float softmax_scale, void* out, float* lse, void* o_part, float* lse_part,
                        int64_t part_rows, void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
-    int sms = 0;
-    if (int32_t s = device_info(&sms)) return s;
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
     if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return HYDRA_ERR_INVALID_ARG;
@@ -561,6 +596,8 @@ int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_
         return HYDRA_ERR_INVALID_ARG;
     if (int32_t s = check_part_rows(pb, part_rows)) return s;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int sms = 0;
+    if (int32_t s = device_info(&sms)) return s;
     if (pb.pairs.empty()) return HYDRA_OK;
 
     const Plan* plan = nullptr;
@@ -581,7 +618,10 @@ int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_
     fp.status = static_cast<StatusBlock*>(workspace);
     fp.wait_limit_ns = g_wait_limit_ns.load();
     const int grid = std::min(plan->n_items, sms);
-    if (launch_fwd(mq, mk, mv, fp, grid, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    {
+        ScopedKernelTimer timer(K_FWD, stream);
+        if (launch_fwd(mq, mk, mv, fp, grid, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    }
     g_launches += 1;
     return HYDRA_OK;
 }
@@ -590,20 +630,20 @@ int32_t hydra_lse_merge(const void* o_part, const float* lse_part, int64_t part_
                         int32_t n_seqs, int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs,
                         void* out, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
-    int sms = 0;
-    if (int32_t s = device_info(&sms)) return s;
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
     if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
     if (workspace_bytes < kStatusBytes) return HYDRA_ERR_WORKSPACE_TOO_SMALL;
     bool any_part = false;
     for (const auto& p : pb.pairs) any_part |= (p.part_row >= 0 && p.q_len > 0);
-    if (!any_part) return HYDRA_OK;
-    if (!o_part || !lse_part || !out || !lse || !aligned16(o_part) || !aligned16(lse_part) ||
-        !aligned16(out) || !aligned16(lse) || part_rows <= 0)
+    if (any_part && (!o_part || !lse_part || !out || !lse || !aligned16(o_part) || !aligned16(lse_part) ||
+        !aligned16(out) || !aligned16(lse) || part_rows <= 0))
         return HYDRA_ERR_INVALID_ARG;
     if (int32_t s = check_part_rows(pb, part_rows)) return s;
+    if (!any_part) return HYDRA_OK;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int sms = 0;
+    if (int32_t s = device_info(&sms)) return s;
     const Plan* plan = nullptr;
     if (int32_t s = get_plan(HYDRA_WS_MERGE, pb, 0, &plan)) return s;
     MergeParams mp{};
@@ -613,7 +653,10 @@ int32_t hydra_lse_merge(const void* o_part, const float* lse_part, int64_t part_
     mp.n_items = plan->n_items;
     mp.o_part = o_part; mp.lse_part = lse_part; mp.out = out; mp.lse = lse;
     mp.T = pb.T; mp.part_rows = part_rows; mp.h = n_heads;
-    if (launch_merge(mp, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    {
+        ScopedKernelTimer timer(K_MERGE, stream);
+        if (launch_merge(mp, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    }
     g_launches += 1;
     return HYDRA_OK;
 }
@@ -624,8 +667,6 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
                        void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes,
                        void* cuda_stream)
 {
-    int sms = 0;
-    if (int32_t s = device_info(&sms)) return s;
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
     if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return HYDRA_ERR_INVALID_ARG;
@@ -645,6 +686,8 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
         if (check_identical_or_disjoint(rq) || check_identical_or_disjoint(rk)) return HYDRA_ERR_INVALID_ARG;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int sms = 0;
+    if (int32_t s = device_info(&sms)) return s;
     const Plan* plan = nullptr;
     if (int32_t s = get_plan(HYDRA_WS_BWD, pb, causal != 0, &plan)) return s;
 
@@ -655,7 +698,10 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
         make_map(&mq_sub, q, pb.T, n_heads, D_QK, SUB) || make_map(&mdo_sub, dout, pb.T, n_heads, D_V, SUB))
         return HYDRA_ERR_CUDA;
     if (int32_t s = reset_status(workspace, stream)) return s;
-    if (launch_bwd_prep(dout, out, dsum, pb.T, n_heads, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    {
+        ScopedKernelTimer timer(K_PREP, stream);
+        if (launch_bwd_prep(dout, out, dsum, pb.T, n_heads, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    }
     g_launches += 1;
 
     BwdParams bp{};
@@ -669,6 +715,7 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
         bp.lists = at<int32_t>(*plan, plan->off_lists2);
         bp.items = at<GroupItem>(*plan, plan->off_items2);
         bp.n_items = plan->n_items2;
+        ScopedKernelTimer timer(K_DKV, stream);
         if (launch_bwd_dkv(mq_sub, mk, mv, mdo_sub, bp, std::min(plan->n_items2, sms), stream) != cudaSuccess)
             return HYDRA_ERR_CUDA;
         g_launches += 1;
@@ -677,10 +724,111 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
         bp.lists = at<int32_t>(*plan, plan->off_lists);
         bp.items = at<GroupItem>(*plan, plan->off_items);
         bp.n_items = plan->n_items;
+        ScopedKernelTimer timer(K_DQ, stream);
         if (launch_bwd_dq(mq, mk, mv, mdo, bp, std::min(plan->n_items, sms), stream) != cudaSuccess)
             return HYDRA_ERR_CUDA;
         g_launches += 1;
     }
+    return HYDRA_OK;
+}
+
+void hydra_profile_enable(int32_t on)
+{
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    g_prof_on = on != 0;
+}
+
+int32_t hydra_profile_collect(double* ms_out, int64_t* launches_out)
+{
+    if (!ms_out || !launches_out) return HYDRA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    for (int i = 0; i < K_COUNT; ++i) { ms_out[i] = 0.0; launches_out[i] = 0; }
+    int32_t status = HYDRA_OK;
+    for (const ProfRecord& r : g_prof_records) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(r.stop) != cudaSuccess || cudaEventElapsedTime(&ms, r.start, r.stop) != cudaSuccess)
+            status = HYDRA_ERR_CUDA;
+        ms_out[r.kind] += ms;
+        launches_out[r.kind] += 1;
+        g_prof_pool.push_back(r.start);
+        g_prof_pool.push_back(r.stop);
+    }
+    g_prof_records.clear();
+    return status;
+}
+
+size_t hydra_host_step_arena_bytes(const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                                   const hydra_pair_t* pairs, int32_t n_pairs)
+{
+    Problem pb;
+    if (make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb) != HYDRA_OK) return 0;
+    int64_t part_rows = 0;
+    for (const auto& p : pb.pairs)
+        if (p.part_row >= 0) part_rows = std::max<int64_t>(part_rows, int64_t{p.part_row} + p.q_len);
+    const size_t th = static_cast<size_t>(std::max<int64_t>(pb.T, 1)) * n_heads;
+    size_t b = 0;
+    b += 3 * align_up(th * D_QK * 2, 256);                   // q, k + dq/dk share nothing: q, k, dq
+    b += 1 * align_up(th * D_QK * 2, 256);                   // dk
+    b += 4 * align_up(th * D_V * 2, 256);                    // v, dout, out, dv
+    b += align_up(th * 4, 256);                              // lse
+    b += align_up(static_cast<size_t>(std::max<int64_t>(part_rows, 1)) * n_heads * D_V * 2, 256);
+    b += align_up(static_cast<size_t>(std::max<int64_t>(part_rows, 1)) * n_heads * 4, 256);
+    b += kStatusBytes + align_up(th * 4, 256);               // workspace of the backward call
+    return b;
+}
+
+int32_t hydra_attn_fwd_bwd_host(const void* q_host, const void* k_host, const void* v_host,
+                                const void* dout_host, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                                const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal,
+                                float softmax_scale, void* out_host, float* lse_host, void* dq_host,
+                                void* dk_host, void* dv_host, void* device_arena, size_t arena_bytes,
+                                void* cuda_stream)
+{
+    Problem pb;
+    if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
+    const void* ptrs[] = {q_host, k_host, v_host, dout_host, out_host, lse_host, dq_host, dk_host, dv_host};
+    for (const void* p : ptrs)
+        if (!p) return HYDRA_ERR_INVALID_ARG;
+    if (!device_arena || (reinterpret_cast<uintptr_t>(device_arena) & 255u)) return HYDRA_ERR_INVALID_ARG;
+    if (arena_bytes < hydra_host_step_arena_bytes(cu, n_seqs, n_heads, pairs, n_pairs))
+        return HYDRA_ERR_WORKSPACE_TOO_SMALL;
+    if (pb.T == 0) return HYDRA_OK;
+    int64_t part_rows = 0;
+    for (const auto& p : pb.pairs)
+        if (p.part_row >= 0) part_rows = std::max<int64_t>(part_rows, int64_t{p.part_row} + p.q_len);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t th = static_cast<size_t>(pb.T) * n_heads;
+    uint8_t* cur = static_cast<uint8_t*>(device_arena);
+    auto carve = [&](size_t bytes) { void* p = cur; cur += align_up(bytes, 256); return p; };
+    void* dq_ = carve(th * D_QK * 2); void* dk_ = carve(th * D_QK * 2);
+    void* q = carve(th * D_QK * 2); void* k = carve(th * D_QK * 2);
+    void* v = carve(th * D_V * 2); void* dout = carve(th * D_V * 2);
+    void* out = carve(th * D_V * 2); void* dv_ = carve(th * D_V * 2);
+    float* lse = static_cast<float*>(carve(th * 4));
+    void* o_part = carve(static_cast<size_t>(std::max<int64_t>(part_rows, 1)) * n_heads * D_V * 2);
+    float* lse_part = static_cast<float*>(carve(static_cast<size_t>(std::max<int64_t>(part_rows, 1)) * n_heads * 4));
+    void* ws = carve(kStatusBytes + align_up(th * 4, 256));
+    const size_t ws_bytes = kStatusBytes + align_up(th * 4, 256);
+    auto h2d = [&](void* d, const void* h, size_t n) { return cudaMemcpyAsync(d, h, n, cudaMemcpyHostToDevice, stream); };
+    auto d2h = [&](void* h, const void* d, size_t n) { return cudaMemcpyAsync(h, d, n, cudaMemcpyDeviceToHost, stream); };
+    if (h2d(q, q_host, th * D_QK * 2) || h2d(k, k_host, th * D_QK * 2) || h2d(v, v_host, th * D_V * 2) ||
+        h2d(dout, dout_host, th * D_V * 2))
+        return HYDRA_ERR_CUDA;
+    const bool any_part = part_rows > 0;
+    if (int32_t s = hydra_attn_fwd(q, k, v, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, out, lse,
+                                   any_part ? o_part : nullptr, any_part ? lse_part : nullptr, part_rows, ws,
+                                   ws_bytes, cuda_stream))
+        return s;
+    if (any_part)
+        if (int32_t s = hydra_lse_merge(o_part, lse_part, part_rows, cu, n_seqs, n_heads, pairs, n_pairs, out,
+                                        lse, ws, ws_bytes, cuda_stream))
+            return s;
+    if (int32_t s = hydra_attn_bwd(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal,
+                                   softmax_scale, dq_, dk_, dv_, ws, ws_bytes, cuda_stream))
+        return s;
+    if (d2h(out_host, out, th * D_V * 2) || d2h(lse_host, lse, th * 4) || d2h(dq_host, dq_, th * D_QK * 2) ||
+        d2h(dk_host, dk_, th * D_QK * 2) || d2h(dv_host, dv_, th * D_V * 2))
+        return HYDRA_ERR_CUDA;
     return HYDRA_OK;
 }
 

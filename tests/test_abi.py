@@ -1,0 +1,153 @@
+"""CPU-side checks of the C ABI: the library loads, exports what include/hydra_attn.h declares,
+its host-only entry points agree bit for bit with the oracle's integer bookkeeping, and argument
+validation returns the documented codes. No kernel runs here."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2609_34318_b200 as P
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    with open(os.path.join(ROOT, "include", "hydra_attn.h")) as f:
+        text = re.sub(r"/\*.*?\*/", "", f.read(), flags=re.S)
+    return sorted(set(re.findall(r"\b(hydra_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_symbols()
+    assert {"hydra_attn_fwd", "hydra_attn_bwd", "hydra_lse_merge"} <= set(names)
+    lib = ctypes.CDLL(P.LIBRARY_PATH)
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in the header but not exported"
+    assert set(n for n in P.EXPORTS) <= set(names)
+
+
+def test_binding_has_the_same_names():
+    for n in declared_symbols():
+        assert hasattr(P, n), f"binding lacks {n}"
+
+
+def test_version_and_status_strings():
+    assert P.hydra_version() >= 1
+    assert P.hydra_status_string(0) == "HYDRA_OK"
+    assert P.hydra_status_string(5) == "HYDRA_ERR_DEVICE_TIMEOUT"
+    assert P.hydra_status_string(99) == "HYDRA_ERR_UNKNOWN"
+
+
+def test_usp_factor_matches_oracle_and_paper_values():
+    assert P.hydra_usp_factor(256, 64) == (64, 4)         # Section 5.2: ring of four at P=256, h=64
+    for degree, heads in [(1, 1), (8, 64), (64, 64), (128, 64), (32, 8), (16, 16), (2, 3)]:
+        assert P.hydra_usp_factor(degree, heads) == oracle.usp_factor(degree, heads)
+    with pytest.raises(P.HydraError):
+        P.hydra_usp_factor(0, 4)
+    with pytest.raises(P.HydraError):
+        P.hydra_usp_factor(12, 8)                         # 8 does not divide 12
+
+
+@pytest.mark.parametrize("lengths,cp_r", [([300], 1), ([262144], 4), ([7, 33, 128, 300], 0),
+                                          ([5, 0, 3, 1000, 1], 2), ([1, 2, 3], 4), ([100, 200], [0, 2])])
+def test_zigzag_pairs_match_the_oracle_bit_for_bit(lengths, cp_r):
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    pairs, part_rows, rank, step = P.hydra_zigzag_pairs(cu, cp_r)
+    ref = oracle.causal_pairs(cu, cp_r)
+    assert len(pairs) == len(ref)
+    rows = 0
+    by_group = {}
+    for p in ref:
+        by_group.setdefault(p["group"], []).append(p)
+    for i, r in enumerate(ref):
+        for name in ("seq", "q_start", "q_len", "k_start", "k_len", "group"):
+            assert int(pairs[i][name]) == r[name], (i, name)
+        assert int(rank[i]) == r["rank"] and int(step[i]) == r["step"]
+        if len(by_group[r["group"]]) > 1:
+            assert int(pairs[i]["part_row"]) == rows
+            rows += r["q_len"]
+        else:
+            assert int(pairs[i]["part_row"]) == -1
+    assert part_rows == rows
+
+
+def test_zigzag_pairs_rejects_bad_input():
+    with pytest.raises(P.HydraError):
+        P.hydra_zigzag_pairs([0, 10, 5], 1)      # decreasing cu_seqlens
+    with pytest.raises(P.HydraError):
+        P.hydra_zigzag_pairs([1, 10], 1)         # does not start at 0
+    with pytest.raises(P.HydraError):
+        P.hydra_zigzag_pairs([0, 10], -1)
+
+
+def test_workspace_bytes():
+    cu = [0, 100, 300]
+    assert P.hydra_workspace_bytes(P.HYDRA_WS_FWD, cu, 4) >= 16
+    small = P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, 4)
+    big = P.hydra_workspace_bytes(P.HYDRA_WS_BWD, [0, 100, 3000], 4)
+    assert small >= 300 * 4 * 4 and big > small               # holds D [h, T] fp32; monotone in T
+    assert P.hydra_workspace_bytes(P.HYDRA_WS_BWD, [0, 100, 50], 4) == 0     # invalid input
+    assert P.hydra_workspace_bytes(7, cu, 4) == 0
+
+
+def _call_fwd(cu, h, pairs, ws=0x1000, ws_bytes=4096, q=0x1000, out=0x1000, part=0x1000, part_rows=0,
+              scale=0.07):
+    return P.hydra_attn_fwd(q, q, q, cu, h, pairs, True, scale, out, out, part, part, part_rows, ws,
+                            ws_bytes, stream=0, check=False)
+
+
+def test_forward_validation_codes_without_a_gpu():
+    cu = [0, 64, 200]
+    ok_pair = dict(seq=1, q_start=0, q_len=136, k_start=0, k_len=136, group=0)
+    assert _call_fwd([0, 64, 32], 2, None) == P.HYDRA_ERR_INVALID_ARG                 # non-monotone
+    assert _call_fwd(cu, 0, None) == P.HYDRA_ERR_INVALID_ARG                          # no heads
+    assert _call_fwd(cu, 2, None, scale=0.0) == P.HYDRA_ERR_INVALID_ARG
+    assert _call_fwd(cu, 2, None, ws=0x1004) == P.HYDRA_ERR_INVALID_ARG               # misaligned
+    assert _call_fwd(cu, 2, None, ws_bytes=8) == P.HYDRA_ERR_WORKSPACE_TOO_SMALL
+    assert _call_fwd(cu, 2, None, q=0) == P.HYDRA_ERR_INVALID_ARG                     # null tensor
+    bad = dict(ok_pair, q_len=137)
+    assert _call_fwd(cu, 2, [bad]) == P.HYDRA_ERR_INVALID_ARG                         # pair leaves its sequence
+    assert _call_fwd(cu, 2, [dict(ok_pair, seq=2)]) == P.HYDRA_ERR_INVALID_ARG
+    assert _call_fwd(cu, 2, [dict(ok_pair, flags=1)]) == P.HYDRA_ERR_INVALID_ARG
+    two = [dict(ok_pair, k_len=60, part_row=0), dict(ok_pair, k_start=60, k_len=76, part_row=100)]
+    assert _call_fwd(cu, 2, two, part_rows=300) == P.HYDRA_ERR_INVALID_ARG            # partial rows overlap
+    assert _call_fwd(cu, 2, two[:1] + [dict(two[1], part_row=136)], part_rows=200) == P.HYDRA_ERR_INVALID_ARG
+    differing = [dict(ok_pair, part_row=0), dict(ok_pair, q_len=100, part_row=136)]
+    assert _call_fwd(cu, 2, differing, part_rows=400) == P.HYDRA_ERR_INVALID_ARG      # group with two q ranges
+    unordered = [dict(ok_pair, group=1), dict(ok_pair, seq=0, q_len=64, k_len=64, group=0)]
+    assert _call_fwd(cu, 2, unordered) == P.HYDRA_ERR_INVALID_ARG
+
+
+def test_backward_requires_identical_or_disjoint_chunks():
+    cu = [0, 256]
+    overlapping = [dict(seq=0, q_start=0, q_len=128, k_start=0, k_len=128, group=0),
+                   dict(seq=0, q_start=64, q_len=128, k_start=0, k_len=128, group=1)]
+    s = P.hydra_attn_bwd(0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, cu, 2, overlapping, True, 0.07,
+                         0x1000, 0x1000, 0x1000, 0x1000, 1 << 20, stream=0, check=False)
+    assert s == P.HYDRA_ERR_INVALID_ARG
+    s = P.hydra_attn_bwd(0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, cu, 2, None, True, 0.07,
+                         0x1000, 0x1000, 0x1000, 0x1000, 64, stream=0, check=False)
+    assert s == P.HYDRA_ERR_WORKSPACE_TOO_SMALL
+
+
+def test_no_cpu_fallback():
+    """With valid arguments and no usable device the call fails loudly instead of computing."""
+    torch = pytest.importorskip("torch")
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    s = _call_fwd([0, 64, 200], 2, None)
+    assert s in (P.HYDRA_ERR_CUDA, P.HYDRA_ERR_NOT_SM100)
+
+
+def test_product_does_not_import_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2609_34318_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                with open(os.path.join(dirpath, f)) as fh:
+                    text = fh.read()
+                assert "import oracle" not in text and "from oracle" not in text, f
+                assert "hydra_oracle" not in text, f

@@ -1,0 +1,156 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 oracle on the same seeded inputs.
+
+Tolerances (stated by the benchmark contract): max |gpu - ref| <= 2e-2 * max |ref| on O, dQ, dK, dV
+and <= 1e-3 absolute on LSE, bf16 inputs with fp32 accumulation.
+"""
+import numpy as np
+import pytest
+
+import hydra_workloads as hw
+import oracle
+from gpu_util import TOL_LSE, TOL_REL, check, pairs_for, row_rel_err, run_gpu, run_oracle
+
+pytestmark = pytest.mark.gpu
+DQK, DV = hw.D_QK, hw.D_V
+
+
+def rand_inputs(rng, T, h, q_scale=1.0):
+    f = lambda d, s=1.0: hw.f32_to_bf16_bits((s * rng.standard_normal((T, h, d))).astype(np.float32))
+    return dict(q=f(DQK, q_scale), k=f(DQK), v=f(DV), do=f(DV))
+
+
+def run_case(lengths, h, cp_r=0, causal=True, x=None, seed=0, label=""):
+    cu = hw.cu_seqlens(lengths)
+    T = int(cu[-1])
+    if x is None:
+        x = rand_inputs(np.random.default_rng(seed), T, h)
+    lib_pairs, rows, ora_pairs = pairs_for(cu, cp_r) if cp_r else (None, 0, None)
+    got = run_gpu(x, cu, h, lib_pairs, rows, causal)
+    ref = run_oracle(x, cu, causal, pairs=ora_pairs)
+    rep = check(got, ref, label=label)
+    return got, ref, rep
+
+
+# ------------------------------------------------------------------------------------------------
+# the two small configurations, in full
+# ------------------------------------------------------------------------------------------------
+def test_tiny_config_all_tensors():
+    w = hw.workload("tiny")
+    x = w.tensors()
+    got, ref, _ = run_case(w.lengths, w.n_heads, x=x, label="tiny ")
+    assert row_rel_err(got["out"], ref["out"]) < 2e-2
+
+
+def test_tiny_two_chunk_split_through_the_merge():
+    w = hw.workload("tiny")
+    x = w.tensors()
+    cu = w.cu()
+    # only the 300-token sequence is cut (2 chunks -> 3 pairs, merged); the others keep one pair
+    lib_pairs, rows, ora_pairs = pairs_for(cu, [0, 0, 0, 1])
+    assert len(lib_pairs) == 6 and rows == 300
+    got = run_gpu(x, cu, w.n_heads, lib_pairs, rows)
+    ref = run_oracle(x, cu, pairs=ora_pairs)
+    check(got, ref, label="tiny split ")
+    # the partial buffers hold what the oracle's per-pair partials say
+    step = got["_step"]
+    o_part = step.o_part.float().cpu().numpy().astype(np.float64)
+    lse_part = step.lse_part.cpu().numpy().astype(np.float64)
+    for lp, op in zip(lib_pairs, ora_pairs):
+        if lp["part_row"] < 0:
+            continue
+        o, l = oracle.attn_partial(x["q"], x["k"], x["v"], cu, op, True, w.scale)
+        r0, n = int(lp["part_row"]), int(lp["q_len"])
+        assert np.abs(o_part[r0:r0 + n] - o).max() <= TOL_REL * np.abs(o).max()
+        assert np.abs(lse_part[:, r0:r0 + n] - l).max() <= TOL_LSE
+
+
+# ------------------------------------------------------------------------------------------------
+# directed shapes: tile edges, ragged tails, unaligned starts
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("lengths", [[1], [7], [127], [128], [129], [255], [256], [257], [300],
+                                     [1, 1, 1, 2], [63, 65, 64], [5, 128, 3, 129, 384, 1],
+                                     [0, 17, 0, 140, 0]])
+def test_boundary_lengths(lengths):
+    run_case(lengths, 2, seed=sum(lengths))
+
+
+@pytest.mark.parametrize("cp_r", [1, 2, 4])
+def test_zigzag_chunks_with_unequal_sizes(cp_r):
+    run_case([1001, 77, 5, 300], 2, cp_r=cp_r, seed=cp_r)
+
+
+def test_non_causal_pairs():
+    run_case([200, 130, 64], 2, causal=False, seed=3)
+
+
+def test_many_heads_and_longer_sequences():
+    run_case([1500, 700, 90], 5, seed=4)
+
+
+# ------------------------------------------------------------------------------------------------
+# directed numerics
+# ------------------------------------------------------------------------------------------------
+def test_spike_upstream_gradient_on_a_late_row():
+    rng = np.random.default_rng(5)
+    L, h = 900, 2
+    x = rand_inputs(rng, L, h)
+    do = np.zeros((L, h, DV), dtype=np.float32)
+    do[L - 3] = rng.standard_normal((h, DV))
+    x["do"] = hw.f32_to_bf16_bits(do)
+    got, ref, _ = run_case([L], h, x=x)          # max |ref| is now set by that one row's gradients
+    assert row_rel_err(got["dq"][L - 3:L - 2], ref["dq"][L - 3:L - 2]) < 2e-2
+    assert np.abs(got["dq"][:L - 3]).max() == 0.0 and np.abs(got["dq"][L - 2:]).max() == 0.0
+
+
+def test_one_hot_values_reveal_which_keys_contribute():
+    rng = np.random.default_rng(6)
+    L, h = 640, 1
+    x = rand_inputs(rng, L, h)
+    v = np.zeros((L, h, DV), dtype=np.float32)
+    v[np.arange(L), 0, np.arange(L) % DV] = 1.0
+    x["v"] = hw.f32_to_bf16_bits(v)
+    got, ref, _ = run_case([L], h, x=x)
+    assert np.abs(got["out"] - ref["out"]).max() < 2e-2 * np.abs(ref["out"]).max()
+
+
+@pytest.mark.parametrize("direction", [+1.0, -1.0])
+def test_monotone_scores_exercise_the_running_max(direction):
+    """<q, k_j> grows (or falls) with j, so the row maximum rises at every kv tile (or never)."""
+    rng = np.random.default_rng(7)
+    L, h = 700, 1
+    x = rand_inputs(rng, L, h)
+    k = 0.05 * rng.standard_normal((L, h, DQK)).astype(np.float32)
+    k[:, :, 0] = direction * np.linspace(-6.0, 6.0, L)[:, None]
+    q = 0.05 * rng.standard_normal((L, h, DQK)).astype(np.float32)
+    q[:, :, 0] = 8.0
+    x["k"], x["q"] = hw.f32_to_bf16_bits(k), hw.f32_to_bf16_bits(q)
+    run_case([L], h, x=x)
+
+
+def test_large_scores():
+    rng = np.random.default_rng(8)
+    L, h = 520, 2
+    x = rand_inputs(rng, L, h, q_scale=8.0)
+    run_case([L], h, x=x)
+
+
+def test_repeatable_bit_for_bit():
+    """No atomics anywhere: two runs on the same inputs give identical bits."""
+    w = hw.workload("tiny")
+    x = w.tensors()
+    a = run_gpu(x, w.cu(), w.n_heads)
+    b = run_gpu(x, w.cu(), w.n_heads)
+    for n in ("out", "lse", "dq", "dk", "dv"):
+        assert np.array_equal(a[n], b[n]), n
+
+
+def test_rows_outside_the_listed_pairs_are_left_untouched():
+    rng = np.random.default_rng(9)
+    lengths = [200, 150]
+    cu = hw.cu_seqlens(lengths)
+    x = rand_inputs(rng, 350, 2)
+    only_second = [dict(seq=1, q_start=0, q_len=150, k_start=0, k_len=150, group=0)]
+    got = run_gpu(x, cu, 2, only_second, 0)
+    assert np.isnan(got["out"][:200]).all() and np.isnan(got["dq"][:200]).all()
+    ref = run_oracle({n: a[200:] for n, a in x.items()}, hw.cu_seqlens([150]))
+    check({n: (got[n][:, 200:] if n == "lse" else got[n][200:]) for n in ref}, ref)
