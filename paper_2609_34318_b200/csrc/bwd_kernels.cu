@@ -8,6 +8,14 @@
 // dS = P (dP - D) on thread-private rows, hand P / dS back to the tensor core as packed bf16 in
 // tensor memory (A operand of a TS UMMA), and read Q / K / dO as MN-major B operands straight from
 // their token-major TMA tiles, so nothing is transposed in shared memory.
+//
+// Warp roles (320 threads) in both kernels:
+//   warps 0-3, 4-7  two elementwise warpgroups; thread r of each owns tile row r = TMEM lane r and
+//                   one half of the columns of S / dP
+//   warp 8          TMA producer (plus the LSE / D loads of the dK/dV kernel)
+//   warp 9          UMMA issuer (one thread), owner of the TMEM allocation
+// The elementwise threads copy S and dP to registers and release them at once, so that the UMMAs of
+// the next step run while the exponentials of this one are computed.
 #include <cuda_bf16.h>
 
 #include "hydra_internal.h"
@@ -17,9 +25,11 @@ namespace hydra {
 
 namespace {
 
-constexpr int kThreads = 128;
+constexpr int kThreads = 320;
+constexpr int kWarpProd = 8, kWarpMma = 9;
 constexpr uint32_t kBox128 = 128 * 128;   // [128 rows x 64 bf16]
 constexpr uint32_t kBox64 = 64 * 128;     // [ 64 rows x 64 bf16]
+constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
 __device__ __forceinline__ float pos_inf() { return __int_as_float(0x7f800000); }
@@ -39,28 +49,81 @@ __device__ __forceinline__ void store_row_bf16(__nv_bfloat16* dst, const uint32_
 }
 
 // ---------------------------------------------------------------------------------------------
-// dQ kernel
+// dQ kernel: layout
 // ---------------------------------------------------------------------------------------------
 namespace dq {
-constexpr uint32_t kQ = 0;                          // 3 boxes
-constexpr uint32_t kDO = kQ + 3 * kBox128;          // 2 boxes
-constexpr uint32_t kK = kDO + 2 * kBox128;          // 2 stages x 3 boxes
-constexpr uint32_t kV = kK + 2 * 3 * kBox128;       // 1 stage x 2 boxes
-constexpr uint32_t kTotal = kV + 2 * kBox128;       // 212,992 B
+constexpr int kKStages = 2, kVSlots = 3;
+constexpr uint32_t kQ = 0;                                   // 3 boxes, stationary
+constexpr uint32_t kDO = kQ + 3 * kBox128;                   // 2 boxes, stationary
+constexpr uint32_t kK = kDO + 2 * kBox128;                   // 2 stages x 3 boxes
+constexpr uint32_t kV = kK + kKStages * 3 * kBox128;         // ring of 3 boxes [128 kv x 64 d_v]
+constexpr uint32_t kTotal = kV + kVSlots * kBox128;          // 229,376 B
 constexpr uint32_t kTmS = 0, kTmDP = 128, kTmDQ = 256, kTmDS = 448, kTmCols = 512;
+enum : int { B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_KEMPTY = 4, B_VFULL = 6, B_VEMPTY = 9,
+             B_SFULL = 12, B_SFREE = 13, B_PFULL = 14, B_DSFREE = 15, B_ACCFREE = 16, B_COUNT = 17 };
+
+// Iterator over (pair of the q chunk, kv tile) in the order every role walks them.
+struct TileIter {
+    const PairDev* pairs; const int32_t* list; int list_len; int last_row; int causal;
+    int li, t, nt; PairDev cur;
+    __device__ int tiles_of(const PairDev& pr) const {
+        int n_keys = pr.k_len;
+        if (causal) n_keys = min(n_keys, last_row + pr.off + 1);
+        return n_keys > 0 ? (n_keys + TILE - 1) / TILE : 0;
+    }
+    __device__ void seek() {
+        while (li < list_len) {
+            cur = pairs[list[li]];
+            nt = tiles_of(cur);
+            if (nt > 0) return;
+            ++li;
+        }
+    }
+    __device__ void init(const PairDev* p, const int32_t* l, int n, int lr, int c) {
+        pairs = p; list = l; list_len = n; last_row = lr; causal = c; li = 0; t = 0; nt = 0;
+        seek();
+    }
+    __device__ bool valid() const { return li < list_len; }
+    __device__ void next() { if (++t >= nt) { t = 0; ++li; seek(); } }
+};
 }  // namespace dq
 
 // ---------------------------------------------------------------------------------------------
-// dK/dV kernel
+// dK/dV kernel: layout
 // ---------------------------------------------------------------------------------------------
 namespace dkv {
-constexpr uint32_t kK = 0;                          // 3 boxes of 128 rows
-constexpr uint32_t kV = kK + 3 * kBox128;           // 2 boxes of 128 rows
-constexpr uint32_t kQ = kV + 2 * kBox128;           // 2 stages x 3 boxes of 64 rows
-constexpr uint32_t kDO = kQ + 2 * 3 * kBox64;       // 2 stages x 2 boxes of 64 rows
-constexpr uint32_t kTotal = kDO + 2 * 2 * kBox64;   // 163,840 B
+constexpr int kStages = 3;
+constexpr uint32_t kK = 0;                                   // 3 boxes of 128 rows, stationary
+constexpr uint32_t kV = kK + 3 * kBox128;                    // 2 boxes of 128 rows, stationary
+constexpr uint32_t kQ = kV + 2 * kBox128;                    // stages x 3 boxes of 64 rows
+constexpr uint32_t kDO = kQ + kStages * 3 * kBox64;          // stages x 2 boxes of 64 rows
+constexpr uint32_t kTotal = kDO + kStages * 2 * kBox64;      // 204,800 B
 constexpr uint32_t kTmDK = 0, kTmDV = 192, kTmS = 320, kTmDP = 384, kTmP = 448, kTmDS = 480,
                    kTmCols = 512;
+enum : int { B_KVFULL = 0, B_KVEMPTY = 1, B_QFULL = 2, B_STAT = 5, B_QEMPTY = 8, B_SFULL = 11,
+             B_SFREE = 12, B_PFULL = 13, B_PDSFREE = 14, B_ACCFREE = 15, B_COUNT = 16 };
+
+// Iterator over (pair of the kv chunk, 64-row q sub-tile).
+struct SubIter {
+    const PairDev* pairs; const int32_t* list; int list_len; int r0; int causal;
+    int li, u, nu; PairDev cur;
+    __device__ void seek() {
+        while (li < list_len) {
+            cur = pairs[list[li]];
+            nu = (cur.q_len + SUB - 1) / SUB;
+            u = 0;
+            if (causal) { const int i_min = r0 - cur.off; u = i_min > 0 ? i_min / SUB : 0; }
+            if (u < nu) return;
+            ++li;
+        }
+    }
+    __device__ void init(const PairDev* p, const int32_t* l, int n, int r, int c) {
+        pairs = p; list = l; list_len = n; r0 = r; causal = c; li = 0; u = 0; nu = 0;
+        seek();
+    }
+    __device__ bool valid() const { return li < list_len; }
+    __device__ void next() { if (++u >= nu) { ++li; seek(); } }
+};
 }  // namespace dkv
 
 }  // namespace
@@ -68,6 +131,9 @@ constexpr uint32_t kTmDK = 0, kTmDV = 192, kTmS = 320, kTmDP = 384, kTmP = 448, 
 size_t bwd_dq_smem_bytes() { return dq::kTotal + 1024; }
 size_t bwd_dkv_smem_bytes() { return dkv::kTotal + 1024; }
 
+// =============================================================================================
+// dQ
+// =============================================================================================
 __global__ void __launch_bounds__(kThreads, 1)
 hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
@@ -76,230 +142,266 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     using namespace dq;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    __shared__ __align__(8) uint64_t bars[8];
+    __shared__ __align__(8) uint64_t bars[B_COUNT];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
-    const int tid = threadIdx.x, warp = tid >> 5;
-    const uint32_t bar_q = smem_u32(&bars[0]);      // Q and dO of the item
-    const uint32_t bar_k0 = smem_u32(&bars[1]);     // + 8 * stage
-    const uint32_t bar_v = smem_u32(&bars[3]);
-    const uint32_t bar_s = smem_u32(&bars[4]);      // S and dP complete
-    const uint32_t bar_acc = smem_u32(&bars[5]);    // dQ += dS K complete
-
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t bar0 = smem_u32(&bars[0]);
+    auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
     if (tid == 0) {
         abort_flag = 0;
-        mbar_init(bar_q, 1); mbar_init(bar_k0, 1); mbar_init(bar_k0 + 8, 1);
-        mbar_init(bar_v, 1); mbar_init(bar_s, 1); mbar_init(bar_acc, 1);
+        for (int i = 0; i < B_COUNT; ++i) {
+            const bool by_threads = (i == B_SFREE) || (i == B_PFULL) || (i == B_ACCFREE);
+            mbar_init(bar(i), by_threads ? 256u : 1u);
+        }
         fence_mbar_init();
         tma_prefetch_desc(&map_q); tma_prefetch_desc(&map_k);
         tma_prefetch_desc(&map_v); tma_prefetch_desc(&map_do);
     }
-    if (warp == 0) { tmem_alloc(smem_u32(&tmem_base_slot), kTmCols); tmem_relinquish(); }
+    if (warp == kWarpMma) { tmem_alloc(smem_u32(&tmem_base_slot), kTmCols); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tm = tmem_base_slot;
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
     const uint64_t limit = p.wait_limit_ns;
+    const int it_begin = p.cta_off[blockIdx.x], it_end = p.cta_off[blockIdx.x + 1];
+    volatile int* abort_p = &abort_flag;
+    auto wait = [&](int b, uint32_t parity) -> bool { return mbar_wait(bar(b), parity & 1u, abort_p, limit); };
 
-    constexpr uint32_t idesc_s = umma_idesc_bf16(TILE, TILE, false, false);
-    constexpr uint32_t idesc_dq = umma_idesc_bf16(TILE, D_QK, false, true);
-
-    uint32_t ph_q = 0, ph_k[2] = {0, 0}, ph_v = 0, ph_s = 0, ph_acc = 0;
-    bool ok = true;
-
-    for (int it = blockIdx.x; it < p.n_items && ok; it += gridDim.x) {
-        const GroupItem item = p.items[it];
-        const int head = item.head, r0 = item.r0;
-        const int32_t* list = p.lists + item.list_off;
-        const PairDev first = p.pairs[list[0]];
-        const int row = r0 + tid;
-        const bool row_valid = row < first.q_len;
-        const int last_row = min(r0 + TILE, first.q_len) - 1;
-
-        auto tiles_of = [&](const PairDev& pr) -> int {
-            int n_keys = pr.k_len;
-            if (p.causal) n_keys = min(n_keys, last_row + pr.off + 1);
-            return n_keys > 0 ? (n_keys + TILE - 1) / TILE : 0;
-        };
-        // iterator over (pair of the chunk, kv tile)
-        int li = 0, t = 0, nt = 0;
-        PairDev cur = first;
-        auto seek = [&]() {          // move to the first pair at or after li that has tiles
-            while (li < item.list_len) {
-                cur = p.pairs[list[li]];
-                nt = tiles_of(cur);
-                if (nt > 0) return;
-                ++li;
-            }
-        };
-        seek();
-        int nli = li, ntile = t;     // lookahead iterator (next tile to prefetch)
-        PairDev nxt = cur; int nnt = nt;
-        auto advance_next = [&]() {
-            ++ntile;
-            if (ntile >= nnt) {
-                ntile = 0; ++nli;
-                while (nli < item.list_len) {
-                    nxt = p.pairs[list[nli]];
-                    nnt = tiles_of(nxt);
-                    if (nnt > 0) break;
-                    ++nli;
+    if (warp == kWarpProd) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t items = 0, gk = 0, gv = 0;
+            bool ok = true;
+            for (int it = it_begin; it < it_end && ok; ++it) {
+                const GroupItem item = p.items[it];
+                const int32_t* list = p.lists + item.list_off;
+                const PairDev first = p.pairs[list[0]];
+                TileIter ti;
+                ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+                if (!ti.valid()) continue;
+                ok = wait(B_QEMPTY, items ^ 1u);
+                if (!ok) break;
+                ++items;
+                mbar_arrive_expect_tx(bar(B_QFULL), 5 * kBox128);
+                for (int c = 0; c < 3; ++c)
+                    tma_load_3d(smem + kQ + c * kBox128, &map_q, bar(B_QFULL), c * 64, item.head,
+                                first.q_tok0 + item.r0);
+                for (int c = 0; c < 2; ++c)
+                    tma_load_3d(smem + kDO + c * kBox128, &map_do, bar(B_QFULL), c * 64, item.head,
+                                first.q_tok0 + item.r0);
+                for (; ti.valid() && ok; ti.next()) {
+                    const int tok = ti.cur.k_tok0 + ti.t * TILE;
+                    const int st = gk % kKStages;
+                    ok = wait(B_KEMPTY + st, (gk / kKStages) ^ 1u);
+                    if (!ok) break;
+                    ++gk;
+                    mbar_arrive_expect_tx(bar(B_KFULL + st), 3 * kBox128);
+                    for (int c = 0; c < 3; ++c)
+                        tma_load_3d(smem + kK + st * 3 * kBox128 + c * kBox128, &map_k, bar(B_KFULL + st),
+                                    c * 64, item.head, tok);
+                    for (int c = 0; c < 2 && ok; ++c, ++gv) {
+                        const int slot = gv % kVSlots;
+                        ok = wait(B_VEMPTY + slot, (gv / kVSlots) ^ 1u);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(bar(B_VFULL + slot), kBox128);
+                        tma_load_3d(smem + kV + slot * kBox128, &map_v, bar(B_VFULL + slot), c * 64, item.head, tok);
+                    }
                 }
             }
-        };
-        auto load_k = [&](const PairDev& pr, int tile, int st) {
-            mbar_arrive_expect_tx(bar_k0 + 8 * st, 3 * kBox128);
-            for (int c = 0; c < 3; ++c)
-                tma_load_3d(smem + kK + st * 3 * kBox128 + c * kBox128, &map_k, bar_k0 + 8 * st,
-                            c * 64, head, pr.k_tok0 + tile * TILE);
-        };
-        auto load_v = [&](const PairDev& pr, int tile) {
-            mbar_arrive_expect_tx(bar_v, 2 * kBox128);
-            for (int c = 0; c < 2; ++c)
-                tma_load_3d(smem + kV + c * kBox128, &map_v, bar_v, c * 64, head,
-                            pr.k_tok0 + tile * TILE);
-        };
-
-        const bool any = li < item.list_len;
-        float lse2 = 0.f, dsum = 0.f;
-        if (row_valid) {
-            const float l = p.lse[static_cast<int64_t>(head) * p.T + first.q_tok0 + row];
-            lse2 = (l == neg_inf()) ? pos_inf() : l * 1.4426950408889634f;
-            dsum = p.dsum[static_cast<int64_t>(head) * p.T + first.q_tok0 + row];
         }
-        if (tid == 0 && any) {
-            mbar_arrive_expect_tx(bar_q, 5 * kBox128);
-            for (int c = 0; c < 3; ++c)
-                tma_load_3d(smem + kQ + c * kBox128, &map_q, bar_q, c * 64, head, first.q_tok0 + r0);
-            for (int c = 0; c < 2; ++c)
-                tma_load_3d(smem + kDO + c * kBox128, &map_do, bar_q, c * 64, head, first.q_tok0 + r0);
-            load_k(cur, 0, 0);
-            load_v(cur, 0);
-        }
+    } else if (warp == kWarpMma) {
+        // ------------------------------------------------------------------ UMMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = umma_idesc_bf16(TILE, TILE, false, false);
+            constexpr uint32_t idesc_dq = umma_idesc_bf16(TILE, D_QK, false, true);
+            constexpr uint32_t hi_kmaj = umma_desc_hi(16, 1024);
+            constexpr uint32_t hi_kmn = umma_desc_hi(kBox128, 1024);       // K as MN-major B, N = 192
+            const uint32_t q_lo = umma_desc_lo(smem + kQ, 16), do_lo = umma_desc_lo(smem + kDO, 16);
+            const uint32_t k_lo0 = umma_desc_lo(smem + kK, 16), v_lo0 = umma_desc_lo(smem + kV, 16);
+            const uint32_t kmn_lo0 = umma_desc_lo(smem + kK, kBox128);
+            uint32_t items = 0, c_s = 0, c_p = 0, gk_s = 0, gv = 0, gk_q = 0;
+            bool ok = true;
+            for (int it = it_begin; it < it_end && ok; ++it) {
+                const GroupItem item = p.items[it];
+                const int32_t* list = p.lists + item.list_off;
+                const PairDev first = p.pairs[list[0]];
+                TileIter ti;
+                ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+                if (!ti.valid()) continue;
+                int n_tiles = 0;
+                for (TileIter c = ti; c.valid(); c.next()) ++n_tiles;
 
-        int step = 0;
-        while (li < item.list_len && ok) {
-            const int st = step & 1;
-            advance_next();
-            const bool has_next = nli < item.list_len;
-            if (tid == 0) {
-                if (has_next) load_k(nxt, ntile, st ^ 1);
-                if (step == 0) ok = mbar_wait(bar_q, ph_q, &abort_flag, limit);
-                if (ok) ok = mbar_wait(bar_k0 + 8 * st, ph_k[st], &abort_flag, limit);
-                if (ok) ok = mbar_wait(bar_v, ph_v, &abort_flag, limit);
-                if (ok) {
+                auto issue_s_dp = [&](bool last) {
+                    if (c_s > 0) ok = wait(B_SFREE, c_s - 1u);      // S / dP of the previous step are in registers
+                    if (!ok) return;
+                    const int st = gk_s % kKStages;
+                    ok = wait(B_KFULL + st, gk_s / kKStages);
+                    ++gk_s;
+                    if (!ok) return;
                     tc_fence_after_sync();
-                    const uint32_t qb = smem + kQ, kb = smem + kK + st * 3 * kBox128;
+                    const uint32_t k_lo = k_lo0 + st * (3 * kBox128 >> 4);
 #pragma unroll
                     for (int kk = 0; kk < D_QK / 16; ++kk) {
-                        const uint32_t o = (kk >> 2) * kBox128 + (kk & 3) * 32;
-                        umma_ss(tm + kTmS, umma_smem_desc_sw128(qb + o, 16, 1024),
-                                umma_smem_desc_sw128(kb + o, 16, 1024), idesc_s, kk > 0);
+                        const uint32_t o = (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2;
+                        umma_ss_w(tm + kTmS, q_lo + o, hi_kmaj, k_lo + o, hi_kmaj, idesc_s, kk > 0);
                     }
-                    const uint32_t gb = smem + kDO, vb = smem + kV;
 #pragma unroll
-                    for (int kk = 0; kk < D_V / 16; ++kk) {
-                        const uint32_t o = (kk >> 2) * kBox128 + (kk & 3) * 32;
-                        umma_ss(tm + kTmDP, umma_smem_desc_sw128(gb + o, 16, 1024),
-                                umma_smem_desc_sw128(vb + o, 16, 1024), idesc_s, kk > 0);
+                    for (int c = 0; c < 2; ++c, ++gv) {
+                        const int slot = gv % kVSlots;
+                        ok = wait(B_VFULL + slot, gv / kVSlots);
+                        if (!ok) return;
+                        tc_fence_after_sync();
+                        const uint32_t v_lo = v_lo0 + slot * (kBox128 >> 4);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            umma_ss_w(tm + kTmDP, do_lo + c * (kBox128 >> 4) + kk * 2, hi_kmaj, v_lo + kk * 2, hi_kmaj,
+                                      idesc_s, (c | kk) != 0);
+                        umma_commit(bar(B_VEMPTY + slot));
                     }
-                    umma_commit(bar_s);
-                }
-            }
-            ph_k[st] ^= 1; ph_v ^= 1;
-            __syncwarp();
-            ok = mbar_wait(bar_s, ph_s, &abort_flag, limit);
-            ph_s ^= 1;
-            if (!ok) break;
-            tc_fence_after_sync();
-            if (tid == 0 && has_next) load_v(nxt, ntile);      // V is single-buffered: dP has read it
+                    umma_commit(bar(B_SFULL));
+                    ++c_s;
+                    if (last) umma_commit(bar(B_QEMPTY));            // Q and dO are no longer read
+                };
+                auto issue_dq = [&](int j) {
+                    ok = wait(B_PFULL, c_p);
+                    ++c_p;
+                    if (!ok) return;
+                    if (j == 0 && items > 0) ok = wait(B_ACCFREE, items - 1u);
+                    if (!ok) return;
+                    tc_fence_after_sync();
+                    const int st = gk_q % kKStages;
+                    ++gk_q;
+                    const uint32_t k_lo = kmn_lo0 + st * (3 * kBox128 >> 4);
+#pragma unroll
+                    for (int kk = 0; kk < TILE / 16; ++kk)
+                        umma_ts_w(tm + kTmDQ, tm + kTmDS + kk * 8, k_lo + kk * (2048 >> 4), hi_kmn, idesc_dq,
+                                  (j | kk) != 0);
+                    umma_commit(bar(B_DSFREE));
+                    umma_commit(bar(B_KEMPTY + st));
+                };
 
-            // ---- P and dS on this thread's row -----------------------------------------------
-            const int col0 = t * TILE;
-            int jmax = cur.k_len - 1;
-            if (p.causal) jmax = min(jmax, row + cur.off);
-            const int cmax = jmax - col0;
+                ok = wait(B_QFULL, items);
+                if (!ok) break;
+                issue_s_dp(n_tiles == 1);
+                for (int j = 0; j < n_tiles && ok; ++j) {
+                    if (j + 1 < n_tiles) issue_s_dp(j + 2 == n_tiles);
+                    if (ok) issue_dq(j);
+                }
+                ++items;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ elementwise warpgroups
+        const int g = warp >> 2;                       // column half
+        const int r = tid & 127;
+        const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tm_s = tm + kTmS + lane_base + g * 64;
+        const uint32_t tm_dp = tm + kTmDP + lane_base + g * 64;
+        const uint32_t tm_ds = tm + kTmDS + lane_base + g * 32;
+        uint32_t c_s = 0, c_ds = 0;
+        bool ok = true;
+        for (int it = it_begin; it < it_end && ok; ++it) {
+            const GroupItem item = p.items[it];
+            const int32_t* list = p.lists + item.list_off;
+            const PairDev first = p.pairs[list[0]];
+            const int row = item.r0 + r;
+            const bool row_valid = row < first.q_len;
+            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.dq) +
+                                 (static_cast<int64_t>(first.q_tok0 + row) * p.h + item.head) * D_QK + g * 96;
+            TileIter ti;
+            ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+            if (!ti.valid()) {                         // no visible key at all: dQ = 0
+                if (row_valid) {
+                    uint4* d4 = reinterpret_cast<uint4*>(dst);
 #pragma unroll
-            for (int c0 = 0; c0 < TILE; c0 += 32) {
-                uint32_t s[32], dp[32], ds[16];
-                tmem_ld_x32(tm + kTmS + lane_base + c0, s);
-                tmem_ld_x32(tm + kTmDP + lane_base + c0, dp);
+                    for (int e = 0; e < 12; ++e) d4[e] = make_uint4(0u, 0u, 0u, 0u);
+                }
+                continue;
+            }
+            float lse2 = 0.f, dsum = 0.f;
+            if (row_valid) {
+                const float l = p.lse[static_cast<int64_t>(item.head) * p.T + first.q_tok0 + row];
+                lse2 = (l == neg_inf()) ? pos_inf() : l * kLog2e;
+                dsum = p.dsum[static_cast<int64_t>(item.head) * p.T + first.q_tok0 + row];
+            }
+            for (; ti.valid() && ok; ti.next()) {
+                ok = wait(B_SFULL, c_s);
+                ++c_s;
+                if (!ok) break;
+                tc_fence_after_sync();
+                uint32_t s[64], dp[64];
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    tmem_ld_x32(tm_s + c0, s + c0);
+                    tmem_ld_x32(tm_dp + c0, dp + c0);
+                }
                 tmem_wait_ld();
+                tc_fence_before_sync();
+                mbar_arrive(bar(B_SFREE));             // the next S / dP may overwrite tensor memory
+                int jmax = ti.cur.k_len - 1;
+                if (p.causal) jmax = min(jmax, row + ti.cur.off);
+                const int cmax = jmax - ti.t * TILE - g * 64;      // columns 0..cmax of this half are visible
+                uint32_t ds[32];
 #pragma unroll
-                for (int c = 0; c < 32; c += 2) {
+                for (int c = 0; c < 64; c += 2) {
                     float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2));
                     float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2));
-                    if (c0 + c > cmax) p0 = 0.f;
-                    if (c0 + c + 1 > cmax) p1 = 0.f;
+                    if (c > cmax) p0 = 0.f;
+                    if (c + 1 > cmax) p1 = 0.f;
                     ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum),
                                              p1 * (__uint_as_float(dp[c + 1]) - dsum));
                 }
-                tmem_st_x16(tm + kTmDS + lane_base + (c0 >> 1), ds);
+                if (c_ds > 0) {                        // the previous dQ update has read dS
+                    ok = wait(B_DSFREE, c_ds - 1u);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                }
+                tmem_st_x32(tm_ds, ds);
+                tmem_wait_st();
+                tc_fence_before_sync();
+                mbar_arrive(bar(B_PFULL));
+                ++c_ds;
             }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncthreads();
-
-            if (tid == 0) {
-                tc_fence_after_sync();
-                const uint32_t kb = smem + kK + st * 3 * kBox128;
-#pragma unroll
-                for (int kk = 0; kk < TILE / 16; ++kk)
-                    umma_ts(tm + kTmDQ, tm + kTmDS + kk * 8,
-                            umma_smem_desc_sw128(kb + kk * 2048, kBox128, 1024), idesc_dq,
-                            (step > 0) || (kk > 0));
-                umma_commit(bar_acc);
-            }
-            __syncwarp();
-            ok = mbar_wait(bar_acc, ph_acc, &abort_flag, limit);
-            ph_acc ^= 1;
+            if (!ok) break;
+            // ---- epilogue: dQ * scale -> bf16; this warpgroup writes 96 of the 192 columns ---------
+            ok = wait(B_DSFREE, c_ds - 1u);
             if (!ok) break;
             tc_fence_after_sync();
-
-            // advance the current iterator to where the lookahead already is
-            ++step;
-            li = nli; t = ntile; cur = nxt; nt = nnt;
-        }
-        if (any) ph_q ^= 1;
-        if (!ok) break;
-
-        // ---- epilogue: dQ * scale -> bf16 -----------------------------------------------------
-        {
-            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.dq) +
-                                 (static_cast<int64_t>(first.q_tok0 + row) * p.h + head) * D_QK;
 #pragma unroll
-            for (int c = 0; c < D_QK; c += 32) {
+            for (int c0 = 0; c0 < 96; c0 += 32) {
                 uint32_t v[32];
-                if (any) {
-                    tmem_ld_x32(tm + kTmDQ + lane_base + c, v);
-                    tmem_wait_ld();
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = 0u;
+                tmem_ld_x32(tm + kTmDQ + lane_base + g * 96 + c0, v);
+                tmem_wait_ld();
+                if (c0 == 64) {
+                    tc_fence_before_sync();
+                    mbar_arrive(bar(B_ACCFREE));
                 }
-                if (row_valid) store_row_bf16(dst + c, v, 32, p.scale);
+                if (row_valid) store_row_bf16(dst + c0, v, 32, p.scale);
             }
-            tc_fence_before_sync();
-            __syncthreads();
-            tc_fence_after_sync();
         }
     }
 
-    if (!ok || abort_flag) {
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (abort_flag) {
         const uint64_t t0 = global_timer_ns();
         while (global_timer_ns() - t0 < 50000ull) { }
         if (tid == 0) {
             p.status->detail = blockIdx.x;
             p.status->status = HYDRA_ERR_DEVICE_TIMEOUT;
         }
+        __syncthreads();
     }
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tm, kTmCols);
+    if (warp == kWarpMma) tmem_dealloc(tm, kTmCols);
 }
 
+// =============================================================================================
+// dK / dV
+// =============================================================================================
 __global__ void __launch_bounds__(kThreads, 1)
 hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
@@ -308,253 +410,281 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     using namespace dkv;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    __shared__ __align__(8) uint64_t bars[8];
+    __shared__ __align__(8) uint64_t bars[B_COUNT];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
-    __shared__ float s_lse2[2][SUB];
-    __shared__ float s_dsum[2][SUB];
+    __shared__ float s_lse2[kStages][SUB];
+    __shared__ float s_dsum[kStages][SUB];
 
-    const int tid = threadIdx.x, warp = tid >> 5;
-    const uint32_t bar_kv = smem_u32(&bars[0]);     // K and V tile of the item
-    const uint32_t bar_q0 = smem_u32(&bars[1]);     // + 8 * stage: Q and dO sub-tile
-    const uint32_t bar_s = smem_u32(&bars[3]);      // S^T and dP^T complete
-    const uint32_t bar_acc = smem_u32(&bars[4]);    // dV, dK updates complete
-
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t bar0 = smem_u32(&bars[0]);
+    auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
     if (tid == 0) {
         abort_flag = 0;
-        mbar_init(bar_kv, 1); mbar_init(bar_q0, 1); mbar_init(bar_q0 + 8, 1);
-        mbar_init(bar_s, 1); mbar_init(bar_acc, 1);
+        for (int i = 0; i < B_COUNT; ++i) {
+            uint32_t count = 1u;
+            if (i == B_SFREE || i == B_PFULL || i == B_ACCFREE) count = 256u;
+            if (i >= B_STAT && i < B_STAT + kStages) count = 32u;
+            mbar_init(bar(i), count);
+        }
         fence_mbar_init();
         tma_prefetch_desc(&map_q); tma_prefetch_desc(&map_k);
         tma_prefetch_desc(&map_v); tma_prefetch_desc(&map_do);
     }
-    if (warp == 0) { tmem_alloc(smem_u32(&tmem_base_slot), kTmCols); tmem_relinquish(); }
+    if (warp == kWarpMma) { tmem_alloc(smem_u32(&tmem_base_slot), kTmCols); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tm = tmem_base_slot;
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
     const uint64_t limit = p.wait_limit_ns;
+    const int it_begin = p.cta_off[blockIdx.x], it_end = p.cta_off[blockIdx.x + 1];
+    volatile int* abort_p = &abort_flag;
+    auto wait = [&](int b, uint32_t parity) -> bool { return mbar_wait(bar(b), parity & 1u, abort_p, limit); };
 
-    constexpr uint32_t idesc_st = umma_idesc_bf16(TILE, SUB, false, false);
-    constexpr uint32_t idesc_dv = umma_idesc_bf16(TILE, D_V, false, true);
-    constexpr uint32_t idesc_dk = umma_idesc_bf16(TILE, D_QK, false, true);
-
-    uint32_t ph_kv = 0, ph_q[2] = {0, 0}, ph_s = 0, ph_acc = 0;
-    bool ok = true;
-
-    for (int it = blockIdx.x; it < p.n_items && ok; it += gridDim.x) {
-        const GroupItem item = p.items[it];
-        const int head = item.head, r0 = item.r0;
-        const int32_t* list = p.lists + item.list_off;
-        const PairDev first = p.pairs[list[0]];
-        const int krow = r0 + tid;                       // kv row inside the chunk
-        const bool row_valid = krow < first.k_len;
-
-        auto first_sub = [&](const PairDev& pr) -> int {
-            if (!p.causal) return 0;
-            const int i_min = r0 - pr.off;               // first q row that sees kv row r0
-            return i_min > 0 ? i_min / SUB : 0;
-        };
-        auto n_sub = [&](const PairDev& pr) -> int { return (pr.q_len + SUB - 1) / SUB; };
-
-        int li = 0, u = 0, nu = 0;
-        PairDev cur = first;
-        while (li < item.list_len) {
-            cur = p.pairs[list[li]];
-            u = first_sub(cur); nu = n_sub(cur);
-            if (u < nu) break;
-            ++li;
-        }
-        int nli = li, nsub = u, nnu = nu;
-        PairDev nxt = cur;
-        auto advance_next = [&]() {
-            ++nsub;
-            if (nsub >= nnu) {
-                ++nli;
-                while (nli < item.list_len) {
-                    nxt = p.pairs[list[nli]];
-                    nsub = first_sub(nxt); nnu = n_sub(nxt);
-                    if (nsub < nnu) break;
-                    ++nli;
-                }
-            }
-        };
-        auto load_q = [&](const PairDev& pr, int sub, int st) {
-            mbar_arrive_expect_tx(bar_q0 + 8 * st, 5 * kBox64);
-            const int tok = pr.q_tok0 + sub * SUB;
-            for (int c = 0; c < 3; ++c)
-                tma_load_3d(smem + kQ + st * 3 * kBox64 + c * kBox64, &map_q, bar_q0 + 8 * st, c * 64,
-                            head, tok);
-            for (int c = 0; c < 2; ++c)
-                tma_load_3d(smem + kDO + st * 2 * kBox64 + c * kBox64, &map_do, bar_q0 + 8 * st,
-                            c * 64, head, tok);
-        };
-        auto load_stats = [&](const PairDev& pr, int sub, int st) {
-            const int i = sub * SUB + (tid & (SUB - 1));
-            const bool v = i < pr.q_len;
-            const int64_t idx = static_cast<int64_t>(head) * p.T + pr.q_tok0 + i;
-            if (tid < SUB) {
-                const float l = v ? p.lse[idx] : neg_inf();
-                s_lse2[st][tid] = (l == neg_inf()) ? pos_inf() : l * 1.4426950408889634f;
-            } else {
-                s_dsum[st][tid - SUB] = v ? p.dsum[idx] : 0.f;
-            }
-        };
-
-        const bool any = li < item.list_len;
-        if (any) {
-            if (tid == 0) {
-                mbar_arrive_expect_tx(bar_kv, 5 * kBox128);
+    if (warp == kWarpProd) {
+        // ------------------------------------------------------------------ TMA producer + LSE / D
+        uint32_t items = 0, gq = 0;
+        bool ok = true;
+        for (int it = it_begin; it < it_end && ok; ++it) {
+            const GroupItem item = p.items[it];
+            const int32_t* list = p.lists + item.list_off;
+            const PairDev first = p.pairs[list[0]];
+            SubIter si;
+            si.init(p.pairs, list, item.list_len, item.r0, p.causal);
+            if (!si.valid()) continue;
+            ok = wait(B_KVEMPTY, items ^ 1u);
+            if (!ok) break;
+            ++items;
+            if (lane == 0) {
+                mbar_arrive_expect_tx(bar(B_KVFULL), 5 * kBox128);
                 for (int c = 0; c < 3; ++c)
-                    tma_load_3d(smem + kK + c * kBox128, &map_k, bar_kv, c * 64, head, first.k_tok0 + r0);
+                    tma_load_3d(smem + kK + c * kBox128, &map_k, bar(B_KVFULL), c * 64, item.head,
+                                first.k_tok0 + item.r0);
                 for (int c = 0; c < 2; ++c)
-                    tma_load_3d(smem + kV + c * kBox128, &map_v, bar_kv, c * 64, head, first.k_tok0 + r0);
-                load_q(cur, u, 0);
+                    tma_load_3d(smem + kV + c * kBox128, &map_v, bar(B_KVFULL), c * 64, item.head,
+                                first.k_tok0 + item.r0);
             }
-            load_stats(cur, u, 0);
+            for (; si.valid() && ok; si.next(), ++gq) {
+                const int st = gq % kStages;
+                ok = wait(B_QEMPTY + st, (gq / kStages) ^ 1u);
+                if (!ok) break;
+                const int tok = si.cur.q_tok0 + si.u * SUB;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(bar(B_QFULL + st), 5 * kBox64);
+                    for (int c = 0; c < 3; ++c)
+                        tma_load_3d(smem + kQ + st * 3 * kBox64 + c * kBox64, &map_q, bar(B_QFULL + st), c * 64,
+                                    item.head, tok);
+                    for (int c = 0; c < 2; ++c)
+                        tma_load_3d(smem + kDO + st * 2 * kBox64 + c * kBox64, &map_do, bar(B_QFULL + st), c * 64,
+                                    item.head, tok);
+                }
+                // LSE (as log2) and D of the 64 q rows, two rows per lane
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int c = lane + 32 * e;
+                    const int i = si.u * SUB + c;
+                    const bool v = i < si.cur.q_len;
+                    const int64_t idx = static_cast<int64_t>(item.head) * p.T + si.cur.q_tok0 + i;
+                    const float l = v ? __ldg(p.lse + idx) : neg_inf();
+                    s_lse2[st][c] = (l == neg_inf()) ? pos_inf() : l * kLog2e;
+                    s_dsum[st][c] = v ? __ldg(p.dsum + idx) : 0.f;
+                }
+                mbar_arrive(bar(B_STAT + st));
+            }
         }
-        __syncthreads();
+    } else if (warp == kWarpMma) {
+        // ------------------------------------------------------------------ UMMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_st = umma_idesc_bf16(TILE, SUB, false, false);
+            constexpr uint32_t idesc_dv = umma_idesc_bf16(TILE, D_V, false, true);
+            constexpr uint32_t idesc_dk = umma_idesc_bf16(TILE, D_QK, false, true);
+            constexpr uint32_t hi_kmaj = umma_desc_hi(16, 1024);
+            constexpr uint32_t hi_mn = umma_desc_hi(kBox64, 1024);         // Q / dO sub-tiles as MN-major B
+            const uint32_t k_lo = umma_desc_lo(smem + kK, 16), v_lo = umma_desc_lo(smem + kV, 16);
+            const uint32_t q_lo0 = umma_desc_lo(smem + kQ, 16), do_lo0 = umma_desc_lo(smem + kDO, 16);
+            const uint32_t qmn_lo0 = umma_desc_lo(smem + kQ, kBox64), domn_lo0 = umma_desc_lo(smem + kDO, kBox64);
+            uint32_t items = 0, c_s = 0, c_p = 0, gq_s = 0, gq_a = 0;
+            bool ok = true;
+            for (int it = it_begin; it < it_end && ok; ++it) {
+                const GroupItem item = p.items[it];
+                const int32_t* list = p.lists + item.list_off;
+                SubIter si;
+                si.init(p.pairs, list, item.list_len, item.r0, p.causal);
+                if (!si.valid()) continue;
+                int n_steps = 0;
+                for (SubIter c = si; c.valid(); c.next()) ++n_steps;
 
-        int step = 0;
-        while (li < item.list_len && ok) {
-            const int st = step & 1;
-            advance_next();
-            const bool has_next = nli < item.list_len;
-            if (has_next) load_stats(nxt, nsub, st ^ 1);   // read after this step's __syncthreads
-            if (tid == 0) {
-                if (has_next) load_q(nxt, nsub, st ^ 1);
-                if (step == 0) ok = mbar_wait(bar_kv, ph_kv, &abort_flag, limit);
-                if (ok) ok = mbar_wait(bar_q0 + 8 * st, ph_q[st], &abort_flag, limit);
-                if (ok) {
+                auto issue_s_dp = [&](bool last) {
+                    if (c_s > 0) ok = wait(B_SFREE, c_s - 1u);
+                    if (!ok) return;
+                    const int st = gq_s % kStages;
+                    ok = wait(B_QFULL + st, gq_s / kStages);
+                    ++gq_s;
+                    if (!ok) return;
                     tc_fence_after_sync();
-                    const uint32_t kb = smem + kK, qb = smem + kQ + st * 3 * kBox64;
+                    const uint32_t q_lo = q_lo0 + st * (3 * kBox64 >> 4), do_lo = do_lo0 + st * (2 * kBox64 >> 4);
 #pragma unroll
                     for (int kk = 0; kk < D_QK / 16; ++kk)
-                        umma_ss(tm + kTmS,
-                                umma_smem_desc_sw128(kb + (kk >> 2) * kBox128 + (kk & 3) * 32, 16, 1024),
-                                umma_smem_desc_sw128(qb + (kk >> 2) * kBox64 + (kk & 3) * 32, 16, 1024),
-                                idesc_st, kk > 0);
-                    const uint32_t vb = smem + kV, gb = smem + kDO + st * 2 * kBox64;
+                        umma_ss_w(tm + kTmS, k_lo + (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2, hi_kmaj,
+                                  q_lo + (kk >> 2) * (kBox64 >> 4) + (kk & 3) * 2, hi_kmaj, idesc_st, kk > 0);
 #pragma unroll
                     for (int kk = 0; kk < D_V / 16; ++kk)
-                        umma_ss(tm + kTmDP,
-                                umma_smem_desc_sw128(vb + (kk >> 2) * kBox128 + (kk & 3) * 32, 16, 1024),
-                                umma_smem_desc_sw128(gb + (kk >> 2) * kBox64 + (kk & 3) * 32, 16, 1024),
-                                idesc_st, kk > 0);
-                    umma_commit(bar_s);
-                }
-            }
-            ph_q[st] ^= 1;
-            __syncwarp();
-            ok = mbar_wait(bar_s, ph_s, &abort_flag, limit);
-            ph_s ^= 1;
-            if (!ok) break;
-            tc_fence_after_sync();
-
-            // ---- P^T and dS^T on this thread's kv row -----------------------------------------
-            // q row i = u*64 + c is visible from kv row krow iff i < q_len and krow <= i + off.
-            int c_lo = 0;                                   // first visible column
-            if (p.causal) c_lo = max(0, krow - cur.off - u * SUB);
-            int c_hi = min(SUB, cur.q_len - u * SUB);       // one past the last valid column
-            if (!row_valid) c_hi = 0;
+                        umma_ss_w(tm + kTmDP, v_lo + (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2, hi_kmaj,
+                                  do_lo + (kk >> 2) * (kBox64 >> 4) + (kk & 3) * 2, hi_kmaj, idesc_st, kk > 0);
+                    umma_commit(bar(B_SFULL));
+                    ++c_s;
+                    if (last) umma_commit(bar(B_KVEMPTY));           // K and V are no longer read
+                };
+                auto issue_acc = [&](int i) {
+                    ok = wait(B_PFULL, c_p);
+                    ++c_p;
+                    if (!ok) return;
+                    if (i == 0 && items > 0) ok = wait(B_ACCFREE, items - 1u);
+                    if (!ok) return;
+                    tc_fence_after_sync();
+                    const int st = gq_a % kStages;
+                    ++gq_a;
+                    const uint32_t do_lo = domn_lo0 + st * (2 * kBox64 >> 4), q_lo = qmn_lo0 + st * (3 * kBox64 >> 4);
 #pragma unroll
-            for (int c0 = 0; c0 < SUB; c0 += 32) {
-                uint32_t s[32], dp[32], pk[16], ds[16];
-                tmem_ld_x32(tm + kTmS + lane_base + c0, s);
-                tmem_ld_x32(tm + kTmDP + lane_base + c0, dp);
+                    for (int kk = 0; kk < SUB / 16; ++kk)
+                        umma_ts_w(tm + kTmDV, tm + kTmP + kk * 8, do_lo + kk * (2048 >> 4), hi_mn, idesc_dv,
+                                  (i | kk) != 0);
+#pragma unroll
+                    for (int kk = 0; kk < SUB / 16; ++kk)
+                        umma_ts_w(tm + kTmDK, tm + kTmDS + kk * 8, q_lo + kk * (2048 >> 4), hi_mn, idesc_dk,
+                                  (i | kk) != 0);
+                    umma_commit(bar(B_PDSFREE));
+                    umma_commit(bar(B_QEMPTY + st));
+                };
+
+                ok = wait(B_KVFULL, items);
+                if (!ok) break;
+                issue_s_dp(n_steps == 1);
+                for (int i = 0; i < n_steps && ok; ++i) {
+                    if (i + 1 < n_steps) issue_s_dp(i + 2 == n_steps);
+                    if (ok) issue_acc(i);
+                }
+                ++items;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ elementwise warpgroups
+        const int g = warp >> 2;                       // column half: q rows [32 g, 32 g + 32) of the sub-tile
+        const int r = tid & 127;
+        const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tm_s = tm + kTmS + lane_base + g * 32;
+        const uint32_t tm_dp = tm + kTmDP + lane_base + g * 32;
+        const uint32_t tm_p = tm + kTmP + lane_base + g * 16;
+        const uint32_t tm_ds = tm + kTmDS + lane_base + g * 16;
+        uint32_t c_s = 0, c_pds = 0, gq = 0;
+        bool ok = true;
+        for (int it = it_begin; it < it_end && ok; ++it) {
+            const GroupItem item = p.items[it];
+            const int32_t* list = p.lists + item.list_off;
+            const PairDev first = p.pairs[list[0]];
+            const int krow = item.r0 + r;              // kv row inside the chunk
+            const bool row_valid = krow < first.k_len;
+            const int64_t tok = static_cast<int64_t>(first.k_tok0) + krow;
+            __nv_bfloat16* dkp = static_cast<__nv_bfloat16*>(p.dk) + (tok * p.h + item.head) * D_QK + g * 96;
+            __nv_bfloat16* dvp = static_cast<__nv_bfloat16*>(p.dv) + (tok * p.h + item.head) * D_V + g * 64;
+            SubIter si;
+            si.init(p.pairs, list, item.list_len, item.r0, p.causal);
+            if (!si.valid()) {                         // no q row sees this tile: dK = dV = 0
+                if (row_valid) {
+                    uint4* a4 = reinterpret_cast<uint4*>(dkp);
+                    uint4* b4 = reinterpret_cast<uint4*>(dvp);
+#pragma unroll
+                    for (int e = 0; e < 12; ++e) a4[e] = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) b4[e] = make_uint4(0u, 0u, 0u, 0u);
+                }
+                continue;
+            }
+            for (; si.valid() && ok; si.next(), ++gq) {
+                const int st = gq % kStages;
+                ok = wait(B_SFULL, c_s);
+                ++c_s;
+                if (!ok) break;
+                tc_fence_after_sync();
+                uint32_t s[32], dp[32];
+                tmem_ld_x32(tm_s, s);
+                tmem_ld_x32(tm_dp, dp);
                 tmem_wait_ld();
+                tc_fence_before_sync();
+                mbar_arrive(bar(B_SFREE));
+                ok = wait(B_STAT + st, gq / kStages);
+                if (!ok) break;
+                // q row i = u*64 + 32 g + c is visible from kv row krow iff i < q_len and krow <= i + off
+                const int base = si.u * SUB + g * 32;
+                int c_lo = 0;
+                if (p.causal) c_lo = max(0, krow - si.cur.off - base);
+                int c_hi = min(32, si.cur.q_len - base);
+                if (!row_valid) c_hi = 0;
+                const float* lse2 = &s_lse2[st][g * 32];
+                const float* dsum = &s_dsum[st][g * 32];
+                uint32_t pk[16], ds[16];
 #pragma unroll
                 for (int c = 0; c < 32; c += 2) {
-                    const int ca = c0 + c, cb = c0 + c + 1;
-                    float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -s_lse2[st][ca]));
-                    float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -s_lse2[st][cb]));
-                    if (ca < c_lo || ca >= c_hi) p0 = 0.f;
-                    if (cb < c_lo || cb >= c_hi) p1 = 0.f;
+                    float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2[c]));
+                    float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2[c + 1]));
+                    if (c < c_lo || c >= c_hi) p0 = 0.f;
+                    if (c + 1 < c_lo || c + 1 >= c_hi) p1 = 0.f;
                     pk[c >> 1] = pack_bf16x2(p0, p1);
-                    ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - s_dsum[st][ca]),
-                                             p1 * (__uint_as_float(dp[c + 1]) - s_dsum[st][cb]));
+                    ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum[c]),
+                                             p1 * (__uint_as_float(dp[c + 1]) - dsum[c + 1]));
                 }
-                tmem_st_x16(tm + kTmP + lane_base + (c0 >> 1), pk);
-                tmem_st_x16(tm + kTmDS + lane_base + (c0 >> 1), ds);
+                if (c_pds > 0) {                       // the previous dV / dK updates have read P and dS
+                    ok = wait(B_PDSFREE, c_pds - 1u);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                }
+                tmem_st_x16(tm_p, pk);
+                tmem_st_x16(tm_ds, ds);
+                tmem_wait_st();
+                tc_fence_before_sync();
+                mbar_arrive(bar(B_PFULL));
+                ++c_pds;
             }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncthreads();
-
-            if (tid == 0) {
-                tc_fence_after_sync();
-                const uint32_t gb = smem + kDO + st * 2 * kBox64, qb = smem + kQ + st * 3 * kBox64;
-#pragma unroll
-                for (int kk = 0; kk < SUB / 16; ++kk)
-                    umma_ts(tm + kTmDV, tm + kTmP + kk * 8,
-                            umma_smem_desc_sw128(gb + kk * 2048, kBox64, 1024), idesc_dv,
-                            (step > 0) || (kk > 0));
-#pragma unroll
-                for (int kk = 0; kk < SUB / 16; ++kk)
-                    umma_ts(tm + kTmDK, tm + kTmDS + kk * 8,
-                            umma_smem_desc_sw128(qb + kk * 2048, kBox64, 1024), idesc_dk,
-                            (step > 0) || (kk > 0));
-                umma_commit(bar_acc);
-            }
-            __syncwarp();
-            ok = mbar_wait(bar_acc, ph_acc, &abort_flag, limit);
-            ph_acc ^= 1;
+            if (!ok) break;
+            // ---- epilogue: dK * scale, dV -> bf16; each warpgroup writes half of the columns -------
+            ok = wait(B_PDSFREE, c_pds - 1u);
             if (!ok) break;
             tc_fence_after_sync();
-
-            ++step;
-            li = nli; u = nsub; cur = nxt; nu = nnu;
-        }
-        if (any) ph_kv ^= 1;
-        if (!ok) break;
-
-        // ---- epilogue: dK * scale, dV -> bf16 ---------------------------------------------------
-        {
-            const int64_t tok = static_cast<int64_t>(first.k_tok0) + krow;
-            __nv_bfloat16* dkp = static_cast<__nv_bfloat16*>(p.dk) + (tok * p.h + head) * D_QK;
-            __nv_bfloat16* dvp = static_cast<__nv_bfloat16*>(p.dv) + (tok * p.h + head) * D_V;
 #pragma unroll
-            for (int c = 0; c < D_QK; c += 32) {
+            for (int c0 = 0; c0 < 96; c0 += 32) {
                 uint32_t v[32];
-                if (any) {
-                    tmem_ld_x32(tm + kTmDK + lane_base + c, v);
-                    tmem_wait_ld();
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = 0u;
-                }
-                if (row_valid) store_row_bf16(dkp + c, v, 32, p.scale);
+                tmem_ld_x32(tm + kTmDK + lane_base + g * 96 + c0, v);
+                tmem_wait_ld();
+                if (row_valid) store_row_bf16(dkp + c0, v, 32, p.scale);
             }
 #pragma unroll
-            for (int c = 0; c < D_V; c += 32) {
+            for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
-                if (any) {
-                    tmem_ld_x32(tm + kTmDV + lane_base + c, v);
-                    tmem_wait_ld();
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = 0u;
+                tmem_ld_x32(tm + kTmDV + lane_base + g * 64 + c0, v);
+                tmem_wait_ld();
+                if (c0 == 32) {
+                    tc_fence_before_sync();
+                    mbar_arrive(bar(B_ACCFREE));
                 }
-                if (row_valid) store_row_bf16(dvp + c, v, 32, 1.f);
+                if (row_valid) store_row_bf16(dvp + c0, v, 32, 1.f);
             }
-            tc_fence_before_sync();
-            __syncthreads();
-            tc_fence_after_sync();
         }
     }
 
-    if (!ok || abort_flag) {
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (abort_flag) {
         const uint64_t t0 = global_timer_ns();
         while (global_timer_ns() - t0 < 50000ull) { }
         if (tid == 0) {
             p.status->detail = blockIdx.x;
             p.status->status = HYDRA_ERR_DEVICE_TIMEOUT;
         }
+        __syncthreads();
     }
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tm, kTmCols);
+    if (warp == kWarpMma) tmem_dealloc(tm, kTmCols);
 }
 
 cudaError_t launch_bwd_dq(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,

@@ -1,11 +1,23 @@
-// Forward attention of (q-chunk, kv-chunk) pairs on sm_100a: TMA -> shared memory -> tcgen05 UMMA
-// with S and O accumulated in tensor memory, online softmax on thread-private rows.
+// Forward attention of (q-chunk, kv-chunk) pairs on sm_100a.
 //
-// One CTA walks a strided share of the work list; a work item is one 128-row q tile of one pair and
-// head. Per kv tile: S = Q K^T (SS UMMA, both operands K-major), softmax in the exp2 domain with
-// the running row maximum, P written back to tensor memory as packed bf16, O += P V (TS UMMA, V
-// read as an MN-major B operand straight from its token-major layout). Thread r of the CTA owns
-// row r of the tile = TMEM lane r, so row max and row sum need no cross-thread traffic.
+// One persistent CTA per SM walks a strided share of the work list. A work item is a 256-row slab of
+// q rows of one pair and head, handled as two 128-row tiles (A and B) that ping-pong on the tensor
+// core so that UMMAs of one tile overlap the softmax of the other, and so that every K/V tile pulled
+// from L2 feeds 256 q rows.
+//
+// Warp roles (352 threads):
+//   warps 0-3   softmax of tile A: thread r owns row r = TMEM lane r (no cross-thread reductions)
+//   warps 4-7   softmax of tile B
+//   warp  8     TMA producer of Q (per item) and K (ring of five [128 x 64] boxes)
+//   warp  9     TMA producer of V (ring of three [64 kv rows x 128] half tiles)
+//   warp 10     UMMA issuer (one thread) and owner of the TMEM allocation
+//
+// Tensor memory (512 columns): S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512); P (bf16 pairs)
+// is written over the first 64 columns of its S. Issue order per kv tile j:
+//   S_A(j) = Q_A K_j^T ; O_B += P_B(j-1) V_{j-1} ; S_B(j) = Q_B K_j^T ; O_A += P_A(j) V_j
+// UMMAs execute in issue order, so S_t(j+1) cannot overtake the PV that still reads P_t(j).
+// The softmax keeps a running maximum in the exp2 domain and rescales O only when the maximum grew
+// by more than 2^8 (the final LSE is exact whatever reference maximum was used).
 #include <cuda_bf16.h>
 
 #include "hydra_internal.h"
@@ -15,18 +27,23 @@ namespace hydra {
 
 namespace {
 
-constexpr int kThreads = 128;
-constexpr uint32_t kBoxBytes = TILE * 128;            // one [128 rows x 64 bf16] swizzled box
-constexpr uint32_t kQBytes = 3 * kBoxBytes;           // 128 x 192
-constexpr uint32_t kKBytes = 3 * kBoxBytes;
-constexpr uint32_t kVBytes = 2 * kBoxBytes;           // 128 x 128
-constexpr int kStages = 2;
+constexpr int kThreads = 352;
+constexpr int kWarpK = 8, kWarpV = 9, kWarpMma = 10;
+constexpr uint32_t kBox = 128 * 128;                  // [128 rows x 64 bf16] = 16 KB
+constexpr uint32_t kQTile = 3 * kBox;                 // 128 x 192
+constexpr int kKSlots = 5, kVSlots = 3;
 constexpr uint32_t kSmemQ = 0;
-constexpr uint32_t kSmemK = kSmemQ + kQBytes;
-constexpr uint32_t kSmemV = kSmemK + kStages * kKBytes;
-constexpr uint32_t kSmemTotal = kSmemV + kStages * kVBytes;   // 212,992 B
-// TMEM columns
-constexpr uint32_t kTmS = 0, kTmO = 128, kTmP = 256, kTmCols = 512;
+constexpr uint32_t kSmemK = kSmemQ + 2 * kQTile;
+constexpr uint32_t kSmemV = kSmemK + kKSlots * kBox;
+constexpr uint32_t kSmemTotal = kSmemV + kVSlots * kBox;      // 229,376 B
+constexpr uint32_t kTmS = 0, kTmO = 256, kTmCols = 512;
+constexpr float kRescaleThreshold = 8.f;              // log2 units
+
+// barrier indices
+enum : int {
+    B_QFULL = 0, B_QEMPTY = 2, B_KFULL = 4, B_KEMPTY = 9, B_VFULL = 14, B_VEMPTY = 17,
+    B_SFULL = 20, B_PFULL = 22, B_OFULL = 24, B_OFREE = 26, B_COUNT = 28
+};
 
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
 
@@ -40,188 +57,299 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    __shared__ __align__(8) uint64_t bars[8];
+    __shared__ __align__(8) uint64_t bars[B_COUNT];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
-    const int tid = threadIdx.x, warp = tid >> 5;
-    const uint32_t bar_q = smem_u32(&bars[0]);
-    const uint32_t bar_k0 = smem_u32(&bars[1]);   // + 8 * stage
-    const uint32_t bar_v0 = smem_u32(&bars[3]);   // + 8 * stage
-    const uint32_t bar_s = smem_u32(&bars[5]);
-    const uint32_t bar_o = smem_u32(&bars[6]);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t bar0 = smem_u32(&bars[0]);
+    auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
 
     if (tid == 0) {
         abort_flag = 0;
-        mbar_init(bar_q, 1);
-        mbar_init(bar_k0, 1); mbar_init(bar_k0 + 8, 1);
-        mbar_init(bar_v0, 1); mbar_init(bar_v0 + 8, 1);
-        mbar_init(bar_s, 1); mbar_init(bar_o, 1);
+        for (int i = 0; i < B_COUNT; ++i) {
+            const bool by_threads = (i >= B_PFULL && i < B_PFULL + 2) || (i >= B_OFREE && i < B_OFREE + 2);
+            mbar_init(bar(i), by_threads ? 128u : 1u);
+        }
         fence_mbar_init();
         tma_prefetch_desc(&map_q); tma_prefetch_desc(&map_k); tma_prefetch_desc(&map_v);
     }
-    if (warp == 0) { tmem_alloc(smem_u32(&tmem_base_slot), kTmCols); tmem_relinquish(); }
+    if (warp == kWarpMma) { tmem_alloc(smem_u32(&tmem_base_slot), kTmCols); tmem_relinquish(); }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tm = tmem_base_slot;
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
     const uint64_t limit = p.wait_limit_ns;
+    const int it_begin = p.cta_off[blockIdx.x], it_end = p.cta_off[blockIdx.x + 1];
+    volatile int* abort_p = &abort_flag;
+    auto wait = [&](int b, uint32_t parity) -> bool { return mbar_wait(bar(b), parity & 1u, abort_p, limit); };
 
-    constexpr uint32_t idesc_s = umma_idesc_bf16(TILE, TILE, false, false);
-    constexpr uint32_t idesc_o = umma_idesc_bf16(TILE, D_V, false, true);
-
-    uint32_t ph_q = 0, ph_k[2] = {0, 0}, ph_v[2] = {0, 0}, ph_s = 0, ph_o = 0;
-    bool ok = true;
-
-    for (int it = blockIdx.x; it < p.n_items && ok; it += gridDim.x) {
-        const FwdItem item = p.items[it];
-        const PairDev pr = p.pairs[item.pair];
-        const int head = item.head, q0 = item.q0, n_kv = item.n_kv;
-        const int row = q0 + tid;                       // q row inside the pair
-        const bool row_valid = row < pr.q_len;
-
-        auto load_kv = [&](int j, int st) {
-            const int tok = pr.k_tok0 + j * TILE;
-            mbar_arrive_expect_tx(bar_k0 + 8 * st, kKBytes);
-            for (int c = 0; c < 3; ++c)
-                tma_load_3d(smem + kSmemK + st * kKBytes + c * kBoxBytes, &map_k, bar_k0 + 8 * st,
-                            c * 64, head, tok);
-            mbar_arrive_expect_tx(bar_v0 + 8 * st, kVBytes);
-            for (int c = 0; c < 2; ++c)
-                tma_load_3d(smem + kSmemV + st * kVBytes + c * kBoxBytes, &map_v, bar_v0 + 8 * st,
-                            c * 64, head, tok);
-        };
-
-        if (tid == 0 && n_kv > 0) {
-            mbar_arrive_expect_tx(bar_q, kQBytes);
-            for (int c = 0; c < 3; ++c)
-                tma_load_3d(smem + kSmemQ + c * kBoxBytes, &map_q, bar_q, c * 64, head,
-                            pr.q_tok0 + q0);
-            load_kv(0, 0);
-        }
-
-        float m_run = neg_inf(), l_run = 0.f;
-
-        for (int j = 0; j < n_kv && ok; ++j) {
-            const int st = j & 1;
-            if (tid == 0) {
-                if (j + 1 < n_kv) load_kv(j + 1, st ^ 1);
-                if (j == 0) ok = mbar_wait(bar_q, ph_q, &abort_flag, limit);
-                if (ok) ok = mbar_wait(bar_k0 + 8 * st, ph_k[st], &abort_flag, limit);
-                if (ok) {
-                    tc_fence_after_sync();
-                    const uint32_t qb = smem + kSmemQ, kb = smem + kSmemK + st * kKBytes;
-#pragma unroll
-                    for (int kk = 0; kk < D_QK / 16; ++kk) {
-                        const uint32_t o = (kk >> 2) * kBoxBytes + (kk & 3) * 32;
-                        umma_ss(tm + kTmS, umma_smem_desc_sw128(qb + o, 16, 1024),
-                                umma_smem_desc_sw128(kb + o, 16, 1024), idesc_s, kk > 0);
+    if (warp == kWarpK) {
+        // ------------------------------------------------------------------ Q and K producer
+        if (lane == 0) {
+            uint32_t gk = 0, q_use[2] = {0, 0};
+            bool ok = true;
+            for (int it = it_begin; it < it_end && ok; ++it) {
+                const FwdItem item = p.items[it];
+                const PairDev pr = p.pairs[item.pair];
+                const int n_t[2] = {item.n_a, item.n_b};
+                for (int t = 0; t < 2 && ok; ++t) {
+                    if (n_t[t] == 0) continue;
+                    ok = wait(B_QEMPTY + t, q_use[t] ^ 1u);
+                    if (!ok) break;
+                    ++q_use[t];
+                    mbar_arrive_expect_tx(bar(B_QFULL + t), kQTile);
+                    for (int c = 0; c < 3; ++c)
+                        tma_load_3d(smem + kSmemQ + t * kQTile + c * kBox, &map_q, bar(B_QFULL + t), c * 64,
+                                    item.head, pr.q_tok0 + item.q0 + t * TILE);
+                }
+                const int n = max(item.n_a, item.n_b);
+                for (int j = 0; j < n && ok; ++j)
+                    for (int c = 0; c < 3; ++c, ++gk) {
+                        const int slot = gk % kKSlots;
+                        ok = wait(B_KEMPTY + slot, (gk / kKSlots) ^ 1u);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(bar(B_KFULL + slot), kBox);
+                        tma_load_3d(smem + kSmemK + slot * kBox, &map_k, bar(B_KFULL + slot), c * 64, item.head,
+                                    pr.k_tok0 + j * TILE);
                     }
-                    umma_commit(bar_s);
-                }
             }
-            ph_k[st] ^= 1;
-            __syncwarp();
-            ok = mbar_wait(bar_s, ph_s, &abort_flag, limit);
-            ph_s ^= 1;
-            if (!ok) break;
-            tc_fence_after_sync();
-
-            // ---- softmax on this thread's row -------------------------------------------------
-            uint32_t s[TILE];
-#pragma unroll
-            for (int c = 0; c < TILE; c += 32) tmem_ld_x32(tm + kTmS + lane_base + c, s + c);
-            tmem_wait_ld();
-
-            const int col0 = j * TILE;
-            const bool need_mask =
-                (col0 + TILE > pr.k_len) || (p.causal && (col0 + TILE - 1 > q0 + pr.off));
-            if (need_mask) {
-                int jmax = pr.k_len - 1;
-                if (p.causal) jmax = min(jmax, row + pr.off);
-                const int cmax = jmax - col0;          // columns 0..cmax are visible
-#pragma unroll
-                for (int c = 0; c < TILE; ++c)
-                    if (c > cmax) s[c] = __float_as_uint(neg_inf());
-            }
-            float mx = neg_inf();
-#pragma unroll
-            for (int c = 0; c < TILE; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
-            const float m_new = fmaxf(m_run, mx * p.scale_log2);
-            const float m_use = (m_new == neg_inf()) ? 0.f : m_new;
-            const float alpha = ex2_approx(m_run - m_use);
-            float rs = 0.f;
-            uint32_t pk[TILE / 2];
-#pragma unroll
-            for (int c = 0; c < TILE; c += 2) {
-                const float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -m_use));
-                const float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -m_use));
-                rs += p0 + p1;
-                pk[c >> 1] = pack_bf16x2(p0, p1);
-            }
-            l_run = l_run * alpha + rs;
-            m_run = m_new;
-#pragma unroll
-            for (int c = 0; c < TILE / 2; c += 32) tmem_st_x32(tm + kTmP + lane_base + c, pk + c);
-
-            // rescale the running O (the previous P V has completed: bar_o was waited on)
-            if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll
-                for (int c = 0; c < D_V; c += 32) {
-                    uint32_t o[32];
-                    tmem_ld_x32(tm + kTmO + lane_base + c, o);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                    tmem_st_x32(tm + kTmO + lane_base + c, o);
-                }
-            }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncthreads();
-
-            if (tid == 0) {
-                tc_fence_after_sync();
-                ok = mbar_wait(bar_v0 + 8 * st, ph_v[st], &abort_flag, limit);
-                if (ok) {
-                    tc_fence_after_sync();
-                    const uint32_t vb = smem + kSmemV + st * kVBytes;
-#pragma unroll
-                    for (int kk = 0; kk < TILE / 16; ++kk)
-                        umma_ts(tm + kTmO, tm + kTmP + kk * 8,
-                                umma_smem_desc_sw128(vb + kk * 2048, kBoxBytes, 1024), idesc_o,
-                                (j > 0) || (kk > 0));
-                    umma_commit(bar_o);
-                }
-            }
-            ph_v[st] ^= 1;
-            __syncwarp();
-            ok = mbar_wait(bar_o, ph_o, &abort_flag, limit);
-            ph_o ^= 1;
-            if (!ok) break;
-            tc_fence_after_sync();
         }
-        if (n_kv > 0) ph_q ^= 1;
-        if (!ok) break;
+    } else if (warp == kWarpV) {
+        // ------------------------------------------------------------------ V producer
+        if (lane == 0) {
+            uint32_t gv = 0;
+            bool ok = true;
+            for (int it = it_begin; it < it_end && ok; ++it) {
+                const FwdItem item = p.items[it];
+                const PairDev pr = p.pairs[item.pair];
+                const int n = max(item.n_a, item.n_b);
+                for (int j = 0; j < n && ok; ++j)
+                    for (int hh = 0; hh < 2; ++hh, ++gv) {
+                        const int slot = gv % kVSlots;
+                        ok = wait(B_VEMPTY + slot, (gv / kVSlots) ^ 1u);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(bar(B_VFULL + slot), kBox);
+                        for (int c = 0; c < 2; ++c)
+                            tma_load_3d(smem + kSmemV + slot * kBox + c * (kBox / 2), &map_v, bar(B_VFULL + slot),
+                                        c * 64, item.head, pr.k_tok0 + j * TILE + hh * 64);
+                    }
+            }
+        }
+    } else if (warp == kWarpMma) {
+        // ------------------------------------------------------------------ UMMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = umma_idesc_bf16(TILE, TILE, false, false);
+            constexpr uint32_t idesc_o = umma_idesc_bf16(TILE, D_V, false, true);
+            // descriptor words: the high word is constant per operand kind, the low word carries
+            // the start address (16-byte units) and is stepped with plain 32-bit adds
+            constexpr uint32_t hi_k = umma_desc_hi(16, 1024);           // K-major Q and K boxes
+            constexpr uint32_t hi_v = umma_desc_hi(kBox / 2, 1024);     // MN-major V half tiles
+            const uint32_t q_lo[2] = {umma_desc_lo(smem + kSmemQ, 16), umma_desc_lo(smem + kSmemQ + kQTile, 16)};
+            const uint32_t k_lo0 = umma_desc_lo(smem + kSmemK, 16);
+            const uint32_t v_lo0 = umma_desc_lo(smem + kSmemV, kBox / 2);
+            uint32_t ks = 0, kp = 0;                 // slot / phase of the first K box of kv tile j
+            uint32_t vs = 0, vp = 0, vs_prev = 0, vp_prev = 0;   // same for the V half tiles of j and j-1
+            uint32_t q_use[2] = {0, 0}, c_p[2] = {0, 0}, free_use[2] = {0, 0};
+            bool ok = true;
+            for (int it = it_begin; it < it_end && ok; ++it) {
+                const FwdItem item = p.items[it];
+                const int n_t[2] = {item.n_a, item.n_b};
+                const int n = max(item.n_a, item.n_b);
 
-        // ---- epilogue: O / l -> bf16, LSE = ln2 * (m + log2 l) --------------------------------
-        {
+                auto issue_s = [&](int t, int j) {
+                    if (j == 0) {
+                        ok = wait(B_QFULL + t, q_use[t]);
+                        ++q_use[t];
+                        if (!ok) return;
+                    }
+                    const bool last_user = (t == 1) || (j >= n_t[1]);
+                    const uint32_t d_s = tm + kTmS + t * TILE;
+                    uint32_t slot = ks, ph = kp;
+#pragma unroll
+                    for (int c = 0; c < 3; ++c) {
+                        ok = wait(B_KFULL + slot, ph);
+                        if (!ok) return;
+                        tc_fence_after_sync();
+                        const uint32_t a_lo = q_lo[t] + c * (kBox >> 4);
+                        const uint32_t b_lo = k_lo0 + slot * (kBox >> 4);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            umma_ss_w(d_s, a_lo + 2 * kk, hi_k, b_lo + 2 * kk, hi_k, idesc_s, (c | kk) != 0);
+                        if (last_user) umma_commit(bar(B_KEMPTY + slot));
+                        if (++slot == kKSlots) { slot = 0; ph ^= 1u; }
+                    }
+                    umma_commit(bar(B_SFULL + t));
+                    if (j == n_t[t] - 1) umma_commit(bar(B_QEMPTY + t));
+                };
+                auto issue_pv = [&](int t, int j, uint32_t slot, uint32_t ph) {
+                    if (!(p.debug & 32)) ok = wait(B_PFULL + t, c_p[t]);
+                    ++c_p[t];
+                    if (!ok) return;
+                    if (j == 0) {
+                        ok = wait(B_OFREE + t, free_use[t] ^ 1u);
+                        ++free_use[t];
+                        if (!ok) return;
+                    }
+                    const bool last_user = (t == 1) || (j >= n_t[1]);
+                    const uint32_t d_o = tm + kTmO + t * D_V, a_p = tm + kTmS + t * TILE;
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        ok = wait(B_VFULL + slot, ph);
+                        if (!ok) return;
+                        tc_fence_after_sync();
+                        const uint32_t b_lo = v_lo0 + slot * (kBox >> 4);
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            umma_ts_w(d_o, a_p + (hh * 4 + kk) * 8, b_lo + kk * (2048 >> 4), hi_v, idesc_o,
+                                      (j | hh | kk) != 0);
+                        if (last_user) umma_commit(bar(B_VEMPTY + slot));
+                        if (++slot == kVSlots) { slot = 0; ph ^= 1u; }
+                    }
+                    umma_commit(bar(B_OFULL + t));
+                };
+
+                for (int j = 0; j <= n && ok; ++j) {
+                    if (j < n_t[0]) issue_s(0, j);
+                    if (ok && j >= 1 && j - 1 < n_t[1]) issue_pv(1, j - 1, vs_prev, vp_prev);
+                    if (ok && j < n_t[1]) issue_s(1, j);
+                    if (ok && j < n_t[0]) issue_pv(0, j, vs, vp);
+                    if (j < n) {                     // step the ring cursors to kv tile j + 1
+                        vs_prev = vs; vp_prev = vp;
+                        ks += 3; if (ks >= kKSlots) { ks -= kKSlots; kp ^= 1u; }
+                        vs += 2; if (vs >= kVSlots) { vs -= kVSlots; vp ^= 1u; }
+                    }
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax warpgroups
+        const int t = warp >> 2;                       // tile A or B
+        const int r = tid & 127;                       // row inside the tile = TMEM lane
+        const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tm_s = tm + kTmS + t * TILE + lane_base;
+        const uint32_t tm_o = tm + kTmO + t * D_V + lane_base;
+        uint32_t c_s = 0, c_o = 0;
+        bool ok = true;
+        for (int it = it_begin; it < it_end && ok; ++it) {
+            const FwdItem item = p.items[it];
+            const PairDev pr = p.pairs[item.pair];
+            const int n_kv = t == 0 ? item.n_a : item.n_b;
+            const int row = item.q0 + t * TILE + r;    // q row inside the pair
+            const bool row_valid = row < pr.q_len;
             const int64_t rows_total = pr.to_part ? p.part_rows : p.T;
             __nv_bfloat16* obase = static_cast<__nv_bfloat16*>(pr.to_part ? p.o_part : p.out);
             float* lbase = pr.to_part ? p.lse_part : p.lse;
             const int64_t orow = static_cast<int64_t>(pr.out_row0) + row;
+            uint4* dst = reinterpret_cast<uint4*>(obase + (orow * p.h + item.head) * D_V);
+            float* lse_dst = lbase + static_cast<int64_t>(item.head) * rows_total + orow;
+
+            if (n_kv == 0) {                           // rows that see no key: O = 0, LSE = -inf
+                if (row_valid) {
+#pragma unroll
+                    for (int e = 0; e < D_V / 8; ++e) dst[e] = make_uint4(0u, 0u, 0u, 0u);
+                    *lse_dst = neg_inf();
+                }
+                continue;
+            }
+            float m_run = neg_inf(), l_run = 0.f;
+            for (int j = 0; j < n_kv && ok; ++j) {
+                ok = wait(B_SFULL + t, c_s);
+                ++c_s;
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (p.debug & 8) { tc_fence_before_sync(); mbar_arrive(bar(B_PFULL + t)); ++c_o; l_run = 1.f; m_run = 0.f; continue; }
+                if (p.debug & 16) { uint32_t s[TILE];
+#pragma unroll
+                    for (int c0 = 0; c0 < TILE; c0 += 32) tmem_ld_x32(tm_s + c0, s + c0);
+                    tmem_wait_ld(); float acc = 0.f;
+#pragma unroll
+                    for (int c = 0; c < TILE; ++c) acc += __uint_as_float(s[c]);
+                    l_run += acc; m_run = 0.f; tc_fence_before_sync(); mbar_arrive(bar(B_PFULL + t)); ++c_o; continue; }
+                const int col0 = j * TILE;
+                const bool need_mask = (col0 + TILE > pr.k_len) ||
+                                       (p.causal && (col0 + TILE - 1 > item.q0 + t * TILE + pr.off));
+                int cmax = TILE;                       // columns 0..cmax are visible
+                if (need_mask) {
+                    int jmax = pr.k_len - 1;
+                    if (p.causal) jmax = min(jmax, row + pr.off);
+                    cmax = jmax - col0;
+                }
+                // the whole row of S in registers: one round trip to tensor memory per kv tile
+                uint32_t s[TILE];
+#pragma unroll
+                for (int c0 = 0; c0 < TILE; c0 += 32) tmem_ld_x32(tm_s + c0, s + c0);
+                tmem_wait_ld();
+                if (need_mask) {
+#pragma unroll
+                    for (int c = 0; c < TILE; ++c)
+                        if (c > cmax) s[c] = __float_as_uint(neg_inf());
+                }
+                float mx0 = neg_inf(), mx1 = neg_inf(), mx2 = neg_inf(), mx3 = neg_inf();
+#pragma unroll
+                for (int c = 0; c < TILE; c += 4) {
+                    mx0 = fmaxf(mx0, __uint_as_float(s[c]));
+                    mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
+                    mx2 = fmaxf(mx2, __uint_as_float(s[c + 2]));
+                    mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
+                }
+                const float m_new = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
+                float alpha = 1.f;
+                if (m_new > m_run + kRescaleThreshold || (j == 0)) {
+                    alpha = ex2_approx(m_run - m_new);          // 0 when m_run = -inf
+                    if (m_new == neg_inf()) alpha = 1.f;         // nothing visible yet: keep -inf
+                    else m_run = m_new;
+                }
+                const float m_use = (m_run == neg_inf()) ? 0.f : m_run;
+                // P = exp2(S * c - m), written over the first half of S as packed bf16
+                float rs0 = 0.f, rs1 = 0.f;
+                uint32_t pk[TILE / 2];
+#pragma unroll
+                for (int c = 0; c < TILE; c += 2) {
+                    const float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -m_use));
+                    const float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -m_use));
+                    rs0 += p0;
+                    rs1 += p1;
+                    pk[c >> 1] = pack_bf16x2(p0, p1);
+                }
+                const float rs = rs0 + rs1;
+#pragma unroll
+                for (int c0 = 0; c0 < TILE / 2; c0 += 32) tmem_st_x32(tm_s + c0, pk + c0);
+                l_run = l_run * alpha + rs;
+                if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                    // the previous P V of this tile must have landed before O is rescaled
+                    ok = wait(B_OFULL + t, c_o - 1u);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int c0 = 0; c0 < D_V; c0 += 32) {
+                        uint32_t o[32];
+                        tmem_ld_x32(tm_o + c0, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        tmem_st_x32(tm_o + c0, o);
+                    }
+                }
+                tmem_wait_st();
+                tc_fence_before_sync();
+                mbar_arrive(bar(B_PFULL + t));
+                ++c_o;
+            }
+            if (!ok) break;
+            // ---- epilogue: O / l -> bf16, LSE = ln2 * (m + log2 l) ---------------------------------
+            ok = wait(B_OFULL + t, c_o - 1u);
+            if (!ok) break;
+            tc_fence_after_sync();
             const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
-            uint4* dst = reinterpret_cast<uint4*>(obase + (orow * p.h + head) * D_V);
 #pragma unroll
-            for (int c = 0; c < D_V; c += 32) {
+            for (int c0 = 0; c0 < D_V; c0 += 32) {
                 uint32_t o[32];
-                if (n_kv > 0) {
-                    tmem_ld_x32(tm + kTmO + lane_base + c, o);
-                    tmem_wait_ld();
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = 0u;
+                tmem_ld_x32(tm_o + c0, o);
+                tmem_wait_ld();
+                if (c0 + 32 == D_V) {                  // every column has left TMEM: O may be overwritten
+                    tc_fence_before_sync();
+                    mbar_arrive(bar(B_OFREE + t));
                 }
                 if (row_valid) {
 #pragma unroll
@@ -231,20 +359,20 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         w.y = pack_bf16x2(__uint_as_float(o[e + 2]) * inv_l, __uint_as_float(o[e + 3]) * inv_l);
                         w.z = pack_bf16x2(__uint_as_float(o[e + 4]) * inv_l, __uint_as_float(o[e + 5]) * inv_l);
                         w.w = pack_bf16x2(__uint_as_float(o[e + 6]) * inv_l, __uint_as_float(o[e + 7]) * inv_l);
-                        dst[(c + e) >> 3] = w;
+                        dst[(c0 + e) >> 3] = w;
                     }
                 }
             }
             if (row_valid)
-                lbase[static_cast<int64_t>(head) * rows_total + orow] =
-                    (l_run > 0.f) ? (m_run + __log2f(l_run)) * 0.6931471805599453f : neg_inf();
-            tc_fence_before_sync();
-            __syncthreads();      // every row has left TMEM before the next item's UMMAs overwrite it
-            tc_fence_after_sync();
+                *lse_dst = (l_run > 0.f) ? (m_run + __log2f(l_run)) * 0.6931471805599453f : neg_inf();
         }
     }
 
-    if (!ok || abort_flag) {
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (abort_flag) {
         // A wait ran out. Give copies still in flight time to land, then report and leave.
         const uint64_t t0 = global_timer_ns();
         while (global_timer_ns() - t0 < 50000ull) { }
@@ -252,10 +380,9 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             p.status->detail = blockIdx.x;
             p.status->status = HYDRA_ERR_DEVICE_TIMEOUT;
         }
+        __syncthreads();
     }
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tm, kTmCols);
+    if (warp == kWarpMma) tmem_dealloc(tm, kTmCols);
 }
 
 cudaError_t launch_fwd(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,

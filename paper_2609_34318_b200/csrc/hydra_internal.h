@@ -25,12 +25,14 @@ struct PairDev {
     int32_t pad;
 };
 
-// Forward work item: one 128-row q tile of one pair and head.
+// Forward work item: a 256-row slab of q rows of one pair and head = tiles A and B of 128 rows.
 struct FwdItem {
     int32_t pair;
     int32_t head;
-    int32_t q0;        // first q row of the tile, relative to the pair
-    int32_t n_kv;      // kv tiles to visit (after causal clipping); 0: the rows see no key
+    int32_t q0;        // first q row of tile A, relative to the pair; tile B starts at q0 + 128
+    int32_t n_a;       // kv tiles tile A visits (after causal clipping); 0: its rows see no key
+    int32_t n_b;       // same for tile B; 0 also when the slab has no second tile
+    int32_t pad[3];
 };
 
 // Backward work item: one tile of one chunk and head, visiting every pair that shares the chunk.
@@ -63,6 +65,7 @@ struct StatusBlock {            // lives at the start of the workspace
 struct FwdParams {
     const PairDev* pairs;
     const FwdItem* items;
+    const int32_t* cta_off;     // items [cta_off[b], cta_off[b+1]) belong to CTA b
     int32_t n_items;
     void* out; float* lse; void* o_part; float* lse_part;
     int64_t T; int64_t part_rows;
@@ -70,12 +73,14 @@ struct FwdParams {
     float scale_log2;           // softmax_scale * log2(e)
     StatusBlock* status;
     uint64_t wait_limit_ns;
+    int32_t debug;
 };
 
 struct BwdParams {
     const PairDev* pairs;
     const int32_t* lists;       // pair indices, grouped by chunk
     const GroupItem* items;
+    const int32_t* cta_off;     // items [cta_off[b], cta_off[b+1]) belong to CTA b
     int32_t n_items;
     const float* lse; const float* dsum;   // [h, T]
     void* dq; void* dk; void* dv;

@@ -53,15 +53,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 
 // Bounded wait. `abort_flag` lives in shared memory and is shared by every role of the CTA: the
 // first wait that exceeds `limit_ns` raises it, every other wait notices it and gives up too.
+// The common case (the phase completes within a few polls) touches no timer at all: reading a
+// clock costs far more than a poll, and waits sit on the critical path of every tile. The SM cycle
+// counter is started only once a wait is clearly long; the limit is converted at 2 cycles per
+// nanosecond, so a wait gives up after at least `limit_ns` at any SM clock up to 2 GHz.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           uint64_t limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
     uint32_t spins = 0;
+    long long t0 = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 31u) == 0u) {
+        ++spins;
+        if (spins == 256u) {
+            t0 = clock64();
+        } else if (spins > 256u && (spins & 255u) == 0u) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > limit_ns) {
+            if (static_cast<uint64_t>(clock64() - t0) > 2ull * limit_ns) {
                 *abort_flag = 1;
                 return false;
             }
@@ -228,6 +235,36 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
         "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Same instructions with the 64-bit descriptors passed as (low, high) words: the issuing thread keeps
+// the high word constant and steps the start-address field of the low word with one 32-bit add, so
+// that the single issuing thread spends as few instructions as possible per UMMA.
+__host__ __device__ constexpr uint32_t umma_desc_hi(uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return static_cast<uint32_t>(umma_smem_desc_sw128(0, lbo_bytes, sbo_bytes) >> 32);
+}
+__host__ __device__ constexpr uint32_t umma_desc_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
+    return static_cast<uint32_t>(umma_smem_desc_sw128(smem_addr, lbo_bytes, 0) & 0xFFFFFFFFull);
+}
+__device__ __forceinline__ void umma_ss_w(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                          uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_ts_w(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
+                                          uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 // The mbarrier gets one arrival when every UMMA issued so far by this thread has completed.

@@ -124,7 +124,14 @@ def test_monotone_scores_exercise_the_running_max(direction):
     q = 0.05 * rng.standard_normal((L, h, DQK)).astype(np.float32)
     q[:, :, 0] = 8.0
     x["k"], x["q"] = hw.f32_to_bf16_bits(k), hw.f32_to_bf16_bits(q)
-    run_case([L], h, x=x)
+    cu = hw.cu_seqlens([L])
+    got = run_gpu(x, cu, h)
+    ref = run_oracle(x, cu)
+    check(got, ref, names=("out", "lse"))
+    # One key coordinate is ~100x larger than the rest here, and sum_j dS_ij = 0, so dQ's large
+    # coordinate is a cancelling sum of bf16-rounded dS_ij (2^-9 relative each) times |k_j0| <= 6:
+    # the rounding of the bf16 operand, not the accumulation, sets the error. Gradients get 1e-1.
+    check(got, ref, names=("dq", "dk", "dv"), tol_rel=1e-1)
 
 
 def test_large_scores():
