@@ -153,7 +153,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         abort_flag = 0;
         for (int i = 0; i < B_COUNT; ++i) {
             const bool by_threads = (i == B_SFREE) || (i == B_PFULL) || (i == B_ACCFREE);
-            mbar_init(bar(i), by_threads ? 256u : 1u);
+            mbar_init(bar(i), by_threads ? 8u : 1u);   // 8 = elementwise warps
         }
         fence_mbar_init();
         tma_prefetch_desc(&map_q); tma_prefetch_desc(&map_k);
@@ -191,7 +191,21 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 for (int c = 0; c < 2; ++c)
                     tma_load_3d(smem + kDO + c * kBox128, &map_do, bar(B_QFULL), c * 64, item.head,
                                 first.q_tok0 + item.r0);
+                // L2 prefetch runs kPrefetch tiles ahead of the loads: a stage frees late (K is read by S
+                // and again by the dQ update), so the load itself must not pay the HBM latency
+                constexpr int kPrefetch = 4;
+                TileIter pf = ti;
+                auto prefetch_tile = [&]() {
+                    if (!pf.valid()) return;
+                    const int ptok = pf.cur.k_tok0 + pf.t * TILE;
+                    for (int c = 0; c < 3; ++c) tma_prefetch_l2_3d(&map_k, c * 64, item.head, ptok);
+                    for (int c = 0; c < 2; ++c) tma_prefetch_l2_3d(&map_v, c * 64, item.head, ptok);
+                    pf.next();
+                };
+                pf.next();
+                for (int a = 0; a < kPrefetch; ++a) prefetch_tile();
                 for (; ti.valid() && ok; ti.next()) {
+                    prefetch_tile();
                     const int tok = ti.cur.k_tok0 + ti.t * TILE;
                     const int st = gk % kKStages;
                     ok = wait(B_KEMPTY + st, (gk / kKStages) ^ 1u);
@@ -213,6 +227,9 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
     } else if (warp == kWarpMma) {
         // ------------------------------------------------------------------ UMMA issuer
+        // Two cursors walk the same (item, kv tile) sequence: `a` issues S = Q K^T and dP = dO V^T,
+        // `b` issues dQ += dS K and trails `a`. Neither blocks the other: each is issued as soon as
+        // its own operands are there (dQ first, because it frees a K stage), also across items.
         if (lane == 0) {
             constexpr uint32_t idesc_s = umma_idesc_bf16(TILE, TILE, false, false);
             constexpr uint32_t idesc_dq = umma_idesc_bf16(TILE, D_QK, false, true);
@@ -221,75 +238,114 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const uint32_t q_lo = umma_desc_lo(smem + kQ, 16), do_lo = umma_desc_lo(smem + kDO, 16);
             const uint32_t k_lo0 = umma_desc_lo(smem + kK, 16), v_lo0 = umma_desc_lo(smem + kV, 16);
             const uint32_t kmn_lo0 = umma_desc_lo(smem + kK, kBox128);
-            uint32_t items = 0, c_s = 0, c_p = 0, gk_s = 0, gv = 0, gk_q = 0;
-            bool ok = true;
-            for (int it = it_begin; it < it_end && ok; ++it) {
-                const GroupItem item = p.items[it];
-                const int32_t* list = p.lists + item.list_off;
-                const PairDev first = p.pairs[list[0]];
-                TileIter ti;
-                ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
-                if (!ti.valid()) continue;
-                int n_tiles = 0;
-                for (TileIter c = ti; c.valid(); c.next()) ++n_tiles;
 
-                auto issue_s_dp = [&](bool last) {
-                    if (c_s > 0) ok = wait(B_SFREE, c_s - 1u);      // S / dP of the previous step are in registers
-                    if (!ok) return;
-                    const int st = gk_s % kKStages;
-                    ok = wait(B_KFULL + st, gk_s / kKStages);
-                    ++gk_s;
-                    if (!ok) return;
-                    tc_fence_after_sync();
-                    const uint32_t k_lo = k_lo0 + st * (3 * kBox128 >> 4);
-#pragma unroll
-                    for (int kk = 0; kk < D_QK / 16; ++kk) {
-                        const uint32_t o = (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2;
-                        umma_ss_w(tm + kTmS, q_lo + o, hi_kmaj, k_lo + o, hi_kmaj, idesc_s, kk > 0);
-                    }
-#pragma unroll
-                    for (int c = 0; c < 2; ++c, ++gv) {
-                        const int slot = gv % kVSlots;
-                        ok = wait(B_VFULL + slot, gv / kVSlots);
-                        if (!ok) return;
-                        tc_fence_after_sync();
-                        const uint32_t v_lo = v_lo0 + slot * (kBox128 >> 4);
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            umma_ss_w(tm + kTmDP, do_lo + c * (kBox128 >> 4) + kk * 2, hi_kmaj, v_lo + kk * 2, hi_kmaj,
-                                      idesc_s, (c | kk) != 0);
-                        umma_commit(bar(B_VEMPTY + slot));
-                    }
-                    umma_commit(bar(B_SFULL));
-                    ++c_s;
-                    if (last) umma_commit(bar(B_QEMPTY));            // Q and dO are no longer read
-                };
-                auto issue_dq = [&](int j) {
-                    ok = wait(B_PFULL, c_p);
-                    ++c_p;
-                    if (!ok) return;
-                    if (j == 0 && items > 0) ok = wait(B_ACCFREE, items - 1u);
-                    if (!ok) return;
-                    tc_fence_after_sync();
-                    const int st = gk_q % kKStages;
-                    ++gk_q;
-                    const uint32_t k_lo = kmn_lo0 + st * (3 * kBox128 >> 4);
-#pragma unroll
-                    for (int kk = 0; kk < TILE / 16; ++kk)
-                        umma_ts_w(tm + kTmDQ, tm + kTmDS + kk * 8, k_lo + kk * (2048 >> 4), hi_kmn, idesc_dq,
-                                  (j | kk) != 0);
-                    umma_commit(bar(B_DSFREE));
-                    umma_commit(bar(B_KEMPTY + st));
-                };
-
-                ok = wait(B_QFULL, items);
-                if (!ok) break;
-                issue_s_dp(n_tiles == 1);
-                for (int j = 0; j < n_tiles && ok; ++j) {
-                    if (j + 1 < n_tiles) issue_s_dp(j + 2 == n_tiles);
-                    if (ok) issue_dq(j);
+            struct Cursor {
+                int it; TileIter ti; bool first;       // first: next tile is the first of its item
+            };
+            auto open_item = [&](Cursor& c) {            // position on the first tile of item c.it (or later)
+                while (c.it < it_end) {
+                    const GroupItem item = p.items[c.it];
+                    const int32_t* list = p.lists + item.list_off;
+                    const PairDev first = p.pairs[list[0]];
+                    c.ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+                    if (c.ti.valid()) { c.first = true; return; }
+                    ++c.it;
                 }
-                ++items;
+            };
+            Cursor a{it_begin, {}, true}, b{it_begin, {}, true};
+            open_item(a);
+            open_item(b);
+            uint32_t n_s = 0, n_q = 0;                   // tiles issued so far by each cursor
+            uint32_t items_a = 0, items_b = 0;           // items opened so far by each cursor
+            uint32_t gv = 0;
+            uint32_t got_a = 0, got_b = 0;               // operands already seen ready for the pending issue
+            uint32_t spins = 0;
+            long long t0 = 0;
+            bool ok = true;
+            auto ready = [&](uint32_t& got, uint32_t bit, int barrier, uint32_t parity) -> bool {
+                if (got & bit) return true;
+                if (mbar_test_wait(bar(barrier), parity & 1u)) { got |= bit; return true; }
+                return false;
+            };
+            while (ok && b.it < it_end) {
+                bool progressed = false;
+                // ---- dQ of tile n_q: needs dS from the elementwise warps; at the start of an item also
+                //      that the previous item's dQ has been read out of tensor memory
+                if (n_q < n_s) {
+                    bool r = ready(got_b, 1u, B_PFULL, n_q);
+                    if (r && b.first && items_b > 0) r = ready(got_b, 2u, B_ACCFREE, items_b - 1u);
+                    if (r) {
+                        tc_fence_after_sync();
+                        const int st = n_q % kKStages;
+                        const uint32_t k_lo = kmn_lo0 + st * (3 * kBox128 >> 4);
+                        const uint32_t acc0 = b.first ? 0u : 1u;
+#pragma unroll
+                        for (int kk = 0; kk < TILE / 16; ++kk)
+                            umma_ts_w(tm + kTmDQ, tm + kTmDS + kk * 8, k_lo + kk * (2048 >> 4), hi_kmn, idesc_dq,
+                                      kk > 0 ? 1u : acc0);
+                        umma_commit(bar(B_DSFREE));
+                        umma_commit(bar(B_KEMPTY + st));
+                        ++n_q;
+                        got_b = 0;
+                        if (b.first) { ++items_b; b.first = false; }
+                        b.ti.next();
+                        if (!b.ti.valid()) { ++b.it; open_item(b); }
+                        progressed = true;
+                    }
+                }
+                // ---- S and dP of tile n_s: needs S/dP of the previous tile copied out, K stage, two V
+                //      boxes, and at the start of an item Q and dO
+                if (a.it < it_end) {
+                    const int st = n_s % kKStages;
+                    bool r = (n_s == 0) || ready(got_a, 1u, B_SFREE, n_s - 1u);
+                    if (r && a.first) r = ready(got_a, 2u, B_QFULL, items_a);
+                    if (r) r = ready(got_a, 4u, B_KFULL + st, n_s / kKStages);
+                    if (r) r = ready(got_a, 8u, B_VFULL + gv % kVSlots, gv / kVSlots);
+                    if (r) r = ready(got_a, 16u, B_VFULL + (gv + 1) % kVSlots, (gv + 1) / kVSlots);
+                    if (r) {
+                        tc_fence_after_sync();
+                        const uint32_t k_lo = k_lo0 + st * (3 * kBox128 >> 4);
+#pragma unroll
+                        for (int kk = 0; kk < D_QK / 16; ++kk) {
+                            const uint32_t o = (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2;
+                            umma_ss_w(tm + kTmS, q_lo + o, hi_kmaj, k_lo + o, hi_kmaj, idesc_s, kk > 0);
+                        }
+#pragma unroll
+                        for (int c = 0; c < 2; ++c, ++gv) {
+                            const int slot = gv % kVSlots;
+                            const uint32_t v_lo = v_lo0 + slot * (kBox128 >> 4);
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk)
+                                umma_ss_w(tm + kTmDP, do_lo + c * (kBox128 >> 4) + kk * 2, hi_kmaj, v_lo + kk * 2,
+                                          hi_kmaj, idesc_s, (c | kk) != 0);
+                            umma_commit(bar(B_VEMPTY + slot));
+                        }
+                        umma_commit(bar(B_SFULL));
+                        ++n_s;
+                        got_a = 0;
+                        if (a.first) { ++items_a; a.first = false; }
+                        a.ti.next();
+                        if (!a.ti.valid()) {                 // last tile of the item: Q and dO are free
+                            umma_commit(bar(B_QEMPTY));
+                            ++a.it;
+                            open_item(a);
+                        }
+                        progressed = true;
+                    }
+                }
+                if (progressed) {
+                    spins = 0;
+                } else {
+                    // back off: a hot polling loop would take issue slots from the elementwise warps
+                    // that share this scheduler
+                    __nanosleep(40);
+                    if (++spins == 4096u) {
+                        t0 = clock64();
+                    } else if (spins > 4096u && (spins & 1023u) == 0u) {
+                        if (*abort_p) ok = false;
+                        else if (static_cast<uint64_t>(clock64() - t0) > 2ull * limit) { *abort_p = 1; ok = false; }
+                    }
+                }
             }
         }
     } else {
@@ -339,7 +395,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 }
                 tmem_wait_ld();
                 tc_fence_before_sync();
-                mbar_arrive(bar(B_SFREE));             // the next S / dP may overwrite tensor memory
+                mbar_arrive_warp(bar(B_SFREE));             // the next S / dP may overwrite tensor memory
                 int jmax = ti.cur.k_len - 1;
                 if (p.causal) jmax = min(jmax, row + ti.cur.off);
                 const int cmax = jmax - ti.t * TILE - g * 64;      // columns 0..cmax of this half are visible
@@ -361,7 +417,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 tmem_st_x32(tm_ds, ds);
                 tmem_wait_st();
                 tc_fence_before_sync();
-                mbar_arrive(bar(B_PFULL));
+                mbar_arrive_warp(bar(B_PFULL));
                 ++c_ds;
             }
             if (!ok) break;
@@ -376,7 +432,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 tmem_wait_ld();
                 if (c0 == 64) {
                     tc_fence_before_sync();
-                    mbar_arrive(bar(B_ACCFREE));
+                    mbar_arrive_warp(bar(B_ACCFREE));
                 }
                 if (row_valid) store_row_bf16(dst + c0, v, 32, p.scale);
             }
@@ -423,8 +479,8 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         abort_flag = 0;
         for (int i = 0; i < B_COUNT; ++i) {
             uint32_t count = 1u;
-            if (i == B_SFREE || i == B_PFULL || i == B_ACCFREE) count = 256u;
-            if (i >= B_STAT && i < B_STAT + kStages) count = 32u;
+            if (i == B_SFREE || i == B_PFULL || i == B_ACCFREE) count = 8u;   // elementwise warps
+            
             mbar_init(bar(i), count);
         }
         fence_mbar_init();
@@ -489,7 +545,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     s_lse2[st][c] = (l == neg_inf()) ? pos_inf() : l * kLog2e;
                     s_dsum[st][c] = v ? __ldg(p.dsum + idx) : 0.f;
                 }
-                mbar_arrive(bar(B_STAT + st));
+                mbar_arrive_warp(bar(B_STAT + st));
             }
         }
     } else if (warp == kWarpMma) {
@@ -611,7 +667,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 tmem_ld_x32(tm_dp, dp);
                 tmem_wait_ld();
                 tc_fence_before_sync();
-                mbar_arrive(bar(B_SFREE));
+                mbar_arrive_warp(bar(B_SFREE));
                 ok = wait(B_STAT + st, gq / kStages);
                 if (!ok) break;
                 // q row i = u*64 + 32 g + c is visible from kv row krow iff i < q_len and krow <= i + off
@@ -642,7 +698,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 tmem_st_x16(tm_ds, ds);
                 tmem_wait_st();
                 tc_fence_before_sync();
-                mbar_arrive(bar(B_PFULL));
+                mbar_arrive_warp(bar(B_PFULL));
                 ++c_pds;
             }
             if (!ok) break;
@@ -664,7 +720,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 tmem_wait_ld();
                 if (c0 == 32) {
                     tc_fence_before_sync();
-                    mbar_arrive(bar(B_ACCFREE));
+                    mbar_arrive_warp(bar(B_ACCFREE));
                 }
                 if (row_valid) store_row_bf16(dvp + c0, v, 32, 1.f);
             }

@@ -69,7 +69,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         abort_flag = 0;
         for (int i = 0; i < B_COUNT; ++i) {
             const bool by_threads = (i >= B_PFULL && i < B_PFULL + 2) || (i >= B_OFREE && i < B_OFREE + 2);
-            mbar_init(bar(i), by_threads ? 128u : 1u);
+            mbar_init(bar(i), by_threads ? 4u : 1u);   // 4 = warps of a softmax warpgroup
         }
         fence_mbar_init();
         tma_prefetch_desc(&map_q); tma_prefetch_desc(&map_k); tma_prefetch_desc(&map_v);
@@ -258,14 +258,14 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 ++c_s;
                 if (!ok) break;
                 tc_fence_after_sync();
-                if (p.debug & 8) { tc_fence_before_sync(); mbar_arrive(bar(B_PFULL + t)); ++c_o; l_run = 1.f; m_run = 0.f; continue; }
+                if (p.debug & 8) { tc_fence_before_sync(); mbar_arrive_warp(bar(B_PFULL + t)); ++c_o; l_run = 1.f; m_run = 0.f; continue; }
                 if (p.debug & 16) { uint32_t s[TILE];
 #pragma unroll
                     for (int c0 = 0; c0 < TILE; c0 += 32) tmem_ld_x32(tm_s + c0, s + c0);
                     tmem_wait_ld(); float acc = 0.f;
 #pragma unroll
                     for (int c = 0; c < TILE; ++c) acc += __uint_as_float(s[c]);
-                    l_run += acc; m_run = 0.f; tc_fence_before_sync(); mbar_arrive(bar(B_PFULL + t)); ++c_o; continue; }
+                    l_run += acc; m_run = 0.f; tc_fence_before_sync(); mbar_arrive_warp(bar(B_PFULL + t)); ++c_o; continue; }
                 const int col0 = j * TILE;
                 const bool need_mask = (col0 + TILE > pr.k_len) ||
                                        (p.causal && (col0 + TILE - 1 > item.q0 + t * TILE + pr.off));
@@ -333,7 +333,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 }
                 tmem_wait_st();
                 tc_fence_before_sync();
-                mbar_arrive(bar(B_PFULL + t));
+                mbar_arrive_warp(bar(B_PFULL + t));
                 ++c_o;
             }
             if (!ok) break;
@@ -349,7 +349,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 tmem_wait_ld();
                 if (c0 + 32 == D_V) {                  // every column has left TMEM: O may be overwritten
                     tc_fence_before_sync();
-                    mbar_arrive(bar(B_OFREE + t));
+                    mbar_arrive_warp(bar(B_OFREE + t));
                 }
                 if (row_valid) {
 #pragma unroll
