@@ -4,7 +4,6 @@
 #include <atomic>
 #include <cmath>
 #include <cstring>
-#include <cstdlib>
 #include <memory>
 #include <mutex>
 #include <vector>
@@ -220,9 +219,10 @@ std::vector<PairDev> device_pairs(const Problem& pb)
     return v;
 }
 
-inline int32_t kv_tiles(const hydra_pair_t& p, int32_t q0, int causal)
+// kv tiles that the q rows [q0, q0 + rows) of a pair visit (0: they see no key)
+inline int32_t kv_tiles(const hydra_pair_t& p, int32_t q0, int causal, int32_t rows = TILE)
 {
-    const int32_t last_row = std::min(q0 + TILE, p.q_len) - 1;
+    const int32_t last_row = std::min(q0 + rows, p.q_len) - 1;
     int64_t n_keys = p.k_len;
     if (causal) n_keys = std::min<int64_t>(n_keys, int64_t{last_row} + (p.q_start - p.k_start) + 1);
     return n_keys > 0 ? static_cast<int32_t>((n_keys + TILE - 1) / TILE) : 0;
@@ -307,9 +307,10 @@ void build_fwd(const Problem& pb, int causal, int n_ctas, Plan& plan, std::vecto
     std::vector<int32_t> block_of, cost;
     for (size_t pi = 0; pi < pb.pairs.size(); ++pi) {
         const auto& p = pb.pairs[pi];
-        for (int32_t q0 = 0; q0 < p.q_len; q0 += 2 * TILE) {
-            const int32_t n_a = kv_tiles(p, q0, causal);
-            const int32_t n_b = q0 + TILE < p.q_len ? kv_tiles(p, q0 + TILE, causal) : 0;
+        // one item = 512 q rows = two 256-row UMMA tiles of a CTA pair
+        for (int32_t q0 = 0; q0 < p.q_len; q0 += 4 * TILE) {
+            const int32_t n_a = kv_tiles(p, q0, causal, 2 * TILE);
+            const int32_t n_b = q0 + 2 * TILE < p.q_len ? kv_tiles(p, q0 + 2 * TILE, causal, 2 * TILE) : 0;
             for (int32_t a = 0; a < pb.h; ++a) {
                 items.push_back(FwdItem{static_cast<int32_t>(pi), a, q0, n_a, n_b, {0, 0, 0}});
                 block_of.push_back(static_cast<int32_t>(pi) * pb.h + a);
@@ -654,12 +655,15 @@ int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_
     if (int32_t s = device_info(&sms)) return s;
     if (pb.pairs.empty()) return HYDRA_OK;
 
+    const int n_clusters = fwd_max_clusters();        // CTA pairs resident at once: the persistent grid
+    if (n_clusters < 1) return HYDRA_ERR_CUDA;
     const Plan* plan = nullptr;
-    if (int32_t s = get_plan(HYDRA_WS_FWD, pb, causal != 0, sms, &plan)) return s;
+    if (int32_t s = get_plan(HYDRA_WS_FWD, pb, causal != 0, n_clusters, &plan)) return s;
     if (plan->n_items == 0) return HYDRA_OK;
+    // each CTA of a pair stages 64 kv rows of K (box of 64 rows) and 64 value columns of V
     CUtensorMap mq, mk, mv;
-    if (make_map(&mq, q, pb.T, n_heads, D_QK, TILE) || make_map(&mk, k, pb.T, n_heads, D_QK, TILE) ||
-        make_map(&mv, v, pb.T, n_heads, D_V, SUB))
+    if (make_map(&mq, q, pb.T, n_heads, D_QK, TILE) || make_map(&mk, k, pb.T, n_heads, D_QK, SUB) ||
+        make_map(&mv, v, pb.T, n_heads, D_V, TILE))
         return HYDRA_ERR_CUDA;
     if (int32_t s = reset_status(workspace, stream)) return s;
     FwdParams fp{};
@@ -672,11 +676,9 @@ int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_
     fp.scale_log2 = softmax_scale * 1.4426950408889634f;
     fp.status = static_cast<StatusBlock*>(workspace);
     fp.wait_limit_ns = g_wait_limit_ns.load();
-    fp.debug = getenv("HYDRA_FWD_DEBUG") ? atoi(getenv("HYDRA_FWD_DEBUG")) : 0;
-    const int grid = sms;
     {
         ScopedKernelTimer timer(K_FWD, stream);
-        if (launch_fwd(mq, mk, mv, fp, grid, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+        if (launch_fwd(mq, mk, mv, fp, n_clusters, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
     }
     g_launches += 1;
     return HYDRA_OK;

@@ -1,21 +1,26 @@
-// Forward attention of (q-chunk, kv-chunk) pairs on sm_100a.
+// Forward attention of (q-chunk, kv-chunk) pairs on sm_100a, on CTA PAIRS (cluster of two,
+// tcgen05 cta_group::2).
 //
-// One persistent CTA per SM walks a strided share of the work list. A work item is a 256-row slab of
-// q rows of one pair and head, handled as two 128-row tiles (A and B) that ping-pong on the tensor
-// core so that UMMAs of one tile overlap the softmax of the other, and so that every K/V tile pulled
-// from L2 feeds 256 q rows.
+// A work item is a 512-row slab of q rows of one pair and head, handled by one CTA pair as two
+// 256-row UMMA tiles (A and B); each CTA owns 128 rows of each tile. The two tiles ping-pong on the
+// tensor cores so that the UMMAs of one overlap the softmax of the other. Every K/V tile is fetched
+// from L2 once per pair and each CTA stages only its half of it (64 kv rows of K for S = Q K^T, 64
+// value columns of V for O += P V), so three stages of K and of V fit next to the two Q tiles: deep
+// enough to cover the latency of a TMA load, which two full-size stages could not.
 //
-// Warp roles (352 threads):
-//   warps 0-3   softmax of tile A: thread r owns row r = TMEM lane r (no cross-thread reductions)
-//   warps 4-7   softmax of tile B
-//   warp  8     TMA producer of Q (per item) and K (ring of five [128 x 64] boxes)
-//   warp  9     TMA producer of V (ring of three [64 kv rows x 128] half tiles)
-//   warp 10     UMMA issuer (one thread) and owner of the TMEM allocation
+// Warp roles per CTA (352 threads):
+//   warps 0-3   softmax of this CTA's rows of tile A: thread r owns row r = TMEM lane r
+//   warps 4-7   softmax of this CTA's rows of tile B
+//   warp  8     TMA producer of Q (per item) and K
+//   warp  9     TMA producer of V
+//   warp 10     leader CTA only: UMMA issuer (one thread); both CTAs: TMEM allocation
+// Barriers live at the same shared-memory offsets in both CTAs. "Full" barriers are used in the
+// leader's copy (both CTAs' TMA loads count their bytes there; both CTAs' softmax warps arrive
+// there); "done" events of the tensor core are committed to both copies at once.
 //
-// Tensor memory (512 columns): S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512); P (bf16 pairs)
-// is written over the first 64 columns of its S. Issue order per kv tile j:
+// Tensor memory (512 columns per CTA): S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512); P (bf16
+// pairs) is written over the first 64 columns of its S. Issue order per kv tile j:
 //   S_A(j) = Q_A K_j^T ; O_B += P_B(j-1) V_{j-1} ; S_B(j) = Q_B K_j^T ; O_A += P_A(j) V_j
-// UMMAs execute in issue order, so S_t(j+1) cannot overtake the PV that still reads P_t(j).
 // The softmax keeps a running maximum in the exp2 domain and rescales O only when the maximum grew
 // by more than 2^8 (the final LSE is exact whatever reference maximum was used).
 #include <cuda_bf16.h>
@@ -30,19 +35,21 @@ namespace {
 constexpr int kThreads = 352;
 constexpr int kWarpK = 8, kWarpV = 9, kWarpMma = 10;
 constexpr uint32_t kBox = 128 * 128;                  // [128 rows x 64 bf16] = 16 KB
-constexpr uint32_t kQTile = 3 * kBox;                 // 128 x 192
-constexpr int kKSlots = 5, kVSlots = 3;
+constexpr uint32_t kHalfBox = 64 * 128;               // [ 64 rows x 64 bf16] =  8 KB
+constexpr uint32_t kQTile = 3 * kBox;                 // this CTA's 128 x 192 rows of a q tile
+constexpr uint32_t kKStage = 3 * kHalfBox;            // this CTA's 64 kv rows x 192
+constexpr uint32_t kVStage = kBox;                    // 128 kv rows x this CTA's 64 value columns
+constexpr int kKStages = 3, kVStages = 3;
 constexpr uint32_t kSmemQ = 0;
 constexpr uint32_t kSmemK = kSmemQ + 2 * kQTile;
-constexpr uint32_t kSmemV = kSmemK + kKSlots * kBox;
-constexpr uint32_t kSmemTotal = kSmemV + kVSlots * kBox;      // 229,376 B
+constexpr uint32_t kSmemV = kSmemK + kKStages * kKStage;
+constexpr uint32_t kSmemTotal = kSmemV + kVStages * kVStage;  // 221,184 B
 constexpr uint32_t kTmS = 0, kTmO = 256, kTmCols = 512;
 constexpr float kRescaleThreshold = 8.f;              // log2 units
 
-// barrier indices
 enum : int {
-    B_QFULL = 0, B_QEMPTY = 2, B_KFULL = 4, B_KEMPTY = 9, B_VFULL = 14, B_VEMPTY = 17,
-    B_SFULL = 20, B_PFULL = 22, B_OFULL = 24, B_OFREE = 26, B_COUNT = 28
+    B_QFULL = 0, B_QEMPTY = 2, B_KFULL = 4, B_KEMPTY = 7, B_VFULL = 10, B_VEMPTY = 13,
+    B_SFULL = 16, B_PFULL = 18, B_OFULL = 20, B_OFREE = 22, B_COUNT = 24
 };
 
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
@@ -51,7 +58,7 @@ __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); 
 
 size_t fwd_smem_bytes() { return kSmemTotal + 1024; }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const FwdParams p)
 {
@@ -62,25 +69,30 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     __shared__ int abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_cta_rank();
+    const bool leader = rank == 0;
     const uint32_t bar0 = smem_u32(&bars[0]);
     auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
 
     if (tid == 0) {
         abort_flag = 0;
         for (int i = 0; i < B_COUNT; ++i) {
-            const bool by_threads = (i >= B_PFULL && i < B_PFULL + 2) || (i >= B_OFREE && i < B_OFREE + 2);
-            mbar_init(bar(i), by_threads ? 4u : 1u);   // 4 = warps of a softmax warpgroup
+            // P-ready and O-drained collect the 4 softmax warps of a tile in each of the 2 CTAs
+            const bool by_warps = (i >= B_PFULL && i < B_PFULL + 2) || (i >= B_OFREE && i < B_OFREE + 2);
+            mbar_init(bar(i), by_warps ? 8u : 1u);
         }
         fence_mbar_init();
         tma_prefetch_desc(&map_q); tma_prefetch_desc(&map_k); tma_prefetch_desc(&map_v);
     }
-    if (warp == kWarpMma) { tmem_alloc(smem_u32(&tmem_base_slot), kTmCols); tmem_relinquish(); }
+    if (warp == kWarpMma) { tmem_alloc_pair(smem_u32(&tmem_base_slot), kTmCols); tmem_relinquish_pair(); }
     tc_fence_before_sync();
     __syncthreads();
+    cluster_sync_all();                                // both CTAs' barriers exist before anyone signals them
     tc_fence_after_sync();
     const uint32_t tm = tmem_base_slot;
     const uint64_t limit = p.wait_limit_ns;
-    const int it_begin = p.cta_off[blockIdx.x], it_end = p.cta_off[blockIdx.x + 1];
+    const int cluster = static_cast<int>(cluster_id_x());
+    const int it_begin = p.cta_off[cluster], it_end = p.cta_off[cluster + 1];
     volatile int* abort_p = &abort_flag;
     auto wait = [&](int b, uint32_t parity) -> bool { return mbar_wait(bar(b), parity & 1u, abort_p, limit); };
 
@@ -98,21 +110,21 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     ok = wait(B_QEMPTY + t, q_use[t] ^ 1u);
                     if (!ok) break;
                     ++q_use[t];
-                    mbar_arrive_expect_tx(bar(B_QFULL + t), kQTile);
+                    if (leader) mbar_arrive_expect_tx(bar(B_QFULL + t), 2 * kQTile);
                     for (int c = 0; c < 3; ++c)
-                        tma_load_3d(smem + kSmemQ + t * kQTile + c * kBox, &map_q, bar(B_QFULL + t), c * 64,
-                                    item.head, pr.q_tok0 + item.q0 + t * TILE);
+                        tma_load_3d_pair(smem + kSmemQ + t * kQTile + c * kBox, &map_q, bar(B_QFULL + t), c * 64,
+                                         item.head, pr.q_tok0 + item.q0 + t * 2 * TILE + rank * TILE);
                 }
                 const int n = max(item.n_a, item.n_b);
-                for (int j = 0; j < n && ok; ++j)
-                    for (int c = 0; c < 3; ++c, ++gk) {
-                        const int slot = gk % kKSlots;
-                        ok = wait(B_KEMPTY + slot, (gk / kKSlots) ^ 1u);
-                        if (!ok) break;
-                        mbar_arrive_expect_tx(bar(B_KFULL + slot), kBox);
-                        tma_load_3d(smem + kSmemK + slot * kBox, &map_k, bar(B_KFULL + slot), c * 64, item.head,
-                                    pr.k_tok0 + j * TILE);
-                    }
+                for (int j = 0; j < n && ok; ++j, ++gk) {
+                    const int slot = gk % kKStages;
+                    ok = wait(B_KEMPTY + slot, (gk / kKStages) ^ 1u);
+                    if (!ok) break;
+                    if (leader) mbar_arrive_expect_tx(bar(B_KFULL + slot), 2 * kKStage);
+                    for (int c = 0; c < 3; ++c)
+                        tma_load_3d_pair(smem + kSmemK + slot * kKStage + c * kHalfBox, &map_k, bar(B_KFULL + slot),
+                                         c * 64, item.head, pr.k_tok0 + j * TILE + rank * 64);
+                }
             }
         }
     } else if (warp == kWarpV) {
@@ -124,32 +136,28 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 const FwdItem item = p.items[it];
                 const PairDev pr = p.pairs[item.pair];
                 const int n = max(item.n_a, item.n_b);
-                for (int j = 0; j < n && ok; ++j)
-                    for (int hh = 0; hh < 2; ++hh, ++gv) {
-                        const int slot = gv % kVSlots;
-                        ok = wait(B_VEMPTY + slot, (gv / kVSlots) ^ 1u);
-                        if (!ok) break;
-                        mbar_arrive_expect_tx(bar(B_VFULL + slot), kBox);
-                        for (int c = 0; c < 2; ++c)
-                            tma_load_3d(smem + kSmemV + slot * kBox + c * (kBox / 2), &map_v, bar(B_VFULL + slot),
-                                        c * 64, item.head, pr.k_tok0 + j * TILE + hh * 64);
-                    }
+                for (int j = 0; j < n && ok; ++j, ++gv) {
+                    const int slot = gv % kVStages;
+                    ok = wait(B_VEMPTY + slot, (gv / kVStages) ^ 1u);
+                    if (!ok) break;
+                    if (leader) mbar_arrive_expect_tx(bar(B_VFULL + slot), 2 * kVStage);
+                    tma_load_3d_pair(smem + kSmemV + slot * kVStage, &map_v, bar(B_VFULL + slot), rank * 64, item.head,
+                                     pr.k_tok0 + j * TILE);
+                }
             }
         }
     } else if (warp == kWarpMma) {
-        // ------------------------------------------------------------------ UMMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = umma_idesc_bf16(TILE, TILE, false, false);
-            constexpr uint32_t idesc_o = umma_idesc_bf16(TILE, D_V, false, true);
-            // descriptor words: the high word is constant per operand kind, the low word carries
-            // the start address (16-byte units) and is stepped with plain 32-bit adds
+        // ------------------------------------------------------------------ UMMA issuer (leader CTA)
+        if (leader && lane == 0) {
+            constexpr uint32_t idesc_s = umma_idesc_bf16(2 * TILE, TILE, false, false);
+            constexpr uint32_t idesc_o = umma_idesc_bf16(2 * TILE, D_V, false, true);
             constexpr uint32_t hi_k = umma_desc_hi(16, 1024);           // K-major Q and K boxes
-            constexpr uint32_t hi_v = umma_desc_hi(kBox / 2, 1024);     // MN-major V half tiles
+            constexpr uint32_t hi_v = umma_desc_hi(kBox, 1024);         // MN-major V (one 64-column chunk)
             const uint32_t q_lo[2] = {umma_desc_lo(smem + kSmemQ, 16), umma_desc_lo(smem + kSmemQ + kQTile, 16)};
             const uint32_t k_lo0 = umma_desc_lo(smem + kSmemK, 16);
-            const uint32_t v_lo0 = umma_desc_lo(smem + kSmemV, kBox / 2);
-            uint32_t ks = 0, kp = 0;                 // slot / phase of the first K box of kv tile j
-            uint32_t vs = 0, vp = 0, vs_prev = 0, vp_prev = 0;   // same for the V half tiles of j and j-1
+            const uint32_t v_lo0 = umma_desc_lo(smem + kSmemV, kBox);
+            uint32_t ks = 0, kp = 0;                 // stage / phase of kv tile j in the K ring
+            uint32_t vs = 0, vp = 0, vs_prev = 0, vp_prev = 0;   // same for V, tiles j and j-1
             uint32_t q_use[2] = {0, 0}, c_p[2] = {0, 0}, free_use[2] = {0, 0};
             bool ok = true;
             for (int it = it_begin; it < it_end && ok; ++it) {
@@ -163,27 +171,22 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         ++q_use[t];
                         if (!ok) return;
                     }
+                    ok = wait(B_KFULL + ks, kp);
+                    if (!ok) return;
+                    tc_fence_after_sync();
                     const bool last_user = (t == 1) || (j >= n_t[1]);
                     const uint32_t d_s = tm + kTmS + t * TILE;
-                    uint32_t slot = ks, ph = kp;
+                    const uint32_t b_lo = k_lo0 + ks * (kKStage >> 4);
 #pragma unroll
-                    for (int c = 0; c < 3; ++c) {
-                        ok = wait(B_KFULL + slot, ph);
-                        if (!ok) return;
-                        tc_fence_after_sync();
-                        const uint32_t a_lo = q_lo[t] + c * (kBox >> 4);
-                        const uint32_t b_lo = k_lo0 + slot * (kBox >> 4);
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            umma_ss_w(d_s, a_lo + 2 * kk, hi_k, b_lo + 2 * kk, hi_k, idesc_s, (c | kk) != 0);
-                        if (last_user) umma_commit(bar(B_KEMPTY + slot));
-                        if (++slot == kKSlots) { slot = 0; ph ^= 1u; }
-                    }
-                    umma_commit(bar(B_SFULL + t));
-                    if (j == n_t[t] - 1) umma_commit(bar(B_QEMPTY + t));
+                    for (int kk = 0; kk < D_QK / 16; ++kk)
+                        umma2_ss_w(d_s, q_lo[t] + (kk >> 2) * (kBox >> 4) + (kk & 3) * 2, hi_k,
+                                   b_lo + (kk >> 2) * (kHalfBox >> 4) + (kk & 3) * 2, hi_k, idesc_s, kk != 0);
+                    if (last_user) umma2_commit(bar(B_KEMPTY + ks));
+                    umma2_commit(bar(B_SFULL + t));
+                    if (j == n_t[t] - 1) umma2_commit(bar(B_QEMPTY + t));
                 };
                 auto issue_pv = [&](int t, int j, uint32_t slot, uint32_t ph) {
-                    if (!(p.debug & 32)) ok = wait(B_PFULL + t, c_p[t]);
+                    ok = wait(B_PFULL + t, c_p[t]);
                     ++c_p[t];
                     if (!ok) return;
                     if (j == 0) {
@@ -191,22 +194,17 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         ++free_use[t];
                         if (!ok) return;
                     }
+                    ok = wait(B_VFULL + slot, ph);
+                    if (!ok) return;
+                    tc_fence_after_sync();
                     const bool last_user = (t == 1) || (j >= n_t[1]);
                     const uint32_t d_o = tm + kTmO + t * D_V, a_p = tm + kTmS + t * TILE;
+                    const uint32_t b_lo = v_lo0 + slot * (kVStage >> 4);
 #pragma unroll
-                    for (int hh = 0; hh < 2; ++hh) {
-                        ok = wait(B_VFULL + slot, ph);
-                        if (!ok) return;
-                        tc_fence_after_sync();
-                        const uint32_t b_lo = v_lo0 + slot * (kBox >> 4);
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            umma_ts_w(d_o, a_p + (hh * 4 + kk) * 8, b_lo + kk * (2048 >> 4), hi_v, idesc_o,
-                                      (j | hh | kk) != 0);
-                        if (last_user) umma_commit(bar(B_VEMPTY + slot));
-                        if (++slot == kVSlots) { slot = 0; ph ^= 1u; }
-                    }
-                    umma_commit(bar(B_OFULL + t));
+                    for (int kk = 0; kk < TILE / 16; ++kk)
+                        umma2_ts_w(d_o, a_p + kk * 8, b_lo + kk * (2048 >> 4), hi_v, idesc_o, (j | kk) != 0);
+                    if (last_user) umma2_commit(bar(B_VEMPTY + slot));
+                    umma2_commit(bar(B_OFULL + t));
                 };
 
                 for (int j = 0; j <= n && ok; ++j) {
@@ -216,8 +214,8 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     if (ok && j < n_t[0]) issue_pv(0, j, vs, vp);
                     if (j < n) {                     // step the ring cursors to kv tile j + 1
                         vs_prev = vs; vp_prev = vp;
-                        ks += 3; if (ks >= kKSlots) { ks -= kKSlots; kp ^= 1u; }
-                        vs += 2; if (vs >= kVSlots) { vs -= kVSlots; vp ^= 1u; }
+                        if (++ks == kKStages) { ks = 0; kp ^= 1u; }
+                        if (++vs == kVStages) { vs = 0; vp ^= 1u; }
                     }
                 }
             }
@@ -225,7 +223,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     } else {
         // ------------------------------------------------------------------ softmax warpgroups
         const int t = warp >> 2;                       // tile A or B
-        const int r = tid & 127;                       // row inside the tile = TMEM lane
+        const int r = tid & 127;                       // row inside this CTA's half of the tile = TMEM lane
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tm_s = tm + kTmS + t * TILE + lane_base;
         const uint32_t tm_o = tm + kTmO + t * D_V + lane_base;
@@ -235,7 +233,8 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             const FwdItem item = p.items[it];
             const PairDev pr = p.pairs[item.pair];
             const int n_kv = t == 0 ? item.n_a : item.n_b;
-            const int row = item.q0 + t * TILE + r;    // q row inside the pair
+            const int row0 = item.q0 + t * 2 * TILE + static_cast<int>(rank) * TILE;   // first row of this CTA
+            const int row = row0 + r;                  // q row inside the pair
             const bool row_valid = row < pr.q_len;
             const int64_t rows_total = pr.to_part ? p.part_rows : p.T;
             __nv_bfloat16* obase = static_cast<__nv_bfloat16*>(pr.to_part ? p.o_part : p.out);
@@ -258,17 +257,8 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 ++c_s;
                 if (!ok) break;
                 tc_fence_after_sync();
-                if (p.debug & 8) { tc_fence_before_sync(); mbar_arrive_warp(bar(B_PFULL + t)); ++c_o; l_run = 1.f; m_run = 0.f; continue; }
-                if (p.debug & 16) { uint32_t s[TILE];
-#pragma unroll
-                    for (int c0 = 0; c0 < TILE; c0 += 32) tmem_ld_x32(tm_s + c0, s + c0);
-                    tmem_wait_ld(); float acc = 0.f;
-#pragma unroll
-                    for (int c = 0; c < TILE; ++c) acc += __uint_as_float(s[c]);
-                    l_run += acc; m_run = 0.f; tc_fence_before_sync(); mbar_arrive_warp(bar(B_PFULL + t)); ++c_o; continue; }
                 const int col0 = j * TILE;
-                const bool need_mask = (col0 + TILE > pr.k_len) ||
-                                       (p.causal && (col0 + TILE - 1 > item.q0 + t * TILE + pr.off));
+                const bool need_mask = (col0 + TILE > pr.k_len) || (p.causal && (col0 + TILE - 1 > row0 + pr.off));
                 int cmax = TILE;                       // columns 0..cmax are visible
                 if (need_mask) {
                     int jmax = pr.k_len - 1;
@@ -333,7 +323,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 }
                 tmem_wait_st();
                 tc_fence_before_sync();
-                mbar_arrive_warp(bar(B_PFULL + t));
+                mbar_arrive_warp_leader(bar(B_PFULL + t));
                 ++c_o;
             }
             if (!ok) break;
@@ -349,7 +339,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 tmem_wait_ld();
                 if (c0 + 32 == D_V) {                  // every column has left TMEM: O may be overwritten
                     tc_fence_before_sync();
-                    mbar_arrive_warp(bar(B_OFREE + t));
+                    mbar_arrive_warp_leader(bar(B_OFREE + t));
                 }
                 if (row_valid) {
 #pragma unroll
@@ -372,6 +362,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     __syncwarp();
     tc_fence_before_sync();
     __syncthreads();
+    cluster_sync_all();                                // the leader's UMMAs read the peer's memories
     if (abort_flag) {
         // A wait ran out. Give copies still in flight time to land, then report and leave.
         const uint64_t t0 = global_timer_ns();
@@ -382,20 +373,34 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
         __syncthreads();
     }
-    if (warp == kWarpMma) tmem_dealloc(tm, kTmCols);
+    if (warp == kWarpMma) tmem_dealloc_pair(tm, kTmCols);
+}
+
+// Number of CTA pairs that can be resident at once (one CTA per SM): the size of the persistent grid.
+int fwd_max_clusters()
+{
+    static int cached = -1;
+    if (cached >= 0) return cached;
+    if (cudaFuncSetAttribute(hydra_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(fwd_smem_bytes())) != cudaSuccess)
+        return 0;
+    int sms = 0, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(sms / 2 * 2));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = fwd_smem_bytes();
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, hydra_fwd_kernel, &cfg) != cudaSuccess) n = 0;
+    cached = n;
+    return n;
 }
 
 cudaError_t launch_fwd(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                       const FwdParams& p, int grid, cudaStream_t stream)
+                       const FwdParams& p, int n_clusters, cudaStream_t stream)
 {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(hydra_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(fwd_smem_bytes()));
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
-    hydra_fwd_kernel<<<grid, kThreads, fwd_smem_bytes(), stream>>>(mq, mk, mv, p);
+    hydra_fwd_kernel<<<2 * n_clusters, kThreads, fwd_smem_bytes(), stream>>>(mq, mk, mv, p);
     return cudaGetLastError();
 }
 

@@ -73,7 +73,6 @@ struct FwdParams {
     float scale_log2;           // softmax_scale * log2(e)
     StatusBlock* status;
     uint64_t wait_limit_ns;
-    int32_t debug;
 };
 
 struct BwdParams {
@@ -103,6 +102,7 @@ struct MergeParams {
 };
 
 size_t fwd_smem_bytes();
+int fwd_max_clusters();
 size_t bwd_dq_smem_bytes();
 size_t bwd_dkv_smem_bytes();
 
