@@ -135,6 +135,34 @@ int32_t hydra_lse_merge(const void* o_part, const float* lse_part, int64_t part_
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * hydra_lse_merge for callers that must not allocate device memory. (No counterpart in the paper:
+ * this is a property of the library, not of the method.) It computes exactly what hydra_lse_merge
+ * computes, with the same kernel, but keeps the per-problem tables (the partials of every q chunk,
+ * cut into blocks of rows) in a fixed array inside the library image instead of in memory obtained
+ * with cudaMalloc, and it needs no workspace. It calls no cudaMalloc, cudaFree or other allocating
+ * routine. It is meant for processes that have handed all device memory to their own pool, and for
+ * latency-critical loops whose rules forbid cudaMalloc because it may synchronise the device.
+ *   - Limits (HYDRA_ERR_UNSUPPORTED beyond them): at most HYDRA_NOALLOC_MAX_GROUPS merged q chunks,
+ *     HYDRA_NOALLOC_MAX_PARTIALS partials in total, and HYDRA_NOALLOC_MAX_BLOCKS blocks of 8 rows
+ *     (sum over merged chunks of ceil(q_len / 8)). The array takes 608 KB on every GPU that loads
+ *     the library, until the process exits.
+ *   - The first call on a device looks up the array's device address with that device current; make
+ *     that first call before any stream capture begins.
+ *   - All calls on a device share the one array and each call rewrites the part it uses: calls
+ *     enqueued on the same stream are safe, calls whose kernels may overlap on the GPU (different
+ *     streams, no dependency) race. The tables are copied from ordinary host memory, so the call
+ *     waits for earlier work on `cuda_stream` before it returns.
+ *   Arguments as for hydra_lse_merge (pairs with part_row == -1 are ignored).
+ */
+#define HYDRA_NOALLOC_MAX_GROUPS 2048
+#define HYDRA_NOALLOC_MAX_PARTIALS 16384
+#define HYDRA_NOALLOC_MAX_BLOCKS 65536
+int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_part, int64_t part_rows,
+                                const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
+                                const hydra_pair_t* pairs, int32_t n_pairs, void* out, float* lse,
+                                void* cuda_stream);
+
+/*
  * Backward of the listed pairs, given the MERGED out and lse and the upstream gradient dout:
  *   D_i = <dout_i, out_i>;  P_ij = exp(s_ij - LSE_i);  dS_ij = P_ij (<dout_i, v_j> - D_i);
  *   dq_i = scale sum_j dS_ij k_j;  dk_j = scale sum_i dS_ij q_i;  dv_j = sum_i P_ij dout_i,

@@ -77,6 +77,8 @@ def _load() -> ctypes.CDLL:
     lib.hydra_profile_collect.argtypes = [vp, vp]
     lib.hydra_host_step_arena_bytes.restype = sz
     lib.hydra_host_step_arena_bytes.argtypes = [vp, i32, i32, vp, i32]
+    lib.hydra_lse_merge_noalloc.restype = i32
+    lib.hydra_lse_merge_noalloc.argtypes = [vp, vp, i64, vp, i32, i32, vp, i32, vp, vp, vp]
     lib.hydra_attn_fwd_bwd_host.restype = i32
     lib.hydra_attn_fwd_bwd_host.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp, i32, i32, f32, vp, vp, vp, vp,
                                             vp, vp, sz, vp]
@@ -89,7 +91,7 @@ EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_
            "hydra_shutdown", "hydra_usp_factor", "hydra_zigzag_pairs", "hydra_workspace_bytes",
            "hydra_attn_fwd", "hydra_lse_merge", "hydra_attn_bwd", "hydra_poll_status",
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
-           "hydra_attn_fwd_bwd_host")
+           "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc")
 KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq")
 
 
@@ -307,4 +309,19 @@ def hydra_attn_fwd_bwd_host(q_host, k_host, v_host, dout_host, cu_seqlens, n_hea
                                      int(arena_bytes), _stream(stream))
     if check:
         _check(s, "hydra_attn_fwd_bwd_host")
+    return s
+
+
+def hydra_lse_merge_noalloc(o_part, lse_part, part_rows: int, cu_seqlens, n_heads: int, pairs, out, lse,
+                            stream=None, check: bool = True) -> int:
+    """The merge for callers that must not allocate device memory (own memory pool, no-cudaMalloc
+    loops): same result as hydra_lse_merge, tables kept in a fixed array inside the library, no
+    workspace. Size limits apply (HYDRA_ERR_UNSUPPORTED beyond them); calls that may overlap on the
+    GPU race on that array; make the first call on a device before any stream capture."""
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    s = _lib.hydra_lse_merge_noalloc(_ptr(o_part), _ptr(lse_part), int(part_rows), cu.ctypes.data, len(cu) - 1,
+                                     n_heads, pp, npairs, _ptr(out), _ptr(lse), _stream(stream))
+    if check:
+        _check(s, "hydra_lse_merge_noalloc")
     return s

@@ -4,6 +4,8 @@
 // Both move every byte once with 16-byte accesses: 16 lanes own one (row, head) vector of 128 bf16.
 #include <cuda_bf16.h>
 
+#include <mutex>
+
 #include "hydra_internal.h"
 
 namespace hydra {
@@ -138,3 +140,135 @@ cudaError_t launch_bwd_prep(const void* dout, const void* out, float* dsum, int6
 }
 
 }  // namespace hydra
+
+// =============================================================================================
+// hydra_lse_merge_noalloc: the merge for callers that must not allocate device memory
+// =============================================================================================
+// hydra_lse_merge keeps its per-problem tables (which q chunk has which partials, cut into blocks of
+// rows) in device memory that the library obtains with cudaMalloc the first time it sees a problem.
+// Some callers cannot have that: a process that has handed all device memory to its own pool and
+// leaves nothing for cudaMalloc to find, or a latency-critical loop whose rules forbid cudaMalloc
+// because it may synchronise the whole device. This entry point runs the same kernel with the tables
+// in a fixed array that is part of the library image, so it calls no cudaMalloc, cudaFree or other
+// allocating routine. The price: a hard size limit, and one array per GPU shared by all calls.
+// The first call on a device looks up the array's device address (cudaGetSymbolAddress, with that
+// device current); make that first call before any stream capture begins.
+namespace hydra {
+namespace {
+
+constexpr int kNoAllocMaxGroups = HYDRA_NOALLOC_MAX_GROUPS;
+constexpr int kNoAllocMaxParts = HYDRA_NOALLOC_MAX_PARTIALS;
+constexpr int kNoAllocMaxItems = HYDRA_NOALLOC_MAX_BLOCKS;
+constexpr size_t kNoAllocGroupsBytes = sizeof(MergeGroup) * kNoAllocMaxGroups;
+constexpr size_t kNoAllocPartsBytes = sizeof(int32_t) * kNoAllocMaxParts;
+constexpr size_t kNoAllocItemsBytes = sizeof(MergeItem) * kNoAllocMaxItems;
+constexpr size_t kNoAllocBytes = kNoAllocGroupsBytes + kNoAllocPartsBytes + kNoAllocItemsBytes;   // 608 KB
+
+// Lives in every GPU context that loads the library, until the process exits. In host code this
+// name is only a handle for cudaGetSymbolAddress, never a pointer to pass to a kernel.
+static __device__ __align__(256) unsigned char g_noalloc_merge_tables[kNoAllocBytes];
+
+// Device address of the array on the current device (looked up once per device).
+cudaError_t noalloc_tables(unsigned char** out)
+{
+    static unsigned char* cached[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!cached[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_noalloc_merge_tables);
+        if (e != cudaSuccess) return e;
+        cached[dev] = static_cast<unsigned char*>(ptr);
+    }
+    *out = cached[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+}  // namespace hydra
+
+extern "C" int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_part, int64_t part_rows,
+                                           const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                                           const hydra_pair_t* pairs, int32_t n_pairs, void* out, float* lse,
+                                           void* cuda_stream)
+{
+    using namespace hydra;
+    if (n_seqs < 1 || !cu || n_heads < 1 || !pairs || n_pairs < 1 || part_rows < 1) return HYDRA_ERR_INVALID_ARG;
+    const void* ptrs[] = {o_part, lse_part, out, lse};
+    for (const void* p : ptrs)
+        if (!p || (reinterpret_cast<uintptr_t>(p) & 15u)) return HYDRA_ERR_INVALID_ARG;
+    if (cu[0] != 0) return HYDRA_ERR_INVALID_ARG;
+    for (int b = 0; b < n_seqs; ++b)
+        if (cu[b + 1] < cu[b]) return HYDRA_ERR_INVALID_ARG;
+
+    // tables in fixed-size host arrays (no heap use either): groups, part_row lists, row blocks;
+    // one set per process, so host-side table building is serialised
+    static std::mutex host_tables_mutex;
+    std::lock_guard<std::mutex> lock(host_tables_mutex);
+    static MergeGroup groups[kNoAllocMaxGroups];
+    static int32_t parts[kNoAllocMaxParts];
+    static MergeItem items[kNoAllocMaxItems];
+    int n_groups = 0, n_parts = 0, n_items = 0;
+    for (int i = 0; i < n_pairs;) {
+        int j = i;
+        while (j < n_pairs && pairs[j].group == pairs[i].group) ++j;
+        const hydra_pair_t& p = pairs[i];
+        if (p.seq < 0 || p.seq >= n_seqs || p.flags != 0 || p.q_start < 0 || p.q_len < 0 ||
+            int64_t{p.q_start} + p.q_len > int64_t{cu[p.seq + 1]} - cu[p.seq])
+            return HYDRA_ERR_INVALID_ARG;
+        if (i > 0 && p.group < pairs[i - 1].group) return HYDRA_ERR_INVALID_ARG;
+        if (p.part_row >= 0 && p.q_len > 0) {
+            if (n_groups >= kNoAllocMaxGroups) return HYDRA_ERR_UNSUPPORTED;
+            MergeGroup g;
+            g.out_tok0 = cu[p.seq] + p.q_start;
+            g.rows = p.q_len;
+            g.list_off = n_parts;
+            g.n_parts = j - i;
+            for (int t = i; t < j; ++t) {
+                const hydra_pair_t& q = pairs[t];
+                if (q.seq != p.seq || q.q_start != p.q_start || q.q_len != p.q_len || q.part_row < 0 ||
+                    int64_t{q.part_row} + q.q_len > part_rows)
+                    return HYDRA_ERR_INVALID_ARG;
+                if (n_parts >= kNoAllocMaxParts) return HYDRA_ERR_UNSUPPORTED;
+                parts[n_parts++] = q.part_row;
+            }
+            for (int32_t r = 0; r < g.rows; r += MERGE_ROWS) {
+                if (n_items >= kNoAllocMaxItems) return HYDRA_ERR_UNSUPPORTED;
+                items[n_items++] = MergeItem{n_groups, r};
+            }
+            groups[n_groups++] = g;
+        } else {
+            for (int t = i; t < j; ++t)
+                if (pairs[t].part_row >= 0 && pairs[t].q_len > 0) return HYDRA_ERR_INVALID_ARG;
+        }
+        i = j;
+    }
+    if (n_items == 0) return HYDRA_OK;
+
+    int major = 0, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+        return HYDRA_ERR_CUDA;
+    if (major != 10) return HYDRA_ERR_NOT_SM100;
+    unsigned char* tables = nullptr;
+    if (noalloc_tables(&tables) != cudaSuccess) return HYDRA_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // Every entry the kernel reads is overwritten here, so nothing of the previous call survives.
+    if (cudaMemcpyAsync(tables, groups, sizeof(MergeGroup) * n_groups, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(tables + kNoAllocGroupsBytes, parts, sizeof(int32_t) * n_parts, cudaMemcpyHostToDevice,
+                        stream) != cudaSuccess ||
+        cudaMemcpyAsync(tables + kNoAllocGroupsBytes + kNoAllocPartsBytes, items, sizeof(MergeItem) * n_items,
+                        cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return HYDRA_ERR_CUDA;
+    MergeParams mp{};
+    mp.groups = reinterpret_cast<const MergeGroup*>(tables);
+    mp.lists = reinterpret_cast<const int32_t*>(tables + kNoAllocGroupsBytes);
+    mp.items = reinterpret_cast<const MergeItem*>(tables + kNoAllocGroupsBytes + kNoAllocPartsBytes);
+    mp.n_items = n_items;
+    mp.o_part = o_part; mp.lse_part = lse_part; mp.out = out; mp.lse = lse;
+    mp.T = cu[n_seqs]; mp.part_rows = part_rows; mp.h = n_heads;
+    hydra_lse_merge_kernel<<<n_items, kThreads, 0, stream>>>(mp);
+    return cudaGetLastError() == cudaSuccess ? HYDRA_OK : HYDRA_ERR_CUDA;
+}
