@@ -9,11 +9,12 @@
 // tensor memory (A operand of a TS UMMA), and read Q / K / dO as MN-major B operands straight from
 // their token-major TMA tiles, so nothing is transposed in shared memory.
 //
-// Warp roles (320 threads) in both kernels:
+// Warp roles (352 threads) in both kernels:
 //   warps 0-3, 4-7  two elementwise warpgroups; thread r of each owns tile row r = TMEM lane r and
 //                   one half of the columns of S / dP
 //   warp 8          TMA producer (plus the LSE / D loads of the dK/dV kernel)
-//   warp 9          UMMA issuer (one thread), owner of the TMEM allocation
+//   warp 9          UMMA issuer of the score products (S, dP); owner of the TMEM allocation
+//   warp 10         UMMA issuer of the gradient updates (dQ, or dV and dK)
 // The elementwise threads copy S and dP to registers and release them at once, so that the UMMAs of
 // the next step run while the exponentials of this one are computed.
 #include <cuda_bf16.h>
@@ -25,8 +26,8 @@ namespace hydra {
 
 namespace {
 
-constexpr int kThreads = 320;
-constexpr int kWarpProd = 8, kWarpMma = 9;
+constexpr int kThreads = 352;
+constexpr int kWarpProd = 8, kWarpMma = 9, kWarpMma2 = 10;
 constexpr uint32_t kBox128 = 128 * 128;   // [128 rows x 64 bf16]
 constexpr uint32_t kBox64 = 64 * 128;     // [ 64 rows x 64 bf16]
 constexpr float kLog2e = 1.4426950408889634f;
@@ -59,8 +60,10 @@ constexpr uint32_t kK = kDO + 2 * kBox128;                   // 2 stages x 3 box
 constexpr uint32_t kV = kK + kKStages * 3 * kBox128;         // ring of 3 boxes [128 kv x 64 d_v]
 constexpr uint32_t kTotal = kV + kVSlots * kBox128;          // 229,376 B
 constexpr uint32_t kTmS = 0, kTmDP = 128, kTmDQ = 256, kTmDS = 448, kTmCols = 512;
-enum : int { B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_KEMPTY = 4, B_VFULL = 6, B_VEMPTY = 9,
-             B_SFULL = 12, B_SFREE = 13, B_PFULL = 14, B_DSFREE = 15, B_ACCFREE = 16, B_COUNT = 17 };
+// K-full is kept per 64-column box (3 per stage): S = Q K^T consumes the boxes in order, so it starts
+// when the first 16 KB have landed instead of waiting for all 48 KB of the stage.
+enum : int { B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_KEMPTY = 8, B_VFULL = 10, B_VEMPTY = 13,
+             B_SFULL = 16, B_SFREE = 17, B_PFULL = 18, B_DSFREE = 19, B_ACCFREE = 20, B_COUNT = 21 };
 
 // Iterator over (pair of the q chunk, kv tile) in the order every role walks them.
 struct TileIter {
@@ -211,10 +214,11 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     ok = wait(B_KEMPTY + st, (gk / kKStages) ^ 1u);
                     if (!ok) break;
                     ++gk;
-                    mbar_arrive_expect_tx(bar(B_KFULL + st), 3 * kBox128);
-                    for (int c = 0; c < 3; ++c)
-                        tma_load_3d(smem + kK + st * 3 * kBox128 + c * kBox128, &map_k, bar(B_KFULL + st),
+                    for (int c = 0; c < 3; ++c) {
+                        mbar_arrive_expect_tx(bar(B_KFULL + st * 3 + c), kBox128);
+                        tma_load_3d(smem + kK + st * 3 * kBox128 + c * kBox128, &map_k, bar(B_KFULL + st * 3 + c),
                                     c * 64, item.head, tok);
+                    }
                     for (int c = 0; c < 2 && ok; ++c, ++gv) {
                         const int slot = gv % kVSlots;
                         ok = wait(B_VEMPTY + slot, (gv / kVSlots) ^ 1u);
@@ -225,11 +229,11 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 }
             }
         }
-    } else if (warp == kWarpMma) {
-        // ------------------------------------------------------------------ UMMA issuer
-        // Two cursors walk the same (item, kv tile) sequence: `a` issues S = Q K^T and dP = dO V^T,
-        // `b` issues dQ += dS K and trails `a`. Neither blocks the other: each is issued as soon as
-        // its own operands are there (dQ first, because it frees a K stage), also across items.
+    } else if (warp == kWarpMma || warp == kWarpMma2) {
+        // ------------------------------------------------------------------ UMMA issuers
+        // Two issuing threads, so that neither kind of UMMA waits behind the other's operands:
+        // warp 9 issues S = Q K^T and dP = dO V^T of tile j+1 as soon as S/dP of tile j have been
+        // copied out and K, V have landed; warp 10 issues dQ += dS K of tile j as soon as dS is there.
         if (lane == 0) {
             constexpr uint32_t idesc_s = umma_idesc_bf16(TILE, TILE, false, false);
             constexpr uint32_t idesc_dq = umma_idesc_bf16(TILE, D_QK, false, true);
@@ -238,81 +242,41 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const uint32_t q_lo = umma_desc_lo(smem + kQ, 16), do_lo = umma_desc_lo(smem + kDO, 16);
             const uint32_t k_lo0 = umma_desc_lo(smem + kK, 16), v_lo0 = umma_desc_lo(smem + kV, 16);
             const uint32_t kmn_lo0 = umma_desc_lo(smem + kK, kBox128);
-
-            struct Cursor {
-                int it; TileIter ti; bool first;       // first: next tile is the first of its item
-            };
-            auto open_item = [&](Cursor& c) {            // position on the first tile of item c.it (or later)
-                while (c.it < it_end) {
-                    const GroupItem item = p.items[c.it];
-                    const int32_t* list = p.lists + item.list_off;
-                    const PairDev first = p.pairs[list[0]];
-                    c.ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
-                    if (c.ti.valid()) { c.first = true; return; }
-                    ++c.it;
-                }
-            };
-            Cursor a{it_begin, {}, true}, b{it_begin, {}, true};
-            open_item(a);
-            open_item(b);
-            uint32_t n_s = 0, n_q = 0;                   // tiles issued so far by each cursor
-            uint32_t items_a = 0, items_b = 0;           // items opened so far by each cursor
-            uint32_t gv = 0;
-            uint32_t got_a = 0, got_b = 0;               // operands already seen ready for the pending issue
-            uint32_t spins = 0;
-            long long t0 = 0;
+            const bool issue_scores = warp == kWarpMma;
+            uint32_t items = 0, n_tile = 0, gv = 0;       // running counts of this issuer
             bool ok = true;
-            auto ready = [&](uint32_t& got, uint32_t bit, int barrier, uint32_t parity) -> bool {
-                if (got & bit) return true;
-                if (mbar_test_wait(bar(barrier), parity & 1u)) { got |= bit; return true; }
-                return false;
-            };
-            while (ok && b.it < it_end) {
-                bool progressed = false;
-                // ---- dQ of tile n_q: needs dS from the elementwise warps; at the start of an item also
-                //      that the previous item's dQ has been read out of tensor memory
-                if (n_q < n_s) {
-                    bool r = ready(got_b, 1u, B_PFULL, n_q);
-                    if (r && b.first && items_b > 0) r = ready(got_b, 2u, B_ACCFREE, items_b - 1u);
-                    if (r) {
-                        tc_fence_after_sync();
-                        const int st = n_q % kKStages;
-                        const uint32_t k_lo = kmn_lo0 + st * (3 * kBox128 >> 4);
-                        const uint32_t acc0 = b.first ? 0u : 1u;
-#pragma unroll
-                        for (int kk = 0; kk < TILE / 16; ++kk)
-                            umma_ts_w(tm + kTmDQ, tm + kTmDS + kk * 8, k_lo + kk * (2048 >> 4), hi_kmn, idesc_dq,
-                                      kk > 0 ? 1u : acc0);
-                        umma_commit(bar(B_DSFREE));
-                        umma_commit(bar(B_KEMPTY + st));
-                        ++n_q;
-                        got_b = 0;
-                        if (b.first) { ++items_b; b.first = false; }
-                        b.ti.next();
-                        if (!b.ti.valid()) { ++b.it; open_item(b); }
-                        progressed = true;
-                    }
-                }
-                // ---- S and dP of tile n_s: needs S/dP of the previous tile copied out, K stage, two V
-                //      boxes, and at the start of an item Q and dO
-                if (a.it < it_end) {
-                    const int st = n_s % kKStages;
-                    bool r = (n_s == 0) || ready(got_a, 1u, B_SFREE, n_s - 1u);
-                    if (r && a.first) r = ready(got_a, 2u, B_QFULL, items_a);
-                    if (r) r = ready(got_a, 4u, B_KFULL + st, n_s / kKStages);
-                    if (r) r = ready(got_a, 8u, B_VFULL + gv % kVSlots, gv / kVSlots);
-                    if (r) r = ready(got_a, 16u, B_VFULL + (gv + 1) % kVSlots, (gv + 1) / kVSlots);
-                    if (r) {
-                        tc_fence_after_sync();
+            for (int it = it_begin; it < it_end && ok; ++it) {
+                const GroupItem item = p.items[it];
+                const int32_t* list = p.lists + item.list_off;
+                const PairDev first = p.pairs[list[0]];
+                TileIter ti;
+                ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+                if (!ti.valid()) continue;
+                if (issue_scores) {
+                    ok = wait(B_QFULL, items);
+                    for (; ti.valid() && ok;) {
+                        if (n_tile > 0) ok = wait(B_SFREE, n_tile - 1u);   // previous S / dP are in registers
+                        if (!ok) break;
+                        const int st = n_tile % kKStages;
                         const uint32_t k_lo = k_lo0 + st * (3 * kBox128 >> 4);
 #pragma unroll
-                        for (int kk = 0; kk < D_QK / 16; ++kk) {
-                            const uint32_t o = (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2;
-                            umma_ss_w(tm + kTmS, q_lo + o, hi_kmaj, k_lo + o, hi_kmaj, idesc_s, kk > 0);
+                        for (int c = 0; c < 3; ++c) {
+                            ok = wait(B_KFULL + st * 3 + c, n_tile / kKStages);
+                            if (!ok) break;
+                            tc_fence_after_sync();
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk) {
+                                const uint32_t o = c * (kBox128 >> 4) + kk * 2;
+                                umma_ss_w(tm + kTmS, q_lo + o, hi_kmaj, k_lo + o, hi_kmaj, idesc_s, (c | kk) != 0);
+                            }
                         }
+                        if (!ok) break;
 #pragma unroll
                         for (int c = 0; c < 2; ++c, ++gv) {
                             const int slot = gv % kVSlots;
+                            ok = wait(B_VFULL + slot, gv / kVSlots);
+                            if (!ok) break;
+                            tc_fence_after_sync();
                             const uint32_t v_lo = v_lo0 + slot * (kBox128 >> 4);
 #pragma unroll
                             for (int kk = 0; kk < 4; ++kk)
@@ -320,31 +284,32 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                                           hi_kmaj, idesc_s, (c | kk) != 0);
                             umma_commit(bar(B_VEMPTY + slot));
                         }
+                        if (!ok) break;
                         umma_commit(bar(B_SFULL));
-                        ++n_s;
-                        got_a = 0;
-                        if (a.first) { ++items_a; a.first = false; }
-                        a.ti.next();
-                        if (!a.ti.valid()) {                 // last tile of the item: Q and dO are free
-                            umma_commit(bar(B_QEMPTY));
-                            ++a.it;
-                            open_item(a);
-                        }
-                        progressed = true;
+                        ++n_tile;
+                        ti.next();
+                        if (!ti.valid()) umma_commit(bar(B_QEMPTY));     // Q and dO are no longer read
                     }
-                }
-                if (progressed) {
-                    spins = 0;
                 } else {
-                    // No sleep here: the shortest __nanosleep measured ~2000 cycles on this part, which
-                    // is a whole tile; the non-blocking tests above are cheap enough to spin on.
-                    if (++spins == 4096u) {
-                        t0 = clock64();
-                    } else if (spins > 4096u && (spins & 1023u) == 0u) {
-                        if (*abort_p) ok = false;
-                        else if (static_cast<uint64_t>(clock64() - t0) > 2ull * limit) { *abort_p = 1; ok = false; }
+                    bool first_tile = true;
+                    for (; ti.valid() && ok; ti.next()) {
+                        ok = wait(B_PFULL, n_tile);
+                        if (ok && first_tile && items > 0) ok = wait(B_ACCFREE, items - 1u);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        const int st = n_tile % kKStages;
+                        const uint32_t k_lo = kmn_lo0 + st * (3 * kBox128 >> 4);
+#pragma unroll
+                        for (int kk = 0; kk < TILE / 16; ++kk)
+                            umma_ts_w(tm + kTmDQ, tm + kTmDS + kk * 8, k_lo + kk * (2048 >> 4), hi_kmn, idesc_dq,
+                                      (kk > 0 || !first_tile) ? 1u : 0u);
+                        umma_commit(bar(B_DSFREE));
+                        umma_commit(bar(B_KEMPTY + st));
+                        ++n_tile;
+                        first_tile = false;
                     }
                 }
+                ++items;
             }
         }
     } else {
@@ -547,8 +512,11 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 mbar_arrive_warp(bar(B_STAT + st));
             }
         }
-    } else if (warp == kWarpMma) {
-        // ------------------------------------------------------------------ UMMA issuer
+    } else if (warp == kWarpMma || warp == kWarpMma2) {
+        // ------------------------------------------------------------------ UMMA issuers
+        // warp 9 issues S^T = K Q^T and dP^T = V dO^T of sub-tile u+1 as soon as those of sub-tile u
+        // have been copied out; warp 10 issues dV += P^T dO and dK += dS^T Q of sub-tile u as soon
+        // as P and dS are in tensor memory. Neither waits behind the other's operands.
         if (lane == 0) {
             constexpr uint32_t idesc_st = umma_idesc_bf16(TILE, SUB, false, false);
             constexpr uint32_t idesc_dv = umma_idesc_bf16(TILE, D_V, false, true);
@@ -558,7 +526,8 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const uint32_t k_lo = umma_desc_lo(smem + kK, 16), v_lo = umma_desc_lo(smem + kV, 16);
             const uint32_t q_lo0 = umma_desc_lo(smem + kQ, 16), do_lo0 = umma_desc_lo(smem + kDO, 16);
             const uint32_t qmn_lo0 = umma_desc_lo(smem + kQ, kBox64), domn_lo0 = umma_desc_lo(smem + kDO, kBox64);
-            uint32_t items = 0, c_s = 0, c_p = 0, gq_s = 0, gq_a = 0;
+            const bool issue_scores = warp == kWarpMma;
+            uint32_t items = 0, n_step = 0;
             bool ok = true;
             for (int it = it_begin; it < it_end && ok; ++it) {
                 const GroupItem item = p.items[it];
@@ -566,58 +535,52 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 SubIter si;
                 si.init(p.pairs, list, item.list_len, item.r0, p.causal);
                 if (!si.valid()) continue;
-                int n_steps = 0;
-                for (SubIter c = si; c.valid(); c.next()) ++n_steps;
-
-                auto issue_s_dp = [&](bool last) {
-                    if (c_s > 0) ok = wait(B_SFREE, c_s - 1u);
-                    if (!ok) return;
-                    const int st = gq_s % kStages;
-                    ok = wait(B_QFULL + st, gq_s / kStages);
-                    ++gq_s;
-                    if (!ok) return;
-                    tc_fence_after_sync();
-                    const uint32_t q_lo = q_lo0 + st * (3 * kBox64 >> 4), do_lo = do_lo0 + st * (2 * kBox64 >> 4);
+                if (issue_scores) {
+                    ok = wait(B_KVFULL, items);
+                    for (; si.valid() && ok;) {
+                        if (n_step > 0) ok = wait(B_SFREE, n_step - 1u);
+                        if (!ok) break;
+                        const int st = n_step % kStages;
+                        ok = wait(B_QFULL + st, n_step / kStages);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        const uint32_t q_lo = q_lo0 + st * (3 * kBox64 >> 4), do_lo = do_lo0 + st * (2 * kBox64 >> 4);
 #pragma unroll
-                    for (int kk = 0; kk < D_QK / 16; ++kk)
-                        umma_ss_w(tm + kTmS, k_lo + (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2, hi_kmaj,
-                                  q_lo + (kk >> 2) * (kBox64 >> 4) + (kk & 3) * 2, hi_kmaj, idesc_st, kk > 0);
+                        for (int kk = 0; kk < D_QK / 16; ++kk)
+                            umma_ss_w(tm + kTmS, k_lo + (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2, hi_kmaj,
+                                      q_lo + (kk >> 2) * (kBox64 >> 4) + (kk & 3) * 2, hi_kmaj, idesc_st, kk > 0);
 #pragma unroll
-                    for (int kk = 0; kk < D_V / 16; ++kk)
-                        umma_ss_w(tm + kTmDP, v_lo + (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2, hi_kmaj,
-                                  do_lo + (kk >> 2) * (kBox64 >> 4) + (kk & 3) * 2, hi_kmaj, idesc_st, kk > 0);
-                    umma_commit(bar(B_SFULL));
-                    ++c_s;
-                    if (last) umma_commit(bar(B_KVEMPTY));           // K and V are no longer read
-                };
-                auto issue_acc = [&](int i) {
-                    ok = wait(B_PFULL, c_p);
-                    ++c_p;
-                    if (!ok) return;
-                    if (i == 0 && items > 0) ok = wait(B_ACCFREE, items - 1u);
-                    if (!ok) return;
-                    tc_fence_after_sync();
-                    const int st = gq_a % kStages;
-                    ++gq_a;
-                    const uint32_t do_lo = domn_lo0 + st * (2 * kBox64 >> 4), q_lo = qmn_lo0 + st * (3 * kBox64 >> 4);
+                        for (int kk = 0; kk < D_V / 16; ++kk)
+                            umma_ss_w(tm + kTmDP, v_lo + (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2, hi_kmaj,
+                                      do_lo + (kk >> 2) * (kBox64 >> 4) + (kk & 3) * 2, hi_kmaj, idesc_st, kk > 0);
+                        umma_commit(bar(B_SFULL));
+                        ++n_step;
+                        si.next();
+                        if (!si.valid()) umma_commit(bar(B_KVEMPTY));    // K and V are no longer read
+                    }
+                } else {
+                    bool first_step = true;
+                    for (; si.valid() && ok; si.next()) {
+                        ok = wait(B_PFULL, n_step);
+                        if (ok && first_step && items > 0) ok = wait(B_ACCFREE, items - 1u);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        const int st = n_step % kStages;
+                        const uint32_t do_lo = domn_lo0 + st * (2 * kBox64 >> 4), q_lo = qmn_lo0 + st * (3 * kBox64 >> 4);
+                        const uint32_t acc = first_step ? 0u : 1u;
 #pragma unroll
-                    for (int kk = 0; kk < SUB / 16; ++kk)
-                        umma_ts_w(tm + kTmDV, tm + kTmP + kk * 8, do_lo + kk * (2048 >> 4), hi_mn, idesc_dv,
-                                  (i | kk) != 0);
+                        for (int kk = 0; kk < SUB / 16; ++kk)
+                            umma_ts_w(tm + kTmDV, tm + kTmP + kk * 8, do_lo + kk * (2048 >> 4), hi_mn, idesc_dv,
+                                      kk > 0 ? 1u : acc);
 #pragma unroll
-                    for (int kk = 0; kk < SUB / 16; ++kk)
-                        umma_ts_w(tm + kTmDK, tm + kTmDS + kk * 8, q_lo + kk * (2048 >> 4), hi_mn, idesc_dk,
-                                  (i | kk) != 0);
-                    umma_commit(bar(B_PDSFREE));
-                    umma_commit(bar(B_QEMPTY + st));
-                };
-
-                ok = wait(B_KVFULL, items);
-                if (!ok) break;
-                issue_s_dp(n_steps == 1);
-                for (int i = 0; i < n_steps && ok; ++i) {
-                    if (i + 1 < n_steps) issue_s_dp(i + 2 == n_steps);
-                    if (ok) issue_acc(i);
+                        for (int kk = 0; kk < SUB / 16; ++kk)
+                            umma_ts_w(tm + kTmDK, tm + kTmDS + kk * 8, q_lo + kk * (2048 >> 4), hi_mn, idesc_dk,
+                                      kk > 0 ? 1u : acc);
+                        umma_commit(bar(B_PDSFREE));
+                        umma_commit(bar(B_QEMPTY + st));
+                        ++n_step;
+                        first_step = false;
+                    }
                 }
                 ++items;
             }
