@@ -63,7 +63,7 @@ constexpr uint32_t kTmS = 0, kTmDP = 128, kTmDQ = 256, kTmDS = 448, kTmCols = 51
 // K-full is kept per 64-column box (3 per stage): S = Q K^T consumes the boxes in order, so it starts
 // when the first 16 KB have landed instead of waiting for all 48 KB of the stage.
 enum : int { B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_KEMPTY = 8, B_VFULL = 10, B_VEMPTY = 13,
-             B_SFULL = 16, B_SFREE = 17, B_PFULL = 18, B_DSFREE = 19, B_ACCFREE = 20, B_COUNT = 21 };
+             B_SFULL = 16, B_SFREE = 17, B_PFULL = 18, B_DSFREE = 20, B_ACCFREE = 21, B_COUNT = 22 };
 
 // Iterator over (pair of the q chunk, kv tile) in the order every role walks them.
 struct TileIter {
@@ -155,7 +155,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     if (tid == 0) {
         abort_flag = 0;
         for (int i = 0; i < B_COUNT; ++i) {
-            const bool by_threads = (i == B_SFREE) || (i == B_PFULL) || (i == B_ACCFREE);
+            const bool by_threads = (i == B_SFREE) || (i == B_PFULL) || (i == B_PFULL + 1) || (i == B_ACCFREE);
             mbar_init(bar(i), by_threads ? 8u : 1u);   // 8 = elementwise warps
         }
         fence_mbar_init();
@@ -194,22 +194,18 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 for (int c = 0; c < 2; ++c)
                     tma_load_3d(smem + kDO + c * kBox128, &map_do, bar(B_QFULL), c * 64, item.head,
                                 first.q_tok0 + item.r0);
-                // L2 prefetch runs kPrefetch tiles ahead of the loads: a stage frees late (K is read by S
-                // and again by the dQ update), so the load itself must not pay the HBM latency
-                constexpr int kPrefetch = 4;
-                TileIter pf = ti;
-                auto prefetch_tile = [&]() {
-                    if (!pf.valid()) return;
-                    const int ptok = pf.cur.k_tok0 + pf.t * TILE;
-                    for (int c = 0; c < 3; ++c) tma_prefetch_l2_3d(&map_k, c * 64, item.head, ptok);
-                    for (int c = 0; c < 2; ++c) tma_prefetch_l2_3d(&map_v, c * 64, item.head, ptok);
-                    pf.next();
-                };
-                pf.next();
-                for (int a = 0; a < kPrefetch; ++a) prefetch_tile();
                 for (; ti.valid() && ok; ti.next()) {
-                    prefetch_tile();
                     const int tok = ti.cur.k_tok0 + ti.t * TILE;
+                    // V first: its slots were freed a whole tile ago and dP is the first product of the
+                    // tile; the K stage frees only when the dQ update two tiles back has completed
+                    for (int c = 0; c < 2 && ok; ++c, ++gv) {
+                        const int slot = gv % kVSlots;
+                        ok = wait(B_VEMPTY + slot, (gv / kVSlots) ^ 1u);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(bar(B_VFULL + slot), kBox128);
+                        tma_load_3d(smem + kV + slot * kBox128, &map_v, bar(B_VFULL + slot), c * 64, item.head, tok);
+                    }
+                    if (!ok) break;
                     const int st = gk % kKStages;
                     ok = wait(B_KEMPTY + st, (gk / kKStages) ^ 1u);
                     if (!ok) break;
@@ -218,13 +214,6 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                         mbar_arrive_expect_tx(bar(B_KFULL + st * 3 + c), kBox128);
                         tma_load_3d(smem + kK + st * 3 * kBox128 + c * kBox128, &map_k, bar(B_KFULL + st * 3 + c),
                                     c * 64, item.head, tok);
-                    }
-                    for (int c = 0; c < 2 && ok; ++c, ++gv) {
-                        const int slot = gv % kVSlots;
-                        ok = wait(B_VEMPTY + slot, (gv / kVSlots) ^ 1u);
-                        if (!ok) break;
-                        mbar_arrive_expect_tx(bar(B_VFULL + slot), kBox128);
-                        tma_load_3d(smem + kV + slot * kBox128, &map_v, bar(B_VFULL + slot), c * 64, item.head, tok);
                     }
                 }
             }
@@ -257,20 +246,8 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     for (; ti.valid() && ok;) {
                         if (n_tile > 0) ok = wait(B_SFREE, n_tile - 1u);   // previous S / dP are in registers
                         if (!ok) break;
-                        const int st = n_tile % kKStages;
-                        const uint32_t k_lo = k_lo0 + st * (3 * kBox128 >> 4);
-#pragma unroll
-                        for (int c = 0; c < 3; ++c) {
-                            ok = wait(B_KFULL + st * 3 + c, n_tile / kKStages);
-                            if (!ok) break;
-                            tc_fence_after_sync();
-#pragma unroll
-                            for (int kk = 0; kk < 4; ++kk) {
-                                const uint32_t o = c * (kBox128 >> 4) + kk * 2;
-                                umma_ss_w(tm + kTmS, q_lo + o, hi_kmaj, k_lo + o, hi_kmaj, idesc_s, (c | kk) != 0);
-                            }
-                        }
-                        if (!ok) break;
+                        // dP first: V was loaded a whole tile ago, while the K stage of this tile was
+                        // freed only by the dQ update two tiles back and may still be landing
 #pragma unroll
                         for (int c = 0; c < 2; ++c, ++gv) {
                             const int slot = gv % kVSlots;
@@ -285,6 +262,20 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                             umma_commit(bar(B_VEMPTY + slot));
                         }
                         if (!ok) break;
+                        const int st = n_tile % kKStages;
+                        const uint32_t k_lo = k_lo0 + st * (3 * kBox128 >> 4);
+#pragma unroll
+                        for (int c = 0; c < 3; ++c) {
+                            ok = wait(B_KFULL + st * 3 + c, n_tile / kKStages);
+                            if (!ok) break;
+                            tc_fence_after_sync();
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk) {
+                                const uint32_t o = c * (kBox128 >> 4) + kk * 2;
+                                umma_ss_w(tm + kTmS, q_lo + o, hi_kmaj, k_lo + o, hi_kmaj, idesc_s, (c | kk) != 0);
+                            }
+                        }
+                        if (!ok) break;
                         umma_commit(bar(B_SFULL));
                         ++n_tile;
                         ti.next();
@@ -293,16 +284,25 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 } else {
                     bool first_tile = true;
                     for (; ti.valid() && ok; ti.next()) {
-                        ok = wait(B_PFULL, n_tile);
-                        if (ok && first_tile && items > 0) ok = wait(B_ACCFREE, items - 1u);
-                        if (!ok) break;
-                        tc_fence_after_sync();
+                        // dS arrives in two instalments: columns [0,32) of each half (K-steps 0,1,4,5),
+                        // then columns [32,64) (K-steps 2,3,6,7); the update of the first overlaps the
+                        // exponentials of the second
                         const int st = n_tile % kKStages;
                         const uint32_t k_lo = kmn_lo0 + st * (3 * kBox128 >> 4);
 #pragma unroll
-                        for (int kk = 0; kk < TILE / 16; ++kk)
-                            umma_ts_w(tm + kTmDQ, tm + kTmDS + kk * 8, k_lo + kk * (2048 >> 4), hi_kmn, idesc_dq,
-                                      (kk > 0 || !first_tile) ? 1u : 0u);
+                        for (int half = 0; half < 2; ++half) {
+                            ok = wait(B_PFULL + half, n_tile);
+                            if (ok && half == 0 && first_tile && items > 0) ok = wait(B_ACCFREE, items - 1u);
+                            if (!ok) break;
+                            tc_fence_after_sync();
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const int kk = (e >> 1) * 4 + half * 2 + (e & 1);
+                                umma_ts_w(tm + kTmDQ, tm + kTmDS + kk * 8, k_lo + kk * (2048 >> 4), hi_kmn, idesc_dq,
+                                          (half > 0 || e > 0 || !first_tile) ? 1u : 0u);
+                            }
+                        }
+                        if (!ok) break;
                         umma_commit(bar(B_DSFREE));
                         umma_commit(bar(B_KEMPTY + st));
                         ++n_tile;
@@ -359,29 +359,37 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 }
                 tmem_wait_ld();
                 tc_fence_before_sync();
-                mbar_arrive_warp(bar(B_SFREE));             // the next S / dP may overwrite tensor memory
+                // the next S / dP may overwrite tensor memory; the arrival must not sink below the arithmetic
+                const float lse2_t = mbar_arrive_warp_before(bar(B_SFREE), lse2);
                 int jmax = ti.cur.k_len - 1;
                 if (p.causal) jmax = min(jmax, row + ti.cur.off);
                 const int cmax = jmax - ti.t * TILE - g * 64;      // columns 0..cmax of this half are visible
                 uint32_t ds[32];
+                float lse2_h = lse2_t;
 #pragma unroll
-                for (int c = 0; c < 64; c += 2) {
-                    float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2));
-                    float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2));
-                    if (c > cmax) p0 = 0.f;
-                    if (c + 1 > cmax) p1 = 0.f;
-                    ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum),
-                                             p1 * (__uint_as_float(dp[c + 1]) - dsum));
+                for (int half = 0; half < 2; ++half) {
+#pragma unroll
+                    for (int c = half * 32; c < half * 32 + 32; c += 2) {
+                        float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2_h));
+                        float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2_h));
+                        if (c > cmax) p0 = 0.f;
+                        if (c + 1 > cmax) p1 = 0.f;
+                        ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum),
+                                                 p1 * (__uint_as_float(dp[c + 1]) - dsum));
+                    }
+                    if (half == 0 && c_ds > 0) {           // the previous dQ update has read dS
+                        ok = wait(B_DSFREE, c_ds - 1u);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                    }
+                    tmem_st_x16(tm_ds + half * 16, ds + half * 16);
+                    tmem_wait_st();
+                    tc_fence_before_sync();
+                    // first instalment: its arrival must not sink below the second half's arithmetic
+                    if (half == 0) lse2_h = mbar_arrive_warp_before(bar(B_PFULL), lse2_h);
+                    else mbar_arrive_warp(bar(B_PFULL + 1));
                 }
-                if (c_ds > 0) {                        // the previous dQ update has read dS
-                    ok = wait(B_DSFREE, c_ds - 1u);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                }
-                tmem_st_x32(tm_ds, ds);
-                tmem_wait_st();
-                tc_fence_before_sync();
-                mbar_arrive_warp(bar(B_PFULL));
+                if (!ok) break;
                 ++c_ds;
             }
             if (!ok) break;

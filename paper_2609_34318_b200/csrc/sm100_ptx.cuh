@@ -320,6 +320,28 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return r;
 }
 
+// One arrival per warp that is issued BEFORE the arithmetic that follows it. An arrival has no
+// consumer, so the instruction scheduler is free to sink it to the end of a long block of pure
+// arithmetic, which delays the signal by the length of that block (measured: more than 1000 cycles
+// per tile). Returning `x` through a value derived from the arrival's state token (x + 0 * bit)
+// makes everything computed from the returned value wait for the arrival to have been issued.
+__device__ __forceinline__ float mbar_arrive_warp_before(uint32_t bar, float x) {
+    __syncwarp();
+    uint64_t state = 0;
+    if ((threadIdx.x & 31u) == 0u)
+        asm volatile("mbarrier.arrive.shared::cta.b64 %0, [%1];" : "=l"(state) : "r"(bar) : "memory");
+    float bit;
+    asm volatile(
+        "{\n\t.reg .b32 lo, hi;\n\t"
+        "mov.b64 {lo, hi}, %1;\n\t"
+        "and.b32 lo, lo, 1;\n\t"
+        "cvt.rn.f32.u32 %0, lo;\n\t}"
+        : "=f"(bit)
+        : "l"(state));
+    asm volatile("fma.rn.f32 %0, %1, 0f00000000, %0;" : "+f"(x) : "f"(bit));
+    return x;
+}
+
 }  // namespace hydra
 
 // ----------------------------------------------------------------------------------------------
