@@ -443,12 +443,14 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     __shared__ int abort_flag;
     __shared__ float s_lse2[kStages][SUB];
     __shared__ float s_dsum[kStages][SUB];
+    __shared__ uint32_t s_bursts;                      // S / dP bursts issued so far (all ones: no more)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t bar0 = smem_u32(&bars[0]);
     auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
     if (tid == 0) {
         abort_flag = 0;
+        s_bursts = 0u;
         for (int i = 0; i < B_COUNT; ++i) {
             uint32_t count = 1u;
             if (i == B_SFREE || i == B_PFULL || i == B_ACCFREE) count = 8u;   // elementwise warps
@@ -468,6 +470,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const int it_begin = p.cta_off[blockIdx.x], it_end = p.cta_off[blockIdx.x + 1];
     volatile int* abort_p = &abort_flag;
     auto wait = [&](int b, uint32_t parity) -> bool { return mbar_wait(bar(b), parity & 1u, abort_p, limit); };
+    volatile uint32_t* bursts_p = &s_bursts;
 
     if (warp == kWarpProd) {
         // ------------------------------------------------------------------ TMA producer + LSE / D
@@ -563,6 +566,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                                       do_lo + (kk >> 2) * (kBox64 >> 4) + (kk & 3) * 2, hi_kmaj, idesc_st, kk > 0);
                         umma_commit(bar(B_SFULL));
                         ++n_step;
+                        *bursts_p = n_step;
                         si.next();
                         if (!si.valid()) umma_commit(bar(B_KVEMPTY));    // K and V are no longer read
                     }
@@ -571,6 +575,13 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     for (; si.valid() && ok; si.next()) {
                         ok = wait(B_PFULL, n_step);
                         if (ok && first_step && items > 0) ok = wait(B_ACCFREE, items - 1u);
+                        // Order hint, not a data dependency: let the score products of the NEXT sub-tile of
+                        // this item enter the tensor pipe first. They are what the elementwise warps wait
+                        // for next; these updates then fill the gap in which S / dP are copied out,
+                        // instead of interleaving with the score products and delaying them.
+                        SubIter peek = si;
+                        peek.next();
+                        if (ok && peek.valid()) ok = counter_wait(bursts_p, n_step + 2u, abort_p, limit);
                         if (!ok) break;
                         tc_fence_after_sync();
                         const int st = n_step % kStages;
@@ -592,6 +603,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 }
                 ++items;
             }
+            if (issue_scores) *bursts_p = 0xffffffffu;         // nothing more to wait for
         }
     } else {
         // ------------------------------------------------------------------ elementwise warpgroups

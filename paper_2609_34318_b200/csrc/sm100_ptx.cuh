@@ -99,6 +99,29 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return true;
 }
 
+// Bounded wait until a counter in shared memory, written by another warp of the CTA, reaches
+// `target`. Used where only the ORDER of two warps' instruction streams matters (no data is handed
+// over), so a plain volatile word is enough; barrier phases would alias if the writer ran two steps
+// ahead.
+__device__ __forceinline__ bool counter_wait(const volatile uint32_t* counter, uint32_t target,
+                                             volatile int* abort_flag, uint64_t limit_ns) {
+    uint32_t spins = 0;
+    long long t0 = 0;
+    while (*counter < target) {
+        ++spins;
+        if (spins == 256u) {
+            t0 = clock64();
+        } else if (spins > 256u && (spins & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if (static_cast<uint64_t>(clock64() - t0) > 2ull * limit_ns) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
 // ----------------------------------------------------------------------------------------------
 // TMA: tiled loads of a box into shared memory, completion counted in bytes on an mbarrier
 // ----------------------------------------------------------------------------------------------
