@@ -63,7 +63,8 @@ constexpr uint32_t kTmS = 0, kTmDP = 128, kTmDQ = 256, kTmDS = 448, kTmCols = 51
 // K-full is kept per 64-column box (3 per stage): S = Q K^T consumes the boxes in order, so it starts
 // when the first 16 KB have landed instead of waiting for all 48 KB of the stage.
 enum : int { B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_KEMPTY = 8, B_VFULL = 10, B_VEMPTY = 13,
-             B_SFULL = 16, B_SFREE = 17, B_PFULL = 18, B_DSFREE = 20, B_ACCFREE = 21, B_COUNT = 22 };
+             B_SFULL = 16, B_SFREE = 17, B_PFULL = 18, B_DSFREE = 20, B_ACCFREE = 21, B_DPFULL = 22, B_DPFREE = 23,
+             B_COUNT = 24 };
 
 // Iterator over (pair of the q chunk, kv tile) in the order every role walks them.
 struct TileIter {
@@ -155,7 +156,8 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     if (tid == 0) {
         abort_flag = 0;
         for (int i = 0; i < B_COUNT; ++i) {
-            const bool by_threads = (i == B_SFREE) || (i == B_PFULL) || (i == B_PFULL + 1) || (i == B_ACCFREE);
+            const bool by_threads = (i == B_SFREE) || (i == B_DPFREE) || (i == B_PFULL) || (i == B_PFULL + 1) ||
+                                    (i == B_ACCFREE);
             mbar_init(bar(i), by_threads ? 8u : 1u);   // 8 = elementwise warps
         }
         fence_mbar_init();
@@ -244,10 +246,13 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 if (issue_scores) {
                     ok = wait(B_QFULL, items);
                     for (; ti.valid() && ok;) {
-                        if (n_tile > 0) ok = wait(B_SFREE, n_tile - 1u);   // previous S / dP are in registers
+                        // dP and S are handed over separately. dP comes first (V was loaded a whole tile
+                        // ago, while the K stage of this tile was freed only by the dQ update two tiles
+                        // back and may still be landing); the elementwise warps copy it out while S is
+                        // still being computed, so the dP of the next tile can follow this S at once and
+                        // fills the time in which S is copied out.
+                        if (n_tile > 0) ok = wait(B_DPFREE, n_tile - 1u);  // previous dP is in registers
                         if (!ok) break;
-                        // dP first: V was loaded a whole tile ago, while the K stage of this tile was
-                        // freed only by the dQ update two tiles back and may still be landing
 #pragma unroll
                         for (int c = 0; c < 2; ++c, ++gv) {
                             const int slot = gv % kVSlots;
@@ -261,6 +266,9 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                                           hi_kmaj, idesc_s, (c | kk) != 0);
                             umma_commit(bar(B_VEMPTY + slot));
                         }
+                        if (!ok) break;
+                        umma_commit(bar(B_DPFULL));
+                        if (n_tile > 0) ok = wait(B_SFREE, n_tile - 1u);   // previous S is in registers
                         if (!ok) break;
                         const int st = n_tile % kKStages;
                         const uint32_t k_lo = k_lo0 + st * (3 * kBox128 >> 4);
@@ -347,35 +355,52 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 dsum = p.dsum[static_cast<int64_t>(item.head) * p.T + first.q_tok0 + row];
             }
             for (; ti.valid() && ok; ti.next()) {
+                uint32_t s[64], dp[64];
+                ok = wait(B_DPFULL, c_s);
+                if (!ok) break;
+                tc_fence_after_sync();
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 32) tmem_ld_x32(tm_dp + c0, dp + c0);
+                tmem_wait_ld();
+                tc_fence_before_sync();
+                mbar_arrive_warp(bar(B_DPFREE));            // the next dP may overwrite tensor memory
                 ok = wait(B_SFULL, c_s);
                 ++c_s;
                 if (!ok) break;
                 tc_fence_after_sync();
-                uint32_t s[64], dp[64];
 #pragma unroll
-                for (int c0 = 0; c0 < 64; c0 += 32) {
-                    tmem_ld_x32(tm_s + c0, s + c0);
-                    tmem_ld_x32(tm_dp + c0, dp + c0);
-                }
+                for (int c0 = 0; c0 < 64; c0 += 32) tmem_ld_x32(tm_s + c0, s + c0);
                 tmem_wait_ld();
                 tc_fence_before_sync();
-                // the next S / dP may overwrite tensor memory; the arrival must not sink below the arithmetic
+                // the next S may overwrite tensor memory; the arrival must not sink below the arithmetic
                 const float lse2_t = mbar_arrive_warp_before(bar(B_SFREE), lse2);
                 int jmax = ti.cur.k_len - 1;
                 if (p.causal) jmax = min(jmax, row + ti.cur.off);
                 const int cmax = jmax - ti.t * TILE - g * 64;      // columns 0..cmax of this half are visible
                 uint32_t ds[32];
                 float lse2_h = lse2_t;
+                // interior tiles (every column visible to every row of the warp) skip the masking
+                const bool masked = __any_sync(0xffffffffu, cmax < 63);
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
+                    if (masked) {
 #pragma unroll
-                    for (int c = half * 32; c < half * 32 + 32; c += 2) {
-                        float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2_h));
-                        float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2_h));
-                        if (c > cmax) p0 = 0.f;
-                        if (c + 1 > cmax) p1 = 0.f;
-                        ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum),
-                                                 p1 * (__uint_as_float(dp[c + 1]) - dsum));
+                        for (int c = half * 32; c < half * 32 + 32; c += 2) {
+                            float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2_h));
+                            float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2_h));
+                            if (c > cmax) p0 = 0.f;
+                            if (c + 1 > cmax) p1 = 0.f;
+                            ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum),
+                                                     p1 * (__uint_as_float(dp[c + 1]) - dsum));
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = half * 32; c < half * 32 + 32; c += 2) {
+                            const float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2_h));
+                            const float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2_h));
+                            ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum),
+                                                     p1 * (__uint_as_float(dp[c + 1]) - dsum));
+                        }
                     }
                     if (half == 0 && c_ds > 0) {           // the previous dQ update has read dS
                         ok = wait(B_DSFREE, c_ds - 1u);
@@ -661,15 +686,27 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 const float* lse2 = &s_lse2[st][g * 32];
                 const float* dsum = &s_dsum[st][g * 32];
                 uint32_t pk[16], ds[16];
+                // interior sub-tiles (every q row visible from every kv row of the warp) skip the masking
+                if (__any_sync(0xffffffffu, c_lo > 0 || c_hi < 32)) {
 #pragma unroll
-                for (int c = 0; c < 32; c += 2) {
-                    float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2[c]));
-                    float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2[c + 1]));
-                    if (c < c_lo || c >= c_hi) p0 = 0.f;
-                    if (c + 1 < c_lo || c + 1 >= c_hi) p1 = 0.f;
-                    pk[c >> 1] = pack_bf16x2(p0, p1);
-                    ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum[c]),
-                                             p1 * (__uint_as_float(dp[c + 1]) - dsum[c + 1]));
+                    for (int c = 0; c < 32; c += 2) {
+                        float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2[c]));
+                        float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2[c + 1]));
+                        if (c < c_lo || c >= c_hi) p0 = 0.f;
+                        if (c + 1 < c_lo || c + 1 >= c_hi) p1 = 0.f;
+                        pk[c >> 1] = pack_bf16x2(p0, p1);
+                        ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum[c]),
+                                                 p1 * (__uint_as_float(dp[c + 1]) - dsum[c + 1]));
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 32; c += 2) {
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2[c]));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2[c + 1]));
+                        pk[c >> 1] = pack_bf16x2(p0, p1);
+                        ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum[c]),
+                                                 p1 * (__uint_as_float(dp[c + 1]) - dsum[c + 1]));
+                    }
                 }
                 if (c_pds > 0) {                       // the previous dV / dK updates have read P and dS
                     ok = wait(B_PDSFREE, c_pds - 1u);
