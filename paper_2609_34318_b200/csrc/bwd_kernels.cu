@@ -225,7 +225,9 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         // Two issuing threads, so that neither kind of UMMA waits behind the other's operands:
         // warp 9 issues S = Q K^T and dP = dO V^T of tile j+1 as soon as S/dP of tile j have been
         // copied out and K, V have landed; warp 10 issues dQ += dS K of tile j as soon as dS is there.
-        if (lane == 0) {
+        // The whole warp walks the work list (uniform control flow, so addresses and descriptors stay
+        // on the uniform datapath); one elected lane issues the UMMAs and commits.
+        {
             constexpr uint32_t idesc_s = umma_idesc_bf16(TILE, TILE, false, false);
             constexpr uint32_t idesc_dq = umma_idesc_bf16(TILE, D_QK, false, true);
             constexpr uint32_t hi_kmaj = umma_desc_hi(16, 1024);
@@ -260,14 +262,16 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                             if (!ok) break;
                             tc_fence_after_sync();
                             const uint32_t v_lo = v_lo0 + slot * (kBox128 >> 4);
+                            if (elect_one()) {
 #pragma unroll
-                            for (int kk = 0; kk < 4; ++kk)
-                                umma_ss_w(tm + kTmDP, do_lo + c * (kBox128 >> 4) + kk * 2, hi_kmaj, v_lo + kk * 2,
-                                          hi_kmaj, idesc_s, (c | kk) != 0);
-                            umma_commit(bar(B_VEMPTY + slot));
+                                for (int kk = 0; kk < 4; ++kk)
+                                    umma_ss_w(tm + kTmDP, do_lo + c * (kBox128 >> 4) + kk * 2, hi_kmaj, v_lo + kk * 2,
+                                              hi_kmaj, idesc_s, (c | kk) != 0);
+                                umma_commit(bar(B_VEMPTY + slot));
+                                if (c == 1) umma_commit(bar(B_DPFULL));
+                            }
                         }
                         if (!ok) break;
-                        umma_commit(bar(B_DPFULL));
                         if (n_tile > 0) ok = wait(B_SFREE, n_tile - 1u);   // previous S is in registers
                         if (!ok) break;
                         const int st = n_tile % kKStages;
@@ -277,17 +281,19 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                             ok = wait(B_KFULL + st * 3 + c, n_tile / kKStages);
                             if (!ok) break;
                             tc_fence_after_sync();
+                            if (elect_one()) {
 #pragma unroll
-                            for (int kk = 0; kk < 4; ++kk) {
-                                const uint32_t o = c * (kBox128 >> 4) + kk * 2;
-                                umma_ss_w(tm + kTmS, q_lo + o, hi_kmaj, k_lo + o, hi_kmaj, idesc_s, (c | kk) != 0);
+                                for (int kk = 0; kk < 4; ++kk) {
+                                    const uint32_t o = c * (kBox128 >> 4) + kk * 2;
+                                    umma_ss_w(tm + kTmS, q_lo + o, hi_kmaj, k_lo + o, hi_kmaj, idesc_s, (c | kk) != 0);
+                                }
+                                if (c == 2) umma_commit(bar(B_SFULL));
                             }
                         }
                         if (!ok) break;
-                        umma_commit(bar(B_SFULL));
                         ++n_tile;
                         ti.next();
-                        if (!ti.valid()) umma_commit(bar(B_QEMPTY));     // Q and dO are no longer read
+                        if (!ti.valid() && elect_one()) umma_commit(bar(B_QEMPTY));     // Q and dO are no longer read
                     }
                 } else {
                     bool first_tile = true;
@@ -303,16 +309,20 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                             if (ok && half == 0 && first_tile && items > 0) ok = wait(B_ACCFREE, items - 1u);
                             if (!ok) break;
                             tc_fence_after_sync();
+                            if (elect_one()) {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const int kk = (e >> 1) * 4 + half * 2 + (e & 1);
-                                umma_ts_w(tm + kTmDQ, tm + kTmDS + kk * 8, k_lo + kk * (2048 >> 4), hi_kmn, idesc_dq,
-                                          (half > 0 || e > 0 || !first_tile) ? 1u : 0u);
+                                for (int e = 0; e < 4; ++e) {
+                                    const int kk = (e >> 1) * 4 + half * 2 + (e & 1);
+                                    umma_ts_w(tm + kTmDQ, tm + kTmDS + kk * 8, k_lo + kk * (2048 >> 4), hi_kmn, idesc_dq,
+                                              (half > 0 || e > 0 || !first_tile) ? 1u : 0u);
+                                }
+                                if (half == 1) {
+                                    umma_commit(bar(B_DSFREE));
+                                    umma_commit(bar(B_KEMPTY + st));
+                                }
                             }
                         }
                         if (!ok) break;
-                        umma_commit(bar(B_DSFREE));
-                        umma_commit(bar(B_KEMPTY + st));
                         ++n_tile;
                         first_tile = false;
                     }
@@ -553,7 +563,8 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // warp 9 issues S^T = K Q^T and dP^T = V dO^T of sub-tile u+1 as soon as those of sub-tile u
         // have been copied out; warp 10 issues dV += P^T dO and dK += dS^T Q of sub-tile u as soon
         // as P and dS are in tensor memory. Neither waits behind the other's operands.
-        if (lane == 0) {
+        // The whole warp walks the work list; one elected lane issues the UMMAs and commits.
+        {
             constexpr uint32_t idesc_st = umma_idesc_bf16(TILE, SUB, false, false);
             constexpr uint32_t idesc_dv = umma_idesc_bf16(TILE, D_V, false, true);
             constexpr uint32_t idesc_dk = umma_idesc_bf16(TILE, D_QK, false, true);
@@ -581,19 +592,21 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                         if (!ok) break;
                         tc_fence_after_sync();
                         const uint32_t q_lo = q_lo0 + st * (3 * kBox64 >> 4), do_lo = do_lo0 + st * (2 * kBox64 >> 4);
-#pragma unroll
-                        for (int kk = 0; kk < D_QK / 16; ++kk)
-                            umma_ss_w(tm + kTmS, k_lo + (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2, hi_kmaj,
-                                      q_lo + (kk >> 2) * (kBox64 >> 4) + (kk & 3) * 2, hi_kmaj, idesc_st, kk > 0);
-#pragma unroll
-                        for (int kk = 0; kk < D_V / 16; ++kk)
-                            umma_ss_w(tm + kTmDP, v_lo + (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2, hi_kmaj,
-                                      do_lo + (kk >> 2) * (kBox64 >> 4) + (kk & 3) * 2, hi_kmaj, idesc_st, kk > 0);
-                        umma_commit(bar(B_SFULL));
                         ++n_step;
-                        *bursts_p = n_step;
                         si.next();
-                        if (!si.valid()) umma_commit(bar(B_KVEMPTY));    // K and V are no longer read
+                        if (elect_one()) {
+#pragma unroll
+                            for (int kk = 0; kk < D_QK / 16; ++kk)
+                                umma_ss_w(tm + kTmS, k_lo + (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2, hi_kmaj,
+                                          q_lo + (kk >> 2) * (kBox64 >> 4) + (kk & 3) * 2, hi_kmaj, idesc_st, kk > 0);
+#pragma unroll
+                            for (int kk = 0; kk < D_V / 16; ++kk)
+                                umma_ss_w(tm + kTmDP, v_lo + (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2, hi_kmaj,
+                                          do_lo + (kk >> 2) * (kBox64 >> 4) + (kk & 3) * 2, hi_kmaj, idesc_st, kk > 0);
+                            umma_commit(bar(B_SFULL));
+                            *bursts_p = n_step;
+                            if (!si.valid()) umma_commit(bar(B_KVEMPTY));    // K and V are no longer read
+                        }
                     }
                 } else {
                     bool first_step = true;
@@ -612,23 +625,25 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                         const int st = n_step % kStages;
                         const uint32_t do_lo = domn_lo0 + st * (2 * kBox64 >> 4), q_lo = qmn_lo0 + st * (3 * kBox64 >> 4);
                         const uint32_t acc = first_step ? 0u : 1u;
+                        if (elect_one()) {
 #pragma unroll
-                        for (int kk = 0; kk < SUB / 16; ++kk)
-                            umma_ts_w(tm + kTmDV, tm + kTmP + kk * 8, do_lo + kk * (2048 >> 4), hi_mn, idesc_dv,
-                                      kk > 0 ? 1u : acc);
+                            for (int kk = 0; kk < SUB / 16; ++kk)
+                                umma_ts_w(tm + kTmDV, tm + kTmP + kk * 8, do_lo + kk * (2048 >> 4), hi_mn, idesc_dv,
+                                          kk > 0 ? 1u : acc);
 #pragma unroll
-                        for (int kk = 0; kk < SUB / 16; ++kk)
-                            umma_ts_w(tm + kTmDK, tm + kTmDS + kk * 8, q_lo + kk * (2048 >> 4), hi_mn, idesc_dk,
-                                      kk > 0 ? 1u : acc);
-                        umma_commit(bar(B_PDSFREE));
-                        umma_commit(bar(B_QEMPTY + st));
+                            for (int kk = 0; kk < SUB / 16; ++kk)
+                                umma_ts_w(tm + kTmDK, tm + kTmDS + kk * 8, q_lo + kk * (2048 >> 4), hi_mn, idesc_dk,
+                                          kk > 0 ? 1u : acc);
+                            umma_commit(bar(B_PDSFREE));
+                            umma_commit(bar(B_QEMPTY + st));
+                        }
                         ++n_step;
                         first_step = false;
                     }
                 }
                 ++items;
             }
-            if (issue_scores) *bursts_p = 0xffffffffu;         // nothing more to wait for
+            if (issue_scores && elect_one()) *bursts_p = 0xffffffffu;         // nothing more to wait for
         }
     } else {
         // ------------------------------------------------------------------ elementwise warpgroups

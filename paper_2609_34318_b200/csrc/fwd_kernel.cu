@@ -148,7 +148,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         }
     } else if (warp == kWarpMma) {
         // ------------------------------------------------------------------ UMMA issuer (leader CTA)
-        if (leader && lane == 0) {
+        if (leader && elect_one()) {
             constexpr uint32_t idesc_s = umma_idesc_bf16(2 * TILE, TILE, false, false);
             constexpr uint32_t idesc_o = umma_idesc_bf16(2 * TILE, D_V, false, true);
             constexpr uint32_t hi_k = umma_desc_hi(16, 1024);           // K-major Q and K boxes

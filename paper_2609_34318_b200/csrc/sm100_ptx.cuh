@@ -73,6 +73,19 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
+// True in exactly one lane of a converged warp. Unlike `lane == 0`, the compiler knows that the
+// code under this predicate runs in a single thread and may keep descriptors, addresses and loop
+// counters on the uniform datapath, which is where TMA and UMMA instructions take their operands.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred = 0;
+    asm volatile(
+        "{\n\t.reg .b32 lane;\n\t.reg .pred p;\n\t"
+        "elect.sync lane|p, 0xffffffff;\n\t"
+        "@p mov.u32 %0, 1;\n\t}"
+        : "+r"(pred));
+    return pred != 0;
+}
+
 // Bounded wait. `abort_flag` lives in shared memory and is shared by every role of the CTA: the
 // first wait that exceeds `limit_ns` raises it, every other wait notices it and gives up too.
 // The common case (the phase completes within a few polls) touches no timer at all: reading a
@@ -455,5 +468,67 @@ __device__ __forceinline__ void umma2_commit(uint32_t bar) {
         "h"(static_cast<uint16_t>(3))
         : "memory");
 }
+
+// ----------------------------------------------------------------------------------------------
+// Four consecutive K-steps in one asm block.
+//
+// The issuing thread is one lane of a warp that shares its sub-core (and its instruction cache)
+// with two busy elementwise warps; it retires an instruction only every several cycles, so the
+// instructions spent per UMMA, not the tensor pipe, set the pace of a burst. Here a K-step costs
+// the UMMA itself plus one add per descriptor: the descriptor's high word and the "accumulate"
+// predicate are set up once per block instead of once per UMMA.
+//   A_STEP / B_STEP: increment of the low descriptor word (bytes >> 4) per K-step; for the TS form
+//   A_STEP is in tensor-memory columns.
+// ----------------------------------------------------------------------------------------------
+#define HYDRA_UMMA_SS_X4(NAME, GROUP)                                                                   \
+    template <int A_STEP, int B_STEP>                                                                  \
+    __device__ __forceinline__ void NAME(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,  \
+                                         uint32_t b_hi, uint32_t idesc, uint32_t accumulate_first) {   \
+        asm volatile(                                                                                  \
+            "{\n\t.reg .pred p, pt;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"                      \
+            "setp.ne.b32 p, %6, 0;\n\t"                                                                \
+            "setp.eq.b32 pt, %6, %6;\n\t"                                                              \
+            "mov.b64 da, {%1, %2};\n\t"                                                                \
+            "mov.b64 db, {%3, %4};\n\t"                                                                \
+            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], da, db, %5, p;\n\t"                      \
+            "add.u32 al, %1, %7;\n\tadd.u32 bl, %3, %8;\n\t"                                          \
+            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %4};\n\t"                                      \
+            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], da, db, %5, pt;\n\t"                     \
+            "add.u32 al, %1, %9;\n\tadd.u32 bl, %3, %10;\n\t"                                         \
+            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %4};\n\t"                                      \
+            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], da, db, %5, pt;\n\t"                     \
+            "add.u32 al, %1, %11;\n\tadd.u32 bl, %3, %12;\n\t"                                        \
+            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %4};\n\t"                                      \
+            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], da, db, %5, pt;\n\t}" ::"r"(d_tmem),     \
+            "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate_first), "n"(A_STEP), \
+            "n"(B_STEP), "n"(2 * A_STEP), "n"(2 * B_STEP), "n"(3 * A_STEP), "n"(3 * B_STEP)             \
+            : "memory");                                                                               \
+    }
+#define HYDRA_UMMA_TS_X4(NAME, GROUP)                                                                   \
+    template <int A_STEP, int B_STEP>                                                                  \
+    __device__ __forceinline__ void NAME(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, \
+                                         uint32_t idesc, uint32_t accumulate_first) {                  \
+        asm volatile(                                                                                  \
+            "{\n\t.reg .pred p, pt;\n\t.reg .b64 db;\n\t.reg .b32 ta, bl;\n\t"                          \
+            "setp.ne.b32 p, %5, 0;\n\t"                                                                \
+            "setp.eq.b32 pt, %5, %5;\n\t"                                                              \
+            "mov.b64 db, {%2, %3};\n\t"                                                                \
+            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], [%1], db, %4, p;\n\t"                    \
+            "add.u32 ta, %1, %6;\n\tadd.u32 bl, %2, %7;\n\tmov.b64 db, {bl, %3};\n\t"                 \
+            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], [ta], db, %4, pt;\n\t"                   \
+            "add.u32 ta, %1, %8;\n\tadd.u32 bl, %2, %9;\n\tmov.b64 db, {bl, %3};\n\t"                 \
+            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], [ta], db, %4, pt;\n\t"                   \
+            "add.u32 ta, %1, %10;\n\tadd.u32 bl, %2, %11;\n\tmov.b64 db, {bl, %3};\n\t"               \
+            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], [ta], db, %4, pt;\n\t}" ::"r"(d_tmem),   \
+            "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate_first), "n"(A_STEP),          \
+            "n"(B_STEP), "n"(2 * A_STEP), "n"(2 * B_STEP), "n"(3 * A_STEP), "n"(3 * B_STEP)             \
+            : "memory");                                                                               \
+    }
+HYDRA_UMMA_SS_X4(umma_ss_x4, "1")
+HYDRA_UMMA_TS_X4(umma_ts_x4, "1")
+HYDRA_UMMA_SS_X4(umma2_ss_x4, "2")
+HYDRA_UMMA_TS_X4(umma2_ts_x4, "2")
+#undef HYDRA_UMMA_SS_X4
+#undef HYDRA_UMMA_TS_X4
 
 }  // namespace hydra
