@@ -406,10 +406,12 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     } else {
 #pragma unroll
                         for (int c = half * 32; c < half * 32 + 32; c += 2) {
-                            const float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2_h));
-                            const float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2_h));
-                            ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum),
-                                                     p1 * (__uint_as_float(dp[c + 1]) - dsum));
+                            float x0, x1, d0, d1;
+                            ffma2(x0, x1, __uint_as_float(s[c]), __uint_as_float(s[c + 1]), p.scale_log2, p.scale_log2,
+                                  -lse2_h, -lse2_h);
+                            fadd2(d0, d1, __uint_as_float(dp[c]), __uint_as_float(dp[c + 1]), -dsum, -dsum);
+                            fmul2(d0, d1, d0, d1, ex2_approx(x0), ex2_approx(x1));
+                            ds[c >> 1] = pack_bf16x2(d0, d1);
                         }
                     }
                     if (half == 0 && c_ds > 0) {           // the previous dQ update has read dS
@@ -716,11 +718,14 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 } else {
 #pragma unroll
                     for (int c = 0; c < 32; c += 2) {
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2[c]));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2[c + 1]));
+                        float x0, x1, d0, d1;
+                        ffma2(x0, x1, __uint_as_float(s[c]), __uint_as_float(s[c + 1]), p.scale_log2, p.scale_log2,
+                              -lse2[c], -lse2[c + 1]);
+                        const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                        fadd2(d0, d1, __uint_as_float(dp[c]), __uint_as_float(dp[c + 1]), -dsum[c], -dsum[c + 1]);
+                        fmul2(d0, d1, d0, d1, p0, p1);
                         pk[c >> 1] = pack_bf16x2(p0, p1);
-                        ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum[c]),
-                                                 p1 * (__uint_as_float(dp[c + 1]) - dsum[c + 1]));
+                        ds[c >> 1] = pack_bf16x2(d0, d1);
                     }
                 }
                 if (c_pds > 0) {                       // the previous dV / dK updates have read P and dS

@@ -49,7 +49,7 @@ constexpr float kRescaleThreshold = 8.f;              // log2 units
 
 enum : int {
     B_QFULL = 0, B_QEMPTY = 2, B_KFULL = 4, B_KEMPTY = 7, B_VFULL = 10, B_VEMPTY = 13,
-    B_SFULL = 16, B_PFULL = 18, B_OFULL = 20, B_OFREE = 22, B_COUNT = 24
+    B_SFULL = 16, B_PFULL = 18, B_OFULL = 20, B_OFREE = 22, B_PFULL2 = 24, B_COUNT = 26
 };
 
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
@@ -78,7 +78,8 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         abort_flag = 0;
         for (int i = 0; i < B_COUNT; ++i) {
             // P-ready and O-drained collect the 4 softmax warps of a tile in each of the 2 CTAs
-            const bool by_warps = (i >= B_PFULL && i < B_PFULL + 2) || (i >= B_OFREE && i < B_OFREE + 2);
+            const bool by_warps = (i >= B_PFULL && i < B_PFULL + 2) || (i >= B_OFREE && i < B_OFREE + 2) ||
+                                  (i >= B_PFULL2 && i < B_PFULL2 + 2);
             mbar_init(bar(i), by_warps ? 8u : 1u);
         }
         fence_mbar_init();
@@ -200,9 +201,17 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     const bool last_user = (t == 1) || (j >= n_t[1]);
                     const uint32_t d_o = tm + kTmO + t * D_V, a_p = tm + kTmS + t * TILE;
                     const uint32_t b_lo = v_lo0 + slot * (kVStage >> 4);
+                    // P arrives in two instalments (columns [0,64) and [64,128)): the first half of the
+                    // product runs while the second half of the exponentials is still being computed
 #pragma unroll
-                    for (int kk = 0; kk < TILE / 16; ++kk)
+                    for (int kk = 0; kk < TILE / 32; ++kk)
                         umma2_ts_w(d_o, a_p + kk * 8, b_lo + kk * (2048 >> 4), hi_v, idesc_o, (j | kk) != 0);
+                    ok = wait(B_PFULL2 + t, c_p[t] - 1u);
+                    if (!ok) return;
+                    tc_fence_after_sync();
+#pragma unroll
+                    for (int kk = TILE / 32; kk < TILE / 16; ++kk)
+                        umma2_ts_w(d_o, a_p + kk * 8, b_lo + kk * (2048 >> 4), hi_v, idesc_o, 1u);
                     if (last_user) umma2_commit(bar(B_VEMPTY + slot));
                     umma2_commit(bar(B_OFULL + t));
                 };
@@ -265,23 +274,27 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     if (p.causal) jmax = min(jmax, row + pr.off);
                     cmax = jmax - col0;
                 }
-                // the whole row of S in registers: one round trip to tensor memory per kv tile
-                uint32_t s[TILE];
-#pragma unroll
-                for (int c0 = 0; c0 < TILE; c0 += 32) tmem_ld_x32(tm_s + c0, s + c0);
-                tmem_wait_ld();
-                if (need_mask) {
-#pragma unroll
-                    for (int c = 0; c < TILE; ++c)
-                        if (c > cmax) s[c] = __float_as_uint(neg_inf());
-                }
+                // pass 1: row maximum, 64 columns at a time (the 168 registers a thread may use do not
+                // hold a whole row of S next to the probabilities without spilling)
                 float mx0 = neg_inf(), mx1 = neg_inf(), mx2 = neg_inf(), mx3 = neg_inf();
 #pragma unroll
-                for (int c = 0; c < TILE; c += 4) {
-                    mx0 = fmaxf(mx0, __uint_as_float(s[c]));
-                    mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
-                    mx2 = fmaxf(mx2, __uint_as_float(s[c + 2]));
-                    mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t s[TILE / 2];
+                    tmem_ld_x32(tm_s + half * 64, s);
+                    tmem_ld_x32(tm_s + half * 64 + 32, s + 32);
+                    tmem_wait_ld();
+                    if (need_mask) {
+#pragma unroll
+                        for (int c = 0; c < TILE / 2; ++c)
+                            if (half * 64 + c > cmax) s[c] = __float_as_uint(neg_inf());
+                    }
+#pragma unroll
+                    for (int c = 0; c < TILE / 2; c += 8) {
+                        mx0 = fmax3(mx0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+                        mx1 = fmax3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+                        mx2 = fmax3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+                        mx3 = fmax3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
+                    }
                 }
                 const float m_new = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
                 float alpha = 1.f;
@@ -291,26 +304,10 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     else m_run = m_new;
                 }
                 const float m_use = (m_run == neg_inf()) ? 0.f : m_run;
-                // P = exp2(S * c - m), written over the first half of S as packed bf16
-                float rs0 = 0.f, rs1 = 0.f;
-                uint32_t pk[TILE / 2];
-#pragma unroll
-                for (int c = 0; c < TILE; c += 2) {
-                    const float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -m_use));
-                    const float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -m_use));
-                    rs0 += p0;
-                    rs1 += p1;
-                    pk[c >> 1] = pack_bf16x2(p0, p1);
-                }
-                const float rs = rs0 + rs1;
-#pragma unroll
-                for (int c0 = 0; c0 < TILE / 2; c0 += 32) tmem_st_x32(tm_s + c0, pk + c0);
-                l_run = l_run * alpha + rs;
                 if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-                    // the previous P V of this tile must have landed before O is rescaled
-                    ok = wait(B_OFULL + t, c_o - 1u);
-                    if (!ok) break;
-                    tc_fence_after_sync();
+                    // Rescale O before any part of this tile's product is added to it. The previous
+                    // P V of this tile has landed: it was issued before this tile's S, which has
+                    // completed, and the tensor pipe runs in issue order.
 #pragma unroll
                     for (int c0 = 0; c0 < D_V; c0 += 32) {
                         uint32_t o[32];
@@ -321,9 +318,44 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                         tmem_st_x32(tm_o + c0, o);
                     }
                 }
-                tmem_wait_st();
-                tc_fence_before_sync();
-                mbar_arrive_warp_leader(bar(B_PFULL + t));
+                // pass 2: P = exp2(S * c - m) as packed bf16, written over the first half of S and handed
+                // to the tensor core in two instalments (columns [0,64), then [64,128)).
+                float rs0 = 0.f, rs1 = 0.f;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t s[TILE / 2], pk[TILE / 4];
+                    tmem_ld_x32(tm_s + half * 64, s);
+                    tmem_ld_x32(tm_s + half * 64 + 32, s + 32);
+                    tmem_wait_ld();
+                    if (need_mask) {
+#pragma unroll
+                        for (int c = 0; c < TILE / 2; c += 2) {
+                            float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -m_use));
+                            float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -m_use));
+                            if (half * 64 + c > cmax) p0 = 0.f;
+                            if (half * 64 + c + 1 > cmax) p1 = 0.f;
+                            rs0 += p0;
+                            rs1 += p1;
+                            pk[c >> 1] = pack_bf16x2(p0, p1);
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < TILE / 2; c += 2) {
+                            float x0, x1;
+                            ffma2(x0, x1, __uint_as_float(s[c]), __uint_as_float(s[c + 1]), p.scale_log2, p.scale_log2,
+                                  -m_use, -m_use);
+                            const float p0 = ex2_approx(x0);
+                            const float p1 = ex2_approx(x1);
+                            fadd2(rs0, rs1, rs0, rs1, p0, p1);
+                            pk[c >> 1] = pack_bf16x2(p0, p1);
+                        }
+                    }
+                    tmem_st_x32(tm_s + half * 32, pk);
+                    tmem_wait_st();
+                    tc_fence_before_sync();
+                    mbar_arrive_warp_leader(bar((half == 0 ? B_PFULL : B_PFULL2) + t));
+                }
+                l_run = l_run * alpha + (rs0 + rs1);
                 ++c_o;
             }
             if (!ok) break;

@@ -349,6 +349,61 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Two fp32 lanes per instruction (sm_100 f32x2): the elementwise warps are bound by instruction
+// issue, not by arithmetic throughput, so pairing neighbouring columns halves the cost of the
+// scale-and-shift and of the row sums.
+__device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0,
+                                      float c1) {
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+__device__ __forceinline__ void fadd2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "add.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void fmul2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "mul.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+// max of three in one instruction
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// 2^x on the FMA pipe, for x <= ~100: round to the nearest integer n with the 1.5 * 2^23 trick, a
+// cubic minimax polynomial for 2^f on f = x - n in [-0.5, 0.5] (relative error 7.5e-5, far below
+// the bf16 rounding of the probabilities it produces), and n added straight into the exponent
+// field. Inputs below -126 (including -inf) give 2^-126, which is zero for every use here. The
+// special-function unit does 16 exponentials per cycle per SM and is the scarcest resource of the
+// softmax; the eight FMA-pipe instructions of this routine cost the SM the same 1/16 cycle per
+// element, so splitting the columns between the two roughly doubles the throughput.
+__device__ __forceinline__ float exp2_poly3(float x) {
+    x = fmaxf(x, -126.f);
+    const float t = x + 12582912.f;                  // 1.5 * 2^23: the low mantissa bits now hold n
+    const float f = x - (t - 12582912.f);
+    float p = fmaf(f, 0.05517134f, 0.24261034f);
+    p = fmaf(p, f, 0.69326097f);
+    p = fmaf(p, f, 0.99992812f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+__device__ __forceinline__ float ld_shared_volatile_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.volatile.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
 // {lo, hi} -> packed bf16x2, round to nearest even; `lo` lands in the low 16 bits.
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
