@@ -383,27 +383,6 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
-// 2^x on the FMA pipe, for x <= ~100: round to the nearest integer n with the 1.5 * 2^23 trick, a
-// cubic minimax polynomial for 2^f on f = x - n in [-0.5, 0.5] (relative error 7.5e-5, far below
-// the bf16 rounding of the probabilities it produces), and n added straight into the exponent
-// field. Inputs below -126 (including -inf) give 2^-126, which is zero for every use here. The
-// special-function unit does 16 exponentials per cycle per SM and is the scarcest resource of the
-// softmax; the eight FMA-pipe instructions of this routine cost the SM the same 1/16 cycle per
-// element, so splitting the columns between the two roughly doubles the throughput.
-__device__ __forceinline__ float exp2_poly3(float x) {
-    x = fmaxf(x, -126.f);
-    const float t = x + 12582912.f;                  // 1.5 * 2^23: the low mantissa bits now hold n
-    const float f = x - (t - 12582912.f);
-    float p = fmaf(f, 0.05517134f, 0.24261034f);
-    p = fmaf(p, f, 0.69326097f);
-    p = fmaf(p, f, 0.99992812f);
-    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
-}
-__device__ __forceinline__ float ld_shared_volatile_f32(uint32_t addr) {
-    float v;
-    asm volatile("ld.volatile.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
-    return v;
-}
 // {lo, hi} -> packed bf16x2, round to nearest even; `lo` lands in the low 16 bits.
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
@@ -523,67 +502,5 @@ __device__ __forceinline__ void umma2_commit(uint32_t bar) {
         "h"(static_cast<uint16_t>(3))
         : "memory");
 }
-
-// ----------------------------------------------------------------------------------------------
-// Four consecutive K-steps in one asm block.
-//
-// The issuing thread is one lane of a warp that shares its sub-core (and its instruction cache)
-// with two busy elementwise warps; it retires an instruction only every several cycles, so the
-// instructions spent per UMMA, not the tensor pipe, set the pace of a burst. Here a K-step costs
-// the UMMA itself plus one add per descriptor: the descriptor's high word and the "accumulate"
-// predicate are set up once per block instead of once per UMMA.
-//   A_STEP / B_STEP: increment of the low descriptor word (bytes >> 4) per K-step; for the TS form
-//   A_STEP is in tensor-memory columns.
-// ----------------------------------------------------------------------------------------------
-#define HYDRA_UMMA_SS_X4(NAME, GROUP)                                                                   \
-    template <int A_STEP, int B_STEP>                                                                  \
-    __device__ __forceinline__ void NAME(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,  \
-                                         uint32_t b_hi, uint32_t idesc, uint32_t accumulate_first) {   \
-        asm volatile(                                                                                  \
-            "{\n\t.reg .pred p, pt;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"                      \
-            "setp.ne.b32 p, %6, 0;\n\t"                                                                \
-            "setp.eq.b32 pt, %6, %6;\n\t"                                                              \
-            "mov.b64 da, {%1, %2};\n\t"                                                                \
-            "mov.b64 db, {%3, %4};\n\t"                                                                \
-            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], da, db, %5, p;\n\t"                      \
-            "add.u32 al, %1, %7;\n\tadd.u32 bl, %3, %8;\n\t"                                          \
-            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %4};\n\t"                                      \
-            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], da, db, %5, pt;\n\t"                     \
-            "add.u32 al, %1, %9;\n\tadd.u32 bl, %3, %10;\n\t"                                         \
-            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %4};\n\t"                                      \
-            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], da, db, %5, pt;\n\t"                     \
-            "add.u32 al, %1, %11;\n\tadd.u32 bl, %3, %12;\n\t"                                        \
-            "mov.b64 da, {al, %2};\n\tmov.b64 db, {bl, %4};\n\t"                                      \
-            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], da, db, %5, pt;\n\t}" ::"r"(d_tmem),     \
-            "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate_first), "n"(A_STEP), \
-            "n"(B_STEP), "n"(2 * A_STEP), "n"(2 * B_STEP), "n"(3 * A_STEP), "n"(3 * B_STEP)             \
-            : "memory");                                                                               \
-    }
-#define HYDRA_UMMA_TS_X4(NAME, GROUP)                                                                   \
-    template <int A_STEP, int B_STEP>                                                                  \
-    __device__ __forceinline__ void NAME(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, \
-                                         uint32_t idesc, uint32_t accumulate_first) {                  \
-        asm volatile(                                                                                  \
-            "{\n\t.reg .pred p, pt;\n\t.reg .b64 db;\n\t.reg .b32 ta, bl;\n\t"                          \
-            "setp.ne.b32 p, %5, 0;\n\t"                                                                \
-            "setp.eq.b32 pt, %5, %5;\n\t"                                                              \
-            "mov.b64 db, {%2, %3};\n\t"                                                                \
-            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], [%1], db, %4, p;\n\t"                    \
-            "add.u32 ta, %1, %6;\n\tadd.u32 bl, %2, %7;\n\tmov.b64 db, {bl, %3};\n\t"                 \
-            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], [ta], db, %4, pt;\n\t"                   \
-            "add.u32 ta, %1, %8;\n\tadd.u32 bl, %2, %9;\n\tmov.b64 db, {bl, %3};\n\t"                 \
-            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], [ta], db, %4, pt;\n\t"                   \
-            "add.u32 ta, %1, %10;\n\tadd.u32 bl, %2, %11;\n\tmov.b64 db, {bl, %3};\n\t"               \
-            "tcgen05.mma.cta_group::" GROUP ".kind::f16 [%0], [ta], db, %4, pt;\n\t}" ::"r"(d_tmem),   \
-            "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate_first), "n"(A_STEP),          \
-            "n"(B_STEP), "n"(2 * A_STEP), "n"(2 * B_STEP), "n"(3 * A_STEP), "n"(3 * B_STEP)             \
-            : "memory");                                                                               \
-    }
-HYDRA_UMMA_SS_X4(umma_ss_x4, "1")
-HYDRA_UMMA_TS_X4(umma_ts_x4, "1")
-HYDRA_UMMA_SS_X4(umma2_ss_x4, "2")
-HYDRA_UMMA_TS_X4(umma2_ts_x4, "2")
-#undef HYDRA_UMMA_SS_X4
-#undef HYDRA_UMMA_TS_X4
 
 }  // namespace hydra
