@@ -343,14 +343,20 @@ def merge_groups(pairs):
     return out
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised in
+# profiles/tensor_kernels_packed32k.md and profiles/merge_prep_short64k_split.md.
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    "fwd:packed32k": 731282432,
+    "bwd_dkv:packed32k": 1010001408,
+    "bwd_dq:packed32k": 873572864,
+    "merge:short64k_split": 764219424,
+    "bwd_prep:short64k_split": 1082259656,
+}
+
+
 def recorded_traffic(kernel: str, workload: str):
-    """DRAM bytes per launch from the ncu capture summarised under profiles/ (None if not captured)."""
-    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
-    if not os.path.exists(path):
-        return None
-    with open(path) as f:
-        table = json.load(f)
-    return table.get(f"{kernel}:{workload}")
+    """DRAM bytes per launch from the ncu capture of this kernel and workload (None if not captured)."""
+    return NCU_DRAM_BYTES_PER_LAUNCH.get(f"{kernel}:{workload}")
 
 
 def main():
