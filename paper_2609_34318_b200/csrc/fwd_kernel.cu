@@ -166,64 +166,76 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 const int n_t[2] = {item.n_a, item.n_b};
                 const int n = max(item.n_a, item.n_b);
 
-                auto issue_s = [&](int t, int j) {
-                    if (j == 0) {
-                        ok = wait(B_QFULL + t, q_use[t]);
-                        ++q_use[t];
+                // One step of a tile's chain: finish kv tile `jpv` (O += P V) and start kv tile `js`
+                // (S = Q K^T), back to back. The polls that are almost always satisfied (K, V, Q
+                // landed; O drained) come first, so that once the softmax has delivered P nothing
+                // but UMMAs and commits stands between the end of one product and the start of the
+                // next: the tile's chain S -> softmax -> P V -> S is the critical path.
+                auto advance = [&](int t, int jpv, uint32_t v_slot, uint32_t v_ph, int js, uint32_t k_slot,
+                                   uint32_t k_ph) {
+                    const bool do_pv = jpv >= 0 && jpv < n_t[t];
+                    const bool do_s = js < n_t[t];
+                    if (do_s) {
+                        if (js == 0) {
+                            ok = wait(B_QFULL + t, q_use[t]);
+                            ++q_use[t];
+                            if (!ok) return;
+                        }
+                        ok = wait(B_KFULL + k_slot, k_ph);
                         if (!ok) return;
                     }
-                    ok = wait(B_KFULL + ks, kp);
-                    if (!ok) return;
-                    tc_fence_after_sync();
-                    const bool last_user = (t == 1) || (j >= n_t[1]);
-                    const uint32_t d_s = tm + kTmS + t * TILE;
-                    const uint32_t b_lo = k_lo0 + ks * (kKStage >> 4);
-#pragma unroll
-                    for (int kk = 0; kk < D_QK / 16; ++kk)
-                        umma2_ss_w(d_s, q_lo[t] + (kk >> 2) * (kBox >> 4) + (kk & 3) * 2, hi_k,
-                                   b_lo + (kk >> 2) * (kHalfBox >> 4) + (kk & 3) * 2, hi_k, idesc_s, kk != 0);
-                    if (last_user) umma2_commit(bar(B_KEMPTY + ks));
-                    umma2_commit(bar(B_SFULL + t));
-                    if (j == n_t[t] - 1) umma2_commit(bar(B_QEMPTY + t));
-                };
-                auto issue_pv = [&](int t, int j, uint32_t slot, uint32_t ph) {
-                    ok = wait(B_PFULL + t, c_p[t]);
-                    ++c_p[t];
-                    if (!ok) return;
-                    if (j == 0) {
-                        ok = wait(B_OFREE + t, free_use[t] ^ 1u);
-                        ++free_use[t];
+                    const uint32_t d_s = tm + kTmS + t * TILE, d_o = tm + kTmO + t * D_V;
+                    if (do_pv) {
+                        ok = wait(B_VFULL + v_slot, v_ph);
                         if (!ok) return;
+                        if (jpv == 0) {
+                            ok = wait(B_OFREE + t, free_use[t] ^ 1u);
+                            ++free_use[t];
+                            if (!ok) return;
+                        }
+                        // P arrives in two instalments (columns [0,64) and [64,128)): the first half of
+                        // the product runs while the second half of the exponentials is being computed
+                        ok = wait(B_PFULL + t, c_p[t]);
+                        if (!ok) return;
+                        tc_fence_after_sync();
+                        const uint32_t b_lo = v_lo0 + v_slot * (kVStage >> 4);
+#pragma unroll
+                        for (int kk = 0; kk < TILE / 32; ++kk)
+                            umma2_ts_w(d_o, d_s + kk * 8, b_lo + kk * (2048 >> 4), hi_v, idesc_o, (jpv | kk) != 0);
+                        ok = wait(B_PFULL2 + t, c_p[t]);
+                        ++c_p[t];
+                        if (!ok) return;
+                        tc_fence_after_sync();
+#pragma unroll
+                        for (int kk = TILE / 32; kk < TILE / 16; ++kk)
+                            umma2_ts_w(d_o, d_s + kk * 8, b_lo + kk * (2048 >> 4), hi_v, idesc_o, 1u);
+                        if ((t == 1) || (jpv >= n_t[1])) umma2_commit(bar(B_VEMPTY + v_slot));   // last reader
+                        umma2_commit(bar(B_OFULL + t));
+                    } else {
+                        tc_fence_after_sync();
                     }
-                    ok = wait(B_VFULL + slot, ph);
-                    if (!ok) return;
-                    tc_fence_after_sync();
-                    const bool last_user = (t == 1) || (j >= n_t[1]);
-                    const uint32_t d_o = tm + kTmO + t * D_V, a_p = tm + kTmS + t * TILE;
-                    const uint32_t b_lo = v_lo0 + slot * (kVStage >> 4);
-                    // P arrives in two instalments (columns [0,64) and [64,128)): the first half of the
-                    // product runs while the second half of the exponentials is still being computed
+                    if (do_s) {
+                        const uint32_t b_lo = k_lo0 + k_slot * (kKStage >> 4);
 #pragma unroll
-                    for (int kk = 0; kk < TILE / 32; ++kk)
-                        umma2_ts_w(d_o, a_p + kk * 8, b_lo + kk * (2048 >> 4), hi_v, idesc_o, (j | kk) != 0);
-                    ok = wait(B_PFULL2 + t, c_p[t] - 1u);
-                    if (!ok) return;
-                    tc_fence_after_sync();
-#pragma unroll
-                    for (int kk = TILE / 32; kk < TILE / 16; ++kk)
-                        umma2_ts_w(d_o, a_p + kk * 8, b_lo + kk * (2048 >> 4), hi_v, idesc_o, 1u);
-                    if (last_user) umma2_commit(bar(B_VEMPTY + slot));
-                    umma2_commit(bar(B_OFULL + t));
+                        for (int kk = 0; kk < D_QK / 16; ++kk)
+                            umma2_ss_w(d_s, q_lo[t] + (kk >> 2) * (kBox >> 4) + (kk & 3) * 2, hi_k,
+                                       b_lo + (kk >> 2) * (kHalfBox >> 4) + (kk & 3) * 2, hi_k, idesc_s, kk != 0);
+                        if ((t == 1) || (js >= n_t[1])) umma2_commit(bar(B_KEMPTY + k_slot));    // last reader
+                        umma2_commit(bar(B_SFULL + t));
+                        if (js == n_t[t] - 1) umma2_commit(bar(B_QEMPTY + t));
+                    }
                 };
 
+                // issue order: S_A(0) | S_B(0) | PV_A(0) S_A(1) | PV_B(0) S_B(1) | PV_A(1) S_A(2) | ...
+                advance(0, -1, 0u, 0u, 0, ks, kp);
                 for (int j = 0; j <= n && ok; ++j) {
-                    if (j < n_t[0]) issue_s(0, j);
-                    if (ok && j >= 1 && j - 1 < n_t[1]) issue_pv(1, j - 1, vs_prev, vp_prev);
-                    if (ok && j < n_t[1]) issue_s(1, j);
-                    if (ok && j < n_t[0]) issue_pv(0, j, vs, vp);
+                    uint32_t ks1 = ks + 1u, kp1 = kp;          // ring position of kv tile j + 1
+                    if (ks1 == kKStages) { ks1 = 0; kp1 ^= 1u; }
+                    advance(1, j - 1, vs_prev, vp_prev, j, ks, kp);
+                    if (ok) advance(0, j, vs, vp, j + 1, ks1, kp1);
                     if (j < n) {                     // step the ring cursors to kv tile j + 1
                         vs_prev = vs; vp_prev = vp;
-                        if (++ks == kKStages) { ks = 0; kp ^= 1u; }
+                        ks = ks1; kp = kp1;
                         if (++vs == kVStages) { vs = 0; vp ^= 1u; }
                     }
                 }
