@@ -91,15 +91,8 @@ class ClockSampler(threading.Thread):
 # --------------------------------------------------------------------------------------------------
 # reference arm: the oracle on the host cores, bounded sample
 # --------------------------------------------------------------------------------------------------
-def oracle_sample(w, budget_s: float):
-    """Leading sequences of the workload, one head, sized so one fwd+bwd takes about `budget_s`."""
-    import oracle
-    probe = hw.Workload("probe", [768], 1)
-    x = probe.tensors([0])
-    t0 = time.perf_counter()
-    out, lse = oracle.attn_fwd(x["q"], x["k"], x["v"], probe.cu(), True, probe.scale)
-    oracle.attn_bwd(x["q"], x["k"], x["v"], x["do"], probe.cu(), True, probe.scale, out, lse)
-    rate = probe.causal_pairs_total / max(time.perf_counter() - t0, 1e-6)      # pairs*head / s
+def _pick_sample(w, rate: float, budget_s: float):
+    """Leading sequences (then more heads) of `w` worth about `budget_s` at `rate` pairs*heads per second."""
     lengths, pairs = [], 0
     for length in w.lengths:
         cost = length * (length + 1) // 2
@@ -110,12 +103,40 @@ def oracle_sample(w, budget_s: float):
             cost = length * (length + 1) // 2
         lengths.append(length)
         pairs += cost
-    return hw.Workload(w.name + "_sample", lengths, 1, cp_r=w.cp_r)
+    heads = 1
+    if len(lengths) == len(w.lengths):                       # the whole batch fits: add heads
+        heads = int(max(1, min(w.n_heads, budget_s * rate // max(pairs, 1))))
+    return hw.Workload(w.name + "_sample", lengths, heads, cp_r=w.cp_r)
+
+
+def oracle_sample(w, budget_s: float):
+    """A bounded sample of the workload (leading sequences, leading heads) whose fwd+bwd takes about
+    `budget_s` on this host. The oracle's rate depends on the problem size (threads, caches), so the
+    size is chosen in two steps: from a small probe, then from a timed run of that first choice."""
+    import oracle
+    probe = hw.Workload("probe", [768], 1)
+    x = probe.tensors([0])
+    t0 = time.perf_counter()
+    out, lse = oracle.attn_fwd(x["q"], x["k"], x["v"], probe.cu(), True, probe.scale)
+    oracle.attn_bwd(x["q"], x["k"], x["v"], x["do"], probe.cu(), True, probe.scale, out, lse)
+    rate = probe.causal_pairs_total / max(time.perf_counter() - t0, 1e-6)      # pairs*head / s
+    first = _pick_sample(w, rate, budget_s / 4)
+    sec = oracle_step(first)
+    if sec > budget_s / 8:
+        rate = first.causal_pairs_total * first.n_heads / sec
+    else:                                                    # too short to trust: assume it scales
+        rate = max(rate, first.causal_pairs_total * first.n_heads / max(sec, 1e-6))
+    return _pick_sample(w, rate, budget_s)
+
+
+def sample_desc(sample, w) -> str:
+    return (f"first {len(sample.lengths)} sequence(s) ({sample.total} tokens), {sample.n_heads} head(s) of "
+            f"{w.name}, fwd+bwd")
 
 
 def oracle_step(sample):
     import oracle
-    x = sample.tensors([0])
+    x = sample.tensors(list(range(sample.n_heads)))
     cu = sample.cu()
     t0 = time.perf_counter()
     out, lse = oracle.attn_fwd(x["q"], x["k"], x["v"], cu, True, sample.scale)
@@ -141,7 +162,7 @@ def run_reference(args, w):
     total = sum(times)
     flops = 3.5 * sample.flops_fwd() * args.steps
     value = flops / total / 1e12
-    desc = f"first {len(sample.lengths)} sequence(s) ({sample.total} tokens), 1 head of {w.name}, fwd+bwd"
+    desc = sample_desc(sample, w)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
@@ -166,6 +187,20 @@ def device_inputs(w, torch, seed_shift: int):
         for a in range(h):
             t[n][:, a, :] = bits_to_tensor(hw.tensor_bits(n, T, [a], seed=hw.SEED + seed_shift))[:, 0, :]
     return t
+
+
+def max_over_ranks(value_ms: float, dist, device) -> float:
+    """The slowest rank's time: what a multi-GPU number is computed from. Works with any backend
+    (`device` is where the backend wants its tensors: "cuda" for nccl, "cpu" for gloo)."""
+    import torch
+    tt = torch.tensor([value_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def whole_job_value(world: int, flops_per_rank_step: float, steps: int, max_ms: float) -> float:
+    """Weak scaling: every rank processes its own microbatch; TFLOP/s of all ranks together."""
+    return world * flops_per_rank_step * steps / (max_ms * 1e-3) / 1e12
 
 
 def run_ours(args, w):
@@ -223,15 +258,13 @@ def run_ours(args, w):
     kernel_ms, kernel_n = P.hydra_profile_collect()
     P.hydra_profile_enable(False)
     if world > 1:
-        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+        total_ms = max_over_ranks(total_ms, dist, "cuda")
     status, detail = step.poll()
     if status != 0:
         raise RuntimeError(f"device status {status} at item {detail}")
 
     flops_step = 3.5 * w.flops_fwd()
-    value = world * flops_step * args.steps / (total_ms * 1e-3) / 1e12
+    value = whole_job_value(world, flops_step, args.steps, total_ms)
 
     # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region ----
     e2e = None
@@ -264,12 +297,10 @@ def run_ours(args, w):
         barrier()
         e2e_ms = e0.elapsed_time(e1)
         if world > 1:
-            tt = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_ms = float(tt.item())
+            e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
         h2d = sum(v.numel() * v.element_size() for v in host.values())
         d2h = sum(v.numel() * v.element_size() for v in ho.values())
-        e2e = {"value": world * flops_step * e_steps / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+        e2e = {"value": whole_job_value(world, flops_step, e_steps, e2e_ms), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e_steps,
                "ms_per_step": e2e_ms / e_steps}
         assert torch.isfinite(ho["dq"].float()).all()
@@ -309,8 +340,7 @@ def run_ours(args, w):
         sec = oracle_step(sample)
         cpu = {"value": 3.5 * sample.flops_fwd() / sec / 1e12, "unit": UNIT, "cores": oracle.n_threads(),
                "kind": "oracle", "seconds": sec,
-               "sample": f"first {len(sample.lengths)} sequence(s) ({sample.total} tokens), 1 head of "
-                         f"{w.name}, fwd+bwd"}
+               "sample": sample_desc(sample, w)}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
