@@ -182,12 +182,17 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
 /*
  * The whole step (forward of every pair, merge, backward; Sections 3.5 and 5.2 as above) with HOST
  * buffers: copies q, k, v, dout to the device, runs hydra_attn_fwd, hydra_lse_merge (if any pair has
- * partial rows) and hydra_attn_bwd, and copies out, lse, dq, dk, dv back, all enqueued on
- * `cuda_stream`. Host buffers have the tensor layouts above; pinned memory makes the copies
- * asynchronous. `device_arena` is device memory, 256-byte aligned, of at least
- * hydra_host_step_arena_bytes(...) bytes, owned by the caller; the library carves every device
- * tensor, the partial buffers and the workspace out of it and allocates nothing itself.
- * Host outputs are valid once the stream has been synchronised.
+ * partial rows) and hydra_attn_bwd, and copies out, lse, dq, dk, dv back. Heads are independent,
+ * so with 4 or more heads the step is pipelined over groups of 2 or 4 heads: the kernels run on
+ * `cuda_stream`, the copies in and out on two internal streams (created once per device, on the
+ * first call), so that both directions of the host link are busy at once. Work enqueued on
+ * `cuda_stream` before the call precedes all of it, and `cuda_stream` completes only when the last
+ * copy out has: host outputs are valid once the stream has been synchronised. Host buffers have
+ * the tensor layouts above; pinned memory makes the copies asynchronous. `device_arena` is device
+ * memory, 256-byte aligned, of at least hydra_host_step_arena_bytes(...) bytes, owned by the
+ * caller; the library carves every device tensor, the partial buffers and the workspace out of it
+ * and allocates no device memory itself. One call at a time per device (the internal streams and
+ * events are shared); more than 128 heads: HYDRA_ERR_UNSUPPORTED.
  */
 size_t hydra_host_step_arena_bytes(const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
                                    const hydra_pair_t* pairs, int32_t n_pairs);

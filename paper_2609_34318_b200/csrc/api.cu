@@ -4,6 +4,7 @@
 #include <atomic>
 #include <cmath>
 #include <cstring>
+#include <map>
 #include <memory>
 #include <mutex>
 #include <vector>
@@ -536,6 +537,37 @@ using namespace hydra;
 // =============================================================================================
 // C ABI
 // =============================================================================================
+namespace {
+// Copy streams and events of hydra_attn_fwd_bwd_host, one set per device, created on first use.
+constexpr size_t kHostLsePad = 64 * 256;                    // alignment slack of the per-group LSE slices
+struct HostPipe {
+    static constexpr int kMaxGroups = 64;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, end = nullptr;
+    cudaEvent_t in_done[kMaxGroups] = {}, comp_done[kMaxGroups] = {};
+};
+HostPipe* host_pipe()
+{
+    static std::mutex mu;
+    static std::map<int, HostPipe> pipes;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = pipes.find(dev);
+    if (it != pipes.end()) return &it->second;
+    HostPipe p;
+    bool ok = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p.end, cudaEventDisableTiming) == cudaSuccess;
+    for (int g = 0; ok && g < HostPipe::kMaxGroups; ++g)
+        ok = cudaEventCreateWithFlags(&p.in_done[g], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&p.comp_done[g], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return nullptr;
+    return &pipes.emplace(dev, p).first->second;
+}
+}  // namespace
+
 extern "C" {
 
 int32_t hydra_version(void) { return 1; }
@@ -834,7 +866,7 @@ size_t hydra_host_step_arena_bytes(const int32_t* cu, int32_t n_seqs, int32_t n_
     b += 3 * align_up(th * D_QK * 2, 256);                   // q, k + dq/dk share nothing: q, k, dq
     b += 1 * align_up(th * D_QK * 2, 256);                   // dk
     b += 4 * align_up(th * D_V * 2, 256);                    // v, dout, out, dv
-    b += align_up(th * 4, 256);                              // lse
+    b += align_up(th * 4, 256) + kHostLsePad;                // lse, one 256-byte aligned slice per head group
     b += align_up(static_cast<size_t>(std::max<int64_t>(part_rows, 1)) * n_heads * D_V * 2, 256);
     b += align_up(static_cast<size_t>(std::max<int64_t>(part_rows, 1)) * n_heads * 4, 256);
     b += kStatusBytes + align_up(th * 4, 256);               // workspace of the backward call
@@ -864,35 +896,98 @@ int32_t hydra_attn_fwd_bwd_host(const void* q_host, const void* k_host, const vo
     const size_t th = static_cast<size_t>(pb.T) * n_heads;
     uint8_t* cur = static_cast<uint8_t*>(device_arena);
     auto carve = [&](size_t bytes) { void* p = cur; cur += align_up(bytes, 256); return p; };
-    void* dq_ = carve(th * D_QK * 2); void* dk_ = carve(th * D_QK * 2);
-    void* q = carve(th * D_QK * 2); void* k = carve(th * D_QK * 2);
-    void* v = carve(th * D_V * 2); void* dout = carve(th * D_V * 2);
-    void* out = carve(th * D_V * 2); void* dv_ = carve(th * D_V * 2);
-    float* lse = static_cast<float*>(carve(th * 4));
+    uint8_t* dq_ = static_cast<uint8_t*>(carve(th * D_QK * 2)); uint8_t* dk_ = static_cast<uint8_t*>(carve(th * D_QK * 2));
+    uint8_t* q = static_cast<uint8_t*>(carve(th * D_QK * 2)); uint8_t* k = static_cast<uint8_t*>(carve(th * D_QK * 2));
+    uint8_t* v = static_cast<uint8_t*>(carve(th * D_V * 2)); uint8_t* dout = static_cast<uint8_t*>(carve(th * D_V * 2));
+    uint8_t* out = static_cast<uint8_t*>(carve(th * D_V * 2)); uint8_t* dv_ = static_cast<uint8_t*>(carve(th * D_V * 2));
+    uint8_t* lse = static_cast<uint8_t*>(carve(th * 4 + kHostLsePad));
     void* o_part = carve(static_cast<size_t>(std::max<int64_t>(part_rows, 1)) * n_heads * D_V * 2);
     float* lse_part = static_cast<float*>(carve(static_cast<size_t>(std::max<int64_t>(part_rows, 1)) * n_heads * 4));
     void* ws = carve(kStatusBytes + align_up(th * 4, 256));
     const size_t ws_bytes = kStatusBytes + align_up(th * 4, 256);
-    auto h2d = [&](void* d, const void* h, size_t n) { return cudaMemcpyAsync(d, h, n, cudaMemcpyHostToDevice, stream); };
-    auto d2h = [&](void* h, const void* d, size_t n) { return cudaMemcpyAsync(h, d, n, cudaMemcpyDeviceToHost, stream); };
-    if (h2d(q, q_host, th * D_QK * 2) || h2d(k, k_host, th * D_QK * 2) || h2d(v, v_host, th * D_V * 2) ||
-        h2d(dout, dout_host, th * D_V * 2))
-        return HYDRA_ERR_CUDA;
     const bool any_part = part_rows > 0;
-    if (int32_t s = hydra_attn_fwd(q, k, v, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, out, lse,
-                                   any_part ? o_part : nullptr, any_part ? lse_part : nullptr, part_rows, ws,
-                                   ws_bytes, cuda_stream))
-        return s;
-    if (any_part)
-        if (int32_t s = hydra_lse_merge(o_part, lse_part, part_rows, cu, n_seqs, n_heads, pairs, n_pairs, out,
-                                        lse, ws, ws_bytes, cuda_stream))
-            return s;
-    if (int32_t s = hydra_attn_bwd(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal,
-                                   softmax_scale, dq_, dk_, dv_, ws, ws_bytes, cuda_stream))
-        return s;
-    if (d2h(out_host, out, th * D_V * 2) || d2h(lse_host, lse, th * 4) || d2h(dq_host, dq_, th * D_QK * 2) ||
-        d2h(dk_host, dk_, th * D_QK * 2) || d2h(dv_host, dv_, th * D_V * 2))
+
+    // Heads are independent, so the step is pipelined over groups of heads: while group g computes,
+    // group g+1 is on its way in and group g-1 on its way out, on two internal copy streams; the PCIe
+    // link then carries both directions at once instead of one after the other. On the device a
+    // group is a compact [T, heads_of_group, d] tensor (the g-th slice of each arena tensor); on the
+    // host it is a strided view of [T, n_heads, d], moved by 2-D copies.
+    HostPipe* pipe = host_pipe();
+    if (!pipe) return HYDRA_ERR_CUDA;
+    // Group size: when the copies dominate (short sequences: bytes grow with T, arithmetic with the
+    // pair count), small groups shorten the fill and the drain of the pipeline and the kernels,
+    // though less efficient on few heads, still hide under the copies; when the arithmetic
+    // dominates, larger groups keep the kernels efficient. Rough rates: 50 GB/s, 700 TFLOP/s.
+    double pair_count = 0.0;
+    for (const auto& p : pb.pairs) {
+        const double full = static_cast<double>(p.q_len) * p.k_len;
+        pair_count += causal ? std::min(full, 0.5 * p.q_len * (p.q_len + 1.0) +
+                                                  static_cast<double>(p.q_len) * std::max(0, p.q_start - p.k_start))
+                             : full;
+    }
+    const double copy_s = static_cast<double>(pb.T) * (2 * D_QK + 2 * D_V) * 2 / 50e9;   // per head, one direction
+    const double math_s = pair_count * 3.5 * 2 * (D_QK + D_V) / 700e12;                  // per head
+    const int32_t hg = n_heads < 4 ? n_heads : (math_s < 0.5 * copy_s ? 2 : 4);
+    const int32_t n_groups = (n_heads + hg - 1) / hg;
+    if (n_groups > HostPipe::kMaxGroups) return HYDRA_ERR_UNSUPPORTED;
+    size_t lse_off[HostPipe::kMaxGroups + 1] = {0};         // LSE slices start on 256-byte boundaries
+    for (int32_t g = 0; g < n_groups; ++g)
+        lse_off[g + 1] = align_up(lse_off[g] + static_cast<size_t>(pb.T) * std::min(hg, n_heads - g * hg) * 4, 256);
+    const size_t T = static_cast<size_t>(pb.T);
+    auto copy2d = [&](void* dst, size_t dpitch, const void* src, size_t spitch, size_t width, cudaMemcpyKind kind,
+                      cudaStream_t st) { return cudaMemcpy2DAsync(dst, dpitch, src, spitch, width, T, kind, st); };
+    if (cudaEventRecord(pipe->start, stream) || cudaStreamWaitEvent(pipe->in, pipe->start, 0) ||
+        cudaStreamWaitEvent(pipe->out, pipe->start, 0))
         return HYDRA_ERR_CUDA;
+    for (int32_t g = 0; g < n_groups; ++g) {
+        const int32_t h0 = g * hg, hn = std::min(hg, n_heads - h0);
+        const size_t oqk = T * h0 * D_QK * 2, ov = T * h0 * D_V * 2;          // the group's slice of the arena tensors
+        const size_t wqk = static_cast<size_t>(hn) * D_QK * 2, wv = static_cast<size_t>(hn) * D_V * 2;
+        const size_t pqk = static_cast<size_t>(n_heads) * D_QK * 2, pv = static_cast<size_t>(n_heads) * D_V * 2;
+        const uint8_t* qh = static_cast<const uint8_t*>(q_host) + static_cast<size_t>(h0) * D_QK * 2;
+        const uint8_t* kh = static_cast<const uint8_t*>(k_host) + static_cast<size_t>(h0) * D_QK * 2;
+        const uint8_t* vh = static_cast<const uint8_t*>(v_host) + static_cast<size_t>(h0) * D_V * 2;
+        const uint8_t* doh = static_cast<const uint8_t*>(dout_host) + static_cast<size_t>(h0) * D_V * 2;
+        if (copy2d(q + oqk, wqk, qh, pqk, wqk, cudaMemcpyHostToDevice, pipe->in) ||
+            copy2d(k + oqk, wqk, kh, pqk, wqk, cudaMemcpyHostToDevice, pipe->in) ||
+            copy2d(v + ov, wv, vh, pv, wv, cudaMemcpyHostToDevice, pipe->in) ||
+            copy2d(dout + ov, wv, doh, pv, wv, cudaMemcpyHostToDevice, pipe->in) ||
+            cudaEventRecord(pipe->in_done[g], pipe->in))
+            return HYDRA_ERR_CUDA;
+    }
+    for (int32_t g = 0; g < n_groups; ++g) {
+        const int32_t h0 = g * hg, hn = std::min(hg, n_heads - h0);
+        const size_t oqk = T * h0 * D_QK * 2, ov = T * h0 * D_V * 2;
+        const size_t wqk = static_cast<size_t>(hn) * D_QK * 2, wv = static_cast<size_t>(hn) * D_V * 2;
+        const size_t pqk = static_cast<size_t>(n_heads) * D_QK * 2, pv = static_cast<size_t>(n_heads) * D_V * 2;
+        float* lse_g = reinterpret_cast<float*>(lse + lse_off[g]);
+        if (cudaStreamWaitEvent(stream, pipe->in_done[g], 0)) return HYDRA_ERR_CUDA;
+        if (int32_t s = hydra_attn_fwd(q + oqk, k + oqk, v + ov, cu, n_seqs, hn, pairs, n_pairs, causal, softmax_scale,
+                                       out + ov, lse_g, any_part ? o_part : nullptr, any_part ? lse_part : nullptr,
+                                       part_rows, ws, ws_bytes, cuda_stream))
+            return s;
+        if (any_part)
+            if (int32_t s = hydra_lse_merge(o_part, lse_part, part_rows, cu, n_seqs, hn, pairs, n_pairs, out + ov,
+                                            lse_g, ws, ws_bytes, cuda_stream))
+                return s;
+        if (int32_t s = hydra_attn_bwd(q + oqk, k + oqk, v + ov, out + ov, lse_g, dout + ov, cu, n_seqs, hn, pairs,
+                                       n_pairs, causal, softmax_scale, dq_ + oqk, dk_ + oqk, dv_ + ov, ws, ws_bytes,
+                                       cuda_stream))
+            return s;
+        uint8_t* outh = static_cast<uint8_t*>(out_host) + static_cast<size_t>(h0) * D_V * 2;
+        uint8_t* dqh = static_cast<uint8_t*>(dq_host) + static_cast<size_t>(h0) * D_QK * 2;
+        uint8_t* dkh = static_cast<uint8_t*>(dk_host) + static_cast<size_t>(h0) * D_QK * 2;
+        uint8_t* dvh = static_cast<uint8_t*>(dv_host) + static_cast<size_t>(h0) * D_V * 2;
+        if (cudaEventRecord(pipe->comp_done[g], stream) || cudaStreamWaitEvent(pipe->out, pipe->comp_done[g], 0) ||
+            copy2d(outh, pv, out + ov, wv, wv, cudaMemcpyDeviceToHost, pipe->out) ||
+            cudaMemcpyAsync(lse_host + T * h0, lse_g, T * hn * 4, cudaMemcpyDeviceToHost, pipe->out) ||
+            copy2d(dqh, pqk, dq_ + oqk, wqk, wqk, cudaMemcpyDeviceToHost, pipe->out) ||
+            copy2d(dkh, pqk, dk_ + oqk, wqk, wqk, cudaMemcpyDeviceToHost, pipe->out) ||
+            copy2d(dvh, pv, dv_ + ov, wv, wv, cudaMemcpyDeviceToHost, pipe->out))
+            return HYDRA_ERR_CUDA;
+    }
+    // the caller's stream completes when the last copy out has completed
+    if (cudaEventRecord(pipe->end, pipe->out) || cudaStreamWaitEvent(stream, pipe->end, 0)) return HYDRA_ERR_CUDA;
     return HYDRA_OK;
 }
 

@@ -1,0 +1,59 @@
+"""The whole step through the C ABI with HOST buffers (`hydra_attn_fwd_bwd_host`) against the oracle.
+
+The entry point pipelines groups of heads over two internal copy streams; the cases cover a head count
+that splits into full groups plus a remainder, a single group, chunked pairs through the merge, and
+two calls in a row on the same arena (the internal streams and events are reused).
+"""
+import numpy as np
+import pytest
+
+import hydra_workloads as hw
+from gpu_util import check, pairs_for, run_oracle
+
+pytestmark = pytest.mark.gpu
+DQK, DV = hw.D_QK, hw.D_V
+
+
+def rand_inputs(rng, T, h):
+    f = lambda d: hw.f32_to_bf16_bits(rng.standard_normal((T, h, d)).astype(np.float32))
+    return dict(q=f(DQK), k=f(DQK), v=f(DV), do=f(DV))
+
+
+def host_step(x, cu, h, lib_pairs, calls=1):
+    import torch
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.runner import bits_to_tensor
+    T = int(cu[-1])
+    host = {n: bits_to_tensor(x[n]).cpu().pin_memory() for n in ("q", "k", "v", "do")}
+    nan16 = lambda d: torch.full((T, h, d), float("nan"), dtype=torch.bfloat16).pin_memory()
+    ho = dict(out=nan16(DV), lse=torch.full((h, T), float("nan"), dtype=torch.float32).pin_memory(),
+              dq=nan16(DQK), dk=nan16(DQK), dv=nan16(DV))
+    arena = torch.empty(P.hydra_host_step_arena_bytes(cu, h, lib_pairs) + 256, dtype=torch.uint8, device="cuda")
+    off = (-arena.data_ptr()) % 256
+    scale = float(np.float32(1.0 / np.sqrt(np.float32(DQK))))
+    for _ in range(calls):
+        P.hydra_attn_fwd_bwd_host(host["q"], host["k"], host["v"], host["do"], cu, h, lib_pairs, True, scale,
+                                  ho["out"], ho["lse"], ho["dq"], ho["dk"], ho["dv"],
+                                  arena.data_ptr() + off, arena.numel() - off)
+    torch.cuda.synchronize()
+    return {n: t.float().numpy().astype(np.float64) for n, t in ho.items()}
+
+
+@pytest.mark.parametrize("h,cp_r", [(9, 0), (3, 0), (8, 1), (6, 2)])
+def test_host_step_matches_the_oracle(h, cp_r):
+    lengths = [130, 257, 64, 1, 300]
+    cu = hw.cu_seqlens(lengths)
+    x = rand_inputs(np.random.default_rng(100 + h), int(cu[-1]), h)
+    lib_pairs, _, ora_pairs = pairs_for(cu, cp_r) if cp_r else (None, 0, None)
+    got = host_step(x, cu, h, lib_pairs)
+    ref = run_oracle(x, cu, True, pairs=ora_pairs)
+    check(got, ref, label=f"host step h={h} cp_r={cp_r}: ")
+
+
+def test_two_host_steps_in_a_row_give_the_same_bits():
+    cu = hw.cu_seqlens([200, 513])
+    x = rand_inputs(np.random.default_rng(7), int(cu[-1]), 12)
+    once = host_step(x, cu, 12, None, calls=1)
+    twice = host_step(x, cu, 12, None, calls=2)
+    for n in once:
+        assert np.array_equal(once[n], twice[n], equal_nan=True), n
