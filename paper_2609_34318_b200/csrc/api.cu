@@ -179,7 +179,6 @@ struct Plan {
     int kind = 0, device = 0;
     DeviceBlob blob;
     size_t off_pairs = 0, off_items = 0, off_lists = 0, off_groups = 0, off_items2 = 0, off_lists2 = 0;
-    size_t off_cta = 0, off_cta2 = 0;
     int32_t n_items = 0, n_items2 = 0;
 };
 
@@ -187,14 +186,14 @@ std::mutex g_plan_mutex;
 std::vector<std::unique_ptr<Plan>> g_plans;
 constexpr size_t kMaxPlans = 32;
 
-std::vector<uint8_t> make_key(int kind, int device, const Problem& pb, int causal, int n_ctas)
+std::vector<uint8_t> make_key(int kind, int device, const Problem& pb, int causal)
 {
     std::vector<uint8_t> key;
     auto put = [&](const void* p, size_t n) {
         const uint8_t* b = static_cast<const uint8_t*>(p);
         key.insert(key.end(), b, b + n);
     };
-    const int32_t head[6] = {kind, device, pb.h, causal, pb.n_seqs, n_ctas};
+    const int32_t head[6] = {kind, device, pb.h, causal, pb.n_seqs, 0};
     put(head, sizeof head);
     put(pb.cu.data(), pb.cu.size() * sizeof(int32_t));
     put(pb.pairs.data(), pb.pairs.size() * sizeof(hydra_pair_t));
@@ -232,53 +231,12 @@ inline int32_t kv_tiles(const hydra_pair_t& p, int32_t q0, int causal, int32_t r
 // Order: blocks of items that share their operands (same pair/chunk and head) stay together so
 // that CTAs running at the same time hit the same K/V (or Q/dO) tiles in L2; blocks go
 // longest-first, and inside a block items go longest-first too (the quadratic load model of
-// Sections 3.2 / 5.1: cost ~ number of inner tiles).
-// The ordered list is then dealt to the `n_ctas` persistent CTAs: each item, in order, goes to the
-// CTA with the least accumulated cost (what a run-time work queue would do under the cost model), so
-// every CTA ends with nearly the same load while CTAs still walk the blocks in the same order.
-// Returns the items grouped by CTA and `cta_off` with n_ctas + 1 offsets.
+// Sections 3.2 / 5.1: cost ~ number of inner tiles). The persistent CTAs pop items from a counter in
+// this order at run time, so a CTA that finishes early takes more items and nothing has to predict
+// how long an item runs.
 struct Keyed { int64_t block_cost; int32_t block; int32_t cost; int32_t idx; };
 template <class Item>
-void order_items(std::vector<Item>& items, const std::vector<int32_t>& block_of,
-                 const std::vector<int32_t>& cost, int n_ctas, std::vector<int32_t>& cta_off);
-
-template <class Item>
-void order_items_impl(std::vector<Item>& items, const std::vector<int32_t>& block_of,
-                      const std::vector<int32_t>& cost, std::vector<int32_t>& sorted_cost);
-
-template <class Item>
-void order_items(std::vector<Item>& items, const std::vector<int32_t>& block_of,
-                 const std::vector<int32_t>& cost, int n_ctas, std::vector<int32_t>& cta_off)
-{
-    std::vector<int32_t> sorted_cost;
-    order_items_impl(items, block_of, cost, sorted_cost);
-    // least-loaded CTA first; ties broken by CTA index so the deal is deterministic
-    using Slot = std::pair<int64_t, int32_t>;
-    std::vector<Slot> heap;
-    for (int32_t c = 0; c < n_ctas; ++c) heap.emplace_back(0, c);
-    auto cmp = [](const Slot& a, const Slot& b) { return a > b; };
-    std::make_heap(heap.begin(), heap.end(), cmp);
-    std::vector<int32_t> owner(items.size());
-    std::vector<int32_t> count(n_ctas, 0);
-    for (size_t i = 0; i < items.size(); ++i) {
-        std::pop_heap(heap.begin(), heap.end(), cmp);
-        Slot& s = heap.back();
-        owner[i] = s.second;
-        ++count[s.second];
-        s.first += sorted_cost[i] + 1;              // + 1: fixed cost of starting an item
-        std::push_heap(heap.begin(), heap.end(), cmp);
-    }
-    cta_off.assign(n_ctas + 1, 0);
-    for (int32_t c = 0; c < n_ctas; ++c) cta_off[c + 1] = cta_off[c] + count[c];
-    std::vector<int32_t> cursor(cta_off.begin(), cta_off.end() - 1);
-    std::vector<Item> dealt(items.size());
-    for (size_t i = 0; i < items.size(); ++i) dealt[cursor[owner[i]]++] = items[i];
-    items.swap(dealt);
-}
-
-template <class Item>
-void order_items_impl(std::vector<Item>& items, const std::vector<int32_t>& block_of,
-                      const std::vector<int32_t>& cost, std::vector<int32_t>& sorted_cost)
+void order_items(std::vector<Item>& items, const std::vector<int32_t>& block_of, const std::vector<int32_t>& cost)
 {
     int32_t n_blocks = 0;
     for (int32_t b : block_of) n_blocks = std::max(n_blocks, b + 1);
@@ -294,15 +252,11 @@ void order_items_impl(std::vector<Item>& items, const std::vector<int32_t>& bloc
         return a.idx < b.idx;
     });
     std::vector<Item> sorted(items.size());
-    sorted_cost.resize(items.size());
-    for (size_t i = 0; i < items.size(); ++i) {
-        sorted[i] = items[k[i].idx];
-        sorted_cost[i] = k[i].cost;
-    }
+    for (size_t i = 0; i < items.size(); ++i) sorted[i] = items[k[i].idx];
     items.swap(sorted);
 }
 
-void build_fwd(const Problem& pb, int causal, int n_ctas, Plan& plan, std::vector<uint8_t>& blob)
+void build_fwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& blob)
 {
     std::vector<FwdItem> items;
     std::vector<int32_t> block_of, cost;
@@ -323,11 +277,9 @@ void build_fwd(const Problem& pb, int causal, int n_ctas, Plan& plan, std::vecto
             }
         }
     }
-    std::vector<int32_t> cta_off;
-    order_items(items, block_of, cost, n_ctas, cta_off);
+    order_items(items, block_of, cost);
     plan.off_pairs = append(blob, device_pairs(pb));
     plan.off_items = append(blob, items);
-    plan.off_cta = append(blob, cta_off);
     plan.n_items = static_cast<int32_t>(items.size());
 }
 
@@ -361,11 +313,10 @@ void build_merge(const Problem& pb, Plan& plan, std::vector<uint8_t>& blob)
 }
 
 // Backward lists: pairs grouped by q chunk (dQ kernel) and by kv chunk (dK/dV kernel).
-void build_bwd(const Problem& pb, int causal, int n_ctas, Plan& plan, std::vector<uint8_t>& blob)
+void build_bwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& blob)
 {
     const int32_t n = static_cast<int32_t>(pb.pairs.size());
-    auto group_by = [&](bool by_q, std::vector<int32_t>& lists, std::vector<GroupItem>& items,
-                        std::vector<int32_t>& cta_off) {
+    auto group_by = [&](bool by_q, std::vector<int32_t>& lists, std::vector<GroupItem>& items) {
         std::vector<int32_t> order(n);
         for (int32_t i = 0; i < n; ++i) order[i] = i;
         auto key = [&](int32_t i) {
@@ -419,29 +370,27 @@ void build_bwd(const Problem& pb, int causal, int n_ctas, Plan& plan, std::vecto
             }
             i = j;
         }
-        order_items(items, block_of, cost, n_ctas, cta_off);
+        order_items(items, block_of, cost);
     };
-    std::vector<int32_t> lists_q, lists_k, cta_q, cta_k;
+    std::vector<int32_t> lists_q, lists_k;
     std::vector<GroupItem> items_q, items_k;
-    group_by(true, lists_q, items_q, cta_q);
-    group_by(false, lists_k, items_k, cta_k);
+    group_by(true, lists_q, items_q);
+    group_by(false, lists_k, items_k);
     plan.off_pairs = append(blob, device_pairs(pb));
     plan.off_lists = append(blob, lists_q);
     plan.off_items = append(blob, items_q);
     plan.off_lists2 = append(blob, lists_k);
     plan.off_items2 = append(blob, items_k);
-    plan.off_cta = append(blob, cta_q);
-    plan.off_cta2 = append(blob, cta_k);
     plan.n_items = static_cast<int32_t>(items_q.size());
     plan.n_items2 = static_cast<int32_t>(items_k.size());
 }
 
 // Returns a cached plan or builds it (cudaMalloc + synchronous upload the first time only).
-int32_t get_plan(int kind, const Problem& pb, int causal, int n_ctas, const Plan** out)
+int32_t get_plan(int kind, const Problem& pb, int causal, const Plan** out)
 {
     int device = 0;
     if (cudaGetDevice(&device) != cudaSuccess) return HYDRA_ERR_CUDA;
-    std::vector<uint8_t> key = make_key(kind, device, pb, causal, n_ctas);
+    std::vector<uint8_t> key = make_key(kind, device, pb, causal);
     std::lock_guard<std::mutex> lock(g_plan_mutex);
     for (size_t i = 0; i < g_plans.size(); ++i)
         if (g_plans[i]->key == key) {
@@ -453,9 +402,9 @@ int32_t get_plan(int kind, const Problem& pb, int causal, int n_ctas, const Plan
     plan->kind = kind;
     plan->device = device;
     std::vector<uint8_t> blob;
-    if (kind == HYDRA_WS_FWD) build_fwd(pb, causal, n_ctas, *plan, blob);
+    if (kind == HYDRA_WS_FWD) build_fwd(pb, causal, *plan, blob);
     else if (kind == HYDRA_WS_MERGE) build_merge(pb, *plan, blob);
-    else build_bwd(pb, causal, n_ctas, *plan, blob);
+    else build_bwd(pb, causal, *plan, blob);
     if (plan->blob.upload(blob) != cudaSuccess) return HYDRA_ERR_CUDA;
     plan->key.swap(key);
     if (g_plans.size() >= kMaxPlans) {
@@ -694,7 +643,7 @@ int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_
     const int n_clusters = fwd_max_clusters();        // CTA pairs resident at once: the persistent grid
     if (n_clusters < 1) return HYDRA_ERR_CUDA;
     const Plan* plan = nullptr;
-    if (int32_t s = get_plan(HYDRA_WS_FWD, pb, causal != 0, n_clusters, &plan)) return s;
+    if (int32_t s = get_plan(HYDRA_WS_FWD, pb, causal != 0, &plan)) return s;
     if (plan->n_items == 0) return HYDRA_OK;
     // each CTA of a pair stages 64 kv rows of K (box of 64 rows) and 64 value columns of V
     CUtensorMap mq, mk, mv;
@@ -706,7 +655,6 @@ int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_
     fp.pairs = at<PairDev>(*plan, plan->off_pairs);
     fp.items = at<FwdItem>(*plan, plan->off_items);
     fp.n_items = plan->n_items;
-    fp.cta_off = at<int32_t>(*plan, plan->off_cta);
     fp.out = out; fp.lse = lse; fp.o_part = o_part; fp.lse_part = lse_part;
     fp.T = pb.T; fp.part_rows = part_rows; fp.h = n_heads; fp.causal = causal != 0;
     fp.scale_log2 = softmax_scale * 1.4426950408889634f;
@@ -739,7 +687,7 @@ int32_t hydra_lse_merge(const void* o_part, const float* lse_part, int64_t part_
     int sms = 0;
     if (int32_t s = device_info(&sms)) return s;
     const Plan* plan = nullptr;
-    if (int32_t s = get_plan(HYDRA_WS_MERGE, pb, 0, sms, &plan)) return s;
+    if (int32_t s = get_plan(HYDRA_WS_MERGE, pb, 0, &plan)) return s;
     MergeParams mp{};
     mp.groups = at<MergeGroup>(*plan, plan->off_groups);
     mp.lists = at<int32_t>(*plan, plan->off_lists);
@@ -783,7 +731,7 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
     int sms = 0;
     if (int32_t s = device_info(&sms)) return s;
     const Plan* plan = nullptr;
-    if (int32_t s = get_plan(HYDRA_WS_BWD, pb, causal != 0, sms, &plan)) return s;
+    if (int32_t s = get_plan(HYDRA_WS_BWD, pb, causal != 0, &plan)) return s;
 
     float* dsum = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kStatusBytes);
     CUtensorMap mq, mk, mv, mdo, mq_sub, mdo_sub;
@@ -809,7 +757,6 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
         bp.lists = at<int32_t>(*plan, plan->off_lists2);
         bp.items = at<GroupItem>(*plan, plan->off_items2);
         bp.n_items = plan->n_items2;
-        bp.cta_off = at<int32_t>(*plan, plan->off_cta2);
         ScopedKernelTimer timer(K_DKV, stream);
         if (launch_bwd_dkv(mq_sub, mk, mv, mdo_sub, bp, sms, stream) != cudaSuccess)
             return HYDRA_ERR_CUDA;
@@ -819,7 +766,6 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
         bp.lists = at<int32_t>(*plan, plan->off_lists);
         bp.items = at<GroupItem>(*plan, plan->off_items);
         bp.n_items = plan->n_items;
-        bp.cta_off = at<int32_t>(*plan, plan->off_cta);
         ScopedKernelTimer timer(K_DQ, stream);
         if (launch_bwd_dq(mq, mk, mv, mdo, bp, sms, stream) != cudaSuccess)
             return HYDRA_ERR_CUDA;

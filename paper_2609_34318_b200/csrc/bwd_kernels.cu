@@ -31,6 +31,7 @@ constexpr int kWarpProd = 8, kWarpMma = 9, kWarpMma2 = 10;
 constexpr uint32_t kBox128 = 128 * 128;   // [128 rows x 64 bf16]
 constexpr uint32_t kBox64 = 64 * 128;     // [ 64 rows x 64 bf16]
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kSched = 4;                  // depth of the in-CTA ring of work-item indices
 
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
 __device__ __forceinline__ float pos_inf() { return __int_as_float(0x7f800000); }
@@ -64,7 +65,7 @@ constexpr uint32_t kTmS = 0, kTmDP = 128, kTmDQ = 256, kTmDS = 448, kTmCols = 51
 // when the first 16 KB have landed instead of waiting for all 48 KB of the stage.
 enum : int { B_QFULL = 0, B_QEMPTY = 1, B_KFULL = 2, B_KEMPTY = 8, B_VFULL = 10, B_VEMPTY = 13,
              B_SFULL = 16, B_SFREE = 17, B_PFULL = 18, B_DSFREE = 20, B_ACCFREE = 21, B_DPFULL = 22, B_DPFREE = 23,
-             B_COUNT = 24 };
+             B_ITEMFULL = 24, B_ITEMEMPTY = 24 + kSched, B_COUNT = 24 + 2 * kSched };
 
 // Iterator over (pair of the q chunk, kv tile) in the order every role walks them.
 struct TileIter {
@@ -105,7 +106,8 @@ constexpr uint32_t kTotal = kDO + kStages * 2 * kBox64;      // 204,800 B
 constexpr uint32_t kTmDK = 0, kTmDV = 192, kTmS = 320, kTmDP = 384, kTmP = 448, kTmDS = 480,
                    kTmCols = 512;
 enum : int { B_KVFULL = 0, B_KVEMPTY = 1, B_QFULL = 2, B_STAT = 5, B_QEMPTY = 8, B_SFULL = 11,
-             B_SFREE = 12, B_PFULL = 13, B_PDSFREE = 14, B_ACCFREE = 15, B_COUNT = 16 };
+             B_SFREE = 12, B_PFULL = 13, B_PDSFREE = 14, B_ACCFREE = 15, B_ITEMFULL = 16, B_ITEMEMPTY = 16 + kSched,
+             B_COUNT = 16 + 2 * kSched };
 
 // Iterator over (pair of the kv chunk, 64-row q sub-tile).
 struct SubIter {
@@ -149,6 +151,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     __shared__ __align__(8) uint64_t bars[B_COUNT];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ int32_t s_sched[kSched];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t bar0 = smem_u32(&bars[0]);
@@ -158,7 +161,8 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         for (int i = 0; i < B_COUNT; ++i) {
             const bool by_threads = (i == B_SFREE) || (i == B_DPFREE) || (i == B_PFULL) || (i == B_PFULL + 1) ||
                                     (i == B_ACCFREE);
-            mbar_init(bar(i), by_threads ? 8u : 1u);   // 8 = elementwise warps
+            const bool by_readers = i >= B_ITEMEMPTY && i < B_ITEMEMPTY + kSched;
+            mbar_init(bar(i), by_readers ? 10u : (by_threads ? 8u : 1u));   // 8 elementwise warps (+ 2 issuers)
         }
         fence_mbar_init();
         tma_prefetch_desc(&map_q); tma_prefetch_desc(&map_k);
@@ -170,16 +174,40 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     tc_fence_after_sync();
     const uint32_t tm = tmem_base_slot;
     const uint64_t limit = p.wait_limit_ns;
-    const int it_begin = p.cta_off[blockIdx.x], it_end = p.cta_off[blockIdx.x + 1];
     volatile int* abort_p = &abort_flag;
     auto wait = [&](int b, uint32_t parity) -> bool { return mbar_wait(bar(b), parity & 1u, abort_p, limit); };
+    // Work queue: the producer pops the next item index from a counter in global memory (so a CTA that
+    // finishes early simply takes more items: no cost model has to predict the run time of an item)
+    // and hands it to the other warps of the CTA through a small ring in shared memory.
+    volatile int32_t* sched = s_sched;
+    auto pop_item = [&](uint32_t k) -> int {                 // producer, one thread
+        const int slot = k % kSched;
+        if (!mbar_wait(bar(B_ITEMEMPTY + slot), ((k / kSched) ^ 1u) & 1u, abort_p, limit)) return -1;
+        int idx = atomicAdd(&p.status->next_item[QUEUE_DQ], 1);
+        if (idx >= p.n_items) idx = -1;
+        sched[slot] = idx;
+        mbar_arrive(bar(B_ITEMFULL + slot));
+        return idx;
+    };
+    auto next_item = [&](uint32_t k) -> int {                // every other warp, all lanes
+        const int slot = k % kSched;
+        if (!mbar_wait(bar(B_ITEMFULL + slot), (k / kSched) & 1u, abort_p, limit)) return -1;
+        const int idx = sched[slot];
+        mbar_arrive_warp(bar(B_ITEMEMPTY + slot));
+        return idx;
+    };
 
     if (warp == kWarpProd) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t items = 0, gk = 0, gv = 0;
             bool ok = true;
-            for (int it = it_begin; it < it_end && ok; ++it) {
+            // one item ahead: the round trip to the counter overlaps the loads of the current item
+            int it_ahead = pop_item(0);
+            for (uint32_t kq = 0; ok; ++kq) {
+                const int it = it_ahead;
+                if (it < 0) break;
+                it_ahead = pop_item(kq + 1);
                 const GroupItem item = p.items[it];
                 const int32_t* list = p.lists + item.list_off;
                 const PairDev first = p.pairs[list[0]];
@@ -238,7 +266,9 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const bool issue_scores = warp == kWarpMma;
             uint32_t items = 0, n_tile = 0, gv = 0;       // running counts of this issuer
             bool ok = true;
-            for (int it = it_begin; it < it_end && ok; ++it) {
+            for (uint32_t kq = 0; ok; ++kq) {
+                const int it = next_item(kq);
+                if (it < 0) break;
                 const GroupItem item = p.items[it];
                 const int32_t* list = p.lists + item.list_off;
                 const PairDev first = p.pairs[list[0]];
@@ -340,7 +370,9 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const uint32_t tm_ds = tm + kTmDS + lane_base + g * 32;
         uint32_t c_s = 0, c_ds = 0;
         bool ok = true;
-        for (int it = it_begin; it < it_end && ok; ++it) {
+        for (uint32_t kq = 0; ok; ++kq) {
+            const int it = next_item(kq);
+            if (it < 0) break;
             const GroupItem item = p.items[it];
             const int32_t* list = p.lists + item.list_off;
             const PairDev first = p.pairs[list[0]];
@@ -478,6 +510,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     __shared__ __align__(8) uint64_t bars[B_COUNT];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ int32_t s_sched[kSched];
     __shared__ float s_lse2[kStages][SUB];
     __shared__ float s_dsum[kStages][SUB];
     __shared__ uint32_t s_bursts;                      // S / dP bursts issued so far (all ones: no more)
@@ -491,6 +524,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         for (int i = 0; i < B_COUNT; ++i) {
             uint32_t count = 1u;
             if (i == B_SFREE || i == B_PFULL || i == B_ACCFREE) count = 8u;   // elementwise warps
+            if (i >= B_ITEMEMPTY && i < B_ITEMEMPTY + kSched) count = 10u;   // + the two issuer warps
             
             mbar_init(bar(i), count);
         }
@@ -504,16 +538,44 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     tc_fence_after_sync();
     const uint32_t tm = tmem_base_slot;
     const uint64_t limit = p.wait_limit_ns;
-    const int it_begin = p.cta_off[blockIdx.x], it_end = p.cta_off[blockIdx.x + 1];
     volatile int* abort_p = &abort_flag;
     auto wait = [&](int b, uint32_t parity) -> bool { return mbar_wait(bar(b), parity & 1u, abort_p, limit); };
+    // Work queue: the producer pops the next item index from a counter in global memory (so a CTA that
+    // finishes early simply takes more items: no cost model has to predict the run time of an item)
+    // and hands it to the other warps of the CTA through a small ring in shared memory.
+    volatile int32_t* sched = s_sched;
+    auto pop_item = [&](uint32_t k) -> int {                 // producer, one thread
+        const int slot = k % kSched;
+        if (!mbar_wait(bar(B_ITEMEMPTY + slot), ((k / kSched) ^ 1u) & 1u, abort_p, limit)) return -1;
+        int idx = atomicAdd(&p.status->next_item[QUEUE_DKV], 1);
+        if (idx >= p.n_items) idx = -1;
+        sched[slot] = idx;
+        mbar_arrive(bar(B_ITEMFULL + slot));
+        return idx;
+    };
+    auto next_item = [&](uint32_t k) -> int {                // every other warp, all lanes
+        const int slot = k % kSched;
+        if (!mbar_wait(bar(B_ITEMFULL + slot), (k / kSched) & 1u, abort_p, limit)) return -1;
+        const int idx = sched[slot];
+        mbar_arrive_warp(bar(B_ITEMEMPTY + slot));
+        return idx;
+    };
     volatile uint32_t* bursts_p = &s_bursts;
 
     if (warp == kWarpProd) {
         // ------------------------------------------------------------------ TMA producer + LSE / D
         uint32_t items = 0, gq = 0;
         bool ok = true;
-        for (int it = it_begin; it < it_end && ok; ++it) {
+        int it_ahead = -1;
+        for (uint32_t kq = 0; ok; ++kq) {
+            int it = 0;
+            if (lane == 0) {                          // one pop per CTA, one item ahead, shared with the other lanes
+                if (kq == 0) it_ahead = pop_item(0);
+                it = it_ahead;
+                if (it >= 0) it_ahead = pop_item(kq + 1);
+            }
+            it = __shfl_sync(0xffffffffu, it, 0);
+            if (it < 0) break;
             const GroupItem item = p.items[it];
             const int32_t* list = p.lists + item.list_off;
             const PairDev first = p.pairs[list[0]];
@@ -578,7 +640,9 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const bool issue_scores = warp == kWarpMma;
             uint32_t items = 0, n_step = 0;
             bool ok = true;
-            for (int it = it_begin; it < it_end && ok; ++it) {
+            for (uint32_t kq = 0; ok; ++kq) {
+                const int it = next_item(kq);
+                if (it < 0) break;
                 const GroupItem item = p.items[it];
                 const int32_t* list = p.lists + item.list_off;
                 SubIter si;
@@ -658,7 +722,9 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const uint32_t tm_ds = tm + kTmDS + lane_base + g * 16;
         uint32_t c_s = 0, c_pds = 0, gq = 0;
         bool ok = true;
-        for (int it = it_begin; it < it_end && ok; ++it) {
+        for (uint32_t kq = 0; ok; ++kq) {
+            const int it = next_item(kq);
+            if (it < 0) break;
             const GroupItem item = p.items[it];
             const int32_t* list = p.lists + item.list_off;
             const PairDev first = p.pairs[list[0]];

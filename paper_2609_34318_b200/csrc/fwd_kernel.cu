@@ -47,9 +47,12 @@ constexpr uint32_t kSmemTotal = kSmemV + kVStages * kVStage;  // 221,184 B
 constexpr uint32_t kTmS = 0, kTmO = 256, kTmCols = 512;
 constexpr float kRescaleThreshold = 8.f;              // log2 units
 
+constexpr int kSched = 4;                             // depth of the in-cluster ring of work-item indices
+
 enum : int {
     B_QFULL = 0, B_QEMPTY = 2, B_KFULL = 4, B_KEMPTY = 7, B_VFULL = 10, B_VEMPTY = 13,
-    B_SFULL = 16, B_PFULL = 18, B_OFULL = 20, B_OFREE = 22, B_PFULL2 = 24, B_COUNT = 26
+    B_SFULL = 16, B_PFULL = 18, B_OFULL = 20, B_OFREE = 22, B_PFULL2 = 24,
+    B_ITEMFULL = 26, B_ITEMEMPTY = 26 + kSched, B_COUNT = 26 + 2 * kSched
 };
 
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
@@ -67,6 +70,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     __shared__ __align__(8) uint64_t bars[B_COUNT];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
+    __shared__ int32_t s_sched[kSched];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_cta_rank();
@@ -80,7 +84,10 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             // P-ready and O-drained collect the 4 softmax warps of a tile in each of the 2 CTAs
             const bool by_warps = (i >= B_PFULL && i < B_PFULL + 2) || (i >= B_OFREE && i < B_OFREE + 2) ||
                                   (i >= B_PFULL2 && i < B_PFULL2 + 2);
-            mbar_init(bar(i), by_warps ? 8u : 1u);
+            // an item slot is free again when every reader of both CTAs has taken the index: 8 softmax
+            // warps and 2 single-thread roles per CTA
+            const bool by_readers = i >= B_ITEMEMPTY && i < B_ITEMEMPTY + kSched;
+            mbar_init(bar(i), by_readers ? 20u : (by_warps ? 8u : 1u));
         }
         fence_mbar_init();
         tma_prefetch_desc(&map_q); tma_prefetch_desc(&map_k); tma_prefetch_desc(&map_v);
@@ -92,17 +99,50 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     tc_fence_after_sync();
     const uint32_t tm = tmem_base_slot;
     const uint64_t limit = p.wait_limit_ns;
-    const int cluster = static_cast<int>(cluster_id_x());
-    const int it_begin = p.cta_off[cluster], it_end = p.cta_off[cluster + 1];
     volatile int* abort_p = &abort_flag;
     auto wait = [&](int b, uint32_t parity) -> bool { return mbar_wait(bar(b), parity & 1u, abort_p, limit); };
+    // Work queue: the leader's producer pops the next item index from a counter in global memory (a
+    // cluster that finishes early simply takes more items: no cost model has to predict the run time
+    // of an item) and hands it to every other role of both CTAs through a small ring that exists in
+    // both CTAs' shared memory.
+    volatile int32_t* sched = s_sched;
+    auto pop_item = [&](uint32_t k) -> int {                 // leader CTA, one thread
+        const int slot = k % kSched;
+        if (!mbar_wait(bar(B_ITEMEMPTY + slot), ((k / kSched) ^ 1u) & 1u, abort_p, limit)) return -1;
+        int idx = atomicAdd(&p.status->next_item[QUEUE_FWD], 1);
+        if (idx >= p.n_items) idx = -1;
+        for (uint32_t r = 0; r < 2; ++r) {
+            st_shared_cluster_s32(cluster_map_shared(smem_u32(&s_sched[slot]), r), idx);
+            mbar_arrive_cluster_release(cluster_map_shared(bar(B_ITEMFULL + slot), r));
+        }
+        return idx;
+    };
+    auto next_item = [&](uint32_t k, bool whole_warp) -> int {   // every other role, either CTA
+        const int slot = k % kSched;
+        if (!mbar_wait_acquire_cluster(bar(B_ITEMFULL + slot), (k / kSched) & 1u, abort_p, limit)) return -1;
+        const int idx = sched[slot];
+        if (whole_warp) mbar_arrive_warp_leader(bar(B_ITEMEMPTY + slot));
+        else mbar_arrive_leader(bar(B_ITEMEMPTY + slot));
+        return idx;
+    };
 
     if (warp == kWarpK) {
         // ------------------------------------------------------------------ Q and K producer
         if (lane == 0) {
             uint32_t gk = 0, q_use[2] = {0, 0};
             bool ok = true;
-            for (int it = it_begin; it < it_end && ok; ++it) {
+            // the leader pops one item ahead: the round trip to the counter and the hand-over to the
+            // other CTA then overlap the loads of the current item
+            int it_ahead = leader ? pop_item(0) : 0;
+            for (uint32_t kq = 0; ok; ++kq) {
+                int it;
+                if (leader) {
+                    it = it_ahead;
+                    if (it >= 0) it_ahead = pop_item(kq + 1);
+                } else {
+                    it = next_item(kq, false);
+                }
+                if (it < 0) break;
                 const FwdItem item = p.items[it];
                 const PairDev pr = p.pairs[item.pair];
                 const int n_t[2] = {item.n_a, item.n_b};
@@ -133,7 +173,9 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (lane == 0) {
             uint32_t gv = 0;
             bool ok = true;
-            for (int it = it_begin; it < it_end && ok; ++it) {
+            for (uint32_t kq = 0; ok; ++kq) {
+                const int it = next_item(kq, false);
+                if (it < 0) break;
                 const FwdItem item = p.items[it];
                 const PairDev pr = p.pairs[item.pair];
                 const int n = max(item.n_a, item.n_b);
@@ -161,7 +203,9 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             uint32_t vs = 0, vp = 0, vs_prev = 0, vp_prev = 0;   // same for V, tiles j and j-1
             uint32_t q_use[2] = {0, 0}, c_p[2] = {0, 0}, free_use[2] = {0, 0};
             bool ok = true;
-            for (int it = it_begin; it < it_end && ok; ++it) {
+            for (uint32_t kq = 0; ok; ++kq) {
+                const int it = next_item(kq, false);
+                if (it < 0) break;
                 const FwdItem item = p.items[it];
                 const int n_t[2] = {item.n_a, item.n_b};
                 const int n = max(item.n_a, item.n_b);
@@ -250,7 +294,9 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         const uint32_t tm_o = tm + kTmO + t * D_V + lane_base;
         uint32_t c_s = 0, c_o = 0;
         bool ok = true;
-        for (int it = it_begin; it < it_end && ok; ++it) {
+        for (uint32_t kq = 0; ok; ++kq) {
+            const int it = next_item(kq, true);
+            if (it < 0) break;
             const FwdItem item = p.items[it];
             const PairDev pr = p.pairs[item.pair];
             const int n_kv = t == 0 ? item.n_a : item.n_b;

@@ -56,16 +56,17 @@ struct MergeItem {
 };
 constexpr int MERGE_ROWS = 8;   // rows of a merge block
 
-struct StatusBlock {            // lives at the start of the workspace
+struct StatusBlock {            // lives at the start of the workspace; zeroed before every call
     int32_t status;
     int32_t pad;
     int64_t detail;
+    int32_t next_item[4];       // work-queue heads of the persistent kernels (forward, dK/dV, dQ)
 };
+enum : int { QUEUE_FWD = 0, QUEUE_DKV = 1, QUEUE_DQ = 2 };
 
 struct FwdParams {
     const PairDev* pairs;
     const FwdItem* items;
-    const int32_t* cta_off;     // items [cta_off[b], cta_off[b+1]) belong to CTA b
     int32_t n_items;
     void* out; float* lse; void* o_part; float* lse_part;
     int64_t T; int64_t part_rows;
@@ -79,7 +80,6 @@ struct BwdParams {
     const PairDev* pairs;
     const int32_t* lists;       // pair indices, grouped by chunk
     const GroupItem* items;
-    const int32_t* cta_off;     // items [cta_off[b], cta_off[b+1]) belong to CTA b
     int32_t n_items;
     const float* lse; const float* dsum;   // [h, T]
     void* dq; void* dk; void* dv;

@@ -454,6 +454,50 @@ __device__ __forceinline__ void mbar_arrive_warp_leader(uint32_t bar) {
     __syncwarp();
     if ((threadIdx.x & 31u) == 0u) mbar_arrive_leader(bar);
 }
+// A word handed from one CTA of the pair to the other through distributed shared memory: the writer
+// stores it in the reader's shared memory and then arrives, with cluster-scope release, on the
+// reader's barrier; the reader waits with cluster-scope acquire.
+__device__ __forceinline__ uint32_t cluster_map_shared(uint32_t addr, uint32_t cta_rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(cta_rank));
+    return r;
+}
+__device__ __forceinline__ void st_shared_cluster_s32(uint32_t cluster_addr, int32_t v) {
+    asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_acquire_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded, as mbar_wait.
+__device__ __forceinline__ bool mbar_wait_acquire_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                          uint64_t limit_ns) {
+    uint32_t spins = 0;
+    long long t0 = 0;
+    while (!mbar_try_wait_acquire_cluster(bar, parity)) {
+        ++spins;
+        if (spins == 256u) {
+            t0 = clock64();
+        } else if (spins > 256u && (spins & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if (static_cast<uint64_t>(clock64() - t0) > 2ull * limit_ns) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+    return true;
+}
 // Box load into THIS CTA's shared memory whose bytes are counted on the leader's barrier.
 __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
                                                  int c1, int c2) {
