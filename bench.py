@@ -376,9 +376,9 @@ def merge_groups(pairs):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised in
 # profiles/tensor_kernels_packed32k.md and profiles/merge_prep_short64k_split.md.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "fwd:packed32k": 731282432,
-    "bwd_dkv:packed32k": 1010001408,
-    "bwd_dq:packed32k": 873572864,
+    "fwd:packed32k": 685094656,
+    "bwd_dkv:packed32k": 995757056,
+    "bwd_dq:packed32k": 875597824,
     "merge:short64k_split": 764219424,
     "bwd_prep:short64k_split": 1082259656,
 }
