@@ -651,15 +651,19 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 if (issue_scores) {
                     ok = wait(B_KVFULL, items);
                     for (; si.valid() && ok;) {
-                        if (n_step > 0) ok = wait(B_SFREE, n_step - 1u);
-                        if (!ok) break;
+                        // the poll that is almost always satisfied (Q / dO landed stages ago) and the
+                        // address arithmetic come first; the wait on the critical path (S / dP of the
+                        // previous sub-tile copied out) comes last, with only the UMMAs behind it
                         const int st = n_step % kStages;
                         ok = wait(B_QFULL + st, n_step / kStages);
                         if (!ok) break;
-                        tc_fence_after_sync();
                         const uint32_t q_lo = q_lo0 + st * (3 * kBox64 >> 4), do_lo = do_lo0 + st * (2 * kBox64 >> 4);
+                        const uint32_t prev = n_step;
                         ++n_step;
                         si.next();
+                        if (prev > 0) ok = wait(B_SFREE, prev - 1u);
+                        if (!ok) break;
+                        tc_fence_after_sync();
                         if (elect_one()) {
 #pragma unroll
                             for (int kk = 0; kk < D_QK / 16; ++kk)
