@@ -19,6 +19,9 @@
  *     the first time a given (cu_seqlens, pairs, h) combination is seen, the internal cudaMalloc of
  *     its cached work lists (freed by hydra_shutdown).
  *   - The caller owns all tensors and the workspace; the library keeps no caller pointer.
+ *   - A workspace carries the status word and the work-queue counters of the kernels of one call:
+ *     each call clears them (on its stream) before it launches, so calls that may run at the same
+ *     time need workspaces of their own; calls on one stream may share one.
  *   - Inputs must be finite: a tile that straddles the end of a sequence reads (and masks) the
  *     rows of its neighbour, and 0 * NaN is NaN.
  *   - Only compute capability 10.0 is supported; there is no fallback path.
