@@ -379,8 +379,8 @@ NCU_DRAM_BYTES_PER_LAUNCH = {
     "fwd:packed32k": 685094656,
     "bwd_dkv:packed32k": 995757056,
     "bwd_dq:packed32k": 875597824,
-    "merge:short64k_split": 764219424,
-    "bwd_prep:short64k_split": 1082259656,
+    "merge:short64k_split": 764355784,
+    "bwd_prep:short64k_split": 1080946776,
 }
 
 

@@ -66,27 +66,50 @@ hydra_lse_merge_kernel(const MergeParams p)
 
     for (int u = unit0; u < rows * p.h; u += kUnitsPerPass) {
         const int r = item.row0 + u / p.h, a = u % p.h;
+        const float* lse_row = p.lse_part + static_cast<int64_t>(a) * p.part_rows + r;
+        // The first two partials (every merged chunk has at least two) are requested before anything
+        // else, together with their LSEs: one round trip to memory instead of two (all LSEs for the
+        // maximum, then O) for most chunks. The running maximum is corrected on the fly for the
+        // partials that follow.
+        const int64_t prow0 = static_cast<int64_t>(part_row[0]) + r;
+        const int64_t prow1 = static_cast<int64_t>(part_row[g.n_parts > 1 ? 1 : 0]) + r;
+        const uint4 v0 = ld_stream(o_part + (prow0 * p.h + a) * kVecPerRow + lane);
+        const uint4 v1 = ld_stream(o_part + (prow1 * p.h + a) * kVecPerRow + lane);
+        const float l0 = __ldg(lse_row + part_row[0]);
+        const float l1 = g.n_parts > 1 ? __ldg(lse_row + part_row[1]) : neg_inf();
         float m = neg_inf();
-        for (int q = 0; q < g.n_parts; ++q)
-            m = fmaxf(m, __ldg(p.lse_part + static_cast<int64_t>(a) * p.part_rows + part_row[q] + r));
         float acc[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[e] = 0.f;
         float z = 0.f;
-        if (m != neg_inf()) {
-            for (int q = 0; q < g.n_parts; ++q) {
-                const int64_t prow = static_cast<int64_t>(part_row[q]) + r;
-                const float w = __expf(__ldg(p.lse_part + static_cast<int64_t>(a) * p.part_rows + prow) - m);
-                if (w == 0.f) continue;
-                z += w;
-                float f[8];
-                unpack8(ld_stream(o_part + (prow * p.h + a) * kVecPerRow + lane), f);
+        auto add = [&](const uint4& v, float l) {          // online update: acc, z are relative to m
+            if (l == neg_inf()) return;                      // a partial that saw no key
+            if (l > m) {
+                const float c = __expf(m - l);               // 0 when m = -inf
+                z *= c;
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e] = fmaf(w, f[e], acc[e]);
+                for (int e = 0; e < 8; ++e) acc[e] *= c;
+                m = l;
             }
+            const float w = __expf(l - m);
+            z += w;
+            float f[8];
+            unpack8(v, f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = fmaf(w, f[e], acc[e]);
+        };
+        add(v0, l0);
+        add(v1, l1);
+        for (int q = 2; q < g.n_parts; ++q) {
+            const int64_t prow = static_cast<int64_t>(part_row[q]) + r;
+            add(ld_stream(o_part + (prow * p.h + a) * kVecPerRow + lane), __ldg(lse_row + part_row[q]));
+        }
+        if (z > 0.f) {
             const float inv = 1.f / z;
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] *= inv;
+        } else {
+            m = neg_inf();
         }
         const int64_t tok = static_cast<int64_t>(g.out_tok0) + r;
         out[(tok * p.h + a) * kVecPerRow + lane] = pack8(acc);
