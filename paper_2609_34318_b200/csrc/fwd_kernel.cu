@@ -23,6 +23,8 @@
 //   S_A(j) = Q_A K_j^T ; O_B += P_B(j-1) V_{j-1} ; S_B(j) = Q_B K_j^T ; O_A += P_A(j) V_j
 // The softmax keeps a running maximum in the exp2 domain and rescales O only when the maximum grew
 // by more than 2^8 (the final LSE is exact whatever reference maximum was used).
+// Items come from a run-time queue: the leader's producer pops an index from a counter in global
+// memory and hands it to every other role of both CTAs through a ring in (distributed) shared memory.
 #include <cuda_bf16.h>
 
 #include "hydra_internal.h"

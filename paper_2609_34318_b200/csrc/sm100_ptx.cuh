@@ -158,14 +158,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
-// Asks the TMA unit to pull a box into L2 only (no shared memory, no barrier): issued a few tiles
-// ahead so that the real load, which can only start once a shared-memory stage is free, hits L2.
-__device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* map, int c0, int c1, int c2) {
-    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(c0),
-                 "r"(c1), "r"(c2)
-                 : "memory");
-}
-
 // ----------------------------------------------------------------------------------------------
 // tcgen05: tensor memory
 // ----------------------------------------------------------------------------------------------
