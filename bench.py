@@ -358,6 +358,94 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_report(args, w):
+    """Per-kernel report of one workload (a JSON object on stdout, not the one-line bench contract):
+    median and best of every kernel over the repetitions, with L2 flushed between repetitions so that
+    the HBM-bound kernels are measured against HBM; fwd-only / bwd-only / total rates against the
+    measured burst, measured sustained and nominal peaks; merge and D-prep GB/s; the time of the first
+    call of the shape (plan build and upload) against a steady call; and, with --per-sequence, every
+    sequence of the batch timed alone next to its share of sum(L^2), the paper's load model."""
+    import statistics
+    import torch
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.runner import AttnStep
+
+    torch.cuda.set_device(0)
+    cu = w.cu()
+    pairs, part_rows = (None, 0)
+    if w.cp_r:
+        pairs, part_rows, _, _ = P.hydra_zigzag_pairs(cu, w.cp_r)
+    t = device_inputs(w, torch, 0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def timed_step(step, x):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        step.forward(x["q"], x["k"], x["v"])
+        step.backward(x["q"], x["k"], x["v"], x["do"])
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    t0 = time.perf_counter()
+    step = AttnStep(cu, w.n_heads, pairs, part_rows, True, float(w.scale))
+    first_ms = timed_step(step, t)
+    first_wall_ms = 1e3 * (time.perf_counter() - t0)
+    for _ in range(max(args.warmup, 3)):
+        timed_step(step, t)
+    P.hydra_profile_enable(True)
+    P.hydra_profile_collect()
+    rows = {k: [] for k in ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "step")}
+    for _ in range(args.steps):
+        flush.zero_()                                        # 256 MB > L2: the next kernels start cold
+        ms = timed_step(step, t)
+        kernel_ms, _ = P.hydra_profile_collect()
+        for k in rows:
+            rows[k].append(ms if k == "step" else kernel_ms.get(k, 0.0))
+    P.hydra_profile_enable(False)
+    peaks, peak_kind = measured_peaks()
+    med = {k: statistics.median(v) for k, v in rows.items()}
+    best = {k: min(v) for k, v in rows.items()}
+    f_fwd = w.flops_fwd()
+    kernels_ms = med["fwd"] + med["merge"] + med["bwd_prep"] + med["bwd_dkv"] + med["bwd_dq"]
+    bwd_ms = med["bwd_prep"] + med["bwd_dkv"] + med["bwd_dq"]
+    tf = lambda flops, ms: flops / (ms * 1e-3) / 1e12 if ms > 0 else None
+    total = tf(3.5 * f_fwd, kernels_ms)
+    th = w.total * w.n_heads
+    merge_bytes = sum((int(n) + 1) * 260.0 * r * w.n_heads for n, r in merge_groups(pairs))
+    gbs = lambda b, ms: b / (ms * 1e-3) / 1e9 if ms > 0 and b > 0 else None
+    report = {
+        "workload": w.name, "repetitions": args.steps, "l2": "256 MB written between repetitions",
+        "median_ms": med, "best_ms": best,
+        "tflops": {"total": total, "fwd_only": tf(f_fwd, med["fwd"] + med["merge"]), "bwd_only": tf(2.5 * f_fwd, bwd_ms),
+                   "total_best": tf(3.5 * f_fwd, sum(best[k] for k in ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq")))},
+        "of_peak": {"measured_burst": total / peaks["bf16_tflops"],
+                    "measured_sustained": total / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                    "nominal_2250": total / 2250.0, "peaks": peak_kind},
+        "merge_gbs": gbs(merge_bytes, med["merge"]), "bwd_prep_gbs": gbs(th * 516.0, med["bwd_prep"]),
+        "hbm_peak_gbs": {"measured": peaks["hbm_gbs"], "nominal": 8000.0},
+        "first_call_ms": {"device": first_ms, "wall_including_plan_build": first_wall_ms,
+                          "steady_step_ms": med["step"]},
+    }
+    if args.per_sequence:
+        # every sequence alone, same kernels: its share of the time next to its share of sum(L^2)
+        shares = []
+        for b, length in enumerate(w.lengths):
+            lo = int(cu[b])
+            xb = {n: v[lo:lo + length].contiguous() for n, v in t.items()}
+            sb = AttnStep(hw.cu_seqlens([length]), w.n_heads, None, 0, True, float(w.scale))
+            timed_step(sb, xb)
+            shares.append((length, min(timed_step(sb, xb) for _ in range(3))))
+        tsum = sum(ms for _, ms in shares)
+        l2sum = float(sum(length * length for length, _ in shares))
+        report["per_sequence"] = [{"L": length, "ms": ms, "time_share": ms / tsum, "L2_share": length * length / l2sum}
+                                  for length, ms in sorted(shares, reverse=True)]
+        report["per_sequence_note"] = ("short sequences sit above their share of sum(L^2): tile quantisation and the "
+                                       "fixed cost of an item")
+    print(json.dumps(report), flush=True)
+
+
 def merge_groups(pairs):
     """(number of partials, rows) of every merged q chunk."""
     if pairs is None:
@@ -398,10 +486,14 @@ def main():
     ap.add_argument("--workload", default="packed32k", choices=list(hw.WORKLOADS))
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--report", action="store_true", help="per-kernel report of the workload instead of the bench line")
+    ap.add_argument("--per-sequence", action="store_true", help="with --report: time every sequence alone")
     args = ap.parse_args()
     w = hw.workload(args.workload)
     if args.impl == "reference":
         run_reference(args, w)
+    elif args.report:
+        run_report(args, w)
     else:
         run_ours(args, w)
 
