@@ -195,7 +195,7 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
  * memory, 256-byte aligned, of at least hydra_host_step_arena_bytes(...) bytes, owned by the
  * caller; the library carves every device tensor, the partial buffers and the workspace out of it
  * and allocates no device memory itself. One call at a time per device (the internal streams and
- * events are shared); more than 128 heads: HYDRA_ERR_UNSUPPORTED.
+ * events are shared).
  */
 size_t hydra_host_step_arena_bytes(const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
                                    const hydra_pair_t* pairs, int32_t n_pairs);

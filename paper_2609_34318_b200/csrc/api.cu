@@ -873,9 +873,9 @@ int32_t hydra_attn_fwd_bwd_host(const void* q_host, const void* k_host, const vo
     }
     const double copy_s = static_cast<double>(pb.T) * (2 * D_QK + 2 * D_V) * 2 / 50e9;   // per head, one direction
     const double math_s = pair_count * 3.5 * 2 * (D_QK + D_V) / 700e12;                  // per head
-    const int32_t hg = n_heads < 4 ? n_heads : (math_s < 0.5 * copy_s ? 2 : 4);
+    int32_t hg = n_heads < 4 ? n_heads : (math_s < 0.5 * copy_s ? 2 : 4);
+    hg = std::max(hg, (n_heads + HostPipe::kMaxGroups - 1) / HostPipe::kMaxGroups);   // at most kMaxGroups groups
     const int32_t n_groups = (n_heads + hg - 1) / hg;
-    if (n_groups > HostPipe::kMaxGroups) return HYDRA_ERR_UNSUPPORTED;
     size_t lse_off[HostPipe::kMaxGroups + 1] = {0};         // LSE slices start on 256-byte boundaries
     for (int32_t g = 0; g < n_groups; ++g)
         lse_off[g + 1] = align_up(lse_off[g] + static_cast<size_t>(pb.T) * std::min(hg, n_heads - g * hg) * 4, 256);
