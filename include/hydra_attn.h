@@ -126,7 +126,7 @@ int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_
                        void* cuda_stream);
 
 /*
- * Log-sum-exp merge of the partials of every group with two or more pairs (the combination step
+ * Log-sum-exp merge of the partials of every group whose pairs carry partial rows (the combination step
  * of ring attention, Section 5.2):  LSE = ln sum_p exp(LSE_p),  O = sum_p exp(LSE_p - LSE) O_p,
  * all n partials at once in fp32 with one rounding to bf16; a partial with LSE_p = -inf has weight
  * zero; all -inf gives O = 0, LSE = -inf. Writes the group's rows of out / lse.
@@ -136,6 +136,22 @@ int32_t hydra_lse_merge(const void* o_part, const float* lse_part, int64_t part_
                         const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
                         const hydra_pair_t* pairs, int32_t n_pairs, void* out, float* lse,
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The same merge in the streaming form a ring engine uses (Section 5.2: the outer ring pipelines
+ * with attention as in standard ring context parallelism): after every ring step the partials of
+ * that step are folded into the running (out, lse) of their q chunks,
+ *   (out, lse) <- (out, lse) (+) partial_1 (+) ... (+) partial_n,
+ * where (+) is the two-way form of the merge above; rows of out / lse that belong to no listed
+ * group are left untouched. The first step of a chunk uses hydra_lse_merge (which accepts groups
+ * of a single partial) or starts from out = 0, lse = -inf. The running out is stored as bf16, so
+ * every step rounds it once; the result equals the one-shot merge up to those roundings.
+ * Arguments as for hydra_lse_merge; out and lse are read and written.
+ */
+int32_t hydra_lse_merge_accumulate(const void* o_part, const float* lse_part, int64_t part_rows,
+                                   const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
+                                   const hydra_pair_t* pairs, int32_t n_pairs, void* out, float* lse,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
  * hydra_lse_merge for callers that must not allocate device memory. (No counterpart in the paper:

@@ -66,6 +66,8 @@ def _load() -> ctypes.CDLL:
                                    vp, sz, vp]
     lib.hydra_lse_merge.restype = i32
     lib.hydra_lse_merge.argtypes = [vp, vp, i64, vp, i32, i32, vp, i32, vp, vp, vp, sz, vp]
+    lib.hydra_lse_merge_accumulate.restype = i32
+    lib.hydra_lse_merge_accumulate.argtypes = [vp, vp, i64, vp, i32, i32, vp, i32, vp, vp, vp, sz, vp]
     lib.hydra_attn_bwd.restype = i32
     lib.hydra_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, i32, i32, f32, vp, vp, vp,
                                    vp, sz, vp]
@@ -91,7 +93,7 @@ EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_
            "hydra_shutdown", "hydra_usp_factor", "hydra_zigzag_pairs", "hydra_workspace_bytes",
            "hydra_attn_fwd", "hydra_lse_merge", "hydra_attn_bwd", "hydra_poll_status",
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
-           "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc")
+           "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc", "hydra_lse_merge_accumulate")
 KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq")
 
 
@@ -237,6 +239,22 @@ def hydra_lse_merge(o_part, lse_part, part_rows: int, cu_seqlens, n_heads: int, 
                              int(workspace_bytes), _stream(stream))
     if check:
         _check(s, "hydra_lse_merge")
+    return s
+
+
+def hydra_lse_merge_accumulate(o_part, lse_part, part_rows: int, cu_seqlens, n_heads: int, pairs, out, lse,
+                               workspace, workspace_bytes: Optional[int] = None, stream=None,
+                               check: bool = True) -> int:
+    """Streaming merge of one ring step: folds the listed partials into the running (out, lse)."""
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = _lib.hydra_lse_merge_accumulate(_ptr(o_part), _ptr(lse_part), int(part_rows), cu.ctypes.data,
+                                        len(cu) - 1, n_heads, pp, npairs, _ptr(out), _ptr(lse), _ptr(workspace),
+                                        int(workspace_bytes), _stream(stream))
+    if check:
+        _check(s, "hydra_lse_merge_accumulate")
     return s
 
 

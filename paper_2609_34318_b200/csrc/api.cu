@@ -668,9 +668,33 @@ int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_
     return HYDRA_OK;
 }
 
+namespace {
+int32_t merge_impl(const void* o_part, const float* lse_part, int64_t part_rows, const int32_t* cu,
+                   int32_t n_seqs, int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs, void* out,
+                   float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream, int32_t accumulate);
+}
+
 int32_t hydra_lse_merge(const void* o_part, const float* lse_part, int64_t part_rows, const int32_t* cu,
                         int32_t n_seqs, int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs,
                         void* out, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    return merge_impl(o_part, lse_part, part_rows, cu, n_seqs, n_heads, pairs, n_pairs, out, lse, workspace,
+                      workspace_bytes, cuda_stream, 0);
+}
+
+int32_t hydra_lse_merge_accumulate(const void* o_part, const float* lse_part, int64_t part_rows,
+                                   const int32_t* cu, int32_t n_seqs, int32_t n_heads, const hydra_pair_t* pairs,
+                                   int32_t n_pairs, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream)
+{
+    return merge_impl(o_part, lse_part, part_rows, cu, n_seqs, n_heads, pairs, n_pairs, out, lse, workspace,
+                      workspace_bytes, cuda_stream, 1);
+}
+
+namespace {
+int32_t merge_impl(const void* o_part, const float* lse_part, int64_t part_rows, const int32_t* cu,
+                   int32_t n_seqs, int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs, void* out,
+                   float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream, int32_t accumulate)
 {
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
@@ -695,6 +719,7 @@ int32_t hydra_lse_merge(const void* o_part, const float* lse_part, int64_t part_
     mp.n_items = plan->n_items;
     mp.o_part = o_part; mp.lse_part = lse_part; mp.out = out; mp.lse = lse;
     mp.T = pb.T; mp.part_rows = part_rows; mp.h = n_heads;
+    mp.accumulate = accumulate;
     {
         ScopedKernelTimer timer(K_MERGE, stream);
         if (launch_merge(mp, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
@@ -702,6 +727,7 @@ int32_t hydra_lse_merge(const void* o_part, const float* lse_part, int64_t part_
     g_launches += 1;
     return HYDRA_OK;
 }
+}  // namespace
 
 int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* out, const float* lse,
                        const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,

@@ -77,6 +77,14 @@ hydra_lse_merge_kernel(const MergeParams p)
         const uint4 v1 = ld_stream(o_part + (prow1 * p.h + a) * kVecPerRow + lane);
         const float l0 = __ldg(lse_row + part_row[0]);
         const float l1 = g.n_parts > 1 ? __ldg(lse_row + part_row[1]) : neg_inf();
+        // streaming form (one ring step at a time): what out / lse hold so far is one more input
+        const int64_t tok = static_cast<int64_t>(g.out_tok0) + r;
+        uint4 v_cur = make_uint4(0u, 0u, 0u, 0u);
+        float l_cur = neg_inf();
+        if (p.accumulate) {
+            v_cur = out[(tok * p.h + a) * kVecPerRow + lane];
+            l_cur = p.lse[static_cast<int64_t>(a) * p.T + tok];
+        }
         float m = neg_inf();
         float acc[8];
 #pragma unroll
@@ -98,6 +106,7 @@ hydra_lse_merge_kernel(const MergeParams p)
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = fmaf(w, f[e], acc[e]);
         };
+        add(v_cur, l_cur);
         add(v0, l0);
         add(v1, l1);
         for (int q = 2; q < g.n_parts; ++q) {
@@ -111,7 +120,6 @@ hydra_lse_merge_kernel(const MergeParams p)
         } else {
             m = neg_inf();
         }
-        const int64_t tok = static_cast<int64_t>(g.out_tok0) + r;
         out[(tok * p.h + a) * kVecPerRow + lane] = pack8(acc);
         if (lane == 0)
             p.lse[static_cast<int64_t>(a) * p.T + tok] = (m == neg_inf()) ? neg_inf() : m + __logf(z);

@@ -99,6 +99,7 @@ struct MergeParams {
     void* out; float* lse;
     int64_t T; int64_t part_rows;
     int32_t h;
+    int32_t accumulate;         // 1: the current (out, lse) rows are one more input of their merge
 };
 
 size_t fwd_smem_bytes();

@@ -1,0 +1,92 @@
+"""The streaming form of the merge (`hydra_lse_merge_accumulate`): a ring engine folds the partials of
+every ring step into the running (out, lse). Emulated on one GPU: the pairs of a zigzag ring are
+processed step by step (all ranks' pairs of a step in one call), and the result must equal the
+unchunked attention of the oracle (chunking and merging is an exact identity up to rounding).
+"""
+import numpy as np
+import pytest
+
+import hydra_workloads as hw
+from gpu_util import TOL_LSE, TOL_REL, check, run_oracle
+
+pytestmark = pytest.mark.gpu
+DQK, DV = hw.D_QK, hw.D_V
+
+
+def rand_inputs(rng, T, h):
+    f = lambda d: hw.f32_to_bf16_bits(rng.standard_normal((T, h, d)).astype(np.float32))
+    return dict(q=f(DQK), k=f(DQK), v=f(DV), do=f(DV))
+
+
+@pytest.mark.parametrize("lengths,cp_r,h", [([1024, 300], 2, 3), ([2048], 4, 2), ([257, 64, 513], 1, 4)])
+def test_ring_steps_accumulate_to_the_unchunked_result(lengths, cp_r, h):
+    import torch
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.runner import bits_to_tensor
+
+    cu = hw.cu_seqlens(lengths)
+    T = int(cu[-1])
+    x = rand_inputs(np.random.default_rng(11 + cp_r), T, h)
+    q, k, v = (bits_to_tensor(x[n]) for n in ("q", "k", "v"))
+    pairs, _, rank, step = P.hydra_zigzag_pairs(cu, cp_r)
+    scale = float(np.float32(1.0 / np.sqrt(np.float32(DQK))))
+    out = torch.full((T, h, DV), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((h, T), float("nan"), dtype=torch.float32, device="cuda")
+    n_steps = int(step.max()) + 1
+    assert n_steps == max(cp_r, 1)
+    for t in range(n_steps):
+        sel = pairs[step == t].copy()
+        assert len(sel) > 0
+        rows = 0
+        for p in sel:                                   # every pair of the step writes a partial
+            p["part_row"] = rows
+            rows += int(p["q_len"])
+        o_part = torch.full((rows, h, DV), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse_part = torch.full((h, rows), float("nan"), dtype=torch.float32, device="cuda")
+        ws = torch.empty(max(P.hydra_workspace_bytes(P.HYDRA_WS_FWD, cu, h, sel), 256), dtype=torch.uint8, device="cuda")
+        P.hydra_attn_fwd(q, k, v, cu, h, sel, True, scale, out, lse, o_part, lse_part, rows, ws)
+        if t == 0:
+            P.hydra_lse_merge(o_part, lse_part, rows, cu, h, sel, out, lse, ws)
+        else:
+            P.hydra_lse_merge_accumulate(o_part, lse_part, rows, cu, h, sel, out, lse, ws)
+    torch.cuda.synchronize()
+    got = dict(out=out.float().cpu().numpy().astype(np.float64), lse=lse.cpu().numpy().astype(np.float64))
+    ref = run_oracle(x, cu, True, backward=False)
+    # every step rounds the running out to bf16 once more than the one-shot merge does
+    check(got, ref, names=("out", "lse"), tol_rel=TOL_REL, tol_lse=TOL_LSE, label=f"ring steps cp_r={cp_r}: ")
+
+
+def test_accumulate_leaves_other_rows_alone_and_matches_the_one_shot_merge():
+    import torch
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.runner import AttnStep, bits_to_tensor
+
+    lengths, cp_r, h = [600, 200], 2, 2
+    cu = hw.cu_seqlens(lengths)
+    T = int(cu[-1])
+    x = rand_inputs(np.random.default_rng(5), T, h)
+    q, k, v = (bits_to_tensor(x[n]) for n in ("q", "k", "v"))
+    pairs, part_rows, _, step = P.hydra_zigzag_pairs(cu, cp_r)
+    one = AttnStep(cu, h, pairs, part_rows, True, None)
+    one.forward(q, k, v)                                 # all pairs at once, one-shot merge
+    scale = float(np.float32(1.0 / np.sqrt(np.float32(DQK))))
+    # only the pairs of sequence 0, two steps; sequence 1's rows must keep their sentinel
+    out = torch.full((T, h, DV), 7.0, dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((h, T), 7.0, dtype=torch.float32, device="cuda")
+    for t in range(cp_r):
+        sel = pairs[(step == t) & (pairs["seq"] == 0)].copy()
+        rows = 0
+        for p in sel:
+            p["part_row"] = rows
+            rows += int(p["q_len"])
+        o_part = torch.empty((rows, h, DV), dtype=torch.bfloat16, device="cuda")
+        lse_part = torch.empty((h, rows), dtype=torch.float32, device="cuda")
+        ws = torch.empty(max(P.hydra_workspace_bytes(P.HYDRA_WS_FWD, cu, h, sel), 256), dtype=torch.uint8, device="cuda")
+        P.hydra_attn_fwd(q, k, v, cu, h, sel, True, scale, out, lse, o_part, lse_part, rows, ws)
+        (P.hydra_lse_merge if t == 0 else P.hydra_lse_merge_accumulate)(o_part, lse_part, rows, cu, h, sel, out, lse, ws)
+    torch.cuda.synchronize()
+    L0 = lengths[0]
+    assert torch.all(out[L0:] == 7.0) and torch.all(lse[:, L0:] == 7.0)
+    a, b = out[:L0].float(), one.out[:L0].float()
+    assert (a - b).abs().max().item() <= 2 ** -7 * b.abs().max().item()      # one extra bf16 rounding
+    assert (lse[:, :L0] - one.lse[:, :L0]).abs().max().item() <= 1e-5
