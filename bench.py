@@ -446,6 +446,43 @@ def run_report(args, w):
     print(json.dumps(report), flush=True)
 
 
+def run_sched(args):
+    """Scheduling time of the load-driven DCP scheduler (host only): the library's heap search on
+    batches of the size the paper schedules (one global batch over a pool of G ranks), and the
+    oracle's direct scans on a bounded sample of the same batch for context."""
+    import math
+    import paper_2609_34318_b200 as P
+    from oracle import scheduler as S
+
+    rng = np.random.default_rng(hw.SEED)
+    out = []
+    for G, tokens_per_rank in ((2048, 8192), (16384, 8192)):
+        B = tokens_per_rank
+        budget = G * B * 4                                   # four micro-batches' worth of tokens
+        lengths, total = [], 0
+        while total < budget:                                # long-tailed mix up to 256K (Section 2.2)
+            L = int(min(262144, max(64, round(math.exp(rng.normal(math.log(1024), 1.4))))))
+            lengths.append(L)
+            total += L
+        t = P.hydra_sched_targets(lengths, G, B, 4, 1e-9)
+        C = max(t.C_star, t.C_mem)
+        best = None
+        for _ in range(5):
+            t0 = time.perf_counter()
+            mb, rank0, cp, n_mb = P.hydra_sched_pack(lengths, G, B, C)
+            dt = time.perf_counter() - t0
+            best = dt if best is None else min(best, dt)
+        sample = lengths[:1500]
+        Cs = max(C, S.ceil2(max(sample) / B))
+        t0 = time.perf_counter()
+        S.pack(sample, G, B, min(G, Cs))
+        oracle_s = time.perf_counter() - t0
+        out.append({"G": G, "B": B, "documents": len(lengths), "tokens": total, "C": int(C), "M_star": int(t.M_star),
+                    "micro_batches": int(n_mb), "library_ms": 1e3 * best, "documents_per_s": len(lengths) / best,
+                    "oracle_direct_scan_s_on_1500_documents": oracle_s})
+    print(json.dumps({"scheduler": out}), flush=True)
+
+
 def merge_groups(pairs):
     """(number of partials, rows) of every merged q chunk."""
     if pairs is None:
@@ -488,7 +525,11 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--report", action="store_true", help="per-kernel report of the workload instead of the bench line")
     ap.add_argument("--per-sequence", action="store_true", help="with --report: time every sequence alone")
+    ap.add_argument("--sched", action="store_true", help="time the host scheduler instead (no GPU needed)")
     args = ap.parse_args()
+    if args.sched:
+        run_sched(args)
+        return
     w = hw.workload(args.workload)
     if args.impl == "reference":
         run_reference(args, w)

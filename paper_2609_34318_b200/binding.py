@@ -66,6 +66,13 @@ def _load() -> ctypes.CDLL:
                                    vp, sz, vp]
     lib.hydra_lse_merge.restype = i32
     lib.hydra_lse_merge.argtypes = [vp, vp, i64, vp, i32, i32, vp, i32, vp, vp, vp, sz, vp]
+    f64 = ctypes.c_double
+    lib.hydra_sched_targets.restype = i32
+    lib.hydra_sched_targets.argtypes = [vp, i32, i32, i64, i32, f64, vp]
+    lib.hydra_sched_cp.restype = i32
+    lib.hydra_sched_cp.argtypes = [i64, i64, i32, i64]
+    lib.hydra_sched_pack.restype = i32
+    lib.hydra_sched_pack.argtypes = [vp, i32, i32, i64, i32, vp, vp, vp, vp]
     lib.hydra_lse_merge_accumulate.restype = i32
     lib.hydra_lse_merge_accumulate.argtypes = [vp, vp, i64, vp, i32, i32, vp, i32, vp, vp, vp, sz, vp]
     lib.hydra_attn_bwd.restype = i32
@@ -93,7 +100,8 @@ EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_
            "hydra_shutdown", "hydra_usp_factor", "hydra_zigzag_pairs", "hydra_workspace_bytes",
            "hydra_attn_fwd", "hydra_lse_merge", "hydra_attn_bwd", "hydra_poll_status",
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
-           "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc", "hydra_lse_merge_accumulate")
+           "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc", "hydra_lse_merge_accumulate",
+           "hydra_sched_targets", "hydra_sched_cp", "hydra_sched_pack")
 KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq")
 
 
@@ -343,3 +351,39 @@ def hydra_lse_merge_noalloc(o_part, lse_part, part_rows: int, cu_seqlens, n_head
     if check:
         _check(s, "hydra_lse_merge_noalloc")
     return s
+
+
+# --------------------------------------------------------------------------------------------------
+# scheduler (include/hydra_sched.h): host only
+# --------------------------------------------------------------------------------------------------
+class SchedTargets(ctypes.Structure):
+    _fields_ = [("s_max", ctypes.c_int64), ("W", ctypes.c_double), ("C_mem", ctypes.c_int32),
+                ("C_star", ctypes.c_int32), ("C_hat", ctypes.c_double), ("Lambda_star", ctypes.c_double),
+                ("M_star", ctypes.c_int64)]
+
+
+def hydra_sched_targets(lengths, G: int, B: int, pp: int, theta_over_c: float) -> SchedTargets:
+    s = np.ascontiguousarray(lengths, dtype=np.int64)
+    out = SchedTargets()
+    _check(_lib.hydra_sched_targets(s.ctypes.data, len(s), int(G), int(B), int(pp), float(theta_over_c),
+                                    ctypes.addressof(out)), "hydra_sched_targets")
+    return out
+
+
+def hydra_sched_cp(s: int, s_max: int, C: int, B: int) -> int:
+    return int(_lib.hydra_sched_cp(int(s), int(s_max), int(C), int(B)))
+
+
+def hydra_sched_pack(lengths, G: int, B: int, C: int, check: bool = True):
+    """Returns (mb, rank0, cp, n_mb): micro-batch, first rank and group size of every document."""
+    s = np.ascontiguousarray(lengths, dtype=np.int64)
+    n = len(s)
+    mb, rank0, cp = (np.zeros(max(n, 1), dtype=np.int32) for _ in range(3))
+    n_mb = ctypes.c_int32(0)
+    st = _lib.hydra_sched_pack(s.ctypes.data, n, int(G), int(B), int(C), mb.ctypes.data, rank0.ctypes.data,
+                               cp.ctypes.data, ctypes.addressof(n_mb))
+    if check:
+        _check(st, "hydra_sched_pack")
+    elif st != HYDRA_OK:
+        return st
+    return mb[:n], rank0[:n], cp[:n], int(n_mb.value)

@@ -13,8 +13,9 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 OUT = os.path.join(PKG, "libhydra_attn.so")
 OBJ_DIR = os.path.join(PKG, "build")
-SOURCES = ["api.cu", "fwd_kernel.cu", "bwd_kernels.cu", "aux_kernels.cu"]
-HEADERS = ["hydra_internal.h", "sm100_ptx.cuh", os.path.join("..", "..", "include", "hydra_attn.h")]
+SOURCES = ["api.cu", "fwd_kernel.cu", "bwd_kernels.cu", "aux_kernels.cu", "sched.cu"]
+HEADERS = ["hydra_internal.h", "sm100_ptx.cuh", os.path.join("..", "..", "include", "hydra_attn.h"),
+           os.path.join("..", "..", "include", "hydra_sched.h")]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-Xptxas", "-v"]
