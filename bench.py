@@ -428,6 +428,43 @@ def run_report(args, w):
         "first_call_ms": {"device": first_ms, "wall_including_plan_build": first_wall_ms,
                           "steady_step_ms": med["step"]},
     }
+    # The backward in its accumulating form (what a ring engine calls once per ring step) and the cast of
+    # the fp32 accumulators to bf16: the pairs of the workload in one call (cost of the fp32
+    # read-modify-write epilogues against the bf16 stores) and, for a cut workload, one call per ring step.
+    acc = [torch.zeros((w.total, w.n_heads, d), dtype=torch.float32, device="cuda") for d in (hw.D_QK, hw.D_QK, hw.D_V)]
+    grads = [torch.empty(a.shape, dtype=torch.bfloat16, device="cuda") for a in acc]
+    all_pairs = pairs if pairs is not None else P.hydra_zigzag_pairs(cu, 0)[0]
+    ring_step = P.hydra_zigzag_pairs(cu, w.cp_r)[3] if w.cp_r else None
+    calls = [all_pairs] if ring_step is None else [all_pairs[ring_step == s_].copy() for s_ in range(int(ring_step.max()) + 1)]
+
+    def accumulate_pass(call_list):
+        for a in acc:
+            a.zero_()
+        flush.zero_()
+        P.hydra_profile_collect()
+        for sel in call_list:
+            P.hydra_attn_bwd_accumulate(t["q"], t["k"], t["v"], step.out, step.lse, t["do"], cu, w.n_heads, sel, True,
+                                        float(w.scale), acc[0], acc[1], acc[2], step.workspace)
+        for a, g in zip(acc, grads):
+            P.hydra_grad_cast(a, g)
+        torch.cuda.synchronize()
+        return P.hydra_profile_collect()[0]
+
+    P.hydra_profile_enable(True)
+    accumulate_pass([all_pairs])
+    one_call = [accumulate_pass([all_pairs]) for _ in range(3)]
+    by_step = [accumulate_pass(calls) for _ in range(3)] if len(calls) > 1 else None
+    P.hydra_profile_enable(False)
+    pick = lambda runs, k: statistics.median(r[k] for r in runs)
+    cast_bytes = sum(a.numel() for a in acc) * 6.0
+    report["accumulating_backward"] = {
+        "one_call_ms": {k: pick(one_call, k) for k in ("bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast")},
+        "grad_cast_gbs": gbs(cast_bytes, pick(one_call, "grad_cast")),
+        "grad_cast_bytes": cast_bytes,
+    }
+    if by_step:
+        report["accumulating_backward"]["ring_steps"] = len(calls)
+        report["accumulating_backward"]["by_step_ms"] = {k: pick(by_step, k) for k in ("bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast")}
     if args.per_sequence:
         # every sequence alone, same kernels: its share of the time next to its share of sum(L^2)
         shares = []

@@ -199,6 +199,31 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The backward of one ring step (Section 5.2: the outer ring pipelines with attention as in
+ * standard ring context parallelism, so a rank sees its chunk pairs a step at a time): the same
+ * computation as hydra_attn_bwd for the listed pairs, but the contributions are ADDED to fp32
+ * accumulators instead of being written as bf16, so that calls for the successive steps sum to the
+ * backward of all pairs. The paper does not print this form; it is what its ring engine needs from
+ * the attention library.
+ *   dq_acc, dk_acc  device fp32 [T, h, 192]; dv_acc device fp32 [T, h, 128]; the caller zeroes them
+ *                   (or loads them with gradients that arrived from a peer) before the first step.
+ *   out, lse        the MERGED forward result of all steps, as for hydra_attn_bwd.
+ * Rows covered by no listed chunk are left untouched. Each accumulator row is owned by one thread
+ * block per call and calls on one stream are ordered, so no atomics are used and the result of a
+ * fixed sequence of calls is deterministic. Calls that share accumulators must be enqueued on one
+ * stream (or ordered by the caller). Workspace, requirements and errors as for hydra_attn_bwd.
+ * hydra_grad_cast converts an accumulator to the bf16 gradient: grad[i] = bf16(acc[i]), i <
+ * n_elements (round to nearest even); acc, grad device pointers, 16-byte aligned.
+ */
+int32_t hydra_attn_bwd_accumulate(const void* q, const void* k, const void* v, const void* out,
+                                  const float* lse, const void* dout, const int32_t* cu_seqlens_host,
+                                  int32_t n_seqs, int32_t n_heads, const hydra_pair_t* pairs,
+                                  int32_t n_pairs, int32_t causal, float softmax_scale, float* dq_acc,
+                                  float* dk_acc, float* dv_acc, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream);
+int32_t hydra_grad_cast(const float* acc, void* grad, int64_t n_elements, void* cuda_stream);
+
+/*
  * The whole step (forward of every pair, merge, backward; Sections 3.5 and 5.2 as above) with HOST
  * buffers: copies q, k, v, dout to the device, runs hydra_attn_fwd, hydra_lse_merge (if any pair has
  * partial rows) and hydra_attn_bwd, and copies out, lse, dq, dk, dv back. Heads are independent,
@@ -225,8 +250,8 @@ int32_t hydra_attn_fwd_bwd_host(const void* q_host, const void* k_host, const vo
 /*
  * Per-kernel timing (measurement aid, not part of the method). While enabled, every kernel launch
  * is bracketed by CUDA events on its stream. hydra_profile_collect waits for the recorded events,
- * adds their durations into ms_out[5] and their counts into launches_out[5] (index: 0 forward,
- * 1 merge, 2 backward prep, 3 backward dK/dV, 4 backward dQ) and forgets them.
+ * adds their durations into ms_out[6] and their counts into launches_out[6] (index: 0 forward,
+ * 1 merge, 2 backward prep, 3 backward dK/dV, 4 backward dQ, 5 gradient cast) and forgets them.
  */
 void hydra_profile_enable(int32_t on);
 int32_t hydra_profile_collect(double* ms_out, int64_t* launches_out);

@@ -78,6 +78,10 @@ def _load() -> ctypes.CDLL:
     lib.hydra_attn_bwd.restype = i32
     lib.hydra_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, i32, i32, f32, vp, vp, vp,
                                    vp, sz, vp]
+    lib.hydra_attn_bwd_accumulate.restype = i32
+    lib.hydra_attn_bwd_accumulate.argtypes = lib.hydra_attn_bwd.argtypes
+    lib.hydra_grad_cast.restype = i32
+    lib.hydra_grad_cast.argtypes = [vp, vp, i64, vp]
     lib.hydra_poll_status.restype = i32
     lib.hydra_poll_status.argtypes = [vp, vp, vp, vp]
     lib.hydra_profile_enable.restype = None
@@ -101,8 +105,9 @@ EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_
            "hydra_attn_fwd", "hydra_lse_merge", "hydra_attn_bwd", "hydra_poll_status",
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
            "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc", "hydra_lse_merge_accumulate",
-           "hydra_sched_targets", "hydra_sched_cp", "hydra_sched_pack")
-KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq")
+           "hydra_sched_targets", "hydra_sched_cp", "hydra_sched_pack", "hydra_attn_bwd_accumulate",
+           "hydra_grad_cast")
+KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast")
 
 
 # ------------------------------------------------------------------------------------------------
@@ -282,6 +287,33 @@ def hydra_attn_bwd(q, k, v, out, lse, dout, cu_seqlens, n_heads: int, pairs, cau
     return s
 
 
+def hydra_attn_bwd_accumulate(q, k, v, out, lse, dout, cu_seqlens, n_heads: int, pairs, causal: bool,
+                              softmax_scale: float, dq_acc, dk_acc, dv_acc, workspace,
+                              workspace_bytes: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """Backward of the listed pairs added to fp32 accumulators (one ring step at a time)."""
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = _lib.hydra_attn_bwd_accumulate(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout),
+                                       cu.ctypes.data, len(cu) - 1, n_heads, pp, npairs, int(bool(causal)),
+                                       ctypes.c_float(float(softmax_scale)), _ptr(dq_acc), _ptr(dk_acc),
+                                       _ptr(dv_acc), _ptr(workspace), int(workspace_bytes), _stream(stream))
+    if check:
+        _check(s, "hydra_attn_bwd_accumulate")
+    return s
+
+
+def hydra_grad_cast(acc, grad, n_elements: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """grad (bf16) = acc (fp32), elementwise."""
+    if n_elements is None:
+        n_elements = acc.numel()
+    s = _lib.hydra_grad_cast(_ptr(acc), _ptr(grad), int(n_elements), _stream(stream))
+    if check:
+        _check(s, "hydra_grad_cast")
+    return s
+
+
 def hydra_poll_status(workspace, stream=None) -> Tuple[int, int]:
     st, detail = ctypes.c_int32(0), ctypes.c_int64(-1)
     _check(_lib.hydra_poll_status(_ptr(workspace), _stream(stream), ctypes.addressof(st),
@@ -295,8 +327,8 @@ def hydra_profile_enable(on: bool) -> None:
 
 def hydra_profile_collect():
     """Returns ({kind: total ms}, {kind: launches}) since the last collect."""
-    ms = (ctypes.c_double * 5)()
-    n = (ctypes.c_int64 * 5)()
+    ms = (ctypes.c_double * len(KERNEL_KINDS))()
+    n = (ctypes.c_int64 * len(KERNEL_KINDS))()
     _check(_lib.hydra_profile_collect(ctypes.addressof(ms), ctypes.addressof(n)), "hydra_profile_collect")
     return dict(zip(KERNEL_KINDS, list(ms))), dict(zip(KERNEL_KINDS, list(n)))
 

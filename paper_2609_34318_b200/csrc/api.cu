@@ -22,7 +22,7 @@ constexpr size_t kStatusBytes = 256;
 // ---------------------------------------------------------------------------------------------
 // optional per-kernel timing with CUDA events on the launching stream
 // ---------------------------------------------------------------------------------------------
-enum KernelKind { K_FWD = 0, K_MERGE, K_PREP, K_DKV, K_DQ, K_COUNT };
+enum KernelKind { K_FWD = 0, K_MERGE, K_PREP, K_DKV, K_DQ, K_CAST, K_COUNT };
 struct ProfRecord { int kind; cudaEvent_t start, stop; };
 std::mutex g_prof_mutex;
 bool g_prof_on = false;
@@ -436,7 +436,7 @@ int32_t device_info(int* sms)
         info[dev].known = true;
     }
     if (info[dev].major != 10) return HYDRA_ERR_NOT_SM100;
-    *sms = info[dev].sms;
+    if (sms) *sms = info[dev].sms;
     return HYDRA_OK;
 }
 
@@ -729,11 +729,12 @@ int32_t merge_impl(const void* o_part, const float* lse_part, int64_t part_rows,
 }
 }  // namespace
 
-int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* out, const float* lse,
-                       const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
-                       const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
-                       void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes,
-                       void* cuda_stream)
+namespace {
+int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                 const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                 const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
+                 void* dq, void* dk, void* dv, bool accumulate, void* workspace, size_t workspace_bytes,
+                 void* cuda_stream)
 {
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
@@ -777,6 +778,7 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
     bp.lse = lse; bp.dsum = dsum; bp.dq = dq; bp.dk = dk; bp.dv = dv;
     bp.T = pb.T; bp.h = n_heads; bp.causal = causal != 0;
     bp.scale = softmax_scale; bp.scale_log2 = softmax_scale * 1.4426950408889634f;
+    bp.accumulate = accumulate ? 1 : 0;
     bp.status = static_cast<StatusBlock*>(workspace);
     bp.wait_limit_ns = g_wait_limit_ns.load();
     if (plan->n_items2 > 0) {
@@ -797,6 +799,42 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
             return HYDRA_ERR_CUDA;
         g_launches += 1;
     }
+    return HYDRA_OK;
+}
+}  // namespace
+
+int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                       const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                       const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
+                       void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream)
+{
+    return bwd_impl(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, dq, dk,
+                    dv, false, workspace, workspace_bytes, cuda_stream);
+}
+
+int32_t hydra_attn_bwd_accumulate(const void* q, const void* k, const void* v, const void* out,
+                                  const float* lse, const void* dout, const int32_t* cu, int32_t n_seqs,
+                                  int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal,
+                                  float softmax_scale, float* dq_acc, float* dk_acc, float* dv_acc,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    return bwd_impl(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, dq_acc,
+                    dk_acc, dv_acc, true, workspace, workspace_bytes, cuda_stream);
+}
+
+int32_t hydra_grad_cast(const float* acc, void* grad, int64_t n_elements, void* cuda_stream)
+{
+    if (n_elements < 0) return HYDRA_ERR_INVALID_ARG;
+    if (n_elements == 0) return HYDRA_OK;
+    if (!acc || !grad || !aligned16(acc) || !aligned16(grad)) return HYDRA_ERR_INVALID_ARG;
+    if (int32_t s = device_info(nullptr)) return s;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    {
+        ScopedKernelTimer timer(K_CAST, stream);
+        if (launch_grad_cast(acc, grad, n_elements, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    }
+    g_launches += 1;
     return HYDRA_OK;
 }
 

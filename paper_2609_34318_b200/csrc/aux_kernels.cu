@@ -1,6 +1,7 @@
 // The bandwidth-bound steps around the tensor-core kernels:
 //   hydra_lse_merge_kernel  n-way log-sum-exp merge of the partial (O, LSE) of a q chunk
 //   hydra_bwd_prep_kernel   D = rowsum(dO * O)
+//   hydra_grad_cast_kernel  fp32 gradient accumulators -> bf16 (after a backward run step by step)
 // Both move every byte once with 16-byte accesses: 16 lanes own one (row, head) vector of 128 bf16.
 #include <cuda_bf16.h>
 
@@ -150,6 +151,39 @@ hydra_bwd_prep_kernel(const uint4* __restrict__ dout, const uint4* __restrict__ 
             dsum[static_cast<int64_t>(a_head) * T + t] = s;
         }
     }
+}
+
+// grad (bf16) = acc (fp32), eight elements per thread: two 16-byte loads, one 16-byte store.
+__global__ void __launch_bounds__(kThreads)
+hydra_grad_cast_kernel(const float4* __restrict__ acc, uint4* __restrict__ grad, int64_t n8, int64_t n,
+                       const float* __restrict__ acc_tail, __nv_bfloat16* __restrict__ grad_tail)
+{
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; i < n8; i += stride) {
+        float4 a, b;
+        asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0, %1, %2, %3}, [%4];"
+                     : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w) : "l"(acc + 2 * i));
+        asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0, %1, %2, %3}, [%4];"
+                     : "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w) : "l"(acc + 2 * i + 1));
+        const float f[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+        grad[i] = pack8(f);
+    }
+    if (blockIdx.x == 0) {                             // fewer than eight elements left over
+        const int64_t t = n8 * 8 + threadIdx.x;
+        if (t < n) grad_tail[t] = __float2bfloat16_rn(acc_tail[t]);
+    }
+}
+
+cudaError_t launch_grad_cast(const float* acc, void* grad, int64_t n, cudaStream_t stream)
+{
+    if (n <= 0) return cudaSuccess;
+    const int64_t n8 = n / 8;
+    const int64_t blocks = (n8 + kThreads - 1) / kThreads;
+    const int grid = static_cast<int>(blocks < 1 ? 1 : (blocks < 148 * 16 ? blocks : 148 * 16));
+    hydra_grad_cast_kernel<<<grid, kThreads, 0, stream>>>(reinterpret_cast<const float4*>(acc),
+                                                          static_cast<uint4*>(grad), n8, n, acc,
+                                                          static_cast<__nv_bfloat16*>(grad));
+    return cudaGetLastError();
 }
 
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream)

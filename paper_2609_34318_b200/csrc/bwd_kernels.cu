@@ -50,6 +50,19 @@ __device__ __forceinline__ void store_row_bf16(__nv_bfloat16* dst, const uint32_
     }
 }
 
+// Accumulating form of the same epilogue: dst (fp32) += v * mul, as 16-byte reductions performed at
+// the L2 cache. Every row is owned by one thread of one CTA per launch and launches on a stream are
+// ordered, so every address receives one addition per launch and the sum does not depend on timing;
+// a reduction is used instead of load-add-store only because it does not make the thread wait for
+// the old value (five dependent round trips to memory per work item otherwise).
+__device__ __forceinline__ void add_row_f32(float* dst, const uint32_t* v, int n, float mul)
+{
+#pragma unroll
+    for (int e = 0; e < n; e += 4)
+        red_add_v4_f32(dst + e, __uint_as_float(v[e + 0]) * mul, __uint_as_float(v[e + 1]) * mul,
+                       __uint_as_float(v[e + 2]) * mul, __uint_as_float(v[e + 3]) * mul);
+}
+
 // ---------------------------------------------------------------------------------------------
 // dQ kernel: layout
 // ---------------------------------------------------------------------------------------------
@@ -378,12 +391,13 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const PairDev first = p.pairs[list[0]];
             const int row = item.r0 + r;
             const bool row_valid = row < first.q_len;
-            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.dq) +
-                                 (static_cast<int64_t>(first.q_tok0 + row) * p.h + item.head) * D_QK + g * 96;
+            const int64_t dst_off = (static_cast<int64_t>(first.q_tok0 + row) * p.h + item.head) * D_QK + g * 96;
+            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.dq) + dst_off;
+            float* dst_acc = static_cast<float*>(p.dq) + dst_off;        // accumulate mode: dq is fp32
             TileIter ti;
             ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
-            if (!ti.valid()) {                         // no visible key at all: dQ = 0
-                if (row_valid) {
+            if (!ti.valid()) {                         // no visible key at all: dQ = 0 (nothing to add)
+                if (row_valid && !p.accumulate) {
                     uint4* d4 = reinterpret_cast<uint4*>(dst);
 #pragma unroll
                     for (int e = 0; e < 12; ++e) d4[e] = make_uint4(0u, 0u, 0u, 0u);
@@ -475,7 +489,10 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     tc_fence_before_sync();
                     mbar_arrive_warp(bar(B_ACCFREE));
                 }
-                if (row_valid) store_row_bf16(dst + c0, v, 32, p.scale);
+                if (row_valid) {
+                    if (p.accumulate) add_row_f32(dst_acc + c0, v, 32, p.scale);
+                    else store_row_bf16(dst + c0, v, 32, p.scale);
+                }
             }
         }
     }
@@ -735,12 +752,16 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const int krow = item.r0 + r;              // kv row inside the chunk
             const bool row_valid = krow < first.k_len;
             const int64_t tok = static_cast<int64_t>(first.k_tok0) + krow;
-            __nv_bfloat16* dkp = static_cast<__nv_bfloat16*>(p.dk) + (tok * p.h + item.head) * D_QK + g * 96;
-            __nv_bfloat16* dvp = static_cast<__nv_bfloat16*>(p.dv) + (tok * p.h + item.head) * D_V + g * 64;
+            const int64_t dk_off = (tok * p.h + item.head) * D_QK + g * 96;
+            const int64_t dv_off = (tok * p.h + item.head) * D_V + g * 64;
+            __nv_bfloat16* dkp = static_cast<__nv_bfloat16*>(p.dk) + dk_off;
+            __nv_bfloat16* dvp = static_cast<__nv_bfloat16*>(p.dv) + dv_off;
+            float* dkp_acc = static_cast<float*>(p.dk) + dk_off;         // accumulate mode: dk, dv are fp32
+            float* dvp_acc = static_cast<float*>(p.dv) + dv_off;
             SubIter si;
             si.init(p.pairs, list, item.list_len, item.r0, p.causal);
-            if (!si.valid()) {                         // no q row sees this tile: dK = dV = 0
-                if (row_valid) {
+            if (!si.valid()) {                         // no q row sees this tile: dK = dV = 0 (nothing to add)
+                if (row_valid && !p.accumulate) {
                     uint4* a4 = reinterpret_cast<uint4*>(dkp);
                     uint4* b4 = reinterpret_cast<uint4*>(dvp);
 #pragma unroll
@@ -820,7 +841,10 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 uint32_t v[32];
                 tmem_ld_x32(tm + kTmDK + lane_base + g * 96 + c0, v);
                 tmem_wait_ld();
-                if (row_valid) store_row_bf16(dkp + c0, v, 32, p.scale);
+                if (row_valid) {
+                    if (p.accumulate) add_row_f32(dkp_acc + c0, v, 32, p.scale);
+                    else store_row_bf16(dkp + c0, v, 32, p.scale);
+                }
             }
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
@@ -831,7 +855,10 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     tc_fence_before_sync();
                     mbar_arrive_warp(bar(B_ACCFREE));
                 }
-                if (row_valid) store_row_bf16(dvp + c0, v, 32, 1.f);
+                if (row_valid) {
+                    if (p.accumulate) add_row_f32(dvp_acc + c0, v, 32, 1.f);
+                    else store_row_bf16(dvp + c0, v, 32, 1.f);
+                }
             }
         }
     }

@@ -82,10 +82,11 @@ struct BwdParams {
     const GroupItem* items;
     int32_t n_items;
     const float* lse; const float* dsum;   // [h, T]
-    void* dq; void* dk; void* dv;
+    void* dq; void* dk; void* dv;   // bf16 [T,h,d], written; or, with accumulate, fp32 [T,h,d], added to
     int64_t T;
     int32_t h; int32_t causal;
     float scale; float scale_log2;
+    int32_t accumulate;
     StatusBlock* status;
     uint64_t wait_limit_ns;
 };
@@ -115,6 +116,7 @@ cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, con
                            const CUtensorMap& mdo_sub, const BwdParams& p, int grid,
                            cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
+cudaError_t launch_grad_cast(const float* acc, void* grad, int64_t n, cudaStream_t stream);
 cudaError_t launch_bwd_prep(const void* dout, const void* out, float* dsum, int64_t T, int32_t h,
                             cudaStream_t stream);
 

@@ -376,6 +376,13 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return d;
 }
 // {lo, hi} -> packed bf16x2, round to nearest even; `lo` lands in the low 16 bits.
+// 16-byte floating-point reduction to global memory (no value comes back, so nothing waits for it)
+__device__ __forceinline__ void red_add_v4_f32(float* addr, float a, float b, float c, float d)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
+                 : "memory");
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));

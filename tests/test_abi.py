@@ -138,6 +138,22 @@ def test_backward_requires_identical_or_disjoint_chunks():
     assert s == P.HYDRA_ERR_WORKSPACE_TOO_SMALL
 
 
+def test_accumulating_backward_and_cast_validate_like_the_plain_calls():
+    cu = [0, 256]
+    overlapping = [dict(seq=0, q_start=0, q_len=128, k_start=0, k_len=128, group=0),
+                   dict(seq=0, q_start=64, q_len=128, k_start=0, k_len=128, group=1)]
+    s = P.hydra_attn_bwd_accumulate(0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, cu, 2, overlapping, True,
+                                    0.07, 0x1000, 0x1000, 0x1000, 0x1000, 1 << 20, stream=0, check=False)
+    assert s == P.HYDRA_ERR_INVALID_ARG
+    s = P.hydra_attn_bwd_accumulate(0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, cu, 2, None, True, 0.07,
+                                    0x1000, 0x1004, 0x1000, 0x1000, 1 << 20, stream=0, check=False)
+    assert s == P.HYDRA_ERR_INVALID_ARG                                               # misaligned accumulator
+    assert P.hydra_grad_cast(0x1000, 0x1000, -1, stream=0, check=False) == P.HYDRA_ERR_INVALID_ARG
+    assert P.hydra_grad_cast(0x1000, 0x1000, 0, stream=0, check=False) == P.HYDRA_OK   # nothing to do
+    assert P.hydra_grad_cast(0, 0x1000, 8, stream=0, check=False) == P.HYDRA_ERR_INVALID_ARG
+    assert P.hydra_grad_cast(0x1000, 0x1008, 8, stream=0, check=False) == P.HYDRA_ERR_INVALID_ARG
+
+
 def test_no_cpu_fallback():
     """With valid arguments and no usable device the call fails loudly instead of computing."""
     torch = pytest.importorskip("torch")
