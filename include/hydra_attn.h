@@ -103,7 +103,20 @@ int32_t hydra_zigzag_pairs(const int32_t* cu_seqlens_host, int32_t n_seqs, const
 /*
  * Bytes of device workspace the call `which` (HYDRA_WS_*) needs for this problem. pairs == NULL
  * with n_pairs == 0 means one whole-sequence pair per sequence. Returns 0 on invalid input.
+ *
+ * HYDRA_WS_BWD has two sizes. The backward always needs the status block and D (4 bytes per token
+ * and head). If, in addition, the workspace has room for dS of every visible (query, key) position
+ * as bf16 (2 bytes per position and head, laid out in 16 KB blocks), the key-side kernel hands dS to
+ * the query-side kernel through the workspace and the latter computes dq = scale * dS k without
+ * recomputing the scores (the backward then executes 1664 instead of 2304 FLOP per position). This
+ * function returns the larger size while the hand-off buffer stays within the limit set with
+ * hydra_set_bwd_scratch_limit (default 4 GiB; 0 switches the hand-off off) and the smaller size
+ * otherwise; hydra_attn_bwd uses the hand-off whenever the workspace it is given is large enough and
+ * the buffer is within the limit. The results of the two forms agree to the rounding of dS to bf16,
+ * which both apply. The size assumes a causal call; a non-causal call needs about twice the buffer
+ * and falls back to recomputation in a workspace sized here.
  */
+void hydra_set_bwd_scratch_limit(uint64_t bytes);
 size_t hydra_workspace_bytes(int32_t which, const int32_t* cu_seqlens_host, int32_t n_seqs,
                              int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs);
 

@@ -78,6 +78,8 @@ def _load() -> ctypes.CDLL:
     lib.hydra_attn_bwd.restype = i32
     lib.hydra_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, vp, i32, i32, f32, vp, vp, vp,
                                    vp, sz, vp]
+    lib.hydra_set_bwd_scratch_limit.restype = None
+    lib.hydra_set_bwd_scratch_limit.argtypes = [ctypes.c_uint64]
     lib.hydra_attn_bwd_accumulate.restype = i32
     lib.hydra_attn_bwd_accumulate.argtypes = lib.hydra_attn_bwd.argtypes
     lib.hydra_grad_cast.restype = i32
@@ -106,7 +108,7 @@ EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
            "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc", "hydra_lse_merge_accumulate",
            "hydra_sched_targets", "hydra_sched_cp", "hydra_sched_pack", "hydra_attn_bwd_accumulate",
-           "hydra_grad_cast")
+           "hydra_grad_cast", "hydra_set_bwd_scratch_limit")
 KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast")
 
 
@@ -302,6 +304,11 @@ def hydra_attn_bwd_accumulate(q, k, v, out, lse, dout, cu_seqlens, n_heads: int,
     if check:
         _check(s, "hydra_attn_bwd_accumulate")
     return s
+
+
+def hydra_set_bwd_scratch_limit(n_bytes: int) -> None:
+    """Largest dS hand-off buffer the backward may ask for and use (0: always recompute)."""
+    _lib.hydra_set_bwd_scratch_limit(int(n_bytes))
 
 
 def hydra_grad_cast(acc, grad, n_elements: Optional[int] = None, stream=None, check: bool = True) -> int:

@@ -180,6 +180,7 @@ struct Plan {
     DeviceBlob blob;
     size_t off_pairs = 0, off_items = 0, off_lists = 0, off_groups = 0, off_items2 = 0, off_lists2 = 0;
     int32_t n_items = 0, n_items2 = 0;
+    int64_t ds_head_blocks = 0;      // backward: blocks of the dS hand-off buffer per head; -1: not usable
 };
 
 std::mutex g_plan_mutex;
@@ -213,7 +214,7 @@ std::vector<PairDev> device_pairs(const Problem& pb)
         d.off = p.q_start - p.k_start;
         d.to_part = p.part_row >= 0;
         d.out_row0 = d.to_part ? p.part_row : d.q_tok0;
-        d.pad = 0;
+        d.ds_base = 0;
         v.push_back(d);
     }
     return v;
@@ -313,6 +314,26 @@ void build_merge(const Problem& pb, Plan& plan, std::vector<uint8_t>& blob)
 }
 
 // Backward lists: pairs grouped by q chunk (dQ kernel) and by kv chunk (dK/dV kernel).
+// Lays the pairs out in the dS hand-off buffer (see DsGeom): returns the number of 16 KB blocks per
+// head and, if `dev` is given, writes every pair's first block. -1 if a pair has a kv tile whose first
+// visible q sub-tile lies beyond the pair's q rows (possible only for pairs that are not chunk pairs of
+// a cut sequence); the backward then recomputes S and dP on the query side instead.
+int64_t ds_layout(const Problem& pb, int causal, std::vector<PairDev>* dev)
+{
+    int64_t blocks = 0;
+    for (size_t i = 0; i < pb.pairs.size(); ++i) {
+        const auto& p = pb.pairs[i];
+        if (dev) (*dev)[i].ds_base = static_cast<int32_t>(blocks);
+        if (p.q_len <= 0 || p.k_len <= 0) continue;
+        const DsGeom g = ds_geom(p.q_len, p.q_start - p.k_start, causal);
+        const int32_t nk = (p.k_len + TILE - 1) / TILE;
+        if (ds_first(g, nk - 1) > g.nu_even) return -1;
+        blocks += ds_rowstart(g, nk);
+        if (blocks > (int64_t{1} << 30)) return -1;
+    }
+    return blocks + 1;                                  // one spare block: a q tile is read as two blocks
+}
+
 void build_bwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& blob)
 {
     const int32_t n = static_cast<int32_t>(pb.pairs.size());
@@ -376,7 +397,9 @@ void build_bwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& 
     std::vector<GroupItem> items_q, items_k;
     group_by(true, lists_q, items_q);
     group_by(false, lists_k, items_k);
-    plan.off_pairs = append(blob, device_pairs(pb));
+    std::vector<PairDev> dev = device_pairs(pb);
+    plan.ds_head_blocks = ds_layout(pb, causal, &dev);
+    plan.off_pairs = append(blob, dev);
     plan.off_lists = append(blob, lists_q);
     plan.off_items = append(blob, items_q);
     plan.off_lists2 = append(blob, lists_k);
@@ -469,6 +492,23 @@ int32_t make_map(CUtensorMap* map, const void* base, int64_t T, int32_t h, int32
     const cuuint32_t es[3] = {1, 1, 1};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides,
                            box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? HYDRA_OK : HYDRA_ERR_CUDA;
+}
+
+// The dS hand-off buffer as a 2-D tensor: rows of 64 bf16, 128 rows per block; a box is two blocks.
+// `store`: the map the key-side kernel writes through (a warp's 32 rows x 32 columns, not swizzled).
+int32_t make_map_ds(CUtensorMap* map, const void* base, int64_t blocks, bool store)
+{
+    EncodeFn enc = encode_fn();
+    if (!enc) return HYDRA_ERR_CUDA;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(SUB), static_cast<cuuint64_t>(blocks) * TILE};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(SUB) * 2};
+    const cuuint32_t box_load[2] = {static_cast<cuuint32_t>(SUB), 2 * TILE}, box_store[2] = {32, 32};
+    const cuuint32_t es[2] = {1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
+                           store ? box_store : box_load, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           store ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? HYDRA_OK : HYDRA_ERR_CUDA;
 }
@@ -605,6 +645,24 @@ int32_t hydra_zigzag_pairs(const int32_t* cu, int32_t n_seqs, const int32_t* cp_
     return n_pairs > max_pairs ? HYDRA_ERR_WORKSPACE_TOO_SMALL : HYDRA_OK;
 }
 
+namespace {
+std::atomic<uint64_t> g_ds_limit_bytes{uint64_t{4} << 30};
+
+size_t bwd_base_bytes(const Problem& pb)
+{
+    return align_up(kStatusBytes + align_up(static_cast<size_t>(pb.T) * pb.h * sizeof(float), 256), 1024);
+}
+// bytes of the dS hand-off buffer, or 0 if it is not to be used (layout not possible, or over the limit)
+size_t bwd_ds_bytes(int64_t head_blocks, int32_t n_heads)
+{
+    if (head_blocks <= 0) return 0;
+    const uint64_t bytes = static_cast<uint64_t>(head_blocks) * n_heads * DS_BLOCK_BYTES;
+    return bytes <= g_ds_limit_bytes.load() ? static_cast<size_t>(bytes) : 0;
+}
+}  // namespace
+
+void hydra_set_bwd_scratch_limit(uint64_t bytes) { g_ds_limit_bytes.store(bytes); }
+
 size_t hydra_workspace_bytes(int32_t which, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
                              const hydra_pair_t* pairs, int32_t n_pairs)
 {
@@ -613,7 +671,12 @@ size_t hydra_workspace_bytes(int32_t which, const int32_t* cu, int32_t n_seqs, i
     switch (which) {
         case HYDRA_WS_FWD:
         case HYDRA_WS_MERGE: return kStatusBytes;
-        case HYDRA_WS_BWD: return kStatusBytes + align_up(static_cast<size_t>(pb.T) * n_heads * sizeof(float), 256);
+        case HYDRA_WS_BWD: {
+            // D, plus the dS hand-off buffer when it stays within the limit (sized for a causal call)
+            const size_t base = bwd_base_bytes(pb);
+            const size_t ds = bwd_ds_bytes(ds_layout(pb, 1, nullptr), n_heads);
+            return ds ? base + ds : base;
+        }
         default: return 0;
     }
 }
@@ -742,6 +805,7 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
     if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
     const size_t need = kStatusBytes + align_up(static_cast<size_t>(pb.T) * n_heads * sizeof(float), 256);
     if (workspace_bytes < need) return HYDRA_ERR_WORKSPACE_TOO_SMALL;
+    const size_t ds_off = bwd_base_bytes(pb);
     if (pb.T == 0 || pb.pairs.empty()) return HYDRA_OK;
     const void* ptrs[] = {q, k, v, out, lse, dout, dq, dk, dv};
     for (const void* p : ptrs)
@@ -781,12 +845,24 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
     bp.accumulate = accumulate ? 1 : 0;
     bp.status = static_cast<StatusBlock*>(workspace);
     bp.wait_limit_ns = g_wait_limit_ns.load();
+    // dS hand-off: the key-side kernel leaves dS^T in the workspace and the query-side kernel only
+    // multiplies it with K, if the buffer fits the workspace given and the limit set
+    const size_t ds_bytes = bwd_ds_bytes(plan->ds_head_blocks, n_heads);
+    const bool hand_off = ds_bytes > 0 && workspace_bytes >= ds_off + ds_bytes;
+    CUtensorMap mds, mds_st;
+    {
+        // without the hand-off the maps are never used; they then cover the D array so that they are valid
+        void* base = hand_off ? static_cast<uint8_t*>(workspace) + ds_off : static_cast<void*>(dsum);
+        const int64_t blocks = hand_off ? plan->ds_head_blocks * n_heads : 1;
+        if (hand_off) { bp.ds = base; bp.ds_head_blocks = plan->ds_head_blocks; }
+        if (make_map_ds(&mds, base, blocks, false) || make_map_ds(&mds_st, base, blocks, true)) return HYDRA_ERR_CUDA;
+    }
     if (plan->n_items2 > 0) {
         bp.lists = at<int32_t>(*plan, plan->off_lists2);
         bp.items = at<GroupItem>(*plan, plan->off_items2);
         bp.n_items = plan->n_items2;
         ScopedKernelTimer timer(K_DKV, stream);
-        if (launch_bwd_dkv(mq_sub, mk, mv, mdo_sub, bp, sms, stream) != cudaSuccess)
+        if (launch_bwd_dkv(mq_sub, mk, mv, mdo_sub, mds_st, bp, sms, stream) != cudaSuccess)
             return HYDRA_ERR_CUDA;
         g_launches += 1;
     }
@@ -795,7 +871,9 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
         bp.items = at<GroupItem>(*plan, plan->off_items);
         bp.n_items = plan->n_items;
         ScopedKernelTimer timer(K_DQ, stream);
-        if (launch_bwd_dq(mq, mk, mv, mdo, bp, sms, stream) != cudaSuccess)
+        const cudaError_t e = hand_off ? launch_bwd_dq_from_ds(mds, mk, bp, sms, stream)
+                                       : launch_bwd_dq(mq, mk, mv, mdo, bp, sms, stream);
+        if (e != cudaSuccess)
             return HYDRA_ERR_CUDA;
         g_launches += 1;
     }

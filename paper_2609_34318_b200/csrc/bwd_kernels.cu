@@ -115,7 +115,8 @@ constexpr uint32_t kK = 0;                                   // 3 boxes of 128 r
 constexpr uint32_t kV = kK + 3 * kBox128;                    // 2 boxes of 128 rows, stationary
 constexpr uint32_t kQ = kV + 2 * kBox128;                    // stages x 3 boxes of 64 rows
 constexpr uint32_t kDO = kQ + kStages * 3 * kBox64;          // stages x 2 boxes of 64 rows
-constexpr uint32_t kTotal = kDO + kStages * 2 * kBox64;      // 204,800 B
+constexpr uint32_t kDsStage = kDO + kStages * 2 * kBox64;    // 8 warps x 2 KB: dS^T on its way to memory
+constexpr uint32_t kTotal = kDsStage + 8 * 2048;             // 221,184 B
 constexpr uint32_t kTmDK = 0, kTmDV = 192, kTmS = 320, kTmDP = 384, kTmP = 448, kTmDS = 480,
                    kTmCols = 512;
 enum : int { B_KVFULL = 0, B_KVEMPTY = 1, B_QFULL = 2, B_STAT = 5, B_QEMPTY = 8, B_SFULL = 11,
@@ -124,7 +125,7 @@ enum : int { B_KVFULL = 0, B_KVEMPTY = 1, B_QFULL = 2, B_STAT = 5, B_QEMPTY = 8,
 
 // Iterator over (pair of the kv chunk, 64-row q sub-tile).
 struct SubIter {
-    const PairDev* pairs; const int32_t* list; int list_len; int r0; int causal;
+    const PairDev* pairs; const int32_t* list; int list_len; int r0; int causal; int even;
     int li, u, nu; PairDev cur;
     __device__ void seek() {
         while (li < list_len) {
@@ -132,12 +133,15 @@ struct SubIter {
             nu = (cur.q_len + SUB - 1) / SUB;
             u = 0;
             if (causal) { const int i_min = r0 - cur.off; u = i_min > 0 ? i_min / SUB : 0; }
+            // with the dS hand-off a q tile is read as two sub-tiles: start at the even one (the extra
+            // sub-tile, if any, is fully masked and contributes zeros)
+            if (even) u &= ~1;
             if (u < nu) return;
             ++li;
         }
     }
-    __device__ void init(const PairDev* p, const int32_t* l, int n, int r, int c) {
-        pairs = p; list = l; list_len = n; r0 = r; causal = c; li = 0; u = 0; nu = 0;
+    __device__ void init(const PairDev* p, const int32_t* l, int n, int r, int c, int ev) {
+        pairs = p; list = l; list_len = n; r0 = r; causal = c; even = ev; li = 0; u = 0; nu = 0;
         seek();
     }
     __device__ bool valid() const { return li < list_len; }
@@ -519,7 +523,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 __global__ void __launch_bounds__(kThreads, 1)
 hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
-                     const BwdParams p)
+                     const __grid_constant__ CUtensorMap map_ds, const BwdParams p)
 {
     using namespace dkv;
     extern __shared__ uint8_t smem_raw[];
@@ -597,7 +601,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const int32_t* list = p.lists + item.list_off;
             const PairDev first = p.pairs[list[0]];
             SubIter si;
-            si.init(p.pairs, list, item.list_len, item.r0, p.causal);
+            si.init(p.pairs, list, item.list_len, item.r0, p.causal, p.ds != nullptr);
             if (!si.valid()) continue;
             ok = wait(B_KVEMPTY, items ^ 1u);
             if (!ok) break;
@@ -663,7 +667,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 const GroupItem item = p.items[it];
                 const int32_t* list = p.lists + item.list_off;
                 SubIter si;
-                si.init(p.pairs, list, item.list_len, item.r0, p.causal);
+                si.init(p.pairs, list, item.list_len, item.r0, p.causal, p.ds != nullptr);
                 if (!si.valid()) continue;
                 if (issue_scores) {
                     ok = wait(B_KVFULL, items);
@@ -742,6 +746,8 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const uint32_t tm_p = tm + kTmP + lane_base + g * 16;
         const uint32_t tm_ds = tm + kTmDS + lane_base + g * 16;
         uint32_t c_s = 0, c_pds = 0, gq = 0;
+        int ds_li = -1;                                // pair whose first hand-off block is in ds_blk0
+        int64_t ds_blk0 = 0;
         bool ok = true;
         for (uint32_t kq = 0; ok; ++kq) {
             const int it = next_item(kq);
@@ -749,6 +755,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const GroupItem item = p.items[it];
             const int32_t* list = p.lists + item.list_off;
             const PairDev first = p.pairs[list[0]];
+            ds_li = -1;
             const int krow = item.r0 + r;              // kv row inside the chunk
             const bool row_valid = krow < first.k_len;
             const int64_t tok = static_cast<int64_t>(first.k_tok0) + krow;
@@ -759,7 +766,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             float* dkp_acc = static_cast<float*>(p.dk) + dk_off;         // accumulate mode: dk, dv are fp32
             float* dvp_acc = static_cast<float*>(p.dv) + dv_off;
             SubIter si;
-            si.init(p.pairs, list, item.list_len, item.r0, p.causal);
+            si.init(p.pairs, list, item.list_len, item.r0, p.causal, p.ds != nullptr);
             if (!si.valid()) {                         // no q row sees this tile: dK = dV = 0 (nothing to add)
                 if (row_valid && !p.accumulate) {
                     uint4* a4 = reinterpret_cast<uint4*>(dkp);
@@ -830,6 +837,35 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 tc_fence_before_sync();
                 mbar_arrive_warp(bar(B_PFULL));
                 ++c_pds;
+                if (p.ds) {
+                    // Hand dS^T to the query-side kernel: the warp's 32 rows x 64 bytes go to a 2 KB slice of
+                    // shared memory and from there to the block in memory as one tiled store (a direct store
+                    // from registers would touch 32 cache lines per instruction).
+                    if (si.li != ds_li) {
+                        ds_li = si.li;
+                        const DsGeom geo = ds_geom(si.cur.q_len, si.cur.off, p.causal);
+                        const int jk = item.r0 / TILE;
+                        ds_blk0 = static_cast<int64_t>(item.head) * p.ds_head_blocks + si.cur.ds_base +
+                                  ds_rowstart(geo, jk) - ds_first(geo, jk);
+                    }
+                    // transpose through the slice so that every store instruction of the warp writes whole
+                    // 64-byte row segments: lane l holds row l; afterwards it holds chunk l % 4 of rows l / 4 + 8 e
+                    const uint32_t slice = smem + kDsStage + warp * 2048;
+                    __syncwarp();                      // the reads of the previous sub-tile are over
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        st_shared_v4(slice + lane * 64 + ((e ^ ((lane >> 1) & 3)) << 4), ds[4 * e], ds[4 * e + 1],
+                                     ds[4 * e + 2], ds[4 * e + 3]);
+                    __syncwarp();
+                    uint8_t* blk = static_cast<uint8_t*>(p.ds) + (ds_blk0 + si.u) * DS_BLOCK_BYTES +
+                                   ((warp & 3) * 32 + (lane >> 2)) * (SUB * 2) + g * 64 + (lane & 3) * 16;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int row = 8 * e + (lane >> 2);
+                        const uint4 w = ld_shared_v4(slice + row * 64 + (((lane & 3) ^ ((row >> 1) & 3)) << 4));
+                        st_global_stream_v4(blk + e * 8 * (SUB * 2), w);
+                    }
+                }
             }
             if (!ok) break;
             // ---- epilogue: dK * scale, dV -> bf16; each warpgroup writes half of the columns -------
@@ -879,6 +915,237 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     if (warp == kWarpMma) tmem_dealloc(tm, kTmCols);
 }
 
+// =============================================================================================
+// dQ from the dS hand-off buffer
+// =============================================================================================
+// When the key-side kernel has left dS^T in memory, dQ = scale * dS K needs no recomputation of S
+// and dP: per (q tile, kv tile) one product of 128 x 192 x 128, both operands straight from their TMA
+// tiles (dS^T blocks as an MN-major A operand, the K tile as an MN-major B operand). The kernel is
+// bound by the stream of dS (2 bytes per 384 FLOP), so it is a plain load -> UMMA -> store pipeline:
+//   warps 0-3  epilogue (thread r = q row r): dQ * scale -> bf16 (or fp32 reductions)
+//   warp  4    TMA producer: per kv tile the two dS^T blocks of the q tile (32 KB) and the K tile (48 KB)
+//   warp  5    UMMA issuer; two accumulators in tensor memory, so the epilogue of one work item
+//              overlaps the products of the next
+namespace dqs {
+constexpr int kThreadsS = 192;
+constexpr int kStages = 2;
+constexpr uint32_t kDsBytes = 2 * DS_BLOCK_BYTES;            // blocks (jk, 2i) and (jk, 2i + 1)
+constexpr uint32_t kStage = kDsBytes + 3 * kBox128;          // + K tile
+constexpr uint32_t kTotal = kStages * kStage;                // 163,840 B
+constexpr uint32_t kTmAcc = 256, kTmCols = 512;              // accumulators at columns 0 and 256
+enum : int { B_FULL = 0, B_EMPTY = kStages, B_ACCFULL = 2 * kStages, B_ACCFREE = 2 * kStages + 2,
+             B_ITEMFULL = 2 * kStages + 4, B_ITEMEMPTY = 2 * kStages + 4 + kSched,
+             B_COUNT = 2 * kStages + 4 + 2 * kSched };
+}  // namespace dqs
+
+size_t bwd_dq_ds_smem_bytes() { return dqs::kTotal + 1024; }
+
+__global__ void __launch_bounds__(dqs::kThreadsS, 1)
+hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __grid_constant__ CUtensorMap map_k,
+                            const BwdParams p)
+{
+    using namespace dqs;
+    using dq::TileIter;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    __shared__ __align__(8) uint64_t bars[B_COUNT];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    __shared__ int32_t s_sched[kSched];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t bar0 = smem_u32(&bars[0]);
+    auto bar = [&](int i) -> uint32_t { return bar0 + 8u * static_cast<uint32_t>(i); };
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int i = 0; i < B_COUNT; ++i) {
+            uint32_t count = 1u;
+            if (i == B_ACCFREE || i == B_ACCFREE + 1) count = 4u;             // epilogue warps
+            if (i >= B_ITEMEMPTY && i < B_ITEMEMPTY + kSched) count = 5u;    // + the issuer warp
+            mbar_init(bar(i), count);
+        }
+        fence_mbar_init();
+        tma_prefetch_desc(&map_ds); tma_prefetch_desc(&map_k);
+    }
+    if (warp == 5) { tmem_alloc(smem_u32(&tmem_base_slot), kTmCols); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tm = tmem_base_slot;
+    const uint64_t limit = p.wait_limit_ns;
+    volatile int* abort_p = &abort_flag;
+    auto wait = [&](int b, uint32_t parity) -> bool { return mbar_wait(bar(b), parity & 1u, abort_p, limit); };
+    volatile int32_t* sched = s_sched;
+    auto pop_item = [&](uint32_t k) -> int {                 // producer, one thread
+        const int slot = k % kSched;
+        if (!mbar_wait(bar(B_ITEMEMPTY + slot), ((k / kSched) ^ 1u) & 1u, abort_p, limit)) return -1;
+        int idx = atomicAdd(&p.status->next_item[QUEUE_DQ], 1);
+        if (idx >= p.n_items) idx = -1;
+        sched[slot] = idx;
+        mbar_arrive(bar(B_ITEMFULL + slot));
+        return idx;
+    };
+    auto next_item = [&](uint32_t k) -> int {                // every other warp, all lanes
+        const int slot = k % kSched;
+        if (!mbar_wait(bar(B_ITEMFULL + slot), (k / kSched) & 1u, abort_p, limit)) return -1;
+        const int idx = sched[slot];
+        mbar_arrive_warp(bar(B_ITEMEMPTY + slot));
+        return idx;
+    };
+
+    if (warp == 4) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t g = 0;
+            bool ok = true;
+            const uint64_t ds_policy = l2_policy_evict_first();
+            int it_ahead = pop_item(0);
+            for (uint32_t kq = 0; ok; ++kq) {
+                const int it = it_ahead;
+                if (it < 0) break;
+                it_ahead = pop_item(kq + 1);
+                const GroupItem item = p.items[it];
+                const int32_t* list = p.lists + item.list_off;
+                const PairDev first = p.pairs[list[0]];
+                TileIter ti;
+                ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+                const int u0 = item.r0 / SUB;                  // first sub-tile of this q tile
+                for (; ti.valid() && ok; ti.next(), ++g) {
+                    const int st = g % kStages;
+                    ok = wait(B_EMPTY + st, (g / kStages) ^ 1u);
+                    if (!ok) break;
+                    const DsGeom geo = ds_geom(ti.cur.q_len, ti.cur.off, p.causal);
+                    const int64_t blk = static_cast<int64_t>(item.head) * p.ds_head_blocks + ti.cur.ds_base +
+                                        ds_rowstart(geo, ti.t) + (u0 - ds_first(geo, ti.t));
+                    const uint32_t dst = smem + st * kStage;
+                    mbar_arrive_expect_tx(bar(B_FULL + st), kStage);
+                    tma_load_2d_hint(dst, &map_ds, bar(B_FULL + st), 0, static_cast<int>(blk * TILE), ds_policy);
+                    for (int c = 0; c < 3; ++c)
+                        tma_load_3d(dst + kDsBytes + c * kBox128, &map_k, bar(B_FULL + st), c * 64, item.head,
+                                    ti.cur.k_tok0 + ti.t * TILE);
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ UMMA issuer
+        constexpr uint32_t idesc = umma_idesc_bf16(TILE, D_QK, true, true);
+        constexpr uint32_t hi_ds = umma_desc_hi(DS_BLOCK_BYTES, 1024);   // dS^T: M chunks of 64 q rows 16 KB apart
+        constexpr uint32_t hi_k = umma_desc_hi(kBox128, 1024);           // K: N chunks of 64 columns 16 KB apart
+        uint32_t g = 0, n_acc = 0;
+        bool ok = true;
+        for (uint32_t kq = 0; ok; ++kq) {
+            const int it = next_item(kq);
+            if (it < 0) break;
+            const GroupItem item = p.items[it];
+            const int32_t* list = p.lists + item.list_off;
+            const PairDev first = p.pairs[list[0]];
+            TileIter ti;
+            ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+            if (!ti.valid()) continue;
+            const uint32_t buf = n_acc & 1u;
+            ok = wait(B_ACCFREE + buf, (n_acc >> 1) ^ 1u);
+            if (!ok) break;
+            bool first_tile = true;
+            for (; ti.valid() && ok; ti.next(), ++g) {
+                const int st = g % kStages;
+                ok = wait(B_FULL + st, g / kStages);
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (elect_one()) {
+                    const uint32_t a_lo = umma_desc_lo(smem + st * kStage, DS_BLOCK_BYTES);
+                    const uint32_t b_lo = umma_desc_lo(smem + st * kStage + kDsBytes, kBox128);
+#pragma unroll
+                    for (int kk = 0; kk < TILE / 16; ++kk)
+                        umma_ss_w(tm + buf * kTmAcc, a_lo + kk * (2048 >> 4), hi_ds, b_lo + kk * (2048 >> 4), hi_k, idesc,
+                                  (kk > 0 || !first_tile) ? 1u : 0u);
+                    umma_commit(bar(B_EMPTY + st));
+                }
+                first_tile = false;
+            }
+            if (ok && elect_one()) umma_commit(bar(B_ACCFULL + buf));
+            __syncwarp();
+            ++n_acc;
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        const int r = tid;                             // q row inside the tile = TMEM lane
+        const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+        uint32_t n_acc = 0;
+        bool ok = true;
+        for (uint32_t kq = 0; ok; ++kq) {
+            const int it = next_item(kq);
+            if (it < 0) break;
+            const GroupItem item = p.items[it];
+            const int32_t* list = p.lists + item.list_off;
+            const PairDev first = p.pairs[list[0]];
+            const int row = item.r0 + r;
+            const bool row_valid = row < first.q_len;
+            const int64_t dst_off = (static_cast<int64_t>(first.q_tok0 + row) * p.h + item.head) * D_QK;
+            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.dq) + dst_off;
+            float* dst_acc = static_cast<float*>(p.dq) + dst_off;
+            TileIter ti;
+            ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+            if (!ti.valid()) {                         // no visible key at all: dQ = 0 (nothing to add)
+                if (row_valid && !p.accumulate) {
+                    uint4* d4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+                    for (int e = 0; e < 24; ++e) d4[e] = make_uint4(0u, 0u, 0u, 0u);
+                }
+                continue;
+            }
+            const uint32_t buf = n_acc & 1u;
+            ok = wait(B_ACCFULL + buf, n_acc >> 1);
+            if (!ok) break;
+            tc_fence_after_sync();
+#pragma unroll
+            for (int c0 = 0; c0 < D_QK; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld_x32(tm + buf * kTmAcc + lane_base + c0, v);
+                tmem_wait_ld();
+                if (c0 + 32 == D_QK) {
+                    tc_fence_before_sync();
+                    mbar_arrive_warp(bar(B_ACCFREE + buf));
+                }
+                if (row_valid) {
+                    if (p.accumulate) add_row_f32(dst_acc + c0, v, 32, p.scale);
+                    else store_row_bf16(dst + c0, v, 32, p.scale);
+                }
+            }
+            ++n_acc;
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (abort_flag) {
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 50000ull) { }
+        if (tid == 0) {
+            p.status->detail = blockIdx.x;
+            p.status->status = HYDRA_ERR_DEVICE_TIMEOUT;
+        }
+        __syncthreads();
+    }
+    if (warp == 5) tmem_dealloc(tm, kTmCols);
+}
+
+cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mds, const CUtensorMap& mk, const BwdParams& p, int grid,
+                                  cudaStream_t stream)
+{
+    static bool configured = false;
+    if (!configured) {
+        const cudaError_t e = cudaFuncSetAttribute(hydra_bwd_dq_from_ds_kernel,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   static_cast<int>(bwd_dq_ds_smem_bytes()));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    hydra_bwd_dq_from_ds_kernel<<<grid, dqs::kThreadsS, bwd_dq_ds_smem_bytes(), stream>>>(mds, mk, p);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_bwd_dq(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                           const CUtensorMap& mdo, const BwdParams& p, int grid, cudaStream_t stream)
 {
@@ -894,7 +1161,8 @@ cudaError_t launch_bwd_dq(const CUtensorMap& mq, const CUtensorMap& mk, const CU
 }
 
 cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, const CUtensorMap& mv,
-                           const CUtensorMap& mdo_sub, const BwdParams& p, int grid, cudaStream_t stream)
+                           const CUtensorMap& mdo_sub, const CUtensorMap& mds_st, const BwdParams& p, int grid,
+                           cudaStream_t stream)
 {
     static bool configured = false;
     if (!configured) {
@@ -903,7 +1171,7 @@ cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, con
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    hydra_bwd_dkv_kernel<<<grid, kThreads, bwd_dkv_smem_bytes(), stream>>>(mq_sub, mk, mv, mdo_sub, p);
+    hydra_bwd_dkv_kernel<<<grid, kThreads, bwd_dkv_smem_bytes(), stream>>>(mq_sub, mk, mv, mdo_sub, mds_st, p);
     return cudaGetLastError();
 }
 

@@ -22,8 +22,37 @@ struct PairDev {
     int32_t off;       // q_start - k_start: key j is visible to q row i iff j <= i + off (causal)
     int32_t out_row0;  // first output row: part_row (partial buffers) or q_tok0 (out / lse)
     int32_t to_part;   // 1: partial buffers, 0: out / lse
-    int32_t pad;
+    int32_t ds_base;   // backward: first block of this pair in the dS hand-off buffer (per head)
 };
+
+// Geometry of the dS hand-off buffer of the backward. The key-side kernel writes dS^T of every
+// (128-row kv tile jk, 64-row q sub-tile u) it visits as one block of 128 rows x 64 bf16 (16 KB); the
+// query-side kernel reads the blocks (jk, 2i) and (jk, 2i + 1) of its q tile i. Per pair the blocks of
+// kv tile jk start at ds_rowstart(jk) and cover the sub-tiles ds_first(jk) .. nu_even - 1, where
+// ds_first is the first sub-tile the causal mask leaves visible, rounded down to an even number, so
+// that the buffer holds the visible trapezoid only. Both kernels and the host evaluate these forms.
+struct DsGeom { int32_t nu_even; int32_t fo; };
+__host__ __device__ inline DsGeom ds_geom(int32_t q_len, int32_t off, int causal)
+{
+    DsGeom g;
+    g.nu_even = ((q_len + SUB - 1) / SUB + 1) & ~1;
+    // fo = floor(-off / 128): kv tile jk sees q tiles jk + fo and later
+    g.fo = !causal ? -(1 << 24) : (off <= 0 ? (-off) / TILE : -((off + TILE - 1) / TILE));
+    return g;
+}
+__host__ __device__ inline int32_t ds_first(const DsGeom& g, int32_t jk)
+{
+    const int32_t m = jk + g.fo;
+    return m > 0 ? 2 * m : 0;
+}
+__host__ __device__ inline int64_t ds_rowstart(const DsGeom& g, int32_t jk)
+{
+    int64_t m = static_cast<int64_t>(jk) + g.fo;
+    if (m < 0) m = 0;
+    const int64_t m0 = g.fo > 0 ? g.fo : 0;
+    return static_cast<int64_t>(jk) * g.nu_even - (m * (m - 1) - m0 * (m0 - 1));
+}
+constexpr uint32_t DS_BLOCK_BYTES = TILE * SUB * 2;   // 16 KB
 
 // Forward work item: a 256-row slab of q rows of one pair and head = tiles A and B of 128 rows.
 struct FwdItem {
@@ -87,6 +116,8 @@ struct BwdParams {
     int32_t h; int32_t causal;
     float scale; float scale_log2;
     int32_t accumulate;
+    void* ds;                   // dS hand-off buffer, or null: the query-side kernel recomputes S and dP
+    int64_t ds_head_blocks;     // blocks per head
     StatusBlock* status;
     uint64_t wait_limit_ns;
 };
@@ -112,8 +143,11 @@ cudaError_t launch_fwd(const CUtensorMap& mq, const CUtensorMap& mk, const CUten
                        const FwdParams& p, int grid, cudaStream_t stream);
 cudaError_t launch_bwd_dq(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                           const CUtensorMap& mdo, const BwdParams& p, int grid, cudaStream_t stream);
+size_t bwd_dq_ds_smem_bytes();
+cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mds, const CUtensorMap& mk, const BwdParams& p, int grid,
+                                  cudaStream_t stream);
 cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, const CUtensorMap& mv,
-                           const CUtensorMap& mdo_sub, const BwdParams& p, int grid,
+                           const CUtensorMap& mdo_sub, const CUtensorMap& mds_st, const BwdParams& p, int grid,
                            cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
 cudaError_t launch_grad_cast(const float* acc, void* grad, int64_t n, cudaStream_t stream);

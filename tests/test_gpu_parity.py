@@ -14,6 +14,17 @@ pytestmark = pytest.mark.gpu
 DQK, DV = hw.D_QK, hw.D_V
 
 
+@pytest.fixture(autouse=True, params=["hand_off", "recompute"])
+def backward_form(request):
+    """Every case runs with both forms of the backward: dS handed from the key-side kernel to the
+    query-side kernel through the workspace (the default while the buffer stays under the limit), and
+    S / dP recomputed on the query side (limit 0)."""
+    import paper_2609_34318_b200 as P
+    P.hydra_set_bwd_scratch_limit(0 if request.param == "recompute" else 4 << 30)
+    yield request.param
+    P.hydra_set_bwd_scratch_limit(4 << 30)
+
+
 def rand_inputs(rng, T, h, q_scale=1.0):
     f = lambda d, s=1.0: hw.f32_to_bf16_bits((s * rng.standard_normal((T, h, d))).astype(np.float32))
     return dict(q=f(DQK, q_scale), k=f(DQK), v=f(DV), do=f(DV))
@@ -161,3 +172,27 @@ def test_rows_outside_the_listed_pairs_are_left_untouched():
     assert np.isnan(got["out"][:200]).all() and np.isnan(got["dq"][:200]).all()
     ref = run_oracle({n: a[200:] for n, a in x.items()}, hw.cu_seqlens([150]))
     check({n: (got[n][:, 200:] if n == "lse" else got[n][200:]) for n in ref}, ref)
+
+
+def test_the_two_backward_forms_are_both_exercised_and_agree(backward_form):
+    import paper_2609_34318_b200 as P
+    lengths, h = [700, 130, 64], 3
+    cu = hw.cu_seqlens(lengths)
+    x = rand_inputs(np.random.default_rng(99), int(cu[-1]), h)
+    ws_here = P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h)
+    P.hydra_set_bwd_scratch_limit(0)
+    ws_small = P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h)
+    P.hydra_set_bwd_scratch_limit(4 << 30)
+    ws_large = P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h)
+    assert ws_large > ws_small >= int(cu[-1]) * h * 4
+    # the hand-off buffer holds the visible (q sub-tile, kv tile) blocks of 16 KB per head
+    blocks = (ws_large - ws_small) // (16384 * h)
+    assert 6 * 12 - 6 * 5 + 2 * 4 - 2 + 2 <= blocks <= 6 * 12 + 2 * 4 + 2 + 2
+    assert ws_here == (ws_small if backward_form == "recompute" else ws_large)
+    got_h = run_gpu(x, cu, h)
+    P.hydra_set_bwd_scratch_limit(0)
+    got_r = run_gpu(x, cu, h)
+    for n in ("dq", "dk", "dv"):
+        scale = np.abs(got_r[n]).max()
+        assert np.abs(got_h[n] - got_r[n]).max() <= 2 ** -7 * scale, n
+    assert np.array_equal(got_h["dk"], got_r["dk"]) and np.array_equal(got_h["dv"], got_r["dv"])
