@@ -497,18 +497,16 @@ int32_t make_map(CUtensorMap* map, const void* base, int64_t T, int32_t h, int32
 }
 
 // The dS hand-off buffer as a 2-D tensor: rows of 64 bf16, 128 rows per block; a box is two blocks.
-// `store`: the map the key-side kernel writes through (a warp's 32 rows x 32 columns, not swizzled).
-int32_t make_map_ds(CUtensorMap* map, const void* base, int64_t blocks, bool store)
+int32_t make_map_ds(CUtensorMap* map, const void* base, int64_t blocks)
 {
     EncodeFn enc = encode_fn();
     if (!enc) return HYDRA_ERR_CUDA;
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(SUB), static_cast<cuuint64_t>(blocks) * TILE};
     const cuuint64_t strides[1] = {static_cast<cuuint64_t>(SUB) * 2};
-    const cuuint32_t box_load[2] = {static_cast<cuuint32_t>(SUB), 2 * TILE}, box_store[2] = {32, 32};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(SUB), 2 * TILE};
     const cuuint32_t es[2] = {1, 1};
-    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
-                           store ? box_store : box_load, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           store ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                           es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? HYDRA_OK : HYDRA_ERR_CUDA;
 }
@@ -849,20 +847,18 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
     // multiplies it with K, if the buffer fits the workspace given and the limit set
     const size_t ds_bytes = bwd_ds_bytes(plan->ds_head_blocks, n_heads);
     const bool hand_off = ds_bytes > 0 && workspace_bytes >= ds_off + ds_bytes;
-    CUtensorMap mds, mds_st;
-    {
-        // without the hand-off the maps are never used; they then cover the D array so that they are valid
-        void* base = hand_off ? static_cast<uint8_t*>(workspace) + ds_off : static_cast<void*>(dsum);
-        const int64_t blocks = hand_off ? plan->ds_head_blocks * n_heads : 1;
-        if (hand_off) { bp.ds = base; bp.ds_head_blocks = plan->ds_head_blocks; }
-        if (make_map_ds(&mds, base, blocks, false) || make_map_ds(&mds_st, base, blocks, true)) return HYDRA_ERR_CUDA;
+    CUtensorMap mds;
+    if (hand_off) {
+        bp.ds = static_cast<uint8_t*>(workspace) + ds_off;
+        bp.ds_head_blocks = plan->ds_head_blocks;
+        if (make_map_ds(&mds, bp.ds, plan->ds_head_blocks * n_heads)) return HYDRA_ERR_CUDA;
     }
     if (plan->n_items2 > 0) {
         bp.lists = at<int32_t>(*plan, plan->off_lists2);
         bp.items = at<GroupItem>(*plan, plan->off_items2);
         bp.n_items = plan->n_items2;
         ScopedKernelTimer timer(K_DKV, stream);
-        if (launch_bwd_dkv(mq_sub, mk, mv, mdo_sub, mds_st, bp, sms, stream) != cudaSuccess)
+        if (launch_bwd_dkv(mq_sub, mk, mv, mdo_sub, bp, sms, stream) != cudaSuccess)
             return HYDRA_ERR_CUDA;
         g_launches += 1;
     }

@@ -523,7 +523,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 __global__ void __launch_bounds__(kThreads, 1)
 hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
-                     const __grid_constant__ CUtensorMap map_ds, const BwdParams p)
+                     const BwdParams p)
 {
     using namespace dkv;
     extern __shared__ uint8_t smem_raw[];
@@ -838,9 +838,9 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 mbar_arrive_warp(bar(B_PFULL));
                 ++c_pds;
                 if (p.ds) {
-                    // Hand dS^T to the query-side kernel: the warp's 32 rows x 64 bytes go to a 2 KB slice of
-                    // shared memory and from there to the block in memory as one tiled store (a direct store
-                    // from registers would touch 32 cache lines per instruction).
+                    // Hand dS^T to the query-side kernel (after P and dS have gone to the tensor core: off the
+                    // chain S -> P, dS -> dV, dK). The block in memory is 128 rows of 64 bf16; a store straight
+                    // from registers would touch 32 cache lines per instruction.
                     if (si.li != ds_li) {
                         ds_li = si.li;
                         const DsGeom geo = ds_geom(si.cur.q_len, si.cur.off, p.causal);
@@ -1161,8 +1161,7 @@ cudaError_t launch_bwd_dq(const CUtensorMap& mq, const CUtensorMap& mk, const CU
 }
 
 cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, const CUtensorMap& mv,
-                           const CUtensorMap& mdo_sub, const CUtensorMap& mds_st, const BwdParams& p, int grid,
-                           cudaStream_t stream)
+                           const CUtensorMap& mdo_sub, const BwdParams& p, int grid, cudaStream_t stream)
 {
     static bool configured = false;
     if (!configured) {
@@ -1171,7 +1170,7 @@ cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, con
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    hydra_bwd_dkv_kernel<<<grid, kThreads, bwd_dkv_smem_bytes(), stream>>>(mq_sub, mk, mv, mdo_sub, mds_st, p);
+    hydra_bwd_dkv_kernel<<<grid, kThreads, bwd_dkv_smem_bytes(), stream>>>(mq_sub, mk, mv, mdo_sub, p);
     return cudaGetLastError();
 }
 

@@ -147,8 +147,7 @@ size_t bwd_dq_ds_smem_bytes();
 cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mds, const CUtensorMap& mk, const BwdParams& p, int grid,
                                   cudaStream_t stream);
 cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, const CUtensorMap& mv,
-                           const CUtensorMap& mdo_sub, const CUtensorMap& mds_st, const BwdParams& p, int grid,
-                           cudaStream_t stream);
+                           const CUtensorMap& mdo_sub, const BwdParams& p, int grid, cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
 cudaError_t launch_grad_cast(const float* acc, void* grad, int64_t n, cudaStream_t stream);
 cudaError_t launch_bwd_prep(const void* dout, const void* out, float* dsum, int64_t T, int32_t h,
