@@ -262,6 +262,15 @@ def run_ours(args, w):
     status, detail = step.poll()
     if status != 0:
         raise RuntimeError(f"device status {status} at item {detail}")
+    # The clock inside the kernels, right after the timed region (same thermal and power state): the
+    # driver's clock query above is sampled between kernels and reads the maximum even when a
+    # power-capped kernel runs well below it.
+    for _ in range(2):
+        step.forward(t["q"], t["k"], t["v"])
+        mhz_fwd = P.hydra_poll_clocks(step.workspace)[0]
+        step.backward(t["q"], t["k"], t["v"], t["do"])
+        _, mhz_dkv, mhz_dq = P.hydra_poll_clocks(step.workspace)
+    clocks["in_kernel_mhz"] = {"fwd": round(mhz_fwd), "bwd_dkv": round(mhz_dkv), "bwd_dq": round(mhz_dq)}
 
     flops_step = 3.5 * w.flops_fwd()
     value = whole_job_value(world, flops_step, args.steps, total_ms)
@@ -538,9 +547,9 @@ def merge_groups(pairs):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised in
 # profiles/tensor_kernels_packed32k.md and profiles/merge_prep_short64k_split.md.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "fwd:packed32k": 685094656,
-    "bwd_dkv:packed32k": 995757056,
-    "bwd_dq:packed32k": 875597824,
+    "fwd:packed32k": 686328000,
+    "bwd_dkv:packed32k": 2752725000,      # with the dS hand-off: 1.76 GB of it is dS written once
+    "bwd_dq:packed32k": 2063804000,       # hydra_bwd_dq_from_ds_kernel: 1.76 GB of it is dS read once
     "merge:short64k_split": 764355784,
     "bwd_prep:short64k_split": 1080946776,
 }

@@ -280,6 +280,17 @@ const char* hydra_status_string(int32_t status);
 int32_t hydra_poll_status(void* workspace, void* cuda_stream, int32_t* device_status,
                           int64_t* detail);
 
+/*
+ * SM clock seen from inside the kernels of the last call that used `workspace` (measurement aid, not
+ * part of the method). The producer thread of thread block 0 of every tensor-core kernel reads the
+ * cycle counter and the nanosecond timer when it starts and when it has issued its last load;
+ * mhz_out[3] receives cycles / microsecond for the forward, the key-side backward and the query-side
+ * backward kernel (0 for a kernel the call did not run). Synchronises the stream. On a power-capped
+ * part this is the clock the kernel really ran at; the driver's clock query, sampled between
+ * kernels, is not.
+ */
+int32_t hydra_poll_clocks(void* workspace, void* cuda_stream, double* mhz_out);
+
 /* Kernel launches issued by this process so far (all entry points), for launch accounting. */
 int64_t hydra_launch_count(void);
 

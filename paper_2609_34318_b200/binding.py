@@ -86,6 +86,8 @@ def _load() -> ctypes.CDLL:
     lib.hydra_grad_cast.argtypes = [vp, vp, i64, vp]
     lib.hydra_poll_status.restype = i32
     lib.hydra_poll_status.argtypes = [vp, vp, vp, vp]
+    lib.hydra_poll_clocks.restype = i32
+    lib.hydra_poll_clocks.argtypes = [vp, vp, vp]
     lib.hydra_profile_enable.restype = None
     lib.hydra_profile_enable.argtypes = [i32]
     lib.hydra_profile_collect.restype = i32
@@ -108,7 +110,7 @@ EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
            "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc", "hydra_lse_merge_accumulate",
            "hydra_sched_targets", "hydra_sched_cp", "hydra_sched_pack", "hydra_attn_bwd_accumulate",
-           "hydra_grad_cast", "hydra_set_bwd_scratch_limit")
+           "hydra_grad_cast", "hydra_set_bwd_scratch_limit", "hydra_poll_clocks")
 KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast")
 
 
@@ -326,6 +328,13 @@ def hydra_poll_status(workspace, stream=None) -> Tuple[int, int]:
     _check(_lib.hydra_poll_status(_ptr(workspace), _stream(stream), ctypes.addressof(st),
                                   ctypes.addressof(detail)), "hydra_poll_status")
     return st.value, detail.value
+
+
+def hydra_poll_clocks(workspace, stream=None) -> Tuple[float, float, float]:
+    """SM MHz inside the forward, key-side backward and query-side backward kernels of the last call."""
+    mhz = (ctypes.c_double * 3)()
+    _check(_lib.hydra_poll_clocks(_ptr(workspace), _stream(stream), ctypes.addressof(mhz)), "hydra_poll_clocks")
+    return tuple(mhz)
 
 
 def hydra_profile_enable(on: bool) -> None:

@@ -1086,4 +1086,15 @@ int32_t hydra_poll_status(void* workspace, void* cuda_stream, int32_t* device_st
     return HYDRA_OK;
 }
 
+int32_t hydra_poll_clocks(void* workspace, void* cuda_stream, double* mhz_out)
+{
+    if (!workspace || !mhz_out) return HYDRA_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return HYDRA_ERR_CUDA;
+    StatusBlock sb;
+    if (cudaMemcpy(&sb, workspace, sizeof sb, cudaMemcpyDeviceToHost) != cudaSuccess) return HYDRA_ERR_CUDA;
+    for (int i = 0; i < 3; ++i)
+        mhz_out[i] = sb.probe_ns[i] ? 1e3 * static_cast<double>(sb.probe_cycles[i]) / static_cast<double>(sb.probe_ns[i]) : 0.0;
+    return HYDRA_OK;
+}
+
 }  // extern "C"

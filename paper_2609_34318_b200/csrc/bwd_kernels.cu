@@ -219,6 +219,8 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (lane == 0) {
             uint32_t items = 0, gk = 0, gv = 0;
             bool ok = true;
+            ClockProbe probe;
+            probe.start();
             // one item ahead: the round trip to the counter overlaps the loads of the current item
             int it_ahead = pop_item(0);
             for (uint32_t kq = 0; ok; ++kq) {
@@ -264,6 +266,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     }
                 }
             }
+            if (blockIdx.x == 0) probe.stop(p.status, QUEUE_DQ);
         }
     } else if (warp == kWarpMma || warp == kWarpMma2) {
         // ------------------------------------------------------------------ UMMA issuers
@@ -588,6 +591,8 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         uint32_t items = 0, gq = 0;
         bool ok = true;
         int it_ahead = -1;
+        ClockProbe probe;
+        probe.start();
         for (uint32_t kq = 0; ok; ++kq) {
             int it = 0;
             if (lane == 0) {                          // one pop per CTA, one item ahead, shared with the other lanes
@@ -643,6 +648,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 mbar_arrive_warp(bar(B_STAT + st));
             }
         }
+        if (blockIdx.x == 0 && lane == 0) probe.stop(p.status, QUEUE_DKV);
     } else if (warp == kWarpMma || warp == kWarpMma2) {
         // ------------------------------------------------------------------ UMMA issuers
         // warp 9 issues S^T = K Q^T and dP^T = V dO^T of sub-tile u+1 as soon as those of sub-tile u
@@ -998,7 +1004,9 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
         if (lane == 0) {
             uint32_t g = 0;
             bool ok = true;
-            const uint64_t ds_policy = l2_policy_evict_first();
+            const uint64_t ds_policy = l2_policy_evict_first();   // dS is read once: leave L2 to the K tiles
+            ClockProbe probe;
+            probe.start();
             int it_ahead = pop_item(0);
             for (uint32_t kq = 0; ok; ++kq) {
                 const int it = it_ahead;
@@ -1025,6 +1033,7 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
                                     ti.cur.k_tok0 + ti.t * TILE);
                 }
             }
+            if (blockIdx.x == 0) probe.stop(p.status, QUEUE_DQ);
         }
     } else if (warp == 5) {
         // ------------------------------------------------------------------ UMMA issuer

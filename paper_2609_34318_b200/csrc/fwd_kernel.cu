@@ -133,6 +133,8 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (lane == 0) {
             uint32_t gk = 0, q_use[2] = {0, 0};
             bool ok = true;
+            ClockProbe probe;
+            probe.start();
             // the leader pops one item ahead: the round trip to the counter and the hand-over to the
             // other CTA then overlap the loads of the current item
             int it_ahead = leader ? pop_item(0) : 0;
@@ -169,6 +171,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                                          c * 64, item.head, pr.k_tok0 + j * TILE + rank * 64);
                 }
             }
+            if (blockIdx.x == 0) probe.stop(p.status, QUEUE_FWD);
         }
     } else if (warp == kWarpV) {
         // ------------------------------------------------------------------ V producer

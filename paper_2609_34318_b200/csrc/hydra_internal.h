@@ -90,8 +90,32 @@ struct StatusBlock {            // lives at the start of the workspace; zeroed b
     int32_t pad;
     int64_t detail;
     int32_t next_item[4];       // work-queue heads of the persistent kernels (forward, dK/dV, dQ)
+    // SM clock seen from inside the tensor-core kernels: cycles and nanoseconds that passed in the
+    // producer thread of CTA 0 between its first and its last instruction (same index as next_item)
+    uint64_t probe_cycles[4];
+    uint64_t probe_ns[4];
 };
 enum : int { QUEUE_FWD = 0, QUEUE_DKV = 1, QUEUE_DQ = 2 };
+
+#ifdef __CUDACC__
+// The clock the driver reports between kernels says little about a 1 ms kernel on a power-capped part;
+// the ratio of the cycle counter to the nanosecond timer inside the kernel does.
+struct ClockProbe {
+    long long c0; uint64_t t0;
+    __device__ __forceinline__ void start()
+    {
+        c0 = clock64();
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    }
+    __device__ __forceinline__ void stop(StatusBlock* sb, int queue) const
+    {
+        uint64_t t1;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+        sb->probe_cycles[queue] = static_cast<uint64_t>(clock64() - c0);
+        sb->probe_ns[queue] = t1 - t0;
+    }
+};
+#endif
 
 struct FwdParams {
     const PairDev* pairs;

@@ -190,3 +190,20 @@ def test_grad_cast_ragged_sizes_and_arguments():
     a = torch.zeros(16, device="cuda")
     assert P.hydra_grad_cast(a, a, -1, check=False) == P.HYDRA_ERR_INVALID_ARG
     assert P.hydra_grad_cast(0, a, 8, check=False) == P.HYDRA_ERR_INVALID_ARG
+
+
+def test_clock_probe_reports_a_plausible_sm_clock():
+    import torch
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.runner import AttnStep, bits_to_tensor
+
+    cu = hw.cu_seqlens([2048, 700])
+    x = rand_inputs(np.random.default_rng(1), int(cu[-1]), 2)
+    q, k, v, do = (bits_to_tensor(x[n]) for n in ("q", "k", "v", "do"))
+    step = AttnStep(cu, 2, None, 0, True, None)
+    step.forward(q, k, v)
+    fwd = P.hydra_poll_clocks(step.workspace)
+    step.backward(q, k, v, do)
+    bwd = P.hydra_poll_clocks(step.workspace)
+    assert 300.0 < fwd[0] < 2500.0 and fwd[1] == 0.0 and fwd[2] == 0.0
+    assert bwd[0] == 0.0 and 300.0 < bwd[1] < 2500.0 and 300.0 < bwd[2] < 2500.0
