@@ -150,26 +150,34 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 const FwdItem item = p.items[it];
                 const PairDev pr = p.pairs[item.pair];
                 const int n_t[2] = {item.n_a, item.n_b};
-                for (int t = 0; t < 2 && ok; ++t) {
-                    if (n_t[t] == 0) continue;
+                const int n = max(item.n_a, item.n_b);
+                auto load_q = [&](int t) {
+                    if (n_t[t] == 0 || !ok) return;
                     ok = wait(B_QEMPTY + t, q_use[t] ^ 1u);
-                    if (!ok) break;
+                    if (!ok) return;
                     ++q_use[t];
                     if (leader) mbar_arrive_expect_tx(bar(B_QFULL + t), 2 * kQTile);
                     for (int c = 0; c < 3; ++c)
                         tma_load_3d_pair(smem + kSmemQ + t * kQTile + c * kBox, &map_q, bar(B_QFULL + t), c * 64,
                                          item.head, pr.q_tok0 + item.q0 + t * 2 * TILE + rank * TILE);
-                }
-                const int n = max(item.n_a, item.n_b);
-                for (int j = 0; j < n && ok; ++j, ++gk) {
+                };
+                auto load_k = [&](int j) {
                     const int slot = gk % kKStages;
                     ok = wait(B_KEMPTY + slot, (gk / kKStages) ^ 1u);
-                    if (!ok) break;
+                    if (!ok) return;
+                    ++gk;
                     if (leader) mbar_arrive_expect_tx(bar(B_KFULL + slot), 2 * kKStage);
                     for (int c = 0; c < 3; ++c)
                         tma_load_3d_pair(smem + kSmemK + slot * kKStage + c * kHalfBox, &map_k, bar(B_KFULL + slot),
                                          c * 64, item.head, pr.k_tok0 + j * TILE + rank * 64);
-                }
+                };
+                // The Q buffer of tile B is released by the very last score product of the previous item,
+                // the K stages one and two tiles earlier: ask for the first K tiles before waiting for it.
+                load_q(0);
+                int j = 0;
+                for (; j < n && j < kKStages - 1 && ok; ++j) load_k(j);
+                load_q(1);
+                for (; j < n && ok; ++j) load_k(j);
             }
             if (blockIdx.x == 0) probe.stop(p.status, QUEUE_FWD);
         }
