@@ -654,6 +654,7 @@ size_t bwd_base_bytes(const Problem& pb)
 size_t bwd_ds_bytes(int64_t head_blocks, int32_t n_heads)
 {
     if (head_blocks <= 0) return 0;
+    if (static_cast<uint64_t>(head_blocks) * n_heads * TILE >= (uint64_t{1} << 31)) return 0;   // row index is 32-bit
     const uint64_t bytes = static_cast<uint64_t>(head_blocks) * n_heads * DS_BLOCK_BYTES;
     return bytes <= g_ds_limit_bytes.load() ? static_cast<size_t>(bytes) : 0;
 }

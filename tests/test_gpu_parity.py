@@ -196,3 +196,63 @@ def test_the_two_backward_forms_are_both_exercised_and_agree(backward_form):
         scale = np.abs(got_r[n]).max()
         assert np.abs(got_h[n] - got_r[n]).max() <= 2 ** -7 * scale, n
     assert np.array_equal(got_h["dk"], got_r["dk"]) and np.array_equal(got_h["dv"], got_r["dv"])
+
+
+# ------------------------------------------------------------------------------------------------
+# geometry: random chunkings and hand-made pairs (both forms of the backward, see the fixture)
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", range(6))
+def test_random_length_mixes_and_per_sequence_ring_degrees(seed):
+    rng = np.random.default_rng(1000 + seed)
+    n = int(rng.integers(1, 6))
+    lengths = [int(x) for x in rng.choice([1, 2, 63, 64, 65, 127, 128, 129, 191, 200, 257, 383, 400, 511, 640, 777],
+                                          size=n)]
+    cp_r = [int(x) for x in rng.choice([0, 1, 2, 3, 4], size=n)]
+    if not any(cp_r):
+        cp_r[0] = 2
+    run_case(lengths, int(rng.integers(1, 4)), cp_r=cp_r, seed=seed, label=f"mix {lengths} cp_r {cp_r}: ")
+
+
+@pytest.mark.parametrize("q_start,q_len,k_start,k_len", [
+    (100, 300, 37, 263),      # off = 63: the first visible q sub-tile of a kv tile is odd
+    (128, 200, 64, 130),      # off = 64
+    (129, 250, 0, 379),       # off = 129, kv chunk reaches the end of the q chunk
+    (0, 300, 0, 300),         # the diagonal pair itself
+    (300, 150, 10, 70),       # kv chunk wholly earlier: no mask inside the pair
+    (64, 129, 1, 192),        # off = 63, ragged tails on both sides
+])
+def test_backward_of_one_hand_made_pair(q_start, q_len, k_start, k_len):
+    """One pair that is not a chunk pair of a cut sequence: dq rows of its q range, dk / dv rows of its
+    kv range, given the out / lse of the whole sequence (what a ring engine passes in)."""
+    import torch
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.runner import AttnStep, bits_to_tensor
+
+    lengths, h = [40, 460, 33], 2
+    cu = hw.cu_seqlens(lengths)
+    T = int(cu[-1])
+    x = rand_inputs(np.random.default_rng(q_start + 7 * k_len), T, h)
+    scale = np.float32(1.0 / np.sqrt(np.float32(DQK)))
+    out, lse = oracle.attn_fwd(x["q"], x["k"], x["v"], cu, True, scale)
+    pair = dict(seq=1, q_start=q_start, q_len=q_len, k_start=k_start, k_len=k_len, group=0)
+    ref = oracle.attn_bwd_pairs(x["q"], x["k"], x["v"], x["do"], cu, [pair], True, scale, lse,
+                                oracle.bwd_prep(x["do"], out))
+    step = AttnStep(cu, h, [pair], 0, True, None)
+    step.out.copy_(bits_to_tensor(hw.f32_to_bf16_bits(out.astype(np.float32))))
+    step.lse.copy_(torch.from_numpy(lse.astype(np.float32)).cuda())
+    for t in (step.dq, step.dk, step.dv):
+        t.fill_(3.0)
+    q, k, v, do = (bits_to_tensor(x[n]) for n in ("q", "k", "v", "do"))
+    step.backward(q, k, v, do)
+    status, detail = step.poll()
+    assert status == 0, (status, detail)
+    got = {n: t.float().cpu().numpy().astype(np.float64) for n, t in (("dq", step.dq), ("dk", step.dk), ("dv", step.dv))}
+    base = int(cu[1])
+    rows = {"dq": (base + q_start, q_len), "dk": (base + k_start, k_len), "dv": (base + k_start, k_len)}
+    for n, r in zip(("dq", "dk", "dv"), ref):
+        lo, ln = rows[n]
+        inside = np.zeros(T, dtype=bool)
+        inside[lo:lo + ln] = True
+        assert np.all(got[n][~inside] == 3.0), f"{n}: rows outside the pair were written"
+        err = np.abs(got[n][inside] - r[inside]).max()
+        assert err <= TOL_REL * np.abs(r).max() + 1e-5, (n, err, np.abs(r).max())
