@@ -929,19 +929,21 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 // tiles (dS^T blocks as an MN-major A operand, the K tile as an MN-major B operand). The kernel is
 // bound by the stream of dS (2 bytes per 384 FLOP), so it is a plain load -> UMMA -> store pipeline:
 //   warps 0-3  epilogue (thread r = q row r): dQ * scale -> bf16 (or fp32 reductions)
-//   warp  4    TMA producer: per kv tile the two dS^T blocks of the q tile (32 KB) and the K tile (48 KB)
+//   warp  4    pops work items; TMA producer of dS^T: per kv tile the two blocks of the q tile (32 KB),
+//              ring of four (dS comes from memory)
 //   warp  5    UMMA issuer; two accumulators in tensor memory, so the epilogue of one work item
 //              overlaps the products of the next
+//   warp  6    TMA producer of the K tiles (48 KB, ring of two: they come from the L2 cache)
+// Per SM the kernel is bound by what TMA can bring in (80 KB per 768 cycles of UMMA).
 namespace dqs {
-constexpr int kThreadsS = 192;
-constexpr int kStages = 2;
+constexpr int kThreadsS = 224;
+constexpr int kDsStages = 4, kKStages = 2;
 constexpr uint32_t kDsBytes = 2 * DS_BLOCK_BYTES;            // blocks (jk, 2i) and (jk, 2i + 1)
-constexpr uint32_t kStage = kDsBytes + 3 * kBox128;          // + K tile
-constexpr uint32_t kTotal = kStages * kStage;                // 163,840 B
+constexpr uint32_t kK = kDsStages * kDsBytes;                // 128 KB of dS^T, then the K tiles
+constexpr uint32_t kTotal = kK + kKStages * 3 * kBox128;     // 229,376 B
 constexpr uint32_t kTmAcc = 256, kTmCols = 512;              // accumulators at columns 0 and 256
-enum : int { B_FULL = 0, B_EMPTY = kStages, B_ACCFULL = 2 * kStages, B_ACCFREE = 2 * kStages + 2,
-             B_ITEMFULL = 2 * kStages + 4, B_ITEMEMPTY = 2 * kStages + 4 + kSched,
-             B_COUNT = 2 * kStages + 4 + 2 * kSched };
+enum : int { B_DSFULL = 0, B_DSEMPTY = 4, B_KFULL = 8, B_KEMPTY = 10, B_ACCFULL = 12, B_ACCFREE = 14,
+             B_ITEMFULL = 16, B_ITEMEMPTY = 16 + kSched, B_COUNT = 16 + 2 * kSched };
 }  // namespace dqs
 
 size_t bwd_dq_ds_smem_bytes() { return dqs::kTotal + 1024; }
@@ -967,7 +969,7 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
         for (int i = 0; i < B_COUNT; ++i) {
             uint32_t count = 1u;
             if (i == B_ACCFREE || i == B_ACCFREE + 1) count = 4u;             // epilogue warps
-            if (i >= B_ITEMEMPTY && i < B_ITEMEMPTY + kSched) count = 5u;    // + the issuer warp
+            if (i >= B_ITEMEMPTY && i < B_ITEMEMPTY + kSched) count = 6u;    // + issuer and K producer warps
             mbar_init(bar(i), count);
         }
         fence_mbar_init();
@@ -1000,7 +1002,7 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
     };
 
     if (warp == 4) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ work queue + dS producer
         if (lane == 0) {
             uint32_t g = 0;
             bool ok = true;
@@ -1019,21 +1021,42 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
                 ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
                 const int u0 = item.r0 / SUB;                  // first sub-tile of this q tile
                 for (; ti.valid() && ok; ti.next(), ++g) {
-                    const int st = g % kStages;
-                    ok = wait(B_EMPTY + st, (g / kStages) ^ 1u);
+                    const int st = g % kDsStages;
+                    ok = wait(B_DSEMPTY + st, (g / kDsStages) ^ 1u);
                     if (!ok) break;
                     const DsGeom geo = ds_geom(ti.cur.q_len, ti.cur.off, p.causal);
                     const int64_t blk = static_cast<int64_t>(item.head) * p.ds_head_blocks + ti.cur.ds_base +
                                         ds_rowstart(geo, ti.t) + (u0 - ds_first(geo, ti.t));
-                    const uint32_t dst = smem + st * kStage;
-                    mbar_arrive_expect_tx(bar(B_FULL + st), kStage);
-                    tma_load_2d_hint(dst, &map_ds, bar(B_FULL + st), 0, static_cast<int>(blk * TILE), ds_policy);
-                    for (int c = 0; c < 3; ++c)
-                        tma_load_3d(dst + kDsBytes + c * kBox128, &map_k, bar(B_FULL + st), c * 64, item.head,
-                                    ti.cur.k_tok0 + ti.t * TILE);
+                    mbar_arrive_expect_tx(bar(B_DSFULL + st), kDsBytes);
+                    tma_load_2d_hint(smem + st * kDsBytes, &map_ds, bar(B_DSFULL + st), 0, static_cast<int>(blk * TILE),
+                                     ds_policy);
                 }
             }
             if (blockIdx.x == 0) probe.stop(p.status, QUEUE_DQ);
+        }
+    } else if (warp == 6) {
+        // ------------------------------------------------------------------ K producer
+        uint32_t g = 0;
+        bool ok = true;
+        for (uint32_t kq = 0; ok; ++kq) {
+            const int it = next_item(kq);
+            if (it < 0) break;
+            const GroupItem item = p.items[it];
+            const int32_t* list = p.lists + item.list_off;
+            const PairDev first = p.pairs[list[0]];
+            TileIter ti;
+            ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+            for (; ti.valid() && ok; ti.next(), ++g) {
+                const int st = g % kKStages;
+                ok = wait(B_KEMPTY + st, (g / kKStages) ^ 1u);
+                if (!ok) break;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(bar(B_KFULL + st), 3 * kBox128);
+                    for (int c = 0; c < 3; ++c)
+                        tma_load_3d(smem + kK + (st * 3 + c) * kBox128, &map_k, bar(B_KFULL + st), c * 64, item.head,
+                                    ti.cur.k_tok0 + ti.t * TILE);
+                }
+            }
         }
     } else if (warp == 5) {
         // ------------------------------------------------------------------ UMMA issuer
@@ -1056,18 +1079,20 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
             if (!ok) break;
             bool first_tile = true;
             for (; ti.valid() && ok; ti.next(), ++g) {
-                const int st = g % kStages;
-                ok = wait(B_FULL + st, g / kStages);
+                const int ds_st = g % kDsStages, k_st = g % kKStages;
+                ok = wait(B_KFULL + k_st, g / kKStages);
+                if (ok) ok = wait(B_DSFULL + ds_st, g / kDsStages);
                 if (!ok) break;
                 tc_fence_after_sync();
                 if (elect_one()) {
-                    const uint32_t a_lo = umma_desc_lo(smem + st * kStage, DS_BLOCK_BYTES);
-                    const uint32_t b_lo = umma_desc_lo(smem + st * kStage + kDsBytes, kBox128);
+                    const uint32_t a_lo = umma_desc_lo(smem + ds_st * kDsBytes, DS_BLOCK_BYTES);
+                    const uint32_t b_lo = umma_desc_lo(smem + kK + k_st * 3 * kBox128, kBox128);
 #pragma unroll
                     for (int kk = 0; kk < TILE / 16; ++kk)
                         umma_ss_w(tm + buf * kTmAcc, a_lo + kk * (2048 >> 4), hi_ds, b_lo + kk * (2048 >> 4), hi_k, idesc,
                                   (kk > 0 || !first_tile) ? 1u : 0u);
-                    umma_commit(bar(B_EMPTY + st));
+                    umma_commit(bar(B_DSEMPTY + ds_st));
+                    umma_commit(bar(B_KEMPTY + k_st));
                 }
                 first_tile = false;
             }
@@ -1075,7 +1100,7 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
             __syncwarp();
             ++n_acc;
         }
-    } else {
+    } else if (warp < 4) {
         // ------------------------------------------------------------------ epilogue warps
         const int r = tid;                             // q row inside the tile = TMEM lane
         const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
