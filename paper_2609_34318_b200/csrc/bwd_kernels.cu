@@ -50,6 +50,34 @@ __device__ __forceinline__ void store_row_bf16(__nv_bfloat16* dst, const uint32_
     }
 }
 
+// Warp-cooperative form of store_row_bf16 for an epilogue that nothing overlaps: lane l holds 32 values
+// of row l of the warp's 32 rows (rows `row_stride` elements apart in memory). Written straight from
+// registers, every store instruction would touch 32 cache lines (16 bytes in each) and the 20 of them an
+// epilogue needs keep the load/store unit busy for thousands of cycles; transposed through a 2 KB slice
+// of shared memory, lane l stores chunk l % 4 of rows l / 4 + 8 e: eight 64-byte segments per instruction.
+// `dst` is this lane's own row pointer, `valid` the ballot of the rows that exist.
+__device__ __forceinline__ void store_rows_bf16_coalesced(uint32_t slice, int lane, __nv_bfloat16* dst,
+                                                          int64_t row_stride, const uint32_t* v, float mul, uint32_t valid)
+{
+    __syncwarp();                                      // earlier reads of the slice are over
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const uint32_t w0 = pack_bf16x2(__uint_as_float(v[8 * e + 0]) * mul, __uint_as_float(v[8 * e + 1]) * mul);
+        const uint32_t w1 = pack_bf16x2(__uint_as_float(v[8 * e + 2]) * mul, __uint_as_float(v[8 * e + 3]) * mul);
+        const uint32_t w2 = pack_bf16x2(__uint_as_float(v[8 * e + 4]) * mul, __uint_as_float(v[8 * e + 5]) * mul);
+        const uint32_t w3 = pack_bf16x2(__uint_as_float(v[8 * e + 6]) * mul, __uint_as_float(v[8 * e + 7]) * mul);
+        st_shared_v4(slice + lane * 64 + ((e ^ ((lane >> 1) & 3)) << 4), w0, w1, w2, w3);
+    }
+    __syncwarp();
+    __nv_bfloat16* base = dst - static_cast<int64_t>(lane) * row_stride + (lane & 3) * 8;   // row 0 of the warp, this lane's chunk
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int row = 8 * e + (lane >> 2);
+        const uint4 w = ld_shared_v4(slice + row * 64 + (((lane & 3) ^ ((row >> 1) & 3)) << 4));
+        if ((valid >> row) & 1u) *reinterpret_cast<uint4*>(base + row * row_stride) = w;
+    }
+}
+
 // Accumulating form of the same epilogue: dst (fp32) += v * mul, as 16-byte reductions performed at
 // the L2 cache. Every row is owned by one thread of one CTA per launch and launches on a stream are
 // ordered, so every address receives one addition per launch and the sum does not depend on timing;
@@ -878,14 +906,17 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             ok = wait(B_PDSFREE, c_pds - 1u);
             if (!ok) break;
             tc_fence_after_sync();
+            const uint32_t rows_valid = __ballot_sync(0xffffffffu, row_valid);
+            const uint32_t out_slice = smem + kDsStage + warp * 2048;
 #pragma unroll
             for (int c0 = 0; c0 < 96; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_x32(tm + kTmDK + lane_base + g * 96 + c0, v);
                 tmem_wait_ld();
-                if (row_valid) {
-                    if (p.accumulate) add_row_f32(dkp_acc + c0, v, 32, p.scale);
-                    else store_row_bf16(dkp + c0, v, 32, p.scale);
+                if (p.accumulate) {
+                    if (row_valid) add_row_f32(dkp_acc + c0, v, 32, p.scale);
+                } else {
+                    store_rows_bf16_coalesced(out_slice, lane, dkp + c0, static_cast<int64_t>(p.h) * D_QK, v, p.scale, rows_valid);
                 }
             }
 #pragma unroll
@@ -897,9 +928,10 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     tc_fence_before_sync();
                     mbar_arrive_warp(bar(B_ACCFREE));
                 }
-                if (row_valid) {
-                    if (p.accumulate) add_row_f32(dvp_acc + c0, v, 32, 1.f);
-                    else store_row_bf16(dvp + c0, v, 32, 1.f);
+                if (p.accumulate) {
+                    if (row_valid) add_row_f32(dvp_acc + c0, v, 32, 1.f);
+                } else {
+                    store_rows_bf16_coalesced(out_slice, lane, dvp + c0, static_cast<int64_t>(p.h) * D_V, v, 1.f, rows_valid);
                 }
             }
         }
