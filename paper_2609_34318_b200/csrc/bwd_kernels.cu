@@ -119,14 +119,15 @@ struct TileIter {
     }
     __device__ void seek() {
         while (li < list_len) {
-            cur = pairs[list[li]];
+            if (li > 0) cur = pairs[list[li]];
             nt = tiles_of(cur);
             if (nt > 0) return;
             ++li;
         }
     }
-    __device__ void init(const PairDev* p, const int32_t* l, int n, int lr, int c) {
-        pairs = p; list = l; list_len = n; last_row = lr; causal = c; li = 0; t = 0; nt = 0;
+    // `first` = pairs[list[0]], which the caller already holds (from the work ring in shared memory)
+    __device__ void init(const PairDev* p, const int32_t* l, int n, int lr, int c, const PairDev& first) {
+        pairs = p; list = l; list_len = n; last_row = lr; causal = c; li = 0; t = 0; nt = 0; cur = first;
         seek();
     }
     __device__ bool valid() const { return li < list_len; }
@@ -157,7 +158,7 @@ struct SubIter {
     int li, u, nu; PairDev cur;
     __device__ void seek() {
         while (li < list_len) {
-            cur = pairs[list[li]];
+            if (li > 0) cur = pairs[list[li]];
             nu = (cur.q_len + SUB - 1) / SUB;
             u = 0;
             if (causal) { const int i_min = r0 - cur.off; u = i_min > 0 ? i_min / SUB : 0; }
@@ -168,8 +169,8 @@ struct SubIter {
             ++li;
         }
     }
-    __device__ void init(const PairDev* p, const int32_t* l, int n, int r, int c, int ev) {
-        pairs = p; list = l; list_len = n; r0 = r; causal = c; even = ev; li = 0; u = 0; nu = 0;
+    __device__ void init(const PairDev* p, const int32_t* l, int n, int r, int c, int ev, const PairDev& first) {
+        pairs = p; list = l; list_len = n; r0 = r; causal = c; even = ev; li = 0; u = 0; nu = 0; cur = first;
         seek();
     }
     __device__ bool valid() const { return li < list_len; }
@@ -197,6 +198,8 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
     __shared__ int32_t s_sched[kSched];
+    __shared__ GroupItem s_item[kSched];              // the work ring carries the item and its first pair, so that
+    __shared__ PairDev s_first[kSched];               // no role starts an item with a walk through global memory
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t bar0 = smem_u32(&bars[0]);
@@ -225,19 +228,37 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // finishes early simply takes more items: no cost model has to predict the run time of an item)
     // and hands it to the other warps of the CTA through a small ring in shared memory.
     volatile int32_t* sched = s_sched;
-    auto pop_item = [&](uint32_t k) -> int {                 // producer, one thread
+    // The pop is split in two: the request to the counter goes out when an item starts, its answer is
+    // looked at after the first loads of that item have been issued; the producer then fetches the
+    // next item's descriptors (three dependent loads from global memory) and puts them in the ring.
+    constexpr int kPopFailed = 0x7fffffff;
+    auto pop_begin = [&](uint32_t k) -> int {               // producer, one thread
         const int slot = k % kSched;
-        if (!mbar_wait(bar(B_ITEMEMPTY + slot), ((k / kSched) ^ 1u) & 1u, abort_p, limit)) return -1;
-        int idx = atomicAdd(&p.status->next_item[QUEUE_DQ], 1);
-        if (idx >= p.n_items) idx = -1;
+        if (!mbar_wait(bar(B_ITEMEMPTY + slot), ((k / kSched) ^ 1u) & 1u, abort_p, limit)) return kPopFailed;
+        return atomicAdd(&p.status->next_item[QUEUE_DQ], 1);
+    };
+    auto pop_end = [&](uint32_t k, int raw, GroupItem& item_out, PairDev& first_out) -> int {
+        if (raw == kPopFailed) return -1;
+        const int slot = k % kSched;
+        const int idx = raw >= p.n_items ? -1 : raw;
+        if (idx >= 0) {
+            item_out = p.items[idx];
+            first_out = p.pairs[p.lists[item_out.list_off]];
+            s_item[slot] = item_out;
+            s_first[slot] = first_out;
+        }
         sched[slot] = idx;
         mbar_arrive(bar(B_ITEMFULL + slot));
         return idx;
     };
-    auto next_item = [&](uint32_t k) -> int {                // every other warp, all lanes
+    auto next_item = [&](uint32_t k, GroupItem& item_out, PairDev& first_out) -> int {   // every other warp, all lanes
         const int slot = k % kSched;
         if (!mbar_wait(bar(B_ITEMFULL + slot), (k / kSched) & 1u, abort_p, limit)) return -1;
         const int idx = sched[slot];
+        if (idx >= 0) {
+            item_out = s_item[slot];
+            first_out = s_first[slot];
+        }
         mbar_arrive_warp(bar(B_ITEMEMPTY + slot));
         return idx;
     };
@@ -249,18 +270,22 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             bool ok = true;
             ClockProbe probe;
             probe.start();
-            // one item ahead: the round trip to the counter overlaps the loads of the current item
-            int it_ahead = pop_item(0);
+            // one item ahead: the round trip to the counter and the descriptor fetch overlap the loads of
+            // the current item
+            GroupItem item_next;
+            PairDev first_next;
+            int it_ahead = pop_end(0, pop_begin(0), item_next, first_next);
             for (uint32_t kq = 0; ok; ++kq) {
                 const int it = it_ahead;
                 if (it < 0) break;
-                it_ahead = pop_item(kq + 1);
-                const GroupItem item = p.items[it];
+                const GroupItem item = item_next;
+                const PairDev first = first_next;
+                const int raw_next = pop_begin(kq + 1);
+                bool popped = false;
                 const int32_t* list = p.lists + item.list_off;
-                const PairDev first = p.pairs[list[0]];
                 TileIter ti;
-                ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
-                if (!ti.valid()) continue;
+                ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal, first);
+                if (!ti.valid()) { it_ahead = pop_end(kq + 1, raw_next, item_next, first_next); continue; }
                 ok = wait(B_QEMPTY, items ^ 1u);
                 if (!ok) break;
                 ++items;
@@ -292,7 +317,9 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                         tma_load_3d(smem + kK + st * 3 * kBox128 + c * kBox128, &map_k, bar(B_KFULL + st * 3 + c),
                                     c * 64, item.head, tok);
                     }
+                    if (!popped) { it_ahead = pop_end(kq + 1, raw_next, item_next, first_next); popped = true; }
                 }
+                if (!popped) it_ahead = pop_end(kq + 1, raw_next, item_next, first_next);
             }
             if (blockIdx.x == 0) probe.stop(p.status, QUEUE_DQ);
         }
@@ -315,13 +342,13 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             uint32_t items = 0, n_tile = 0, gv = 0;       // running counts of this issuer
             bool ok = true;
             for (uint32_t kq = 0; ok; ++kq) {
-                const int it = next_item(kq);
+                GroupItem item;
+                PairDev first;
+                const int it = next_item(kq, item, first);
                 if (it < 0) break;
-                const GroupItem item = p.items[it];
                 const int32_t* list = p.lists + item.list_off;
-                const PairDev first = p.pairs[list[0]];
                 TileIter ti;
-                ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+                ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal, first);
                 if (!ti.valid()) continue;
                 if (issue_scores) {
                     ok = wait(B_QFULL, items);
@@ -419,18 +446,18 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         uint32_t c_s = 0, c_ds = 0;
         bool ok = true;
         for (uint32_t kq = 0; ok; ++kq) {
-            const int it = next_item(kq);
+            GroupItem item;
+            PairDev first;
+            const int it = next_item(kq, item, first);
             if (it < 0) break;
-            const GroupItem item = p.items[it];
             const int32_t* list = p.lists + item.list_off;
-            const PairDev first = p.pairs[list[0]];
             const int row = item.r0 + r;
             const bool row_valid = row < first.q_len;
             const int64_t dst_off = (static_cast<int64_t>(first.q_tok0 + row) * p.h + item.head) * D_QK + g * 96;
             __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.dq) + dst_off;
             float* dst_acc = static_cast<float*>(p.dq) + dst_off;        // accumulate mode: dq is fp32
             TileIter ti;
-            ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+            ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal, first);
             if (!ti.valid()) {                         // no visible key at all: dQ = 0 (nothing to add)
                 if (row_valid && !p.accumulate) {
                     uint4* d4 = reinterpret_cast<uint4*>(dst);
@@ -563,6 +590,8 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
     __shared__ int32_t s_sched[kSched];
+    __shared__ GroupItem s_item[kSched];              // the work ring carries the item and its first pair, so that
+    __shared__ PairDev s_first[kSched];               // no role starts an item with a walk through global memory
     __shared__ float s_lse2[kStages][SUB];
     __shared__ float s_dsum[kStages][SUB];
     __shared__ uint32_t s_bursts;                      // S / dP bursts issued so far (all ones: no more)
@@ -596,19 +625,37 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // finishes early simply takes more items: no cost model has to predict the run time of an item)
     // and hands it to the other warps of the CTA through a small ring in shared memory.
     volatile int32_t* sched = s_sched;
-    auto pop_item = [&](uint32_t k) -> int {                 // producer, one thread
+    // The pop is split in two: the request to the counter goes out when an item starts, its answer is
+    // looked at after the first loads of that item have been issued; the producer then fetches the
+    // next item's descriptors (three dependent loads from global memory) and puts them in the ring.
+    constexpr int kPopFailed = 0x7fffffff;
+    auto pop_begin = [&](uint32_t k) -> int {               // producer, one thread
         const int slot = k % kSched;
-        if (!mbar_wait(bar(B_ITEMEMPTY + slot), ((k / kSched) ^ 1u) & 1u, abort_p, limit)) return -1;
-        int idx = atomicAdd(&p.status->next_item[QUEUE_DKV], 1);
-        if (idx >= p.n_items) idx = -1;
+        if (!mbar_wait(bar(B_ITEMEMPTY + slot), ((k / kSched) ^ 1u) & 1u, abort_p, limit)) return kPopFailed;
+        return atomicAdd(&p.status->next_item[QUEUE_DKV], 1);
+    };
+    auto pop_end = [&](uint32_t k, int raw, GroupItem& item_out, PairDev& first_out) -> int {
+        if (raw == kPopFailed) return -1;
+        const int slot = k % kSched;
+        const int idx = raw >= p.n_items ? -1 : raw;
+        if (idx >= 0) {
+            item_out = p.items[idx];
+            first_out = p.pairs[p.lists[item_out.list_off]];
+            s_item[slot] = item_out;
+            s_first[slot] = first_out;
+        }
         sched[slot] = idx;
         mbar_arrive(bar(B_ITEMFULL + slot));
         return idx;
     };
-    auto next_item = [&](uint32_t k) -> int {                // every other warp, all lanes
+    auto next_item = [&](uint32_t k, GroupItem& item_out, PairDev& first_out) -> int {   // every other warp, all lanes
         const int slot = k % kSched;
         if (!mbar_wait(bar(B_ITEMFULL + slot), (k / kSched) & 1u, abort_p, limit)) return -1;
         const int idx = sched[slot];
+        if (idx >= 0) {
+            item_out = s_item[slot];
+            first_out = s_first[slot];
+        }
         mbar_arrive_warp(bar(B_ITEMEMPTY + slot));
         return idx;
     };
@@ -621,21 +668,29 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         int it_ahead = -1;
         ClockProbe probe;
         probe.start();
+        GroupItem item_next;                          // lane 0: descriptors of the item popped ahead
+        PairDev first_next;
         for (uint32_t kq = 0; ok; ++kq) {
-            int it = 0;
+            int it = 0, raw_next = 0;
             if (lane == 0) {                          // one pop per CTA, one item ahead, shared with the other lanes
-                if (kq == 0) it_ahead = pop_item(0);
+                if (kq == 0) it_ahead = pop_end(0, pop_begin(0), item_next, first_next);
                 it = it_ahead;
-                if (it >= 0) it_ahead = pop_item(kq + 1);
+                if (it >= 0) raw_next = pop_begin(kq + 1);
             }
+            bool popped = false;
             it = __shfl_sync(0xffffffffu, it, 0);
             if (it < 0) break;
-            const GroupItem item = p.items[it];
+            __syncwarp();
+            // lane 0 wrote this item's descriptors into the ring when it popped it (before the barrier above)
+            const GroupItem item = s_item[kq % kSched];
+            const PairDev first = s_first[kq % kSched];
             const int32_t* list = p.lists + item.list_off;
-            const PairDev first = p.pairs[list[0]];
             SubIter si;
-            si.init(p.pairs, list, item.list_len, item.r0, p.causal, p.ds != nullptr);
-            if (!si.valid()) continue;
+            si.init(p.pairs, list, item.list_len, item.r0, p.causal, p.ds != nullptr, first);
+            if (!si.valid()) {
+                if (lane == 0) it_ahead = pop_end(kq + 1, raw_next, item_next, first_next);
+                continue;
+            }
             ok = wait(B_KVEMPTY, items ^ 1u);
             if (!ok) break;
             ++items;
@@ -674,7 +729,12 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     s_dsum[st][c] = v ? __ldg(p.dsum + idx) : 0.f;
                 }
                 mbar_arrive_warp(bar(B_STAT + st));
+                if (!popped) {
+                    if (lane == 0) it_ahead = pop_end(kq + 1, raw_next, item_next, first_next);
+                    popped = true;
+                }
             }
+            if (!popped && lane == 0) it_ahead = pop_end(kq + 1, raw_next, item_next, first_next);
         }
         if (blockIdx.x == 0 && lane == 0) probe.stop(p.status, QUEUE_DKV);
     } else if (warp == kWarpMma || warp == kWarpMma2) {
@@ -696,12 +756,13 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             uint32_t items = 0, n_step = 0;
             bool ok = true;
             for (uint32_t kq = 0; ok; ++kq) {
-                const int it = next_item(kq);
+                GroupItem item;
+                PairDev first;
+                const int it = next_item(kq, item, first);
                 if (it < 0) break;
-                const GroupItem item = p.items[it];
                 const int32_t* list = p.lists + item.list_off;
                 SubIter si;
-                si.init(p.pairs, list, item.list_len, item.r0, p.causal, p.ds != nullptr);
+                si.init(p.pairs, list, item.list_len, item.r0, p.causal, p.ds != nullptr, first);
                 if (!si.valid()) continue;
                 if (issue_scores) {
                     ok = wait(B_KVFULL, items);
@@ -784,11 +845,11 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         int64_t ds_blk0 = 0;
         bool ok = true;
         for (uint32_t kq = 0; ok; ++kq) {
-            const int it = next_item(kq);
+            GroupItem item;
+            PairDev first;
+            const int it = next_item(kq, item, first);
             if (it < 0) break;
-            const GroupItem item = p.items[it];
             const int32_t* list = p.lists + item.list_off;
-            const PairDev first = p.pairs[list[0]];
             ds_li = -1;
             const int krow = item.r0 + r;              // kv row inside the chunk
             const bool row_valid = krow < first.k_len;
@@ -800,7 +861,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             float* dkp_acc = static_cast<float*>(p.dk) + dk_off;         // accumulate mode: dk, dv are fp32
             float* dvp_acc = static_cast<float*>(p.dv) + dv_off;
             SubIter si;
-            si.init(p.pairs, list, item.list_len, item.r0, p.causal, p.ds != nullptr);
+            si.init(p.pairs, list, item.list_len, item.r0, p.causal, p.ds != nullptr, first);
             if (!si.valid()) {                         // no q row sees this tile: dK = dV = 0 (nothing to add)
                 if (row_valid && !p.accumulate) {
                     uint4* a4 = reinterpret_cast<uint4*>(dkp);
@@ -992,6 +1053,8 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
     __shared__ int32_t s_sched[kSched];
+    __shared__ GroupItem s_item[kSched];              // the work ring carries the item and its first pair, so that
+    __shared__ PairDev s_first[kSched];               // no role starts an item with a walk through global memory
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t bar0 = smem_u32(&bars[0]);
@@ -1016,19 +1079,37 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
     volatile int* abort_p = &abort_flag;
     auto wait = [&](int b, uint32_t parity) -> bool { return mbar_wait(bar(b), parity & 1u, abort_p, limit); };
     volatile int32_t* sched = s_sched;
-    auto pop_item = [&](uint32_t k) -> int {                 // producer, one thread
+    // The pop is split in two: the request to the counter goes out when an item starts, its answer is
+    // looked at after the first loads of that item have been issued; the producer then fetches the
+    // next item's descriptors (three dependent loads from global memory) and puts them in the ring.
+    constexpr int kPopFailed = 0x7fffffff;
+    auto pop_begin = [&](uint32_t k) -> int {               // producer, one thread
         const int slot = k % kSched;
-        if (!mbar_wait(bar(B_ITEMEMPTY + slot), ((k / kSched) ^ 1u) & 1u, abort_p, limit)) return -1;
-        int idx = atomicAdd(&p.status->next_item[QUEUE_DQ], 1);
-        if (idx >= p.n_items) idx = -1;
+        if (!mbar_wait(bar(B_ITEMEMPTY + slot), ((k / kSched) ^ 1u) & 1u, abort_p, limit)) return kPopFailed;
+        return atomicAdd(&p.status->next_item[QUEUE_DQ], 1);
+    };
+    auto pop_end = [&](uint32_t k, int raw, GroupItem& item_out, PairDev& first_out) -> int {
+        if (raw == kPopFailed) return -1;
+        const int slot = k % kSched;
+        const int idx = raw >= p.n_items ? -1 : raw;
+        if (idx >= 0) {
+            item_out = p.items[idx];
+            first_out = p.pairs[p.lists[item_out.list_off]];
+            s_item[slot] = item_out;
+            s_first[slot] = first_out;
+        }
         sched[slot] = idx;
         mbar_arrive(bar(B_ITEMFULL + slot));
         return idx;
     };
-    auto next_item = [&](uint32_t k) -> int {                // every other warp, all lanes
+    auto next_item = [&](uint32_t k, GroupItem& item_out, PairDev& first_out) -> int {   // every other warp, all lanes
         const int slot = k % kSched;
         if (!mbar_wait(bar(B_ITEMFULL + slot), (k / kSched) & 1u, abort_p, limit)) return -1;
         const int idx = sched[slot];
+        if (idx >= 0) {
+            item_out = s_item[slot];
+            first_out = s_first[slot];
+        }
         mbar_arrive_warp(bar(B_ITEMEMPTY + slot));
         return idx;
     };
@@ -1041,16 +1122,19 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
             const uint64_t ds_policy = l2_policy_evict_first();   // dS is read once: leave L2 to the K tiles
             ClockProbe probe;
             probe.start();
-            int it_ahead = pop_item(0);
+            GroupItem item_next;
+            PairDev first_next;
+            int it_ahead = pop_end(0, pop_begin(0), item_next, first_next);
             for (uint32_t kq = 0; ok; ++kq) {
                 const int it = it_ahead;
                 if (it < 0) break;
-                it_ahead = pop_item(kq + 1);
-                const GroupItem item = p.items[it];
+                const GroupItem item = item_next;
+                const PairDev first = first_next;
+                const int raw_next = pop_begin(kq + 1);
+                bool popped = false;
                 const int32_t* list = p.lists + item.list_off;
-                const PairDev first = p.pairs[list[0]];
                 TileIter ti;
-                ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+                ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal, first);
                 const int u0 = item.r0 / SUB;                  // first sub-tile of this q tile
                 for (; ti.valid() && ok; ti.next(), ++g) {
                     const int st = g % kDsStages;
@@ -1062,7 +1146,9 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
                     mbar_arrive_expect_tx(bar(B_DSFULL + st), kDsBytes);
                     tma_load_2d_hint(smem + st * kDsBytes, &map_ds, bar(B_DSFULL + st), 0, static_cast<int>(blk * TILE),
                                      ds_policy);
+                    if (!popped) { it_ahead = pop_end(kq + 1, raw_next, item_next, first_next); popped = true; }
                 }
+                if (!popped) it_ahead = pop_end(kq + 1, raw_next, item_next, first_next);
             }
             if (blockIdx.x == 0) probe.stop(p.status, QUEUE_DQ);
         }
@@ -1071,13 +1157,13 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
         uint32_t g = 0;
         bool ok = true;
         for (uint32_t kq = 0; ok; ++kq) {
-            const int it = next_item(kq);
+            GroupItem item;
+            PairDev first;
+            const int it = next_item(kq, item, first);
             if (it < 0) break;
-            const GroupItem item = p.items[it];
             const int32_t* list = p.lists + item.list_off;
-            const PairDev first = p.pairs[list[0]];
             TileIter ti;
-            ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+            ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal, first);
             for (; ti.valid() && ok; ti.next(), ++g) {
                 const int st = g % kKStages;
                 ok = wait(B_KEMPTY + st, (g / kKStages) ^ 1u);
@@ -1098,13 +1184,13 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
         uint32_t g = 0, n_acc = 0;
         bool ok = true;
         for (uint32_t kq = 0; ok; ++kq) {
-            const int it = next_item(kq);
+            GroupItem item;
+            PairDev first;
+            const int it = next_item(kq, item, first);
             if (it < 0) break;
-            const GroupItem item = p.items[it];
             const int32_t* list = p.lists + item.list_off;
-            const PairDev first = p.pairs[list[0]];
             TileIter ti;
-            ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+            ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal, first);
             if (!ti.valid()) continue;
             const uint32_t buf = n_acc & 1u;
             ok = wait(B_ACCFREE + buf, (n_acc >> 1) ^ 1u);
@@ -1139,18 +1225,18 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
         uint32_t n_acc = 0;
         bool ok = true;
         for (uint32_t kq = 0; ok; ++kq) {
-            const int it = next_item(kq);
+            GroupItem item;
+            PairDev first;
+            const int it = next_item(kq, item, first);
             if (it < 0) break;
-            const GroupItem item = p.items[it];
             const int32_t* list = p.lists + item.list_off;
-            const PairDev first = p.pairs[list[0]];
             const int row = item.r0 + r;
             const bool row_valid = row < first.q_len;
             const int64_t dst_off = (static_cast<int64_t>(first.q_tok0 + row) * p.h + item.head) * D_QK;
             __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.dq) + dst_off;
             float* dst_acc = static_cast<float*>(p.dq) + dst_off;
             TileIter ti;
-            ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal);
+            ti.init(p.pairs, list, item.list_len, min(item.r0 + TILE, first.q_len) - 1, p.causal, first);
             if (!ti.valid()) {                         // no visible key at all: dQ = 0 (nothing to add)
                 if (row_valid && !p.accumulate) {
                     uint4* d4 = reinterpret_cast<uint4*>(dst);
