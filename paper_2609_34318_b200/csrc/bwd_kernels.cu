@@ -969,30 +969,34 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             tc_fence_after_sync();
             const uint32_t rows_valid = __ballot_sync(0xffffffffu, row_valid);
             const uint32_t out_slice = smem + kDsStage + warp * 2048;
+            // five chunks of 32 columns (dK: 3, dV: 2); the load of the next chunk is in flight while the
+            // current one is packed, transposed and stored
+            auto chunk_addr = [&](int c) -> uint32_t {
+                return c < 3 ? tm + kTmDK + lane_base + g * 96 + c * 32 : tm + kTmDV + lane_base + g * 64 + (c - 3) * 32;
+            };
+            uint32_t va[32], vb[32];
+            tmem_ld_x32(chunk_addr(0), va);
 #pragma unroll
-            for (int c0 = 0; c0 < 96; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld_x32(tm + kTmDK + lane_base + g * 96 + c0, v);
+            for (int c = 0; c < 5; ++c) {
+                uint32_t* cur = (c & 1) ? vb : va;
+                uint32_t* nxt = (c & 1) ? va : vb;
                 tmem_wait_ld();
-                if (p.accumulate) {
-                    if (row_valid) add_row_f32(dkp_acc + c0, v, 32, p.scale);
-                } else {
-                    store_rows_bf16_coalesced(out_slice, lane, dkp + c0, static_cast<int64_t>(p.h) * D_QK, v, p.scale, rows_valid);
-                }
-            }
-#pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld_x32(tm + kTmDV + lane_base + g * 64 + c0, v);
-                tmem_wait_ld();
-                if (c0 == 32) {
+                if (c + 1 < 5) tmem_ld_x32(chunk_addr(c + 1), nxt);
+                if (c == 4) {                          // every column has left tensor memory
                     tc_fence_before_sync();
                     mbar_arrive_warp(bar(B_ACCFREE));
                 }
+                const bool is_dk = c < 3;
+                const int c0 = is_dk ? c * 32 : (c - 3) * 32;
                 if (p.accumulate) {
-                    if (row_valid) add_row_f32(dvp_acc + c0, v, 32, 1.f);
+                    if (row_valid) {
+                        if (is_dk) add_row_f32(dkp_acc + c0, cur, 32, p.scale);
+                        else add_row_f32(dvp_acc + c0, cur, 32, 1.f);
+                    }
+                } else if (is_dk) {
+                    store_rows_bf16_coalesced(out_slice, lane, dkp + c0, static_cast<int64_t>(p.h) * D_QK, cur, p.scale, rows_valid);
                 } else {
-                    store_rows_bf16_coalesced(out_slice, lane, dvp + c0, static_cast<int64_t>(p.h) * D_V, v, 1.f, rows_valid);
+                    store_rows_bf16_coalesced(out_slice, lane, dvp + c0, static_cast<int64_t>(p.h) * D_V, cur, 1.f, rows_valid);
                 }
             }
         }
