@@ -52,7 +52,8 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p)
 
 // One block = MERGE_ROWS consecutive rows of one chunk, all heads.  For (row, head):
 //   M = max_p LSE_p;  Z = sum_p exp(LSE_p - M);  LSE = M + ln Z;  O = sum_p (exp(LSE_p - M) / Z) O_p
-__global__ void __launch_bounds__(kThreads)
+template <bool kAccumulate>
+__global__ void __launch_bounds__(kThreads, 6)
 hydra_lse_merge_kernel(const MergeParams p)
 {
     const MergeItem item = p.items[blockIdx.x];
@@ -82,7 +83,7 @@ hydra_lse_merge_kernel(const MergeParams p)
         const int64_t tok = static_cast<int64_t>(g.out_tok0) + r;
         uint4 v_cur = make_uint4(0u, 0u, 0u, 0u);
         float l_cur = neg_inf();
-        if (p.accumulate) {
+        if (kAccumulate) {
             v_cur = out[(tok * p.h + a) * kVecPerRow + lane];
             l_cur = p.lse[static_cast<int64_t>(a) * p.T + tok];
         }
@@ -107,7 +108,7 @@ hydra_lse_merge_kernel(const MergeParams p)
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = fmaf(w, f[e], acc[e]);
         };
-        add(v_cur, l_cur);
+        if (kAccumulate) add(v_cur, l_cur);
         add(v0, l0);
         add(v1, l1);
         for (int q = 2; q < g.n_parts; ++q) {
@@ -189,7 +190,8 @@ cudaError_t launch_grad_cast(const float* acc, void* grad, int64_t n, cudaStream
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream)
 {
     if (p.n_items == 0) return cudaSuccess;
-    hydra_lse_merge_kernel<<<p.n_items, kThreads, 0, stream>>>(p);
+    if (p.accumulate) hydra_lse_merge_kernel<true><<<p.n_items, kThreads, 0, stream>>>(p);
+    else hydra_lse_merge_kernel<false><<<p.n_items, kThreads, 0, stream>>>(p);
     return cudaGetLastError();
 }
 
@@ -334,6 +336,6 @@ extern "C" int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_
     mp.n_items = n_items;
     mp.o_part = o_part; mp.lse_part = lse_part; mp.out = out; mp.lse = lse;
     mp.T = cu[n_seqs]; mp.part_rows = part_rows; mp.h = n_heads;
-    hydra_lse_merge_kernel<<<n_items, kThreads, 0, stream>>>(mp);
+    hydra_lse_merge_kernel<false><<<n_items, kThreads, 0, stream>>>(mp);
     return cudaGetLastError() == cudaSuccess ? HYDRA_OK : HYDRA_ERR_CUDA;
 }
