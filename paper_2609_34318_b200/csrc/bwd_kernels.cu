@@ -78,6 +78,29 @@ __device__ __forceinline__ void store_rows_bf16_coalesced(uint32_t slice, int la
     }
 }
 
+// The accumulating counterpart: 16 fp32 columns (64 bytes per row) per call through the same slice, then
+// 16-byte reductions of whole 64-byte row segments.
+__device__ __forceinline__ void add_rows_f32_coalesced(uint32_t slice, int lane, float* dst, int64_t row_stride,
+                                                       const uint32_t* v, float mul, uint32_t valid)
+{
+    __syncwarp();
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+        st_shared_v4(slice + lane * 64 + ((e ^ ((lane >> 1) & 3)) << 4), __float_as_uint(__uint_as_float(v[4 * e + 0]) * mul),
+                     __float_as_uint(__uint_as_float(v[4 * e + 1]) * mul), __float_as_uint(__uint_as_float(v[4 * e + 2]) * mul),
+                     __float_as_uint(__uint_as_float(v[4 * e + 3]) * mul));
+    __syncwarp();
+    float* base = dst - static_cast<int64_t>(lane) * row_stride + (lane & 3) * 4;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const int row = 8 * e + (lane >> 2);
+        const uint4 w = ld_shared_v4(slice + row * 64 + (((lane & 3) ^ ((row >> 1) & 3)) << 4));
+        if ((valid >> row) & 1u)
+            red_add_v4_f32(base + row * row_stride, __uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z),
+                           __uint_as_float(w.w));
+    }
+}
+
 // Accumulating form of the same epilogue: dst (fp32) += v * mul, as 16-byte reductions performed at
 // the L2 cache. Every row is owned by one thread of one CTA per launch and launches on a stream are
 // ordered, so every address receives one addition per launch and the sum does not depend on timing;
@@ -989,9 +1012,14 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 const bool is_dk = c < 3;
                 const int c0 = is_dk ? c * 32 : (c - 3) * 32;
                 if (p.accumulate) {
-                    if (row_valid) {
-                        if (is_dk) add_row_f32(dkp_acc + c0, cur, 32, p.scale);
-                        else add_row_f32(dvp_acc + c0, cur, 32, 1.f);
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        if (is_dk)
+                            add_rows_f32_coalesced(out_slice, lane, dkp_acc + c0 + half * 16, static_cast<int64_t>(p.h) * D_QK,
+                                                   cur + half * 16, p.scale, rows_valid);
+                        else
+                            add_rows_f32_coalesced(out_slice, lane, dvp_acc + c0 + half * 16, static_cast<int64_t>(p.h) * D_V,
+                                                   cur + half * 16, 1.f, rows_valid);
                     }
                 } else if (is_dk) {
                     store_rows_bf16_coalesced(out_slice, lane, dkp + c0, static_cast<int64_t>(p.h) * D_QK, cur, p.scale, rows_valid);
