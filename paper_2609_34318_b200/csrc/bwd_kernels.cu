@@ -1053,19 +1053,21 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 // and dP: per (q tile, kv tile) one product of 128 x 192 x 128, both operands straight from their TMA
 // tiles (dS^T blocks as an MN-major A operand, the K tile as an MN-major B operand). The kernel is
 // bound by the stream of dS (2 bytes per 384 FLOP), so it is a plain load -> UMMA -> store pipeline:
-//   warps 0-3  epilogue (thread r = q row r): dQ * scale -> bf16 (or fp32 reductions)
+//   warps 0-3  epilogue (thread r = q row r): dQ * scale -> bf16 (or fp32 reductions), rows transposed
+//              through 2 KB of shared memory per warp so that whole 64-byte segments are stored
 //   warp  4    pops work items; TMA producer of dS^T: per kv tile the two blocks of the q tile (32 KB),
-//              ring of four (dS comes from memory)
+//              ring of three (dS comes from memory)
 //   warp  5    UMMA issuer; two accumulators in tensor memory, so the epilogue of one work item
 //              overlaps the products of the next
 //   warp  6    TMA producer of the K tiles (48 KB, ring of two: they come from the L2 cache)
 // Per SM the kernel is bound by what TMA can bring in (80 KB per 768 cycles of UMMA).
 namespace dqs {
 constexpr int kThreadsS = 224;
-constexpr int kDsStages = 4, kKStages = 2;
+constexpr int kDsStages = 3, kKStages = 2;
 constexpr uint32_t kDsBytes = 2 * DS_BLOCK_BYTES;            // blocks (jk, 2i) and (jk, 2i + 1)
-constexpr uint32_t kK = kDsStages * kDsBytes;                // 128 KB of dS^T, then the K tiles
-constexpr uint32_t kTotal = kK + kKStages * 3 * kBox128;     // 229,376 B
+constexpr uint32_t kK = kDsStages * kDsBytes;                // 96 KB of dS^T, then the K tiles
+constexpr uint32_t kOut = kK + kKStages * 3 * kBox128;       // 4 epilogue warps x 2 KB: dQ rows on their way out
+constexpr uint32_t kTotal = kOut + 4 * 2048;                 // 204,800 B
 constexpr uint32_t kTmAcc = 256, kTmCols = 512;              // accumulators at columns 0 and 256
 enum : int { B_DSFULL = 0, B_DSEMPTY = 4, B_KFULL = 8, B_KEMPTY = 10, B_ACCFULL = 12, B_ACCFREE = 14,
              B_ITEMFULL = 16, B_ITEMEMPTY = 16 + kSched, B_COUNT = 16 + 2 * kSched };
@@ -1281,6 +1283,8 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
             ok = wait(B_ACCFULL + buf, n_acc >> 1);
             if (!ok) break;
             tc_fence_after_sync();
+            const uint32_t rows_valid = __ballot_sync(0xffffffffu, row_valid);
+            const uint32_t out_slice = smem + kOut + warp * 2048;
 #pragma unroll
             for (int c0 = 0; c0 < D_QK; c0 += 32) {
                 uint32_t v[32];
@@ -1290,9 +1294,13 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
                     tc_fence_before_sync();
                     mbar_arrive_warp(bar(B_ACCFREE + buf));
                 }
-                if (row_valid) {
-                    if (p.accumulate) add_row_f32(dst_acc + c0, v, 32, p.scale);
-                    else store_row_bf16(dst + c0, v, 32, p.scale);
+                if (p.accumulate) {
+#pragma unroll
+                    for (int half = 0; half < 2; ++half)
+                        add_rows_f32_coalesced(out_slice, lane, dst_acc + c0 + half * 16, static_cast<int64_t>(p.h) * D_QK,
+                                               v + half * 16, p.scale, rows_valid);
+                } else {
+                    store_rows_bf16_coalesced(out_slice, lane, dst + c0, static_cast<int64_t>(p.h) * D_QK, v, p.scale, rows_valid);
                 }
             }
             ++n_acc;
