@@ -256,3 +256,32 @@ def test_backward_of_one_hand_made_pair(q_start, q_len, k_start, k_len):
         assert np.all(got[n][~inside] == 3.0), f"{n}: rows outside the pair were written"
         err = np.abs(got[n][inside] - r[inside]).max()
         assert err <= TOL_REL * np.abs(r).max() + 1e-5, (n, err, np.abs(r).max())
+
+
+def test_non_causal_backward_with_room_for_the_dense_hand_off(backward_form):
+    """hydra_workspace_bytes sizes the dS buffer for a causal call; a non-causal call needs the whole
+    rectangle of every pair and uses the hand-off only when the caller gives it that much room."""
+    import torch
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.runner import AttnStep, bits_to_tensor
+
+    lengths, h = [300, 129, 64], 2
+    cu = hw.cu_seqlens(lengths)
+    x = rand_inputs(np.random.default_rng(42), int(cu[-1]), h)
+    step = AttnStep(cu, h, None, 0, False, None)
+    if backward_form == "hand_off":
+        # rectangle of every sequence in 16 KB blocks of 128 kv rows x 64 q rows, with slack
+        blocks = sum(((L + 127) // 128) * (2 * ((L + 127) // 128)) for L in lengths) + 2
+        step.workspace = torch.empty(step.workspace.numel() + blocks * 16384 * h, dtype=torch.uint8, device="cuda")
+    q, k, v, do = (bits_to_tensor(x[n]) for n in ("q", "k", "v", "do"))
+    for t in (step.dq, step.dk, step.dv):
+        t.fill_(float("nan"))
+    step.forward(q, k, v)
+    step.backward(q, k, v, do)
+    status, detail = step.poll()
+    assert status == 0, (status, detail)
+    T = int(cu[-1])
+    got = {"out": step.out[:T].float().cpu().numpy().astype(np.float64), "lse": step.lse[:, :T].cpu().numpy().astype(np.float64),
+           "dq": step.dq[:T].float().cpu().numpy().astype(np.float64), "dk": step.dk[:T].float().cpu().numpy().astype(np.float64),
+           "dv": step.dv[:T].float().cpu().numpy().astype(np.float64)}
+    check(got, run_oracle(x, cu, False), label="non-causal, roomy workspace: ")
