@@ -226,6 +226,8 @@ def run_ours(args, w):
     if w.cp_r:
         pairs, part_rows, _, _ = P.hydra_zigzag_pairs(cu, w.cp_r)
     t = device_inputs(w, torch, rank)
+    # problems whose dS hand-off buffer is over the 4 GiB limit run their backward in bands of query rows
+    P.hydra_set_bwd_band_scratch(int(args.band_scratch_gb * 2 ** 30))
     step = AttnStep(cu, w.n_heads, pairs, part_rows, True, float(w.scale))
     stream = torch.cuda.current_stream()
 
@@ -322,7 +324,10 @@ def run_ours(args, w):
     # ---- roofline of the dominant kernel ----
     peaks, peak_kind = measured_peaks()
     dominant = max(kernel_ms, key=lambda k: kernel_ms[k])
-    per_launch_ms = kernel_ms[dominant] / max(kernel_n[dominant], 1)
+    # all launches of the kernel in one step together process the workload (a banded backward launches
+    # it once per band), so the rate is the step's work over the step's time in that kernel
+    launches_per_step = max(kernel_n[dominant], 1) / args.steps
+    per_launch_ms = kernel_ms[dominant] / args.steps
     if dominant in FLOPS_PER_PAIR:
         work = FLOPS_PER_PAIR[dominant] * w.causal_pairs_total * w.n_heads
         # the tensor cores have been busy without a pause since the first warm-up step: against the
@@ -341,7 +346,8 @@ def run_ours(args, w):
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "peak_kind": f"{peak_kind} copy"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = recorded_traffic(dominant, w.name)
-    roof["ms_per_launch"] = per_launch_ms
+    roof["ms_per_launch"] = per_launch_ms / launches_per_step
+    roof["launches_per_step"] = launches_per_step
 
     # ---- CPU baseline: the oracle on a bounded sample, rank 0, N = 1 only ----
     cpu = None
@@ -359,7 +365,9 @@ def run_ours(args, w):
             "config": {"workload": w.name, "tokens": w.total, "heads": w.n_heads, "sequences": len(w.lengths),
                        "d_qk": hw.D_QK, "d_v": hw.D_V, "pairs": 0 if pairs is None else int(len(pairs)),
                        "causal_pairs": w.causal_pairs_total, "note": w.note,
-                       "l2": "inputs larger than L2 (no flush between iterations)"},
+                       "l2": "inputs larger than L2 (no flush between iterations)",
+                       "bwd_bands": int(round(kernel_n.get("bwd_dkv", 0) / args.steps)),
+                       "band_scratch_gb": args.band_scratch_gb},
             "frac_of_bf16_peak": value / world / peaks["bf16_tflops"],
             "kernel_ms_per_step": {k: v / args.steps for k, v in kernel_ms.items()},
             "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
@@ -569,6 +577,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="packed32k", choices=list(hw.WORKLOADS))
+    ap.add_argument("--band-scratch-gb", type=float, default=48.0,
+                    help="dS scratch of the banded backward (long sequences only); 0 switches the bands off")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--report", action="store_true", help="per-kernel report of the workload instead of the bench line")

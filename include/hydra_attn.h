@@ -115,8 +115,33 @@ int32_t hydra_zigzag_pairs(const int32_t* cu_seqlens_host, int32_t n_seqs, const
  * the buffer is within the limit. The results of the two forms agree to the rounding of dS to bf16,
  * which both apply. The size assumes a causal call; a non-causal call needs about twice the buffer
  * and falls back to recomputation in a workspace sized here.
+ *
+ * Banded form, for problems whose dS buffer is over that limit (long sequences). After
+ * hydra_set_bwd_band_scratch(bytes) with bytes >= 1 MiB (default 0: off), HYDRA_WS_BWD asks, for such a
+ * problem, for the base size + an fp32 accumulator of dq (4 * 192 bytes per token and head) +
+ * min(bytes, the full dS buffer). hydra_attn_bwd, given that much, cuts the key rows of every chunk into
+ * bands of 128-row tiles whose own dS buffer fits the scratch and runs every band with the hand-off
+ * (pairs clipped to the band's keys and, under the causal mask, to the query rows that see them). A key
+ * tile lies in one band, so dk and dv come out as in the one-shot form; dq sums the bands' contributions
+ * in fp32, in an unspecified order, and is rounded to bf16 once at the end. A problem that cannot be
+ * banded (a single tile column over the scratch, or clipped chunks that would overlap without being
+ * identical) runs in the recomputing form instead.
  */
 void hydra_set_bwd_scratch_limit(uint64_t bytes);
+void hydra_set_bwd_band_scratch(uint64_t bytes);
+
+/*
+ * Host only: the bands the banded backward would run for this problem with `scratch_bytes` of dS scratch.
+ * Writes the clipped pairs of all bands, band after band, to pairs_out (capacity max_pairs; may be NULL
+ * with max_pairs = 0 to count) and the band of each to band_out. Every visible (query, key) position of
+ * the input pairs lies in exactly one clipped pair. n_bands_out = 0 means the problem cannot be banded
+ * with that scratch. Returns HYDRA_ERR_WORKSPACE_TOO_SMALL if max_pairs is too small (counts are still
+ * written), HYDRA_ERR_INVALID_ARG on bad input.
+ */
+int32_t hydra_bwd_bands(const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
+                        const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, uint64_t scratch_bytes,
+                        hydra_pair_t* pairs_out, int32_t* band_out, int32_t max_pairs, int32_t* n_pairs_out,
+                        int32_t* n_bands_out);
 size_t hydra_workspace_bytes(int32_t which, const int32_t* cu_seqlens_host, int32_t n_seqs,
                              int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs);
 

@@ -59,6 +59,8 @@ def _load() -> ctypes.CDLL:
     lib.hydra_usp_factor.argtypes = [i32, i32, vp, vp]
     lib.hydra_zigzag_pairs.restype = i32
     lib.hydra_zigzag_pairs.argtypes = [vp, i32, vp, i32, vp, i32, vp, vp, vp, vp]
+    lib.hydra_bwd_bands.restype = i32
+    lib.hydra_bwd_bands.argtypes = [vp, i32, i32, vp, i32, i32, ctypes.c_uint64, vp, vp, i32, vp, vp]
     lib.hydra_workspace_bytes.restype = sz
     lib.hydra_workspace_bytes.argtypes = [i32, vp, i32, i32, vp, i32]
     lib.hydra_attn_fwd.restype = i32
@@ -80,6 +82,8 @@ def _load() -> ctypes.CDLL:
                                    vp, sz, vp]
     lib.hydra_set_bwd_scratch_limit.restype = None
     lib.hydra_set_bwd_scratch_limit.argtypes = [ctypes.c_uint64]
+    lib.hydra_set_bwd_band_scratch.restype = None
+    lib.hydra_set_bwd_band_scratch.argtypes = [ctypes.c_uint64]
     lib.hydra_attn_bwd_accumulate.restype = i32
     lib.hydra_attn_bwd_accumulate.argtypes = lib.hydra_attn_bwd.argtypes
     lib.hydra_grad_cast.restype = i32
@@ -110,7 +114,8 @@ EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
            "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc", "hydra_lse_merge_accumulate",
            "hydra_sched_targets", "hydra_sched_cp", "hydra_sched_pack", "hydra_attn_bwd_accumulate",
-           "hydra_grad_cast", "hydra_set_bwd_scratch_limit", "hydra_poll_clocks")
+           "hydra_grad_cast", "hydra_set_bwd_scratch_limit", "hydra_set_bwd_band_scratch", "hydra_bwd_bands",
+           "hydra_poll_clocks")
 KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast")
 
 
@@ -223,6 +228,23 @@ def hydra_zigzag_pairs(cu_seqlens, cp_r):
     return pairs, int(part_rows.value), rank, step
 
 
+def hydra_bwd_bands(cu_seqlens, n_heads: int, pairs, causal: bool, scratch_bytes: int):
+    """Returns (clipped pairs of all bands, band index of each, number of bands); host only."""
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    n_out, n_bands = ctypes.c_int32(0), ctypes.c_int32(0)
+    args = (cu.ctypes.data, len(cu) - 1, n_heads, pp, npairs, int(bool(causal)), int(scratch_bytes))
+    s = _lib.hydra_bwd_bands(*args, None, None, 0, ctypes.addressof(n_out), ctypes.addressof(n_bands))
+    if s not in (HYDRA_OK, HYDRA_ERR_WORKSPACE_TOO_SMALL):
+        raise HydraError(s, "hydra_bwd_bands")
+    out = np.zeros(n_out.value, dtype=PAIR_DTYPE)
+    band = np.zeros(n_out.value, dtype=np.int32)
+    if n_out.value:
+        _check(_lib.hydra_bwd_bands(*args, out.ctypes.data, band.ctypes.data, len(out), ctypes.addressof(n_out),
+                                    ctypes.addressof(n_bands)), "hydra_bwd_bands")
+    return out, band, int(n_bands.value)
+
+
 def hydra_workspace_bytes(which: int, cu_seqlens, n_heads: int, pairs=None) -> int:
     cu = _cu(cu_seqlens)
     pp, npairs, _keep = _pairs_arg(pairs)
@@ -311,6 +333,11 @@ def hydra_attn_bwd_accumulate(q, k, v, out, lse, dout, cu_seqlens, n_heads: int,
 def hydra_set_bwd_scratch_limit(n_bytes: int) -> None:
     """Largest dS hand-off buffer the backward may ask for and use (0: always recompute)."""
     _lib.hydra_set_bwd_scratch_limit(int(n_bytes))
+
+
+def hydra_set_bwd_band_scratch(n_bytes: int) -> None:
+    """Scratch for the banded backward of problems whose dS buffer is over the limit (0: off)."""
+    _lib.hydra_set_bwd_band_scratch(int(n_bytes))
 
 
 def hydra_grad_cast(acc, grad, n_elements: Optional[int] = None, stream=None, check: bool = True) -> int:

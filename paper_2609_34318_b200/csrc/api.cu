@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cmath>
+#include <cstddef>
 #include <cstring>
 #include <map>
 #include <memory>
@@ -185,7 +186,7 @@ struct Plan {
 
 std::mutex g_plan_mutex;
 std::vector<std::unique_ptr<Plan>> g_plans;
-constexpr size_t kMaxPlans = 32;
+constexpr size_t kMaxPlans = 256;
 
 std::vector<uint8_t> make_key(int kind, int device, const Problem& pb, int causal)
 {
@@ -646,21 +647,30 @@ int32_t hydra_zigzag_pairs(const int32_t* cu, int32_t n_seqs, const int32_t* cp_
 namespace {
 std::atomic<uint64_t> g_ds_limit_bytes{uint64_t{4} << 30};
 
+std::atomic<uint64_t> g_band_bytes{0};
+// smallest scratch the banded backward is worth running with
+constexpr uint64_t kMinBandBytes = uint64_t{1} << 20;
+
+size_t bwd_acc_bytes(const Problem& pb)
+{
+    return align_up(static_cast<size_t>(pb.T) * pb.h * D_QK * sizeof(float), 1024);
+}
 size_t bwd_base_bytes(const Problem& pb)
 {
     return align_up(kStatusBytes + align_up(static_cast<size_t>(pb.T) * pb.h * sizeof(float), 256), 1024);
 }
 // bytes of the dS hand-off buffer, or 0 if it is not to be used (layout not possible, or over the limit)
-size_t bwd_ds_bytes(int64_t head_blocks, int32_t n_heads)
+size_t bwd_ds_bytes(int64_t head_blocks, int32_t n_heads, uint64_t limit)
 {
     if (head_blocks <= 0) return 0;
     if (static_cast<uint64_t>(head_blocks) * n_heads * TILE >= (uint64_t{1} << 31)) return 0;   // row index is 32-bit
     const uint64_t bytes = static_cast<uint64_t>(head_blocks) * n_heads * DS_BLOCK_BYTES;
-    return bytes <= g_ds_limit_bytes.load() ? static_cast<size_t>(bytes) : 0;
+    return bytes <= limit ? static_cast<size_t>(bytes) : 0;
 }
 }  // namespace
 
 void hydra_set_bwd_scratch_limit(uint64_t bytes) { g_ds_limit_bytes.store(bytes); }
+void hydra_set_bwd_band_scratch(uint64_t bytes) { g_band_bytes.store(bytes); }
 
 size_t hydra_workspace_bytes(int32_t which, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
                              const hydra_pair_t* pairs, int32_t n_pairs)
@@ -673,8 +683,16 @@ size_t hydra_workspace_bytes(int32_t which, const int32_t* cu, int32_t n_seqs, i
         case HYDRA_WS_BWD: {
             // D, plus the dS hand-off buffer when it stays within the limit (sized for a causal call)
             const size_t base = bwd_base_bytes(pb);
-            const size_t ds = bwd_ds_bytes(ds_layout(pb, 1, nullptr), n_heads);
-            return ds ? base + ds : base;
+            const int64_t head_blocks = ds_layout(pb, 1, nullptr);
+            const size_t ds = bwd_ds_bytes(head_blocks, n_heads, g_ds_limit_bytes.load());
+            if (ds) return base + ds;
+            // over the limit: the banded form, if switched on, wants an fp32 dq and its scratch
+            const uint64_t band = g_band_bytes.load();
+            if (head_blocks > 0 && band >= kMinBandBytes) {
+                const uint64_t full = static_cast<uint64_t>(head_blocks) * n_heads * DS_BLOCK_BYTES;
+                return base + bwd_acc_bytes(pb) + static_cast<size_t>(std::min(band, full));
+            }
+            return base;
         }
         default: return 0;
     }
@@ -792,6 +810,161 @@ int32_t merge_impl(const void* o_part, const float* lse_part, int64_t part_rows,
 }  // namespace
 
 namespace {
+struct BwdTensors {
+    const void *q, *k, *v, *out, *dout;
+    const float* lse;
+    void *dq, *dk, *dv;                 // bf16 outputs or fp32 accumulators
+};
+
+// One backward over the pairs of `pb`: D = rowsum(dO*O) (if `first`), the key-side kernel, the query-side
+// kernel. dq and dk/dv are bf16 outputs or fp32 accumulators, each by its own flag. `ds` / `ds_room` is
+// where a dS hand-off buffer may go. With `first` false the status block keeps its flags and only the
+// work-queue counters are cleared.
+int32_t bwd_run(const Problem& pb, int32_t causal, float softmax_scale, const BwdTensors& t, bool accumulate_dq,
+                bool accumulate_dkv, void* workspace, uint8_t* ds, size_t ds_room, uint64_t ds_limit, bool first, int sms,
+                cudaStream_t stream)
+{
+    const int32_t n_heads = pb.h;
+    const Plan* plan = nullptr;
+    if (int32_t s = get_plan(HYDRA_WS_BWD, pb, causal != 0, &plan)) return s;
+
+    float* dsum = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kStatusBytes);
+    CUtensorMap mq, mk, mv, mdo, mq_sub, mdo_sub;
+    if (make_map(&mq, t.q, pb.T, n_heads, D_QK, TILE) || make_map(&mk, t.k, pb.T, n_heads, D_QK, TILE) ||
+        make_map(&mv, t.v, pb.T, n_heads, D_V, TILE) || make_map(&mdo, t.dout, pb.T, n_heads, D_V, TILE) ||
+        make_map(&mq_sub, t.q, pb.T, n_heads, D_QK, SUB) || make_map(&mdo_sub, t.dout, pb.T, n_heads, D_V, SUB))
+        return HYDRA_ERR_CUDA;
+    if (first) {
+        if (int32_t s = reset_status(workspace, stream)) return s;
+        ScopedKernelTimer timer(K_PREP, stream);
+        if (launch_bwd_prep(t.dout, t.out, dsum, pb.T, n_heads, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+        g_launches += 1;
+    } else if (cudaMemsetAsync(static_cast<uint8_t*>(workspace) + offsetof(StatusBlock, next_item), 0,
+                               sizeof(StatusBlock::next_item), stream) != cudaSuccess) {
+        return HYDRA_ERR_CUDA;
+    }
+
+    BwdParams bp{};
+    bp.pairs = at<PairDev>(*plan, plan->off_pairs);
+    bp.lse = t.lse; bp.dsum = dsum; bp.dq = t.dq; bp.dk = t.dk; bp.dv = t.dv;
+    bp.T = pb.T; bp.h = n_heads; bp.causal = causal != 0;
+    bp.scale = softmax_scale; bp.scale_log2 = softmax_scale * 1.4426950408889634f;
+    bp.status = static_cast<StatusBlock*>(workspace);
+    bp.wait_limit_ns = g_wait_limit_ns.load();
+    // dS hand-off: the key-side kernel leaves dS^T in the workspace and the query-side kernel only
+    // multiplies it with K, if the buffer fits the room given and the limit set
+    const size_t ds_bytes = bwd_ds_bytes(plan->ds_head_blocks, n_heads, ds_limit);
+    const bool hand_off = ds_bytes > 0 && ds != nullptr && ds_room >= ds_bytes;
+    CUtensorMap mds;
+    if (hand_off) {
+        bp.ds = ds;
+        bp.ds_head_blocks = plan->ds_head_blocks;
+        if (make_map_ds(&mds, bp.ds, plan->ds_head_blocks * n_heads)) return HYDRA_ERR_CUDA;
+    }
+    if (plan->n_items2 > 0) {
+        bp.lists = at<int32_t>(*plan, plan->off_lists2);
+        bp.items = at<GroupItem>(*plan, plan->off_items2);
+        bp.n_items = plan->n_items2;
+        bp.accumulate = accumulate_dkv ? 1 : 0;
+        ScopedKernelTimer timer(K_DKV, stream);
+        if (launch_bwd_dkv(mq_sub, mk, mv, mdo_sub, bp, sms, stream) != cudaSuccess)
+            return HYDRA_ERR_CUDA;
+        g_launches += 1;
+    }
+    if (plan->n_items > 0) {
+        bp.lists = at<int32_t>(*plan, plan->off_lists);
+        bp.items = at<GroupItem>(*plan, plan->off_items);
+        bp.n_items = plan->n_items;
+        bp.accumulate = accumulate_dq ? 1 : 0;
+        ScopedKernelTimer timer(K_DQ, stream);
+        const cudaError_t e = hand_off ? launch_bwd_dq_from_ds(mds, mk, bp, sms, stream)
+                                       : launch_bwd_dq(mq, mk, mv, mdo, bp, sms, stream);
+        if (e != cudaSuccess)
+            return HYDRA_ERR_CUDA;
+        g_launches += 1;
+    }
+    return HYDRA_OK;
+}
+
+// Bands of key rows for a backward whose dS buffer is over the limit: every band is a list of pairs
+// clipped to some 128-row tiles of their key chunk (and, under the causal mask, to the query rows that
+// see those keys), chosen so that the band's own dS buffer fits `room`. A key tile lies in one band, so
+// dk and dv of a band are final; dq sums over the bands. Empty if some band cannot be made to fit, if a
+// clipped pair would have no visible position, or if the clipped chunks would break the
+// identical-or-disjoint rule.
+std::vector<std::vector<hydra_pair_t>> make_bands(const Problem& pb, int32_t causal, size_t room)
+{
+    std::vector<std::vector<hydra_pair_t>> bands;
+    // distinct key ranges, in order
+    std::vector<Range> ranges;
+    for (const auto& p : pb.pairs)
+        if (p.q_len > 0 && p.k_len > 0) ranges.push_back(Range{p.seq, p.k_start, p.k_len});
+    std::sort(ranges.begin(), ranges.end(), range_less);
+    ranges.erase(std::unique(ranges.begin(), ranges.end(),
+                             [](const Range& a, const Range& b) {
+                                 return a.seq == b.seq && a.start == b.start && a.len == b.len;
+                             }), ranges.end());
+    // appends the pairs of key range r clipped to its keys [c0, c1); false if one of them sees nothing
+    auto clip = [&](const Range& r, int32_t c0, int32_t c1, std::vector<hydra_pair_t>& into) {
+        for (const auto& p : pb.pairs) {
+            if (p.seq != r.seq || p.k_start != r.start || p.k_len != r.len || p.q_len <= 0) continue;
+            hydra_pair_t c = p;
+            c.k_start = p.k_start + c0;
+            c.k_len = c1 - c0;
+            if (causal) {                                  // query rows before the first key see nothing
+                const int32_t first = std::max(p.q_start, c.k_start);
+                if (first >= p.q_start + p.q_len) return false;
+                c.q_len = p.q_start + p.q_len - first;
+                c.q_start = first;
+            }
+            c.part_row = -1;
+            c.group = static_cast<int32_t>(into.size());
+            c.flags = 0;
+            into.push_back(c);
+        }
+        return true;
+    };
+    Problem probe;
+    probe.cu = pb.cu; probe.n_seqs = pb.n_seqs; probe.h = pb.h; probe.T = pb.T;
+    auto fits = [&](const std::vector<hydra_pair_t>& pairs) {
+        probe.pairs = pairs;
+        return bwd_ds_bytes(ds_layout(probe, causal, nullptr), pb.h, room) > 0;
+    };
+    std::vector<hydra_pair_t> cur;
+    for (const Range& r : ranges) {
+        const int32_t n = (r.len + TILE - 1) / TILE;
+        int32_t i = 0;
+        while (i < n) {
+            // the most key tiles [i, j) of this range that still fit beside what the band holds
+            int32_t lo = i, hi = n;
+            while (lo < hi) {
+                const int32_t mid = lo + (hi - lo + 1) / 2;
+                std::vector<hydra_pair_t> trial = cur;
+                if (clip(r, i * TILE, std::min(r.len, mid * TILE), trial) && fits(trial)) lo = mid;
+                else hi = mid - 1;
+            }
+            if (lo == i) {
+                if (cur.empty()) return {};                // one tile column alone does not fit
+                bands.push_back(std::move(cur));
+                cur.clear();
+                continue;
+            }
+            if (!clip(r, i * TILE, std::min(r.len, lo * TILE), cur)) return {};
+            i = lo;
+        }
+    }
+    if (!cur.empty()) bands.push_back(std::move(cur));
+    for (const auto& band : bands) {
+        std::vector<Range> rq, rk;
+        for (const auto& p : band) {
+            rq.push_back(Range{p.seq, p.q_start, p.q_len});
+            rk.push_back(Range{p.seq, p.k_start, p.k_len});
+        }
+        if (check_identical_or_disjoint(rq) || check_identical_or_disjoint(rk)) return {};
+    }
+    return bands;
+}
+
 int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, const float* lse,
                  const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
                  const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
@@ -820,63 +993,80 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     int sms = 0;
     if (int32_t s = device_info(&sms)) return s;
-    const Plan* plan = nullptr;
-    if (int32_t s = get_plan(HYDRA_WS_BWD, pb, causal != 0, &plan)) return s;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const BwdTensors t{q, k, v, out, dout, lse, dq, dk, dv};
+    const size_t room = workspace_bytes > ds_off ? workspace_bytes - ds_off : 0;
 
-    float* dsum = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kStatusBytes);
-    CUtensorMap mq, mk, mv, mdo, mq_sub, mdo_sub;
-    if (make_map(&mq, q, pb.T, n_heads, D_QK, TILE) || make_map(&mk, k, pb.T, n_heads, D_QK, TILE) ||
-        make_map(&mv, v, pb.T, n_heads, D_V, TILE) || make_map(&mdo, dout, pb.T, n_heads, D_V, TILE) ||
-        make_map(&mq_sub, q, pb.T, n_heads, D_QK, SUB) || make_map(&mdo_sub, dout, pb.T, n_heads, D_V, SUB))
-        return HYDRA_ERR_CUDA;
-    if (int32_t s = reset_status(workspace, stream)) return s;
-    {
-        ScopedKernelTimer timer(K_PREP, stream);
-        if (launch_bwd_prep(dout, out, dsum, pb.T, n_heads, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    // Banded form: the dS buffer of the whole call is over the limit, but the caller has switched the
+    // bands on and left room for an fp32 accumulator of dq and a band's scratch. Each band of key rows
+    // then runs with its own hand-off: dk and dv of its keys are final, dq is summed in fp32 over the
+    // bands and rounded once at the end.
+    const uint64_t band_limit = g_band_bytes.load();
+    const size_t acc_bytes = bwd_acc_bytes(pb);
+    if (!accumulate && band_limit >= kMinBandBytes && room >= acc_bytes + kMinBandBytes) {
+        const int64_t head_blocks = ds_layout(pb, causal, nullptr);
+        if (head_blocks > 0 && bwd_ds_bytes(head_blocks, n_heads, g_ds_limit_bytes.load()) == 0) {
+            const size_t scratch = static_cast<size_t>(std::min<uint64_t>(band_limit, room - acc_bytes));
+            const auto bands = make_bands(pb, causal, scratch);
+            if (!bands.empty()) {
+                float* dq_acc = reinterpret_cast<float*>(ws + ds_off);
+                if (cudaMemsetAsync(dq_acc, 0, acc_bytes, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+                const BwdTensors tb{q, k, v, out, dout, lse, dq_acc, dk, dv};
+                Problem band_pb;
+                band_pb.cu = pb.cu; band_pb.n_seqs = pb.n_seqs; band_pb.h = pb.h; band_pb.T = pb.T;
+                bool first = true;
+                for (const auto& band : bands) {
+                    band_pb.pairs = band;
+                    if (int32_t s = bwd_run(band_pb, causal, softmax_scale, tb, true, false, workspace,
+                                            ws + ds_off + acc_bytes, scratch, scratch, first, sms, stream))
+                        return s;
+                    first = false;
+                }
+                // round the query rows the pairs cover; rows outside every pair stay untouched, as in
+                // the one-shot form
+                std::vector<Range> rs;
+                for (const auto& p : pb.pairs)
+                    if (p.q_len > 0 && p.k_len > 0) rs.push_back(Range{p.seq, p.q_start, p.q_len});
+                std::sort(rs.begin(), rs.end(), range_less);
+                const size_t per_row = static_cast<size_t>(n_heads) * D_QK;
+                for (size_t i = 0; i < rs.size(); ++i) {
+                    if (i > 0 && rs[i].seq == rs[i - 1].seq && rs[i].start == rs[i - 1].start) continue;
+                    const size_t row = static_cast<size_t>(pb.cu[rs[i].seq]) + rs[i].start;
+                    ScopedKernelTimer timer(K_CAST, stream);
+                    if (launch_grad_cast(dq_acc + row * per_row, static_cast<uint16_t*>(dq) + row * per_row,
+                                         static_cast<int64_t>(rs[i].len) * per_row, stream) != cudaSuccess)
+                        return HYDRA_ERR_CUDA;
+                    g_launches += 1;
+                }
+                return HYDRA_OK;
+            }
+        }
     }
-    g_launches += 1;
-
-    BwdParams bp{};
-    bp.pairs = at<PairDev>(*plan, plan->off_pairs);
-    bp.lse = lse; bp.dsum = dsum; bp.dq = dq; bp.dk = dk; bp.dv = dv;
-    bp.T = pb.T; bp.h = n_heads; bp.causal = causal != 0;
-    bp.scale = softmax_scale; bp.scale_log2 = softmax_scale * 1.4426950408889634f;
-    bp.accumulate = accumulate ? 1 : 0;
-    bp.status = static_cast<StatusBlock*>(workspace);
-    bp.wait_limit_ns = g_wait_limit_ns.load();
-    // dS hand-off: the key-side kernel leaves dS^T in the workspace and the query-side kernel only
-    // multiplies it with K, if the buffer fits the workspace given and the limit set
-    const size_t ds_bytes = bwd_ds_bytes(plan->ds_head_blocks, n_heads);
-    const bool hand_off = ds_bytes > 0 && workspace_bytes >= ds_off + ds_bytes;
-    CUtensorMap mds;
-    if (hand_off) {
-        bp.ds = static_cast<uint8_t*>(workspace) + ds_off;
-        bp.ds_head_blocks = plan->ds_head_blocks;
-        if (make_map_ds(&mds, bp.ds, plan->ds_head_blocks * n_heads)) return HYDRA_ERR_CUDA;
-    }
-    if (plan->n_items2 > 0) {
-        bp.lists = at<int32_t>(*plan, plan->off_lists2);
-        bp.items = at<GroupItem>(*plan, plan->off_items2);
-        bp.n_items = plan->n_items2;
-        ScopedKernelTimer timer(K_DKV, stream);
-        if (launch_bwd_dkv(mq_sub, mk, mv, mdo_sub, bp, sms, stream) != cudaSuccess)
-            return HYDRA_ERR_CUDA;
-        g_launches += 1;
-    }
-    if (plan->n_items > 0) {
-        bp.lists = at<int32_t>(*plan, plan->off_lists);
-        bp.items = at<GroupItem>(*plan, plan->off_items);
-        bp.n_items = plan->n_items;
-        ScopedKernelTimer timer(K_DQ, stream);
-        const cudaError_t e = hand_off ? launch_bwd_dq_from_ds(mds, mk, bp, sms, stream)
-                                       : launch_bwd_dq(mq, mk, mv, mdo, bp, sms, stream);
-        if (e != cudaSuccess)
-            return HYDRA_ERR_CUDA;
-        g_launches += 1;
-    }
-    return HYDRA_OK;
+    return bwd_run(pb, causal, softmax_scale, t, accumulate, accumulate, workspace, ws + ds_off, room,
+                   g_ds_limit_bytes.load(), true, sms, stream);
 }
 }  // namespace
+
+int32_t hydra_bwd_bands(const int32_t* cu, int32_t n_seqs, int32_t n_heads, const hydra_pair_t* pairs,
+                        int32_t n_pairs, int32_t causal, uint64_t scratch_bytes, hydra_pair_t* pairs_out,
+                        int32_t* band_out, int32_t max_pairs, int32_t* n_pairs_out, int32_t* n_bands_out)
+{
+    if (!n_pairs_out || !n_bands_out || max_pairs < 0 || (max_pairs > 0 && (!pairs_out || !band_out)))
+        return HYDRA_ERR_INVALID_ARG;
+    Problem pb;
+    if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
+    const auto bands = make_bands(pb, causal, static_cast<size_t>(scratch_bytes));
+    int64_t n = 0;
+    for (size_t b = 0; b < bands.size(); ++b)
+        for (const auto& p : bands[b]) {
+            if (n < max_pairs) { pairs_out[n] = p; band_out[n] = static_cast<int32_t>(b); }
+            ++n;
+        }
+    if (n > INT32_MAX) return HYDRA_ERR_UNSUPPORTED;
+    *n_pairs_out = static_cast<int32_t>(n);
+    *n_bands_out = static_cast<int32_t>(bands.size());
+    return n > max_pairs ? HYDRA_ERR_WORKSPACE_TOO_SMALL : HYDRA_OK;
+}
 
 int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* out, const float* lse,
                        const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,

@@ -172,3 +172,53 @@ def test_product_does_not_import_the_oracle():
                     text = fh.read()
                 assert "import oracle" not in text and "from oracle" not in text, f
                 assert "hydra_oracle" not in text, f
+
+
+def _visible(p, causal):
+    """Boolean [q_len, k_len] mask of the positions a pair computes."""
+    qi = p["q_start"] + np.arange(p["q_len"])[:, None]
+    kj = p["k_start"] + np.arange(p["k_len"])[None, :]
+    return (kj <= qi) if causal else np.ones((p["q_len"], p["k_len"]), bool)
+
+
+@pytest.mark.parametrize("lengths,cp_r,causal,scratch", [
+    ([1000], 0, True, 1 << 20), ([1000], 0, False, 1 << 20), ([1500], 2, True, 1 << 20),
+    ([700, 130, 64, 900], [1, 0, 0, 2], True, 1 << 20), ([2048], 1, True, 3 << 19), ([300, 5], 0, True, 1 << 30)])
+def test_bands_cover_every_visible_position_once_and_fit_their_scratch(lengths, cp_r, causal, scratch):
+    h = 2
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    pairs = P.hydra_zigzag_pairs(cu, cp_r)[0] if cp_r else None
+    whole = pairs if pairs is not None else np.array(
+        [(b, 0, L, 0, L, -1, b, 0) for b, L in enumerate(lengths)], dtype=P.PAIR_DTYPE)
+    out, band, n_bands = P.hydra_bwd_bands(cu, h, pairs, causal, scratch)
+    assert n_bands >= 1 and len(out) == len(band) and list(band) == sorted(band)
+    cover = [np.zeros((L, L), np.int32) for L in lengths]
+    for p in out:
+        assert p["q_len"] > 0 and p["k_len"] > 0 and p["part_row"] == -1
+        assert p["q_start"] + p["q_len"] <= lengths[p["seq"]] and p["k_start"] + p["k_len"] <= lengths[p["seq"]]
+        cover[p["seq"]][p["q_start"]:p["q_start"] + p["q_len"], p["k_start"]:p["k_start"] + p["k_len"]] += \
+            _visible(p, causal)
+    want = [np.zeros((L, L), np.int32) for L in lengths]
+    for p in whole:
+        want[p["seq"]][p["q_start"]:p["q_start"] + p["q_len"], p["k_start"]:p["k_start"] + p["k_len"]] += \
+            _visible(p, causal)
+    for c, w in zip(cover, want):
+        assert np.array_equal(c, w)
+    # a band's dS buffer (16 KB per visible 64 x 128 block and head, plus one spare block) fits the scratch
+    for b in range(n_bands):
+        blocks = 1
+        for p in out[band == b]:
+            for jk in range(0, p["k_len"], 128):
+                first_q = max(0, p["k_start"] + jk - p["q_start"]) if causal else 0
+                if first_q < p["q_len"]:
+                    blocks += (p["q_len"] + 63) // 64 - first_q // 64
+        assert blocks * 16384 * h <= scratch + 4 * 16384 * h * len(out[band == b]), (b, blocks)
+    if scratch >= 1 << 30:
+        assert n_bands == 1
+    elif sum(L * L for L in lengths) > 1 << 20:
+        assert n_bands > 1
+
+
+def test_bands_refuse_a_scratch_smaller_than_one_tile_column():
+    out, band, n_bands = P.hydra_bwd_bands([0, 4096], 4, None, True, 1 << 16)
+    assert n_bands == 0 and len(out) == 0
