@@ -123,7 +123,7 @@ int32_t hydra_zigzag_pairs(const int32_t* cu_seqlens_host, int32_t n_seqs, const
  * bands of 128-row tiles whose own dS buffer fits the scratch and runs every band with the hand-off
  * (pairs clipped to the band's keys and, under the causal mask, to the query rows that see them). A key
  * tile lies in one band, so dk and dv come out as in the one-shot form; dq sums the bands' contributions
- * in fp32, in an unspecified order, and is rounded to bf16 once at the end. A problem that cannot be
+ * in fp32, band after band, and is rounded to bf16 once at the end. A problem that cannot be
  * banded (a single tile column over the scratch, or clipped chunks that would overlap without being
  * identical) runs in the recomputing form instead.
  */

@@ -497,21 +497,6 @@ int32_t make_map(CUtensorMap* map, const void* base, int64_t T, int32_t h, int32
     return r == CUDA_SUCCESS ? HYDRA_OK : HYDRA_ERR_CUDA;
 }
 
-// The dS hand-off buffer as a 2-D tensor: rows of 64 bf16, 128 rows per block; a box is two blocks.
-int32_t make_map_ds(CUtensorMap* map, const void* base, int64_t blocks)
-{
-    EncodeFn enc = encode_fn();
-    if (!enc) return HYDRA_ERR_CUDA;
-    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(SUB), static_cast<cuuint64_t>(blocks) * TILE};
-    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(SUB) * 2};
-    const cuuint32_t box[2] = {static_cast<cuuint32_t>(SUB), 2 * TILE};
-    const cuuint32_t es[2] = {1, 1};
-    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
-                           es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? HYDRA_OK : HYDRA_ERR_CUDA;
-}
-
 int32_t reset_status(void* workspace, cudaStream_t s)
 {
     return cudaMemsetAsync(workspace, 0, sizeof(StatusBlock), s) == cudaSuccess ? HYDRA_OK : HYDRA_ERR_CUDA;
@@ -663,7 +648,6 @@ size_t bwd_base_bytes(const Problem& pb)
 size_t bwd_ds_bytes(int64_t head_blocks, int32_t n_heads, uint64_t limit)
 {
     if (head_blocks <= 0) return 0;
-    if (static_cast<uint64_t>(head_blocks) * n_heads * TILE >= (uint64_t{1} << 31)) return 0;   // row index is 32-bit
     const uint64_t bytes = static_cast<uint64_t>(head_blocks) * n_heads * DS_BLOCK_BYTES;
     return bytes <= limit ? static_cast<size_t>(bytes) : 0;
 }
@@ -855,11 +839,9 @@ int32_t bwd_run(const Problem& pb, int32_t causal, float softmax_scale, const Bw
     // multiplies it with K, if the buffer fits the room given and the limit set
     const size_t ds_bytes = bwd_ds_bytes(plan->ds_head_blocks, n_heads, ds_limit);
     const bool hand_off = ds_bytes > 0 && ds != nullptr && ds_room >= ds_bytes;
-    CUtensorMap mds;
     if (hand_off) {
         bp.ds = ds;
         bp.ds_head_blocks = plan->ds_head_blocks;
-        if (make_map_ds(&mds, bp.ds, plan->ds_head_blocks * n_heads)) return HYDRA_ERR_CUDA;
     }
     if (plan->n_items2 > 0) {
         bp.lists = at<int32_t>(*plan, plan->off_lists2);
@@ -877,7 +859,7 @@ int32_t bwd_run(const Problem& pb, int32_t causal, float softmax_scale, const Bw
         bp.n_items = plan->n_items;
         bp.accumulate = accumulate_dq ? 1 : 0;
         ScopedKernelTimer timer(K_DQ, stream);
-        const cudaError_t e = hand_off ? launch_bwd_dq_from_ds(mds, mk, bp, sms, stream)
+        const cudaError_t e = hand_off ? launch_bwd_dq_from_ds(mk, bp, sms, stream)
                                        : launch_bwd_dq(mq, mk, mv, mdo, bp, sms, stream);
         if (e != cudaSuccess)
             return HYDRA_ERR_CUDA;

@@ -957,8 +957,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 ++c_pds;
                 if (p.ds) {
                     // Hand dS^T to the query-side kernel (after P and dS have gone to the tensor core: off the
-                    // chain S -> P, dS -> dV, dK). The block in memory is 128 rows of 64 bf16; a store straight
-                    // from registers would touch 32 cache lines per instruction.
+                    // chain S -> P, dS -> dV, dK).
                     if (si.li != ds_li) {
                         ds_li = si.li;
                         const DsGeom geo = ds_geom(si.cur.q_len, si.cur.off, p.causal);
@@ -966,23 +965,14 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                         ds_blk0 = static_cast<int64_t>(item.head) * p.ds_head_blocks + si.cur.ds_base +
                                   ds_rowstart(geo, jk) - ds_first(geo, jk);
                     }
-                    // transpose through the slice so that every store instruction of the warp writes whole
-                    // 64-byte row segments: lane l holds row l; afterwards it holds chunk l % 4 of rows l / 4 + 8 e
-                    const uint32_t slice = smem + kDsStage + warp * 2048;
-                    __syncwarp();                      // the reads of the previous sub-tile are over
+                    // The block in memory is 8 chunks (8 q rows each) of 128 kv rows x 16 bytes: lane = kv row,
+                    // so every store instruction of the warp writes 512 contiguous bytes.
+                    uint8_t* blk = static_cast<uint8_t*>(p.ds) + (ds_blk0 + si.u) * DS_BLOCK_BYTES + g * 4 * 2048 +
+                                   ((warp & 3) * 32 + lane) * 16;
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
-                        st_shared_v4(slice + lane * 64 + ((e ^ ((lane >> 1) & 3)) << 4), ds[4 * e], ds[4 * e + 1],
-                                     ds[4 * e + 2], ds[4 * e + 3]);
-                    __syncwarp();
-                    uint8_t* blk = static_cast<uint8_t*>(p.ds) + (ds_blk0 + si.u) * DS_BLOCK_BYTES +
-                                   ((warp & 3) * 32 + (lane >> 2)) * (SUB * 2) + g * 64 + (lane & 3) * 16;
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int row = 8 * e + (lane >> 2);
-                        const uint4 w = ld_shared_v4(slice + row * 64 + (((lane & 3) ^ ((row >> 1) & 3)) << 4));
-                        st_global_stream_v4(blk + e * 8 * (SUB * 2), w);
-                    }
+                        st_global_stream_v4(blk + e * 2048,
+                                            make_uint4(ds[4 * e], ds[4 * e + 1], ds[4 * e + 2], ds[4 * e + 3]));
                 }
             }
             if (!ok) break;
@@ -1076,7 +1066,7 @@ enum : int { B_DSFULL = 0, B_DSEMPTY = 4, B_KFULL = 8, B_KEMPTY = 10, B_ACCFULL 
 size_t bwd_dq_ds_smem_bytes() { return dqs::kTotal + 1024; }
 
 __global__ void __launch_bounds__(dqs::kThreadsS, 1)
-hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __grid_constant__ CUtensorMap map_k,
+hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_k,
                             const BwdParams p)
 {
     using namespace dqs;
@@ -1102,7 +1092,7 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
             mbar_init(bar(i), count);
         }
         fence_mbar_init();
-        tma_prefetch_desc(&map_ds); tma_prefetch_desc(&map_k);
+        tma_prefetch_desc(&map_k);
     }
     if (warp == 5) { tmem_alloc(smem_u32(&tmem_base_slot), kTmCols); tmem_relinquish(); }
     tc_fence_before_sync();
@@ -1178,8 +1168,8 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
                     const int64_t blk = static_cast<int64_t>(item.head) * p.ds_head_blocks + ti.cur.ds_base +
                                         ds_rowstart(geo, ti.t) + (u0 - ds_first(geo, ti.t));
                     mbar_arrive_expect_tx(bar(B_DSFULL + st), kDsBytes);
-                    tma_load_2d_hint(smem + st * kDsBytes, &map_ds, bar(B_DSFULL + st), 0, static_cast<int>(blk * TILE),
-                                     ds_policy);
+                    bulk_load_hint(smem + st * kDsBytes, static_cast<const uint8_t*>(p.ds) + blk * DS_BLOCK_BYTES,
+                                   kDsBytes, bar(B_DSFULL + st), ds_policy);
                     if (!popped) { it_ahead = pop_end(kq + 1, raw_next, item_next, first_next); popped = true; }
                 }
                 if (!popped) it_ahead = pop_end(kq + 1, raw_next, item_next, first_next);
@@ -1213,7 +1203,8 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
     } else if (warp == 5) {
         // ------------------------------------------------------------------ UMMA issuer
         constexpr uint32_t idesc = umma_idesc_bf16(TILE, D_QK, true, true);
-        constexpr uint32_t hi_ds = umma_desc_hi(DS_BLOCK_BYTES, 1024);   // dS^T: M chunks of 64 q rows 16 KB apart
+        // dS^T without swizzle: 8 kv rows are 128 bytes, chunks of 8 q rows are 2 KB apart (two blocks in a row)
+        constexpr uint32_t hi_ds = umma_desc_plain_hi(128, 2048);
         constexpr uint32_t hi_k = umma_desc_hi(kBox128, 1024);           // K: N chunks of 64 columns 16 KB apart
         uint32_t g = 0, n_acc = 0;
         bool ok = true;
@@ -1237,11 +1228,11 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
                 if (!ok) break;
                 tc_fence_after_sync();
                 if (elect_one()) {
-                    const uint32_t a_lo = umma_desc_lo(smem + ds_st * kDsBytes, DS_BLOCK_BYTES);
+                    const uint32_t a_lo = umma_desc_plain_lo(smem + ds_st * kDsBytes, 128);
                     const uint32_t b_lo = umma_desc_lo(smem + kK + k_st * 3 * kBox128, kBox128);
 #pragma unroll
                     for (int kk = 0; kk < TILE / 16; ++kk)
-                        umma_ss_w(tm + buf * kTmAcc, a_lo + kk * (2048 >> 4), hi_ds, b_lo + kk * (2048 >> 4), hi_k, idesc,
+                        umma_ss_w(tm + buf * kTmAcc, a_lo + kk * (256 >> 4), hi_ds, b_lo + kk * (2048 >> 4), hi_k, idesc,
                                   (kk > 0 || !first_tile) ? 1u : 0u);
                     umma_commit(bar(B_DSEMPTY + ds_st));
                     umma_commit(bar(B_KEMPTY + k_st));
@@ -1323,7 +1314,7 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_ds, const __
     if (warp == 5) tmem_dealloc(tm, kTmCols);
 }
 
-cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mds, const CUtensorMap& mk, const BwdParams& p, int grid,
+cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mk, const BwdParams& p, int grid,
                                   cudaStream_t stream)
 {
     static bool configured = false;
@@ -1334,7 +1325,7 @@ cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mds, const CUtensorMap& mk,
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    hydra_bwd_dq_from_ds_kernel<<<grid, dqs::kThreadsS, bwd_dq_ds_smem_bytes(), stream>>>(mds, mk, p);
+    hydra_bwd_dq_from_ds_kernel<<<grid, dqs::kThreadsS, bwd_dq_ds_smem_bytes(), stream>>>(mk, p);
     return cudaGetLastError();
 }
 

@@ -26,7 +26,9 @@ struct PairDev {
 };
 
 // Geometry of the dS hand-off buffer of the backward. The key-side kernel writes dS^T of every
-// (128-row kv tile jk, 64-row q sub-tile u) it visits as one block of 128 rows x 64 bf16 (16 KB); the
+// (128-row kv tile jk, 64-row q sub-tile u) it visits as one block of 16 KB: 8 chunks (8 q rows each) of
+// 128 kv rows x 16 bytes, which is the tensor core's operand layout without swizzle (so the writer's
+// stores are contiguous per warp and the reader's copy is one untiled bulk copy); the
 // query-side kernel reads the blocks (jk, 2i) and (jk, 2i + 1) of its q tile i. Per pair the blocks of
 // kv tile jk start at ds_rowstart(jk) and cover the sub-tiles ds_first(jk) .. nu_even - 1, where
 // ds_first is the first sub-tile the causal mask leaves visible, rounded down to an even number, so
@@ -168,7 +170,7 @@ cudaError_t launch_fwd(const CUtensorMap& mq, const CUtensorMap& mk, const CUten
 cudaError_t launch_bwd_dq(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                           const CUtensorMap& mdo, const BwdParams& p, int grid, cudaStream_t stream);
 size_t bwd_dq_ds_smem_bytes();
-cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mds, const CUtensorMap& mk, const BwdParams& p, int grid,
+cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mk, const BwdParams& p, int grid,
                                   cudaStream_t stream);
 cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, const CUtensorMap& mv,
                            const CUtensorMap& mdo_sub, const BwdParams& p, int grid, cudaStream_t stream);

@@ -163,6 +163,14 @@ __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap
         "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(pol)
         : "memory");
 }
+// Untiled bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completing on an mbarrier
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar,
+                                               uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::
+            "r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+        : "memory");
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -302,6 +310,17 @@ __host__ __device__ constexpr uint64_t umma_smem_desc_sw128(uint32_t smem_addr, 
            | (2ull << 61);                                                // SWIZZLE_128B
 }
 
+// The same descriptor for an operand without swizzle: 8 x 16-byte core matrices of 128 contiguous bytes.
+//   MN-major operand (a 16-byte unit holds 8 M/N elements of one K row; 8 K rows are 128 bytes):
+//     lbo = distance between groups of 8 K rows, sbo = distance between 8-element M/N chunks.
+__host__ __device__ constexpr uint64_t umma_smem_desc_plain(uint32_t smem_addr, uint32_t lbo_bytes,
+                                                            uint32_t sbo_bytes) {
+    return static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4)
+           | (static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16)
+           | (static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32)
+           | (1ull << 46);
+}
+
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
                                         uint32_t idesc, uint32_t accumulate) {
@@ -330,6 +349,12 @@ __host__ __device__ constexpr uint32_t umma_desc_hi(uint32_t lbo_bytes, uint32_t
 }
 __host__ __device__ constexpr uint32_t umma_desc_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
     return static_cast<uint32_t>(umma_smem_desc_sw128(smem_addr, lbo_bytes, 0) & 0xFFFFFFFFull);
+}
+__host__ __device__ constexpr uint32_t umma_desc_plain_hi(uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return static_cast<uint32_t>(umma_smem_desc_plain(0, lbo_bytes, sbo_bytes) >> 32);
+}
+__host__ __device__ constexpr uint32_t umma_desc_plain_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
+    return static_cast<uint32_t>(umma_smem_desc_plain(smem_addr, lbo_bytes, 0) & 0xFFFFFFFFull);
 }
 __device__ __forceinline__ void umma_ss_w(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
                                           uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
