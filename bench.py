@@ -557,9 +557,9 @@ def merge_groups(pairs):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised in
 # profiles/tensor_kernels_packed32k.md and profiles/merge_prep_short64k_split.md.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "fwd:packed32k": 685904000,
-    "bwd_dkv:packed32k": 2796371000,      # with the dS hand-off: 1.76 GB of it is dS written once
-    "bwd_dq:packed32k": 2069275000,       # hydra_bwd_dq_from_ds_kernel: 1.76 GB of it is dS read once
+    "fwd:packed32k": 686360000,
+    "bwd_dkv:packed32k": 2809982000,      # with the dS hand-off: 1.76 GB of it is dS written once
+    "bwd_dq:packed32k": 2072652000,       # hydra_bwd_dq_from_ds_kernel: 1.76 GB of it is dS read once
     "merge:short64k_split": 764355784,
     "bwd_prep:short64k_split": 1080946776,
 }

@@ -137,9 +137,35 @@ def gradient_identities(w, step, t):
         assert ((qdq - kdk).abs() / mag).max().item() < 2e-2, (w.name, b, "<q,dQ> != <k,dK>")
 
 
-def test_skewed_128k_sampled_rows_and_identities():
+@pytest.fixture(params=["bands_off", "banded_48gb"])
+def long_backward_form(request):
+    """The two forms of the backward on the long configurations: dq recomputing S and dP (the dS buffer of
+    the whole problem is over the limit), and the form bench.py times: bands of key rows with 48 GB of dS
+    scratch."""
+    import paper_2609_34318_b200 as P
+    P.hydra_set_bwd_band_scratch((48 << 30) if request.param == "banded_48gb" else 0)
+    yield request.param
+    P.hydra_set_bwd_band_scratch(0)
+
+
+def bands_ran(w, form, launches):
+    """The banded form launches the two backward kernels once per band."""
+    import paper_2609_34318_b200 as P
+    if form != "banded_48gb":
+        assert launches <= 6
+        return
+    cu = w.cu()
+    lib_pairs = pairs_for(cu, w.cp_r)[0] if w.cp_r else None
+    n_bands = P.hydra_bwd_bands(cu, w.n_heads, lib_pairs, True, 48 << 30)[2]
+    assert n_bands >= 2 and launches >= 2 * n_bands + 2, (n_bands, launches)
+
+
+def test_skewed_128k_sampled_rows_and_identities(long_backward_form):
+    import paper_2609_34318_b200 as P
     w = hw.workload("skewed128k")
+    n0 = P.hydra_launch_count()
     step, t, _ = run_workload(w)
+    bands_ran(w, long_backward_form, P.hydra_launch_count() - n0)
     cu = w.cu()
     b_long = int(np.argmax(w.lengths))
     lo, hi = int(cu[b_long]), int(cu[b_long + 1])
@@ -152,9 +178,12 @@ def test_skewed_128k_sampled_rows_and_identities():
     assert torch.isfinite(step.out.float()).all()
 
 
-def test_ring_256k_sampled_rows_and_identities():
+def test_ring_256k_sampled_rows_and_identities(long_backward_form):
+    import paper_2609_34318_b200 as P
     w = hw.workload("ring256k")
+    n0 = P.hydra_launch_count()
     step, t, ora_pairs = run_workload(w)
+    bands_ran(w, long_backward_form, P.hydra_launch_count() - n0)
     assert len(ora_pairs) == 36
     L = w.total
     rng = np.random.default_rng(2)
