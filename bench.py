@@ -407,6 +407,7 @@ def run_report(args, w):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1)
 
+    P.hydra_set_bwd_band_scratch(int(args.band_scratch_gb * 2 ** 30))
     t0 = time.perf_counter()
     step = AttnStep(cu, w.n_heads, pairs, part_rows, True, float(w.scale))
     first_ms = timed_step(step, t)
@@ -415,11 +416,13 @@ def run_report(args, w):
         timed_step(step, t)
     P.hydra_profile_enable(True)
     P.hydra_profile_collect()
-    rows = {k: [] for k in ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "step")}
+    rows = {k: [] for k in ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast", "step")}
+    bands = 1
     for _ in range(args.steps):
         flush.zero_()                                        # 256 MB > L2: the next kernels start cold
         ms = timed_step(step, t)
-        kernel_ms, _ = P.hydra_profile_collect()
+        kernel_ms, kernel_n = P.hydra_profile_collect()
+        bands = max(bands, int(kernel_n.get("bwd_dkv", 1)))
         for k in rows:
             rows[k].append(ms if k == "step" else kernel_ms.get(k, 0.0))
     P.hydra_profile_enable(False)
@@ -427,8 +430,8 @@ def run_report(args, w):
     med = {k: statistics.median(v) for k, v in rows.items()}
     best = {k: min(v) for k, v in rows.items()}
     f_fwd = w.flops_fwd()
-    kernels_ms = med["fwd"] + med["merge"] + med["bwd_prep"] + med["bwd_dkv"] + med["bwd_dq"]
-    bwd_ms = med["bwd_prep"] + med["bwd_dkv"] + med["bwd_dq"]
+    kernels_ms = med["fwd"] + med["merge"] + med["bwd_prep"] + med["bwd_dkv"] + med["bwd_dq"] + med["grad_cast"]
+    bwd_ms = med["bwd_prep"] + med["bwd_dkv"] + med["bwd_dq"] + med["grad_cast"]
     tf = lambda flops, ms: flops / (ms * 1e-3) / 1e12 if ms > 0 else None
     total = tf(3.5 * f_fwd, kernels_ms)
     th = w.total * w.n_heads
@@ -438,7 +441,9 @@ def run_report(args, w):
         "workload": w.name, "repetitions": args.steps, "l2": "256 MB written between repetitions",
         "median_ms": med, "best_ms": best,
         "tflops": {"total": total, "fwd_only": tf(f_fwd, med["fwd"] + med["merge"]), "bwd_only": tf(2.5 * f_fwd, bwd_ms),
-                   "total_best": tf(3.5 * f_fwd, sum(best[k] for k in ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq")))},
+                   "total_best": tf(3.5 * f_fwd, sum(best[k] for k in ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq",
+                                                                       "grad_cast")))},
+        "bwd_bands": bands, "band_scratch_gb": args.band_scratch_gb,
         "of_peak": {"measured_burst": total / peaks["bf16_tflops"],
                     "measured_sustained": total / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
                     "nominal_2250": total / 2250.0, "peaks": peak_kind},

@@ -22,3 +22,4 @@ from .attention import (  # noqa: F401
     zigzag_chunks,
     zigzag_rank,
 )
+from .ulysses import all_to_all, ulysses_pack, ulysses_unpack  # noqa: F401,E402

@@ -76,3 +76,39 @@ def test_weak_scaling_aggregate_is_linear_in_ranks():
     one = bench.whole_job_value(1, 1.0e12, 10, 5.0)
     eight = bench.whole_job_value(8, 1.0e12, 10, 5.0)
     assert eight == pytest.approx(8 * one)
+
+
+def _ulysses_rank(rank: int, world: int, port: int, out_dir: str):
+    """One rank of a Ulysses group over gloo: pack, a real all-to-all, check the head split; then the way
+    back through a second all-to-all and unpack."""
+    import oracle
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        n, h, d = 5, 6, 4
+        hg = h // world
+        X = np.arange(world * n * h * d, dtype=np.int64).reshape(world * n, h, d).astype(np.uint16)   # same on all ranks
+        mine = X[rank * n:(rank + 1) * n]
+        # the transport carries the 16-bit elements widened to int32 (gloo has no 16-bit all-to-all)
+        send = torch.from_numpy(oracle.ulysses_pack(mine, world).astype(np.int32))
+        recv = torch.empty_like(send)
+        dist.all_to_all_single(recv, send)                           # equal blocks along dim 0
+        got = recv.numpy().astype(np.uint16).reshape(world * n, hg, d)
+        ok_in = bool(np.array_equal(got, X[:, rank * hg:(rank + 1) * hg, :]))
+        back = torch.from_numpy(got.reshape(world, n, hg, d).astype(np.int32))
+        recv2 = torch.empty_like(back)
+        dist.all_to_all_single(recv2, back)
+        ok_out = bool(np.array_equal(oracle.ulysses_unpack(recv2.numpy().astype(np.uint16)), mine))
+        with open(os.path.join(out_dir, f"uly{rank}.json"), "w") as f:
+            json.dump({"in": ok_in, "out": ok_out}, f)
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_ulysses_pack_unpack_around_a_real_all_to_all(tmp_path):
+    world, port = 2, _free_port()
+    mp.spawn(_ulysses_rank, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    for i in range(world):
+        r = json.load(open(tmp_path / f"uly{i}.json"))
+        assert r["in"] and r["out"]
