@@ -489,6 +489,32 @@ def run_report(args, w):
     if by_step:
         report["accumulating_backward"]["ring_steps"] = len(calls)
         report["accumulating_backward"]["by_step_ms"] = {k: pick(by_step, k) for k in ("bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast")}
+    # The local permutations around the head <-> sequence all-to-all of an inner Ulysses group of 4 (q of
+    # this workload; 4 bytes moved per element), with L2 flushed before each.
+    del acc, grads
+    if w.n_heads % 4 == 0:
+        send = torch.empty((4, w.total, w.n_heads // 4, hw.D_QK), dtype=torch.bfloat16, device="cuda")
+        back = torch.empty_like(t["q"])
+        P.hydra_profile_enable(True)
+        runs = []
+        for _ in range(5):
+            flush.zero_()
+            P.hydra_profile_collect()
+            P.hydra_ulysses_pack(t["q"], w.total, w.n_heads, hw.D_QK, 4, send)
+            torch.cuda.synchronize()
+            pack_ms = P.hydra_profile_collect()[0]["ulysses"]
+            flush.zero_()
+            P.hydra_ulysses_unpack(send, w.total, w.n_heads, hw.D_QK, 4, back)
+            torch.cuda.synchronize()
+            runs.append((pack_ms, P.hydra_profile_collect()[0]["ulysses"]))
+        P.hydra_profile_enable(False)
+        assert torch.equal(back, t["q"])
+        moved = t["q"].numel() * 4.0
+        report["ulysses_cp4"] = {"bytes": moved, "pack_ms": statistics.median(r[0] for r in runs),
+                                 "unpack_ms": statistics.median(r[1] for r in runs),
+                                 "pack_gbs": gbs(moved, statistics.median(r[0] for r in runs)),
+                                 "unpack_gbs": gbs(moved, statistics.median(r[1] for r in runs))}
+        del send, back
     if args.per_sequence:
         # every sequence alone, same kernels: its share of the time next to its share of sum(L^2)
         shares = []

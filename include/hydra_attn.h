@@ -286,10 +286,35 @@ int32_t hydra_attn_fwd_bwd_host(const void* q_host, const void* k_host, const vo
                                 size_t arena_bytes, void* cuda_stream);
 
 /*
+ * The local halves of the Ulysses all-to-all (Section 3.3: all-to-all transposes partition the attention
+ * heads across the cp_u ranks of a group; Eq. (ulysses) counts the volume, about 4 S h / P elements per
+ * rank for q, k, v and the output). Elements are 2 bytes wide (bf16) and are moved, not interpreted.
+ *   hydra_ulysses_pack    x device [n_tokens, n_heads, head_dim] (this rank's tokens, all heads)
+ *                         -> send device [cp_u, n_tokens, n_heads / cp_u, head_dim]:
+ *                         send[j, t, b, :] = x[t, j * (n_heads / cp_u) + b, :]; block j goes to rank j.
+ *                         With equal n_tokens on every rank the received buffer is
+ *                         [cp_u * n_tokens, n_heads / cp_u, head_dim], tokens in rank order: the layout
+ *                         hydra_attn_fwd takes, without another copy.
+ *   hydra_ulysses_unpack  recv device [cp_u, n_tokens, n_heads / cp_u, head_dim] (block j from rank j: this
+ *                         rank's tokens, rank j's heads) -> y device [n_tokens, n_heads, head_dim], the
+ *                         inverse permutation (the way back after attention; on that way the split by
+ *                         token owner before the exchange is contiguous and needs no kernel).
+ * Requirements: cp_u divides n_heads; (n_heads / cp_u) * head_dim * 2 is a multiple of 16 bytes (else
+ * HYDRA_ERR_UNSUPPORTED, as is a tensor of more than 60 GB); pointers 16-byte aligned, distinct buffers (not
+ * in place). One kernel launch on
+ * cuda_stream, HBM-bound: 4 bytes moved per element. HYDRA_ERR_INVALID_ARG on bad arguments.
+ */
+int32_t hydra_ulysses_pack(const void* x, int64_t n_tokens, int32_t n_heads, int32_t head_dim, int32_t cp_u,
+                           void* send, void* cuda_stream);
+int32_t hydra_ulysses_unpack(const void* recv, int64_t n_tokens, int32_t n_heads, int32_t head_dim, int32_t cp_u,
+                             void* y, void* cuda_stream);
+
+/*
  * Per-kernel timing (measurement aid, not part of the method). While enabled, every kernel launch
  * is bracketed by CUDA events on its stream. hydra_profile_collect waits for the recorded events,
- * adds their durations into ms_out[6] and their counts into launches_out[6] (index: 0 forward,
- * 1 merge, 2 backward prep, 3 backward dK/dV, 4 backward dQ, 5 gradient cast) and forgets them.
+ * adds their durations into ms_out[7] and their counts into launches_out[7] (index: 0 forward,
+ * 1 merge, 2 backward prep, 3 backward dK/dV, 4 backward dQ, 5 gradient cast, 6 Ulysses pack / unpack)
+ * and forgets them.
  */
 void hydra_profile_enable(int32_t on);
 int32_t hydra_profile_collect(double* ms_out, int64_t* launches_out);

@@ -59,6 +59,10 @@ def _load() -> ctypes.CDLL:
     lib.hydra_usp_factor.argtypes = [i32, i32, vp, vp]
     lib.hydra_zigzag_pairs.restype = i32
     lib.hydra_zigzag_pairs.argtypes = [vp, i32, vp, i32, vp, i32, vp, vp, vp, vp]
+    for name in ("hydra_ulysses_pack", "hydra_ulysses_unpack"):
+        fn = getattr(lib, name)
+        fn.restype = i32
+        fn.argtypes = [vp, ctypes.c_int64, i32, i32, i32, vp, vp]
     lib.hydra_bwd_bands.restype = i32
     lib.hydra_bwd_bands.argtypes = [vp, i32, i32, vp, i32, i32, ctypes.c_uint64, vp, vp, i32, vp, vp]
     lib.hydra_workspace_bytes.restype = sz
@@ -114,9 +118,9 @@ EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
            "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc", "hydra_lse_merge_accumulate",
            "hydra_sched_targets", "hydra_sched_cp", "hydra_sched_pack", "hydra_attn_bwd_accumulate",
-           "hydra_grad_cast", "hydra_set_bwd_scratch_limit", "hydra_set_bwd_band_scratch", "hydra_bwd_bands",
+           "hydra_grad_cast", "hydra_set_bwd_scratch_limit", "hydra_set_bwd_band_scratch", "hydra_bwd_bands", "hydra_ulysses_pack", "hydra_ulysses_unpack",
            "hydra_poll_clocks")
-KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast")
+KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast", "ulysses")
 
 
 # ------------------------------------------------------------------------------------------------
@@ -333,6 +337,26 @@ def hydra_attn_bwd_accumulate(q, k, v, out, lse, dout, cu_seqlens, n_heads: int,
 def hydra_set_bwd_scratch_limit(n_bytes: int) -> None:
     """Largest dS hand-off buffer the backward may ask for and use (0: always recompute)."""
     _lib.hydra_set_bwd_scratch_limit(int(n_bytes))
+
+
+def hydra_ulysses_pack(x, n_tokens: int, n_heads: int, head_dim: int, cp_u: int, send, stream=None,
+                       check: bool = True) -> int:
+    """send[j, t, b, :] = x[t, j * (n_heads / cp_u) + b, :] (2-byte elements)."""
+    s = _lib.hydra_ulysses_pack(_ptr(x), int(n_tokens), int(n_heads), int(head_dim), int(cp_u), _ptr(send),
+                                _stream(stream))
+    if check:
+        _check(s, "hydra_ulysses_pack")
+    return s
+
+
+def hydra_ulysses_unpack(recv, n_tokens: int, n_heads: int, head_dim: int, cp_u: int, y, stream=None,
+                         check: bool = True) -> int:
+    """y[t, j * (n_heads / cp_u) + b, :] = recv[j, t, b, :] (2-byte elements)."""
+    s = _lib.hydra_ulysses_unpack(_ptr(recv), int(n_tokens), int(n_heads), int(head_dim), int(cp_u), _ptr(y),
+                                  _stream(stream))
+    if check:
+        _check(s, "hydra_ulysses_unpack")
+    return s
 
 
 def hydra_set_bwd_band_scratch(n_bytes: int) -> None:

@@ -24,7 +24,7 @@ constexpr size_t kStatusBytes = 256;
 // ---------------------------------------------------------------------------------------------
 // optional per-kernel timing with CUDA events on the launching stream
 // ---------------------------------------------------------------------------------------------
-enum KernelKind { K_FWD = 0, K_MERGE, K_PREP, K_DKV, K_DQ, K_CAST, K_COUNT };
+enum KernelKind { K_FWD = 0, K_MERGE, K_PREP, K_DKV, K_DQ, K_CAST, K_ULYSSES, K_COUNT };
 struct ProfRecord { int kind; cudaEvent_t start, stop; };
 std::mutex g_prof_mutex;
 bool g_prof_on = false;
@@ -1314,6 +1314,38 @@ int32_t hydra_attn_fwd_bwd_host(const void* q_host, const void* k_host, const vo
     // the caller's stream completes when the last copy out has completed
     if (cudaEventRecord(pipe->end, pipe->out) || cudaStreamWaitEvent(stream, pipe->end, 0)) return HYDRA_ERR_CUDA;
     return HYDRA_OK;
+}
+
+namespace {
+int32_t ulysses_impl(bool pack, const void* x, int64_t n_tokens, int32_t n_heads, int32_t head_dim, int32_t cp_u,
+                     void* out, void* cuda_stream)
+{
+    if (n_tokens < 0 || n_heads < 1 || head_dim < 1 || cp_u < 1 || n_heads % cp_u) return HYDRA_ERR_INVALID_ARG;
+    const int64_t chunk_bytes = static_cast<int64_t>(n_heads / cp_u) * head_dim * 2;
+    if (chunk_bytes % 16) return HYDRA_ERR_UNSUPPORTED;
+    if (n_tokens == 0) return HYDRA_OK;
+    if (!x || !out || x == out || !aligned16(x) || !aligned16(out)) return HYDRA_ERR_INVALID_ARG;
+    // the kernel indexes 16-byte units with 32 bits: tensors up to 60 GB
+    if (n_tokens > (int64_t{60} << 30) / (chunk_bytes * cp_u)) return HYDRA_ERR_UNSUPPORTED;
+    if (int32_t s = device_info(nullptr)) return s;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ScopedKernelTimer timer(K_ULYSSES, stream);
+    if (launch_ulysses(pack, x, out, n_tokens, cp_u, chunk_bytes / 16, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    g_launches += 1;
+    return HYDRA_OK;
+}
+}  // namespace
+
+int32_t hydra_ulysses_pack(const void* x, int64_t n_tokens, int32_t n_heads, int32_t head_dim, int32_t cp_u,
+                           void* send, void* cuda_stream)
+{
+    return ulysses_impl(true, x, n_tokens, n_heads, head_dim, cp_u, send, cuda_stream);
+}
+
+int32_t hydra_ulysses_unpack(const void* recv, int64_t n_tokens, int32_t n_heads, int32_t head_dim, int32_t cp_u,
+                             void* y, void* cuda_stream)
+{
+    return ulysses_impl(false, recv, n_tokens, n_heads, head_dim, cp_u, y, cuda_stream);
 }
 
 int32_t hydra_poll_status(void* workspace, void* cuda_stream, int32_t* device_status, int64_t* detail)

@@ -176,6 +176,8 @@ cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, con
                            const CUtensorMap& mdo_sub, const BwdParams& p, int grid, cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
 cudaError_t launch_grad_cast(const float* acc, void* grad, int64_t n, cudaStream_t stream);
+cudaError_t launch_ulysses(bool pack, const void* src, void* dst, int64_t n_tokens, int32_t cp_u, int64_t chunk_units,
+                           cudaStream_t stream);
 cudaError_t launch_bwd_prep(const void* dout, const void* out, float* dsum, int64_t T, int32_t h,
                             cudaStream_t stream);
 

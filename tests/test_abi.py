@@ -222,3 +222,15 @@ def test_bands_cover_every_visible_position_once_and_fit_their_scratch(lengths, 
 def test_bands_refuse_a_scratch_smaller_than_one_tile_column():
     out, band, n_bands = P.hydra_bwd_bands([0, 4096], 4, None, True, 1 << 16)
     assert n_bands == 0 and len(out) == 0
+
+
+def test_ulysses_pack_validation_without_a_gpu():
+    args = dict(stream=0, check=False)
+    assert P.hydra_ulysses_pack(0x1000, 8, 6, 8, 4, 0x2000, **args) == P.HYDRA_ERR_INVALID_ARG     # 4 does not divide 6
+    assert P.hydra_ulysses_pack(0x1000, 8, 3, 4, 3, 0x2000, **args) == P.HYDRA_ERR_UNSUPPORTED     # 8-byte chunks
+    assert P.hydra_ulysses_pack(0x1000, 0, 4, 8, 2, 0x2000, **args) == P.HYDRA_OK                  # nothing to move
+    assert P.hydra_ulysses_pack(0x1000, 8, 4, 8, 2, 0x1000, **args) == P.HYDRA_ERR_INVALID_ARG     # in place
+    assert P.hydra_ulysses_unpack(0x1008, 8, 4, 8, 2, 0x2000, **args) == P.HYDRA_ERR_INVALID_ARG   # misaligned
+    assert P.hydra_ulysses_unpack(0, 8, 4, 8, 2, 0x2000, **args) == P.HYDRA_ERR_INVALID_ARG
+    assert P.hydra_ulysses_pack(0x1000, 1 << 34, 64, 192, 4, 0x2000, **args) == P.HYDRA_ERR_UNSUPPORTED
+    assert P.hydra_ulysses_pack(0x1000, -1, 4, 8, 2, 0x2000, **args) == P.HYDRA_ERR_INVALID_ARG
