@@ -23,3 +23,4 @@ from .attention import (  # noqa: F401
     zigzag_rank,
 )
 from .ulysses import all_to_all, ulysses_pack, ulysses_unpack  # noqa: F401,E402
+from .gqa import attn_bwd_gqa, attn_bwd_pairs_gqa, attn_fwd_gqa, expand_kv, reduce_kv  # noqa: F401,E402
