@@ -515,6 +515,35 @@ def run_report(args, w):
                                  "pack_gbs": gbs(moved, statistics.median(r[0] for r in runs)),
                                  "unpack_gbs": gbs(moved, statistics.median(r[1] for r in runs))}
         del send, back
+    # Grouped-query form (eight query heads per KV head, as in the GQA model of Section 6): forward and the
+    # accumulating backward, same q / dO, K and V of h / 8 heads.
+    if w.n_heads % 8 == 0:
+        h_kv = w.n_heads // 8
+        kg, vg = t["k"][:, :h_kv].contiguous(), t["v"][:, :h_kv].contiguous()
+        gacc = [torch.zeros((w.total, hh, d), dtype=torch.float32, device="cuda")
+                for hh, d in ((w.n_heads, hw.D_QK), (h_kv, hw.D_QK), (h_kv, hw.D_V))]
+
+        def gqa_pass():
+            flush.zero_()
+            P.hydra_profile_collect()
+            P.hydra_attn_fwd_gqa(t["q"], kg, vg, cu, w.n_heads, h_kv, pairs, True, float(w.scale), step.out, step.lse,
+                                 step.o_part if step.has_partials else None,
+                                 step.lse_part if step.has_partials else None, part_rows, step.workspace)
+            if step.has_partials:
+                P.hydra_lse_merge(step.o_part, step.lse_part, part_rows, cu, w.n_heads, pairs, step.out, step.lse,
+                                  step.workspace)
+            P.hydra_attn_bwd_accumulate_gqa(t["q"], kg, vg, step.out, step.lse, t["do"], cu, w.n_heads, h_kv, pairs,
+                                            True, float(w.scale), gacc[0], gacc[1], gacc[2], step.workspace)
+            torch.cuda.synchronize()
+            return P.hydra_profile_collect()[0]
+
+        P.hydra_profile_enable(True)
+        gqa_pass()
+        gruns = [gqa_pass() for _ in range(3)]
+        P.hydra_profile_enable(False)
+        gms = {k: pick(gruns, k) for k in ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq")}
+        report["gqa_8_to_1"] = {"kv_heads": h_kv, "ms": gms, "tflops": tf(3.5 * f_fwd, sum(gms.values()))}
+        del gacc, kg, vg
     if args.per_sequence:
         # every sequence alone, same kernels: its share of the time next to its share of sum(L^2)
         shares = []

@@ -262,6 +262,30 @@ int32_t hydra_attn_bwd_accumulate(const void* q, const void* k, const void* v, c
 int32_t hydra_grad_cast(const float* acc, void* grad, int64_t n_elements, void* cuda_stream);
 
 /*
+ * Grouped-query form (Table "Notation": h query heads and h_kv KV heads per rank; the GQA model of
+ * Section 6 shares eight KV heads). With g = n_heads / n_kv_heads, query head a reads KV head a / g
+ * (integer division); n_kv_heads must divide n_heads. k device bf16 [T, n_kv_heads, 192], v device bf16
+ * [T, n_kv_heads, 128]; everything else as in hydra_attn_fwd / hydra_attn_bwd_accumulate, which are the
+ * case n_kv_heads == n_heads.
+ * The backward exists in the accumulating form only: dk_acc device fp32 [T, n_kv_heads, 192], dv_acc device
+ * fp32 [T, n_kv_heads, 128] receive, per KV head, the SUM over the g query heads that read it (the work
+ * items of the g query heads add into the same rows with fp32 reductions, so the order of the g terms, and
+ * with it the last bits of dk / dv, may differ from run to run); dq_acc device fp32 [T, n_heads, 192].
+ * The caller zeroes the accumulators and rounds them with hydra_grad_cast.
+ */
+int32_t hydra_attn_fwd_gqa(const void* q, const void* k, const void* v, const int32_t* cu_seqlens_host,
+                           int32_t n_seqs, int32_t n_heads, int32_t n_kv_heads, const hydra_pair_t* pairs,
+                           int32_t n_pairs, int32_t causal, float softmax_scale, void* out, float* lse,
+                           void* o_part, float* lse_part, int64_t part_rows, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream);
+int32_t hydra_attn_bwd_accumulate_gqa(const void* q, const void* k, const void* v, const void* out,
+                                      const float* lse, const void* dout, const int32_t* cu_seqlens_host,
+                                      int32_t n_seqs, int32_t n_heads, int32_t n_kv_heads,
+                                      const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal,
+                                      float softmax_scale, float* dq_acc, float* dk_acc, float* dv_acc,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * The whole step (forward of every pair, merge, backward; Sections 3.5 and 5.2 as above) with HOST
  * buffers: copies q, k, v, dout to the device, runs hydra_attn_fwd, hydra_lse_merge (if any pair has
  * partial rows) and hydra_attn_bwd, and copies out, lse, dq, dk, dv back. Heads are independent,

@@ -90,6 +90,12 @@ def _load() -> ctypes.CDLL:
     lib.hydra_set_bwd_band_scratch.argtypes = [ctypes.c_uint64]
     lib.hydra_attn_bwd_accumulate.restype = i32
     lib.hydra_attn_bwd_accumulate.argtypes = lib.hydra_attn_bwd.argtypes
+    lib.hydra_attn_fwd_gqa.restype = i32
+    lib.hydra_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, i32, i32, f32, vp, vp, vp, vp, i64,
+                                       vp, sz, vp]
+    lib.hydra_attn_bwd_accumulate_gqa.restype = i32
+    a = list(lib.hydra_attn_bwd.argtypes)
+    lib.hydra_attn_bwd_accumulate_gqa.argtypes = a[:9] + [i32] + a[9:]
     lib.hydra_grad_cast.restype = i32
     lib.hydra_grad_cast.argtypes = [vp, vp, i64, vp]
     lib.hydra_poll_status.restype = i32
@@ -118,7 +124,7 @@ EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
            "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc", "hydra_lse_merge_accumulate",
            "hydra_sched_targets", "hydra_sched_cp", "hydra_sched_pack", "hydra_attn_bwd_accumulate",
-           "hydra_grad_cast", "hydra_set_bwd_scratch_limit", "hydra_set_bwd_band_scratch", "hydra_bwd_bands", "hydra_ulysses_pack", "hydra_ulysses_unpack",
+           "hydra_grad_cast", "hydra_set_bwd_scratch_limit", "hydra_set_bwd_band_scratch", "hydra_bwd_bands", "hydra_ulysses_pack", "hydra_ulysses_unpack", "hydra_attn_fwd_gqa", "hydra_attn_bwd_accumulate_gqa",
            "hydra_poll_clocks")
 KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast", "ulysses")
 
@@ -331,6 +337,41 @@ def hydra_attn_bwd_accumulate(q, k, v, out, lse, dout, cu_seqlens, n_heads: int,
                                        _ptr(dv_acc), _ptr(workspace), int(workspace_bytes), _stream(stream))
     if check:
         _check(s, "hydra_attn_bwd_accumulate")
+    return s
+
+
+def hydra_attn_fwd_gqa(q, k, v, cu_seqlens, n_heads: int, n_kv_heads: int, pairs, causal: bool,
+                       softmax_scale: float, out, lse, o_part, lse_part, part_rows: int, workspace,
+                       workspace_bytes: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """hydra_attn_fwd with k, v of n_kv_heads heads: query head a reads KV head a // (n_heads / n_kv_heads)."""
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = _lib.hydra_attn_fwd_gqa(_ptr(q), _ptr(k), _ptr(v), cu.ctypes.data, len(cu) - 1, n_heads, n_kv_heads, pp,
+                                npairs, int(bool(causal)), ctypes.c_float(float(softmax_scale)), _ptr(out),
+                                _ptr(lse), _ptr(o_part), _ptr(lse_part), int(part_rows), _ptr(workspace),
+                                int(workspace_bytes), _stream(stream))
+    if check:
+        _check(s, "hydra_attn_fwd_gqa")
+    return s
+
+
+def hydra_attn_bwd_accumulate_gqa(q, k, v, out, lse, dout, cu_seqlens, n_heads: int, n_kv_heads: int, pairs,
+                                  causal: bool, softmax_scale: float, dq_acc, dk_acc, dv_acc, workspace,
+                                  workspace_bytes: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """hydra_attn_bwd_accumulate with shared KV heads: dk_acc, dv_acc have n_kv_heads heads."""
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = _lib.hydra_attn_bwd_accumulate_gqa(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout),
+                                           cu.ctypes.data, len(cu) - 1, n_heads, n_kv_heads, pp, npairs,
+                                           int(bool(causal)), ctypes.c_float(float(softmax_scale)), _ptr(dq_acc),
+                                           _ptr(dk_acc), _ptr(dv_acc), _ptr(workspace), int(workspace_bytes),
+                                           _stream(stream))
+    if check:
+        _check(s, "hydra_attn_bwd_accumulate_gqa")
     return s
 
 

@@ -755,8 +755,19 @@ int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_
                        float softmax_scale, void* out, float* lse, void* o_part, float* lse_part,
                        int64_t part_rows, void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
+    return hydra_attn_fwd_gqa(q, k, v, cu, n_seqs, n_heads, n_heads, pairs, n_pairs, causal, softmax_scale, out, lse,
+                              o_part, lse_part, part_rows, workspace, workspace_bytes, cuda_stream);
+}
+
+int32_t hydra_attn_fwd_gqa(const void* q, const void* k, const void* v, const int32_t* cu, int32_t n_seqs,
+                           int32_t n_heads, int32_t n_kv_heads, const hydra_pair_t* pairs, int32_t n_pairs,
+                           int32_t causal, float softmax_scale, void* out, float* lse, void* o_part,
+                           float* lse_part, int64_t part_rows, void* workspace, size_t workspace_bytes,
+                           void* cuda_stream)
+{
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
+    if (n_kv_heads < 1 || n_heads % n_kv_heads) return HYDRA_ERR_INVALID_ARG;
     if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return HYDRA_ERR_INVALID_ARG;
     if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
     if (workspace_bytes < kStatusBytes) return HYDRA_ERR_WORKSPACE_TOO_SMALL;
@@ -779,8 +790,8 @@ int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_
     if (plan->n_items == 0) return HYDRA_OK;
     // each CTA of a pair stages 64 kv rows of K (box of 64 rows) and 64 value columns of V
     CUtensorMap mq, mk, mv;
-    if (make_map(&mq, q, pb.T, n_heads, D_QK, TILE) || make_map(&mk, k, pb.T, n_heads, D_QK, SUB) ||
-        make_map(&mv, v, pb.T, n_heads, D_V, TILE))
+    if (make_map(&mq, q, pb.T, n_heads, D_QK, TILE) || make_map(&mk, k, pb.T, n_kv_heads, D_QK, SUB) ||
+        make_map(&mv, v, pb.T, n_kv_heads, D_V, TILE))
         return HYDRA_ERR_CUDA;
     if (int32_t s = reset_status(workspace, stream)) return s;
     FwdParams fp{};
@@ -789,6 +800,7 @@ int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_
     fp.n_items = plan->n_items;
     fp.out = out; fp.lse = lse; fp.o_part = o_part; fp.lse_part = lse_part;
     fp.T = pb.T; fp.part_rows = part_rows; fp.h = n_heads; fp.causal = causal != 0;
+    fp.kv_group = n_heads / n_kv_heads;
     fp.scale_log2 = softmax_scale * 1.4426950408889634f;
     fp.status = static_cast<StatusBlock*>(workspace);
     fp.wait_limit_ns = g_wait_limit_ns.load();
@@ -872,8 +884,8 @@ struct BwdTensors {
 // kernel. dq and dk/dv are bf16 outputs or fp32 accumulators, each by its own flag. `ds` / `ds_room` is
 // where a dS hand-off buffer may go. With `first` false the status block keeps its flags and only the
 // work-queue counters are cleared.
-int32_t bwd_run(const Problem& pb, int32_t causal, float softmax_scale, const BwdTensors& t, bool accumulate_dq,
-                bool accumulate_dkv, void* workspace, uint8_t* ds, size_t ds_room, uint64_t ds_limit, bool first, int sms,
+int32_t bwd_run(const Problem& pb, int32_t n_kv_heads, int32_t causal, float softmax_scale, const BwdTensors& t,
+                bool accumulate_dq, bool accumulate_dkv, void* workspace, uint8_t* ds, size_t ds_room, uint64_t ds_limit, bool first, int sms,
                 cudaStream_t stream)
 {
     const int32_t n_heads = pb.h;
@@ -882,8 +894,8 @@ int32_t bwd_run(const Problem& pb, int32_t causal, float softmax_scale, const Bw
 
     float* dsum = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kStatusBytes);
     CUtensorMap mq, mk, mv, mdo, mq_sub, mdo_sub;
-    if (make_map(&mq, t.q, pb.T, n_heads, D_QK, TILE) || make_map(&mk, t.k, pb.T, n_heads, D_QK, TILE) ||
-        make_map(&mv, t.v, pb.T, n_heads, D_V, TILE) || make_map(&mdo, t.dout, pb.T, n_heads, D_V, TILE) ||
+    if (make_map(&mq, t.q, pb.T, n_heads, D_QK, TILE) || make_map(&mk, t.k, pb.T, n_kv_heads, D_QK, TILE) ||
+        make_map(&mv, t.v, pb.T, n_kv_heads, D_V, TILE) || make_map(&mdo, t.dout, pb.T, n_heads, D_V, TILE) ||
         make_map(&mq_sub, t.q, pb.T, n_heads, D_QK, SUB) || make_map(&mdo_sub, t.dout, pb.T, n_heads, D_V, SUB))
         return HYDRA_ERR_CUDA;
     if (first) {
@@ -900,6 +912,7 @@ int32_t bwd_run(const Problem& pb, int32_t causal, float softmax_scale, const Bw
     bp.pairs = at<PairDev>(*plan, plan->off_pairs);
     bp.lse = t.lse; bp.dsum = dsum; bp.dq = t.dq; bp.dk = t.dk; bp.dv = t.dv;
     bp.T = pb.T; bp.h = n_heads; bp.causal = causal != 0;
+    bp.kv_group = n_heads / n_kv_heads;
     bp.scale = softmax_scale; bp.scale_log2 = softmax_scale * 1.4426950408889634f;
     bp.status = static_cast<StatusBlock*>(workspace);
     bp.wait_limit_ns = g_wait_limit_ns.load();
@@ -1019,10 +1032,13 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
                  const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
                  const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
                  void* dq, void* dk, void* dv, bool accumulate, void* workspace, size_t workspace_bytes,
-                 void* cuda_stream)
+                 void* cuda_stream, int32_t n_kv_heads)
 {
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
+    if (n_kv_heads < 1 || n_heads % n_kv_heads) return HYDRA_ERR_INVALID_ARG;
+    // the query heads of a group add into one dk / dv row: only the accumulating form can do that
+    if (n_kv_heads != n_heads && !accumulate) return HYDRA_ERR_UNSUPPORTED;
     if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return HYDRA_ERR_INVALID_ARG;
     if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
     const size_t need = kStatusBytes + align_up(static_cast<size_t>(pb.T) * n_heads * sizeof(float), 256);
@@ -1067,7 +1083,7 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
                 bool first = true;
                 for (const auto& band : bands) {
                     band_pb.pairs = band;
-                    if (int32_t s = bwd_run(band_pb, causal, softmax_scale, tb, true, false, workspace,
+                    if (int32_t s = bwd_run(band_pb, n_heads, causal, softmax_scale, tb, true, false, workspace,
                                             ws + ds_off + acc_bytes, scratch, scratch, first, sms, stream))
                         return s;
                     first = false;
@@ -1092,7 +1108,7 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
             }
         }
     }
-    return bwd_run(pb, causal, softmax_scale, t, accumulate, accumulate, workspace, ws + ds_off, room,
+    return bwd_run(pb, n_kv_heads, causal, softmax_scale, t, accumulate, accumulate, workspace, ws + ds_off, room,
                    g_ds_limit_bytes.load(), true, sms, stream);
 }
 }  // namespace
@@ -1125,7 +1141,7 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
                        void* cuda_stream)
 {
     return bwd_impl(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, dq, dk,
-                    dv, false, workspace, workspace_bytes, cuda_stream);
+                    dv, false, workspace, workspace_bytes, cuda_stream, n_heads);
 }
 
 int32_t hydra_attn_bwd_accumulate(const void* q, const void* k, const void* v, const void* out,
@@ -1135,7 +1151,18 @@ int32_t hydra_attn_bwd_accumulate(const void* q, const void* k, const void* v, c
                                   void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
     return bwd_impl(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, dq_acc,
-                    dk_acc, dv_acc, true, workspace, workspace_bytes, cuda_stream);
+                    dk_acc, dv_acc, true, workspace, workspace_bytes, cuda_stream, n_heads);
+}
+
+int32_t hydra_attn_bwd_accumulate_gqa(const void* q, const void* k, const void* v, const void* out,
+                                      const float* lse, const void* dout, const int32_t* cu, int32_t n_seqs,
+                                      int32_t n_heads, int32_t n_kv_heads, const hydra_pair_t* pairs,
+                                      int32_t n_pairs, int32_t causal, float softmax_scale, float* dq_acc,
+                                      float* dk_acc, float* dv_acc, void* workspace, size_t workspace_bytes,
+                                      void* cuda_stream)
+{
+    return bwd_impl(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, dq_acc,
+                    dk_acc, dv_acc, true, workspace, workspace_bytes, cuda_stream, n_kv_heads);
 }
 
 int32_t hydra_grad_cast(const float* acc, void* grad, int64_t n_elements, void* cuda_stream)

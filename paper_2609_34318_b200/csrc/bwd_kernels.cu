@@ -328,7 +328,8 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                         ok = wait(B_VEMPTY + slot, (gv / kVSlots) ^ 1u);
                         if (!ok) break;
                         mbar_arrive_expect_tx(bar(B_VFULL + slot), kBox128);
-                        tma_load_3d(smem + kV + slot * kBox128, &map_v, bar(B_VFULL + slot), c * 64, item.head, tok);
+                        tma_load_3d(smem + kV + slot * kBox128, &map_v, bar(B_VFULL + slot), c * 64,
+                                    item.head / p.kv_group, tok);
                     }
                     if (!ok) break;
                     const int st = gk % kKStages;
@@ -338,7 +339,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     for (int c = 0; c < 3; ++c) {
                         mbar_arrive_expect_tx(bar(B_KFULL + st * 3 + c), kBox128);
                         tma_load_3d(smem + kK + st * 3 * kBox128 + c * kBox128, &map_k, bar(B_KFULL + st * 3 + c),
-                                    c * 64, item.head, tok);
+                                    c * 64, item.head / p.kv_group, tok);
                     }
                     if (!popped) { it_ahead = pop_end(kq + 1, raw_next, item_next, first_next); popped = true; }
                 }
@@ -720,10 +721,10 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (lane == 0) {
                 mbar_arrive_expect_tx(bar(B_KVFULL), 5 * kBox128);
                 for (int c = 0; c < 3; ++c)
-                    tma_load_3d(smem + kK + c * kBox128, &map_k, bar(B_KVFULL), c * 64, item.head,
+                    tma_load_3d(smem + kK + c * kBox128, &map_k, bar(B_KVFULL), c * 64, item.head / p.kv_group,
                                 first.k_tok0 + item.r0);
                 for (int c = 0; c < 2; ++c)
-                    tma_load_3d(smem + kV + c * kBox128, &map_v, bar(B_KVFULL), c * 64, item.head,
+                    tma_load_3d(smem + kV + c * kBox128, &map_v, bar(B_KVFULL), c * 64, item.head / p.kv_group,
                                 first.k_tok0 + item.r0);
             }
             for (; si.valid() && ok; si.next(), ++gq) {
@@ -877,8 +878,11 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const int krow = item.r0 + r;              // kv row inside the chunk
             const bool row_valid = krow < first.k_len;
             const int64_t tok = static_cast<int64_t>(first.k_tok0) + krow;
-            const int64_t dk_off = (tok * p.h + item.head) * D_QK + g * 96;
-            const int64_t dv_off = (tok * p.h + item.head) * D_V + g * 64;
+            // with shared KV heads (accumulating form only) the query heads of a group add into one dk / dv row
+            const int64_t kv_heads = p.h / p.kv_group;
+            const int64_t kv_row = tok * kv_heads + item.head / p.kv_group;
+            const int64_t dk_off = kv_row * D_QK + g * 96;
+            const int64_t dv_off = kv_row * D_V + g * 64;
             __nv_bfloat16* dkp = static_cast<__nv_bfloat16*>(p.dk) + dk_off;
             __nv_bfloat16* dvp = static_cast<__nv_bfloat16*>(p.dv) + dv_off;
             float* dkp_acc = static_cast<float*>(p.dk) + dk_off;         // accumulate mode: dk, dv are fp32
@@ -1005,16 +1009,16 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
                         if (is_dk)
-                            add_rows_f32_coalesced(out_slice, lane, dkp_acc + c0 + half * 16, static_cast<int64_t>(p.h) * D_QK,
+                            add_rows_f32_coalesced(out_slice, lane, dkp_acc + c0 + half * 16, kv_heads * D_QK,
                                                    cur + half * 16, p.scale, rows_valid);
                         else
-                            add_rows_f32_coalesced(out_slice, lane, dvp_acc + c0 + half * 16, static_cast<int64_t>(p.h) * D_V,
+                            add_rows_f32_coalesced(out_slice, lane, dvp_acc + c0 + half * 16, kv_heads * D_V,
                                                    cur + half * 16, 1.f, rows_valid);
                     }
                 } else if (is_dk) {
-                    store_rows_bf16_coalesced(out_slice, lane, dkp + c0, static_cast<int64_t>(p.h) * D_QK, cur, p.scale, rows_valid);
+                    store_rows_bf16_coalesced(out_slice, lane, dkp + c0, kv_heads * D_QK, cur, p.scale, rows_valid);
                 } else {
-                    store_rows_bf16_coalesced(out_slice, lane, dvp + c0, static_cast<int64_t>(p.h) * D_V, cur, 1.f, rows_valid);
+                    store_rows_bf16_coalesced(out_slice, lane, dvp + c0, kv_heads * D_V, cur, 1.f, rows_valid);
                 }
             }
         }
@@ -1195,8 +1199,8 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_k,
                 if (lane == 0) {
                     mbar_arrive_expect_tx(bar(B_KFULL + st), 3 * kBox128);
                     for (int c = 0; c < 3; ++c)
-                        tma_load_3d(smem + kK + (st * 3 + c) * kBox128, &map_k, bar(B_KFULL + st), c * 64, item.head,
-                                    ti.cur.k_tok0 + ti.t * TILE);
+                        tma_load_3d(smem + kK + (st * 3 + c) * kBox128, &map_k, bar(B_KFULL + st), c * 64,
+                                    item.head / p.kv_group, ti.cur.k_tok0 + ti.t * TILE);
                 }
             }
         }

@@ -169,7 +169,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     if (leader) mbar_arrive_expect_tx(bar(B_KFULL + slot), 2 * kKStage);
                     for (int c = 0; c < 3; ++c)
                         tma_load_3d_pair(smem + kSmemK + slot * kKStage + c * kHalfBox, &map_k, bar(B_KFULL + slot),
-                                         c * 64, item.head, pr.k_tok0 + j * TILE + rank * 64);
+                                         c * 64, item.head / p.kv_group, pr.k_tok0 + j * TILE + rank * 64);
                 };
                 // The Q buffer of tile B is released by the very last score product of the previous item,
                 // the K stages one and two tiles earlier: ask for the first K tiles before waiting for it.
@@ -197,8 +197,8 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     ok = wait(B_VEMPTY + slot, (gv / kVStages) ^ 1u);
                     if (!ok) break;
                     if (leader) mbar_arrive_expect_tx(bar(B_VFULL + slot), 2 * kVStage);
-                    tma_load_3d_pair(smem + kSmemV + slot * kVStage, &map_v, bar(B_VFULL + slot), rank * 64, item.head,
-                                     pr.k_tok0 + j * TILE);
+                    tma_load_3d_pair(smem + kSmemV + slot * kVStage, &map_v, bar(B_VFULL + slot), rank * 64,
+                                     item.head / p.kv_group, pr.k_tok0 + j * TILE);
                 }
             }
         }

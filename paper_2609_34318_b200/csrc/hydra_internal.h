@@ -126,6 +126,7 @@ struct FwdParams {
     void* out; float* lse; void* o_part; float* lse_part;
     int64_t T; int64_t part_rows;
     int32_t h; int32_t causal;
+    int32_t kv_group;           // query heads per KV head (1: every head has its own K, V)
     float scale_log2;           // softmax_scale * log2(e)
     StatusBlock* status;
     uint64_t wait_limit_ns;
@@ -140,6 +141,7 @@ struct BwdParams {
     void* dq; void* dk; void* dv;   // bf16 [T,h,d], written; or, with accumulate, fp32 [T,h,d], added to
     int64_t T;
     int32_t h; int32_t causal;
+    int32_t kv_group;           // query heads per KV head; k, v, dk, dv have h / kv_group heads
     float scale; float scale_log2;
     int32_t accumulate;
     void* ds;                   // dS hand-off buffer, or null: the query-side kernel recomputes S and dP

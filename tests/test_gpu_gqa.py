@@ -1,0 +1,85 @@
+"""Grouped-query attention (shared KV heads) on the GPU against the oracle: forward, merge of cut sequences,
+and the accumulating backward whose dk / dv rows sum over the query heads of a group. Same tolerances as the
+per-head path."""
+import numpy as np
+import pytest
+
+import hydra_workloads as hw
+import oracle
+from gpu_util import check, pairs_for
+
+pytestmark = pytest.mark.gpu
+DQK, DV = hw.D_QK, hw.D_V
+
+
+@pytest.fixture(params=["hand_off", "recompute"])
+def backward_form(request):
+    import paper_2609_34318_b200 as P
+    P.hydra_set_bwd_scratch_limit(0 if request.param == "recompute" else 4 << 30)
+    yield request.param
+    P.hydra_set_bwd_scratch_limit(4 << 30)
+
+
+def inputs(rng, T, h, h_kv):
+    f = lambda heads, d: hw.f32_to_bf16_bits(rng.standard_normal((T, heads, d)).astype(np.float32))
+    return dict(q=f(h, DQK), k=f(h_kv, DQK), v=f(h_kv, DV), do=f(h, DV))
+
+
+def run_gpu_gqa(x, cu, h, h_kv, lib_pairs, part_rows, causal=True):
+    import torch
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.runner import bits_to_tensor
+    T = int(cu[-1])
+    scale = float(np.float32(1.0 / np.sqrt(np.float32(DQK))))
+    q, k, v, do = (bits_to_tensor(x[n]) for n in ("q", "k", "v", "do"))
+    bf, f32 = torch.bfloat16, torch.float32
+    out = torch.full((T, h, DV), float("nan"), dtype=bf, device="cuda")
+    lse = torch.full((h, T), float("nan"), dtype=f32, device="cuda")
+    o_part = torch.full((max(part_rows, 1), h, DV), float("nan"), dtype=bf, device="cuda")
+    lse_part = torch.full((h, max(part_rows, 1)), float("nan"), dtype=f32, device="cuda")
+    ws = torch.empty(max(P.hydra_workspace_bytes(w, cu, h, lib_pairs) for w in (P.HYDRA_WS_FWD, P.HYDRA_WS_BWD)),
+                     dtype=torch.uint8, device="cuda")
+    has_parts = lib_pairs is not None and bool((lib_pairs["part_row"] >= 0).any())
+    P.hydra_attn_fwd_gqa(q, k, v, cu, h, h_kv, lib_pairs, causal, scale, out, lse,
+                         o_part if has_parts else None, lse_part if has_parts else None, part_rows, ws)
+    if has_parts:
+        P.hydra_lse_merge(o_part, lse_part, part_rows, cu, h, lib_pairs, out, lse, ws)
+    acc = [torch.zeros((T, heads, d), dtype=f32, device="cuda") for heads, d in ((h, DQK), (h_kv, DQK), (h_kv, DV))]
+    P.hydra_attn_bwd_accumulate_gqa(q, k, v, out, lse, do, cu, h, h_kv, lib_pairs, causal, scale, acc[0], acc[1],
+                                    acc[2], ws)
+    grads = [torch.empty(a.shape, dtype=bf, device="cuda") for a in acc]
+    for a, g in zip(acc, grads):
+        P.hydra_grad_cast(a, g)
+    status, detail = P.hydra_poll_status(ws)
+    assert status == 0, (status, detail)
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    return dict(out=f64(out), lse=f64(lse), dq=f64(grads[0]), dk=f64(grads[1]), dv=f64(grads[2]))
+
+
+@pytest.mark.parametrize("lengths,h,h_kv,cp_r", [
+    ([300, 129, 64], 4, 2, 0), ([700], 6, 1, 0), ([640, 200], 8, 2, 2), ([257], 4, 4, 0), ([1, 130, 513], 8, 4, 1)])
+def test_gqa_forward_and_backward_match_the_oracle(backward_form, lengths, h, h_kv, cp_r):
+    cu = hw.cu_seqlens(lengths)
+    x = inputs(np.random.default_rng(11 + h + h_kv), int(cu[-1]), h, h_kv)
+    lib_pairs, rows, ora_pairs = pairs_for(cu, cp_r) if cp_r else (None, 0, None)
+    got = run_gpu_gqa(x, cu, h, h_kv, lib_pairs, rows)
+    scale = np.float32(1.0 / np.sqrt(np.float32(DQK)))
+    out, lse = oracle.attn_fwd_gqa(x["q"], x["k"], x["v"], cu, True, scale)
+    if ora_pairs is None:
+        dq, dk, dv = oracle.attn_bwd_gqa(x["q"], x["k"], x["v"], x["do"], cu, True, scale, out, lse)
+    else:
+        d = oracle.bwd_prep(x["do"], out)
+        dq, dk, dv = oracle.attn_bwd_pairs_gqa(x["q"], x["k"], x["v"], x["do"], cu, ora_pairs, True, scale, lse, d)
+    check(got, dict(out=out, lse=lse, dq=dq, dk=dk, dv=dv), label=f"gqa {lengths} h={h}/{h_kv}: ")
+
+
+def test_gqa_backward_needs_the_accumulating_form_and_valid_head_counts():
+    import torch
+    import paper_2609_34318_b200 as P
+    cu = hw.cu_seqlens([64])
+    t = torch.zeros(64 * 4 * DQK, dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
+    s = P.hydra_attn_fwd_gqa(t, t, t, cu, 4, 3, None, True, 0.07, t, t, None, None, 0, ws, check=False)
+    assert s == P.HYDRA_ERR_INVALID_ARG                                       # 3 does not divide 4
+    s = P.hydra_attn_bwd_accumulate_gqa(t, t, t, t, t, t, cu, 4, 0, None, True, 0.07, t, t, t, ws, check=False)
+    assert s == P.HYDRA_ERR_INVALID_ARG
