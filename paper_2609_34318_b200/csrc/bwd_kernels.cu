@@ -167,7 +167,7 @@ constexpr uint32_t kK = 0;                                   // 3 boxes of 128 r
 constexpr uint32_t kV = kK + 3 * kBox128;                    // 2 boxes of 128 rows, stationary
 constexpr uint32_t kQ = kV + 2 * kBox128;                    // stages x 3 boxes of 64 rows
 constexpr uint32_t kDO = kQ + kStages * 3 * kBox64;          // stages x 2 boxes of 64 rows
-constexpr uint32_t kDsStage = kDO + kStages * 2 * kBox64;    // 8 warps x 2 KB: dS^T on its way to memory
+constexpr uint32_t kDsStage = kDO + kStages * 2 * kBox64;    // 8 warps x 2 KB: dK / dV rows on their way to memory
 constexpr uint32_t kTotal = kDsStage + 8 * 2048;             // 221,184 B
 constexpr uint32_t kTmDK = 0, kTmDV = 192, kTmS = 320, kTmDP = 384, kTmP = 448, kTmDS = 480,
                    kTmCols = 512;
@@ -1044,13 +1044,14 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 // dQ from the dS hand-off buffer
 // =============================================================================================
 // When the key-side kernel has left dS^T in memory, dQ = scale * dS K needs no recomputation of S
-// and dP: per (q tile, kv tile) one product of 128 x 192 x 128, both operands straight from their TMA
-// tiles (dS^T blocks as an MN-major A operand, the K tile as an MN-major B operand). The kernel is
+// and dP: per (q tile, kv tile) one product of 128 x 192 x 128, both operands as they arrive (the dS^T
+// blocks, stored by the key-side kernel in the unswizzled MN-major operand layout, as the A operand; the K
+// tile from its swizzled TMA boxes as an MN-major B operand). The kernel is
 // bound by the stream of dS (2 bytes per 384 FLOP), so it is a plain load -> UMMA -> store pipeline:
 //   warps 0-3  epilogue (thread r = q row r): dQ * scale -> bf16 (or fp32 reductions), rows transposed
 //              through 2 KB of shared memory per warp so that whole 64-byte segments are stored
-//   warp  4    pops work items; TMA producer of dS^T: per kv tile the two blocks of the q tile (32 KB),
-//              ring of three (dS comes from memory)
+//   warp  4    pops work items; producer of dS^T: per kv tile the two adjacent blocks of the q tile as one
+//              untiled 32 KB bulk copy, ring of three (dS comes from memory)
 //   warp  5    UMMA issuer; two accumulators in tensor memory, so the epilogue of one work item
 //              overlaps the products of the next
 //   warp  6    TMA producer of the K tiles (48 KB, ring of two: they come from the L2 cache)
