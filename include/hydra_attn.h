@@ -267,12 +267,26 @@ int32_t hydra_grad_cast(const float* acc, void* grad, int64_t n_elements, void* 
  * (integer division); n_kv_heads must divide n_heads. k device bf16 [T, n_kv_heads, 192], v device bf16
  * [T, n_kv_heads, 128]; everything else as in hydra_attn_fwd / hydra_attn_bwd_accumulate, which are the
  * case n_kv_heads == n_heads.
- * The backward exists in the accumulating form only: dk_acc device fp32 [T, n_kv_heads, 192], dv_acc device
- * fp32 [T, n_kv_heads, 128] receive, per KV head, the SUM over the g query heads that read it (the work
- * items of the g query heads add into the same rows with fp32 reductions, so the order of the g terms, and
- * with it the last bits of dk / dv, may differ from run to run); dq_acc device fp32 [T, n_heads, 192].
- * The caller zeroes the accumulators and rounds them with hydra_grad_cast.
+ * In the backward dk, dv of a KV head are the SUM over the g query heads that read it: the work items of
+ * the g query heads add into the same fp32 rows with reductions, so the order of the g terms, and with it
+ * the last bits of dk / dv, may differ from run to run.
+ *   hydra_attn_bwd_accumulate_gqa  dq_acc device fp32 [T, n_heads, 192], dk_acc device fp32
+ *                                  [T, n_kv_heads, 192], dv_acc device fp32 [T, n_kv_heads, 128]: the
+ *                                  caller zeroes them and rounds them with hydra_grad_cast.
+ *   hydra_attn_bwd_gqa             one shot: dq device bf16 [T, n_heads, 192], dk device bf16
+ *                                  [T, n_kv_heads, 192], dv device bf16 [T, n_kv_heads, 128]. dk and dv are
+ *                                  summed in fp32 in the workspace and rounded once; the workspace must
+ *                                  have hydra_workspace_bytes_gqa(HYDRA_WS_BWD, ...) bytes (the per-head
+ *                                  size plus 4 * (192 + 128) bytes per token and KV head), else
+ *                                  HYDRA_ERR_WORKSPACE_TOO_SMALL. The banded form does not apply.
  */
+size_t hydra_workspace_bytes_gqa(int32_t which, const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
+                                 int32_t n_kv_heads, const hydra_pair_t* pairs, int32_t n_pairs);
+int32_t hydra_attn_bwd_gqa(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                           const void* dout, const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
+                           int32_t n_kv_heads, const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal,
+                           float softmax_scale, void* dq, void* dk, void* dv, void* workspace,
+                           size_t workspace_bytes, void* cuda_stream);
 int32_t hydra_attn_fwd_gqa(const void* q, const void* k, const void* v, const int32_t* cu_seqlens_host,
                            int32_t n_seqs, int32_t n_heads, int32_t n_kv_heads, const hydra_pair_t* pairs,
                            int32_t n_pairs, int32_t causal, float softmax_scale, void* out, float* lse,

@@ -93,9 +93,13 @@ def _load() -> ctypes.CDLL:
     lib.hydra_attn_fwd_gqa.restype = i32
     lib.hydra_attn_fwd_gqa.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, i32, i32, f32, vp, vp, vp, vp, i64,
                                        vp, sz, vp]
+    lib.hydra_workspace_bytes_gqa.restype = sz
+    lib.hydra_workspace_bytes_gqa.argtypes = [i32, vp, i32, i32, i32, vp, i32]
     lib.hydra_attn_bwd_accumulate_gqa.restype = i32
     a = list(lib.hydra_attn_bwd.argtypes)
     lib.hydra_attn_bwd_accumulate_gqa.argtypes = a[:9] + [i32] + a[9:]
+    lib.hydra_attn_bwd_gqa.restype = i32
+    lib.hydra_attn_bwd_gqa.argtypes = a[:9] + [i32] + a[9:]
     lib.hydra_grad_cast.restype = i32
     lib.hydra_grad_cast.argtypes = [vp, vp, i64, vp]
     lib.hydra_poll_status.restype = i32
@@ -124,7 +128,7 @@ EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
            "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc", "hydra_lse_merge_accumulate",
            "hydra_sched_targets", "hydra_sched_cp", "hydra_sched_pack", "hydra_attn_bwd_accumulate",
-           "hydra_grad_cast", "hydra_set_bwd_scratch_limit", "hydra_set_bwd_band_scratch", "hydra_bwd_bands", "hydra_ulysses_pack", "hydra_ulysses_unpack", "hydra_attn_fwd_gqa", "hydra_attn_bwd_accumulate_gqa",
+           "hydra_grad_cast", "hydra_set_bwd_scratch_limit", "hydra_set_bwd_band_scratch", "hydra_bwd_bands", "hydra_ulysses_pack", "hydra_ulysses_unpack", "hydra_attn_fwd_gqa", "hydra_attn_bwd_accumulate_gqa", "hydra_attn_bwd_gqa", "hydra_workspace_bytes_gqa",
            "hydra_poll_clocks")
 KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast", "ulysses")
 
@@ -354,6 +358,29 @@ def hydra_attn_fwd_gqa(q, k, v, cu_seqlens, n_heads: int, n_kv_heads: int, pairs
                                 int(workspace_bytes), _stream(stream))
     if check:
         _check(s, "hydra_attn_fwd_gqa")
+    return s
+
+
+def hydra_workspace_bytes_gqa(which: int, cu_seqlens, n_heads: int, n_kv_heads: int, pairs=None) -> int:
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    return int(_lib.hydra_workspace_bytes_gqa(which, cu.ctypes.data, len(cu) - 1, n_heads, n_kv_heads, pp, npairs))
+
+
+def hydra_attn_bwd_gqa(q, k, v, out, lse, dout, cu_seqlens, n_heads: int, n_kv_heads: int, pairs, causal: bool,
+                       softmax_scale: float, dq, dk, dv, workspace, workspace_bytes: Optional[int] = None,
+                       stream=None, check: bool = True) -> int:
+    """hydra_attn_bwd with shared KV heads: dk, dv (bf16) have n_kv_heads heads."""
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = _lib.hydra_attn_bwd_gqa(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout), cu.ctypes.data,
+                                len(cu) - 1, n_heads, n_kv_heads, pp, npairs, int(bool(causal)),
+                                ctypes.c_float(float(softmax_scale)), _ptr(dq), _ptr(dk), _ptr(dv),
+                                _ptr(workspace), int(workspace_bytes), _stream(stream))
+    if check:
+        _check(s, "hydra_attn_bwd_gqa")
     return s
 
 

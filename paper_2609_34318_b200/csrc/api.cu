@@ -708,6 +708,10 @@ size_t bwd_acc_bytes(const Problem& pb)
 {
     return align_up(static_cast<size_t>(pb.T) * pb.h * D_QK * sizeof(float), 1024);
 }
+size_t bwd_kv_acc_bytes(const Problem& pb, int32_t n_kv_heads)
+{
+    return align_up(static_cast<size_t>(pb.T) * n_kv_heads * (D_QK + D_V) * sizeof(float), 1024);
+}
 size_t bwd_base_bytes(const Problem& pb)
 {
     return align_up(kStatusBytes + align_up(static_cast<size_t>(pb.T) * pb.h * sizeof(float), 256), 1024);
@@ -727,8 +731,20 @@ void hydra_set_bwd_band_scratch(uint64_t bytes) { g_band_bytes.store(bytes); }
 size_t hydra_workspace_bytes(int32_t which, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
                              const hydra_pair_t* pairs, int32_t n_pairs)
 {
+    return hydra_workspace_bytes_gqa(which, cu, n_seqs, n_heads, n_heads, pairs, n_pairs);
+}
+
+size_t hydra_workspace_bytes_gqa(int32_t which, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                                 int32_t n_kv_heads, const hydra_pair_t* pairs, int32_t n_pairs)
+{
     Problem pb;
     if (make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb) != HYDRA_OK) return 0;
+    if (n_kv_heads < 1 || n_heads % n_kv_heads) return 0;
+    if (which == HYDRA_WS_BWD && n_kv_heads != n_heads) {
+        // one-shot grouped-query backward: fp32 dk, dv of the KV heads, then the dS buffer if within the limit
+        const size_t ds = bwd_ds_bytes(ds_layout(pb, 1, nullptr), n_heads, g_ds_limit_bytes.load());
+        return bwd_base_bytes(pb) + bwd_kv_acc_bytes(pb, n_kv_heads) + ds;
+    }
     switch (which) {
         case HYDRA_WS_FWD:
         case HYDRA_WS_MERGE: return kStatusBytes;
@@ -1037,8 +1053,6 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
     if (n_kv_heads < 1 || n_heads % n_kv_heads) return HYDRA_ERR_INVALID_ARG;
-    // the query heads of a group add into one dk / dv row: only the accumulating form can do that
-    if (n_kv_heads != n_heads && !accumulate) return HYDRA_ERR_UNSUPPORTED;
     if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return HYDRA_ERR_INVALID_ARG;
     if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
     const size_t need = kStatusBytes + align_up(static_cast<size_t>(pb.T) * n_heads * sizeof(float), 256);
@@ -1062,6 +1076,38 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     const BwdTensors t{q, k, v, out, dout, lse, dq, dk, dv};
     const size_t room = workspace_bytes > ds_off ? workspace_bytes - ds_off : 0;
+
+    // One-shot grouped-query form: the query heads of a group add into one dk / dv row, which only the
+    // accumulating epilogue can do. dk, dv are summed in fp32 in the workspace and rounded at the end; dq
+    // (one query head per row) is written as bf16 as usual.
+    if (!accumulate && n_kv_heads != n_heads) {
+        const size_t kv_bytes = bwd_kv_acc_bytes(pb, n_kv_heads);
+        if (room < kv_bytes) return HYDRA_ERR_WORKSPACE_TOO_SMALL;
+        float* dk_acc = reinterpret_cast<float*>(ws + ds_off);
+        float* dv_acc = dk_acc + static_cast<size_t>(pb.T) * n_kv_heads * D_QK;
+        if (cudaMemsetAsync(dk_acc, 0, kv_bytes, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+        const BwdTensors tg{q, k, v, out, dout, lse, dq, dk_acc, dv_acc};
+        if (int32_t s = bwd_run(pb, n_kv_heads, causal, softmax_scale, tg, false, true, workspace,
+                                ws + ds_off + kv_bytes, room - kv_bytes, g_ds_limit_bytes.load(), true, sms, stream))
+            return s;
+        std::vector<Range> rs;
+        for (const auto& p : pb.pairs)
+            if (p.q_len > 0 && p.k_len > 0) rs.push_back(Range{p.seq, p.k_start, p.k_len});
+        std::sort(rs.begin(), rs.end(), range_less);
+        for (size_t i = 0; i < rs.size(); ++i) {
+            if (i > 0 && rs[i].seq == rs[i - 1].seq && rs[i].start == rs[i - 1].start) continue;
+            const size_t row = static_cast<size_t>(pb.cu[rs[i].seq]) + rs[i].start;
+            const size_t rk = static_cast<size_t>(n_kv_heads) * D_QK, rv = static_cast<size_t>(n_kv_heads) * D_V;
+            ScopedKernelTimer timer(K_CAST, stream);
+            if (launch_grad_cast(dk_acc + row * rk, static_cast<uint16_t*>(dk) + row * rk,
+                                 static_cast<int64_t>(rs[i].len) * rk, stream) != cudaSuccess ||
+                launch_grad_cast(dv_acc + row * rv, static_cast<uint16_t*>(dv) + row * rv,
+                                 static_cast<int64_t>(rs[i].len) * rv, stream) != cudaSuccess)
+                return HYDRA_ERR_CUDA;
+            g_launches += 2;
+        }
+        return HYDRA_OK;
+    }
 
     // Banded form: the dS buffer of the whole call is over the limit, but the caller has switched the
     // bands on and left room for an fp32 accumulator of dq and a band's scratch. Each band of key rows
@@ -1152,6 +1198,15 @@ int32_t hydra_attn_bwd_accumulate(const void* q, const void* k, const void* v, c
 {
     return bwd_impl(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, dq_acc,
                     dk_acc, dv_acc, true, workspace, workspace_bytes, cuda_stream, n_heads);
+}
+
+int32_t hydra_attn_bwd_gqa(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                           const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads, int32_t n_kv_heads,
+                           const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
+                           void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    return bwd_impl(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, dq, dk,
+                    dv, false, workspace, workspace_bytes, cuda_stream, n_kv_heads);
 }
 
 int32_t hydra_attn_bwd_accumulate_gqa(const void* q, const void* k, const void* v, const void* out,

@@ -73,7 +73,52 @@ def test_gqa_forward_and_backward_match_the_oracle(backward_form, lengths, h, h_
     check(got, dict(out=out, lse=lse, dq=dq, dk=dk, dv=dv), label=f"gqa {lengths} h={h}/{h_kv}: ")
 
 
-def test_gqa_backward_needs_the_accumulating_form_and_valid_head_counts():
+@pytest.mark.parametrize("lengths,h,h_kv,cp_r", [([300, 129, 64], 4, 2, 0), ([640, 200], 8, 1, 2)])
+def test_gqa_one_shot_backward_matches_the_oracle(backward_form, lengths, h, h_kv, cp_r):
+    import torch
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.runner import bits_to_tensor
+    cu = hw.cu_seqlens(lengths)
+    T = int(cu[-1])
+    x = inputs(np.random.default_rng(23), T, h, h_kv)
+    lib_pairs, rows, ora_pairs = pairs_for(cu, cp_r) if cp_r else (None, 0, None)
+    scale = float(np.float32(1.0 / np.sqrt(np.float32(DQK))))
+    q, k, v, do = (bits_to_tensor(x[n]) for n in ("q", "k", "v", "do"))
+    bf = torch.bfloat16
+    out = torch.empty((T, h, DV), dtype=bf, device="cuda")
+    lse = torch.empty((h, T), dtype=torch.float32, device="cuda")
+    o_part = torch.empty((max(rows, 1), h, DV), dtype=bf, device="cuda")
+    lse_part = torch.empty((h, max(rows, 1)), dtype=torch.float32, device="cuda")
+    need = P.hydra_workspace_bytes_gqa(P.HYDRA_WS_BWD, cu, h, h_kv, lib_pairs)
+    assert need >= P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h, lib_pairs) + T * h_kv * (DQK + DV) * 4
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    has_parts = rows > 0
+    P.hydra_attn_fwd_gqa(q, k, v, cu, h, h_kv, lib_pairs, True, scale, out, lse, o_part if has_parts else None,
+                         lse_part if has_parts else None, rows, ws)
+    if has_parts:
+        P.hydra_lse_merge(o_part, lse_part, rows, cu, h, lib_pairs, out, lse, ws)
+    dq = torch.full((T, h, DQK), float("nan"), dtype=bf, device="cuda")
+    dk = torch.full((T, h_kv, DQK), float("nan"), dtype=bf, device="cuda")
+    dv = torch.full((T, h_kv, DV), float("nan"), dtype=bf, device="cuda")
+    small = P.hydra_attn_bwd_gqa(q, k, v, out, lse, do, cu, h, h_kv, lib_pairs, True, scale, dq, dk, dv, ws,
+                                 workspace_bytes=P.hydra_workspace_bytes(P.HYDRA_WS_FWD, cu, h) + T * h * 4 + 4096,
+                                 check=False)
+    assert small == P.HYDRA_ERR_WORKSPACE_TOO_SMALL
+    P.hydra_attn_bwd_gqa(q, k, v, out, lse, do, cu, h, h_kv, lib_pairs, True, scale, dq, dk, dv, ws)
+    status, detail = P.hydra_poll_status(ws)
+    assert status == 0, (status, detail)
+    f64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    o_ref, l_ref = oracle.attn_fwd_gqa(x["q"], x["k"], x["v"], cu, True, np.float32(scale))
+    if ora_pairs is None:
+        ref = oracle.attn_bwd_gqa(x["q"], x["k"], x["v"], x["do"], cu, True, np.float32(scale), o_ref, l_ref)
+    else:
+        d = oracle.bwd_prep(x["do"], o_ref)
+        ref = oracle.attn_bwd_pairs_gqa(x["q"], x["k"], x["v"], x["do"], cu, ora_pairs, True, np.float32(scale), l_ref, d)
+    check(dict(out=f64(out), lse=f64(lse), dq=f64(dq), dk=f64(dk), dv=f64(dv)),
+          dict(out=o_ref, lse=l_ref, dq=ref[0], dk=ref[1], dv=ref[2]), label=f"gqa one-shot {lengths}: ")
+
+
+def test_gqa_entry_points_reject_bad_head_counts():
     import torch
     import paper_2609_34318_b200 as P
     cu = hw.cu_seqlens([64])
