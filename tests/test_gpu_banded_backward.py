@@ -81,3 +81,21 @@ def test_banded_backward_non_causal(banded):
     got = {n: getattr(step, n)[:T].float().cpu().numpy().astype(np.float64) for n in ("out", "dq", "dk", "dv")}
     got["lse"] = step.lse[:, :T].cpu().numpy().astype(np.float64)
     check(got, run_oracle(x, cu, False), label="banded non-causal: ")
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_banded_backward_random_mixes(banded, seed):
+    """Random length mixes and ring degrees with a random scratch between 1 and 3 MiB: whatever the bands
+    turn out to be (or if the problem is small enough to need none), the result is the oracle's."""
+    P = banded
+    rng = np.random.default_rng(500 + seed)
+    n = int(rng.integers(1, 5))
+    lengths = [int(v) for v in rng.choice([65, 128, 200, 383, 640, 777, 1025, 1500], size=n)]
+    cp_r = [int(v) for v in rng.choice([0, 1, 2], size=n)]
+    h = int(rng.integers(1, 4))
+    P.hydra_set_bwd_band_scratch(int(rng.integers(1 << 20, 3 << 20)))
+    cu = hw.cu_seqlens(lengths)
+    x = rand_inputs(rng, int(cu[-1]), h)
+    lib_pairs, rows, ora_pairs = pairs_for(cu, cp_r) if any(cp_r) else (None, 0, None)
+    got = run_gpu(x, cu, h, lib_pairs, rows, True)
+    check(got, run_oracle(x, cu, True, pairs=ora_pairs), label=f"banded mix {lengths} cp_r {cp_r} h {h}: ")

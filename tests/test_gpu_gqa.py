@@ -128,3 +128,25 @@ def test_gqa_entry_points_reject_bad_head_counts():
     assert s == P.HYDRA_ERR_INVALID_ARG                                       # 3 does not divide 4
     s = P.hydra_attn_bwd_accumulate_gqa(t, t, t, t, t, t, cu, 4, 0, None, True, 0.07, t, t, t, ws, check=False)
     assert s == P.HYDRA_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_gqa_random_mixes(backward_form, seed):
+    rng = np.random.default_rng(900 + seed)
+    n = int(rng.integers(1, 5))
+    lengths = [int(v) for v in rng.choice([1, 64, 129, 200, 383, 640, 777], size=n)]
+    cp_r = [int(v) for v in rng.choice([0, 1, 2, 3], size=n)]
+    h_kv = int(rng.integers(1, 3))
+    h = h_kv * int(rng.choice([1, 2, 4]))
+    cu = hw.cu_seqlens(lengths)
+    x = inputs(rng, int(cu[-1]), h, h_kv)
+    lib_pairs, rows, ora_pairs = pairs_for(cu, cp_r) if any(cp_r) else (None, 0, None)
+    got = run_gpu_gqa(x, cu, h, h_kv, lib_pairs, rows)
+    scale = np.float32(1.0 / np.sqrt(np.float32(DQK)))
+    out, lse = oracle.attn_fwd_gqa(x["q"], x["k"], x["v"], cu, True, scale)
+    if ora_pairs is None:
+        dq, dk, dv = oracle.attn_bwd_gqa(x["q"], x["k"], x["v"], x["do"], cu, True, scale, out, lse)
+    else:
+        d = oracle.bwd_prep(x["do"], out)
+        dq, dk, dv = oracle.attn_bwd_pairs_gqa(x["q"], x["k"], x["v"], x["do"], cu, ora_pairs, True, scale, lse, d)
+    check(got, dict(out=out, lse=lse, dq=dq, dk=dk, dv=dv), label=f"gqa mix {lengths} {cp_r} h={h}/{h_kv}: ")
