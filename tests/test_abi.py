@@ -234,3 +234,31 @@ def test_ulysses_pack_validation_without_a_gpu():
     assert P.hydra_ulysses_unpack(0, 8, 4, 8, 2, 0x2000, **args) == P.HYDRA_ERR_INVALID_ARG
     assert P.hydra_ulysses_pack(0x1000, 1 << 34, 64, 192, 4, 0x2000, **args) == P.HYDRA_ERR_UNSUPPORTED
     assert P.hydra_ulysses_pack(0x1000, -1, 4, 8, 2, 0x2000, **args) == P.HYDRA_ERR_INVALID_ARG
+
+
+def test_workspace_bytes_with_the_band_scratch():
+    """Over the dS limit the backward asks for the base size alone, or, with the bands switched on, for the
+    base size + an fp32 dq + the scratch (capped by the full dS buffer)."""
+    cu, h = [0, 20000], 4
+    try:
+        P.hydra_set_bwd_scratch_limit(1 << 30)
+        P.hydra_set_bwd_band_scratch(0)
+        base = P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h)
+        assert 20000 * h * 4 <= base < 20000 * h * 4 + (1 << 16)          # D only: dS (1.6 GB) is over the limit
+        P.hydra_set_bwd_band_scratch(256 << 20)
+        banded = P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h)
+        acc = 20000 * h * 192 * 4
+        assert base + acc + (256 << 20) <= banded <= base + acc + (256 << 20) + 4096
+        P.hydra_set_bwd_band_scratch(64 << 30)                            # more than the whole buffer: capped
+        capped = P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h)
+        full = 20000 * 20000 // 2 * 2 * h
+        assert base + acc + full <= capped <= base + acc + int(full * 1.05) + (1 << 20)
+        P.hydra_set_bwd_scratch_limit(4 << 30)                            # under the limit: the bands play no part
+        assert P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h) <= base + int(full * 1.05) + (1 << 20)
+        # grouped-query form: fp32 dk, dv of the KV heads on top
+        g = P.hydra_workspace_bytes_gqa(P.HYDRA_WS_BWD, cu, h, 2)
+        assert g >= P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h) + 20000 * 2 * (192 + 128) * 4
+        assert P.hydra_workspace_bytes_gqa(P.HYDRA_WS_BWD, cu, h, 3) == 0  # 3 does not divide 4
+    finally:
+        P.hydra_set_bwd_scratch_limit(4 << 30)
+        P.hydra_set_bwd_band_scratch(0)
