@@ -116,10 +116,13 @@ int32_t hydra_zigzag_pairs(const int32_t* cu_seqlens_host, int32_t n_seqs, const
  * which both apply. The size assumes a causal call; a non-causal call needs about twice the buffer
  * and falls back to recomputation in a workspace sized here.
  *
- * Banded form, for problems whose dS buffer is over that limit (long sequences). After
- * hydra_set_bwd_band_scratch(bytes) with bytes >= 1 MiB (default 0: off), HYDRA_WS_BWD asks, for such a
- * problem, for the base size + an fp32 accumulator of dq (4 * 192 bytes per token and head) +
- * min(bytes, the full dS buffer). hydra_attn_bwd, given that much, cuts the key rows of every chunk into
+ * Banded form, for problems whose dS buffer is over that limit (long sequences). The band scratch is set
+ * with hydra_set_bwd_band_scratch(bytes): a byte count >= 1 MiB, 0 (bands off), or HYDRA_BAND_AUTO (the
+ * default): as much as the dS limit, for problems whose whole dS buffer is at most 16 times the limit,
+ * and off for larger ones (hundreds of small bands cost more than the recomputation they save: give
+ * those an explicit scratch of tens of GB). With a scratch in effect HYDRA_WS_BWD asks, for a problem over
+ * the limit, for the base size + an fp32 accumulator of dq (4 * 192 bytes per token and head) +
+ * min(scratch, the full dS buffer). hydra_attn_bwd, given that much, cuts the key rows of every chunk into
  * bands of 128-row tiles whose own dS buffer fits the scratch and runs every band with the hand-off
  * (pairs clipped to the band's keys and, under the causal mask, to the query rows that see them). A key
  * tile lies in one band, so dk and dv come out as in the one-shot form; dq sums the bands' contributions
@@ -127,6 +130,7 @@ int32_t hydra_zigzag_pairs(const int32_t* cu_seqlens_host, int32_t n_seqs, const
  * banded (a single tile column over the scratch, or clipped chunks that would overlap without being
  * identical) runs in the recomputing form instead.
  */
+#define HYDRA_BAND_AUTO (~(uint64_t)0)
 void hydra_set_bwd_scratch_limit(uint64_t bytes);
 void hydra_set_bwd_band_scratch(uint64_t bytes);
 

@@ -427,8 +427,12 @@ def hydra_ulysses_unpack(recv, n_tokens: int, n_heads: int, head_dim: int, cp_u:
     return s
 
 
+HYDRA_BAND_AUTO = (1 << 64) - 1
+
+
 def hydra_set_bwd_band_scratch(n_bytes: int) -> None:
-    """Scratch for the banded backward of problems whose dS buffer is over the limit (0: off)."""
+    """Scratch for the banded backward of problems whose dS buffer is over the limit (0: off;
+    HYDRA_BAND_AUTO, the default: the dS limit, for problems of at most 16 such bands)."""
     _lib.hydra_set_bwd_band_scratch(int(n_bytes))
 
 

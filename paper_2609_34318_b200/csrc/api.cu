@@ -700,9 +700,22 @@ int32_t hydra_zigzag_pairs(const int32_t* cu, int32_t n_seqs, const int32_t* cp_
 namespace {
 std::atomic<uint64_t> g_ds_limit_bytes{uint64_t{4} << 30};
 
-std::atomic<uint64_t> g_band_bytes{0};
 // smallest scratch the banded backward is worth running with
 constexpr uint64_t kMinBandBytes = uint64_t{1} << 20;
+// Band scratch: a byte count, 0 (bands off) or HYDRA_BAND_AUTO: as much as the dS limit, for problems whose
+// whole dS buffer is at most 16 times that (a band boundary costs about as much as 1 / 30 of a 48 GB band,
+// so hundreds of small bands would cost more than the recomputation they save).
+std::atomic<uint64_t> g_band_bytes{HYDRA_BAND_AUTO};
+constexpr uint64_t kAutoBandsMax = 16;
+uint64_t band_scratch_for(int64_t head_blocks, int32_t n_heads)
+{
+    const uint64_t set = g_band_bytes.load();
+    if (set != HYDRA_BAND_AUTO) return set;
+    if (head_blocks <= 0) return 0;
+    const uint64_t limit = g_ds_limit_bytes.load();
+    const uint64_t full = static_cast<uint64_t>(head_blocks) * n_heads * DS_BLOCK_BYTES;
+    return (limit >= kMinBandBytes && full <= kAutoBandsMax * limit) ? limit : 0;
+}
 
 size_t bwd_acc_bytes(const Problem& pb)
 {
@@ -755,7 +768,7 @@ size_t hydra_workspace_bytes_gqa(int32_t which, const int32_t* cu, int32_t n_seq
             const size_t ds = bwd_ds_bytes(head_blocks, n_heads, g_ds_limit_bytes.load());
             if (ds) return base + ds;
             // over the limit: the banded form, if switched on, wants an fp32 dq and its scratch
-            const uint64_t band = g_band_bytes.load();
+            const uint64_t band = band_scratch_for(head_blocks, n_heads);
             if (head_blocks > 0 && band >= kMinBandBytes) {
                 const uint64_t full = static_cast<uint64_t>(head_blocks) * n_heads * DS_BLOCK_BYTES;
                 return base + bwd_acc_bytes(pb) + static_cast<size_t>(std::min(band, full));
@@ -1113,11 +1126,12 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
     // bands on and left room for an fp32 accumulator of dq and a band's scratch. Each band of key rows
     // then runs with its own hand-off: dk and dv of its keys are final, dq is summed in fp32 over the
     // bands and rounded once at the end.
-    const uint64_t band_limit = g_band_bytes.load();
     const size_t acc_bytes = bwd_acc_bytes(pb);
-    if (!accumulate && band_limit >= kMinBandBytes && room >= acc_bytes + kMinBandBytes) {
+    if (!accumulate && room >= acc_bytes + kMinBandBytes) {
         const int64_t head_blocks = ds_layout(pb, causal, nullptr);
-        if (head_blocks > 0 && bwd_ds_bytes(head_blocks, n_heads, g_ds_limit_bytes.load()) == 0) {
+        const uint64_t band_limit = band_scratch_for(head_blocks, n_heads);
+        if (head_blocks > 0 && band_limit >= kMinBandBytes &&
+            bwd_ds_bytes(head_blocks, n_heads, g_ds_limit_bytes.load()) == 0) {
             const size_t scratch = static_cast<size_t>(std::min<uint64_t>(band_limit, room - acc_bytes));
             const auto bands = make_bands(pb, causal, scratch);
             if (!bands.empty()) {

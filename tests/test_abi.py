@@ -253,6 +253,12 @@ def test_workspace_bytes_with_the_band_scratch():
         capped = P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h)
         full = 20000 * 20000 // 2 * 2 * h
         assert base + acc + full <= capped <= base + acc + int(full * 1.05) + (1 << 20)
+        # the default: as much scratch as the dS limit while the whole buffer is at most 16 times the limit
+        P.hydra_set_bwd_band_scratch(P.HYDRA_BAND_AUTO)
+        P.hydra_set_bwd_scratch_limit(256 << 20)                          # 1.6 GB of dS: 7 bands
+        assert P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h) == banded
+        P.hydra_set_bwd_scratch_limit(64 << 20)                           # 25 bands: too many, recompute instead
+        assert P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h) == base
         P.hydra_set_bwd_scratch_limit(4 << 30)                            # under the limit: the bands play no part
         assert P.hydra_workspace_bytes(P.HYDRA_WS_BWD, cu, h) <= base + int(full * 1.05) + (1 << 20)
         # grouped-query form: fp32 dk, dv of the KV heads on top
@@ -261,4 +267,4 @@ def test_workspace_bytes_with_the_band_scratch():
         assert P.hydra_workspace_bytes_gqa(P.HYDRA_WS_BWD, cu, h, 3) == 0  # 3 does not divide 4
     finally:
         P.hydra_set_bwd_scratch_limit(4 << 30)
-        P.hydra_set_bwd_band_scratch(0)
+        P.hydra_set_bwd_band_scratch(P.HYDRA_BAND_AUTO)

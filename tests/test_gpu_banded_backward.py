@@ -25,7 +25,7 @@ def banded():
     P.hydra_set_bwd_band_scratch(1 << 20)
     yield P
     P.hydra_set_bwd_scratch_limit(4 << 30)
-    P.hydra_set_bwd_band_scratch(0)
+    P.hydra_set_bwd_band_scratch(P.HYDRA_BAND_AUTO)
 
 
 @pytest.mark.parametrize("lengths,h,cp_r", [([1000], 2, 0), ([1500], 2, 2), ([700, 130, 64, 900], 2, [1, 0, 0, 2]),

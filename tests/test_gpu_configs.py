@@ -145,7 +145,7 @@ def long_backward_form(request):
     import paper_2609_34318_b200 as P
     P.hydra_set_bwd_band_scratch((48 << 30) if request.param == "banded_48gb" else 0)
     yield request.param
-    P.hydra_set_bwd_band_scratch(0)
+    P.hydra_set_bwd_band_scratch(P.HYDRA_BAND_AUTO)
 
 
 def bands_ran(w, form, launches):
