@@ -162,8 +162,8 @@ hydra_bwd_prep_kernel(const uint4* __restrict__ dout, const uint4* __restrict__ 
 
 // grad (bf16) = acc (fp32), eight elements per thread: two 16-byte loads, one 16-byte store.
 __global__ void __launch_bounds__(kThreads)
-hydra_grad_cast_kernel(const float4* __restrict__ acc, uint4* __restrict__ grad, int64_t n8, int64_t n,
-                       const float* __restrict__ acc_tail, __nv_bfloat16* __restrict__ grad_tail)
+hydra_grad_cast_kernel(const float4* acc, uint4* grad, int64_t n8, int64_t n, const float* acc_tail,
+                       __nv_bfloat16* grad_tail)
 {
     const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
     for (int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; i < n8; i += stride) {
