@@ -268,3 +268,38 @@ def test_workspace_bytes_with_the_band_scratch():
     finally:
         P.hydra_set_bwd_scratch_limit(4 << 30)
         P.hydra_set_bwd_band_scratch(P.HYDRA_BAND_AUTO)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_bands_cover_random_problems_exactly_once(seed):
+    rng = np.random.default_rng(7000 + seed)
+    n = int(rng.integers(1, 5))
+    lengths = [int(v) for v in rng.choice([1, 65, 128, 200, 383, 640, 777, 1025, 1500], size=n)]
+    cp_r = [int(v) for v in rng.choice([0, 1, 2, 3], size=n)]
+    causal = bool(rng.integers(0, 2))
+    h = int(rng.integers(1, 4))
+    scratch = int(rng.integers(1 << 20, 4 << 20))
+    cu = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    pairs = P.hydra_zigzag_pairs(cu, cp_r)[0] if any(cp_r) else None
+    whole = pairs if pairs is not None else np.array(
+        [(b, 0, L, 0, L, -1, b, 0) for b, L in enumerate(lengths)], dtype=P.PAIR_DTYPE)
+    out, band, n_bands = P.hydra_bwd_bands(cu, h, pairs, causal, scratch)
+    if n_bands == 0:                       # a single tile column over the scratch: the caller recomputes
+        assert max(lengths) * 128 * 2 * h * 2 > scratch // 2
+        return
+    cover = [np.zeros((L, L), np.int32) for L in lengths]
+    for p in out:
+        cover[p["seq"]][p["q_start"]:p["q_start"] + p["q_len"], p["k_start"]:p["k_start"] + p["k_len"]] += \
+            _visible(p, causal)
+    want = [np.zeros((L, L), np.int32) for L in lengths]
+    for p in whole:
+        if p["q_len"] > 0 and p["k_len"] > 0:
+            want[p["seq"]][p["q_start"]:p["q_start"] + p["q_len"], p["k_start"]:p["k_start"] + p["k_len"]] += \
+                _visible(p, causal)
+    for c, w in zip(cover, want):
+        assert np.array_equal(c, w)
+    # a key tile of a chunk lies in one band only (dk, dv of a band are final)
+    owner = {}
+    for p, b in zip(out, band):
+        for k0 in range(p["k_start"], p["k_start"] + p["k_len"], 128):
+            assert owner.setdefault((int(p["seq"]), int(k0)), int(b)) == int(b)
