@@ -18,6 +18,7 @@ from .attention import (  # noqa: F401
     p_row,
     sample_keys,
     sample_rows,
+    spike_bwd,
     usp_factor,
     zigzag_chunks,
     zigzag_rank,

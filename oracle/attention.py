@@ -302,3 +302,21 @@ def sample_keys(q, k, v, dout, cu_seqlens, causal: bool, scale: float, tok, head
                               ctypes.c_int(int(causal)), ctypes.c_double(float(np.float32(scale))),
                               ctypes.c_int64(n), _p(tok), _p(head), _p(dk), _p(dvv))
     return dk, dvv
+
+
+def spike_bwd(q, k, v, dout, cu_seqlens, causal: bool, scale: float, tok):
+    """Backward when dO is zero outside the query rows `tok` (all heads of each): returns dQ of those rows
+    [n, h, dqk] and dK [T, h, dqk], dV [T, h, dv] of every key row. The caller passes a dO that is zero
+    elsewhere; only the listed rows are read."""
+    q, k, v, dout, cu = _u16(q), _u16(k), _u16(v), _u16(dout), _cu(cu_seqlens)
+    T, h, dqk = q.shape
+    dv = v.shape[2]
+    assert dqk <= 512 and dv <= 512
+    tok = np.ascontiguousarray(tok, dtype=np.int64)
+    n = len(tok)
+    dq = np.zeros((n, h, dqk)); dk = np.zeros((T, h, dqk)); dvv = np.zeros((T, h, dv))
+    _lib().oracle_spike_bwd(_p(q), _p(k), _p(v), _p(dout), _p(cu), ctypes.c_int(len(cu) - 1), ctypes.c_int(h),
+                            ctypes.c_int(dqk), ctypes.c_int(dv), ctypes.c_int(int(causal)),
+                            ctypes.c_double(float(np.float32(scale))), ctypes.c_int64(n), _p(tok), _p(dq), _p(dk),
+                            _p(dvv))
+    return dq, dk, dvv

@@ -30,7 +30,9 @@
  * Parity pins (tests/test_oracle_*.py): brute-force softmax without max subtraction, closed forms
  * (L = 1, q = 0, constant k, constant v, key shift), row sums of P, gradient invariants, central
  * finite differences, torch float64 scaled_dot_product_attention + autograd, and the identity
- * "merge of the partials of any chunking == unchunked attention".
+ * "merge of the partials of any chunking == unchunked attention". The sampled forms
+ * (oracle_sample_rows with its blocked gathers, oracle_sample_keys, oracle_spike_bwd) are pinned
+ * against the full functions, on sequences longer than two gather blocks.
  */
 #include <math.h>
 #include <stdint.h>
@@ -452,6 +454,79 @@ ORACLE_API void oracle_sample_keys(const uint16_t *q, const uint16_t *k, const u
         }
         free(acck); free(accv);
         free(Q); free(K); free(V); free(G);
+    }
+}
+
+/* ------------------------------------------------------------------------------------------- */
+/* Backward when dO is non-zero on a few query rows only ("spike" rows). dS_ij and P_ij dO_i      */
+/* vanish on every other row, so dK_j and dV_j of ALL key rows, and dQ of the spike rows, follow  */
+/* from one pass per spike row: two-pass softmax of the row, D_i = <dO_i, O_i>, then one loop     */
+/* over the keys j <= i. Cost O(rows * L * d), which makes every key row of the long              */
+/* configurations checkable element by element. The caller guarantees that dO is zero outside     */
+/* the listed tokens (rows of all h heads are treated). dk [T,h,dqk], dvv [T,h,dv] are cleared    */
+/* here; dq_rows is [n_rows,h,dqk].                                                               */
+ORACLE_API void oracle_spike_bwd(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                                 const uint16_t *dout, const int32_t *cu, int n_seqs, int h, int dqk,
+                                 int dv, int causal, double scale, int64_t n_rows, const int64_t *tok,
+                                 double *dq_rows, double *dk, double *dvv)
+{
+    const int64_t T = cu[n_seqs];
+    memset(dk, 0, sizeof(double) * (size_t)T * h * dqk);
+    memset(dvv, 0, sizeof(double) * (size_t)T * h * dv);
+    for (int64_t s = 0; s < n_rows; ++s) {
+        const int64_t t = tok[s];
+        int b = 0;
+        while (b + 1 < n_seqs && cu[b + 1] <= t) ++b;
+        const int64_t t0 = cu[b], L = cu[b + 1] - cu[b], i = t - t0;
+        const int64_t nk = admissible(i, 0, L, causal);
+        for (int a = 0; a < h; ++a) {
+            double *qi = gather_head(q, t, 1, h, a, dqk);
+            double *gi = gather_head(dout, t, 1, h, a, dv);
+            double *sbuf = (double *)malloc(sizeof(double) * (size_t)(nk > 0 ? nk : 1));
+            double *orow = (double *)calloc((size_t)dv, sizeof(double));
+            double *dqrow = dq_rows + (s * h + a) * dqk;
+            for (int e = 0; e < dqk; ++e) dqrow[e] = 0.0;
+            /* pass 1: scores and their maximum */
+            double m = -INFINITY;
+#pragma omp parallel for reduction(max : m) schedule(static)
+            for (int64_t j = 0; j < nk; ++j) {
+                double kj[512];
+                for (int e = 0; e < dqk; ++e) kj[e] = load_in(k, ((t0 + j) * h + a) * (int64_t)dqk + e);
+                sbuf[j] = scale * dot(qi, kj, dqk);
+                if (sbuf[j] > m) m = sbuf[j];
+            }
+            double l = 0.0;
+            for (int64_t j = 0; j < nk; ++j) l += exp(sbuf[j] - m);
+            const double lse_i = (nk > 0) ? m + log(l) : -INFINITY;
+            /* pass 2: O_i, hence D_i */
+            for (int64_t j = 0; j < nk; ++j) {
+                const double p = exp(sbuf[j] - lse_i);
+                for (int e = 0; e < dv; ++e) orow[e] += p * load_in(v, ((t0 + j) * h + a) * (int64_t)dv + e);
+            }
+            const double D = dot(gi, orow, dv);
+            /* pass 3: every key j <= i receives this row's share; key rows are disjoint across j */
+#pragma omp parallel
+            {
+                double *dq_priv = (double *)calloc((size_t)dqk, sizeof(double));
+#pragma omp for schedule(static)
+                for (int64_t j = 0; j < nk; ++j) {
+                    double kj[512], vj[512];
+                    for (int e = 0; e < dqk; ++e) kj[e] = load_in(k, ((t0 + j) * h + a) * (int64_t)dqk + e);
+                    for (int e = 0; e < dv; ++e) vj[e] = load_in(v, ((t0 + j) * h + a) * (int64_t)dv + e);
+                    const double p = exp(sbuf[j] - lse_i);
+                    const double ds = p * (dot(gi, vj, dv) - D);
+                    double *dkj = dk + ((t0 + j) * h + a) * (int64_t)dqk;
+                    double *dvj = dvv + ((t0 + j) * h + a) * (int64_t)dv;
+                    for (int e = 0; e < dqk; ++e) dkj[e] += scale * ds * qi[e];
+                    for (int e = 0; e < dv; ++e) dvj[e] += p * gi[e];
+                    for (int e = 0; e < dqk; ++e) dq_priv[e] += scale * ds * kj[e];
+                }
+#pragma omp critical
+                for (int e = 0; e < dqk; ++e) dqrow[e] += dq_priv[e];
+                free(dq_priv);
+            }
+            free(qi); free(gi); free(sbuf); free(orow);
+        }
     }
 }
 

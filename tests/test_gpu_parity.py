@@ -140,9 +140,42 @@ def test_monotone_scores_exercise_the_running_max(direction):
     ref = run_oracle(x, cu)
     check(got, ref, names=("out", "lse"))
     # One key coordinate is ~100x larger than the rest here, and sum_j dS_ij = 0, so dQ's large
-    # coordinate is a cancelling sum of bf16-rounded dS_ij (2^-9 relative each) times |k_j0| <= 6:
-    # the rounding of the bf16 operand, not the accumulation, sets the error. Gradients get 1e-1.
-    check(got, ref, names=("dq", "dk", "dv"), tol_rel=1e-1)
+    # coordinate is a cancelling sum of dS_ij times |k_j0| <= 6. Any backward that feeds P and dS to the
+    # tensor cores as bf16 operands (the method's precision: bf16 inputs, fp32 accumulation) rounds each
+    # dS_ij by 2^-9 relative before that sum. Shown, not asserted: the same fp64 arithmetic with only P, dS
+    # and the stored O rounded to bf16 (a dense numpy evaluation written here) is what the GPU must match
+    # within the contract's 2e-2; against the unrounded oracle the bound is set from that model's own
+    # distance to the oracle.
+    model = bf16_operand_backward(x, L, float(np.float32(1.0 / np.sqrt(np.float32(DQK)))))
+    for n in ("dq", "dk", "dv"):
+        g, m, r = got[n][:, 0], model[n], ref[n][:, 0]
+        err_model = np.abs(g - m).max() / np.abs(r).max()
+        err_oracle = np.abs(g - r).max() / np.abs(r).max()
+        model_oracle = np.abs(m - r).max() / np.abs(r).max()
+        print(f"monotone {direction:+.0f} {n}: gpu-model {err_model:.2e} gpu-oracle {err_oracle:.2e} "
+              f"model-oracle {model_oracle:.2e}")
+        assert err_model <= TOL_REL, (n, err_model)
+        assert err_oracle <= TOL_REL + 1.5 * model_oracle, (n, err_oracle, model_oracle)
+
+
+def bf16_round(a):
+    return hw.bf16_bits_to_f64(hw.f32_to_bf16_bits(np.asarray(a, dtype=np.float32)))
+
+
+def bf16_operand_backward(x, L, scale):
+    """Single sequence, head 0, causal: fp64 attention backward in which the three quantities a bf16-operand
+    kernel rounds before they reach a product are rounded to bf16 (P for dV, dS for dQ and dK, the stored O in
+    D = <dO, O>); everything else stays fp64. Dense numpy, independent of the oracle's code."""
+    q, k, v, g = (hw.bf16_bits_to_f64(x[n])[:L, 0] for n in ("q", "k", "v", "do"))
+    s = scale * (q @ k.T)
+    s[np.triu_indices(L, 1)] = -np.inf
+    m = s.max(1, keepdims=True)
+    e = np.exp(s - m)
+    p = e / e.sum(1, keepdims=True)
+    o = bf16_round(p @ v)
+    d = (g * o).sum(1, keepdims=True)
+    ds = bf16_round(p * (g @ v.T - d))
+    return dict(dq=scale * ds @ k, dk=scale * ds.T @ q, dv=bf16_round(p).T @ g)
 
 
 def test_large_scores():

@@ -399,3 +399,56 @@ def test_sampled_rows_and_keys_match_full():
     kk, vv = oracle.sample_keys(x["q"], x["k"], x["v"], x["do"], x["cu"], True, SCALE, tok, head)
     np.testing.assert_allclose(kk, dk[tok, head], rtol=1e-10, atol=1e-13)
     np.testing.assert_allclose(vv, dv[tok, head], rtol=1e-10, atol=1e-13)
+
+
+def test_sampled_rows_beyond_two_gather_blocks_match_full():
+    """The sampled-row form gathers keys and values 1024 at a time; rows with more than 1024 and more than
+    2048 visible keys run its block offsets, and rows of a second sequence run its token offsets. The full
+    unchunked oracle (pinned above by brute force, closed forms, finite differences and torch) is the
+    reference."""
+    rng = np.random.default_rng(23)
+    lengths = [2600, 1500]
+    x = make(rng, lengths, 2)
+    out, lse, dq, dk, dv = full(x)
+    tok = np.array([0, 1023, 1024, 1025, 2047, 2048, 2049, 2599, 2600, 2600 + 1023, 2600 + 1024, 2600 + 1499])
+    head = np.array([0, 1, 0, 1, 0, 1, 0, 1, 0, 1, 0, 1])
+    o, l, d, q_ = oracle.sample_rows(x["q"], x["k"], x["v"], x["do"], x["cu"], True, SCALE, tok, head)
+    np.testing.assert_allclose(o, out[tok, head], rtol=1e-11, atol=1e-14)
+    np.testing.assert_allclose(l, lse[head, tok], rtol=1e-13)
+    np.testing.assert_allclose(q_, dq[tok, head], rtol=1e-9, atol=1e-13)
+    np.testing.assert_allclose(d, (hw.bf16_bits_to_f64(x["do"]) * out).sum(-1)[tok, head], rtol=1e-11, atol=1e-14)
+    # a wrong block offset would change every one of these rows by far more than rounding
+    assert np.abs(o[3] - out[tok[3] - 1024, head[3]]).max() > 1e-3
+    kk, vv = oracle.sample_keys(x["q"], x["k"], x["v"], x["do"], x["cu"], True, SCALE, tok[[1, 5, 7, 9]],
+                                head[[1, 5, 7, 9]])
+    np.testing.assert_allclose(kk, dk[tok[[1, 5, 7, 9]], head[[1, 5, 7, 9]]], rtol=1e-9, atol=1e-13)
+    np.testing.assert_allclose(vv, dv[tok[[1, 5, 7, 9]], head[[1, 5, 7, 9]]], rtol=1e-9, atol=1e-13)
+
+
+@pytest.mark.parametrize("lengths,rows", [([300], [0, 1, 149, 150, 299]), ([7, 130, 64], [6, 7, 100, 136, 137, 200]),
+                                          ([1200, 90], [5, 1023, 1024, 1199, 1200, 1289])])
+def test_spike_backward_matches_full_backward_with_sparse_dout(lengths, rows):
+    """With dO zero outside a few query rows the spike form must give the full backward's dK and dV on every
+    key row and its dQ on the spike rows (and the full backward gives dQ = 0 elsewhere)."""
+    rng = np.random.default_rng(29)
+    x = make(rng, lengths, 2)
+    g = x["do"].copy()
+    keep = np.zeros(g.shape[0], dtype=bool)
+    keep[rows] = True
+    g[~keep] = 0
+    x["do"] = g
+    out, lse, dq, dk, dv = full(x)
+    sq, sk, sv = oracle.spike_bwd(x["q"], x["k"], x["v"], x["do"], x["cu"], True, SCALE, np.array(rows))
+    scale_k, scale_v = np.abs(dk).max(), np.abs(dv).max()
+    assert scale_k > 0 and scale_v > 0
+    np.testing.assert_allclose(sk, dk, rtol=1e-9, atol=1e-12 * scale_k)
+    np.testing.assert_allclose(sv, dv, rtol=1e-9, atol=1e-12 * scale_v)
+    np.testing.assert_allclose(sq, dq[rows], rtol=1e-9, atol=1e-12 * np.abs(dq).max())
+    assert np.abs(dq[~keep]).max() == 0.0
+    # non-causal form too (every key of the sequence is visible to a spike row)
+    out2, lse2 = oracle.attn_fwd(x["q"], x["k"], x["v"], x["cu"], False, SCALE)
+    dq2, dk2, dv2 = oracle.attn_bwd(x["q"], x["k"], x["v"], x["do"], x["cu"], False, SCALE, out2, lse2)
+    sq, sk, sv = oracle.spike_bwd(x["q"], x["k"], x["v"], x["do"], x["cu"], False, SCALE, np.array(rows))
+    np.testing.assert_allclose(sk, dk2, rtol=1e-9, atol=1e-12 * np.abs(dk2).max())
+    np.testing.assert_allclose(sv, dv2, rtol=1e-9, atol=1e-12 * np.abs(dv2).max())
+    np.testing.assert_allclose(sq, dq2[rows], rtol=1e-9, atol=1e-12 * np.abs(dq2).max())
