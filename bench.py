@@ -203,6 +203,90 @@ def whole_job_value(world: int, flops_per_rank_step: float, steps: int, max_ms: 
     return world * flops_per_rank_step * steps / (max_ms * 1e-3) / 1e12
 
 
+def measure_secondary(args, name: str, steps: int, peaks, peak_kind):
+    """The other configuration the target is quoted on (the 256K sequence cut for a ring of four), timed the
+    same way on the same GPU right after the headline workload: a few steps of forward of the 36 chunk pairs,
+    merge and (banded) backward. Its inputs are seeded N(0,1) bf16 drawn on the device (the numpy recipe of the
+    parity tests takes minutes at this size; the timing does not depend on the values)."""
+    import torch
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.runner import AttnStep
+
+    w = hw.workload(name)
+    cu = w.cu()
+    pairs, part_rows = (None, 0)
+    if w.cp_r:
+        pairs, part_rows, _, _ = P.hydra_zigzag_pairs(cu, w.cp_r)
+    torch.cuda.reset_peak_memory_stats()
+    held0 = torch.cuda.memory_allocated()
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(hw.SEED)
+    t = {n: torch.randn((w.total, w.n_heads, hw.D_V if n in ("v", "do") else hw.D_QK), generator=gen,
+                        device="cuda", dtype=torch.float32).to(torch.bfloat16) for n in ("q", "k", "v", "do")}
+    step = AttnStep(cu, w.n_heads, pairs, part_rows, True, float(w.scale))
+    stream = torch.cuda.current_stream()
+
+    def one_step():
+        step.forward(t["q"], t["k"], t["v"])
+        step.backward(t["q"], t["k"], t["v"], t["do"])
+
+    warm = 3
+    for _ in range(warm):
+        one_step()
+    status, detail = step.poll()
+    if status != 0:
+        raise RuntimeError(f"{name}: device status {status} at item {detail}")
+    sampler = ClockSampler(torch.cuda.current_device())
+    P.hydra_profile_enable(True)
+    P.hydra_profile_collect()
+    torch.cuda.synchronize()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        one_step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    total_ms = e0.elapsed_time(e1)
+    kernel_ms, kernel_n = P.hydra_profile_collect()
+    P.hydra_profile_enable(False)
+    status, detail = step.poll()
+    if status != 0:
+        raise RuntimeError(f"{name}: device status {status} at item {detail}")
+    step.forward(t["q"], t["k"], t["v"])
+    mhz_fwd = P.hydra_poll_clocks(step.workspace)[0]
+    step.backward(t["q"], t["k"], t["v"], t["do"])
+    _, mhz_dkv, mhz_dq = P.hydra_poll_clocks(step.workspace)
+    clocks["in_kernel_mhz"] = {"fwd": round(mhz_fwd), "bwd_dkv": round(mhz_dkv), "bwd_dq": round(mhz_dq)}
+    held = torch.cuda.max_memory_allocated() - held0
+    value = 3.5 * w.flops_fwd() * steps / (total_ms * 1e-3) / 1e12
+    dominant = max(kernel_ms, key=lambda k: kernel_ms[k])
+    work = FLOPS_PER_PAIR[dominant] * w.causal_pairs_total * w.n_heads if dominant in FLOPS_PER_PAIR else 0.0
+    # the steps are seconds long and follow each other without a pause: the power-capped (sustained) peak
+    peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    achieved = work / (kernel_ms[dominant] / steps * 1e-3) / 1e12
+    merge_bytes = sum((int(n) + 1) * 260.0 * r * w.n_heads for n, r in merge_groups(pairs))
+    merge_ms = kernel_ms.get("merge", 0.0) / steps
+    out = {"workload": name, "value": value, "unit": UNIT, "steps": steps, "warmup": warm,
+           "ms_per_step": total_ms / steps,
+           "kernel_ms_per_step": {k: v / steps for k, v in kernel_ms.items()},
+           "frac_of_bf16_peak": {"measured_burst": value / peaks["bf16_tflops"], "measured_sustained": value / peak},
+           "roofline": {"kernel": dominant, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                        "peak_kind": f"{peak_kind} sustained bf16", "frac": achieved / peak,
+                        "launches_per_step": kernel_n[dominant] / steps},
+           "merge_gbs": merge_bytes / (merge_ms * 1e-3) / 1e9 if merge_ms > 0 else None,
+           "bwd_bands": int(round(kernel_n.get("bwd_dkv", 0) / steps)), "band_scratch_gb": args.band_scratch_gb,
+           "device_bytes_held": int(held), "clocks": clocks,
+           "config": {"tokens": w.total, "heads": w.n_heads, "pairs": 0 if pairs is None else int(len(pairs)),
+                      "causal_pairs": w.causal_pairs_total, "note": w.note,
+                      "inputs": "seeded N(0,1) bf16 drawn on the device",
+                      "l2": "inputs larger than L2 (no flush between iterations)"}}
+    del step, t
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
@@ -345,9 +429,20 @@ def run_ours(args, w):
         roof = {"kernel": dominant, "bound": "hbm", "achieved": work / (per_launch_ms * 1e-3) / 1e9,
                 "peak": peaks["hbm_gbs"], "unit": "GB/s", "peak_kind": f"{peak_kind} copy"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = recorded_traffic(dominant, w.name)
+    roof["traffic"], roof["traffic_source"] = recorded_traffic(dominant, w.name)
     roof["ms_per_launch"] = per_launch_ms / launches_per_step
     roof["launches_per_step"] = launches_per_step
+
+    # ---- the second configuration of the target (N = 1 only): a few steps of the 256K ring workload ----
+    secondary = None
+    if world == 1 and args.secondary and args.secondary != w.name:
+        if args.no_e2e:
+            del step
+        else:
+            del arena
+        t.clear()
+        torch.cuda.empty_cache()
+        secondary = measure_secondary(args, args.secondary, args.secondary_steps, peaks, peak_kind)
 
     # ---- CPU baseline: the oracle on a bounded sample, rank 0, N = 1 only ----
     cpu = None
@@ -371,7 +466,7 @@ def run_ours(args, w):
             "frac_of_bf16_peak": value / world / peaks["bf16_tflops"],
             "kernel_ms_per_step": {k: v / args.steps for k, v in kernel_ms.items()},
             "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
-            "clocks": clocks}
+            "clocks": clocks, "secondary": secondary}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -614,20 +709,35 @@ def merge_groups(pairs):
     return out
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised in
-# profiles/tensor_kernels_packed32k.md and profiles/merge_prep_short64k_split.md.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from ncu captures of this kernel on this workload
+# (summaries with the full commands are kept with the other profiler summaries). Each figure carries the
+# hash of the kernel sources it was captured from: when a source has changed since, the figure is no longer
+# printed (traffic = null) instead of being repeated for a kernel it does not describe.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "fwd:packed32k": 686360000,
-    "bwd_dkv:packed32k": 2809982000,      # with the dS hand-off: 1.76 GB of it is dS written once
-    "bwd_dq:packed32k": 2072652000,       # hydra_bwd_dq_from_ds_kernel: 1.76 GB of it is dS read once
-    "merge:short64k_split": 764355784,
-    "bwd_prep:short64k_split": 1080946776,
+    # (kernel, workload): (bytes per launch, source files, their hash at capture time, capture date)
 }
 
 
+def kernel_source_hash(files) -> str:
+    import hashlib
+    h = hashlib.sha1()
+    for name in files:
+        with open(os.path.join(ROOT, "paper_2609_34318_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
+
+
 def recorded_traffic(kernel: str, workload: str):
-    """DRAM bytes per launch from the ncu capture of this kernel and workload (None if not captured)."""
-    return NCU_DRAM_BYTES_PER_LAUNCH.get(f"{kernel}:{workload}")
+    """(DRAM bytes per launch, where the figure comes from) for this kernel and workload; (None, why) if it was
+    not captured or the kernel's sources have changed since the capture."""
+    rec = NCU_DRAM_BYTES_PER_LAUNCH.get((kernel, workload))
+    if rec is None:
+        return None, "no ncu capture of this kernel on this workload"
+    nbytes, files, src_hash, date = rec
+    now = kernel_source_hash(files)
+    if now != src_hash:
+        return None, f"stale: ncu capture of {date} was of sources {src_hash}, the kernel is now {now}"
+    return nbytes, f"ncu capture of {date}, kernel sources {src_hash} (dram__bytes_read.sum + dram__bytes_write.sum, one launch)"
 
 
 def main():
@@ -639,6 +749,9 @@ def main():
     ap.add_argument("--workload", default="packed32k", choices=list(hw.WORKLOADS))
     ap.add_argument("--band-scratch-gb", type=float, default=48.0,
                     help="dS scratch of the banded backward (long sequences only); 0 switches the bands off")
+    ap.add_argument("--secondary", default="ring256k",
+                    help="second workload timed after the headline one at N = 1 ('' = none)")
+    ap.add_argument("--secondary-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--report", action="store_true", help="per-kernel report of the workload instead of the bench line")

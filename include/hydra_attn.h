@@ -180,9 +180,8 @@ int32_t hydra_lse_merge(const void* o_part, const float* lse_part, int64_t part_
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * The same merge in the streaming form a ring engine uses (Section 5.2: the outer ring pipelines
- * with attention as in standard ring context parallelism): after every ring step the partials of
- * that step are folded into the running (out, lse) of their q chunks,
+ * The same merge in its streaming form, one ring step at a time (Section 5.2, outer ring): after
+ * every ring step the partials of that step are folded into the running (out, lse) of their q chunks,
  *   (out, lse) <- (out, lse) (+) partial_1 (+) ... (+) partial_n,
  * where (+) is the two-way form of the merge above; rows of out / lse that belong to no listed
  * group are left untouched. The first step of a chunk uses hydra_lse_merge (which accepts groups
@@ -209,10 +208,17 @@ int32_t hydra_lse_merge_accumulate(const void* o_part, const float* lse_part, in
  *     the library, until the process exits.
  *   - The first call on a device looks up the array's device address with that device current; make
  *     that first call before any stream capture begins.
+ *   - No call may be made while `cuda_stream` is capturing: the tables travel from static host arrays
+ *     that the next call overwrites, which a captured copy would read again at every replay. Such a
+ *     call is refused with HYDRA_ERR_UNSUPPORTED before anything is touched.
  *   - All calls on a device share the one array and each call rewrites the part it uses: calls
  *     enqueued on the same stream are safe, calls whose kernels may overlap on the GPU (different
  *     streams, no dependency) race. The tables are copied from ordinary host memory, so the call
- *     waits for earlier work on `cuda_stream` before it returns.
+ *     waits for earlier work on `cuda_stream` before it returns; the host-side tables are one set
+ *     per process behind one lock, so calls from several threads (also for different GPUs) take
+ *     turns, each holding the lock through that wait.
+ *   - As hydra_lse_merge, it refuses (HYDRA_ERR_INVALID_ARG) partial rows that overlap and merged q
+ *     chunks whose output rows overlap.
  *   Arguments as for hydra_lse_merge (pairs with part_row == -1 are ignored).
  */
 #define HYDRA_NOALLOC_MAX_GROUPS 2048
@@ -241,18 +247,19 @@ int32_t hydra_attn_bwd(const void* q, const void* k, const void* v, const void* 
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * The backward of one ring step (Section 5.2: the outer ring pipelines with attention as in
- * standard ring context parallelism, so a rank sees its chunk pairs a step at a time): the same
- * computation as hydra_attn_bwd for the listed pairs, but the contributions are ADDED to fp32
+ * The backward of one ring step (Section 5.2, outer ring: a rank meets its chunk pairs a step at a
+ * time, as the visiting K/V chunks arrive): the same computation as hydra_attn_bwd for the listed pairs, but the contributions are ADDED to fp32
  * accumulators instead of being written as bf16, so that calls for the successive steps sum to the
  * backward of all pairs. The paper does not print this form; it is what its ring engine needs from
  * the attention library.
  *   dq_acc, dk_acc  device fp32 [T, h, 192]; dv_acc device fp32 [T, h, 128]; the caller zeroes them
  *                   (or loads them with gradients that arrived from a peer) before the first step.
  *   out, lse        the MERGED forward result of all steps, as for hydra_attn_bwd.
- * Rows covered by no listed chunk are left untouched. Each accumulator row is owned by one thread
- * block per call and calls on one stream are ordered, so no atomics are used and the result of a
- * fixed sequence of calls is deterministic. Calls that share accumulators must be enqueued on one
+ * Rows covered by no listed chunk are left untouched. The additions are fp32 reductions performed at
+ * the L2 cache (red.global.add). Each accumulator address receives exactly one addition per call
+ * (one thread block owns the row) and calls on one stream are ordered, so the result of a fixed
+ * sequence of per-head calls does not depend on timing. (The grouped-query form is the exception:
+ * the query heads of a group add into the same dk / dv rows in no fixed order.) Calls that share accumulators must be enqueued on one
  * stream (or ordered by the caller). Workspace, requirements and errors as for hydra_attn_bwd.
  * hydra_grad_cast converts an accumulator to the bf16 gradient: grad[i] = bf16(acc[i]), i <
  * n_elements (round to nearest even); acc, grad device pointers, 16-byte aligned.
@@ -328,7 +335,7 @@ int32_t hydra_attn_fwd_bwd_host(const void* q_host, const void* k_host, const vo
                                 size_t arena_bytes, void* cuda_stream);
 
 /*
- * The local halves of the Ulysses all-to-all (Section 3.3: all-to-all transposes partition the attention
+ * The local halves of the Ulysses all-to-all (Section 3.5: all-to-all transposes partition the attention
  * heads across the cp_u ranks of a group; Eq. (ulysses) counts the volume, about 4 S h / P elements per
  * rank for q, k, v and the output). Elements are 2 bytes wide (bf16) and are moved, not interpreted.
  *   hydra_ulysses_pack    x device [n_tokens, n_heads, head_dim] (this rank's tokens, all heads)

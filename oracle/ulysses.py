@@ -1,4 +1,4 @@
-"""Oracle of the local halves of the Ulysses all-to-all (Section 3.3: the all-to-all transposes that
+"""Oracle of the local halves of the Ulysses all-to-all (Section 3.5: the all-to-all transposes that
 partition the attention heads across the ranks of a group; Eq. (ulysses) counts their volume).
 
 TEST INFRASTRUCTURE ONLY. Nothing in the product path imports this module.

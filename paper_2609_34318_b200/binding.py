@@ -514,7 +514,9 @@ def hydra_lse_merge_noalloc(o_part, lse_part, part_rows: int, cu_seqlens, n_head
     """The merge for callers that must not allocate device memory (own memory pool, no-cudaMalloc
     loops): same result as hydra_lse_merge, tables kept in a fixed array inside the library, no
     workspace. Size limits apply (HYDRA_ERR_UNSUPPORTED beyond them); calls that may overlap on the
-    GPU race on that array; make the first call on a device before any stream capture."""
+    GPU race on that array; make the first call on a device before any stream capture, and never call
+    it on a stream that is capturing (refused with HYDRA_ERR_UNSUPPORTED: the tables travel from host
+    arrays the next call overwrites). Host-side table building is serialised per process."""
     cu = _cu(cu_seqlens)
     pp, npairs, _keep = _pairs_arg(pairs)
     s = _lib.hydra_lse_merge_noalloc(_ptr(o_part), _ptr(lse_part), int(part_rows), cu.ctypes.data, len(cu) - 1,

@@ -571,6 +571,17 @@ int32_t reset_status(void* workspace, cudaStream_t s)
 }
 
 }  // namespace
+
+cudaError_t launch_merge_counted(const MergeParams& p, cudaStream_t stream)
+{
+    cudaError_t e;
+    {
+        ScopedKernelTimer timer(K_MERGE, stream);
+        e = launch_merge(p, stream);
+    }
+    if (e == cudaSuccess && p.n_items > 0) g_launches += 1;
+    return e;
+}
 }  // namespace hydra
 
 using namespace hydra;
@@ -893,11 +904,7 @@ int32_t merge_impl(const void* o_part, const float* lse_part, int64_t part_rows,
     mp.o_part = o_part; mp.lse_part = lse_part; mp.out = out; mp.lse = lse;
     mp.T = pb.T; mp.part_rows = part_rows; mp.h = n_heads;
     mp.accumulate = accumulate;
-    {
-        ScopedKernelTimer timer(K_MERGE, stream);
-        if (launch_merge(mp, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
-    }
-    g_launches += 1;
+    if (launch_merge_counted(mp, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
     return HYDRA_OK;
 }
 }  // namespace

@@ -6,7 +6,9 @@
 // Both move every byte once with 16-byte accesses: 16 lanes own one (row, head) vector of 128 bf16.
 #include <cuda_bf16.h>
 
+#include <algorithm>
 #include <mutex>
+#include <utility>
 
 #include "hydra_internal.h"
 
@@ -336,6 +338,7 @@ extern "C" int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_
     static MergeGroup groups[kNoAllocMaxGroups];
     static int32_t parts[kNoAllocMaxParts];
     static MergeItem items[kNoAllocMaxItems];
+    static std::pair<int64_t, int64_t> part_iv[kNoAllocMaxParts], out_iv[kNoAllocMaxGroups];   // [first, end) rows
     int n_groups = 0, n_parts = 0, n_items = 0;
     for (int i = 0; i < n_pairs;) {
         int j = i;
@@ -358,12 +361,14 @@ extern "C" int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_
                     int64_t{q.part_row} + q.q_len > part_rows)
                     return HYDRA_ERR_INVALID_ARG;
                 if (n_parts >= kNoAllocMaxParts) return HYDRA_ERR_UNSUPPORTED;
+                part_iv[n_parts] = {q.part_row, int64_t{q.part_row} + q.q_len};
                 parts[n_parts++] = q.part_row;
             }
             for (int32_t r = 0; r < g.rows; r += MERGE_ROWS) {
                 if (n_items >= kNoAllocMaxItems) return HYDRA_ERR_UNSUPPORTED;
                 items[n_items++] = MergeItem{n_groups, r};
             }
+            out_iv[n_groups] = {g.out_tok0, int64_t{g.out_tok0} + g.rows};
             groups[n_groups++] = g;
         } else {
             for (int t = i; t < j; ++t)
@@ -372,6 +377,14 @@ extern "C" int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_
         i = j;
     }
     if (n_items == 0) return HYDRA_OK;
+    // as in hydra_lse_merge: the partials may not share rows of the partial buffers, and two merged q
+    // chunks may not write the same rows of out / lse (std::sort works in place: no heap)
+    std::sort(part_iv, part_iv + n_parts);
+    for (int i = 1; i < n_parts; ++i)
+        if (part_iv[i].first < part_iv[i - 1].second) return HYDRA_ERR_INVALID_ARG;
+    std::sort(out_iv, out_iv + n_groups);
+    for (int i = 1; i < n_groups; ++i)
+        if (out_iv[i].first < out_iv[i - 1].second) return HYDRA_ERR_INVALID_ARG;
 
     int major = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -381,6 +394,11 @@ extern "C" int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_
     unsigned char* tables = nullptr;
     if (noalloc_tables(&tables) != cudaSuccess) return HYDRA_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // The tables below travel from static host arrays that the next call overwrites: a captured copy would
+    // read them again at every replay of the graph, so a capturing stream is refused before anything moves.
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &capturing) != cudaSuccess) return HYDRA_ERR_CUDA;
+    if (capturing != cudaStreamCaptureStatusNone) return HYDRA_ERR_UNSUPPORTED;
     // Every entry the kernel reads is overwritten here, so nothing of the previous call survives.
     if (cudaMemcpyAsync(tables, groups, sizeof(MergeGroup) * n_groups, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
         cudaMemcpyAsync(tables + kNoAllocGroupsBytes, parts, sizeof(int32_t) * n_parts, cudaMemcpyHostToDevice,
@@ -395,6 +413,6 @@ extern "C" int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_
     mp.n_items = n_items;
     mp.o_part = o_part; mp.lse_part = lse_part; mp.out = out; mp.lse = lse;
     mp.T = cu[n_seqs]; mp.part_rows = part_rows; mp.h = n_heads;
-    hydra_lse_merge_kernel<false><<<n_items, kThreads, 0, stream>>>(mp);
-    return cudaGetLastError() == cudaSuccess ? HYDRA_OK : HYDRA_ERR_CUDA;
+    // counted and timed like every other merge launch (hydra_launch_count, hydra_profile_collect)
+    return launch_merge_counted(mp, stream) == cudaSuccess ? HYDRA_OK : HYDRA_ERR_CUDA;
 }

@@ -1319,17 +1319,27 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_k,
     if (warp == 5) tmem_dealloc(tm, kTmCols);
 }
 
+
+// cudaFuncSetAttribute applies to the device that is current when it is called, so the opt-in to more than
+// 48 KB of dynamic shared memory is made once per device ordinal, not once per process.
+template <class Kernel>
+cudaError_t configure_once_per_device(Kernel kernel, size_t smem_bytes, bool (&done)[64])
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (done[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_bytes));
+    if (e == cudaSuccess) done[dev] = true;
+    return e;
+}
+
 cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mk, const BwdParams& p, int grid,
                                   cudaStream_t stream)
 {
-    static bool configured = false;
-    if (!configured) {
-        const cudaError_t e = cudaFuncSetAttribute(hydra_bwd_dq_from_ds_kernel,
-                                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   static_cast<int>(bwd_dq_ds_smem_bytes()));
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static bool configured[64] = {};
+    if (cudaError_t e = configure_once_per_device(hydra_bwd_dq_from_ds_kernel, bwd_dq_ds_smem_bytes(), configured)) return e;
     hydra_bwd_dq_from_ds_kernel<<<grid, dqs::kThreadsS, bwd_dq_ds_smem_bytes(), stream>>>(mk, p);
     return cudaGetLastError();
 }
@@ -1337,13 +1347,8 @@ cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mk, const BwdParams& p, int
 cudaError_t launch_bwd_dq(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                           const CUtensorMap& mdo, const BwdParams& p, int grid, cudaStream_t stream)
 {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(hydra_bwd_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(bwd_dq_smem_bytes()));
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static bool configured[64] = {};
+    if (cudaError_t e = configure_once_per_device(hydra_bwd_dq_kernel, bwd_dq_smem_bytes(), configured)) return e;
     hydra_bwd_dq_kernel<<<grid, kThreads, bwd_dq_smem_bytes(), stream>>>(mq, mk, mv, mdo, p);
     return cudaGetLastError();
 }
@@ -1351,13 +1356,8 @@ cudaError_t launch_bwd_dq(const CUtensorMap& mq, const CUtensorMap& mk, const CU
 cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, const CUtensorMap& mv,
                            const CUtensorMap& mdo_sub, const BwdParams& p, int grid, cudaStream_t stream)
 {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(hydra_bwd_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(bwd_dkv_smem_bytes()));
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static bool configured[64] = {};
+    if (cudaError_t e = configure_once_per_device(hydra_bwd_dkv_kernel, bwd_dkv_smem_bytes(), configured)) return e;
     hydra_bwd_dkv_kernel<<<grid, kThreads, bwd_dkv_smem_bytes(), stream>>>(mq_sub, mk, mv, mdo_sub, p);
     return cudaGetLastError();
 }

@@ -480,15 +480,17 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 }
 
 // Number of CTA pairs that can be resident at once (one CTA per SM): the size of the persistent grid.
+// Kept per device ordinal: the shared-memory opt-in applies to the device that is current when it is made.
 int fwd_max_clusters()
 {
-    static int cached = -1;
-    if (cached >= 0) return cached;
+    static int cached_by_device[64];
+    static bool known[64] = {};
+    int sms = 0, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (known[dev]) return cached_by_device[dev];
     if (cudaFuncSetAttribute(hydra_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(fwd_smem_bytes())) != cudaSuccess)
         return 0;
-    int sms = 0, dev = 0;
-    cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(sms / 2 * 2));
@@ -496,7 +498,8 @@ int fwd_max_clusters()
     cfg.dynamicSmemBytes = fwd_smem_bytes();
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, hydra_fwd_kernel, &cfg) != cudaSuccess) n = 0;
-    cached = n;
+    cached_by_device[dev] = n;
+    known[dev] = n > 0;
     return n;
 }
 

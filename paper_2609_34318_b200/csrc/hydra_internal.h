@@ -177,6 +177,8 @@ cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mk, const BwdParams& p, int
 cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, const CUtensorMap& mv,
                            const CUtensorMap& mdo_sub, const BwdParams& p, int grid, cudaStream_t stream);
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
+// launch_merge plus the library's launch counter and per-kernel timer (defined beside them, in api.cu)
+cudaError_t launch_merge_counted(const MergeParams& p, cudaStream_t stream);
 cudaError_t launch_grad_cast(const float* acc, void* grad, int64_t n, cudaStream_t stream);
 cudaError_t launch_ulysses(bool pack, const void* src, void* dst, int64_t n_tokens, int32_t cp_u, int64_t chunk_units,
                            cudaStream_t stream);

@@ -214,7 +214,8 @@ int32_t hydra_sched_pack(const int64_t* lengths, int32_t n, int32_t G, int64_t B
             lightest.push(RankLoad{g.load_n, g.size, g.opened, gid, g.version});
             if (rank_load_less(max_load_n, max_size, g.load_n, g.size)) { max_load_n = g.load_n; max_size = g.size; }
             ++pos;
-            // "k has shrunk and MB balanced"
+            // early-close test of Algorithm 1, Phase 2: the next document needs a smaller degree, no rank is
+            // free, and the micro-batch is balanced
             if (pos < n && free_ranks == 0 && cp_degree(lengths[order[pos]], s_max, C, B) < k) {
                 while (lightest.top().version != groups[lightest.top().gid].version) lightest.pop();
                 const RankLoad lo = lightest.top();

@@ -21,7 +21,8 @@ def run_bench(*args):
 
 
 def test_our_arm_prints_the_whole_contract():
-    d = run_bench("--workload", "tiny_split", "--steps", "4", "--warmup", "3")
+    d = run_bench("--workload", "tiny_split", "--steps", "4", "--warmup", "3", "--secondary", "tiny",
+                  "--secondary-steps", "2")
     for k in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
               "vs_baseline", "dtype", "data", "config", "roofline", "cpu_baseline", "e2e", "gpu_launches", "clocks"):
         assert k in d, k
@@ -30,7 +31,7 @@ def test_our_arm_prints_the_whole_contract():
     assert d["scaling"] == "weak" and d["vs_baseline"] is None
     assert d["config"]["workload"] == "tiny_split" and "model" not in d["config"]
     r = d["roofline"]
-    for k in ("bound", "achieved", "peak", "unit", "frac", "traffic"):
+    for k in ("bound", "achieved", "peak", "unit", "frac", "traffic", "traffic_source"):
         assert k in r, k
     assert r["bound"] in ("hbm", "tensor", "alu") and r["peak"] > 0
     assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
@@ -42,6 +43,12 @@ def test_our_arm_prints_the_whole_contract():
     # per step: forward, merge, D-prep and the two backward kernels
     assert d["gpu_launches"] == 5 * d["steps"]
     assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(d["clocks"])
+    # the second workload of the target, timed after the headline one (here a small stand-in)
+    s2 = d["secondary"]
+    for k in ("workload", "value", "ms_per_step", "kernel_ms_per_step", "roofline", "bwd_bands", "band_scratch_gb",
+              "device_bytes_held", "clocks"):
+        assert k in s2, k
+    assert s2["workload"] == "tiny" and s2["value"] > 0 and s2["steps"] == 2
 
 
 def test_reference_arm_prints_its_line():

@@ -1,4 +1,4 @@
-"""Pins of the Ulysses pack / unpack oracle to what Section 3.3 fixes: after the all-to-all every rank
+"""Pins of the Ulysses pack / unpack oracle to what Section 3.5 fixes: after the all-to-all every rank
 holds all tokens of the group for its own h / P heads, the way back restores the token split, and the
 volume is Eq. (ulysses)'s. None of these re-evaluates the oracle's own index formula."""
 import os
@@ -21,7 +21,7 @@ def tagged(S, h, d):
 
 @pytest.mark.parametrize("world,n,h,d", [(2, 3, 4, 2), (4, 5, 8, 3), (1, 4, 3, 2), (8, 2, 8, 1), (2, 1, 16, 4)])
 def test_after_the_exchange_every_rank_holds_all_tokens_of_its_own_heads(world, n, h, d):
-    """Section 3.3: the transposes partition the heads across the ranks. The expected result is a slice
+    """Section 3.5: the transposes partition the heads across the ranks. The expected result is a slice
     of the global tensor, taken with numpy indexing, not with the oracle's loops."""
     X = tagged(world * n, h, d)                                     # the group's sequence, [S, h, d]
     local = [X[r * n:(r + 1) * n] for r in range(world)]            # token split

@@ -1,17 +1,21 @@
-"""hydra_lse_merge_noalloc against hydra_lse_merge.
+"""hydra_lse_merge_noalloc against hydra_lse_merge and against the oracle's merge.
 
 The no-alloc entry point exists for callers that cannot call cudaMalloc (a process that gave all
 device memory to its own pool, or a loop whose rules forbid a call that may synchronise the device).
-It must give what the ordinary merge gives. Both run the same kernel on the same partials, so the
-results are expected to agree to the bit; the comparison still uses the suite's tolerances.
-Two calls in a row, on different problems, check that the shared table array is rewritten each time.
-This file sorts last on purpose: a run that stops at the first failure has then run everything else.
+It must give what the ordinary merge gives: both are compared on the same partials with the suite's
+tolerances, and the no-alloc result is also compared, element by element, with the fp64 oracle's merge of
+those same partials (the two GPU entry points share a kernel, so agreeing with each other proves little).
+Two calls in a row, on different problems, check that the shared table array is rewritten each time, and
+the device's free memory must be the same before and after the second call: the property the entry point
+exists for. This file sorts last on purpose: a run that stops at the first failure has then run
+everything else.
 """
 import numpy as np
 import pytest
 import torch
 
 import hydra_workloads as hw
+import oracle
 from gpu_util import TOL_LSE, TOL_REL
 
 pytestmark = pytest.mark.gpu
@@ -34,9 +38,34 @@ def _partials(lengths, h, cp_r, seed):
     return P, cu, pairs, part_rows, step
 
 
-def _merge_both_ways(lengths, h, cp_r, seed):
+def _oracle_merge(cu, pairs, o_part, lse_part, T, h):
+    """fp64 merge (the oracle's) of the GPU's own partials, per merged q chunk; NaN elsewhere."""
+    o_np = o_part.float().cpu().numpy().astype(np.float64)
+    l_np = lse_part.cpu().numpy().astype(np.float64)
+    out = np.full((T, h, hw.D_V), np.nan)
+    lse = np.full((h, T), np.nan)
+    i = 0
+    while i < len(pairs):
+        j = i
+        while j < len(pairs) and pairs[j]["group"] == pairs[i]["group"]:
+            j += 1
+        p = pairs[i]
+        if p["part_row"] >= 0 and p["q_len"] > 0:
+            n = int(p["q_len"])
+            os_ = [o_np[int(pairs[t]["part_row"]):int(pairs[t]["part_row"]) + n] for t in range(i, j)]
+            ls_ = [l_np[:, int(pairs[t]["part_row"]):int(pairs[t]["part_row"]) + n] for t in range(i, j)]
+            mo, ml = oracle.lse_merge(os_, ls_)
+            t0 = int(cu[p["seq"]]) + int(p["q_start"])
+            out[t0:t0 + n] = mo
+            lse[:, t0:t0 + n] = ml
+        i = j
+    return out, lse
+
+
+def _merge_both_ways(lengths, h, cp_r, seed, memory_must_stay_flat):
     P, cu, pairs, part_rows, step = _partials(lengths, h, cp_r, seed)
-    merged = np.zeros(int(cu[-1]), dtype=bool)
+    T = int(cu[-1])
+    merged = np.zeros(T, dtype=bool)
     for p in pairs:
         if p["part_row"] >= 0:
             t0 = int(cu[p["seq"]]) + int(p["q_start"])
@@ -45,14 +74,30 @@ def _merge_both_ways(lengths, h, cp_r, seed):
     out_a, lse_a = torch.full_like(step.out, float("nan")), torch.full_like(step.lse, float("nan"))
     out_b, lse_b = torch.full_like(step.out, float("nan")), torch.full_like(step.lse, float("nan"))
     P.hydra_lse_merge(step.o_part, step.lse_part, part_rows, cu, h, pairs, out_a, lse_a, step.workspace)
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    launches_before = P.hydra_launch_count()
     P.hydra_lse_merge_noalloc(step.o_part, step.lse_part, part_rows, cu, h, pairs, out_b, lse_b)
     torch.cuda.synchronize()
+    free_after = torch.cuda.mem_get_info()[0]
+    assert P.hydra_launch_count() == launches_before + 1          # counted like every other launch
+    if memory_must_stay_flat:
+        # the first call on a device may make the driver load the module's data; from the second call
+        # on, the device's free memory must not move at all
+        assert free_after == free_before, (free_before, free_after)
     idx = torch.from_numpy(np.nonzero(merged)[0]).cuda()
     a, b = out_a[idx].float().cpu().numpy(), out_b[idx].float().cpu().numpy()
     la, lb = lse_a[:, idx].cpu().numpy(), lse_b[:, idx].cpu().numpy()
     assert np.isfinite(b).all() and np.isfinite(lb).all()
     assert np.abs(a - b).max() <= TOL_REL * np.abs(a).max()
     assert np.abs(la - lb).max() <= TOL_LSE
+    # against the oracle's merge of the same partials, element by element
+    ref_o, ref_l = _oracle_merge(cu, pairs, step.o_part, step.lse_part, T, h)
+    rows = np.nonzero(merged)[0]
+    got_o = out_b.float().cpu().numpy().astype(np.float64)[rows]
+    got_l = lse_b.cpu().numpy().astype(np.float64)[:, rows]
+    assert np.abs(got_o - ref_o[rows]).max() <= TOL_REL * np.abs(ref_o[rows]).max()
+    assert np.abs(got_l - ref_l[:, rows]).max() <= TOL_LSE
     # rows of chunks that have a single pair are not the merge's business: both leave them alone
     rest = torch.from_numpy(np.nonzero(~merged)[0]).cuda()
     if len(rest):
@@ -60,8 +105,8 @@ def _merge_both_ways(lengths, h, cp_r, seed):
 
 
 def test_no_alloc_merge_matches_the_ordinary_merge_twice_in_a_row():
-    _merge_both_ways([300, 77, 1001], 4, 1, seed=11)        # three chunked sequences, two chunks each
-    _merge_both_ways([2000, 5, 640], 3, 4, seed=12)         # a different problem: ring of four
+    _merge_both_ways([300, 77, 1001], 4, 1, seed=11, memory_must_stay_flat=False)   # two chunks per sequence
+    _merge_both_ways([2000, 5, 640], 3, 4, seed=12, memory_must_stay_flat=True)     # another problem: ring of 4
 
 
 def test_no_alloc_merge_rejects_what_exceeds_its_fixed_tables():
@@ -75,3 +120,19 @@ def test_no_alloc_merge_rejects_what_exceeds_its_fixed_tables():
     s = P.hydra_lse_merge_noalloc(dummy, dummy, part_rows, cu, 1, pairs, dummy, dummy, check=False)
     assert s == P.HYDRA_ERR_UNSUPPORTED
     assert P.hydra_status_string(s) == "HYDRA_ERR_UNSUPPORTED"
+
+
+def test_no_alloc_merge_rejects_overlapping_rows_like_the_ordinary_merge():
+    import paper_2609_34318_b200 as P
+    cu = hw.cu_seqlens([64])
+    pairs, part_rows, _, _ = P.hydra_zigzag_pairs(cu, 1)
+    dummy = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    n0 = P.hydra_launch_count()
+    bad = pairs.copy()
+    merged = np.nonzero(bad["part_row"] >= 0)[0]
+    assert len(merged) >= 2
+    bad["part_row"][merged[1]] = bad["part_row"][merged[0]]          # two partials on the same rows
+    for fn, extra in ((P.hydra_lse_merge_noalloc, ()), (P.hydra_lse_merge, (dummy,))):
+        s = fn(dummy, dummy, part_rows, cu, 1, bad, dummy, dummy, *extra, check=False)
+        assert s == P.HYDRA_ERR_INVALID_ARG, (fn.__name__, s)
+    assert P.hydra_launch_count() == n0
