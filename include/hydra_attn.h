@@ -399,6 +399,21 @@ int64_t hydra_launch_count(void);
  */
 void hydra_set_wait_limit_ns(uint64_t ns);
 
+/*
+ * Test hook for the bounded waits above (no counterpart in the paper: it is how the library's own
+ * failure path is exercised without faulting a GPU). While `ns` is non-zero for a
+ * kernel, the thread of every thread block that hands out work items idles for `ns` nanoseconds
+ * (at most 20 ms) at the start of that kernel's next launches and then hands out nothing and loads
+ * nothing: the other roles wait for a signal that is never given, their waits run out at the limit set
+ * with hydra_set_wait_limit_ns, the kernel records HYDRA_ERR_DEVICE_TIMEOUT with the index of a thread
+ * block in `detail` and returns by itself (no trap, no endless loop, nothing in flight). Outputs of such
+ * a launch are not written. ns = 0 (the default) switches the hook off; it costs one predicate per launch.
+ */
+#define HYDRA_STALL_FWD 0
+#define HYDRA_STALL_BWD_DKV 1
+#define HYDRA_STALL_BWD_DQ 2    /* either form of the query-side kernel */
+void hydra_debug_stall(int32_t kernel, uint64_t ns);
+
 int32_t hydra_version(void);
 
 /* Frees the cached work lists (device and pinned host memory). Safe to call at any time. */

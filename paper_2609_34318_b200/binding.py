@@ -54,6 +54,8 @@ def _load() -> ctypes.CDLL:
     lib.hydra_launch_count.restype = i64
     lib.hydra_set_wait_limit_ns.argtypes = [ctypes.c_uint64]
     lib.hydra_set_wait_limit_ns.restype = None
+    lib.hydra_debug_stall.argtypes = [i32, ctypes.c_uint64]
+    lib.hydra_debug_stall.restype = None
     lib.hydra_shutdown.restype = None
     lib.hydra_usp_factor.restype = i32
     lib.hydra_usp_factor.argtypes = [i32, i32, vp, vp]
@@ -122,7 +124,7 @@ def _load() -> ctypes.CDLL:
 
 _lib = _load()
 LIBRARY_PATH = _build.OUT
-EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_set_wait_limit_ns",
+EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_set_wait_limit_ns", "hydra_debug_stall",
            "hydra_shutdown", "hydra_usp_factor", "hydra_zigzag_pairs", "hydra_workspace_bytes",
            "hydra_attn_fwd", "hydra_lse_merge", "hydra_attn_bwd", "hydra_poll_status",
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
@@ -207,6 +209,15 @@ def hydra_launch_count() -> int:
 
 def hydra_set_wait_limit_ns(ns: int) -> None:
     _lib.hydra_set_wait_limit_ns(int(ns))
+
+
+HYDRA_STALL_FWD, HYDRA_STALL_BWD_DKV, HYDRA_STALL_BWD_DQ = 0, 1, 2
+
+
+def hydra_debug_stall(kernel: int, ns: int) -> None:
+    """Test hook: the work-issuing thread of every thread block of `kernel` idles for `ns` (at most 20 ms) and
+    then issues nothing, so that the bounded waits of the other roles run out (0 switches it off)."""
+    _lib.hydra_debug_stall(int(kernel), int(ns))
 
 
 def hydra_shutdown() -> None:

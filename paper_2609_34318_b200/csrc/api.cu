@@ -18,6 +18,7 @@ namespace {
 
 std::atomic<int64_t> g_launches{0};
 std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};
+std::atomic<uint64_t> g_debug_stall_ns[3];           // test hook, see hydra_debug_stall
 
 constexpr size_t kStatusBytes = 256;
 
@@ -642,6 +643,11 @@ int64_t hydra_launch_count(void) { return g_launches.load(); }
 
 void hydra_set_wait_limit_ns(uint64_t ns) { g_wait_limit_ns.store(ns ? ns : 1); }
 
+void hydra_debug_stall(int32_t kernel, uint64_t ns)
+{
+    if (kernel >= 0 && kernel < 3) g_debug_stall_ns[kernel].store(ns);
+}
+
 void hydra_shutdown(void)
 {
     std::lock_guard<std::mutex> lock(g_plan_mutex);
@@ -844,6 +850,7 @@ int32_t hydra_attn_fwd_gqa(const void* q, const void* k, const void* v, const in
     fp.scale_log2 = softmax_scale * 1.4426950408889634f;
     fp.status = static_cast<StatusBlock*>(workspace);
     fp.wait_limit_ns = g_wait_limit_ns.load();
+    fp.debug_stall_ns = g_debug_stall_ns[HYDRA_STALL_FWD].load();
     {
         ScopedKernelTimer timer(K_FWD, stream);
         if (launch_fwd(mq, mk, mv, fp, n_clusters, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
@@ -965,6 +972,7 @@ int32_t bwd_run(const Problem& pb, int32_t n_kv_heads, int32_t causal, float sof
         bp.items = at<GroupItem>(*plan, plan->off_items2);
         bp.n_items = plan->n_items2;
         bp.accumulate = accumulate_dkv ? 1 : 0;
+        bp.debug_stall_ns = g_debug_stall_ns[HYDRA_STALL_BWD_DKV].load();
         ScopedKernelTimer timer(K_DKV, stream);
         if (launch_bwd_dkv(mq_sub, mk, mv, mdo_sub, bp, sms, stream) != cudaSuccess)
             return HYDRA_ERR_CUDA;
@@ -975,6 +983,7 @@ int32_t bwd_run(const Problem& pb, int32_t n_kv_heads, int32_t causal, float sof
         bp.items = at<GroupItem>(*plan, plan->off_items);
         bp.n_items = plan->n_items;
         bp.accumulate = accumulate_dq ? 1 : 0;
+        bp.debug_stall_ns = g_debug_stall_ns[HYDRA_STALL_BWD_DQ].load();
         ScopedKernelTimer timer(K_DQ, stream);
         const cudaError_t e = hand_off ? launch_bwd_dq_from_ds(mk, bp, sms, stream)
                                        : launch_bwd_dq(mq, mk, mv, mdo, bp, sms, stream);

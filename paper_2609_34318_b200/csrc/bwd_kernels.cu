@@ -297,7 +297,9 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             // the current item
             GroupItem item_next;
             PairDev first_next;
-            int it_ahead = pop_end(0, pop_begin(0), item_next, first_next);
+            // test hook: idle, then hand out and load nothing; every other role's wait then runs out
+            if (p.debug_stall_ns) { debug_stall(p.debug_stall_ns); ok = false; }
+            int it_ahead = ok ? pop_end(0, pop_begin(0), item_next, first_next) : -1;
             for (uint32_t kq = 0; ok; ++kq) {
                 const int it = it_ahead;
                 if (it < 0) break;
@@ -694,6 +696,12 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         probe.start();
         GroupItem item_next;                          // lane 0: descriptors of the item popped ahead
         PairDev first_next;
+        // test hook: idle, then hand out and load nothing; every other role's wait then runs out
+        if (p.debug_stall_ns) {
+            if (lane == 0) debug_stall(p.debug_stall_ns);
+            __syncwarp();
+            ok = false;
+        }
         for (uint32_t kq = 0; ok; ++kq) {
             int it = 0, raw_next = 0;
             if (lane == 0) {                          // one pop per CTA, one item ahead, shared with the other lanes
@@ -1153,7 +1161,9 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_k,
             probe.start();
             GroupItem item_next;
             PairDev first_next;
-            int it_ahead = pop_end(0, pop_begin(0), item_next, first_next);
+            // test hook: idle, then hand out and load nothing; every other role's wait then runs out
+            if (p.debug_stall_ns) { debug_stall(p.debug_stall_ns); ok = false; }
+            int it_ahead = ok ? pop_end(0, pop_begin(0), item_next, first_next) : -1;
             for (uint32_t kq = 0; ok; ++kq) {
                 const int it = it_ahead;
                 if (it < 0) break;

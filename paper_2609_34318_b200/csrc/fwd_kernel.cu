@@ -135,9 +135,11 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             bool ok = true;
             ClockProbe probe;
             probe.start();
+            // test hook: idle, then hand out and load nothing; every other role's wait then runs out
+            if (p.debug_stall_ns) { debug_stall(p.debug_stall_ns); ok = false; }
             // the leader pops one item ahead: the round trip to the counter and the hand-over to the
             // other CTA then overlap the loads of the current item
-            int it_ahead = leader ? pop_item(0) : 0;
+            int it_ahead = (leader && ok) ? pop_item(0) : 0;
             for (uint32_t kq = 0; ok; ++kq) {
                 int it;
                 if (leader) {

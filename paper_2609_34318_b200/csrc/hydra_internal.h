@@ -130,6 +130,7 @@ struct FwdParams {
     float scale_log2;           // softmax_scale * log2(e)
     StatusBlock* status;
     uint64_t wait_limit_ns;
+    uint64_t debug_stall_ns;    // test hook (hydra_debug_stall): 0 in normal operation
 };
 
 struct BwdParams {
@@ -148,6 +149,7 @@ struct BwdParams {
     int64_t ds_head_blocks;     // blocks per head
     StatusBlock* status;
     uint64_t wait_limit_ns;
+    uint64_t debug_stall_ns;    // test hook (hydra_debug_stall): 0 in normal operation
 };
 
 struct MergeParams {

@@ -112,6 +112,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return true;
 }
 
+// Test hook: idle for `ns` nanoseconds (never more than 20 ms), by the clock of the whole GPU.
+__device__ __forceinline__ void debug_stall(uint64_t ns) {
+    const uint64_t limit = ns < 20000000ull ? ns : 20000000ull;
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < limit) { }
+}
+
 // Bounded wait until a counter in shared memory, written by another warp of the CTA, reaches
 // `target`. Used where only the ORDER of two warps' instruction streams matters (no data is handed
 // over), so a plain volatile word is enough; barrier phases would alias if the writer ran two steps

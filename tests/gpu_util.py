@@ -19,11 +19,43 @@ def pairs_for(cu, cp_r):
     return lib_pairs, part_rows, oracle.causal_pairs(cu, cp_r)
 
 
+GUARD_BYTES = 4096          # sentinel band before and after every output and the workspace
+GUARD_FILL = 0xA5
+
+
+def guard(step, names=("out", "lse", "o_part", "lse_part", "dq", "dk", "dv", "workspace")):
+    """Re-homes the listed buffers of an AttnStep inside larger allocations whose margins hold a sentinel
+    byte, and returns the function that checks the margins (compute-sanitizer is not available: a write
+    before the first or past the last byte of a buffer shows here instead)."""
+    import torch
+    bands = []
+    for n in names:
+        old = getattr(step, n)
+        nbytes = old.numel() * old.element_size()
+        room = (nbytes + 255) // 256 * 256
+        raw = torch.full((room + 2 * GUARD_BYTES,), GUARD_FILL, dtype=torch.uint8, device=old.device)
+        assert raw.data_ptr() % 256 == 0
+        new = raw[GUARD_BYTES:GUARD_BYTES + nbytes].view(old.dtype).view(old.shape)
+        new.copy_(old)
+        setattr(step, n, new)
+        bands.append((n, raw, nbytes))
+
+    def verify(where=""):
+        for n, raw, nbytes in bands:
+            lo = raw[:GUARD_BYTES]
+            hi = raw[GUARD_BYTES + nbytes:]
+            assert bool((lo == GUARD_FILL).all()), f"{where}{n}: bytes written before the buffer"
+            assert bool((hi == GUARD_FILL).all()), f"{where}{n}: bytes written past the buffer"
+    return verify
+
+
 def run_gpu(x, cu, h, pairs=None, part_rows=0, causal=True, scale=None, backward=True, poison=True):
-    """x: dict of uint16 bit arrays q, k, v, do. Returns dict of float64 numpy results."""
+    """x: dict of uint16 bit arrays q, k, v, do. Returns dict of float64 numpy results. Every output and the
+    workspace sit between sentinel bands that are checked after the calls."""
     import torch
     from paper_2609_34318_b200.runner import AttnStep, bits_to_tensor
     step = AttnStep(cu, h, pairs, part_rows, causal, scale)
+    verify_guards = guard(step)
     if poison:
         for t in (step.out, step.lse, step.dq, step.dk, step.dv, step.o_part, step.lse_part):
             t.fill_(float("nan"))
@@ -35,6 +67,7 @@ def run_gpu(x, cu, h, pairs=None, part_rows=0, causal=True, scale=None, backward
     status, detail = step.poll()
     assert status == 0, f"device status {status} (item {detail})"
     torch.cuda.synchronize()
+    verify_guards()
     T = int(cu[-1])
     res["out"] = step.out[:T].float().cpu().numpy().astype(np.float64)
     res["lse"] = step.lse[:, :T].cpu().numpy().astype(np.float64)

@@ -264,7 +264,10 @@ def spike_check(w, n_chunks, seed):
         worst[name] = float(ratio.max())
         bad = np.nonzero(live)[0][ratio > TOL_REL]
         assert len(bad) == 0, (w.name, name, "key blocks over 2e-2 of their own maximum", bad[:8], ratio.max())
-        assert e_blk[~live].max(initial=0.0) == 0.0, (w.name, name, "non-zero gradient where no query row sees the key")
+        # blocks whose reference is identically zero: no spike row sees them, or only the first row of a
+        # sequence does (one key: dP = D exactly, which fp32 reproduces to ~1e-8)
+        assert e_blk[~live].max(initial=0.0) <= 1e-6 * np.abs(ref).max(), \
+            (w.name, name, "gradient where the reference is identically zero", e_blk[~live].max(initial=0.0))
     idx = torch.as_tensor(np.asarray(rows, dtype=np.int64), device="cuda")
     g_dq = step.dq.index_select(0, idx).index_select(1, hsel).float().cpu().numpy().astype(np.float64)
     assert np.abs(g_dq - dq_ref).max() <= TOL_REL * np.abs(dq_ref).max(), (w.name, "dq")
