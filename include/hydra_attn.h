@@ -335,6 +335,35 @@ int32_t hydra_attn_fwd_bwd_host(const void* q_host, const void* k_host, const vo
                                 size_t arena_bytes, void* cuda_stream);
 
 /*
+ * The same entry points with the head dimensions as arguments. Two pairs are built: d_qk = 192, d_v = 128
+ * (the multi-head-latent model the configurations name: every other entry point is this case) and
+ * d_qk = d_v = 128 (the grouped-query model of the scale-out simulation, Section 6: eight KV heads; the
+ * paper gives no head dimension for it, 128 is the customary one). Any other pair returns
+ * HYDRA_ERR_UNSUPPORTED (hydra_workspace_bytes_dims: 0). q, k and dq, dk then have d_qk columns per head,
+ * v, out, dout and dv have d_v; everything else (layouts, partial buffers, workspace rules, banded and
+ * grouped-query forms, errors) is as in the entry points without the suffix.
+ */
+size_t hydra_workspace_bytes_dims(int32_t which, const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
+                                  int32_t n_kv_heads, int32_t d_qk, int32_t d_v, const hydra_pair_t* pairs,
+                                  int32_t n_pairs);
+int32_t hydra_attn_fwd_dims(const void* q, const void* k, const void* v, const int32_t* cu_seqlens_host,
+                            int32_t n_seqs, int32_t n_heads, int32_t n_kv_heads, int32_t d_qk, int32_t d_v,
+                            const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
+                            void* out, float* lse, void* o_part, float* lse_part, int64_t part_rows,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+int32_t hydra_attn_bwd_dims(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                            const void* dout, const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
+                            int32_t n_kv_heads, int32_t d_qk, int32_t d_v, const hydra_pair_t* pairs,
+                            int32_t n_pairs, int32_t causal, float softmax_scale, void* dq, void* dk, void* dv,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+int32_t hydra_attn_bwd_accumulate_dims(const void* q, const void* k, const void* v, const void* out,
+                                       const float* lse, const void* dout, const int32_t* cu_seqlens_host,
+                                       int32_t n_seqs, int32_t n_heads, int32_t n_kv_heads, int32_t d_qk,
+                                       int32_t d_v, const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal,
+                                       float softmax_scale, float* dq_acc, float* dk_acc, float* dv_acc,
+                                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * The local halves of the Ulysses all-to-all (Section 3.5: all-to-all transposes partition the attention
  * heads across the cp_u ranks of a group; Eq. (ulysses) counts the volume, about 4 S h / P elements per
  * rank for q, k, v and the output). Elements are 2 bytes wide (bf16) and are moved, not interpreted.
@@ -416,7 +445,19 @@ void hydra_debug_stall(int32_t kernel, uint64_t ns);
 
 int32_t hydra_version(void);
 
-/* Frees the cached work lists (device and pinned host memory). Safe to call at any time. */
+/*
+ * Device memory the library itself owns. The work tables of a problem (pairs, work items, lists) are built
+ * on the host, cached by content, and copied on the caller's stream (cudaMemcpyAsync from pinned staging)
+ * into a table arena that is allocated ONCE per device, by the first compute call on that device (default
+ * 32 MiB; hydra_set_plan_arena_bytes changes the size used by the next first call or the first call after
+ * hydra_shutdown). After that first call no entry point allocates or frees device memory or waits for the
+ * device, however many distinct problems are seen: when the arena is full its older half is recycled, and
+ * the stream that recycles it waits on the device for the kernels that last read it. The one exception is a
+ * problem whose tables exceed half the arena (about 500 000 work items at the default size): it gets an
+ * allocation of its own, once. A first call on a device should precede any stream capture.
+ * hydra_shutdown waits for the device and frees the arena, the cached tables and the pinned staging.
+ */
+void hydra_set_plan_arena_bytes(uint64_t bytes);
 void hydra_shutdown(void);
 
 #if defined(__GNUC__)

@@ -57,6 +57,8 @@ def _load() -> ctypes.CDLL:
     lib.hydra_debug_stall.argtypes = [i32, ctypes.c_uint64]
     lib.hydra_debug_stall.restype = None
     lib.hydra_shutdown.restype = None
+    lib.hydra_set_plan_arena_bytes.argtypes = [ctypes.c_uint64]
+    lib.hydra_set_plan_arena_bytes.restype = None
     lib.hydra_usp_factor.restype = i32
     lib.hydra_usp_factor.argtypes = [i32, i32, vp, vp]
     lib.hydra_zigzag_pairs.restype = i32
@@ -102,6 +104,16 @@ def _load() -> ctypes.CDLL:
     lib.hydra_attn_bwd_accumulate_gqa.argtypes = a[:9] + [i32] + a[9:]
     lib.hydra_attn_bwd_gqa.restype = i32
     lib.hydra_attn_bwd_gqa.argtypes = a[:9] + [i32] + a[9:]
+    # the same entry points with the head dimensions as arguments (d_qk, d_v after n_kv_heads)
+    lib.hydra_attn_fwd_dims.restype = i32
+    f = list(lib.hydra_attn_fwd_gqa.argtypes)
+    lib.hydra_attn_fwd_dims.argtypes = f[:7] + [i32, i32] + f[7:]
+    lib.hydra_workspace_bytes_dims.restype = sz
+    lib.hydra_workspace_bytes_dims.argtypes = [i32, vp, i32, i32, i32, i32, i32, vp, i32]
+    g = list(lib.hydra_attn_bwd_gqa.argtypes)
+    for name in ("hydra_attn_bwd_dims", "hydra_attn_bwd_accumulate_dims"):
+        getattr(lib, name).restype = i32
+        getattr(lib, name).argtypes = g[:10] + [i32, i32] + g[10:]
     lib.hydra_grad_cast.restype = i32
     lib.hydra_grad_cast.argtypes = [vp, vp, i64, vp]
     lib.hydra_poll_status.restype = i32
@@ -124,13 +136,14 @@ def _load() -> ctypes.CDLL:
 
 _lib = _load()
 LIBRARY_PATH = _build.OUT
-EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_set_wait_limit_ns", "hydra_debug_stall",
+EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_set_wait_limit_ns", "hydra_debug_stall", "hydra_set_plan_arena_bytes",
            "hydra_shutdown", "hydra_usp_factor", "hydra_zigzag_pairs", "hydra_workspace_bytes",
            "hydra_attn_fwd", "hydra_lse_merge", "hydra_attn_bwd", "hydra_poll_status",
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
            "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc", "hydra_lse_merge_accumulate",
            "hydra_sched_targets", "hydra_sched_cp", "hydra_sched_pack", "hydra_attn_bwd_accumulate",
            "hydra_grad_cast", "hydra_set_bwd_scratch_limit", "hydra_set_bwd_band_scratch", "hydra_bwd_bands", "hydra_ulysses_pack", "hydra_ulysses_unpack", "hydra_attn_fwd_gqa", "hydra_attn_bwd_accumulate_gqa", "hydra_attn_bwd_gqa", "hydra_workspace_bytes_gqa",
+           "hydra_attn_fwd_dims", "hydra_attn_bwd_dims", "hydra_attn_bwd_accumulate_dims", "hydra_workspace_bytes_dims",
            "hydra_poll_clocks")
 KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast", "ulysses")
 
@@ -222,6 +235,12 @@ def hydra_debug_stall(kernel: int, ns: int) -> None:
 
 def hydra_shutdown() -> None:
     _lib.hydra_shutdown()
+
+
+def hydra_set_plan_arena_bytes(nbytes: int) -> None:
+    """Size of the per-device arena that holds the work tables (used by the next first call on a device, or
+    the first call after hydra_shutdown)."""
+    _lib.hydra_set_plan_arena_bytes(int(nbytes))
 
 
 def hydra_usp_factor(degree: int, heads: int) -> Tuple[int, int]:
@@ -411,6 +430,65 @@ def hydra_attn_bwd_accumulate_gqa(q, k, v, out, lse, dout, cu_seqlens, n_heads: 
     if check:
         _check(s, "hydra_attn_bwd_accumulate_gqa")
     return s
+
+
+def hydra_workspace_bytes_dims(which: int, cu_seqlens, n_heads: int, n_kv_heads: int, d_qk: int, d_v: int,
+                               pairs=None) -> int:
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    return int(_lib.hydra_workspace_bytes_dims(which, cu.ctypes.data, len(cu) - 1, n_heads, n_kv_heads, int(d_qk),
+                                               int(d_v), pp, npairs))
+
+
+def hydra_attn_fwd_dims(q, k, v, cu_seqlens, n_heads: int, n_kv_heads: int, d_qk: int, d_v: int, pairs, causal: bool,
+                        softmax_scale: float, out, lse, o_part, lse_part, part_rows: int, workspace,
+                        workspace_bytes: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """hydra_attn_fwd_gqa with the head dimensions as arguments: (192, 128) or (128, 128)."""
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = _lib.hydra_attn_fwd_dims(_ptr(q), _ptr(k), _ptr(v), cu.ctypes.data, len(cu) - 1, n_heads, n_kv_heads,
+                                 int(d_qk), int(d_v), pp, npairs, int(bool(causal)),
+                                 ctypes.c_float(float(softmax_scale)), _ptr(out), _ptr(lse), _ptr(o_part),
+                                 _ptr(lse_part), int(part_rows), _ptr(workspace), int(workspace_bytes),
+                                 _stream(stream))
+    if check:
+        _check(s, "hydra_attn_fwd_dims")
+    return s
+
+
+def _bwd_dims(fn_name, q, k, v, out, lse, dout, cu_seqlens, n_heads, n_kv_heads, d_qk, d_v, pairs, causal,
+              softmax_scale, dq, dk, dv, workspace, workspace_bytes, stream, check):
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = getattr(_lib, fn_name)(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout), cu.ctypes.data,
+                               len(cu) - 1, n_heads, n_kv_heads, int(d_qk), int(d_v), pp, npairs,
+                               int(bool(causal)), ctypes.c_float(float(softmax_scale)), _ptr(dq), _ptr(dk),
+                               _ptr(dv), _ptr(workspace), int(workspace_bytes), _stream(stream))
+    if check:
+        _check(s, fn_name)
+    return s
+
+
+def hydra_attn_bwd_dims(q, k, v, out, lse, dout, cu_seqlens, n_heads: int, n_kv_heads: int, d_qk: int, d_v: int,
+                        pairs, causal: bool, softmax_scale: float, dq, dk, dv, workspace,
+                        workspace_bytes: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """hydra_attn_bwd_gqa with the head dimensions as arguments: (192, 128) or (128, 128)."""
+    return _bwd_dims("hydra_attn_bwd_dims", q, k, v, out, lse, dout, cu_seqlens, n_heads, n_kv_heads, d_qk, d_v,
+                     pairs, causal, softmax_scale, dq, dk, dv, workspace, workspace_bytes, stream, check)
+
+
+def hydra_attn_bwd_accumulate_dims(q, k, v, out, lse, dout, cu_seqlens, n_heads: int, n_kv_heads: int, d_qk: int,
+                                   d_v: int, pairs, causal: bool, softmax_scale: float, dq_acc, dk_acc, dv_acc,
+                                   workspace, workspace_bytes: Optional[int] = None, stream=None,
+                                   check: bool = True) -> int:
+    """hydra_attn_bwd_accumulate_gqa with the head dimensions as arguments: (192, 128) or (128, 128)."""
+    return _bwd_dims("hydra_attn_bwd_accumulate_dims", q, k, v, out, lse, dout, cu_seqlens, n_heads, n_kv_heads,
+                     d_qk, d_v, pairs, causal, softmax_scale, dq_acc, dk_acc, dv_acc, workspace, workspace_bytes,
+                     stream, check)
 
 
 def hydra_set_bwd_scratch_limit(n_bytes: int) -> None:

@@ -14,6 +14,8 @@ CSRC = os.path.join(PKG, "csrc")
 OUT = os.path.join(PKG, "libhydra_attn.so")
 OBJ_DIR = os.path.join(PKG, "build")
 SOURCES = ["api.cu", "fwd_kernel.cu", "bwd_kernels.cu", "aux_kernels.cu", "sched.cu"]
+# the tensor-core kernel files are compiled a second time for q / k heads of 128 (own symbol names)
+VARIANTS = [("fwd_kernel.cu", "d128", ["-DHYDRA_KERNEL_DQK=128"]), ("bwd_kernels.cu", "d128", ["-DHYDRA_KERNEL_DQK=128"])]
 HEADERS = ["hydra_internal.h", "sm100_ptx.cuh", os.path.join("..", "..", "include", "hydra_attn.h"),
            os.path.join("..", "..", "include", "hydra_sched.h")]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
@@ -24,7 +26,7 @@ FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std
 def _source_hash() -> str:
     """Content hash of everything the library is built from (file times do not survive a copy)."""
     import hashlib
-    h = hashlib.sha1(" ".join(FLAGS).encode())
+    h = hashlib.sha1((" ".join(FLAGS) + repr(VARIANTS)).encode())
     for name in SOURCES + HEADERS:
         with open(os.path.join(CSRC, name), "rb") as f:
             h.update(f.read())
@@ -38,9 +40,10 @@ def _stale() -> bool:
         return f.read().strip() != _source_hash()
 
 
-def _compile(src: str) -> str:
-    obj = os.path.join(OBJ_DIR, src.replace(".cu", ".o"))
-    cmd = [NVCC] + FLAGS + ["-c", os.path.join(CSRC, src), "-o", obj]
+def _compile(job) -> str:
+    src, tag, defines = job
+    obj = os.path.join(OBJ_DIR, src.replace(".cu", (("_" + tag) if tag else "") + ".o"))
+    cmd = [NVCC] + FLAGS + list(defines) + ["-c", os.path.join(CSRC, src), "-o", obj]
     r = subprocess.run(cmd, capture_output=True, text=True)
     with open(obj + ".log", "w") as f:
         f.write(" ".join(cmd) + "\n" + r.stdout + r.stderr)
@@ -53,8 +56,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return OUT
     os.makedirs(OBJ_DIR, exist_ok=True)
-    with ThreadPoolExecutor(max_workers=len(SOURCES)) as pool:
-        objs = list(pool.map(_compile, SOURCES))
+    jobs = [(src, "", []) for src in SOURCES] + VARIANTS
+    with ThreadPoolExecutor(max_workers=len(jobs)) as pool:
+        objs = list(pool.map(_compile, jobs))
     tmp = OUT + f".tmp{os.getpid()}"
     cmd = [NVCC, "-shared", "-o", tmp] + objs + ["-Xcompiler", "-fPIC"]
     r = subprocess.run(cmd, capture_output=True, text=True)

@@ -70,6 +70,7 @@ struct Problem {
     std::vector<hydra_pair_t> pairs;
     int32_t n_seqs = 0, h = 0;
     int64_t T = 0;
+    int32_t dqk = D_QK;     // q / k head dimension of the call: 192 or 128 (the value dimension is 128)
 };
 
 int32_t make_problem(const int32_t* cu, int32_t n_seqs, int32_t h, const hydra_pair_t* pairs,
@@ -154,8 +155,18 @@ int32_t check_identical_or_disjoint(std::vector<Range> r)
 }
 
 // ---------------------------------------------------------------------------------------------
-// plans: device-resident work lists, cached by content
+// plans: work lists built on the host, cached by content, resident on the device in a fixed arena
 // ---------------------------------------------------------------------------------------------
+// A training loop meets a new cu_seqlens with every micro-batch, so a new problem must cost neither a device
+// allocation nor a device-wide stall. The tables of a plan are built on the host (and cached by content:
+// every layer of a micro-batch asks for the same ones), staged in pinned host memory and copied with
+// cudaMemcpyAsync, on the caller's stream, into an arena that the library allocates ONCE per device (the
+// first call on that device). The arena is used as two halves: tables are appended to the active half; when
+// it is full the other half becomes active, the plans that lived there stop being resident (they are
+// uploaded again when they are next used) and the uploading stream first waits, on the device, for the
+// kernels that last read that half (an event per stream that used it). No cudaMalloc, no cudaFree and no
+// host-side wait happens after the first call on a device, whatever the number of distinct problems. The
+// one exception: a plan larger than half the arena gets an allocation of its own (and is cached).
 struct DeviceBlob {
     void* ptr = nullptr;
     ~DeviceBlob() { if (ptr) cudaFree(ptr); }
@@ -180,15 +191,162 @@ size_t append(std::vector<uint8_t>& blob, const std::vector<T>& v)
 struct Plan {
     std::vector<uint8_t> key;
     int kind = 0, device = 0;
-    DeviceBlob blob;
+    std::vector<uint8_t> blob;       // the tables, as they go to the device
     size_t off_pairs = 0, off_items = 0, off_lists = 0, off_groups = 0, off_items2 = 0, off_lists2 = 0;
     int32_t n_items = 0, n_items2 = 0;
     int64_t ds_head_blocks = 0;      // backward: blocks of the dS hand-off buffer per head; -1: not usable
+    // residency on the device (guarded by g_plan_mutex)
+    int half = -1;                   // arena half the tables were last copied to
+    uint64_t epoch = 0;              // generation of that half at the time: resident iff it still is the half's
+    size_t dev_off = 0;
+    cudaStream_t up_stream = nullptr;    // stream that carried the copy, and its completion
+    cudaEvent_t uploaded = nullptr;
+    DeviceBlob own;                  // a plan too large for the arena owns its device copy
+    ~Plan() { if (uploaded) cudaEventDestroy(uploaded); }
 };
 
 std::mutex g_plan_mutex;
-std::vector<std::unique_ptr<Plan>> g_plans;
+std::vector<std::shared_ptr<Plan>> g_plans;
 constexpr size_t kMaxPlans = 256;
+
+struct PlanArena {
+    uint8_t* base = nullptr;
+    size_t half_bytes = 0;
+    int active = 0;
+    size_t used = 0;
+    uint64_t epoch[2] = {0, 0};
+    uint64_t next_epoch = 1;
+    // kernels that read tables of a half: one event per stream, re-recorded at every use
+    std::vector<std::pair<cudaStream_t, cudaEvent_t>> users[2];
+    std::vector<cudaEvent_t> spare_events;
+    // "the previous readers of this half are done", recorded on the stream that switched to it; uploads on
+    // other streams wait for it
+    cudaEvent_t freed[2] = {nullptr, nullptr};
+    cudaStream_t freed_on[2] = {nullptr, nullptr};
+    // pinned staging: a slot is reused once the copy that read it has completed
+    struct Slot { uint8_t* host = nullptr; size_t cap = 0; cudaEvent_t done = nullptr; bool used = false; };
+    static constexpr int kSlots = 16;
+    Slot slots[kSlots];
+    int next_slot = 0;
+};
+PlanArena g_arena[64];
+std::atomic<uint64_t> g_arena_bytes{uint64_t{32} << 20};
+
+void arena_release(PlanArena& a)                         // device idle, g_plan_mutex held
+{
+    if (a.base) cudaFree(a.base);
+    a.base = nullptr; a.half_bytes = 0; a.used = 0; a.active = 0;
+    for (int h = 0; h < 2; ++h) {
+        for (auto& u : a.users[h]) cudaEventDestroy(u.second);
+        a.users[h].clear();
+        if (a.freed[h]) cudaEventDestroy(a.freed[h]);
+        a.freed[h] = nullptr; a.freed_on[h] = nullptr;
+        a.epoch[h] = a.next_epoch++;                     // nothing is resident any more
+    }
+    for (cudaEvent_t e : a.spare_events) cudaEventDestroy(e);
+    a.spare_events.clear();
+    for (auto& sl : a.slots) {
+        if (sl.host) cudaFreeHost(sl.host);
+        if (sl.done) cudaEventDestroy(sl.done);
+        sl = PlanArena::Slot{};
+    }
+}
+
+// Makes the tables of `plan` resident on the current device and returns their address. g_plan_mutex held.
+int32_t arena_place(Plan& plan, int device, cudaStream_t stream, const uint8_t** tables)
+{
+    if (plan.own.ptr) { *tables = static_cast<const uint8_t*>(plan.own.ptr); return HYDRA_OK; }
+    PlanArena& a = g_arena[device];
+    if (!a.base) {                                       // first call on this device: the one allocation
+        const size_t half = align_up(std::max<uint64_t>(g_arena_bytes.load() / 2, 4096), 256);
+        void* ptr = nullptr;
+        if (cudaMalloc(&ptr, 2 * half) != cudaSuccess) return HYDRA_ERR_CUDA;
+        a.base = static_cast<uint8_t*>(ptr);
+        a.half_bytes = half;
+        a.epoch[0] = a.next_epoch++;
+        a.epoch[1] = a.next_epoch++;
+    }
+    if (plan.half >= 0 && plan.epoch == a.epoch[plan.half]) {
+        // resident; a stream other than the one that carried the copy waits for the copy (free once complete)
+        if (stream != plan.up_stream && cudaStreamWaitEvent(stream, plan.uploaded, 0) != cudaSuccess) return HYDRA_ERR_CUDA;
+        *tables = a.base + plan.half * a.half_bytes + plan.dev_off;
+        return HYDRA_OK;
+    }
+    const size_t need = align_up(std::max<size_t>(plan.blob.size(), 16), 256);
+    if (need > a.half_bytes) {                           // documented exception: its own allocation, once
+        if (plan.own.upload(plan.blob) != cudaSuccess) return HYDRA_ERR_CUDA;
+        *tables = static_cast<const uint8_t*>(plan.own.ptr);
+        return HYDRA_OK;
+    }
+    if (a.used + need > a.half_bytes) {
+        // switch halves: what lived in the other half is no longer resident, and this stream waits (on the
+        // device) for the kernels that last read it before anything is copied over their tables
+        a.active ^= 1;
+        a.used = 0;
+        a.epoch[a.active] = a.next_epoch++;
+        for (auto& u : a.users[a.active]) {
+            if (cudaStreamWaitEvent(stream, u.second, 0) != cudaSuccess) return HYDRA_ERR_CUDA;
+            a.spare_events.push_back(u.second);
+        }
+        a.users[a.active].clear();
+        if (!a.freed[a.active] && cudaEventCreateWithFlags(&a.freed[a.active], cudaEventDisableTiming) != cudaSuccess)
+            return HYDRA_ERR_CUDA;
+        if (cudaEventRecord(a.freed[a.active], stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+        a.freed_on[a.active] = stream;
+    }
+    const int half = a.active;
+    if (a.freed[half] && a.freed_on[half] != stream && cudaStreamWaitEvent(stream, a.freed[half], 0) != cudaSuccess)
+        return HYDRA_ERR_CUDA;
+    // staging slot: pinned, reused once the copy that read it has completed (sixteen uploads ago, so the host
+    // may run several micro-batches ahead of the device before this ever waits)
+    PlanArena::Slot& sl = a.slots[a.next_slot];
+    a.next_slot = (a.next_slot + 1) % PlanArena::kSlots;
+    if (sl.used && cudaEventSynchronize(sl.done) != cudaSuccess) return HYDRA_ERR_CUDA;
+    if (sl.cap < need) {
+        if (sl.host) cudaFreeHost(sl.host);
+        sl.host = nullptr; sl.cap = 0;
+        const size_t cap = std::max<size_t>(need, size_t{256} << 10);
+        void* hp = nullptr;
+        if (cudaHostAlloc(&hp, cap, cudaHostAllocDefault) != cudaSuccess) return HYDRA_ERR_CUDA;
+        sl.host = static_cast<uint8_t*>(hp);
+        sl.cap = cap;
+    }
+    if (!sl.done && cudaEventCreateWithFlags(&sl.done, cudaEventDisableTiming) != cudaSuccess) return HYDRA_ERR_CUDA;
+    if (!plan.uploaded && cudaEventCreateWithFlags(&plan.uploaded, cudaEventDisableTiming) != cudaSuccess)
+        return HYDRA_ERR_CUDA;
+    if (!plan.blob.empty()) std::memcpy(sl.host, plan.blob.data(), plan.blob.size());
+    uint8_t* dst = a.base + half * a.half_bytes + a.used;
+    if (!plan.blob.empty() &&
+        cudaMemcpyAsync(dst, sl.host, plan.blob.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return HYDRA_ERR_CUDA;
+    if (cudaEventRecord(sl.done, stream) != cudaSuccess || cudaEventRecord(plan.uploaded, stream) != cudaSuccess)
+        return HYDRA_ERR_CUDA;
+    sl.used = true;
+    plan.half = half;
+    plan.epoch = a.epoch[half];
+    plan.dev_off = a.used;
+    plan.up_stream = stream;
+    a.used += need;
+    *tables = dst;
+    return HYDRA_OK;
+}
+
+// After the launches that read the tables of `plan`: remember that `stream` has to be waited for before the
+// plan's half of the arena is overwritten. g_plan_mutex held.
+void arena_note_use(const Plan& plan, int device, cudaStream_t stream)
+{
+    if (plan.own.ptr || plan.half < 0) return;
+    PlanArena& a = g_arena[device];
+    if (plan.epoch != a.epoch[plan.half]) return;
+    auto& users = a.users[plan.half];
+    for (auto& u : users)
+        if (u.first == stream) { cudaEventRecord(u.second, stream); return; }
+    cudaEvent_t e = nullptr;
+    if (!a.spare_events.empty()) { e = a.spare_events.back(); a.spare_events.pop_back(); }
+    else if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return;
+    cudaEventRecord(e, stream);
+    users.emplace_back(stream, e);
+}
 
 std::vector<uint8_t> make_key(int kind, int device, const Problem& pb, int causal)
 {
@@ -333,18 +491,26 @@ void build_fwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& 
     std::vector<int32_t> block_of, cost;
     for (size_t pi = 0; pi < pb.pairs.size(); ++pi) {
         const auto& p = pb.pairs[pi];
-        // one item = 512 q rows = two 256-row UMMA tiles of a CTA pair
-        for (int32_t q0 = 0; q0 < p.q_len; q0 += 4 * TILE) {
-            const int32_t n_a = kv_tiles(p, q0, causal, 2 * TILE);
-            const int32_t n_b = q0 + 2 * TILE < p.q_len ? kv_tiles(p, q0 + 2 * TILE, causal, 2 * TILE) : 0;
+        // One item = two consecutive 256-row UMMA tiles (A, then B) of a CTA pair. The slabs are aligned to
+        // the END of the q chunk: with an odd number of 256-row tiles the chunk's FIRST tile goes alone (it
+        // visits the fewest kv tiles), so the ragged last tile rides with a full neighbour instead of running
+        // its many kv tiles with the tensor cores half idle (32K packed workload: 1008 -> 942 kv steps per
+        // head, steps with a single active tile 266 -> 134).
+        const int32_t n_tiles = (p.q_len + 2 * TILE - 1) / (2 * TILE);
+        for (int32_t q0 = (n_tiles & 1) ? -2 * TILE : 0; q0 < p.q_len; q0 += 4 * TILE) {
+            const bool lone = q0 < 0;                       // tile A only, at row 0
+            const int32_t qa = lone ? 0 : q0;
+            const int32_t n_a = kv_tiles(p, qa, causal, 2 * TILE);
+            // n_b = -1: the item has no second tile (0 would mean: a tile whose rows see no key)
+            const int32_t n_b = (!lone && qa + 2 * TILE < p.q_len) ? kv_tiles(p, qa + 2 * TILE, causal, 2 * TILE) : -1;
             for (int32_t a = 0; a < pb.h; ++a) {
-                items.push_back(FwdItem{static_cast<int32_t>(pi), a, q0, n_a, n_b, {0, 0, 0}});
+                items.push_back(FwdItem{static_cast<int32_t>(pi), a, qa, n_a, n_b, {0, 0, 0}});
                 block_of.push_back(static_cast<int32_t>(pi) * pb.h + a);
                 // the two tiles advance in lockstep (one kv tile each per step of the issue order), so
                 // the time of an item goes with the longer tile, not with the sum: a slab whose second
                 // tile is empty costs as much per kv tile as a full one (measured: with the sum the
                 // slowest cluster of the 32K packed workload ended 17 % after the mean, now 4 %)
-                cost.push_back(2 * std::max(n_a, n_b));
+                cost.push_back(2 * std::max(n_a, std::max(n_b, 0)));
             }
         }
     }
@@ -478,40 +644,64 @@ void build_bwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& 
     plan.n_items2 = static_cast<int32_t>(items_k.size());
 }
 
-// Returns a cached plan or builds it (cudaMalloc + synchronous upload the first time only).
-int32_t get_plan(int kind, const Problem& pb, int causal, const Plan** out)
+// A plan on loan for the launches of one call: holds the plan cache's lock from the look-up to the last
+// launch (so that no other thread can recycle the arena half between the two), and on release records, on
+// the call's stream, that the tables have a reader.
+class PlanLease {
+public:
+    PlanLease() = default;
+    PlanLease(const PlanLease&) = delete;
+    PlanLease& operator=(const PlanLease&) = delete;
+    ~PlanLease()
+    {
+        if (!lock_.owns_lock()) return;
+        if (plan_) arena_note_use(*plan_, device_, stream_);
+    }
+    // Finds the plan (building it on the host the first time) and makes its tables resident.
+    int32_t acquire(int kind, const Problem& pb, int causal, cudaStream_t stream);
+    const Plan& plan() const { return *plan_; }
+    template <class T>
+    const T* at(size_t off) const { return reinterpret_cast<const T*>(tables_ + off); }
+
+private:
+    std::unique_lock<std::mutex> lock_;
+    std::shared_ptr<Plan> plan_;
+    const uint8_t* tables_ = nullptr;
+    int device_ = 0;
+    cudaStream_t stream_ = nullptr;
+};
+
+int32_t PlanLease::acquire(int kind, const Problem& pb, int causal, cudaStream_t stream)
 {
-    int device = 0;
-    if (cudaGetDevice(&device) != cudaSuccess) return HYDRA_ERR_CUDA;
-    std::vector<uint8_t> key = make_key(kind, device, pb, causal);
-    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    if (cudaGetDevice(&device_) != cudaSuccess || device_ < 0 || device_ >= 64) return HYDRA_ERR_CUDA;
+    stream_ = stream;
+    std::vector<uint8_t> key = make_key(kind, device_, pb, causal);
+    lock_ = std::unique_lock<std::mutex>(g_plan_mutex);
     for (size_t i = 0; i < g_plans.size(); ++i)
         if (g_plans[i]->key == key) {
             if (i + 1 != g_plans.size()) std::rotate(g_plans.begin() + i, g_plans.begin() + i + 1, g_plans.end());
-            *out = g_plans.back().get();
-            return HYDRA_OK;
+            plan_ = g_plans.back();
+            break;
         }
-    auto plan = std::make_unique<Plan>();
-    plan->kind = kind;
-    plan->device = device;
-    std::vector<uint8_t> blob;
-    if (kind == HYDRA_WS_FWD) build_fwd(pb, causal, *plan, blob);
-    else if (kind == HYDRA_WS_MERGE) build_merge(pb, *plan, blob);
-    else build_bwd(pb, causal, *plan, blob);
-    if (plan->blob.upload(blob) != cudaSuccess) return HYDRA_ERR_CUDA;
-    plan->key.swap(key);
-    if (g_plans.size() >= kMaxPlans) {
-        // evicting frees device memory a kernel in flight may still read: drain first
-        cudaDeviceSynchronize();
-        g_plans.erase(g_plans.begin());
+    if (!plan_) {
+        auto plan = std::make_shared<Plan>();
+        plan->kind = kind;
+        plan->device = device_;
+        if (kind == HYDRA_WS_FWD) build_fwd(pb, causal, *plan, plan->blob);
+        else if (kind == HYDRA_WS_MERGE) build_merge(pb, *plan, plan->blob);
+        else build_bwd(pb, causal, *plan, plan->blob);
+        plan->key.swap(key);
+        if (g_plans.size() >= kMaxPlans) {
+            // an evicted plan that owns device memory frees it: drain the device first (arena plans own none)
+            if (g_plans.front()->own.ptr) cudaDeviceSynchronize();
+            g_plans.erase(g_plans.begin());
+        }
+        g_plans.push_back(plan);
+        plan_ = std::move(plan);
     }
-    g_plans.push_back(std::move(plan));
-    *out = g_plans.back().get();
+    if (int32_t s = arena_place(*plan_, device_, stream, &tables_)) { plan_.reset(); return s; }
     return HYDRA_OK;
 }
-
-template <class T>
-const T* at(const Plan& p, size_t off) { return reinterpret_cast<const T*>(static_cast<const uint8_t*>(p.blob.ptr) + off); }
 
 // ---------------------------------------------------------------------------------------------
 // device properties and tensor maps
@@ -564,6 +754,28 @@ int32_t make_map(CUtensorMap* map, const void* base, int64_t T, int32_t h, int32
                            box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? HYDRA_OK : HYDRA_ERR_CUDA;
+}
+
+// The kernels of one q / k head dimension.
+struct KernelSet {
+    int (*fwd_max_clusters)();
+    cudaError_t (*launch_fwd)(const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, const FwdParams&, int,
+                              cudaStream_t);
+    cudaError_t (*launch_bwd_dq)(const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, const CUtensorMap&,
+                                 const BwdParams&, int, cudaStream_t);
+    cudaError_t (*launch_bwd_dq_from_ds)(const CUtensorMap&, const BwdParams&, int, cudaStream_t);
+    cudaError_t (*launch_bwd_dkv)(const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, const CUtensorMap&,
+                                  const BwdParams&, int, cudaStream_t);
+};
+const KernelSet* kernel_set(int32_t d_qk, int32_t d_v)
+{
+    static const KernelSet k192{fwd_max_clusters, launch_fwd, launch_bwd_dq, launch_bwd_dq_from_ds, launch_bwd_dkv};
+    static const KernelSet k128{fwd_max_clusters_d128, launch_fwd_d128, launch_bwd_dq_d128, launch_bwd_dq_from_ds_d128,
+                                launch_bwd_dkv_d128};
+    if (d_v != D_V) return nullptr;
+    if (d_qk == 192) return &k192;
+    if (d_qk == 128) return &k128;
+    return nullptr;
 }
 
 int32_t reset_status(void* workspace, cudaStream_t s)
@@ -651,9 +863,23 @@ void hydra_debug_stall(int32_t kernel, uint64_t ns)
 void hydra_shutdown(void)
 {
     std::lock_guard<std::mutex> lock(g_plan_mutex);
-    if (!g_plans.empty()) cudaDeviceSynchronize();
+    int current = 0, count = 0;
+    const bool have_device = cudaGetDevice(&current) == cudaSuccess && cudaGetDeviceCount(&count) == cudaSuccess;
+    for (int d = 0; have_device && d < count && d < 64; ++d) {
+        bool owns = g_arena[d].base != nullptr;
+        for (const auto& p : g_plans) owns |= (p->device == d && p->own.ptr != nullptr);
+        if (!owns) continue;
+        if (cudaSetDevice(d) != cudaSuccess) continue;
+        cudaDeviceSynchronize();                       // kernels in flight may still read the tables
+        for (auto it = g_plans.begin(); it != g_plans.end();)
+            it = ((*it)->device == d) ? g_plans.erase(it) : it + 1;
+        arena_release(g_arena[d]);
+    }
+    if (have_device) cudaSetDevice(current);
     g_plans.clear();
 }
+
+void hydra_set_plan_arena_bytes(uint64_t bytes) { g_arena_bytes.store(bytes); }
 
 int32_t hydra_usp_factor(int32_t degree, int32_t heads, int32_t* cp_u, int32_t* cp_r)
 {
@@ -736,11 +962,11 @@ uint64_t band_scratch_for(int64_t head_blocks, int32_t n_heads)
 
 size_t bwd_acc_bytes(const Problem& pb)
 {
-    return align_up(static_cast<size_t>(pb.T) * pb.h * D_QK * sizeof(float), 1024);
+    return align_up(static_cast<size_t>(pb.T) * pb.h * pb.dqk * sizeof(float), 1024);
 }
 size_t bwd_kv_acc_bytes(const Problem& pb, int32_t n_kv_heads)
 {
-    return align_up(static_cast<size_t>(pb.T) * n_kv_heads * (D_QK + D_V) * sizeof(float), 1024);
+    return align_up(static_cast<size_t>(pb.T) * n_kv_heads * (pb.dqk + D_V) * sizeof(float), 1024);
 }
 size_t bwd_base_bytes(const Problem& pb)
 {
@@ -767,9 +993,17 @@ size_t hydra_workspace_bytes(int32_t which, const int32_t* cu, int32_t n_seqs, i
 size_t hydra_workspace_bytes_gqa(int32_t which, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
                                  int32_t n_kv_heads, const hydra_pair_t* pairs, int32_t n_pairs)
 {
+    return hydra_workspace_bytes_dims(which, cu, n_seqs, n_heads, n_kv_heads, D_QK, D_V, pairs, n_pairs);
+}
+
+size_t hydra_workspace_bytes_dims(int32_t which, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                                  int32_t n_kv_heads, int32_t d_qk, int32_t d_v, const hydra_pair_t* pairs,
+                                  int32_t n_pairs)
+{
     Problem pb;
     if (make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb) != HYDRA_OK) return 0;
-    if (n_kv_heads < 1 || n_heads % n_kv_heads) return 0;
+    if (n_kv_heads < 1 || n_heads % n_kv_heads || !kernel_set(d_qk, d_v)) return 0;
+    pb.dqk = d_qk;
     if (which == HYDRA_WS_BWD && n_kv_heads != n_heads) {
         // one-shot grouped-query backward: fp32 dk, dv of the KV heads, then the dS buffer if within the limit
         const size_t ds = bwd_ds_bytes(ds_layout(pb, 1, nullptr), n_heads, g_ds_limit_bytes.load());
@@ -811,8 +1045,22 @@ int32_t hydra_attn_fwd_gqa(const void* q, const void* k, const void* v, const in
                            float* lse_part, int64_t part_rows, void* workspace, size_t workspace_bytes,
                            void* cuda_stream)
 {
+    return hydra_attn_fwd_dims(q, k, v, cu, n_seqs, n_heads, n_kv_heads, D_QK, D_V, pairs, n_pairs, causal,
+                               softmax_scale, out, lse, o_part, lse_part, part_rows, workspace, workspace_bytes,
+                               cuda_stream);
+}
+
+int32_t hydra_attn_fwd_dims(const void* q, const void* k, const void* v, const int32_t* cu, int32_t n_seqs,
+                            int32_t n_heads, int32_t n_kv_heads, int32_t d_qk, int32_t d_v,
+                            const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
+                            void* out, float* lse, void* o_part, float* lse_part, int64_t part_rows,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    const KernelSet* ks = kernel_set(d_qk, d_v);
+    if (!ks) return HYDRA_ERR_UNSUPPORTED;
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
+    pb.dqk = d_qk;
     if (n_kv_heads < 1 || n_heads % n_kv_heads) return HYDRA_ERR_INVALID_ARG;
     if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return HYDRA_ERR_INVALID_ARG;
     if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
@@ -829,20 +1077,21 @@ int32_t hydra_attn_fwd_gqa(const void* q, const void* k, const void* v, const in
     if (int32_t s = device_info(&sms)) return s;
     if (pb.pairs.empty()) return HYDRA_OK;
 
-    const int n_clusters = fwd_max_clusters();        // CTA pairs resident at once: the persistent grid
+    const int n_clusters = ks->fwd_max_clusters();        // CTA pairs resident at once: the persistent grid
     if (n_clusters < 1) return HYDRA_ERR_CUDA;
-    const Plan* plan = nullptr;
-    if (int32_t s = get_plan(HYDRA_WS_FWD, pb, causal != 0, &plan)) return s;
+    PlanLease lease;
+    if (int32_t s = lease.acquire(HYDRA_WS_FWD, pb, causal != 0, stream)) return s;
+    const Plan* plan = &lease.plan();
     if (plan->n_items == 0) return HYDRA_OK;
     // each CTA of a pair stages 64 kv rows of K (box of 64 rows) and 64 value columns of V
     CUtensorMap mq, mk, mv;
-    if (make_map(&mq, q, pb.T, n_heads, D_QK, TILE) || make_map(&mk, k, pb.T, n_kv_heads, D_QK, SUB) ||
+    if (make_map(&mq, q, pb.T, n_heads, pb.dqk, TILE) || make_map(&mk, k, pb.T, n_kv_heads, pb.dqk, SUB) ||
         make_map(&mv, v, pb.T, n_kv_heads, D_V, TILE))
         return HYDRA_ERR_CUDA;
     if (int32_t s = reset_status(workspace, stream)) return s;
     FwdParams fp{};
-    fp.pairs = at<PairDev>(*plan, plan->off_pairs);
-    fp.items = at<FwdItem>(*plan, plan->off_items);
+    fp.pairs = lease.at<PairDev>(plan->off_pairs);
+    fp.items = lease.at<FwdItem>(plan->off_items);
     fp.n_items = plan->n_items;
     fp.out = out; fp.lse = lse; fp.o_part = o_part; fp.lse_part = lse_part;
     fp.T = pb.T; fp.part_rows = part_rows; fp.h = n_heads; fp.causal = causal != 0;
@@ -853,7 +1102,7 @@ int32_t hydra_attn_fwd_gqa(const void* q, const void* k, const void* v, const in
     fp.debug_stall_ns = g_debug_stall_ns[HYDRA_STALL_FWD].load();
     {
         ScopedKernelTimer timer(K_FWD, stream);
-        if (launch_fwd(mq, mk, mv, fp, n_clusters, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+        if (ks->launch_fwd(mq, mk, mv, fp, n_clusters, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
     }
     g_launches += 1;
     return HYDRA_OK;
@@ -901,12 +1150,13 @@ int32_t merge_impl(const void* o_part, const float* lse_part, int64_t part_rows,
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     int sms = 0;
     if (int32_t s = device_info(&sms)) return s;
-    const Plan* plan = nullptr;
-    if (int32_t s = get_plan(HYDRA_WS_MERGE, pb, 0, &plan)) return s;
+    PlanLease lease;
+    if (int32_t s = lease.acquire(HYDRA_WS_MERGE, pb, 0, stream)) return s;
+    const Plan* plan = &lease.plan();
     MergeParams mp{};
-    mp.groups = at<MergeGroup>(*plan, plan->off_groups);
-    mp.lists = at<int32_t>(*plan, plan->off_lists);
-    mp.items = at<MergeItem>(*plan, plan->off_items);
+    mp.groups = lease.at<MergeGroup>(plan->off_groups);
+    mp.lists = lease.at<int32_t>(plan->off_lists);
+    mp.items = lease.at<MergeItem>(plan->off_items);
     mp.n_items = plan->n_items;
     mp.o_part = o_part; mp.lse_part = lse_part; mp.out = out; mp.lse = lse;
     mp.T = pb.T; mp.part_rows = part_rows; mp.h = n_heads;
@@ -932,14 +1182,17 @@ int32_t bwd_run(const Problem& pb, int32_t n_kv_heads, int32_t causal, float sof
                 cudaStream_t stream)
 {
     const int32_t n_heads = pb.h;
-    const Plan* plan = nullptr;
-    if (int32_t s = get_plan(HYDRA_WS_BWD, pb, causal != 0, &plan)) return s;
+    const KernelSet* ks = kernel_set(pb.dqk, D_V);
+    if (!ks) return HYDRA_ERR_UNSUPPORTED;
+    PlanLease lease;
+    if (int32_t s = lease.acquire(HYDRA_WS_BWD, pb, causal != 0, stream)) return s;
+    const Plan* plan = &lease.plan();
 
     float* dsum = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kStatusBytes);
     CUtensorMap mq, mk, mv, mdo, mq_sub, mdo_sub;
-    if (make_map(&mq, t.q, pb.T, n_heads, D_QK, TILE) || make_map(&mk, t.k, pb.T, n_kv_heads, D_QK, TILE) ||
+    if (make_map(&mq, t.q, pb.T, n_heads, pb.dqk, TILE) || make_map(&mk, t.k, pb.T, n_kv_heads, pb.dqk, TILE) ||
         make_map(&mv, t.v, pb.T, n_kv_heads, D_V, TILE) || make_map(&mdo, t.dout, pb.T, n_heads, D_V, TILE) ||
-        make_map(&mq_sub, t.q, pb.T, n_heads, D_QK, SUB) || make_map(&mdo_sub, t.dout, pb.T, n_heads, D_V, SUB))
+        make_map(&mq_sub, t.q, pb.T, n_heads, pb.dqk, SUB) || make_map(&mdo_sub, t.dout, pb.T, n_heads, D_V, SUB))
         return HYDRA_ERR_CUDA;
     if (first) {
         if (int32_t s = reset_status(workspace, stream)) return s;
@@ -952,7 +1205,7 @@ int32_t bwd_run(const Problem& pb, int32_t n_kv_heads, int32_t causal, float sof
     }
 
     BwdParams bp{};
-    bp.pairs = at<PairDev>(*plan, plan->off_pairs);
+    bp.pairs = lease.at<PairDev>(plan->off_pairs);
     bp.lse = t.lse; bp.dsum = dsum; bp.dq = t.dq; bp.dk = t.dk; bp.dv = t.dv;
     bp.T = pb.T; bp.h = n_heads; bp.causal = causal != 0;
     bp.kv_group = n_heads / n_kv_heads;
@@ -968,25 +1221,25 @@ int32_t bwd_run(const Problem& pb, int32_t n_kv_heads, int32_t causal, float sof
         bp.ds_head_blocks = plan->ds_head_blocks;
     }
     if (plan->n_items2 > 0) {
-        bp.lists = at<int32_t>(*plan, plan->off_lists2);
-        bp.items = at<GroupItem>(*plan, plan->off_items2);
+        bp.lists = lease.at<int32_t>(plan->off_lists2);
+        bp.items = lease.at<GroupItem>(plan->off_items2);
         bp.n_items = plan->n_items2;
         bp.accumulate = accumulate_dkv ? 1 : 0;
         bp.debug_stall_ns = g_debug_stall_ns[HYDRA_STALL_BWD_DKV].load();
         ScopedKernelTimer timer(K_DKV, stream);
-        if (launch_bwd_dkv(mq_sub, mk, mv, mdo_sub, bp, sms, stream) != cudaSuccess)
+        if (ks->launch_bwd_dkv(mq_sub, mk, mv, mdo_sub, bp, sms, stream) != cudaSuccess)
             return HYDRA_ERR_CUDA;
         g_launches += 1;
     }
     if (plan->n_items > 0) {
-        bp.lists = at<int32_t>(*plan, plan->off_lists);
-        bp.items = at<GroupItem>(*plan, plan->off_items);
+        bp.lists = lease.at<int32_t>(plan->off_lists);
+        bp.items = lease.at<GroupItem>(plan->off_items);
         bp.n_items = plan->n_items;
         bp.accumulate = accumulate_dq ? 1 : 0;
         bp.debug_stall_ns = g_debug_stall_ns[HYDRA_STALL_BWD_DQ].load();
         ScopedKernelTimer timer(K_DQ, stream);
-        const cudaError_t e = hand_off ? launch_bwd_dq_from_ds(mk, bp, sms, stream)
-                                       : launch_bwd_dq(mq, mk, mv, mdo, bp, sms, stream);
+        const cudaError_t e = hand_off ? ks->launch_bwd_dq_from_ds(mk, bp, sms, stream)
+                                       : ks->launch_bwd_dq(mq, mk, mv, mdo, bp, sms, stream);
         if (e != cudaSuccess)
             return HYDRA_ERR_CUDA;
         g_launches += 1;
@@ -1033,7 +1286,7 @@ std::vector<std::vector<hydra_pair_t>> make_bands(const Problem& pb, int32_t cau
         return true;
     };
     Problem probe;
-    probe.cu = pb.cu; probe.n_seqs = pb.n_seqs; probe.h = pb.h; probe.T = pb.T;
+    probe.cu = pb.cu; probe.n_seqs = pb.n_seqs; probe.h = pb.h; probe.T = pb.T; probe.dqk = pb.dqk;
     auto fits = [&](const std::vector<hydra_pair_t>& pairs) {
         probe.pairs = pairs;
         return bwd_ds_bytes(ds_layout(probe, causal, nullptr), pb.h, room) > 0;
@@ -1077,10 +1330,12 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
                  const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
                  const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
                  void* dq, void* dk, void* dv, bool accumulate, void* workspace, size_t workspace_bytes,
-                 void* cuda_stream, int32_t n_kv_heads)
+                 void* cuda_stream, int32_t n_kv_heads, int32_t d_qk = D_QK, int32_t d_v = D_V)
 {
+    if (!kernel_set(d_qk, d_v)) return HYDRA_ERR_UNSUPPORTED;
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
+    pb.dqk = d_qk;
     if (n_kv_heads < 1 || n_heads % n_kv_heads) return HYDRA_ERR_INVALID_ARG;
     if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return HYDRA_ERR_INVALID_ARG;
     if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
@@ -1113,7 +1368,7 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
         const size_t kv_bytes = bwd_kv_acc_bytes(pb, n_kv_heads);
         if (room < kv_bytes) return HYDRA_ERR_WORKSPACE_TOO_SMALL;
         float* dk_acc = reinterpret_cast<float*>(ws + ds_off);
-        float* dv_acc = dk_acc + static_cast<size_t>(pb.T) * n_kv_heads * D_QK;
+        float* dv_acc = dk_acc + static_cast<size_t>(pb.T) * n_kv_heads * pb.dqk;
         if (cudaMemsetAsync(dk_acc, 0, kv_bytes, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
         const BwdTensors tg{q, k, v, out, dout, lse, dq, dk_acc, dv_acc};
         if (int32_t s = bwd_run(pb, n_kv_heads, causal, softmax_scale, tg, false, true, workspace,
@@ -1126,7 +1381,7 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
         for (size_t i = 0; i < rs.size(); ++i) {
             if (i > 0 && rs[i].seq == rs[i - 1].seq && rs[i].start == rs[i - 1].start) continue;
             const size_t row = static_cast<size_t>(pb.cu[rs[i].seq]) + rs[i].start;
-            const size_t rk = static_cast<size_t>(n_kv_heads) * D_QK, rv = static_cast<size_t>(n_kv_heads) * D_V;
+            const size_t rk = static_cast<size_t>(n_kv_heads) * pb.dqk, rv = static_cast<size_t>(n_kv_heads) * D_V;
             ScopedKernelTimer timer(K_CAST, stream);
             if (launch_grad_cast(dk_acc + row * rk, static_cast<uint16_t*>(dk) + row * rk,
                                  static_cast<int64_t>(rs[i].len) * rk, stream) != cudaSuccess ||
@@ -1155,7 +1410,7 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
                 if (cudaMemsetAsync(dq_acc, 0, acc_bytes, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
                 const BwdTensors tb{q, k, v, out, dout, lse, dq_acc, dk, dv};
                 Problem band_pb;
-                band_pb.cu = pb.cu; band_pb.n_seqs = pb.n_seqs; band_pb.h = pb.h; band_pb.T = pb.T;
+                band_pb.cu = pb.cu; band_pb.n_seqs = pb.n_seqs; band_pb.h = pb.h; band_pb.T = pb.T; band_pb.dqk = pb.dqk;
                 bool first = true;
                 for (const auto& band : bands) {
                     band_pb.pairs = band;
@@ -1170,7 +1425,7 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
                 for (const auto& p : pb.pairs)
                     if (p.q_len > 0 && p.k_len > 0) rs.push_back(Range{p.seq, p.q_start, p.q_len});
                 std::sort(rs.begin(), rs.end(), range_less);
-                const size_t per_row = static_cast<size_t>(n_heads) * D_QK;
+                const size_t per_row = static_cast<size_t>(n_heads) * pb.dqk;
                 for (size_t i = 0; i < rs.size(); ++i) {
                     if (i > 0 && rs[i].seq == rs[i - 1].seq && rs[i].start == rs[i - 1].start) continue;
                     const size_t row = static_cast<size_t>(pb.cu[rs[i].seq]) + rs[i].start;
@@ -1248,6 +1503,27 @@ int32_t hydra_attn_bwd_accumulate_gqa(const void* q, const void* k, const void* 
 {
     return bwd_impl(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, dq_acc,
                     dk_acc, dv_acc, true, workspace, workspace_bytes, cuda_stream, n_kv_heads);
+}
+
+int32_t hydra_attn_bwd_dims(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                            const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads, int32_t n_kv_heads,
+                            int32_t d_qk, int32_t d_v, const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal,
+                            float softmax_scale, void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes,
+                            void* cuda_stream)
+{
+    return bwd_impl(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, dq, dk,
+                    dv, false, workspace, workspace_bytes, cuda_stream, n_kv_heads, d_qk, d_v);
+}
+
+int32_t hydra_attn_bwd_accumulate_dims(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                                       const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                                       int32_t n_kv_heads, int32_t d_qk, int32_t d_v, const hydra_pair_t* pairs,
+                                       int32_t n_pairs, int32_t causal, float softmax_scale, float* dq_acc,
+                                       float* dk_acc, float* dv_acc, void* workspace, size_t workspace_bytes,
+                                       void* cuda_stream)
+{
+    return bwd_impl(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, dq_acc,
+                    dk_acc, dv_acc, true, workspace, workspace_bytes, cuda_stream, n_kv_heads, d_qk, d_v);
 }
 
 int32_t hydra_grad_cast(const float* acc, void* grad, int64_t n_elements, void* cuda_stream)

@@ -22,10 +22,27 @@
 #include "hydra_internal.h"
 #include "sm100_ptx.cuh"
 
+// This file is compiled once per supported q / k head dimension (HYDRA_KERNEL_DQK = 192, the default, or
+// 128); the value dimension is 128 in both. HYDRA_K() gives the kernels and launchers of the second
+// build their own names. The tensor-memory maps are those of d_qk = 192 in both builds (at 128 a third of
+// the dQ / dK columns stays unused).
+#ifndef HYDRA_KERNEL_DQK
+#define HYDRA_KERNEL_DQK 192
+#endif
+#if HYDRA_KERNEL_DQK == 192
+#define HYDRA_K(name) name
+#elif HYDRA_KERNEL_DQK == 128
+#define HYDRA_K(name) name##_d128
+#else
+#error "unsupported q / k head dimension"
+#endif
+
 namespace hydra {
 
 namespace {
 
+constexpr int kDqk = HYDRA_KERNEL_DQK;
+constexpr int kQkBoxes = kDqk / 64;        // 64-column boxes of a q / k row
 constexpr int kThreads = 352;
 constexpr int kWarpProd = 8, kWarpMma = 9, kWarpMma2 = 10;
 constexpr uint32_t kBox128 = 128 * 128;   // [128 rows x 64 bf16]
@@ -119,11 +136,11 @@ __device__ __forceinline__ void add_row_f32(float* dst, const uint32_t* v, int n
 // ---------------------------------------------------------------------------------------------
 namespace dq {
 constexpr int kKStages = 2, kVSlots = 3;
-constexpr uint32_t kQ = 0;                                   // 3 boxes, stationary
-constexpr uint32_t kDO = kQ + 3 * kBox128;                   // 2 boxes, stationary
-constexpr uint32_t kK = kDO + 2 * kBox128;                   // 2 stages x 3 boxes
-constexpr uint32_t kV = kK + kKStages * 3 * kBox128;         // ring of 3 boxes [128 kv x 64 d_v]
-constexpr uint32_t kTotal = kV + kVSlots * kBox128;          // 229,376 B
+constexpr uint32_t kQ = 0;                                   // kQkBoxes boxes of 64 columns, stationary
+constexpr uint32_t kDO = kQ + kQkBoxes * kBox128;                   // 2 boxes, stationary
+constexpr uint32_t kK = kDO + 2 * kBox128;                   // 2 stages x kQkBoxes boxes
+constexpr uint32_t kV = kK + kKStages * kQkBoxes * kBox128;         // ring of 3 boxes [128 kv x 64 d_v]
+constexpr uint32_t kTotal = kV + kVSlots * kBox128;          // 229,376 B at d_qk = 192
 constexpr uint32_t kTmS = 0, kTmDP = 128, kTmDQ = 256, kTmDS = 448, kTmCols = 512;
 // K-full is kept per 64-column box (3 per stage): S = Q K^T consumes the boxes in order, so it starts
 // when the first 16 KB have landed instead of waiting for all 48 KB of the stage.
@@ -163,12 +180,12 @@ struct TileIter {
 // ---------------------------------------------------------------------------------------------
 namespace dkv {
 constexpr int kStages = 3;
-constexpr uint32_t kK = 0;                                   // 3 boxes of 128 rows, stationary
-constexpr uint32_t kV = kK + 3 * kBox128;                    // 2 boxes of 128 rows, stationary
-constexpr uint32_t kQ = kV + 2 * kBox128;                    // stages x 3 boxes of 64 rows
-constexpr uint32_t kDO = kQ + kStages * 3 * kBox64;          // stages x 2 boxes of 64 rows
+constexpr uint32_t kK = 0;                                   // kQkBoxes boxes of 128 rows, stationary
+constexpr uint32_t kV = kK + kQkBoxes * kBox128;                    // 2 boxes of 128 rows, stationary
+constexpr uint32_t kQ = kV + 2 * kBox128;                    // stages x kQkBoxes boxes of 64 rows
+constexpr uint32_t kDO = kQ + kStages * kQkBoxes * kBox64;          // stages x 2 boxes of 64 rows
 constexpr uint32_t kDsStage = kDO + kStages * 2 * kBox64;    // 8 warps x 2 KB: dK / dV rows on their way to memory
-constexpr uint32_t kTotal = kDsStage + 8 * 2048;             // 221,184 B
+constexpr uint32_t kTotal = kDsStage + 8 * 2048;             // 221,184 B at d_qk = 192
 constexpr uint32_t kTmDK = 0, kTmDV = 192, kTmS = 320, kTmDP = 384, kTmP = 448, kTmDS = 480,
                    kTmCols = 512;
 enum : int { B_KVFULL = 0, B_KVEMPTY = 1, B_QFULL = 2, B_STAT = 5, B_QEMPTY = 8, B_SFULL = 11,
@@ -203,14 +220,14 @@ struct SubIter {
 
 }  // namespace
 
-size_t bwd_dq_smem_bytes() { return dq::kTotal + 1024; }
-size_t bwd_dkv_smem_bytes() { return dkv::kTotal + 1024; }
+size_t HYDRA_K(bwd_dq_smem_bytes)() { return dq::kTotal + 1024; }
+size_t HYDRA_K(bwd_dkv_smem_bytes)() { return dkv::kTotal + 1024; }
 
 // =============================================================================================
 // dQ
 // =============================================================================================
 __global__ void __launch_bounds__(kThreads, 1)
-hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+HYDRA_K(hydra_bwd_dq_kernel)(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
                     const BwdParams p)
 {
@@ -314,8 +331,8 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 ok = wait(B_QEMPTY, items ^ 1u);
                 if (!ok) break;
                 ++items;
-                mbar_arrive_expect_tx(bar(B_QFULL), 5 * kBox128);
-                for (int c = 0; c < 3; ++c)
+                mbar_arrive_expect_tx(bar(B_QFULL), (kQkBoxes + 2) * kBox128);
+                for (int c = 0; c < kQkBoxes; ++c)
                     tma_load_3d(smem + kQ + c * kBox128, &map_q, bar(B_QFULL), c * 64, item.head,
                                 first.q_tok0 + item.r0);
                 for (int c = 0; c < 2; ++c)
@@ -338,9 +355,9 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     ok = wait(B_KEMPTY + st, (gk / kKStages) ^ 1u);
                     if (!ok) break;
                     ++gk;
-                    for (int c = 0; c < 3; ++c) {
+                    for (int c = 0; c < kQkBoxes; ++c) {
                         mbar_arrive_expect_tx(bar(B_KFULL + st * 3 + c), kBox128);
-                        tma_load_3d(smem + kK + st * 3 * kBox128 + c * kBox128, &map_k, bar(B_KFULL + st * 3 + c),
+                        tma_load_3d(smem + kK + st * kQkBoxes * kBox128 + c * kBox128, &map_k, bar(B_KFULL + st * 3 + c),
                                     c * 64, item.head / p.kv_group, tok);
                     }
                     if (!popped) { it_ahead = pop_end(kq + 1, raw_next, item_next, first_next); popped = true; }
@@ -358,7 +375,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         // on the uniform datapath); one elected lane issues the UMMAs and commits.
         {
             constexpr uint32_t idesc_s = umma_idesc_bf16(TILE, TILE, false, false);
-            constexpr uint32_t idesc_dq = umma_idesc_bf16(TILE, D_QK, false, true);
+            constexpr uint32_t idesc_dq = umma_idesc_bf16(TILE, kDqk, false, true);
             constexpr uint32_t hi_kmaj = umma_desc_hi(16, 1024);
             constexpr uint32_t hi_kmn = umma_desc_hi(kBox128, 1024);       // K as MN-major B, N = 192
             const uint32_t q_lo = umma_desc_lo(smem + kQ, 16), do_lo = umma_desc_lo(smem + kDO, 16);
@@ -406,9 +423,9 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                         if (n_tile > 0) ok = wait(B_SFREE, n_tile - 1u);   // previous S is in registers
                         if (!ok) break;
                         const int st = n_tile % kKStages;
-                        const uint32_t k_lo = k_lo0 + st * (3 * kBox128 >> 4);
+                        const uint32_t k_lo = k_lo0 + st * (kQkBoxes * kBox128 >> 4);
 #pragma unroll
-                        for (int c = 0; c < 3; ++c) {
+                        for (int c = 0; c < kQkBoxes; ++c) {
                             ok = wait(B_KFULL + st * 3 + c, n_tile / kKStages);
                             if (!ok) break;
                             tc_fence_after_sync();
@@ -418,7 +435,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                                     const uint32_t o = c * (kBox128 >> 4) + kk * 2;
                                     umma_ss_w(tm + kTmS, q_lo + o, hi_kmaj, k_lo + o, hi_kmaj, idesc_s, (c | kk) != 0);
                                 }
-                                if (c == 2) umma_commit(bar(B_SFULL));
+                                if (c == kQkBoxes - 1) umma_commit(bar(B_SFULL));
                             }
                         }
                         if (!ok) break;
@@ -433,7 +450,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                         // then columns [32,64) (K-steps 2,3,6,7); the update of the first overlaps the
                         // exponentials of the second
                         const int st = n_tile % kKStages;
-                        const uint32_t k_lo = kmn_lo0 + st * (3 * kBox128 >> 4);
+                        const uint32_t k_lo = kmn_lo0 + st * (kQkBoxes * kBox128 >> 4);
 #pragma unroll
                         for (int half = 0; half < 2; ++half) {
                             ok = wait(B_PFULL + half, n_tile);
@@ -479,7 +496,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const int32_t* list = p.lists + item.list_off;
             const int row = item.r0 + r;
             const bool row_valid = row < first.q_len;
-            const int64_t dst_off = (static_cast<int64_t>(first.q_tok0 + row) * p.h + item.head) * D_QK + g * 96;
+            const int64_t dst_off = (static_cast<int64_t>(first.q_tok0 + row) * p.h + item.head) * kDqk + g * (kDqk / 2);
             __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.dq) + dst_off;
             float* dst_acc = static_cast<float*>(p.dq) + dst_off;        // accumulate mode: dq is fp32
             TileIter ti;
@@ -488,7 +505,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 if (row_valid && !p.accumulate) {
                     uint4* d4 = reinterpret_cast<uint4*>(dst);
 #pragma unroll
-                    for (int e = 0; e < 12; ++e) d4[e] = make_uint4(0u, 0u, 0u, 0u);
+                    for (int e = 0; e < kDqk / 16; ++e) d4[e] = make_uint4(0u, 0u, 0u, 0u);
                 }
                 continue;
             }
@@ -564,16 +581,16 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 ++c_ds;
             }
             if (!ok) break;
-            // ---- epilogue: dQ * scale -> bf16; this warpgroup writes 96 of the 192 columns ---------
+            // ---- epilogue: dQ * scale -> bf16; this warpgroup writes half of the columns ---------
             ok = wait(B_DSFREE, c_ds - 1u);
             if (!ok) break;
             tc_fence_after_sync();
 #pragma unroll
-            for (int c0 = 0; c0 < 96; c0 += 32) {
+            for (int c0 = 0; c0 < kDqk / 2; c0 += 32) {
                 uint32_t v[32];
-                tmem_ld_x32(tm + kTmDQ + lane_base + g * 96 + c0, v);
+                tmem_ld_x32(tm + kTmDQ + lane_base + g * (kDqk / 2) + c0, v);
                 tmem_wait_ld();
-                if (c0 == 64) {
+                if (c0 + 32 == kDqk / 2) {
                     tc_fence_before_sync();
                     mbar_arrive_warp(bar(B_ACCFREE));
                 }
@@ -605,7 +622,7 @@ hydra_bwd_dq_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 // dK / dV
 // =============================================================================================
 __global__ void __launch_bounds__(kThreads, 1)
-hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+HYDRA_K(hydra_bwd_dkv_kernel)(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
                      const BwdParams p)
 {
@@ -727,8 +744,8 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (!ok) break;
             ++items;
             if (lane == 0) {
-                mbar_arrive_expect_tx(bar(B_KVFULL), 5 * kBox128);
-                for (int c = 0; c < 3; ++c)
+                mbar_arrive_expect_tx(bar(B_KVFULL), (kQkBoxes + 2) * kBox128);
+                for (int c = 0; c < kQkBoxes; ++c)
                     tma_load_3d(smem + kK + c * kBox128, &map_k, bar(B_KVFULL), c * 64, item.head / p.kv_group,
                                 first.k_tok0 + item.r0);
                 for (int c = 0; c < 2; ++c)
@@ -741,9 +758,9 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 if (!ok) break;
                 const int tok = si.cur.q_tok0 + si.u * SUB;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(bar(B_QFULL + st), 5 * kBox64);
-                    for (int c = 0; c < 3; ++c)
-                        tma_load_3d(smem + kQ + st * 3 * kBox64 + c * kBox64, &map_q, bar(B_QFULL + st), c * 64,
+                    mbar_arrive_expect_tx(bar(B_QFULL + st), (kQkBoxes + 2) * kBox64);
+                    for (int c = 0; c < kQkBoxes; ++c)
+                        tma_load_3d(smem + kQ + st * kQkBoxes * kBox64 + c * kBox64, &map_q, bar(B_QFULL + st), c * 64,
                                     item.head, tok);
                     for (int c = 0; c < 2; ++c)
                         tma_load_3d(smem + kDO + st * 2 * kBox64 + c * kBox64, &map_do, bar(B_QFULL + st), c * 64,
@@ -778,7 +795,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         {
             constexpr uint32_t idesc_st = umma_idesc_bf16(TILE, SUB, false, false);
             constexpr uint32_t idesc_dv = umma_idesc_bf16(TILE, D_V, false, true);
-            constexpr uint32_t idesc_dk = umma_idesc_bf16(TILE, D_QK, false, true);
+            constexpr uint32_t idesc_dk = umma_idesc_bf16(TILE, kDqk, false, true);
             constexpr uint32_t hi_kmaj = umma_desc_hi(16, 1024);
             constexpr uint32_t hi_mn = umma_desc_hi(kBox64, 1024);         // Q / dO sub-tiles as MN-major B
             const uint32_t k_lo = umma_desc_lo(smem + kK, 16), v_lo = umma_desc_lo(smem + kV, 16);
@@ -805,7 +822,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                         const int st = n_step % kStages;
                         ok = wait(B_QFULL + st, n_step / kStages);
                         if (!ok) break;
-                        const uint32_t q_lo = q_lo0 + st * (3 * kBox64 >> 4), do_lo = do_lo0 + st * (2 * kBox64 >> 4);
+                        const uint32_t q_lo = q_lo0 + st * (kQkBoxes * kBox64 >> 4), do_lo = do_lo0 + st * (2 * kBox64 >> 4);
                         const uint32_t prev = n_step;
                         ++n_step;
                         si.next();
@@ -814,7 +831,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                         tc_fence_after_sync();
                         if (elect_one()) {
 #pragma unroll
-                            for (int kk = 0; kk < D_QK / 16; ++kk)
+                            for (int kk = 0; kk < kDqk / 16; ++kk)
                                 umma_ss_w(tm + kTmS, k_lo + (kk >> 2) * (kBox128 >> 4) + (kk & 3) * 2, hi_kmaj,
                                           q_lo + (kk >> 2) * (kBox64 >> 4) + (kk & 3) * 2, hi_kmaj, idesc_st, kk > 0);
 #pragma unroll
@@ -841,7 +858,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                         if (!ok) break;
                         tc_fence_after_sync();
                         const int st = n_step % kStages;
-                        const uint32_t do_lo = domn_lo0 + st * (2 * kBox64 >> 4), q_lo = qmn_lo0 + st * (3 * kBox64 >> 4);
+                        const uint32_t do_lo = domn_lo0 + st * (2 * kBox64 >> 4), q_lo = qmn_lo0 + st * (kQkBoxes * kBox64 >> 4);
                         const uint32_t acc = first_step ? 0u : 1u;
                         if (elect_one()) {
 #pragma unroll
@@ -889,7 +906,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             // with shared KV heads (accumulating form only) the query heads of a group add into one dk / dv row
             const int64_t kv_heads = p.h / p.kv_group;
             const int64_t kv_row = tok * kv_heads + item.head / p.kv_group;
-            const int64_t dk_off = kv_row * D_QK + g * 96;
+            const int64_t dk_off = kv_row * kDqk + g * (kDqk / 2);
             const int64_t dv_off = kv_row * D_V + g * 64;
             __nv_bfloat16* dkp = static_cast<__nv_bfloat16*>(p.dk) + dk_off;
             __nv_bfloat16* dvp = static_cast<__nv_bfloat16*>(p.dv) + dv_off;
@@ -902,7 +919,7 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     uint4* a4 = reinterpret_cast<uint4*>(dkp);
                     uint4* b4 = reinterpret_cast<uint4*>(dvp);
 #pragma unroll
-                    for (int e = 0; e < 12; ++e) a4[e] = make_uint4(0u, 0u, 0u, 0u);
+                    for (int e = 0; e < kDqk / 16; ++e) a4[e] = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) b4[e] = make_uint4(0u, 0u, 0u, 0u);
                 }
@@ -994,37 +1011,39 @@ hydra_bwd_dkv_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             tc_fence_after_sync();
             const uint32_t rows_valid = __ballot_sync(0xffffffffu, row_valid);
             const uint32_t out_slice = smem + kDsStage + warp * 2048;
-            // five chunks of 32 columns (dK: 3, dV: 2); the load of the next chunk is in flight while the
-            // current one is packed, transposed and stored
+            // chunks of 32 columns (dK: kDkChunks, then dV: 2); the load of the next chunk is in flight while
+            // the current one is packed, transposed and stored
+            constexpr int kDkChunks = kDqk / 64, kChunks = kDkChunks + 2;
             auto chunk_addr = [&](int c) -> uint32_t {
-                return c < 3 ? tm + kTmDK + lane_base + g * 96 + c * 32 : tm + kTmDV + lane_base + g * 64 + (c - 3) * 32;
+                return c < kDkChunks ? tm + kTmDK + lane_base + g * (kDqk / 2) + c * 32
+                                     : tm + kTmDV + lane_base + g * 64 + (c - kDkChunks) * 32;
             };
             uint32_t va[32], vb[32];
             tmem_ld_x32(chunk_addr(0), va);
 #pragma unroll
-            for (int c = 0; c < 5; ++c) {
+            for (int c = 0; c < kChunks; ++c) {
                 uint32_t* cur = (c & 1) ? vb : va;
                 uint32_t* nxt = (c & 1) ? va : vb;
                 tmem_wait_ld();
-                if (c + 1 < 5) tmem_ld_x32(chunk_addr(c + 1), nxt);
-                if (c == 4) {                          // every column has left tensor memory
+                if (c + 1 < kChunks) tmem_ld_x32(chunk_addr(c + 1), nxt);
+                if (c == kChunks - 1) {                          // every column has left tensor memory
                     tc_fence_before_sync();
                     mbar_arrive_warp(bar(B_ACCFREE));
                 }
-                const bool is_dk = c < 3;
-                const int c0 = is_dk ? c * 32 : (c - 3) * 32;
+                const bool is_dk = c < kDkChunks;
+                const int c0 = is_dk ? c * 32 : (c - kDkChunks) * 32;
                 if (p.accumulate) {
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
                         if (is_dk)
-                            add_rows_f32_coalesced(out_slice, lane, dkp_acc + c0 + half * 16, kv_heads * D_QK,
+                            add_rows_f32_coalesced(out_slice, lane, dkp_acc + c0 + half * 16, kv_heads * kDqk,
                                                    cur + half * 16, p.scale, rows_valid);
                         else
                             add_rows_f32_coalesced(out_slice, lane, dvp_acc + c0 + half * 16, kv_heads * D_V,
                                                    cur + half * 16, 1.f, rows_valid);
                     }
                 } else if (is_dk) {
-                    store_rows_bf16_coalesced(out_slice, lane, dkp + c0, kv_heads * D_QK, cur, p.scale, rows_valid);
+                    store_rows_bf16_coalesced(out_slice, lane, dkp + c0, kv_heads * kDqk, cur, p.scale, rows_valid);
                 } else {
                     store_rows_bf16_coalesced(out_slice, lane, dvp + c0, kv_heads * D_V, cur, 1.f, rows_valid);
                 }
@@ -1069,17 +1088,17 @@ constexpr int kThreadsS = 224;
 constexpr int kDsStages = 3, kKStages = 2;
 constexpr uint32_t kDsBytes = 2 * DS_BLOCK_BYTES;            // blocks (jk, 2i) and (jk, 2i + 1)
 constexpr uint32_t kK = kDsStages * kDsBytes;                // 96 KB of dS^T, then the K tiles
-constexpr uint32_t kOut = kK + kKStages * 3 * kBox128;       // 4 epilogue warps x 2 KB: dQ rows on their way out
-constexpr uint32_t kTotal = kOut + 4 * 2048;                 // 204,800 B
+constexpr uint32_t kOut = kK + kKStages * kQkBoxes * kBox128;       // 4 epilogue warps x 2 KB: dQ rows on their way out
+constexpr uint32_t kTotal = kOut + 4 * 2048;                 // 204,800 B at d_qk = 192
 constexpr uint32_t kTmAcc = 256, kTmCols = 512;              // accumulators at columns 0 and 256
 enum : int { B_DSFULL = 0, B_DSEMPTY = 4, B_KFULL = 8, B_KEMPTY = 10, B_ACCFULL = 12, B_ACCFREE = 14,
              B_ITEMFULL = 16, B_ITEMEMPTY = 16 + kSched, B_COUNT = 16 + 2 * kSched };
 }  // namespace dqs
 
-size_t bwd_dq_ds_smem_bytes() { return dqs::kTotal + 1024; }
+size_t HYDRA_K(bwd_dq_ds_smem_bytes)() { return dqs::kTotal + 1024; }
 
 __global__ void __launch_bounds__(dqs::kThreadsS, 1)
-hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_k,
+HYDRA_K(hydra_bwd_dq_from_ds_kernel)(const __grid_constant__ CUtensorMap map_k,
                             const BwdParams p)
 {
     using namespace dqs;
@@ -1208,16 +1227,16 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_k,
                 ok = wait(B_KEMPTY + st, (g / kKStages) ^ 1u);
                 if (!ok) break;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(bar(B_KFULL + st), 3 * kBox128);
-                    for (int c = 0; c < 3; ++c)
-                        tma_load_3d(smem + kK + (st * 3 + c) * kBox128, &map_k, bar(B_KFULL + st), c * 64,
+                    mbar_arrive_expect_tx(bar(B_KFULL + st), kQkBoxes * kBox128);
+                    for (int c = 0; c < kQkBoxes; ++c)
+                        tma_load_3d(smem + kK + (st * kQkBoxes + c) * kBox128, &map_k, bar(B_KFULL + st), c * 64,
                                     item.head / p.kv_group, ti.cur.k_tok0 + ti.t * TILE);
                 }
             }
         }
     } else if (warp == 5) {
         // ------------------------------------------------------------------ UMMA issuer
-        constexpr uint32_t idesc = umma_idesc_bf16(TILE, D_QK, true, true);
+        constexpr uint32_t idesc = umma_idesc_bf16(TILE, kDqk, true, true);
         // dS^T without swizzle: 8 kv rows are 128 bytes, chunks of 8 q rows are 2 KB apart (two blocks in a row)
         constexpr uint32_t hi_ds = umma_desc_plain_hi(128, 2048);
         constexpr uint32_t hi_k = umma_desc_hi(kBox128, 1024);           // K: N chunks of 64 columns 16 KB apart
@@ -1244,7 +1263,7 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_k,
                 tc_fence_after_sync();
                 if (elect_one()) {
                     const uint32_t a_lo = umma_desc_plain_lo(smem + ds_st * kDsBytes, 128);
-                    const uint32_t b_lo = umma_desc_lo(smem + kK + k_st * 3 * kBox128, kBox128);
+                    const uint32_t b_lo = umma_desc_lo(smem + kK + k_st * kQkBoxes * kBox128, kBox128);
 #pragma unroll
                     for (int kk = 0; kk < TILE / 16; ++kk)
                         umma_ss_w(tm + buf * kTmAcc, a_lo + kk * (256 >> 4), hi_ds, b_lo + kk * (2048 >> 4), hi_k, idesc,
@@ -1272,7 +1291,7 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_k,
             const int32_t* list = p.lists + item.list_off;
             const int row = item.r0 + r;
             const bool row_valid = row < first.q_len;
-            const int64_t dst_off = (static_cast<int64_t>(first.q_tok0 + row) * p.h + item.head) * D_QK;
+            const int64_t dst_off = (static_cast<int64_t>(first.q_tok0 + row) * p.h + item.head) * kDqk;
             __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.dq) + dst_off;
             float* dst_acc = static_cast<float*>(p.dq) + dst_off;
             TileIter ti;
@@ -1281,7 +1300,7 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_k,
                 if (row_valid && !p.accumulate) {
                     uint4* d4 = reinterpret_cast<uint4*>(dst);
 #pragma unroll
-                    for (int e = 0; e < 24; ++e) d4[e] = make_uint4(0u, 0u, 0u, 0u);
+                    for (int e = 0; e < kDqk / 8; ++e) d4[e] = make_uint4(0u, 0u, 0u, 0u);
                 }
                 continue;
             }
@@ -1292,21 +1311,21 @@ hydra_bwd_dq_from_ds_kernel(const __grid_constant__ CUtensorMap map_k,
             const uint32_t rows_valid = __ballot_sync(0xffffffffu, row_valid);
             const uint32_t out_slice = smem + kOut + warp * 2048;
 #pragma unroll
-            for (int c0 = 0; c0 < D_QK; c0 += 32) {
+            for (int c0 = 0; c0 < kDqk; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_x32(tm + buf * kTmAcc + lane_base + c0, v);
                 tmem_wait_ld();
-                if (c0 + 32 == D_QK) {
+                if (c0 + 32 == kDqk) {
                     tc_fence_before_sync();
                     mbar_arrive_warp(bar(B_ACCFREE + buf));
                 }
                 if (p.accumulate) {
 #pragma unroll
                     for (int half = 0; half < 2; ++half)
-                        add_rows_f32_coalesced(out_slice, lane, dst_acc + c0 + half * 16, static_cast<int64_t>(p.h) * D_QK,
+                        add_rows_f32_coalesced(out_slice, lane, dst_acc + c0 + half * 16, static_cast<int64_t>(p.h) * kDqk,
                                                v + half * 16, p.scale, rows_valid);
                 } else {
-                    store_rows_bf16_coalesced(out_slice, lane, dst + c0, static_cast<int64_t>(p.h) * D_QK, v, p.scale, rows_valid);
+                    store_rows_bf16_coalesced(out_slice, lane, dst + c0, static_cast<int64_t>(p.h) * kDqk, v, p.scale, rows_valid);
                 }
             }
             ++n_acc;
@@ -1345,30 +1364,30 @@ cudaError_t configure_once_per_device(Kernel kernel, size_t smem_bytes, bool (&d
     return e;
 }
 
-cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mk, const BwdParams& p, int grid,
+cudaError_t HYDRA_K(launch_bwd_dq_from_ds)(const CUtensorMap& mk, const BwdParams& p, int grid,
                                   cudaStream_t stream)
 {
     static bool configured[64] = {};
-    if (cudaError_t e = configure_once_per_device(hydra_bwd_dq_from_ds_kernel, bwd_dq_ds_smem_bytes(), configured)) return e;
-    hydra_bwd_dq_from_ds_kernel<<<grid, dqs::kThreadsS, bwd_dq_ds_smem_bytes(), stream>>>(mk, p);
+    if (cudaError_t e = configure_once_per_device(HYDRA_K(hydra_bwd_dq_from_ds_kernel), HYDRA_K(bwd_dq_ds_smem_bytes)(), configured)) return e;
+    HYDRA_K(hydra_bwd_dq_from_ds_kernel)<<<grid, dqs::kThreadsS, HYDRA_K(bwd_dq_ds_smem_bytes)(), stream>>>(mk, p);
     return cudaGetLastError();
 }
 
-cudaError_t launch_bwd_dq(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+cudaError_t HYDRA_K(launch_bwd_dq)(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                           const CUtensorMap& mdo, const BwdParams& p, int grid, cudaStream_t stream)
 {
     static bool configured[64] = {};
-    if (cudaError_t e = configure_once_per_device(hydra_bwd_dq_kernel, bwd_dq_smem_bytes(), configured)) return e;
-    hydra_bwd_dq_kernel<<<grid, kThreads, bwd_dq_smem_bytes(), stream>>>(mq, mk, mv, mdo, p);
+    if (cudaError_t e = configure_once_per_device(HYDRA_K(hydra_bwd_dq_kernel), HYDRA_K(bwd_dq_smem_bytes)(), configured)) return e;
+    HYDRA_K(hydra_bwd_dq_kernel)<<<grid, kThreads, HYDRA_K(bwd_dq_smem_bytes)(), stream>>>(mq, mk, mv, mdo, p);
     return cudaGetLastError();
 }
 
-cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, const CUtensorMap& mv,
+cudaError_t HYDRA_K(launch_bwd_dkv)(const CUtensorMap& mq_sub, const CUtensorMap& mk, const CUtensorMap& mv,
                            const CUtensorMap& mdo_sub, const BwdParams& p, int grid, cudaStream_t stream)
 {
     static bool configured[64] = {};
-    if (cudaError_t e = configure_once_per_device(hydra_bwd_dkv_kernel, bwd_dkv_smem_bytes(), configured)) return e;
-    hydra_bwd_dkv_kernel<<<grid, kThreads, bwd_dkv_smem_bytes(), stream>>>(mq_sub, mk, mv, mdo_sub, p);
+    if (cudaError_t e = configure_once_per_device(HYDRA_K(hydra_bwd_dkv_kernel), HYDRA_K(bwd_dkv_smem_bytes)(), configured)) return e;
+    HYDRA_K(hydra_bwd_dkv_kernel)<<<grid, kThreads, HYDRA_K(bwd_dkv_smem_bytes)(), stream>>>(mq_sub, mk, mv, mdo_sub, p);
     return cudaGetLastError();
 }
 

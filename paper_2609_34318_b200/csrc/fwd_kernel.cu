@@ -30,22 +30,38 @@
 #include "hydra_internal.h"
 #include "sm100_ptx.cuh"
 
+// This file is compiled once per supported q / k head dimension (HYDRA_KERNEL_DQK = 192, the default, or
+// 128); the value dimension is 128 in both. HYDRA_K() gives the kernels and launchers of the second
+// build their own names.
+#ifndef HYDRA_KERNEL_DQK
+#define HYDRA_KERNEL_DQK 192
+#endif
+#if HYDRA_KERNEL_DQK == 192
+#define HYDRA_K(name) name
+#elif HYDRA_KERNEL_DQK == 128
+#define HYDRA_K(name) name##_d128
+#else
+#error "unsupported q / k head dimension"
+#endif
+
 namespace hydra {
 
 namespace {
 
+constexpr int kDqk = HYDRA_KERNEL_DQK;
+constexpr int kQkBoxes = kDqk / 64;                    // 64-column boxes of a q / k row
 constexpr int kThreads = 352;
 constexpr int kWarpK = 8, kWarpV = 9, kWarpMma = 10;
 constexpr uint32_t kBox = 128 * 128;                  // [128 rows x 64 bf16] = 16 KB
 constexpr uint32_t kHalfBox = 64 * 128;               // [ 64 rows x 64 bf16] =  8 KB
-constexpr uint32_t kQTile = 3 * kBox;                 // this CTA's 128 x 192 rows of a q tile
-constexpr uint32_t kKStage = 3 * kHalfBox;            // this CTA's 64 kv rows x 192
+constexpr uint32_t kQTile = kQkBoxes * kBox;          // this CTA's 128 rows of a q tile
+constexpr uint32_t kKStage = kQkBoxes * kHalfBox;     // this CTA's 64 kv rows of a k tile
 constexpr uint32_t kVStage = kBox;                    // 128 kv rows x this CTA's 64 value columns
 constexpr int kKStages = 3, kVStages = 3;
 constexpr uint32_t kSmemQ = 0;
 constexpr uint32_t kSmemK = kSmemQ + 2 * kQTile;
 constexpr uint32_t kSmemV = kSmemK + kKStages * kKStage;
-constexpr uint32_t kSmemTotal = kSmemV + kVStages * kVStage;  // 221,184 B
+constexpr uint32_t kSmemTotal = kSmemV + kVStages * kVStage;  // 221,184 B at d_qk = 192
 constexpr uint32_t kTmS = 0, kTmO = 256, kTmCols = 512;
 constexpr float kRescaleThreshold = 8.f;              // log2 units
 
@@ -61,10 +77,10 @@ __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); 
 
 }  // namespace
 
-size_t fwd_smem_bytes() { return kSmemTotal + 1024; }
+size_t HYDRA_K(fwd_smem_bytes)() { return kSmemTotal + 1024; }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+HYDRA_K(hydra_fwd_kernel)(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const __grid_constant__ CUtensorMap map_v, const FwdParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -154,12 +170,12 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                 const int n_t[2] = {item.n_a, item.n_b};
                 const int n = max(item.n_a, item.n_b);
                 auto load_q = [&](int t) {
-                    if (n_t[t] == 0 || !ok) return;
+                    if (n_t[t] <= 0 || !ok) return;
                     ok = wait(B_QEMPTY + t, q_use[t] ^ 1u);
                     if (!ok) return;
                     ++q_use[t];
                     if (leader) mbar_arrive_expect_tx(bar(B_QFULL + t), 2 * kQTile);
-                    for (int c = 0; c < 3; ++c)
+                    for (int c = 0; c < kQkBoxes; ++c)
                         tma_load_3d_pair(smem + kSmemQ + t * kQTile + c * kBox, &map_q, bar(B_QFULL + t), c * 64,
                                          item.head, pr.q_tok0 + item.q0 + t * 2 * TILE + rank * TILE);
                 };
@@ -169,7 +185,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     if (!ok) return;
                     ++gk;
                     if (leader) mbar_arrive_expect_tx(bar(B_KFULL + slot), 2 * kKStage);
-                    for (int c = 0; c < 3; ++c)
+                    for (int c = 0; c < kQkBoxes; ++c)
                         tma_load_3d_pair(smem + kSmemK + slot * kKStage + c * kHalfBox, &map_k, bar(B_KFULL + slot),
                                          c * 64, item.head / p.kv_group, pr.k_tok0 + j * TILE + rank * 64);
                 };
@@ -276,7 +292,7 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
                     if (do_s) {
                         const uint32_t b_lo = k_lo0 + k_slot * (kKStage >> 4);
 #pragma unroll
-                        for (int kk = 0; kk < D_QK / 16; ++kk)
+                        for (int kk = 0; kk < kDqk / 16; ++kk)
                             umma2_ss_w(d_s, q_lo[t] + (kk >> 2) * (kBox >> 4) + (kk & 3) * 2, hi_k,
                                        b_lo + (kk >> 2) * (kHalfBox >> 4) + (kk & 3) * 2, hi_k, idesc_s, kk != 0);
                         if ((t == 1) || (js >= n_t[1])) umma2_commit(bar(B_KEMPTY + k_slot));    // last reader
@@ -325,8 +341,8 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
             uint4* dst = reinterpret_cast<uint4*>(obase + (orow * p.h + item.head) * D_V);
             float* lse_dst = lbase + static_cast<int64_t>(item.head) * rows_total + orow;
 
-            if (n_kv == 0) {                           // rows that see no key: O = 0, LSE = -inf
-                if (row_valid) {
+            if (n_kv <= 0) {                           // rows that see no key: O = 0, LSE = -inf
+                if (row_valid && n_kv == 0) {           // (n_kv < 0: no such tile in this item)
 #pragma unroll
                     for (int e = 0; e < D_V / 8; ++e) dst[e] = make_uint4(0u, 0u, 0u, 0u);
                     *lse_dst = neg_inf();
@@ -483,32 +499,32 @@ hydra_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
 // Number of CTA pairs that can be resident at once (one CTA per SM): the size of the persistent grid.
 // Kept per device ordinal: the shared-memory opt-in applies to the device that is current when it is made.
-int fwd_max_clusters()
+int HYDRA_K(fwd_max_clusters)()
 {
     static int cached_by_device[64];
     static bool known[64] = {};
     int sms = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
     if (known[dev]) return cached_by_device[dev];
-    if (cudaFuncSetAttribute(hydra_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(fwd_smem_bytes())) != cudaSuccess)
+    if (cudaFuncSetAttribute(HYDRA_K(hydra_fwd_kernel), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(HYDRA_K(fwd_smem_bytes)())) != cudaSuccess)
         return 0;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(sms / 2 * 2));
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = fwd_smem_bytes();
+    cfg.dynamicSmemBytes = HYDRA_K(fwd_smem_bytes)();
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, hydra_fwd_kernel, &cfg) != cudaSuccess) n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, HYDRA_K(hydra_fwd_kernel), &cfg) != cudaSuccess) n = 0;
     cached_by_device[dev] = n;
     known[dev] = n > 0;
     return n;
 }
 
-cudaError_t launch_fwd(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+cudaError_t HYDRA_K(launch_fwd)(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                        const FwdParams& p, int n_clusters, cudaStream_t stream)
 {
-    hydra_fwd_kernel<<<2 * n_clusters, kThreads, fwd_smem_bytes(), stream>>>(mq, mk, mv, p);
+    HYDRA_K(hydra_fwd_kernel)<<<2 * n_clusters, kThreads, HYDRA_K(fwd_smem_bytes)(), stream>>>(mq, mk, mv, p);
     return cudaGetLastError();
 }
 

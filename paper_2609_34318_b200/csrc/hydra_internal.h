@@ -56,13 +56,13 @@ __host__ __device__ inline int64_t ds_rowstart(const DsGeom& g, int32_t jk)
 }
 constexpr uint32_t DS_BLOCK_BYTES = TILE * SUB * 2;   // 16 KB
 
-// Forward work item: a 256-row slab of q rows of one pair and head = tiles A and B of 128 rows.
+// Forward work item: up to 512 q rows of one pair and head = tiles A and B of 256 rows (128 per CTA of the pair).
 struct FwdItem {
     int32_t pair;
     int32_t head;
     int32_t q0;        // first q row of tile A, relative to the pair; tile B starts at q0 + 128
     int32_t n_a;       // kv tiles tile A visits (after causal clipping); 0: its rows see no key
-    int32_t n_b;       // same for tile B; 0 also when the slab has no second tile
+    int32_t n_b;       // same for tile B; -1 when the item has no second tile (its rows belong to another item)
     int32_t pad[3];
 };
 
@@ -164,20 +164,25 @@ struct MergeParams {
     int32_t accumulate;         // 1: the current (out, lse) rows are one more input of their merge
 };
 
-size_t fwd_smem_bytes();
-int fwd_max_clusters();
-size_t bwd_dq_smem_bytes();
-size_t bwd_dkv_smem_bytes();
-
-cudaError_t launch_fwd(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                       const FwdParams& p, int grid, cudaStream_t stream);
-cudaError_t launch_bwd_dq(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                          const CUtensorMap& mdo, const BwdParams& p, int grid, cudaStream_t stream);
-size_t bwd_dq_ds_smem_bytes();
-cudaError_t launch_bwd_dq_from_ds(const CUtensorMap& mk, const BwdParams& p, int grid,
-                                  cudaStream_t stream);
-cudaError_t launch_bwd_dkv(const CUtensorMap& mq_sub, const CUtensorMap& mk, const CUtensorMap& mv,
-                           const CUtensorMap& mdo_sub, const BwdParams& p, int grid, cudaStream_t stream);
+// The tensor-core kernels exist once per supported q / k head dimension (the kernel files are compiled
+// twice): the unsuffixed set for d_qk = 192, the _d128 set for d_qk = 128; d_v = 128 in both.
+#define HYDRA_DECLARE_KERNEL_SET(SUFFIX)                                                                              \
+    size_t fwd_smem_bytes##SUFFIX();                                                                                  \
+    int fwd_max_clusters##SUFFIX();                                                                                   \
+    size_t bwd_dq_smem_bytes##SUFFIX();                                                                               \
+    size_t bwd_dkv_smem_bytes##SUFFIX();                                                                              \
+    size_t bwd_dq_ds_smem_bytes##SUFFIX();                                                                            \
+    cudaError_t launch_fwd##SUFFIX(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,               \
+                                   const FwdParams& p, int grid, cudaStream_t stream);                                \
+    cudaError_t launch_bwd_dq##SUFFIX(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,            \
+                                      const CUtensorMap& mdo, const BwdParams& p, int grid, cudaStream_t stream);     \
+    cudaError_t launch_bwd_dq_from_ds##SUFFIX(const CUtensorMap& mk, const BwdParams& p, int grid,                    \
+                                              cudaStream_t stream);                                                   \
+    cudaError_t launch_bwd_dkv##SUFFIX(const CUtensorMap& mq_sub, const CUtensorMap& mk, const CUtensorMap& mv,       \
+                                       const CUtensorMap& mdo_sub, const BwdParams& p, int grid, cudaStream_t stream);
+HYDRA_DECLARE_KERNEL_SET()
+HYDRA_DECLARE_KERNEL_SET(_d128)
+#undef HYDRA_DECLARE_KERNEL_SET
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream);
 // launch_merge plus the library's launch counter and per-kernel timer (defined beside them, in api.cu)
 cudaError_t launch_merge_counted(const MergeParams& p, cudaStream_t stream);

@@ -452,3 +452,32 @@ def test_spike_backward_matches_full_backward_with_sparse_dout(lengths, rows):
     np.testing.assert_allclose(sk, dk2, rtol=1e-9, atol=1e-12 * np.abs(dk2).max())
     np.testing.assert_allclose(sv, dv2, rtol=1e-9, atol=1e-12 * np.abs(dv2).max())
     np.testing.assert_allclose(sq, dq2[rows], rtol=1e-9, atol=1e-12 * np.abs(dq2).max())
+
+
+def test_oracle_at_head_dimension_128_against_brute_force():
+    """The oracle takes its head dimensions from the arrays; heads of 128 / 128 (the grouped-query model's)
+    are pinned by the same dense numpy evaluation without max subtraction as 192 / 128."""
+    rng = np.random.default_rng(31)
+    lengths, h, d = [19, 40, 1], 2, 128
+    T = sum(lengths)
+    x = dict(q=rand_bits(rng, (T, h, d)), k=rand_bits(rng, (T, h, d)), v=rand_bits(rng, (T, h, d)),
+             do=rand_bits(rng, (T, h, d)), cu=hw.cu_seqlens(lengths))
+    sc = np.float32(1.0 / np.sqrt(np.float32(d)))
+    out, lse = oracle.attn_fwd(x["q"], x["k"], x["v"], x["cu"], True, sc)
+    dq, dk, dv = oracle.attn_bwd(x["q"], x["k"], x["v"], x["do"], x["cu"], True, sc, out, lse)
+    q, k, v, g = (hw.bf16_bits_to_f64(x[n]) for n in ("q", "k", "v", "do"))
+    for b in range(len(lengths)):
+        lo, hi = int(x["cu"][b]), int(x["cu"][b + 1])
+        L = hi - lo
+        for a in range(h):
+            S = float(sc) * q[lo:hi, a] @ k[lo:hi, a].T
+            E = np.exp(S) * np.tril(np.ones((L, L)))
+            P_ = E / E.sum(1, keepdims=True)
+            O = P_ @ v[lo:hi, a]
+            G = g[lo:hi, a]
+            dS = P_ * (G @ v[lo:hi, a].T - (G * O).sum(1, keepdims=True))
+            np.testing.assert_allclose(out[lo:hi, a], O, rtol=1e-12, atol=1e-14)
+            np.testing.assert_allclose(lse[a, lo:hi], np.log(E.sum(1)), rtol=1e-13)
+            np.testing.assert_allclose(dq[lo:hi, a], float(sc) * dS @ k[lo:hi, a], rtol=1e-10, atol=1e-13)
+            np.testing.assert_allclose(dk[lo:hi, a], float(sc) * dS.T @ q[lo:hi, a], rtol=1e-10, atol=1e-13)
+            np.testing.assert_allclose(dv[lo:hi, a], P_.T @ G, rtol=1e-10, atol=1e-13)
