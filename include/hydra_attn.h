@@ -388,10 +388,51 @@ int32_t hydra_ulysses_unpack(const void* recv, int64_t n_tokens, int32_t n_heads
                              void* y, void* cuda_stream);
 
 /*
+ * The elementwise steps of a gated multi-head-latent attention block that surround the attention kernel
+ * (Section 5.2, "Exposed All-to-All Overlap": the query's rotary embedding; the KV up-projection's output
+ * split into the value and the key's position-free part; the key's rotary embedding and concatenation; the
+ * gate). The paper names the steps and the order in which their results become final, not their formulas;
+ * the readings taken here:
+ *   rotary embedding  the columns [rope_offset, rope_offset + rope_dim) of every head are rotated in pairs
+ *                     (2i, 2i+1) by the angle positions[t] * theta^(-2i / rope_dim):
+ *                       y_2i = x_2i cos - x_2i+1 sin,  y_2i+1 = x_2i sin + x_2i+1 cos;
+ *                     positions[t] is the token's index inside its packed sequence; inverse != 0 rotates by
+ *                     the opposite angle, which is the backward of the step (a rotation's adjoint).
+ *   key / value       the up-projection emits, per token and head, [d_nope key columns | d_v value columns];
+ *                     the rotary part of the key is ONE vector of d_rope columns per token, shared by all
+ *                     heads: k[t, a, :] = [kv_up[t, a, 0:d_nope] | rope(k_pe[t, :])], v[t, a, :] =
+ *                     kv_up[t, a, d_nope:]. With d_nope = 128, d_rope = 64, d_v = 128 these are the
+ *                     [T, h, 192] / [T, h, 128] tensors hydra_attn_fwd takes. The backward is the adjoint:
+ *                     dkv_up = [dk[.., 0:d_nope] | dv], dk_pe[t, :] = rope^-1(sum_a dk[t, a, d_nope:]) (the sum
+ *                     over the heads in fp32, rounded once).
+ *   gate              y = out * sigmoid(gate), elementwise, gate being the gate projection's output with the
+ *                     shape of out; backward d_out = dy * sigmoid(gate), d_gate = dy * out * sigmoid(gate) *
+ *                     (1 - sigmoid(gate)).
+ * All tensors device bf16, positions device int32 [n_tokens]; arithmetic in fp32 (the rotary angle is formed
+ * and reduced in double precision), one rounding per output element. hydra_mla_rope may run in place (y == x);
+ * all other outputs must not alias inputs. Dimensions must be even, rope_dim <= 256, theta > 1; the gate
+ * takes n_elements % 8 == 0 and 16-byte aligned pointers (else HYDRA_ERR_INVALID_ARG). One launch each on
+ * cuda_stream, bound by HBM: every byte moves once.
+ */
+int32_t hydra_mla_rope(const void* x, const int32_t* positions, int64_t n_tokens, int32_t n_heads, int32_t head_dim,
+                       int32_t rope_offset, int32_t rope_dim, float theta, int32_t inverse, void* y,
+                       void* cuda_stream);
+int32_t hydra_mla_kv_assemble(const void* kv_up, const void* k_pe, const int32_t* positions, int64_t n_tokens,
+                              int32_t n_heads, int32_t d_nope, int32_t d_rope, int32_t d_v, float theta, void* k,
+                              void* v, void* cuda_stream);
+int32_t hydra_mla_kv_assemble_bwd(const void* dk, const void* dv, const int32_t* positions, int64_t n_tokens,
+                                  int32_t n_heads, int32_t d_nope, int32_t d_rope, int32_t d_v, float theta,
+                                  void* dkv_up, void* dk_pe, void* cuda_stream);
+int32_t hydra_gate_apply(const void* out, const void* gate, int64_t n_elements, void* y, void* cuda_stream);
+int32_t hydra_gate_apply_bwd(const void* dy, const void* out, const void* gate, int64_t n_elements, void* d_out,
+                             void* d_gate, void* cuda_stream);
+
+/*
  * Per-kernel timing (measurement aid, not part of the method). While enabled, every kernel launch
  * is bracketed by CUDA events on its stream. hydra_profile_collect waits for the recorded events,
- * adds their durations into ms_out[7] and their counts into launches_out[7] (index: 0 forward,
- * 1 merge, 2 backward prep, 3 backward dK/dV, 4 backward dQ, 5 gradient cast, 6 Ulysses pack / unpack)
+ * adds their durations into ms_out[8] and their counts into launches_out[8] (index: 0 forward,
+ * 1 merge, 2 backward prep, 3 backward dK/dV, 4 backward dQ, 5 gradient cast, 6 Ulysses pack / unpack,
+ * 7 the elementwise steps of the gated MLA block)
  * and forgets them.
  */
 void hydra_profile_enable(int32_t on);
@@ -458,6 +499,20 @@ int32_t hydra_version(void);
  * hydra_shutdown waits for the device and frees the arena, the cached tables and the pinned staging.
  */
 void hydra_set_plan_arena_bytes(uint64_t bytes);
+/*
+ * In training the forward of a problem is followed by its merge and its backward. hydra_attn_fwd therefore
+ * builds, on the host and right after it has launched its kernel, the work tables those calls will ask for
+ * (if they are not cached yet), so that this host work runs while the GPU computes the forward. Nothing is
+ * uploaded and no result changes. on = 0 switches it off (forward-only use); the default is on.
+ */
+void hydra_set_plan_prefetch(int32_t on);
+/*
+ * Host only (no GPU needed): seconds the host takes to build the work tables of one call of kind `which`
+ * (HYDRA_WS_FWD / MERGE / BWD) for this problem, uncached. What a new cu_seqlens costs before its first launch.
+ * Negative on invalid arguments.
+ */
+double hydra_plan_build_seconds(int32_t which, const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
+                                const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal);
 void hydra_shutdown(void);
 
 #if defined(__GNUC__)

@@ -59,6 +59,10 @@ def _load() -> ctypes.CDLL:
     lib.hydra_shutdown.restype = None
     lib.hydra_set_plan_arena_bytes.argtypes = [ctypes.c_uint64]
     lib.hydra_set_plan_arena_bytes.restype = None
+    lib.hydra_plan_build_seconds.restype = ctypes.c_double
+    lib.hydra_plan_build_seconds.argtypes = [i32, vp, i32, i32, vp, i32, i32]
+    lib.hydra_set_plan_prefetch.argtypes = [i32]
+    lib.hydra_set_plan_prefetch.restype = None
     lib.hydra_usp_factor.restype = i32
     lib.hydra_usp_factor.argtypes = [i32, i32, vp, vp]
     lib.hydra_zigzag_pairs.restype = i32
@@ -116,6 +120,15 @@ def _load() -> ctypes.CDLL:
         getattr(lib, name).argtypes = g[:10] + [i32, i32] + g[10:]
     lib.hydra_grad_cast.restype = i32
     lib.hydra_grad_cast.argtypes = [vp, vp, i64, vp]
+    lib.hydra_mla_rope.restype = i32
+    lib.hydra_mla_rope.argtypes = [vp, vp, i64, i32, i32, i32, i32, f32, i32, vp, vp]
+    for name in ("hydra_mla_kv_assemble", "hydra_mla_kv_assemble_bwd"):
+        getattr(lib, name).restype = i32
+        getattr(lib, name).argtypes = [vp, vp, vp, i64, i32, i32, i32, i32, f32, vp, vp, vp]
+    lib.hydra_gate_apply.restype = i32
+    lib.hydra_gate_apply.argtypes = [vp, vp, i64, vp, vp]
+    lib.hydra_gate_apply_bwd.restype = i32
+    lib.hydra_gate_apply_bwd.argtypes = [vp, vp, vp, i64, vp, vp, vp]
     lib.hydra_poll_status.restype = i32
     lib.hydra_poll_status.argtypes = [vp, vp, vp, vp]
     lib.hydra_poll_clocks.restype = i32
@@ -136,16 +149,17 @@ def _load() -> ctypes.CDLL:
 
 _lib = _load()
 LIBRARY_PATH = _build.OUT
-EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_set_wait_limit_ns", "hydra_debug_stall", "hydra_set_plan_arena_bytes",
+EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_set_wait_limit_ns", "hydra_debug_stall", "hydra_set_plan_arena_bytes", "hydra_set_plan_prefetch", "hydra_plan_build_seconds",
            "hydra_shutdown", "hydra_usp_factor", "hydra_zigzag_pairs", "hydra_workspace_bytes",
            "hydra_attn_fwd", "hydra_lse_merge", "hydra_attn_bwd", "hydra_poll_status",
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
            "hydra_attn_fwd_bwd_host", "hydra_lse_merge_noalloc", "hydra_lse_merge_accumulate",
            "hydra_sched_targets", "hydra_sched_cp", "hydra_sched_pack", "hydra_attn_bwd_accumulate",
            "hydra_grad_cast", "hydra_set_bwd_scratch_limit", "hydra_set_bwd_band_scratch", "hydra_bwd_bands", "hydra_ulysses_pack", "hydra_ulysses_unpack", "hydra_attn_fwd_gqa", "hydra_attn_bwd_accumulate_gqa", "hydra_attn_bwd_gqa", "hydra_workspace_bytes_gqa",
+           "hydra_mla_rope", "hydra_mla_kv_assemble", "hydra_mla_kv_assemble_bwd", "hydra_gate_apply", "hydra_gate_apply_bwd",
            "hydra_attn_fwd_dims", "hydra_attn_bwd_dims", "hydra_attn_bwd_accumulate_dims", "hydra_workspace_bytes_dims",
            "hydra_poll_clocks")
-KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast", "ulysses")
+KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast", "ulysses", "mla_ops")
 
 
 # ------------------------------------------------------------------------------------------------
@@ -235,6 +249,18 @@ def hydra_debug_stall(kernel: int, ns: int) -> None:
 
 def hydra_shutdown() -> None:
     _lib.hydra_shutdown()
+
+
+def hydra_plan_build_seconds(which: int, cu_seqlens, n_heads: int, pairs=None, causal: bool = True) -> float:
+    """Host-only: seconds to build the (uncached) work tables of one call of kind `which` for this problem."""
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    return float(_lib.hydra_plan_build_seconds(which, cu.ctypes.data, len(cu) - 1, n_heads, pp, npairs, int(bool(causal))))
+
+
+def hydra_set_plan_prefetch(on: bool) -> None:
+    """Build the merge / backward tables of a problem on the host while its forward runs (default on)."""
+    _lib.hydra_set_plan_prefetch(int(bool(on)))
 
 
 def hydra_set_plan_arena_bytes(nbytes: int) -> None:
@@ -489,6 +515,50 @@ def hydra_attn_bwd_accumulate_dims(q, k, v, out, lse, dout, cu_seqlens, n_heads:
     return _bwd_dims("hydra_attn_bwd_accumulate_dims", q, k, v, out, lse, dout, cu_seqlens, n_heads, n_kv_heads,
                      d_qk, d_v, pairs, causal, softmax_scale, dq_acc, dk_acc, dv_acc, workspace, workspace_bytes,
                      stream, check)
+
+
+def hydra_mla_rope(x, positions, n_tokens: int, n_heads: int, head_dim: int, rope_offset: int, rope_dim: int,
+                   theta: float, inverse: bool, y, stream=None, check: bool = True) -> int:
+    """Rotary embedding of columns [rope_offset, rope_offset + rope_dim) of every head (y may be x)."""
+    s = _lib.hydra_mla_rope(_ptr(x), _ptr(positions), int(n_tokens), n_heads, head_dim, rope_offset, rope_dim,
+                            ctypes.c_float(float(theta)), int(bool(inverse)), _ptr(y), _stream(stream))
+    if check:
+        _check(s, "hydra_mla_rope")
+    return s
+
+
+def hydra_mla_kv_assemble(kv_up, k_pe, positions, n_tokens: int, n_heads: int, d_nope: int, d_rope: int, d_v: int,
+                          theta: float, k, v, stream=None, check: bool = True) -> int:
+    """k = [key part of kv_up | rope(k_pe) shared by all heads], v = value part of kv_up."""
+    s = _lib.hydra_mla_kv_assemble(_ptr(kv_up), _ptr(k_pe), _ptr(positions), int(n_tokens), n_heads, d_nope, d_rope,
+                                   d_v, ctypes.c_float(float(theta)), _ptr(k), _ptr(v), _stream(stream))
+    if check:
+        _check(s, "hydra_mla_kv_assemble")
+    return s
+
+
+def hydra_mla_kv_assemble_bwd(dk, dv, positions, n_tokens: int, n_heads: int, d_nope: int, d_rope: int, d_v: int,
+                              theta: float, dkv_up, dk_pe, stream=None, check: bool = True) -> int:
+    s = _lib.hydra_mla_kv_assemble_bwd(_ptr(dk), _ptr(dv), _ptr(positions), int(n_tokens), n_heads, d_nope, d_rope,
+                                       d_v, ctypes.c_float(float(theta)), _ptr(dkv_up), _ptr(dk_pe), _stream(stream))
+    if check:
+        _check(s, "hydra_mla_kv_assemble_bwd")
+    return s
+
+
+def hydra_gate_apply(out, gate, n_elements: int, y, stream=None, check: bool = True) -> int:
+    s = _lib.hydra_gate_apply(_ptr(out), _ptr(gate), int(n_elements), _ptr(y), _stream(stream))
+    if check:
+        _check(s, "hydra_gate_apply")
+    return s
+
+
+def hydra_gate_apply_bwd(dy, out, gate, n_elements: int, d_out, d_gate, stream=None, check: bool = True) -> int:
+    s = _lib.hydra_gate_apply_bwd(_ptr(dy), _ptr(out), _ptr(gate), int(n_elements), _ptr(d_out), _ptr(d_gate),
+                                  _stream(stream))
+    if check:
+        _check(s, "hydra_gate_apply_bwd")
+    return s
 
 
 def hydra_set_bwd_scratch_limit(n_bytes: int) -> None:

@@ -2,13 +2,13 @@
 // with a small cache, tensor-map encoding and kernel launches.
 #include <algorithm>
 #include <atomic>
+#include <chrono>
 #include <cmath>
 #include <cstddef>
 #include <cstring>
 #include <map>
 #include <memory>
 #include <mutex>
-#include <queue>
 #include <vector>
 
 #include "hydra_internal.h"
@@ -25,7 +25,7 @@ constexpr size_t kStatusBytes = 256;
 // ---------------------------------------------------------------------------------------------
 // optional per-kernel timing with CUDA events on the launching stream
 // ---------------------------------------------------------------------------------------------
-enum KernelKind { K_FWD = 0, K_MERGE, K_PREP, K_DKV, K_DQ, K_CAST, K_ULYSSES, K_COUNT };
+enum KernelKind { K_FWD = 0, K_MERGE, K_PREP, K_DKV, K_DQ, K_CAST, K_ULYSSES, K_MLA, K_COUNT };
 struct ProfRecord { int kind; cudaEvent_t start, stop; };
 std::mutex g_prof_mutex;
 bool g_prof_on = false;
@@ -223,9 +223,13 @@ struct PlanArena {
     // other streams wait for it
     cudaEvent_t freed[2] = {nullptr, nullptr};
     cudaStream_t freed_on[2] = {nullptr, nullptr};
-    // pinned staging: a slot is reused once the copy that read it has completed
-    struct Slot { uint8_t* host = nullptr; size_t cap = 0; cudaEvent_t done = nullptr; bool used = false; };
-    static constexpr int kSlots = 16;
+    // pinned staging: a slot is reused once the copy that read it has completed. The slots are slices of one
+    // pinned allocation made with the arena (page-locking memory takes a fraction of a millisecond, too long
+    // for the first call of a new shape); tables larger than a slice get a pinned buffer of their own.
+    struct Slot { uint8_t* host = nullptr; size_t cap = 0; cudaEvent_t done = nullptr; bool used = false; bool own = false; };
+    static constexpr int kSlots = 8;
+    static constexpr size_t kSlotBytes = size_t{2} << 20;
+    uint8_t* stage_base = nullptr;
     Slot slots[kSlots];
     int next_slot = 0;
 };
@@ -246,10 +250,12 @@ void arena_release(PlanArena& a)                         // device idle, g_plan_
     for (cudaEvent_t e : a.spare_events) cudaEventDestroy(e);
     a.spare_events.clear();
     for (auto& sl : a.slots) {
-        if (sl.host) cudaFreeHost(sl.host);
+        if (sl.host && sl.own) cudaFreeHost(sl.host);
         if (sl.done) cudaEventDestroy(sl.done);
         sl = PlanArena::Slot{};
     }
+    if (a.stage_base) cudaFreeHost(a.stage_base);
+    a.stage_base = nullptr;
 }
 
 // Makes the tables of `plan` resident on the current device and returns their address. g_plan_mutex held.
@@ -265,6 +271,15 @@ int32_t arena_place(Plan& plan, int device, cudaStream_t stream, const uint8_t**
         a.half_bytes = half;
         a.epoch[0] = a.next_epoch++;
         a.epoch[1] = a.next_epoch++;
+        void* hp = nullptr;
+        if (cudaHostAlloc(&hp, PlanArena::kSlots * PlanArena::kSlotBytes, cudaHostAllocDefault) != cudaSuccess)
+            return HYDRA_ERR_CUDA;
+        a.stage_base = static_cast<uint8_t*>(hp);
+        for (int i = 0; i < PlanArena::kSlots; ++i) {
+            a.slots[i].host = a.stage_base + i * PlanArena::kSlotBytes;
+            a.slots[i].cap = PlanArena::kSlotBytes;
+            if (cudaEventCreateWithFlags(&a.slots[i].done, cudaEventDisableTiming) != cudaSuccess) return HYDRA_ERR_CUDA;
+        }
     }
     if (plan.half >= 0 && plan.epoch == a.epoch[plan.half]) {
         // resident; a stream other than the one that carried the copy waits for the copy (free once complete)
@@ -297,19 +312,19 @@ int32_t arena_place(Plan& plan, int device, cudaStream_t stream, const uint8_t**
     const int half = a.active;
     if (a.freed[half] && a.freed_on[half] != stream && cudaStreamWaitEvent(stream, a.freed[half], 0) != cudaSuccess)
         return HYDRA_ERR_CUDA;
-    // staging slot: pinned, reused once the copy that read it has completed (sixteen uploads ago, so the host
-    // may run several micro-batches ahead of the device before this ever waits)
+    // staging slot: pinned, reused once the copy that read it has completed (eight uploads ago, so the host
+    // may run two micro-batches ahead of the device before this ever waits)
     PlanArena::Slot& sl = a.slots[a.next_slot];
     a.next_slot = (a.next_slot + 1) % PlanArena::kSlots;
     if (sl.used && cudaEventSynchronize(sl.done) != cudaSuccess) return HYDRA_ERR_CUDA;
-    if (sl.cap < need) {
-        if (sl.host) cudaFreeHost(sl.host);
-        sl.host = nullptr; sl.cap = 0;
-        const size_t cap = std::max<size_t>(need, size_t{256} << 10);
+    if (sl.cap < need) {                                 // rare: tables of more than 2 MB
+        if (sl.host && sl.own) cudaFreeHost(sl.host);
+        sl.host = nullptr; sl.cap = 0; sl.own = false;
         void* hp = nullptr;
-        if (cudaHostAlloc(&hp, cap, cudaHostAllocDefault) != cudaSuccess) return HYDRA_ERR_CUDA;
+        if (cudaHostAlloc(&hp, need, cudaHostAllocDefault) != cudaSuccess) return HYDRA_ERR_CUDA;
         sl.host = static_cast<uint8_t*>(hp);
-        sl.cap = cap;
+        sl.cap = need;
+        sl.own = true;
     }
     if (!sl.done && cudaEventCreateWithFlags(&sl.done, cudaEventDisableTiming) != cudaSuccess) return HYDRA_ERR_CUDA;
     if (!plan.uploaded && cudaEventCreateWithFlags(&plan.uploaded, cudaEventDisableTiming) != cudaSuccess)
@@ -415,80 +430,145 @@ template <class Item>
 void order_items(std::vector<Item>& items, const std::vector<int32_t>& block_of, const std::vector<int32_t>& cost,
                  int workers)
 {
+    const size_t n = items.size();
     int32_t n_blocks = 0;
     for (int32_t b : block_of) n_blocks = std::max(n_blocks, b + 1);
     std::vector<int64_t> block_cost(n_blocks, 0);
-    for (size_t i = 0; i < items.size(); ++i) block_cost[block_of[i]] += cost[i];
-    std::vector<Keyed> k(items.size());
-    for (size_t i = 0; i < items.size(); ++i)
-        k[i] = Keyed{block_cost[block_of[i]], block_of[i], cost[i], static_cast<int32_t>(i)};
-    // ascending by cost: the candidates for the tail
-    std::vector<int32_t> asc(items.size());
-    for (size_t i = 0; i < items.size(); ++i) asc[i] = static_cast<int32_t>(i);
-    std::sort(asc.begin(), asc.end(), [&](int32_t a, int32_t b) {
-        return cost[a] != cost[b] ? cost[a] < cost[b] : a > b;
+    for (size_t i = 0; i < n; ++i) block_cost[block_of[i]] += cost[i];
+    // the block order, sorted once; a trial order is this one with its tail items taken out and appended
+    std::vector<Keyed> base(n);
+    for (size_t i = 0; i < n; ++i)
+        base[i] = Keyed{block_cost[block_of[i]], block_of[i], cost[i], static_cast<int32_t>(i)};
+    std::sort(base.begin(), base.end(), [](const Keyed& a, const Keyed& b) {
+        if (a.block_cost != b.block_cost) return a.block_cost > b.block_cost;
+        if (a.block != b.block) return a.block < b.block;
+        if (a.cost != b.cost) return a.cost > b.cost;
+        return a.idx < b.idx;
     });
+    // ascending by cost: the candidates for the tail (sorted only if a tail is tried at all)
+    std::vector<int32_t> asc;
     int32_t longest = 0;
     int64_t total = 0;
     for (int32_t c : cost) { longest = std::max(longest, c); total += c + kItemOverhead; }
     // the order with a tail worth `want` units of work
+    std::vector<uint8_t> in_tail(n);
     auto ordered = [&](int64_t want) {
-        std::vector<uint8_t> in_tail(items.size(), 0);
+        if (asc.empty()) {
+            asc.resize(n);
+            for (size_t i = 0; i < n; ++i) asc[i] = static_cast<int32_t>(i);
+            std::sort(asc.begin(), asc.end(), [&](int32_t a, int32_t b) {
+                return cost[a] != cost[b] ? cost[a] < cost[b] : a > b;
+            });
+        }
+        std::fill(in_tail.begin(), in_tail.end(), 0);
+        std::vector<Keyed> tail;
         int64_t have = 0;
         for (int32_t i : asc) {
             if (have >= want) break;
             in_tail[i] = 1;
             have += cost[i] + kItemOverhead;
+            tail.push_back(Keyed{block_cost[block_of[i]], block_of[i], cost[i], i});
         }
-        std::vector<Keyed> o = k;
-        std::sort(o.begin(), o.end(), [&](const Keyed& a, const Keyed& b) {
-            if (in_tail[a.idx] != in_tail[b.idx]) return in_tail[a.idx] < in_tail[b.idx];
-            if (in_tail[a.idx]) {
-                if (a.cost != b.cost) return a.cost > b.cost;
-                if (a.block != b.block) return a.block < b.block;
-                return a.idx < b.idx;
-            }
-            if (a.block_cost != b.block_cost) return a.block_cost > b.block_cost;
-            if (a.block != b.block) return a.block < b.block;
+        std::sort(tail.begin(), tail.end(), [](const Keyed& a, const Keyed& b) {
             if (a.cost != b.cost) return a.cost > b.cost;
+            if (a.block != b.block) return a.block < b.block;
             return a.idx < b.idx;
         });
+        std::vector<Keyed> o;
+        o.reserve(n);
+        for (const Keyed& e : base)
+            if (!in_tail[e.idx]) o.push_back(e);
+        o.insert(o.end(), tail.begin(), tail.end());
         return o;
     };
-    // when the last worker ends if the workers pop the items in this order (time = cost + a fixed part)
+    // When the last worker ends if the workers pop the items in this order (time = cost + a fixed part). Times
+    // are small integers and an item always starts at the earliest free time, which never decreases, so the
+    // workers' free times live in a calendar (count of workers per time value) with a cursor that only moves
+    // forward: O(items + end time), a few nanoseconds per item (a heap cost 1 ms for the 8000 items of the
+    // 32K workload's backward, as long as the kernels of the step). List scheduling ends within one longest
+    // item of the even share, which bounds the calendar.
+    const int64_t even = (total + workers - 1) / workers;
+    std::vector<int32_t> calendar(static_cast<size_t>(even + longest + kItemOverhead + 2));
     auto makespan = [&](const std::vector<Keyed>& o) {
-        std::priority_queue<int64_t, std::vector<int64_t>, std::greater<int64_t>> free_at;
-        for (int w = 0; w < workers; ++w) free_at.push(0);
+        std::fill(calendar.begin(), calendar.end(), 0);
+        calendar[0] = workers;
+        size_t now = 0;
         int64_t end = 0;
         for (const Keyed& e : o) {
-            const int64_t t = free_at.top() + e.cost + kItemOverhead;
-            free_at.pop();
-            free_at.push(t);
-            end = std::max(end, t);
+            while (calendar[now] == 0) ++now;
+            --calendar[now];
+            const size_t t = now + static_cast<size_t>(e.cost + kItemOverhead);
+            ++calendar[t];
+            end = std::max<int64_t>(end, static_cast<int64_t>(t));
         }
         return end;
     };
     // Taking items out of their blocks costs locality (measured: -5 % on workloads of many short sequences
     // when a tail was always cut), so the smallest tail that brings the simulated end within 5 % of the
     // even share is taken, and none if the block order already gets there.
-    const int64_t even = (total + workers - 1) / workers;
     const int64_t full_tail = static_cast<int64_t>(workers) * (longest + kItemOverhead);
-    k = ordered(0);
+    std::vector<Keyed> k = base;
     int64_t best = makespan(k);
     for (int step = 1; step <= 4 && best * 100 > even * 105; ++step) {
         std::vector<Keyed> o = ordered(full_tail * step / 4);
         const int64_t m = makespan(o);
         if (m < best) { best = m; k.swap(o); }
     }
-    std::vector<Item> sorted(items.size());
-    for (size_t i = 0; i < items.size(); ++i) sorted[i] = items[k[i].idx];
+    std::vector<Item> sorted(n);
+    for (size_t i = 0; i < n; ++i) sorted[i] = items[k[i].idx];
     items.swap(sorted);
+}
+
+// The items of a plan come in groups (a pair, or a chunk) that repeat for every head with the same costs, so
+// the block order above (blocks = (group, head), longest block first, the items of a block longest first)
+// needs only the GROUPS sorted, and the list is then written out in one pass. That matters because a
+// training loop meets new cu_seqlens with every micro-batch: sorting the 22 000 items of the many-short
+// workload took milliseconds on the host, as long as the kernels they feed. List scheduling ends within one
+// longest item of the even share, so when the longest item is under 5 % of that share the block order needs
+// no check; only otherwise (few, long, equal sequences: few items) is the queue simulated as above.
+struct GroupEntry { int32_t a, b, c, cost; };
+template <class Item, class Make>
+std::vector<Item> order_by_groups(std::vector<std::vector<GroupEntry>>& groups, int32_t h, int workers, Make make)
+{
+    std::vector<int64_t> group_cost(groups.size(), 0);
+    int64_t total = 0, n_items = 0;
+    int32_t longest = 0;
+    for (size_t g = 0; g < groups.size(); ++g) {
+        std::stable_sort(groups[g].begin(), groups[g].end(),
+                         [](const GroupEntry& x, const GroupEntry& y) { return x.cost > y.cost; });
+        for (const GroupEntry& e : groups[g]) {
+            group_cost[g] += e.cost;
+            total += static_cast<int64_t>(e.cost + kItemOverhead) * h;
+            longest = std::max(longest, e.cost);
+        }
+        n_items += static_cast<int64_t>(groups[g].size()) * h;
+    }
+    std::vector<int32_t> order(groups.size());
+    for (size_t g = 0; g < groups.size(); ++g) order[g] = static_cast<int32_t>(g);
+    std::sort(order.begin(), order.end(), [&](int32_t x, int32_t y) {
+        return group_cost[x] != group_cost[y] ? group_cost[x] > group_cost[y] : x < y;
+    });
+    std::vector<Item> items;
+    items.reserve(static_cast<size_t>(n_items));
+    const int64_t even = (total + workers - 1) / workers;
+    const bool settled = static_cast<int64_t>(longest + kItemOverhead) * 20 <= even;
+    std::vector<int32_t> block_of, cost;
+    for (int32_t g : order)
+        for (int32_t a = 0; a < h; ++a)
+            for (const GroupEntry& e : groups[g]) {
+                items.push_back(make(g, a, e));
+                if (!settled) {
+                    block_of.push_back(g * h + a);
+                    cost.push_back(e.cost);
+                }
+            }
+    if (!settled) order_items(items, block_of, cost, workers);
+    return items;
 }
 
 void build_fwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& blob)
 {
-    std::vector<FwdItem> items;
-    std::vector<int32_t> block_of, cost;
+    std::vector<std::vector<GroupEntry>> groups(pb.pairs.size());
     for (size_t pi = 0; pi < pb.pairs.size(); ++pi) {
         const auto& p = pb.pairs[pi];
         // One item = two consecutive 256-row UMMA tiles (A, then B) of a CTA pair. The slabs are aligned to
@@ -503,18 +583,16 @@ void build_fwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& 
             const int32_t n_a = kv_tiles(p, qa, causal, 2 * TILE);
             // n_b = -1: the item has no second tile (0 would mean: a tile whose rows see no key)
             const int32_t n_b = (!lone && qa + 2 * TILE < p.q_len) ? kv_tiles(p, qa + 2 * TILE, causal, 2 * TILE) : -1;
-            for (int32_t a = 0; a < pb.h; ++a) {
-                items.push_back(FwdItem{static_cast<int32_t>(pi), a, qa, n_a, n_b, {0, 0, 0}});
-                block_of.push_back(static_cast<int32_t>(pi) * pb.h + a);
-                // the two tiles advance in lockstep (one kv tile each per step of the issue order), so
-                // the time of an item goes with the longer tile, not with the sum: a slab whose second
-                // tile is empty costs as much per kv tile as a full one (measured: with the sum the
-                // slowest cluster of the 32K packed workload ended 17 % after the mean, now 4 %)
-                cost.push_back(2 * std::max(n_a, std::max(n_b, 0)));
-            }
+            // the two tiles advance in lockstep (one kv tile each per step of the issue order), so the time
+            // of an item goes with the longer tile, not with the sum: a slab whose second tile is empty costs
+            // as much per kv tile as a full one (measured: with the sum the slowest cluster of the 32K packed
+            // workload ended 17 % after the mean, now 4 %)
+            groups[pi].push_back(GroupEntry{qa, n_a, n_b, 2 * std::max(n_a, std::max(n_b, 0))});
         }
     }
-    order_items(items, block_of, cost, plan_workers(2));
+    const std::vector<FwdItem> items = order_by_groups<FwdItem>(
+        groups, pb.h, plan_workers(2),
+        [](int32_t g, int32_t a, const GroupEntry& e) { return FwdItem{g, a, e.a, e.b, e.c, {0, 0, 0}}; });
     plan.off_pairs = append(blob, device_pairs(pb));
     plan.off_items = append(blob, items);
     plan.n_items = static_cast<int32_t>(items.size());
@@ -582,8 +660,8 @@ void build_bwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& 
         };
         std::stable_sort(order.begin(), order.end(),
                          [&](int32_t a, int32_t b) { return range_less(key(a), key(b)); });
-        std::vector<int32_t> block_of, cost;
-        int32_t block = 0;
+        std::vector<std::vector<GroupEntry>> groups;       // one per chunk that has work
+        std::vector<std::pair<int32_t, int32_t>> list_of;  // its (list_off, list_len)
         int32_t i = 0;
         while (i < n) {
             int32_t j = i;
@@ -601,6 +679,8 @@ void build_bwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& 
             }
             const int32_t list_len = static_cast<int32_t>(lists.size()) - list_off;
             if (r.len > 0 && list_len > 0) {
+                groups.emplace_back();
+                list_of.emplace_back(list_off, list_len);
                 for (int32_t r0 = 0; r0 < r.len; r0 += TILE) {
                     int32_t c = 0;
                     for (int32_t t = 0; t < list_len; ++t) {
@@ -617,17 +697,14 @@ void build_bwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& 
                             c += std::max(0, n_sub - first);
                         }
                     }
-                    for (int32_t a = 0; a < pb.h; ++a) {
-                        items.push_back(GroupItem{list_off, list_len, a, r0});
-                        block_of.push_back(block * pb.h + a);
-                        cost.push_back(c);
-                    }
+                    groups.back().push_back(GroupEntry{r0, 0, 0, c});
                 }
-                ++block;
             }
             i = j;
         }
-        order_items(items, block_of, cost, plan_workers(1));
+        items = order_by_groups<GroupItem>(groups, pb.h, plan_workers(1), [&](int32_t g, int32_t a, const GroupEntry& e) {
+            return GroupItem{list_of[g].first, list_of[g].second, a, e.a};
+        });
     };
     std::vector<int32_t> lists_q, lists_k;
     std::vector<GroupItem> items_q, items_k;
@@ -652,10 +729,12 @@ public:
     PlanLease() = default;
     PlanLease(const PlanLease&) = delete;
     PlanLease& operator=(const PlanLease&) = delete;
-    ~PlanLease()
+    ~PlanLease() { release(); }
+    void release()
     {
         if (!lock_.owns_lock()) return;
         if (plan_) arena_note_use(*plan_, device_, stream_);
+        lock_.unlock();
     }
     // Finds the plan (building it on the host the first time) and makes its tables resident.
     int32_t acquire(int kind, const Problem& pb, int causal, cudaStream_t stream);
@@ -671,36 +750,54 @@ private:
     cudaStream_t stream_ = nullptr;
 };
 
+// The cached plan of a problem, built on the host if it is new. g_plan_mutex held.
+std::shared_ptr<Plan> find_or_build_plan(int kind, int device, const Problem& pb, int causal)
+{
+    std::vector<uint8_t> key = make_key(kind, device, pb, causal);
+    for (size_t i = 0; i < g_plans.size(); ++i)
+        if (g_plans[i]->key == key) {
+            if (i + 1 != g_plans.size()) std::rotate(g_plans.begin() + i, g_plans.begin() + i + 1, g_plans.end());
+            return g_plans.back();
+        }
+    auto plan = std::make_shared<Plan>();
+    plan->kind = kind;
+    plan->device = device;
+    if (kind == HYDRA_WS_FWD) build_fwd(pb, causal, *plan, plan->blob);
+    else if (kind == HYDRA_WS_MERGE) build_merge(pb, *plan, plan->blob);
+    else build_bwd(pb, causal, *plan, plan->blob);
+    plan->key.swap(key);
+    if (g_plans.size() >= kMaxPlans) {
+        // an evicted plan that owns device memory frees it: drain the device first (arena plans own none)
+        if (g_plans.front()->own.ptr) cudaDeviceSynchronize();
+        g_plans.erase(g_plans.begin());
+    }
+    g_plans.push_back(plan);
+    return plan;
+}
+
 int32_t PlanLease::acquire(int kind, const Problem& pb, int causal, cudaStream_t stream)
 {
     if (cudaGetDevice(&device_) != cudaSuccess || device_ < 0 || device_ >= 64) return HYDRA_ERR_CUDA;
     stream_ = stream;
-    std::vector<uint8_t> key = make_key(kind, device_, pb, causal);
     lock_ = std::unique_lock<std::mutex>(g_plan_mutex);
-    for (size_t i = 0; i < g_plans.size(); ++i)
-        if (g_plans[i]->key == key) {
-            if (i + 1 != g_plans.size()) std::rotate(g_plans.begin() + i, g_plans.begin() + i + 1, g_plans.end());
-            plan_ = g_plans.back();
-            break;
-        }
-    if (!plan_) {
-        auto plan = std::make_shared<Plan>();
-        plan->kind = kind;
-        plan->device = device_;
-        if (kind == HYDRA_WS_FWD) build_fwd(pb, causal, *plan, plan->blob);
-        else if (kind == HYDRA_WS_MERGE) build_merge(pb, *plan, plan->blob);
-        else build_bwd(pb, causal, *plan, plan->blob);
-        plan->key.swap(key);
-        if (g_plans.size() >= kMaxPlans) {
-            // an evicted plan that owns device memory frees it: drain the device first (arena plans own none)
-            if (g_plans.front()->own.ptr) cudaDeviceSynchronize();
-            g_plans.erase(g_plans.begin());
-        }
-        g_plans.push_back(plan);
-        plan_ = std::move(plan);
-    }
+    plan_ = find_or_build_plan(kind, device_, pb, causal);
     if (int32_t s = arena_place(*plan_, device_, stream, &tables_)) { plan_.reset(); return s; }
     return HYDRA_OK;
+}
+
+// A forward of a new problem is followed, in training, by the merge and the backward of the same problem:
+// their tables are built on the host right after the forward kernel has been launched, while the GPU runs
+// it, instead of when their own calls arrive and the GPU has nothing to do (host work only: nothing is
+// uploaded). hydra_set_plan_prefetch(0) switches this off for forward-only use.
+std::atomic<int> g_plan_prefetch{1};
+void prefetch_plans(const Problem& pb, int causal, bool any_part)
+{
+    if (!g_plan_prefetch.load()) return;
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return;
+    std::lock_guard<std::mutex> lock(g_plan_mutex);
+    if (any_part) find_or_build_plan(HYDRA_WS_MERGE, device, pb, 0);
+    find_or_build_plan(HYDRA_WS_BWD, device, pb, causal);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -880,6 +977,22 @@ void hydra_shutdown(void)
 }
 
 void hydra_set_plan_arena_bytes(uint64_t bytes) { g_arena_bytes.store(bytes); }
+
+void hydra_set_plan_prefetch(int32_t on) { g_plan_prefetch.store(on != 0); }
+
+double hydra_plan_build_seconds(int32_t which, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                                const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal)
+{
+    Problem pb;
+    if (make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb) != HYDRA_OK) return -1.0;
+    Plan plan;
+    const auto t0 = std::chrono::steady_clock::now();
+    if (which == HYDRA_WS_FWD) build_fwd(pb, causal != 0, plan, plan.blob);
+    else if (which == HYDRA_WS_MERGE) build_merge(pb, plan, plan.blob);
+    else if (which == HYDRA_WS_BWD) build_bwd(pb, causal != 0, plan, plan.blob);
+    else return -1.0;
+    return std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count();
+}
 
 int32_t hydra_usp_factor(int32_t degree, int32_t heads, int32_t* cp_u, int32_t* cp_r)
 {
@@ -1105,6 +1218,8 @@ int32_t hydra_attn_fwd_dims(const void* q, const void* k, const void* v, const i
         if (ks->launch_fwd(mq, mk, mv, fp, n_clusters, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
     }
     g_launches += 1;
+    lease.release();                                   // the tables have their reader on record
+    prefetch_plans(pb, causal != 0, any_part);
     return HYDRA_OK;
 }
 
@@ -1326,6 +1441,26 @@ std::vector<std::vector<hydra_pair_t>> make_bands(const Problem& pb, int32_t cau
     return bands;
 }
 
+// Token rows [first, end) that the listed ranges cover, sorted, with ranges that touch or overlap joined: a
+// packed batch whose chunks tile its sequences is one run, so a cast over it is one launch (a batch of 230
+// short sequences used to take 460 launches of a few microseconds each).
+std::vector<std::pair<size_t, size_t>> covered_rows(const Problem& pb, bool key_side)
+{
+    std::vector<std::pair<size_t, size_t>> rows;
+    for (const auto& p : pb.pairs) {
+        if (p.q_len <= 0 || p.k_len <= 0) continue;
+        const size_t first = static_cast<size_t>(pb.cu[p.seq]) + (key_side ? p.k_start : p.q_start);
+        rows.emplace_back(first, first + static_cast<size_t>(key_side ? p.k_len : p.q_len));
+    }
+    std::sort(rows.begin(), rows.end());
+    std::vector<std::pair<size_t, size_t>> runs;
+    for (const auto& r : rows) {
+        if (!runs.empty() && r.first <= runs.back().second) runs.back().second = std::max(runs.back().second, r.second);
+        else runs.push_back(r);
+    }
+    return runs;
+}
+
 int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, const float* lse,
                  const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
                  const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
@@ -1374,19 +1509,14 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
         if (int32_t s = bwd_run(pb, n_kv_heads, causal, softmax_scale, tg, false, true, workspace,
                                 ws + ds_off + kv_bytes, room - kv_bytes, g_ds_limit_bytes.load(), true, sms, stream))
             return s;
-        std::vector<Range> rs;
-        for (const auto& p : pb.pairs)
-            if (p.q_len > 0 && p.k_len > 0) rs.push_back(Range{p.seq, p.k_start, p.k_len});
-        std::sort(rs.begin(), rs.end(), range_less);
-        for (size_t i = 0; i < rs.size(); ++i) {
-            if (i > 0 && rs[i].seq == rs[i - 1].seq && rs[i].start == rs[i - 1].start) continue;
-            const size_t row = static_cast<size_t>(pb.cu[rs[i].seq]) + rs[i].start;
-            const size_t rk = static_cast<size_t>(n_kv_heads) * pb.dqk, rv = static_cast<size_t>(n_kv_heads) * D_V;
+        const size_t rk = static_cast<size_t>(n_kv_heads) * pb.dqk, rv = static_cast<size_t>(n_kv_heads) * D_V;
+        for (const auto& run : covered_rows(pb, true)) {
+            const size_t row = run.first, n = run.second - run.first;
             ScopedKernelTimer timer(K_CAST, stream);
             if (launch_grad_cast(dk_acc + row * rk, static_cast<uint16_t*>(dk) + row * rk,
-                                 static_cast<int64_t>(rs[i].len) * rk, stream) != cudaSuccess ||
+                                 static_cast<int64_t>(n * rk), stream) != cudaSuccess ||
                 launch_grad_cast(dv_acc + row * rv, static_cast<uint16_t*>(dv) + row * rv,
-                                 static_cast<int64_t>(rs[i].len) * rv, stream) != cudaSuccess)
+                                 static_cast<int64_t>(n * rv), stream) != cudaSuccess)
                 return HYDRA_ERR_CUDA;
             g_launches += 2;
         }
@@ -1421,17 +1551,12 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
                 }
                 // round the query rows the pairs cover; rows outside every pair stay untouched, as in
                 // the one-shot form
-                std::vector<Range> rs;
-                for (const auto& p : pb.pairs)
-                    if (p.q_len > 0 && p.k_len > 0) rs.push_back(Range{p.seq, p.q_start, p.q_len});
-                std::sort(rs.begin(), rs.end(), range_less);
                 const size_t per_row = static_cast<size_t>(n_heads) * pb.dqk;
-                for (size_t i = 0; i < rs.size(); ++i) {
-                    if (i > 0 && rs[i].seq == rs[i - 1].seq && rs[i].start == rs[i - 1].start) continue;
-                    const size_t row = static_cast<size_t>(pb.cu[rs[i].seq]) + rs[i].start;
+                for (const auto& run : covered_rows(pb, false)) {
+                    const size_t row = run.first, n = run.second - run.first;
                     ScopedKernelTimer timer(K_CAST, stream);
                     if (launch_grad_cast(dq_acc + row * per_row, static_cast<uint16_t*>(dq) + row * per_row,
-                                         static_cast<int64_t>(rs[i].len) * per_row, stream) != cudaSuccess)
+                                         static_cast<int64_t>(n * per_row), stream) != cudaSuccess)
                         return HYDRA_ERR_CUDA;
                     g_launches += 1;
                 }
@@ -1734,6 +1859,104 @@ int32_t hydra_ulysses_unpack(const void* recv, int64_t n_tokens, int32_t n_heads
                              void* y, void* cuda_stream)
 {
     return ulysses_impl(false, recv, n_tokens, n_heads, head_dim, cp_u, y, cuda_stream);
+}
+
+namespace {
+bool rope_shape_ok(int32_t head_dim, int32_t rope_offset, int32_t rope_dim)
+{
+    return head_dim >= 2 && head_dim % 2 == 0 && rope_offset >= 0 && rope_offset % 2 == 0 && rope_dim >= 2 &&
+           rope_dim % 2 == 0 && rope_dim <= 256 && rope_offset + rope_dim <= head_dim;
+}
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+}  // namespace
+
+int32_t hydra_mla_rope(const void* x, const int32_t* positions, int64_t n_tokens, int32_t n_heads, int32_t head_dim,
+                       int32_t rope_offset, int32_t rope_dim, float theta, int32_t inverse, void* y, void* cuda_stream)
+{
+    if (n_tokens < 0 || n_heads < 1 || !rope_shape_ok(head_dim, rope_offset, rope_dim) || !(theta > 1.f) ||
+        !std::isfinite(theta))
+        return HYDRA_ERR_INVALID_ARG;
+    if (n_tokens == 0) return HYDRA_OK;
+    if (!x || !y || !positions || !aligned4(x) || !aligned4(y) || !aligned4(positions)) return HYDRA_ERR_INVALID_ARG;
+    if (int32_t s = device_info(nullptr)) return s;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ScopedKernelTimer timer(K_MLA, stream);
+    if (launch_rope(x, positions, y, n_tokens, n_heads, head_dim, rope_offset, rope_dim, theta, inverse != 0, stream) !=
+        cudaSuccess)
+        return HYDRA_ERR_CUDA;
+    g_launches += 1;
+    return HYDRA_OK;
+}
+
+int32_t hydra_mla_kv_assemble(const void* kv_up, const void* k_pe, const int32_t* positions, int64_t n_tokens,
+                              int32_t n_heads, int32_t d_nope, int32_t d_rope, int32_t d_v, float theta, void* k, void* v,
+                              void* cuda_stream)
+{
+    if (n_tokens < 0 || n_heads < 1 || d_nope < 2 || d_nope % 2 || d_v < 2 || d_v % 2 ||
+        !rope_shape_ok(d_rope, 0, d_rope) || !(theta > 1.f) || !std::isfinite(theta))
+        return HYDRA_ERR_INVALID_ARG;
+    if (n_tokens == 0) return HYDRA_OK;
+    const void* ptrs[] = {kv_up, k_pe, positions, k, v};
+    for (const void* p : ptrs)
+        if (!p || !aligned4(p)) return HYDRA_ERR_INVALID_ARG;
+    if (int32_t s = device_info(nullptr)) return s;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ScopedKernelTimer timer(K_MLA, stream);
+    if (launch_mla_kv_assemble(kv_up, k_pe, positions, k, v, n_tokens, n_heads, d_nope, d_rope, d_v, theta, stream) !=
+        cudaSuccess)
+        return HYDRA_ERR_CUDA;
+    g_launches += 1;
+    return HYDRA_OK;
+}
+
+int32_t hydra_mla_kv_assemble_bwd(const void* dk, const void* dv, const int32_t* positions, int64_t n_tokens,
+                                  int32_t n_heads, int32_t d_nope, int32_t d_rope, int32_t d_v, float theta, void* dkv_up,
+                                  void* dk_pe, void* cuda_stream)
+{
+    if (n_tokens < 0 || n_heads < 1 || d_nope < 2 || d_nope % 2 || d_v < 2 || d_v % 2 ||
+        !rope_shape_ok(d_rope, 0, d_rope) || !(theta > 1.f) || !std::isfinite(theta))
+        return HYDRA_ERR_INVALID_ARG;
+    if (n_tokens == 0) return HYDRA_OK;
+    const void* ptrs[] = {dk, dv, positions, dkv_up, dk_pe};
+    for (const void* p : ptrs)
+        if (!p || !aligned4(p)) return HYDRA_ERR_INVALID_ARG;
+    if (int32_t s = device_info(nullptr)) return s;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ScopedKernelTimer timer(K_MLA, stream);
+    if (launch_mla_kv_assemble_bwd(dk, dv, positions, dkv_up, dk_pe, n_tokens, n_heads, d_nope, d_rope, d_v, theta,
+                                   stream) != cudaSuccess)
+        return HYDRA_ERR_CUDA;
+    g_launches += 1;
+    return HYDRA_OK;
+}
+
+int32_t hydra_gate_apply(const void* out, const void* gate, int64_t n_elements, void* y, void* cuda_stream)
+{
+    if (n_elements < 0 || n_elements % 8) return HYDRA_ERR_INVALID_ARG;
+    if (n_elements == 0) return HYDRA_OK;
+    if (!out || !gate || !y || !aligned16(out) || !aligned16(gate) || !aligned16(y)) return HYDRA_ERR_INVALID_ARG;
+    if (int32_t s = device_info(nullptr)) return s;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ScopedKernelTimer timer(K_MLA, stream);
+    if (launch_gate(out, gate, y, n_elements / 8, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    g_launches += 1;
+    return HYDRA_OK;
+}
+
+int32_t hydra_gate_apply_bwd(const void* dy, const void* out, const void* gate, int64_t n_elements, void* d_out,
+                             void* d_gate, void* cuda_stream)
+{
+    if (n_elements < 0 || n_elements % 8) return HYDRA_ERR_INVALID_ARG;
+    if (n_elements == 0) return HYDRA_OK;
+    const void* ptrs[] = {dy, out, gate, d_out, d_gate};
+    for (const void* p : ptrs)
+        if (!p || !aligned16(p)) return HYDRA_ERR_INVALID_ARG;
+    if (int32_t s = device_info(nullptr)) return s;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    ScopedKernelTimer timer(K_MLA, stream);
+    if (launch_gate_bwd(dy, out, gate, d_out, d_gate, n_elements / 8, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+    g_launches += 1;
+    return HYDRA_OK;
 }
 
 int32_t hydra_poll_status(void* workspace, void* cuda_stream, int32_t* device_status, int64_t* detail)

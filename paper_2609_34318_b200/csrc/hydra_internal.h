@@ -189,6 +189,19 @@ cudaError_t launch_merge_counted(const MergeParams& p, cudaStream_t stream);
 cudaError_t launch_grad_cast(const float* acc, void* grad, int64_t n, cudaStream_t stream);
 cudaError_t launch_ulysses(bool pack, const void* src, void* dst, int64_t n_tokens, int32_t cp_u, int64_t chunk_units,
                            cudaStream_t stream);
+// the elementwise steps of a gated MLA block around the attention kernel (mla_ops.cu)
+cudaError_t launch_rope(const void* x, const int32_t* positions, void* y, int64_t n_tokens, int32_t n_heads,
+                        int32_t head_dim, int32_t rope_offset, int32_t rope_dim, float theta, int inverse,
+                        cudaStream_t stream);
+cudaError_t launch_mla_kv_assemble(const void* kv_up, const void* k_pe, const int32_t* positions, void* k, void* v,
+                                   int64_t n_tokens, int32_t n_heads, int32_t nope, int32_t rope_dim, int32_t dv,
+                                   float theta, cudaStream_t stream);
+cudaError_t launch_mla_kv_assemble_bwd(const void* dk, const void* dv, const int32_t* positions, void* dkv_up,
+                                       void* dk_pe, int64_t n_tokens, int32_t n_heads, int32_t nope, int32_t rope_dim,
+                                       int32_t dvd, float theta, cudaStream_t stream);
+cudaError_t launch_gate(const void* out, const void* gate, void* y, int64_t n8, cudaStream_t stream);
+cudaError_t launch_gate_bwd(const void* dy, const void* out, const void* gate, void* d_out, void* d_gate, int64_t n8,
+                            cudaStream_t stream);
 cudaError_t launch_bwd_prep(const void* dout, const void* out, float* dsum, int64_t T, int32_t h,
                             cudaStream_t stream);
 

@@ -1,0 +1,258 @@
+// The elementwise steps of a gated multi-head-latent attention block around the attention kernel
+// (Section 5.2, "Exposed All-to-All Overlap": the query's rotary embedding; the split of the KV
+// up-projection's output into the value and the key's position-free part; the key's rotary embedding and
+// concatenation; the output gate), forward and backward. All are bound by HBM: every byte moves once, with
+// 16-byte or 4-byte accesses that are contiguous per warp. The paper names the steps, not their formulas;
+// the readings taken (rotary pairs (2i, 2i+1), angle = position * theta^(-2i/rope_dim); one rotary key
+// vector per token shared by all heads; up-projection rows laid out [key part | value]; gate = sigmoid)
+// are stated with each entry point in the header.
+#include <cuda_bf16.h>
+
+#include <cmath>
+
+#include "hydra_internal.h"
+
+namespace hydra {
+namespace {
+
+constexpr int kRopeThreads = 128;
+constexpr int kMaxRopePairs = 128;          // rotary dimensions up to 256
+
+__device__ __forceinline__ float2 bf2_to_f2(uint32_t w)
+{
+    return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+__device__ __forceinline__ uint32_t f2_to_bf2(float lo, float hi)
+{
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// cos / sin of position * theta^(-2i/rope_dim), i < rope_dim / 2, for one token, into shared memory. The
+// angle is formed and reduced modulo 2 pi in double precision: at position 262143 a single-precision
+// product is off by hundredths of a radian.
+__device__ __forceinline__ void rope_table(float* s_cos, float* s_sin, int32_t pos, int32_t rope_dim, double log_theta,
+                                           int inverse)
+{
+    for (int i = threadIdx.x; i < rope_dim / 2; i += blockDim.x) {
+        const double freq = exp(-log_theta * (2.0 * i) / rope_dim);
+        double ang = static_cast<double>(pos) * freq;
+        ang -= 6.283185307179586476925 * floor(ang / 6.283185307179586476925);
+        float sn, cs;
+        sincosf(static_cast<float>(ang), &sn, &cs);
+        s_cos[i] = cs;
+        s_sin[i] = inverse ? -sn : sn;
+    }
+}
+
+// y[t, a, :] = x[t, a, :] with the pairs (2i, 2i+1) of columns [rope_offset, rope_offset + rope_dim) rotated
+// by the token's angles. One block per token (grid-stride), the heads' rows as 4-byte pairs.
+__global__ void __launch_bounds__(kRopeThreads)
+hydra_rope_kernel(const uint32_t* __restrict__ x, const int32_t* __restrict__ positions, uint32_t* __restrict__ y,
+                  int64_t n_tokens, int32_t n_heads, int32_t head_dim, int32_t rope_offset, int32_t rope_dim,
+                  double log_theta, int inverse, int in_place)
+{
+    __shared__ float s_cos[kMaxRopePairs], s_sin[kMaxRopePairs];
+    const int pairs_per_head = head_dim / 2, p0 = rope_offset / 2, p1 = (rope_offset + rope_dim) / 2;
+    for (int64_t t = blockIdx.x; t < n_tokens; t += gridDim.x) {
+        __syncthreads();                               // the previous token's table is no longer read
+        rope_table(s_cos, s_sin, positions[t], rope_dim, log_theta, inverse);
+        __syncthreads();
+        const int64_t row0 = t * n_heads * pairs_per_head;
+        if (in_place) {                                // only the rotary columns move
+            const int n = n_heads * (p1 - p0);
+            for (int e = threadIdx.x; e < n; e += kRopeThreads) {
+                const int a = e / (p1 - p0), i = e - a * (p1 - p0);
+                const int64_t idx = row0 + static_cast<int64_t>(a) * pairs_per_head + p0 + i;
+                const float2 v = bf2_to_f2(x[idx]);
+                y[idx] = f2_to_bf2(v.x * s_cos[i] - v.y * s_sin[i], v.x * s_sin[i] + v.y * s_cos[i]);
+            }
+        } else {
+            const int n = n_heads * pairs_per_head;
+            for (int e = threadIdx.x; e < n; e += kRopeThreads) {
+                const int c = e % pairs_per_head;
+                uint32_t w = x[row0 + e];
+                if (c >= p0 && c < p1) {
+                    const float2 v = bf2_to_f2(w);
+                    const int i = c - p0;
+                    w = f2_to_bf2(v.x * s_cos[i] - v.y * s_sin[i], v.x * s_sin[i] + v.y * s_cos[i]);
+                }
+                y[row0 + e] = w;
+            }
+        }
+    }
+}
+
+// k[t, a, :] = [kv_up[t, a, 0:nope] | rope(k_pe[t, :])], v[t, a, :] = kv_up[t, a, nope:nope+dv]
+__global__ void __launch_bounds__(kRopeThreads)
+hydra_mla_kv_assemble_kernel(const uint32_t* __restrict__ kv_up, const uint32_t* __restrict__ k_pe,
+                             const int32_t* __restrict__ positions, uint32_t* __restrict__ k, uint32_t* __restrict__ v,
+                             int64_t n_tokens, int32_t n_heads, int32_t nope, int32_t rope_dim, int32_t dv,
+                             double log_theta)
+{
+    __shared__ float s_cos[kMaxRopePairs], s_sin[kMaxRopePairs];
+    __shared__ uint32_t s_pe[kMaxRopePairs];
+    const int np = nope / 2, rp = rope_dim / 2, vp = dv / 2;
+    const int up_pairs = np + vp, k_pairs = np + rp;
+    for (int64_t t = blockIdx.x; t < n_tokens; t += gridDim.x) {
+        __syncthreads();
+        rope_table(s_cos, s_sin, positions[t], rope_dim, log_theta, 0);
+        __syncthreads();
+        for (int i = threadIdx.x; i < rp; i += kRopeThreads) {
+            const float2 w = bf2_to_f2(k_pe[t * rp + i]);
+            s_pe[i] = f2_to_bf2(w.x * s_cos[i] - w.y * s_sin[i], w.x * s_sin[i] + w.y * s_cos[i]);
+        }
+        __syncthreads();
+        const int64_t up0 = t * n_heads * up_pairs, k0 = t * n_heads * k_pairs, v0 = t * n_heads * vp;
+        for (int e = threadIdx.x; e < n_heads * up_pairs; e += kRopeThreads) {
+            const int a = e / up_pairs, c = e - a * up_pairs;
+            const uint32_t w = kv_up[up0 + e];
+            if (c < np) k[k0 + static_cast<int64_t>(a) * k_pairs + c] = w;
+            else v[v0 + static_cast<int64_t>(a) * vp + (c - np)] = w;
+        }
+        for (int e = threadIdx.x; e < n_heads * rp; e += kRopeThreads) {
+            const int a = e / rp, i = e - a * rp;
+            k[k0 + static_cast<int64_t>(a) * k_pairs + np + i] = s_pe[i];
+        }
+    }
+}
+
+// The adjoint: dkv_up[t, a, :] = [dk[t, a, 0:nope] | dv[t, a, :]],
+// dk_pe[t, :] = rope^-1( sum_a dk[t, a, nope:nope+rope_dim] ) (summed in fp32, rounded once).
+__global__ void __launch_bounds__(kRopeThreads)
+hydra_mla_kv_assemble_bwd_kernel(const uint32_t* __restrict__ dk, const uint32_t* __restrict__ dv,
+                                 const int32_t* __restrict__ positions, uint32_t* __restrict__ dkv_up,
+                                 uint32_t* __restrict__ dk_pe, int64_t n_tokens, int32_t n_heads, int32_t nope,
+                                 int32_t rope_dim, int32_t dvd, double log_theta)
+{
+    __shared__ float s_cos[kMaxRopePairs], s_sin[kMaxRopePairs];
+    const int np = nope / 2, rp = rope_dim / 2, vp = dvd / 2;
+    const int up_pairs = np + vp, k_pairs = np + rp;
+    for (int64_t t = blockIdx.x; t < n_tokens; t += gridDim.x) {
+        __syncthreads();
+        rope_table(s_cos, s_sin, positions[t], rope_dim, log_theta, 1);
+        __syncthreads();
+        const int64_t up0 = t * n_heads * up_pairs, k0 = t * n_heads * k_pairs, v0 = t * n_heads * vp;
+        for (int e = threadIdx.x; e < n_heads * up_pairs; e += kRopeThreads) {
+            const int a = e / up_pairs, c = e - a * up_pairs;
+            dkv_up[up0 + e] = c < np ? dk[k0 + static_cast<int64_t>(a) * k_pairs + c]
+                                     : dv[v0 + static_cast<int64_t>(a) * vp + (c - np)];
+        }
+        for (int i = threadIdx.x; i < rp; i += kRopeThreads) {
+            float sx = 0.f, sy = 0.f;
+            for (int a = 0; a < n_heads; ++a) {
+                const float2 w = bf2_to_f2(dk[k0 + static_cast<int64_t>(a) * k_pairs + np + i]);
+                sx += w.x;
+                sy += w.y;
+            }
+            dk_pe[t * rp + i] = f2_to_bf2(sx * s_cos[i] - sy * s_sin[i], sx * s_sin[i] + sy * s_cos[i]);
+        }
+    }
+}
+
+__device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + __expf(-x)); }
+
+// y = out * sigmoid(gate), eight elements per thread
+__global__ void __launch_bounds__(256)
+hydra_gate_kernel(const uint4* __restrict__ out, const uint4* __restrict__ gate, uint4* __restrict__ y, int64_t n8)
+{
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x; i < n8; i += static_cast<int64_t>(gridDim.x) * 256) {
+        const uint4 o = out[i], g = gate[i];
+        const uint32_t* ow = reinterpret_cast<const uint32_t*>(&o);
+        const uint32_t* gw = reinterpret_cast<const uint32_t*>(&g);
+        uint4 r;
+        uint32_t* rw = reinterpret_cast<uint32_t*>(&r);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 a = bf2_to_f2(ow[e]), b = bf2_to_f2(gw[e]);
+            rw[e] = f2_to_bf2(a.x * sigmoidf_(b.x), a.y * sigmoidf_(b.y));
+        }
+        y[i] = r;
+    }
+}
+
+// d_out = dy * sigmoid(gate);  d_gate = dy * out * sigmoid(gate) * (1 - sigmoid(gate))
+__global__ void __launch_bounds__(256)
+hydra_gate_bwd_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ out, const uint4* __restrict__ gate,
+                      uint4* __restrict__ d_out, uint4* __restrict__ d_gate, int64_t n8)
+{
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x; i < n8; i += static_cast<int64_t>(gridDim.x) * 256) {
+        const uint4 d = dy[i], o = out[i], g = gate[i];
+        const uint32_t* dw = reinterpret_cast<const uint32_t*>(&d);
+        const uint32_t* ow = reinterpret_cast<const uint32_t*>(&o);
+        const uint32_t* gw = reinterpret_cast<const uint32_t*>(&g);
+        uint4 ro, rg;
+        uint32_t* row = reinterpret_cast<uint32_t*>(&ro);
+        uint32_t* rgw = reinterpret_cast<uint32_t*>(&rg);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 a = bf2_to_f2(dw[e]), b = bf2_to_f2(ow[e]), c = bf2_to_f2(gw[e]);
+            const float s0 = sigmoidf_(c.x), s1 = sigmoidf_(c.y);
+            row[e] = f2_to_bf2(a.x * s0, a.y * s1);
+            rgw[e] = f2_to_bf2(a.x * b.x * s0 * (1.f - s0), a.y * b.y * s1 * (1.f - s1));
+        }
+        d_out[i] = ro;
+        d_gate[i] = rg;
+    }
+}
+
+int grid_for(int64_t work_items, int per_block)
+{
+    const int64_t blocks = (work_items + per_block - 1) / per_block;
+    return static_cast<int>(blocks < 1 ? 1 : (blocks < 148 * 16 ? blocks : 148 * 16));
+}
+
+}  // namespace
+
+cudaError_t launch_rope(const void* x, const int32_t* positions, void* y, int64_t n_tokens, int32_t n_heads,
+                        int32_t head_dim, int32_t rope_offset, int32_t rope_dim, float theta, int inverse,
+                        cudaStream_t stream)
+{
+    if (n_tokens == 0) return cudaSuccess;
+    hydra_rope_kernel<<<grid_for(n_tokens, 1), kRopeThreads, 0, stream>>>(
+        static_cast<const uint32_t*>(x), positions, static_cast<uint32_t*>(y), n_tokens, n_heads, head_dim, rope_offset,
+        rope_dim, std::log(static_cast<double>(theta)), inverse, x == y ? 1 : 0);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mla_kv_assemble(const void* kv_up, const void* k_pe, const int32_t* positions, void* k, void* v,
+                                   int64_t n_tokens, int32_t n_heads, int32_t nope, int32_t rope_dim, int32_t dv,
+                                   float theta, cudaStream_t stream)
+{
+    if (n_tokens == 0) return cudaSuccess;
+    hydra_mla_kv_assemble_kernel<<<grid_for(n_tokens, 1), kRopeThreads, 0, stream>>>(
+        static_cast<const uint32_t*>(kv_up), static_cast<const uint32_t*>(k_pe), positions, static_cast<uint32_t*>(k),
+        static_cast<uint32_t*>(v), n_tokens, n_heads, nope, rope_dim, dv, std::log(static_cast<double>(theta)));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mla_kv_assemble_bwd(const void* dk, const void* dv, const int32_t* positions, void* dkv_up,
+                                       void* dk_pe, int64_t n_tokens, int32_t n_heads, int32_t nope, int32_t rope_dim,
+                                       int32_t dvd, float theta, cudaStream_t stream)
+{
+    if (n_tokens == 0) return cudaSuccess;
+    hydra_mla_kv_assemble_bwd_kernel<<<grid_for(n_tokens, 1), kRopeThreads, 0, stream>>>(
+        static_cast<const uint32_t*>(dk), static_cast<const uint32_t*>(dv), positions, static_cast<uint32_t*>(dkv_up),
+        static_cast<uint32_t*>(dk_pe), n_tokens, n_heads, nope, rope_dim, dvd, std::log(static_cast<double>(theta)));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gate(const void* out, const void* gate, void* y, int64_t n8, cudaStream_t stream)
+{
+    if (n8 == 0) return cudaSuccess;
+    hydra_gate_kernel<<<grid_for(n8, 256), 256, 0, stream>>>(static_cast<const uint4*>(out), static_cast<const uint4*>(gate),
+                                                             static_cast<uint4*>(y), n8);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gate_bwd(const void* dy, const void* out, const void* gate, void* d_out, void* d_gate, int64_t n8,
+                            cudaStream_t stream)
+{
+    if (n8 == 0) return cudaSuccess;
+    hydra_gate_bwd_kernel<<<grid_for(n8, 256), 256, 0, stream>>>(
+        static_cast<const uint4*>(dy), static_cast<const uint4*>(out), static_cast<const uint4*>(gate),
+        static_cast<uint4*>(d_out), static_cast<uint4*>(d_gate), n8);
+    return cudaGetLastError();
+}
+
+}  // namespace hydra

@@ -303,3 +303,17 @@ def test_bands_cover_random_problems_exactly_once(seed):
     for p, b in zip(out, band):
         for k0 in range(p["k_start"], p["k_start"] + p["k_len"], 128):
             assert owner.setdefault((int(p["seq"]), int(k0)), int(b)) == int(b)
+
+
+def test_plan_build_timer_is_host_only_and_bounded():
+    """The work tables of a call are built on the host; the timer needs no GPU. A new cu_seqlens must not cost
+    more than the kernels it feeds: the many-short batch (690 chunk pairs, 32 heads, 22 000 forward items)
+    builds each of its three tables in well under ten milliseconds even on a slow host."""
+    import hydra_workloads as hw
+    w = hw.workload("short64k_split")
+    cu = w.cu()
+    pairs, _, _, _ = P.hydra_zigzag_pairs(cu, w.cp_r)
+    for kind in (P.HYDRA_WS_FWD, P.HYDRA_WS_MERGE, P.HYDRA_WS_BWD):
+        t = min(P.hydra_plan_build_seconds(kind, cu, w.n_heads, pairs) for _ in range(3))
+        assert 0.0 <= t < 10e-3, (kind, t)
+    assert P.hydra_plan_build_seconds(7, cu, w.n_heads, pairs) < 0
