@@ -435,7 +435,7 @@ def run_ours(args, w):
 
     # ---- the second configuration of the target (N = 1 only): a few steps of the 256K ring workload ----
     secondary = None
-    if world == 1 and args.secondary and args.secondary != w.name:
+    if world == 1 and args.secondary not in ("", "none") and args.secondary != w.name:
         if args.no_e2e:
             del step
         else:
@@ -773,8 +773,15 @@ def merge_groups(pairs):
 # (summaries with the full commands are kept with the other profiler summaries). Each figure carries the
 # hash of the kernel sources it was captured from: when a source has changed since, the figure is no longer
 # printed (traffic = null) instead of being repeated for a kernel it does not describe.
+_TENSOR_DEPS = ("sm100_ptx.cuh", "hydra_internal.h")
 NCU_DRAM_BYTES_PER_LAUNCH = {
     # (kernel, workload): (bytes per launch, source files, their hash at capture time, capture date)
+    ("fwd", "packed32k"): (689471000, ("fwd_kernel.cu",) + _TENSOR_DEPS, "2e5bf8da80b4", "2026-11-25"),
+    # with the dS hand-off: 1.76 GB of the key-side kernel's writes and of the query-side kernel's reads are dS
+    ("bwd_dkv", "packed32k"): (2804055000, ("bwd_kernels.cu",) + _TENSOR_DEPS, "ac66daf4ebb2", "2026-11-25"),
+    ("bwd_dq", "packed32k"): (2069059000, ("bwd_kernels.cu",) + _TENSOR_DEPS, "ac66daf4ebb2", "2026-11-25"),
+    ("merge", "short64k_split"): (769407400, ("aux_kernels.cu", "hydra_internal.h"), "010f8444e435", "2026-11-25"),
+    ("bwd_prep", "short64k_split"): (1082133344, ("aux_kernels.cu", "hydra_internal.h"), "010f8444e435", "2026-11-25"),
 }
 
 
@@ -810,7 +817,7 @@ def main():
     ap.add_argument("--band-scratch-gb", type=float, default=48.0,
                     help="dS scratch of the banded backward (long sequences only); 0 switches the bands off")
     ap.add_argument("--secondary", default="ring256k",
-                    help="second workload timed after the headline one at N = 1 ('' = none)")
+                    help="second workload timed after the headline one at N = 1 ('none' = skip it)")
     ap.add_argument("--secondary-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
