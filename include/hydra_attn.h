@@ -364,6 +364,55 @@ int32_t hydra_attn_bwd_accumulate_dims(const void* q, const void* k, const void*
                                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Local layouts: what a rank of an outer ring calls (Section 5.2: the outer ring circulates K/V chunks and
+ * pipelines with attention; Section 3.5, Eq. (ring)). Such a rank holds only its own q chunks and, at a ring
+ * step, the visiting kv chunks; its tensors are not the packed batch. A chunk table says where the chunks of
+ * the sequences sit:
+ *   hydra_chunk_t { seq, start, len, row }   positions [start, start + len) of sequence seq occupy rows
+ *                                            [row, row + len) of the tensor
+ * q_chunks describes the q-side tensors (q, out, lse, dout, dq: q_rows rows; lse is [n_heads, q_rows]),
+ * kv_chunks the kv-side tensors (k, v, dk, dv: kv_rows rows). The pairs keep their sequence-local positions
+ * (the causal mask needs them); every pair's q range must lie inside one q chunk and its kv range inside one
+ * kv chunk, chunks of one table must not share rows (else HYDRA_ERR_INVALID_ARG). cu_seqlens_host still gives
+ * the lengths of the whole sequences. Everything else is as in hydra_attn_fwd_dims / hydra_lse_merge(_accumulate)
+ * / hydra_attn_bwd_accumulate_dims: the forward of a step's pairs writes partials (or out / lse directly for a
+ * chunk with one pair), the merge folds them into the running (out, lse) when `accumulate` is non-zero, the
+ * backward adds the step's contributions into fp32 accumulators laid out like the tensors they belong to
+ * (dq_acc with q_rows rows; dk_acc, dv_acc with kv_rows rows: they travel round the ring with their chunks).
+ * The exchange of the chunks between the GPUs is the caller's (a peer copy or NCCL send / receive into this
+ * GPU's own memory before the call: the kernels only ever read local memory).
+ */
+typedef struct {
+    int32_t seq;
+    int32_t start, len;
+    int32_t row;
+} hydra_chunk_t;
+size_t hydra_workspace_bytes_local(int32_t which, const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
+                                   int32_t n_kv_heads, int32_t d_qk, int32_t d_v, const hydra_chunk_t* q_chunks,
+                                   int32_t n_q_chunks, int64_t q_rows, const hydra_chunk_t* kv_chunks,
+                                   int32_t n_kv_chunks, int64_t kv_rows, const hydra_pair_t* pairs, int32_t n_pairs);
+int32_t hydra_attn_fwd_local(const void* q, const void* k, const void* v, const int32_t* cu_seqlens_host,
+                             int32_t n_seqs, int32_t n_heads, int32_t n_kv_heads, int32_t d_qk, int32_t d_v,
+                             const hydra_chunk_t* q_chunks, int32_t n_q_chunks, int64_t q_rows,
+                             const hydra_chunk_t* kv_chunks, int32_t n_kv_chunks, int64_t kv_rows,
+                             const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
+                             void* out, float* lse, void* o_part, float* lse_part, int64_t part_rows,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream);
+int32_t hydra_lse_merge_local(const void* o_part, const float* lse_part, int64_t part_rows,
+                              const int32_t* cu_seqlens_host, int32_t n_seqs, int32_t n_heads,
+                              const hydra_chunk_t* q_chunks, int32_t n_q_chunks, int64_t q_rows,
+                              const hydra_pair_t* pairs, int32_t n_pairs, int32_t accumulate, void* out, float* lse,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+int32_t hydra_attn_bwd_accumulate_local(const void* q, const void* k, const void* v, const void* out,
+                                        const float* lse, const void* dout, const int32_t* cu_seqlens_host,
+                                        int32_t n_seqs, int32_t n_heads, int32_t n_kv_heads, int32_t d_qk,
+                                        int32_t d_v, const hydra_chunk_t* q_chunks, int32_t n_q_chunks,
+                                        int64_t q_rows, const hydra_chunk_t* kv_chunks, int32_t n_kv_chunks,
+                                        int64_t kv_rows, const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal,
+                                        float softmax_scale, float* dq_acc, float* dk_acc, float* dv_acc,
+                                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * The local halves of the Ulysses all-to-all (Section 3.5: all-to-all transposes partition the attention
  * heads across the cp_u ranks of a group; Eq. (ulysses) counts the volume, about 4 S h / P elements per
  * rank for q, k, v and the output). Elements are 2 bytes wide (bf16) and are moved, not interpreted.

@@ -37,6 +37,19 @@ PAIR_DTYPE = np.dtype([("seq", "<i4"), ("q_start", "<i4"), ("q_len", "<i4"), ("k
                        ("k_len", "<i4"), ("part_row", "<i4"), ("group", "<i4"), ("flags", "<i4")])
 
 
+CHUNK_DTYPE = np.dtype([("seq", "<i4"), ("start", "<i4"), ("len", "<i4"), ("row", "<i4")])
+
+
+def as_chunks(chunks) -> np.ndarray:
+    """A chunk table (include/hydra_attn.h, hydra_chunk_t): structured array, or an iterable of (seq, start, len, row)."""
+    if isinstance(chunks, np.ndarray) and chunks.dtype == CHUNK_DTYPE:
+        return np.ascontiguousarray(chunks)
+    out = np.zeros(len(chunks), dtype=CHUNK_DTYPE)
+    for i, c in enumerate(chunks):
+        out[i] = tuple(c[n] for n in ("seq", "start", "len", "row")) if isinstance(c, dict) else tuple(c)
+    return out
+
+
 class HydraError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -120,6 +133,18 @@ def _load() -> ctypes.CDLL:
         getattr(lib, name).argtypes = g[:10] + [i32, i32] + g[10:]
     lib.hydra_grad_cast.restype = i32
     lib.hydra_grad_cast.argtypes = [vp, vp, i64, vp]
+    # local layouts (a rank of an outer ring): chunk tables after the head dimensions
+    tables = [vp, i32, i64, vp, i32, i64]
+    lib.hydra_workspace_bytes_local.restype = sz
+    lib.hydra_workspace_bytes_local.argtypes = [i32, vp, i32, i32, i32, i32, i32] + tables + [vp, i32]
+    lib.hydra_attn_fwd_local.restype = i32
+    lib.hydra_attn_fwd_local.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32] + tables + \
+        [vp, i32, i32, f32, vp, vp, vp, vp, i64, vp, sz, vp]
+    lib.hydra_lse_merge_local.restype = i32
+    lib.hydra_lse_merge_local.argtypes = [vp, vp, i64, vp, i32, i32, vp, i32, i64, vp, i32, i32, vp, vp, vp, sz, vp]
+    lib.hydra_attn_bwd_accumulate_local.restype = i32
+    lib.hydra_attn_bwd_accumulate_local.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32] + tables + \
+        [vp, i32, i32, f32, vp, vp, vp, vp, sz, vp]
     lib.hydra_mla_rope.restype = i32
     lib.hydra_mla_rope.argtypes = [vp, vp, i64, i32, i32, i32, i32, f32, i32, vp, vp]
     for name in ("hydra_mla_kv_assemble", "hydra_mla_kv_assemble_bwd"):
@@ -157,6 +182,7 @@ EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_
            "hydra_sched_targets", "hydra_sched_cp", "hydra_sched_pack", "hydra_attn_bwd_accumulate",
            "hydra_grad_cast", "hydra_set_bwd_scratch_limit", "hydra_set_bwd_band_scratch", "hydra_bwd_bands", "hydra_ulysses_pack", "hydra_ulysses_unpack", "hydra_attn_fwd_gqa", "hydra_attn_bwd_accumulate_gqa", "hydra_attn_bwd_gqa", "hydra_workspace_bytes_gqa",
            "hydra_mla_rope", "hydra_mla_kv_assemble", "hydra_mla_kv_assemble_bwd", "hydra_gate_apply", "hydra_gate_apply_bwd",
+           "hydra_attn_fwd_local", "hydra_lse_merge_local", "hydra_attn_bwd_accumulate_local", "hydra_workspace_bytes_local",
            "hydra_attn_fwd_dims", "hydra_attn_bwd_dims", "hydra_attn_bwd_accumulate_dims", "hydra_workspace_bytes_dims",
            "hydra_poll_clocks")
 KERNEL_KINDS = ("fwd", "merge", "bwd_prep", "bwd_dkv", "bwd_dq", "grad_cast", "ulysses", "mla_ops")
@@ -558,6 +584,75 @@ def hydra_gate_apply_bwd(dy, out, gate, n_elements: int, d_out, d_gate, stream=N
                                   _stream(stream))
     if check:
         _check(s, "hydra_gate_apply_bwd")
+    return s
+
+
+def _tables(q_chunks, q_rows, kv_chunks, kv_rows):
+    qc, kc = as_chunks(q_chunks), as_chunks(kv_chunks)
+    return (qc.ctypes.data, len(qc), int(q_rows), kc.ctypes.data, len(kc), int(kv_rows)), (qc, kc)
+
+
+def hydra_workspace_bytes_local(which: int, cu_seqlens, n_heads: int, n_kv_heads: int, d_qk: int, d_v: int, q_chunks,
+                                q_rows: int, kv_chunks, kv_rows: int, pairs) -> int:
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    t, _k2 = _tables(q_chunks, q_rows, kv_chunks, kv_rows)
+    return int(_lib.hydra_workspace_bytes_local(which, cu.ctypes.data, len(cu) - 1, n_heads, n_kv_heads, int(d_qk),
+                                                int(d_v), *t, pp, npairs))
+
+
+def hydra_attn_fwd_local(q, k, v, cu_seqlens, n_heads: int, n_kv_heads: int, d_qk: int, d_v: int, q_chunks, q_rows: int,
+                         kv_chunks, kv_rows: int, pairs, causal: bool, softmax_scale: float, out, lse, o_part,
+                         lse_part, part_rows: int, workspace, workspace_bytes: Optional[int] = None, stream=None,
+                         check: bool = True) -> int:
+    """Forward of the listed pairs on LOCAL tensors (a rank of an outer ring): chunk tables say where the chunks sit."""
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    t, _k2 = _tables(q_chunks, q_rows, kv_chunks, kv_rows)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = _lib.hydra_attn_fwd_local(_ptr(q), _ptr(k), _ptr(v), cu.ctypes.data, len(cu) - 1, n_heads, n_kv_heads,
+                                  int(d_qk), int(d_v), *t, pp, npairs, int(bool(causal)),
+                                  ctypes.c_float(float(softmax_scale)), _ptr(out), _ptr(lse), _ptr(o_part),
+                                  _ptr(lse_part), int(part_rows), _ptr(workspace), int(workspace_bytes),
+                                  _stream(stream))
+    if check:
+        _check(s, "hydra_attn_fwd_local")
+    return s
+
+
+def hydra_lse_merge_local(o_part, lse_part, part_rows: int, cu_seqlens, n_heads: int, q_chunks, q_rows: int, pairs,
+                          accumulate: bool, out, lse, workspace, workspace_bytes: Optional[int] = None, stream=None,
+                          check: bool = True) -> int:
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    qc = as_chunks(q_chunks)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = _lib.hydra_lse_merge_local(_ptr(o_part), _ptr(lse_part), int(part_rows), cu.ctypes.data, len(cu) - 1, n_heads,
+                                   qc.ctypes.data, len(qc), int(q_rows), pp, npairs, int(bool(accumulate)), _ptr(out),
+                                   _ptr(lse), _ptr(workspace), int(workspace_bytes), _stream(stream))
+    if check:
+        _check(s, "hydra_lse_merge_local")
+    return s
+
+
+def hydra_attn_bwd_accumulate_local(q, k, v, out, lse, dout, cu_seqlens, n_heads: int, n_kv_heads: int, d_qk: int,
+                                    d_v: int, q_chunks, q_rows: int, kv_chunks, kv_rows: int, pairs, causal: bool,
+                                    softmax_scale: float, dq_acc, dk_acc, dv_acc, workspace,
+                                    workspace_bytes: Optional[int] = None, stream=None, check: bool = True) -> int:
+    cu = _cu(cu_seqlens)
+    pp, npairs, _keep = _pairs_arg(pairs)
+    t, _k2 = _tables(q_chunks, q_rows, kv_chunks, kv_rows)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    s = _lib.hydra_attn_bwd_accumulate_local(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout),
+                                             cu.ctypes.data, len(cu) - 1, n_heads, n_kv_heads, int(d_qk), int(d_v), *t,
+                                             pp, npairs, int(bool(causal)), ctypes.c_float(float(softmax_scale)),
+                                             _ptr(dq_acc), _ptr(dk_acc), _ptr(dv_acc), _ptr(workspace),
+                                             int(workspace_bytes), _stream(stream))
+    if check:
+        _check(s, "hydra_attn_bwd_accumulate_local")
     return s
 
 

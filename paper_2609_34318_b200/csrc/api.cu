@@ -71,6 +71,19 @@ struct Problem {
     int32_t n_seqs = 0, h = 0;
     int64_t T = 0;
     int32_t dqk = D_QK;     // q / k head dimension of the call: 192 or 128 (the value dimension is 128)
+    // Local layouts (a rank of a ring holds only its own q chunks and the visiting kv chunks): where the
+    // chunks of the sequences sit in the q-side tensors (q, out, lse, dout, dq) and in the kv-side tensors
+    // (k, v, dk, dv). Empty tables = the packed layout, row = cu[seq] + position, Tq = Tk = T.
+    std::vector<hydra_chunk_t> qc, kc;
+    int64_t Tq = 0, Tk = 0;
+    static int64_t row_in(const std::vector<hydra_chunk_t>& table, int32_t seq, int32_t pos)
+    {
+        for (const hydra_chunk_t& c : table)
+            if (c.seq == seq && pos >= c.start && pos < c.start + c.len) return int64_t{c.row} + (pos - c.start);
+        return -1;
+    }
+    int64_t q_row(int32_t seq, int32_t pos) const { return qc.empty() ? int64_t{cu[seq]} + pos : row_in(qc, seq, pos); }
+    int64_t k_row(int32_t seq, int32_t pos) const { return kc.empty() ? int64_t{cu[seq]} + pos : row_in(kc, seq, pos); }
 };
 
 int32_t make_problem(const int32_t* cu, int32_t n_seqs, int32_t h, const hydra_pair_t* pairs,
@@ -89,6 +102,9 @@ int32_t make_problem(const int32_t* cu, int32_t n_seqs, int32_t h, const hydra_p
     }
     out.T = out.cu[n_seqs];
     if (out.T > (int64_t{1} << 30)) return HYDRA_ERR_UNSUPPORTED;
+    out.Tq = out.Tk = out.T;
+    out.qc.clear();
+    out.kc.clear();
     out.pairs.clear();
     if (pairs == nullptr) {
         for (int b = 0; b < n_seqs; ++b) {
@@ -115,6 +131,44 @@ int32_t make_problem(const int32_t* cu, int32_t n_seqs, int32_t h, const hydra_p
             if (p.group == o.group && p.part_row < 0) return HYDRA_ERR_INVALID_ARG;  // two direct writers
         }
         out.pairs.push_back(p);
+    }
+    return HYDRA_OK;
+}
+
+// The same with local layouts: every chunk lies inside its sequence and inside its tensor, chunks of one table
+// do not share rows, and every pair's q range lies inside one q chunk and its kv range inside one kv chunk.
+int32_t make_problem_local(const int32_t* cu, int32_t n_seqs, int32_t h, const hydra_chunk_t* q_chunks,
+                           int32_t n_q_chunks, int64_t q_rows, const hydra_chunk_t* kv_chunks, int32_t n_kv_chunks,
+                           int64_t kv_rows, const hydra_pair_t* pairs, int32_t n_pairs, Problem& out)
+{
+    if (!pairs || n_pairs < 1 || !q_chunks || n_q_chunks < 1 || !kv_chunks || n_kv_chunks < 1) return HYDRA_ERR_INVALID_ARG;
+    if (q_rows < 1 || kv_rows < 1 || q_rows > (int64_t{1} << 30) || kv_rows > (int64_t{1} << 30)) return HYDRA_ERR_INVALID_ARG;
+    if (int32_t s = make_problem(cu, n_seqs, h, pairs, n_pairs, out)) return s;
+    auto take = [&](const hydra_chunk_t* src, int32_t n, int64_t rows, std::vector<hydra_chunk_t>& dst) {
+        dst.assign(src, src + n);
+        std::vector<std::pair<int64_t, int64_t>> iv;
+        for (const hydra_chunk_t& c : dst) {
+            if (c.seq < 0 || c.seq >= n_seqs || c.start < 0 || c.len < 0 || c.row < 0) return false;
+            if (int64_t{c.start} + c.len > int64_t{out.cu[c.seq + 1]} - out.cu[c.seq]) return false;
+            if (int64_t{c.row} + c.len > rows) return false;
+            if (c.len > 0) iv.emplace_back(c.row, int64_t{c.row} + c.len);
+        }
+        std::sort(iv.begin(), iv.end());
+        for (size_t i = 1; i < iv.size(); ++i)
+            if (iv[i].first < iv[i - 1].second) return false;
+        return true;
+    };
+    if (!take(q_chunks, n_q_chunks, q_rows, out.qc) || !take(kv_chunks, n_kv_chunks, kv_rows, out.kc))
+        return HYDRA_ERR_INVALID_ARG;
+    out.Tq = q_rows;
+    out.Tk = kv_rows;
+    for (const hydra_pair_t& p : out.pairs) {
+        if (p.q_len > 0 && (out.q_row(p.seq, p.q_start) < 0 ||
+                            out.q_row(p.seq, p.q_start + p.q_len - 1) != out.q_row(p.seq, p.q_start) + p.q_len - 1))
+            return HYDRA_ERR_INVALID_ARG;
+        if (p.k_len > 0 && (out.k_row(p.seq, p.k_start) < 0 ||
+                            out.k_row(p.seq, p.k_start + p.k_len - 1) != out.k_row(p.seq, p.k_start) + p.k_len - 1))
+            return HYDRA_ERR_INVALID_ARG;
     }
     return HYDRA_OK;
 }
@@ -374,6 +428,12 @@ std::vector<uint8_t> make_key(int kind, int device, const Problem& pb, int causa
     put(head, sizeof head);
     put(pb.cu.data(), pb.cu.size() * sizeof(int32_t));
     put(pb.pairs.data(), pb.pairs.size() * sizeof(hydra_pair_t));
+    if (!pb.qc.empty() || !pb.kc.empty()) {
+        const int64_t dims[4] = {pb.Tq, pb.Tk, static_cast<int64_t>(pb.qc.size()), static_cast<int64_t>(pb.kc.size())};
+        put(dims, sizeof dims);
+        put(pb.qc.data(), pb.qc.size() * sizeof(hydra_chunk_t));
+        put(pb.kc.data(), pb.kc.size() * sizeof(hydra_chunk_t));
+    }
     return key;
 }
 
@@ -383,9 +443,9 @@ std::vector<PairDev> device_pairs(const Problem& pb)
     v.reserve(pb.pairs.size());
     for (const auto& p : pb.pairs) {
         PairDev d;
-        d.q_tok0 = pb.cu[p.seq] + p.q_start;
+        d.q_tok0 = p.q_len > 0 ? static_cast<int32_t>(pb.q_row(p.seq, p.q_start)) : 0;
         d.q_len = p.q_len;
-        d.k_tok0 = pb.cu[p.seq] + p.k_start;
+        d.k_tok0 = p.k_len > 0 ? static_cast<int32_t>(pb.k_row(p.seq, p.k_start)) : 0;
         d.k_len = p.k_len;
         d.off = p.q_start - p.k_start;
         d.to_part = p.part_row >= 0;
@@ -610,7 +670,7 @@ void build_merge(const Problem& pb, Plan& plan, std::vector<uint8_t>& blob)
         const auto& p = pb.pairs[i];
         if (p.part_row >= 0 && p.q_len > 0) {
             MergeGroup g;
-            g.out_tok0 = pb.cu[p.seq] + p.q_start;
+            g.out_tok0 = static_cast<int32_t>(pb.q_row(p.seq, p.q_start));
             g.rows = p.q_len;
             g.list_off = static_cast<int32_t>(lists.size());
             g.n_parts = static_cast<int32_t>(j - i);
@@ -1075,15 +1135,15 @@ uint64_t band_scratch_for(int64_t head_blocks, int32_t n_heads)
 
 size_t bwd_acc_bytes(const Problem& pb)
 {
-    return align_up(static_cast<size_t>(pb.T) * pb.h * pb.dqk * sizeof(float), 1024);
+    return align_up(static_cast<size_t>(pb.Tq) * pb.h * pb.dqk * sizeof(float), 1024);
 }
 size_t bwd_kv_acc_bytes(const Problem& pb, int32_t n_kv_heads)
 {
-    return align_up(static_cast<size_t>(pb.T) * n_kv_heads * (pb.dqk + D_V) * sizeof(float), 1024);
+    return align_up(static_cast<size_t>(pb.Tk) * n_kv_heads * (pb.dqk + D_V) * sizeof(float), 1024);
 }
 size_t bwd_base_bytes(const Problem& pb)
 {
-    return align_up(kStatusBytes + align_up(static_cast<size_t>(pb.T) * pb.h * sizeof(float), 256), 1024);
+    return align_up(kStatusBytes + align_up(static_cast<size_t>(pb.Tq) * pb.h * sizeof(float), 256), 1024);
 }
 // bytes of the dS hand-off buffer, or 0 if it is not to be used (layout not possible, or over the limit)
 size_t bwd_ds_bytes(int64_t head_blocks, int32_t n_heads, uint64_t limit)
@@ -1143,6 +1203,12 @@ size_t hydra_workspace_bytes_dims(int32_t which, const int32_t* cu, int32_t n_se
     }
 }
 
+namespace {
+int32_t fwd_core(Problem& pb, const void* q, const void* k, const void* v, int32_t n_kv_heads, int32_t causal,
+                 float softmax_scale, void* out, float* lse, void* o_part, float* lse_part, int64_t part_rows,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+}
+
 int32_t hydra_attn_fwd(const void* q, const void* k, const void* v, const int32_t* cu, int32_t n_seqs,
                        int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal,
                        float softmax_scale, void* out, float* lse, void* o_part, float* lse_part,
@@ -1169,11 +1235,39 @@ int32_t hydra_attn_fwd_dims(const void* q, const void* k, const void* v, const i
                             void* out, float* lse, void* o_part, float* lse_part, int64_t part_rows,
                             void* workspace, size_t workspace_bytes, void* cuda_stream)
 {
-    const KernelSet* ks = kernel_set(d_qk, d_v);
-    if (!ks) return HYDRA_ERR_UNSUPPORTED;
+    if (!kernel_set(d_qk, d_v)) return HYDRA_ERR_UNSUPPORTED;
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
     pb.dqk = d_qk;
+    return fwd_core(pb, q, k, v, n_kv_heads, causal, softmax_scale, out, lse, o_part, lse_part, part_rows, workspace,
+                    workspace_bytes, cuda_stream);
+}
+
+int32_t hydra_attn_fwd_local(const void* q, const void* k, const void* v, const int32_t* cu, int32_t n_seqs,
+                             int32_t n_heads, int32_t n_kv_heads, int32_t d_qk, int32_t d_v,
+                             const hydra_chunk_t* q_chunks, int32_t n_q_chunks, int64_t q_rows,
+                             const hydra_chunk_t* kv_chunks, int32_t n_kv_chunks, int64_t kv_rows,
+                             const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
+                             void* out, float* lse, void* o_part, float* lse_part, int64_t part_rows,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (!kernel_set(d_qk, d_v)) return HYDRA_ERR_UNSUPPORTED;
+    Problem pb;
+    if (int32_t s = make_problem_local(cu, n_seqs, n_heads, q_chunks, n_q_chunks, q_rows, kv_chunks, n_kv_chunks,
+                                       kv_rows, pairs, n_pairs, pb))
+        return s;
+    pb.dqk = d_qk;
+    return fwd_core(pb, q, k, v, n_kv_heads, causal, softmax_scale, out, lse, o_part, lse_part, part_rows, workspace,
+                    workspace_bytes, cuda_stream);
+}
+
+namespace {
+int32_t fwd_core(Problem& pb, const void* q, const void* k, const void* v, int32_t n_kv_heads, int32_t causal,
+                 float softmax_scale, void* out, float* lse, void* o_part, float* lse_part, int64_t part_rows,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    const int32_t n_heads = pb.h;
+    const KernelSet* ks = kernel_set(pb.dqk, D_V);
     if (n_kv_heads < 1 || n_heads % n_kv_heads) return HYDRA_ERR_INVALID_ARG;
     if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return HYDRA_ERR_INVALID_ARG;
     if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
@@ -1198,8 +1292,8 @@ int32_t hydra_attn_fwd_dims(const void* q, const void* k, const void* v, const i
     if (plan->n_items == 0) return HYDRA_OK;
     // each CTA of a pair stages 64 kv rows of K (box of 64 rows) and 64 value columns of V
     CUtensorMap mq, mk, mv;
-    if (make_map(&mq, q, pb.T, n_heads, pb.dqk, TILE) || make_map(&mk, k, pb.T, n_kv_heads, pb.dqk, SUB) ||
-        make_map(&mv, v, pb.T, n_kv_heads, D_V, TILE))
+    if (make_map(&mq, q, pb.Tq, n_heads, pb.dqk, TILE) || make_map(&mk, k, pb.Tk, n_kv_heads, pb.dqk, SUB) ||
+        make_map(&mv, v, pb.Tk, n_kv_heads, D_V, TILE))
         return HYDRA_ERR_CUDA;
     if (int32_t s = reset_status(workspace, stream)) return s;
     FwdParams fp{};
@@ -1207,7 +1301,7 @@ int32_t hydra_attn_fwd_dims(const void* q, const void* k, const void* v, const i
     fp.items = lease.at<FwdItem>(plan->off_items);
     fp.n_items = plan->n_items;
     fp.out = out; fp.lse = lse; fp.o_part = o_part; fp.lse_part = lse_part;
-    fp.T = pb.T; fp.part_rows = part_rows; fp.h = n_heads; fp.causal = causal != 0;
+    fp.T = pb.Tq; fp.part_rows = part_rows; fp.h = n_heads; fp.causal = causal != 0;
     fp.kv_group = n_heads / n_kv_heads;
     fp.scale_log2 = softmax_scale * 1.4426950408889634f;
     fp.status = static_cast<StatusBlock*>(workspace);
@@ -1222,10 +1316,13 @@ int32_t hydra_attn_fwd_dims(const void* q, const void* k, const void* v, const i
     prefetch_plans(pb, causal != 0, any_part);
     return HYDRA_OK;
 }
+}  // namespace
 
 namespace {
 int32_t merge_impl(const void* o_part, const float* lse_part, int64_t part_rows, const int32_t* cu,
                    int32_t n_seqs, int32_t n_heads, const hydra_pair_t* pairs, int32_t n_pairs, void* out,
+                   float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream, int32_t accumulate);
+int32_t merge_core(const Problem& pb, const void* o_part, const float* lse_part, int64_t part_rows, void* out,
                    float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream, int32_t accumulate);
 }
 
@@ -1253,6 +1350,13 @@ int32_t merge_impl(const void* o_part, const float* lse_part, int64_t part_rows,
 {
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
+    return merge_core(pb, o_part, lse_part, part_rows, out, lse, workspace, workspace_bytes, cuda_stream, accumulate);
+}
+
+int32_t merge_core(const Problem& pb, const void* o_part, const float* lse_part, int64_t part_rows, void* out,
+                   float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream, int32_t accumulate)
+{
+    const int32_t n_heads = pb.h;
     if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
     if (workspace_bytes < kStatusBytes) return HYDRA_ERR_WORKSPACE_TOO_SMALL;
     bool any_part = false;
@@ -1274,7 +1378,7 @@ int32_t merge_impl(const void* o_part, const float* lse_part, int64_t part_rows,
     mp.items = lease.at<MergeItem>(plan->off_items);
     mp.n_items = plan->n_items;
     mp.o_part = o_part; mp.lse_part = lse_part; mp.out = out; mp.lse = lse;
-    mp.T = pb.T; mp.part_rows = part_rows; mp.h = n_heads;
+    mp.T = pb.Tq; mp.part_rows = part_rows; mp.h = n_heads;
     mp.accumulate = accumulate;
     if (launch_merge_counted(mp, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
     return HYDRA_OK;
@@ -1305,14 +1409,14 @@ int32_t bwd_run(const Problem& pb, int32_t n_kv_heads, int32_t causal, float sof
 
     float* dsum = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kStatusBytes);
     CUtensorMap mq, mk, mv, mdo, mq_sub, mdo_sub;
-    if (make_map(&mq, t.q, pb.T, n_heads, pb.dqk, TILE) || make_map(&mk, t.k, pb.T, n_kv_heads, pb.dqk, TILE) ||
-        make_map(&mv, t.v, pb.T, n_kv_heads, D_V, TILE) || make_map(&mdo, t.dout, pb.T, n_heads, D_V, TILE) ||
-        make_map(&mq_sub, t.q, pb.T, n_heads, pb.dqk, SUB) || make_map(&mdo_sub, t.dout, pb.T, n_heads, D_V, SUB))
+    if (make_map(&mq, t.q, pb.Tq, n_heads, pb.dqk, TILE) || make_map(&mk, t.k, pb.Tk, n_kv_heads, pb.dqk, TILE) ||
+        make_map(&mv, t.v, pb.Tk, n_kv_heads, D_V, TILE) || make_map(&mdo, t.dout, pb.Tq, n_heads, D_V, TILE) ||
+        make_map(&mq_sub, t.q, pb.Tq, n_heads, pb.dqk, SUB) || make_map(&mdo_sub, t.dout, pb.Tq, n_heads, D_V, SUB))
         return HYDRA_ERR_CUDA;
     if (first) {
         if (int32_t s = reset_status(workspace, stream)) return s;
         ScopedKernelTimer timer(K_PREP, stream);
-        if (launch_bwd_prep(t.dout, t.out, dsum, pb.T, n_heads, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+        if (launch_bwd_prep(t.dout, t.out, dsum, pb.Tq, n_heads, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
         g_launches += 1;
     } else if (cudaMemsetAsync(static_cast<uint8_t*>(workspace) + offsetof(StatusBlock, next_item), 0,
                                sizeof(StatusBlock::next_item), stream) != cudaSuccess) {
@@ -1322,7 +1426,7 @@ int32_t bwd_run(const Problem& pb, int32_t n_kv_heads, int32_t causal, float sof
     BwdParams bp{};
     bp.pairs = lease.at<PairDev>(plan->off_pairs);
     bp.lse = t.lse; bp.dsum = dsum; bp.dq = t.dq; bp.dk = t.dk; bp.dv = t.dv;
-    bp.T = pb.T; bp.h = n_heads; bp.causal = causal != 0;
+    bp.T = pb.Tq; bp.h = n_heads; bp.causal = causal != 0;
     bp.kv_group = n_heads / n_kv_heads;
     bp.scale = softmax_scale; bp.scale_log2 = softmax_scale * 1.4426950408889634f;
     bp.status = static_cast<StatusBlock*>(workspace);
@@ -1401,7 +1505,7 @@ std::vector<std::vector<hydra_pair_t>> make_bands(const Problem& pb, int32_t cau
         return true;
     };
     Problem probe;
-    probe.cu = pb.cu; probe.n_seqs = pb.n_seqs; probe.h = pb.h; probe.T = pb.T; probe.dqk = pb.dqk;
+    probe.cu = pb.cu; probe.n_seqs = pb.n_seqs; probe.h = pb.h; probe.T = pb.T; probe.Tq = pb.Tq; probe.Tk = pb.Tk; probe.dqk = pb.dqk;
     auto fits = [&](const std::vector<hydra_pair_t>& pairs) {
         probe.pairs = pairs;
         return bwd_ds_bytes(ds_layout(probe, causal, nullptr), pb.h, room) > 0;
@@ -1449,7 +1553,7 @@ std::vector<std::pair<size_t, size_t>> covered_rows(const Problem& pb, bool key_
     std::vector<std::pair<size_t, size_t>> rows;
     for (const auto& p : pb.pairs) {
         if (p.q_len <= 0 || p.k_len <= 0) continue;
-        const size_t first = static_cast<size_t>(pb.cu[p.seq]) + (key_side ? p.k_start : p.q_start);
+        const size_t first = static_cast<size_t>(key_side ? pb.k_row(p.seq, p.k_start) : pb.q_row(p.seq, p.q_start));
         rows.emplace_back(first, first + static_cast<size_t>(key_side ? p.k_len : p.q_len));
     }
     std::sort(rows.begin(), rows.end());
@@ -1461,6 +1565,10 @@ std::vector<std::pair<size_t, size_t>> covered_rows(const Problem& pb, bool key_
     return runs;
 }
 
+int32_t bwd_core(Problem& pb, const void* q, const void* k, const void* v, const void* out, const float* lse,
+                 const void* dout, int32_t causal, float softmax_scale, void* dq, void* dk, void* dv, bool accumulate,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream, int32_t n_kv_heads);
+
 int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, const float* lse,
                  const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
                  const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal, float softmax_scale,
@@ -1471,10 +1579,19 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
     Problem pb;
     if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
     pb.dqk = d_qk;
+    return bwd_core(pb, q, k, v, out, lse, dout, causal, softmax_scale, dq, dk, dv, accumulate, workspace,
+                    workspace_bytes, cuda_stream, n_kv_heads);
+}
+
+int32_t bwd_core(Problem& pb, const void* q, const void* k, const void* v, const void* out, const float* lse,
+                 const void* dout, int32_t causal, float softmax_scale, void* dq, void* dk, void* dv, bool accumulate,
+                 void* workspace, size_t workspace_bytes, void* cuda_stream, int32_t n_kv_heads)
+{
+    const int32_t n_heads = pb.h;
     if (n_kv_heads < 1 || n_heads % n_kv_heads) return HYDRA_ERR_INVALID_ARG;
     if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return HYDRA_ERR_INVALID_ARG;
     if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
-    const size_t need = kStatusBytes + align_up(static_cast<size_t>(pb.T) * n_heads * sizeof(float), 256);
+    const size_t need = kStatusBytes + align_up(static_cast<size_t>(pb.Tq) * n_heads * sizeof(float), 256);
     if (workspace_bytes < need) return HYDRA_ERR_WORKSPACE_TOO_SMALL;
     const size_t ds_off = bwd_base_bytes(pb);
     if (pb.T == 0 || pb.pairs.empty()) return HYDRA_OK;
@@ -1503,7 +1620,7 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
         const size_t kv_bytes = bwd_kv_acc_bytes(pb, n_kv_heads);
         if (room < kv_bytes) return HYDRA_ERR_WORKSPACE_TOO_SMALL;
         float* dk_acc = reinterpret_cast<float*>(ws + ds_off);
-        float* dv_acc = dk_acc + static_cast<size_t>(pb.T) * n_kv_heads * pb.dqk;
+        float* dv_acc = dk_acc + static_cast<size_t>(pb.Tk) * n_kv_heads * pb.dqk;
         if (cudaMemsetAsync(dk_acc, 0, kv_bytes, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
         const BwdTensors tg{q, k, v, out, dout, lse, dq, dk_acc, dv_acc};
         if (int32_t s = bwd_run(pb, n_kv_heads, causal, softmax_scale, tg, false, true, workspace,
@@ -1540,7 +1657,7 @@ int32_t bwd_impl(const void* q, const void* k, const void* v, const void* out, c
                 if (cudaMemsetAsync(dq_acc, 0, acc_bytes, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
                 const BwdTensors tb{q, k, v, out, dout, lse, dq_acc, dk, dv};
                 Problem band_pb;
-                band_pb.cu = pb.cu; band_pb.n_seqs = pb.n_seqs; band_pb.h = pb.h; band_pb.T = pb.T; band_pb.dqk = pb.dqk;
+                band_pb.cu = pb.cu; band_pb.n_seqs = pb.n_seqs; band_pb.h = pb.h; band_pb.T = pb.T; band_pb.Tq = pb.Tq; band_pb.Tk = pb.Tk; band_pb.dqk = pb.dqk;
                 bool first = true;
                 for (const auto& band : bands) {
                     band_pb.pairs = band;
@@ -1649,6 +1766,66 @@ int32_t hydra_attn_bwd_accumulate_dims(const void* q, const void* k, const void*
 {
     return bwd_impl(q, k, v, out, lse, dout, cu, n_seqs, n_heads, pairs, n_pairs, causal, softmax_scale, dq_acc,
                     dk_acc, dv_acc, true, workspace, workspace_bytes, cuda_stream, n_kv_heads, d_qk, d_v);
+}
+
+int32_t hydra_lse_merge_local(const void* o_part, const float* lse_part, int64_t part_rows, const int32_t* cu,
+                              int32_t n_seqs, int32_t n_heads, const hydra_chunk_t* q_chunks, int32_t n_q_chunks,
+                              int64_t q_rows, const hydra_pair_t* pairs, int32_t n_pairs, int32_t accumulate, void* out,
+                              float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    // the merge touches q-side tensors only: the kv table is the q table (every pair's kv range is unused here)
+    Problem pb;
+    if (int32_t s = make_problem(cu, n_seqs, n_heads, pairs, n_pairs, pb)) return s;
+    if (!q_chunks || n_q_chunks < 1 || q_rows < 1 || q_rows > (int64_t{1} << 30)) return HYDRA_ERR_INVALID_ARG;
+    pb.qc.assign(q_chunks, q_chunks + n_q_chunks);
+    pb.Tq = q_rows;
+    for (const hydra_chunk_t& c : pb.qc)
+        if (c.seq < 0 || c.seq >= n_seqs || c.start < 0 || c.len < 0 || c.row < 0 || int64_t{c.row} + c.len > q_rows ||
+            int64_t{c.start} + c.len > int64_t{pb.cu[c.seq + 1]} - pb.cu[c.seq])
+            return HYDRA_ERR_INVALID_ARG;
+    for (const hydra_pair_t& p : pb.pairs)
+        if (p.q_len > 0 && p.part_row >= 0 &&
+            (pb.q_row(p.seq, p.q_start) < 0 ||
+             pb.q_row(p.seq, p.q_start + p.q_len - 1) != pb.q_row(p.seq, p.q_start) + p.q_len - 1))
+            return HYDRA_ERR_INVALID_ARG;
+    return merge_core(pb, o_part, lse_part, part_rows, out, lse, workspace, workspace_bytes, cuda_stream,
+                      accumulate != 0);
+}
+
+int32_t hydra_attn_bwd_accumulate_local(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                                        const void* dout, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                                        int32_t n_kv_heads, int32_t d_qk, int32_t d_v, const hydra_chunk_t* q_chunks,
+                                        int32_t n_q_chunks, int64_t q_rows, const hydra_chunk_t* kv_chunks,
+                                        int32_t n_kv_chunks, int64_t kv_rows, const hydra_pair_t* pairs,
+                                        int32_t n_pairs, int32_t causal, float softmax_scale, float* dq_acc,
+                                        float* dk_acc, float* dv_acc, void* workspace, size_t workspace_bytes,
+                                        void* cuda_stream)
+{
+    if (!kernel_set(d_qk, d_v)) return HYDRA_ERR_UNSUPPORTED;
+    Problem pb;
+    if (int32_t s = make_problem_local(cu, n_seqs, n_heads, q_chunks, n_q_chunks, q_rows, kv_chunks, n_kv_chunks,
+                                       kv_rows, pairs, n_pairs, pb))
+        return s;
+    pb.dqk = d_qk;
+    return bwd_core(pb, q, k, v, out, lse, dout, causal, softmax_scale, dq_acc, dk_acc, dv_acc, true, workspace,
+                    workspace_bytes, cuda_stream, n_kv_heads);
+}
+
+size_t hydra_workspace_bytes_local(int32_t which, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
+                                   int32_t n_kv_heads, int32_t d_qk, int32_t d_v, const hydra_chunk_t* q_chunks,
+                                   int32_t n_q_chunks, int64_t q_rows, const hydra_chunk_t* kv_chunks,
+                                   int32_t n_kv_chunks, int64_t kv_rows, const hydra_pair_t* pairs, int32_t n_pairs)
+{
+    Problem pb;
+    if (!kernel_set(d_qk, d_v) || n_kv_heads < 1 || n_heads % n_kv_heads) return 0;
+    if (make_problem_local(cu, n_seqs, n_heads, q_chunks, n_q_chunks, q_rows, kv_chunks, n_kv_chunks, kv_rows, pairs,
+                           n_pairs, pb) != HYDRA_OK)
+        return 0;
+    pb.dqk = d_qk;
+    if (which == HYDRA_WS_FWD || which == HYDRA_WS_MERGE) return kStatusBytes;
+    if (which != HYDRA_WS_BWD) return 0;
+    // the accumulating backward: D of the local q rows, plus the dS hand-off buffer when it is within the limit
+    return bwd_base_bytes(pb) + bwd_ds_bytes(ds_layout(pb, 1, nullptr), n_heads, g_ds_limit_bytes.load());
 }
 
 int32_t hydra_grad_cast(const float* acc, void* grad, int64_t n_elements, void* cuda_stream)

@@ -1,0 +1,127 @@
+"""A whole outer ring on one GPU: cp_r ranks, each with ONLY its own q / k / v chunks in local tensors, run the
+step loop of paper_2609_34318_b200.ring (forward with the kv chunks passed round, merge into the running
+(out, lse), backward with the dk / dv accumulators travelling with their chunks) through the local-layout
+entry points; the exchange is a device copy between the ranks' buffers (every rank is a thread of this
+process; no kernel of one rank waits for a kernel of another). Gathered back to the packed batch, the results
+must be the unchunked oracle's: the chunked and merged computation is an exact identity."""
+import queue
+import threading
+
+import numpy as np
+import pytest
+import torch
+
+import hydra_workloads as hw
+from gpu_util import check, run_oracle
+
+pytestmark = pytest.mark.gpu
+DQK, DV = hw.D_QK, hw.D_V
+
+
+class MailboxTransport:
+    """shift(): hand copies of the tensors to the next rank's mailbox, take the previous rank's from one's own."""
+    def __init__(self, boxes, rank):
+        self.boxes, self.rank, self.world = boxes, rank, len(boxes)
+
+    def shift(self, send, recv):
+        self.boxes[(self.rank + 1) % self.world].put([t.clone() for t in send])
+        me = self
+
+        class _Handle:
+            def wait(self_inner):
+                got = me.boxes[me.rank].get(timeout=120)
+                assert len(got) == len(recv)
+                for dst, src in zip(recv, got):
+                    dst.copy_(src)
+        return _Handle()
+
+
+def run_ring(lengths, h, cp_r, seed, h_kv=None, d_qk=DQK):
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.ring import HydraCompute, RingRank, RingSchedule
+    from paper_2609_34318_b200.runner import bits_to_tensor
+    h_kv = h_kv or h
+    cu = hw.cu_seqlens(lengths)
+    T = int(cu[-1])
+    rng = np.random.default_rng(seed)
+    f = lambda heads, d: hw.f32_to_bf16_bits(rng.standard_normal((T, heads, d)).astype(np.float32))
+    x = dict(q=f(h, d_qk), k=f(h_kv, d_qk), v=f(h_kv, DV), do=f(h, DV))
+    sched = RingSchedule(cu, cp_r)
+    boxes = [queue.Queue() for _ in range(cp_r)]
+    res, errs = {}, []
+
+    def rank_main(r):
+        try:
+            torch.cuda.set_device(0)
+            rows = torch.from_numpy(sched.global_rows(r)).cuda()
+            loc = {n: bits_to_tensor(x[n]).index_select(0, rows).contiguous() for n in x}
+            rr = RingRank(sched, r, HydraCompute(h, h_kv, d_qk, DV), MailboxTransport(boxes, r))
+            out, lse = rr.forward(loc["q"], loc["k"], loc["v"])
+            dq, dk, dv = rr.backward(loc["k"], loc["v"], loc["do"])
+            st, detail = P.hydra_poll_status(rr.workspace)
+            assert st == 0, (r, st, detail)
+            torch.cuda.synchronize()
+            res[r] = dict(rows=rows.cpu().numpy(), out=out[:len(rows)].float().cpu().numpy(),
+                          lse=lse[:, :len(rows)].cpu().numpy(), dq=dq.cpu().numpy(), dk=dk.cpu().numpy(),
+                          dv=dv.cpu().numpy(), log=list(rr.log))
+        except Exception as e:  # noqa: BLE001
+            errs.append((r, repr(e)))
+            for b in boxes:                       # do not leave the other ranks waiting
+                b.put([])
+
+    threads = [threading.Thread(target=rank_main, args=(r,)) for r in range(cp_r)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=300)
+    assert not errs, errs
+    got = dict(out=np.zeros((T, h, DV)), lse=np.zeros((h, T)), dq=np.zeros((T, h, d_qk)),
+               dk=np.zeros((T, h_kv, d_qk)), dv=np.zeros((T, h_kv, DV)))
+    for r in range(cp_r):
+        rows = res[r]["rows"]
+        got["out"][rows] = res[r]["out"]
+        got["lse"][:, rows] = res[r]["lse"]
+        for n in ("dq", "dk", "dv"):
+            # the accumulators are fp32; the contract's gradients are their bf16 rounding
+            got[n][rows] = hw.bf16_bits_to_f64(hw.f32_to_bf16_bits(res[r][n]))
+        assert res[r]["log"] == [("fwd", t, (r - t) % cp_r) for t in range(cp_r)] + \
+                                [("bwd", t, (r - t) % cp_r) for t in range(cp_r)]
+    return x, cu, got
+
+
+@pytest.mark.parametrize("lengths,h,cp_r", [([300], 4, 1), ([1000, 333], 2, 2), ([2048], 2, 4), ([700, 65, 1301, 9], 3, 4)])
+def test_ring_of_local_ranks_matches_the_unchunked_oracle(lengths, h, cp_r):
+    x, cu, got = run_ring(lengths, h, cp_r, seed=61 + cp_r)
+    check(got, run_oracle(x, cu), label=f"ring of {cp_r} over {lengths}: ")
+
+
+def test_ring_with_shared_kv_heads_of_128():
+    """The paper's grouped-query model on a ring: heads of 128, four query heads per KV head."""
+    import oracle
+    lengths, h, h_kv, cp_r, d = [900, 260], 8, 2, 2, 128
+    x, cu, got = run_ring(lengths, h, cp_r, seed=67, h_kv=h_kv, d_qk=d)
+    scale = np.float32(1.0 / np.sqrt(np.float32(d)))
+    out, lse = oracle.attn_fwd_gqa(x["q"], x["k"], x["v"], cu, True, scale)
+    dq, dk, dv = oracle.attn_bwd_gqa(x["q"], x["k"], x["v"], x["do"], cu, True, scale, out, lse)
+    check(got, dict(out=out, lse=lse, dq=dq, dk=dk, dv=dv), label="ring, grouped-query 128: ")
+
+
+def test_local_layout_arguments_are_validated():
+    import paper_2609_34318_b200 as P
+    cu = hw.cu_seqlens([256])
+    pairs, _, _, _ = P.hydra_zigzag_pairs(cu, 1)
+    z = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    qc = [(0, 0, 128, 0), (0, 128, 128, 128)]
+    ok_args = dict(q_chunks=qc, q_rows=256, kv_chunks=qc, kv_rows=256)
+    n0 = P.hydra_launch_count()
+
+    def fwd(**kw):
+        a = dict(ok_args, **kw)
+        return P.hydra_attn_fwd_local(z, z, z, cu, 1, 1, DQK, DV, a["q_chunks"], a["q_rows"], a["kv_chunks"],
+                                      a["kv_rows"], pairs, True, 0.1, z, z, z, z, 256, z, check=False)
+    assert fwd(q_chunks=[(0, 0, 128, 0), (0, 128, 128, 64)]) == P.HYDRA_ERR_INVALID_ARG      # chunks share rows
+    assert fwd(q_rows=200) == P.HYDRA_ERR_INVALID_ARG                                        # chunk past the tensor
+    assert fwd(kv_chunks=[(0, 0, 128, 0)]) == P.HYDRA_ERR_INVALID_ARG                        # a pair's keys are nowhere
+    # a q range that spans two chunks whose rows are not contiguous
+    assert fwd(q_chunks=[(0, 0, 100, 0), (0, 100, 156, 130)], q_rows=300) == P.HYDRA_ERR_INVALID_ARG
+    assert P.hydra_launch_count() == n0
