@@ -207,15 +207,20 @@ class RingRank:
         for a in self.dkv_acc[cur]:
             a.zero_()
         for t in range(R):
+            # the kv chunks move on while this step computes (they are only read); the gradients they have
+            # gathered follow once this rank has added its share. After the last step that hop brings every
+            # accumulator home.
+            kv_handle = None
+            if t + 1 < R:
+                kv_handle = self.transport.shift(list(self.kv[cur]), list(self.kv[cur ^ 1]))
             self.log.append(("bwd", t, self.sched.source(self.rank, t)))
             self.compute.backward_step(self.sched, self.rank, t, self.q, self.kv[cur][0], self.kv[cur][1], self.out,
                                        self.lse, dout, self.dq_acc, self.dkv_acc[cur][0], self.dkv_acc[cur][1],
                                        self.workspace)
-            # the chunks move on with the gradients they have gathered so far; after the last step that hop
-            # brings every accumulator home
-            send = list(self.dkv_acc[cur]) + (list(self.kv[cur]) if t + 1 < R else [])
-            recv = list(self.dkv_acc[cur ^ 1]) + (list(self.kv[cur ^ 1]) if t + 1 < R else [])
-            self.transport.shift(send, recv).wait()
+            acc_handle = self.transport.shift(list(self.dkv_acc[cur]), list(self.dkv_acc[cur ^ 1]))
+            if kv_handle is not None:
+                kv_handle.wait()
+            acc_handle.wait()
             cur ^= 1
         dk, dv = self.dkv_acc[cur]
         return self.dq_acc[:rows], dk[:rows], dv[:rows]

@@ -105,3 +105,32 @@ def test_three_hundred_distinct_shapes_allocate_nothing_and_stay_correct():
         torch.cuda.synchronize()
         P.hydra_shutdown()
         P.hydra_set_plan_arena_bytes(32 << 20)
+
+
+def test_results_do_not_depend_on_the_table_prefetch():
+    """hydra_attn_fwd builds the tables of the merge and the backward ahead of their calls (host work only); with
+    that switched off the same problems must give the same bits."""
+    import paper_2609_34318_b200 as P
+    from gpu_util import pairs_for, run_gpu
+    rng = np.random.default_rng(43)
+    cases = [([300, 77, 1001], 1), ([513, 64], 0), ([640, 200, 65], 2)]
+    results = {}
+    for prefetch in (True, False):
+        P.hydra_shutdown()                              # forget every cached table: both passes build their own
+        P.hydra_set_plan_prefetch(prefetch)
+        try:
+            for i, (lengths, cp_r) in enumerate(cases):
+                cu = hw.cu_seqlens(lengths)
+                T = int(cu[-1])
+                r = np.random.default_rng(100 + i)
+                x = {n: hw.f32_to_bf16_bits(r.standard_normal((T, 2, DV if n in ("v", "do") else DQK)).astype(np.float32))
+                     for n in ("q", "k", "v", "do")}
+                lib_pairs, rows, _ = pairs_for(cu, cp_r) if cp_r else (None, 0, None)
+                got = run_gpu(x, cu, 2, lib_pairs, rows)
+                results[(prefetch, i)] = {n: got[n] for n in ("out", "lse", "dq", "dk", "dv")}
+        finally:
+            P.hydra_set_plan_prefetch(True)
+    for i in range(len(cases)):
+        for n in ("out", "lse", "dq", "dk", "dv"):
+            assert np.array_equal(results[(True, i)][n], results[(False, i)][n], equal_nan=True), (i, n)
+    del rng
