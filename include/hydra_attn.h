@@ -15,9 +15,10 @@
  *     T = cu_seqlens[n_seqs]; sequence b owns tokens [cu_seqlens[b], cu_seqlens[b+1]).
  *   - Every call returns a status (HYDRA_OK = 0). Work is enqueued on `cuda_stream` (a
  *     cudaStream_t passed as void*; NULL = the legacy default stream); results are valid once the
- *     stream has been synchronised. No call synchronises the device except hydra_poll_status and,
- *     the first time a given (cu_seqlens, pairs, h) combination is seen, the internal cudaMalloc of
- *     its cached work lists (freed by hydra_shutdown).
+ *     stream has been synchronised. No call synchronises the device except hydra_poll_status,
+ *     hydra_shutdown and the first compute call on a device, which allocates the library's table
+ *     arena (see hydra_set_plan_arena_bytes): a new (cu_seqlens, pairs, h) combination costs host
+ *     work and an asynchronous copy on `cuda_stream`, no allocation and no wait.
  *   - The caller owns all tensors and the workspace; the library keeps no caller pointer.
  *   - A workspace carries the status word and the work-queue counters of the kernels of one call:
  *     each call clears them (on its stream) before it launches, so calls that may run at the same
@@ -198,8 +199,8 @@ int32_t hydra_lse_merge_accumulate(const void* o_part, const float* lse_part, in
  * hydra_lse_merge for callers that must not allocate device memory. (No counterpart in the paper:
  * this is a property of the library, not of the method.) It computes exactly what hydra_lse_merge
  * computes, with the same kernel, but keeps the per-problem tables (the partials of every q chunk,
- * cut into blocks of rows) in a fixed array inside the library image instead of in memory obtained
- * with cudaMalloc, and it needs no workspace. It calls no cudaMalloc, cudaFree or other allocating
+ * cut into blocks of rows) in a fixed array inside the library image instead of in the arena that the
+ * other entry points obtain with cudaMalloc at their first call, and it needs no workspace. It calls no cudaMalloc, cudaFree or other allocating
  * routine. It is meant for processes that have handed all device memory to their own pool, and for
  * latency-critical loops whose rules forbid cudaMalloc because it may synchronise the device.
  *   - Limits (HYDRA_ERR_UNSUPPORTED beyond them): at most HYDRA_NOALLOC_MAX_GROUPS merged q chunks,

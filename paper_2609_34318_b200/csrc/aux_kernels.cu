@@ -279,7 +279,8 @@ cudaError_t launch_bwd_prep(const void* dout, const void* out, float* dsum, int6
 // hydra_lse_merge_noalloc: the merge for callers that must not allocate device memory
 // =============================================================================================
 // hydra_lse_merge keeps its per-problem tables (which q chunk has which partials, cut into blocks of
-// rows) in device memory that the library obtains with cudaMalloc the first time it sees a problem.
+// rows) in an arena of device memory that the library obtains with cudaMalloc at its first call on a
+// device (and a problem with very large tables gets an allocation of its own).
 // Some callers cannot have that: a process that has handed all device memory to its own pool and
 // leaves nothing for cudaMalloc to find, or a latency-critical loop whose rules forbid cudaMalloc
 // because it may synchronise the whole device. This entry point runs the same kernel with the tables
