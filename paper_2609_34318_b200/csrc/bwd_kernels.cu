@@ -635,8 +635,10 @@ HYDRA_K(hydra_bwd_dkv_kernel)(const __grid_constant__ CUtensorMap map_q, const _
     __shared__ int32_t s_sched[kSched];
     __shared__ GroupItem s_item[kSched];              // the work ring carries the item and its first pair, so that
     __shared__ PairDev s_first[kSched];               // no role starts an item with a walk through global memory
-    __shared__ float s_lse2[kStages][SUB];
-    __shared__ float s_dsum[kStages][SUB];
+    // -LSE * log2(e) and -D of the q rows of a sub-tile (negated by the producer: they are addends of packed
+    // two-element operations, which have no operand negation; 16-byte aligned: read four columns at a time)
+    __shared__ __align__(16) float s_lse2[kStages][SUB];
+    __shared__ __align__(16) float s_dsum[kStages][SUB];
     __shared__ uint32_t s_bursts;                      // S / dP bursts issued so far (all ones: no more)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -774,8 +776,8 @@ HYDRA_K(hydra_bwd_dkv_kernel)(const __grid_constant__ CUtensorMap map_q, const _
                     const bool v = i < si.cur.q_len;
                     const int64_t idx = static_cast<int64_t>(item.head) * p.T + si.cur.q_tok0 + i;
                     const float l = v ? __ldg(p.lse + idx) : neg_inf();
-                    s_lse2[st][c] = (l == neg_inf()) ? pos_inf() : l * kLog2e;
-                    s_dsum[st][c] = v ? __ldg(p.dsum + idx) : 0.f;
+                    s_lse2[st][c] = (l == neg_inf()) ? neg_inf() : -(l * kLog2e);
+                    s_dsum[st][c] = v ? -__ldg(p.dsum + idx) : 0.f;
                 }
                 mbar_arrive_warp(bar(B_STAT + st));
                 if (!popped) {
@@ -945,32 +947,42 @@ HYDRA_K(hydra_bwd_dkv_kernel)(const __grid_constant__ CUtensorMap map_q, const _
                 if (p.causal) c_lo = max(0, krow - si.cur.off - base);
                 int c_hi = min(32, si.cur.q_len - base);
                 if (!row_valid) c_hi = 0;
-                const float* lse2 = &s_lse2[st][g * 32];
-                const float* dsum = &s_dsum[st][g * 32];
+                const float4* nlse4 = reinterpret_cast<const float4*>(&s_lse2[st][g * 32]);
+                const float4* ndsum4 = reinterpret_cast<const float4*>(&s_dsum[st][g * 32]);
                 uint32_t pk[16], ds[16];
                 // interior sub-tiles (every q row visible from every kv row of the warp) skip the masking
                 if (__any_sync(0xffffffffu, c_lo > 0 || c_hi < 32)) {
 #pragma unroll
-                    for (int c = 0; c < 32; c += 2) {
-                        float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2[c]));
-                        float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2[c + 1]));
-                        if (c < c_lo || c >= c_hi) p0 = 0.f;
-                        if (c + 1 < c_lo || c + 1 >= c_hi) p1 = 0.f;
-                        pk[c >> 1] = pack_bf16x2(p0, p1);
-                        ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum[c]),
-                                                 p1 * (__uint_as_float(dp[c + 1]) - dsum[c + 1]));
+                    for (int c = 0; c < 32; c += 4) {
+                        const float4 nl = nlse4[c >> 2], nd = ndsum4[c >> 2];
+                        const float nlv[4] = {nl.x, nl.y, nl.z, nl.w}, ndv[4] = {nd.x, nd.y, nd.z, nd.w};
+#pragma unroll
+                        for (int e = 0; e < 4; e += 2) {
+                            float p0 = ex2_approx(fmaf(__uint_as_float(s[c + e]), p.scale_log2, nlv[e]));
+                            float p1 = ex2_approx(fmaf(__uint_as_float(s[c + e + 1]), p.scale_log2, nlv[e + 1]));
+                            if (c + e < c_lo || c + e >= c_hi) p0 = 0.f;
+                            if (c + e + 1 < c_lo || c + e + 1 >= c_hi) p1 = 0.f;
+                            pk[(c + e) >> 1] = pack_bf16x2(p0, p1);
+                            ds[(c + e) >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c + e]) + ndv[e]),
+                                                           p1 * (__uint_as_float(dp[c + e + 1]) + ndv[e + 1]));
+                        }
                     }
                 } else {
 #pragma unroll
-                    for (int c = 0; c < 32; c += 2) {
-                        float x0, x1, d0, d1;
-                        ffma2(x0, x1, __uint_as_float(s[c]), __uint_as_float(s[c + 1]), p.scale_log2, p.scale_log2,
-                              -lse2[c], -lse2[c + 1]);
-                        const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
-                        fadd2(d0, d1, __uint_as_float(dp[c]), __uint_as_float(dp[c + 1]), -dsum[c], -dsum[c + 1]);
-                        fmul2(d0, d1, d0, d1, p0, p1);
-                        pk[c >> 1] = pack_bf16x2(p0, p1);
-                        ds[c >> 1] = pack_bf16x2(d0, d1);
+                    for (int c = 0; c < 32; c += 4) {
+                        const float4 nl = nlse4[c >> 2], nd = ndsum4[c >> 2];
+                        const float nlv[4] = {nl.x, nl.y, nl.z, nl.w}, ndv[4] = {nd.x, nd.y, nd.z, nd.w};
+#pragma unroll
+                        for (int e = 0; e < 4; e += 2) {
+                            float x0, x1, d0, d1;
+                            ffma2(x0, x1, __uint_as_float(s[c + e]), __uint_as_float(s[c + e + 1]), p.scale_log2,
+                                  p.scale_log2, nlv[e], nlv[e + 1]);
+                            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                            fadd2(d0, d1, __uint_as_float(dp[c + e]), __uint_as_float(dp[c + e + 1]), ndv[e], ndv[e + 1]);
+                            fmul2(d0, d1, d0, d1, p0, p1);
+                            pk[(c + e) >> 1] = pack_bf16x2(p0, p1);
+                            ds[(c + e) >> 1] = pack_bf16x2(d0, d1);
+                        }
                     }
                 }
                 if (c_pds > 0) {                       // the previous dV / dK updates have read P and dS
