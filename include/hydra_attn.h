@@ -557,6 +557,17 @@ void hydra_set_plan_arena_bytes(uint64_t bytes);
  */
 void hydra_set_plan_prefetch(int32_t on);
 /*
+ * The forward has two kernels. Pairs whose q range AND kv range are at most `len` tokens long go to the
+ * short-sequence kernel (one CTA per SM, two independent 128-row q tiles in flight, steps of 64 keys: the
+ * regime of Section 2.2, where most sequences are short and a tile's chain of dependent steps, not the tensor
+ * core, sets the pace), all others to the CTA-pair kernel; if the short pairs carry less than a quarter of a
+ * call's work, that call uses the CTA-pair kernel alone. Both compute the same function to the same tolerance
+ * (not bit for bit: their summation orders differ). len = 0 switches the short-sequence kernel off; the
+ * default is 1536 (where the two kernels take equal time on sequences of one length). Takes effect with the next
+ * call.
+ */
+void hydra_set_fwd_short_len(int32_t len);
+/*
  * Host only (no GPU needed): seconds the host takes to build the work tables of one call of kind `which`
  * (HYDRA_WS_FWD / MERGE / BWD) for this problem, uncached. What a new cu_seqlens costs before its first launch.
  * Negative on invalid arguments.

@@ -76,6 +76,8 @@ def _load() -> ctypes.CDLL:
     lib.hydra_plan_build_seconds.argtypes = [i32, vp, i32, i32, vp, i32, i32]
     lib.hydra_set_plan_prefetch.argtypes = [i32]
     lib.hydra_set_plan_prefetch.restype = None
+    lib.hydra_set_fwd_short_len.argtypes = [i32]
+    lib.hydra_set_fwd_short_len.restype = None
     lib.hydra_usp_factor.restype = i32
     lib.hydra_usp_factor.argtypes = [i32, i32, vp, vp]
     lib.hydra_zigzag_pairs.restype = i32
@@ -174,7 +176,7 @@ def _load() -> ctypes.CDLL:
 
 _lib = _load()
 LIBRARY_PATH = _build.OUT
-EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_set_wait_limit_ns", "hydra_debug_stall", "hydra_set_plan_arena_bytes", "hydra_set_plan_prefetch", "hydra_plan_build_seconds",
+EXPORTS = ("hydra_version", "hydra_status_string", "hydra_launch_count", "hydra_set_wait_limit_ns", "hydra_debug_stall", "hydra_set_plan_arena_bytes", "hydra_set_plan_prefetch", "hydra_set_fwd_short_len", "hydra_plan_build_seconds",
            "hydra_shutdown", "hydra_usp_factor", "hydra_zigzag_pairs", "hydra_workspace_bytes",
            "hydra_attn_fwd", "hydra_lse_merge", "hydra_attn_bwd", "hydra_poll_status",
            "hydra_profile_enable", "hydra_profile_collect", "hydra_host_step_arena_bytes",
@@ -287,6 +289,11 @@ def hydra_plan_build_seconds(which: int, cu_seqlens, n_heads: int, pairs=None, c
 def hydra_set_plan_prefetch(on: bool) -> None:
     """Build the merge / backward tables of a problem on the host while its forward runs (default on)."""
     _lib.hydra_set_plan_prefetch(int(bool(on)))
+
+
+def hydra_set_fwd_short_len(length: int) -> None:
+    """Pairs with q and kv ranges of at most `length` tokens use the short-sequence forward kernel (0: off)."""
+    _lib.hydra_set_fwd_short_len(int(length))
 
 
 def hydra_set_plan_arena_bytes(nbytes: int) -> None:

@@ -13,9 +13,10 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 OUT = os.path.join(PKG, "libhydra_attn.so")
 OBJ_DIR = os.path.join(PKG, "build")
-SOURCES = ["api.cu", "fwd_kernel.cu", "bwd_kernels.cu", "aux_kernels.cu", "mla_ops.cu", "sched.cu"]
+SOURCES = ["api.cu", "fwd_kernel.cu", "fwd_short_kernel.cu", "bwd_kernels.cu", "aux_kernels.cu", "mla_ops.cu", "sched.cu"]
 # the tensor-core kernel files are compiled a second time for q / k heads of 128 (own symbol names)
-VARIANTS = [("fwd_kernel.cu", "d128", ["-DHYDRA_KERNEL_DQK=128"]), ("bwd_kernels.cu", "d128", ["-DHYDRA_KERNEL_DQK=128"])]
+VARIANTS = [("fwd_kernel.cu", "d128", ["-DHYDRA_KERNEL_DQK=128"]), ("fwd_short_kernel.cu", "d128", ["-DHYDRA_KERNEL_DQK=128"]),
+            ("bwd_kernels.cu", "d128", ["-DHYDRA_KERNEL_DQK=128"])]
 HEADERS = ["hydra_internal.h", "sm100_ptx.cuh", os.path.join("..", "..", "include", "hydra_attn.h"),
            os.path.join("..", "..", "include", "hydra_sched.h")]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")

@@ -417,6 +417,11 @@ void arena_note_use(const Plan& plan, int device, cudaStream_t stream)
     users.emplace_back(stream, e);
 }
 
+// Pairs whose q range and kv range are both at most this long go to the short-sequence forward kernel
+// (0: none do). See build_fwd.
+std::atomic<int32_t> g_fwd_short_len{1536};
+static_assert(FWD_SHORT_KEYS == SUB, "the short forward kernel reads K through the 64-row map of the CTA-pair kernel");
+
 std::vector<uint8_t> make_key(int kind, int device, const Problem& pb, int causal)
 {
     std::vector<uint8_t> key;
@@ -424,7 +429,8 @@ std::vector<uint8_t> make_key(int kind, int device, const Problem& pb, int causa
         const uint8_t* b = static_cast<const uint8_t*>(p);
         key.insert(key.end(), b, b + n);
     };
-    const int32_t head[6] = {kind, device, pb.h, causal, pb.n_seqs, 0};
+    // the forward's tables depend on which pairs go to the short-sequence kernel
+    const int32_t head[6] = {kind, device, pb.h, causal, pb.n_seqs, kind == HYDRA_WS_FWD ? g_fwd_short_len.load() : 0};
     put(head, sizeof head);
     put(pb.cu.data(), pb.cu.size() * sizeof(int32_t));
     put(pb.pairs.data(), pb.pairs.size() * sizeof(hydra_pair_t));
@@ -626,11 +632,44 @@ std::vector<Item> order_by_groups(std::vector<std::vector<GroupEntry>>& groups, 
     return items;
 }
 
+// Steps of FWD_SHORT_KEYS keys that the q rows [q0, q0 + rows) of a pair visit in the short-sequence kernel
+inline int32_t kv_steps_short(const hydra_pair_t& p, int32_t q0, int32_t rows, int causal)
+{
+    int64_t n_keys = p.k_len;
+    if (causal) n_keys = std::min<int64_t>(n_keys, int64_t{q0} + rows - 1 + (p.q_start - p.k_start) + 1);
+    return n_keys > 0 ? static_cast<int32_t>((n_keys + FWD_SHORT_KEYS - 1) / FWD_SHORT_KEYS) : 0;
+}
+
 void build_fwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& blob)
 {
-    std::vector<std::vector<GroupEntry>> groups(pb.pairs.size());
+    // Which pairs go to the short-sequence kernel (one CTA per SM, two independent 128-row tiles in flight,
+    // steps of 64 keys): those whose q range and kv range are both short. On such pairs the CTA-pair kernel is
+    // bound by the length of a tile's chain of steps, and more, shorter chains per SM win; on long pairs its
+    // operand sharing and its 256-row tiles do. A second launch has a price of its own (its start and its
+    // tail), so the short kernel is used only if the short pairs carry at least a quarter of the call's work.
+    const int32_t short_len = g_fwd_short_len.load();
+    std::vector<uint8_t> is_short(pb.pairs.size(), 0);
+    {
+        double work_short = 0, work_all = 0;
+        for (size_t pi = 0; pi < pb.pairs.size(); ++pi) {
+            const auto& p = pb.pairs[pi];
+            const double w = static_cast<double>(p.q_len) * p.k_len;
+            work_all += w;
+            if (short_len > 0 && p.q_len <= short_len && p.k_len <= short_len) { is_short[pi] = 1; work_short += w; }
+        }
+        if (work_short * 4 < work_all) std::fill(is_short.begin(), is_short.end(), 0);
+    }
+    std::vector<std::vector<GroupEntry>> groups(pb.pairs.size()), groups_short(pb.pairs.size());
     for (size_t pi = 0; pi < pb.pairs.size(); ++pi) {
         const auto& p = pb.pairs[pi];
+        if (is_short[pi]) {
+            for (int32_t q0 = 0; q0 < p.q_len; q0 += TILE) {
+                const int32_t rows = std::min(TILE, p.q_len - q0);
+                const int32_t n_kv = kv_steps_short(p, q0, rows, causal);
+                groups_short[pi].push_back(GroupEntry{q0, n_kv, rows, n_kv});
+            }
+            continue;
+        }
         // One item = two consecutive 256-row UMMA tiles (A, then B) of a CTA pair. The slabs are aligned to
         // the END of the q chunk: with an odd number of 256-row tiles the chunk's FIRST tile goes alone (it
         // visits the fewest kv tiles), so the ragged last tile rides with a full neighbour instead of running
@@ -653,9 +692,19 @@ void build_fwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& 
     const std::vector<FwdItem> items = order_by_groups<FwdItem>(
         groups, pb.h, plan_workers(2),
         [](int32_t g, int32_t a, const GroupEntry& e) { return FwdItem{g, a, e.a, e.b, e.c, {0, 0, 0}}; });
-    plan.off_pairs = append(blob, device_pairs(pb));
+    const std::vector<PairDev> dev_pairs = device_pairs(pb);
+    // the short kernel's items carry what they need of their pair (its slots start an item from this alone)
+    const std::vector<FwdShortItem> short_items = order_by_groups<FwdShortItem>(
+        groups_short, pb.h, 2 * plan_workers(1), [&](int32_t g, int32_t a, const GroupEntry& e) {
+            const PairDev& d = dev_pairs[g];
+            return FwdShortItem{d.q_tok0 + e.a, e.c, d.k_tok0, d.k_len, e.a + d.off, e.b, a, d.out_row0 + e.a,
+                                d.to_part, {0, 0, 0}};
+        });
+    plan.off_pairs = append(blob, dev_pairs);
     plan.off_items = append(blob, items);
     plan.n_items = static_cast<int32_t>(items.size());
+    plan.off_items2 = append(blob, short_items);
+    plan.n_items2 = static_cast<int32_t>(short_items.size());
 }
 
 void build_merge(const Problem& pb, Plan& plan, std::vector<uint8_t>& blob)
@@ -918,6 +967,8 @@ struct KernelSet {
     int (*fwd_max_clusters)();
     cudaError_t (*launch_fwd)(const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, const FwdParams&, int,
                               cudaStream_t);
+    cudaError_t (*launch_fwd_short)(const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, const FwdParams&, int,
+                                    cudaStream_t);
     cudaError_t (*launch_bwd_dq)(const CUtensorMap&, const CUtensorMap&, const CUtensorMap&, const CUtensorMap&,
                                  const BwdParams&, int, cudaStream_t);
     cudaError_t (*launch_bwd_dq_from_ds)(const CUtensorMap&, const BwdParams&, int, cudaStream_t);
@@ -926,8 +977,8 @@ struct KernelSet {
 };
 const KernelSet* kernel_set(int32_t d_qk, int32_t d_v)
 {
-    static const KernelSet k192{fwd_max_clusters, launch_fwd, launch_bwd_dq, launch_bwd_dq_from_ds, launch_bwd_dkv};
-    static const KernelSet k128{fwd_max_clusters_d128, launch_fwd_d128, launch_bwd_dq_d128, launch_bwd_dq_from_ds_d128,
+    static const KernelSet k192{fwd_max_clusters, launch_fwd, launch_fwd_short, launch_bwd_dq, launch_bwd_dq_from_ds, launch_bwd_dkv};
+    static const KernelSet k128{fwd_max_clusters_d128, launch_fwd_d128, launch_fwd_short_d128, launch_bwd_dq_d128, launch_bwd_dq_from_ds_d128,
                                 launch_bwd_dkv_d128};
     if (d_v != D_V) return nullptr;
     if (d_qk == 192) return &k192;
@@ -1039,6 +1090,8 @@ void hydra_shutdown(void)
 void hydra_set_plan_arena_bytes(uint64_t bytes) { g_arena_bytes.store(bytes); }
 
 void hydra_set_plan_prefetch(int32_t on) { g_plan_prefetch.store(on != 0); }
+
+void hydra_set_fwd_short_len(int32_t len) { g_fwd_short_len.store(len > 0 ? len : 0); }
 
 double hydra_plan_build_seconds(int32_t which, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
                                 const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal)
@@ -1284,22 +1337,17 @@ int32_t fwd_core(Problem& pb, const void* q, const void* k, const void* v, int32
     if (int32_t s = device_info(&sms)) return s;
     if (pb.pairs.empty()) return HYDRA_OK;
 
-    const int n_clusters = ks->fwd_max_clusters();        // CTA pairs resident at once: the persistent grid
-    if (n_clusters < 1) return HYDRA_ERR_CUDA;
     PlanLease lease;
     if (int32_t s = lease.acquire(HYDRA_WS_FWD, pb, causal != 0, stream)) return s;
     const Plan* plan = &lease.plan();
-    if (plan->n_items == 0) return HYDRA_OK;
-    // each CTA of a pair stages 64 kv rows of K (box of 64 rows) and 64 value columns of V
-    CUtensorMap mq, mk, mv;
-    if (make_map(&mq, q, pb.Tq, n_heads, pb.dqk, TILE) || make_map(&mk, k, pb.Tk, n_kv_heads, pb.dqk, SUB) ||
-        make_map(&mv, v, pb.Tk, n_kv_heads, D_V, TILE))
-        return HYDRA_ERR_CUDA;
+    if (plan->n_items == 0 && plan->n_items2 == 0) return HYDRA_OK;
     if (int32_t s = reset_status(workspace, stream)) return s;
     FwdParams fp{};
     fp.pairs = lease.at<PairDev>(plan->off_pairs);
     fp.items = lease.at<FwdItem>(plan->off_items);
     fp.n_items = plan->n_items;
+    fp.short_items = lease.at<FwdShortItem>(plan->off_items2);
+    fp.n_short = plan->n_items2;
     fp.out = out; fp.lse = lse; fp.o_part = o_part; fp.lse_part = lse_part;
     fp.T = pb.Tq; fp.part_rows = part_rows; fp.h = n_heads; fp.causal = causal != 0;
     fp.kv_group = n_heads / n_kv_heads;
@@ -1307,11 +1355,29 @@ int32_t fwd_core(Problem& pb, const void* q, const void* k, const void* v, int32
     fp.status = static_cast<StatusBlock*>(workspace);
     fp.wait_limit_ns = g_wait_limit_ns.load();
     fp.debug_stall_ns = g_debug_stall_ns[HYDRA_STALL_FWD].load();
-    {
+    CUtensorMap mq, mk;
+    if (make_map(&mq, q, pb.Tq, n_heads, pb.dqk, TILE) || make_map(&mk, k, pb.Tk, n_kv_heads, pb.dqk, SUB))
+        return HYDRA_ERR_CUDA;
+    if (plan->n_items > 0) {
+        // long pairs, on CTA pairs: each CTA of a pair stages 64 kv rows of K (box of 64 rows) and 64 value
+        // columns of V
+        const int n_clusters = ks->fwd_max_clusters();    // CTA pairs resident at once: the persistent grid
+        if (n_clusters < 1) return HYDRA_ERR_CUDA;
+        CUtensorMap mv;
+        if (make_map(&mv, v, pb.Tk, n_kv_heads, D_V, TILE)) return HYDRA_ERR_CUDA;
         ScopedKernelTimer timer(K_FWD, stream);
         if (ks->launch_fwd(mq, mk, mv, fp, n_clusters, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+        g_launches += 1;
     }
-    g_launches += 1;
+    if (plan->n_items2 > 0) {
+        // short pairs: one CTA per SM with two work items in flight, K and V in boxes of 64 keys
+        CUtensorMap mv_sub;
+        if (make_map(&mv_sub, v, pb.Tk, n_kv_heads, D_V, FWD_SHORT_KEYS)) return HYDRA_ERR_CUDA;
+        const int grid = std::min(sms, (plan->n_items2 + 1) / 2);
+        ScopedKernelTimer timer(K_FWD, stream);
+        if (ks->launch_fwd_short(mq, mk, mv_sub, fp, grid, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
+        g_launches += 1;
+    }
     lease.release();                                   // the tables have their reader on record
     prefetch_plans(pb, causal != 0, any_part);
     return HYDRA_OK;

@@ -12,6 +12,7 @@ constexpr int D_QK = HYDRA_D_QK;
 constexpr int D_V = HYDRA_D_V;
 constexpr int TILE = 128;       // rows of a q tile and of a kv tile
 constexpr int SUB = 64;         // rows of a q sub-tile in the key-side backward kernel
+constexpr int FWD_SHORT_KEYS = 64;   // keys per step of the short-sequence forward kernel
 
 // One (q-chunk, kv-chunk) pair with absolute token offsets, as the kernels see it.
 struct PairDev {
@@ -66,6 +67,21 @@ struct FwdItem {
     int32_t pad[3];
 };
 
+// Work item of the short-sequence forward kernel: one 128-row q tile of one pair and head, self-contained
+// (a slot of that kernel reads nothing else to start it).
+struct FwdShortItem {
+    int32_t q_tok0;    // token index of the tile's first q row
+    int32_t rows;      // q rows of the tile that exist (1..128)
+    int32_t k_tok0;    // token index of the pair's first kv row
+    int32_t k_len;
+    int32_t off;       // key j is visible to row r of the tile iff j <= r + off (causal)
+    int32_t n_kv;      // steps of FWD_SHORT_KEYS keys the tile visits; 0: its rows see no key
+    int32_t head;
+    int32_t out_row0;  // output row of the tile's first q row (partial buffers or out / lse)
+    int32_t to_part;   // 1: partial buffers, 0: out / lse
+    int32_t pad[3];
+};
+
 // Backward work item: one tile of one chunk and head, visiting every pair that shares the chunk.
 struct GroupItem {
     int32_t list_off;  // first entry of the chunk's pair list
@@ -91,13 +107,13 @@ struct StatusBlock {            // lives at the start of the workspace; zeroed b
     int32_t status;
     int32_t pad;
     int64_t detail;
-    int32_t next_item[4];       // work-queue heads of the persistent kernels (forward, dK/dV, dQ)
+    int32_t next_item[4];       // work-queue heads of the persistent kernels (forward, dK/dV, dQ, short forward)
     // SM clock seen from inside the tensor-core kernels: cycles and nanoseconds that passed in the
     // producer thread of CTA 0 between its first and its last instruction (same index as next_item)
     uint64_t probe_cycles[4];
     uint64_t probe_ns[4];
 };
-enum : int { QUEUE_FWD = 0, QUEUE_DKV = 1, QUEUE_DQ = 2 };
+enum : int { QUEUE_FWD = 0, QUEUE_DKV = 1, QUEUE_DQ = 2, QUEUE_FWD_SHORT = 3 };
 
 #ifdef __CUDACC__
 // The clock the driver reports between kernels says little about a 1 ms kernel on a power-capped part;
@@ -123,6 +139,8 @@ struct FwdParams {
     const PairDev* pairs;
     const FwdItem* items;
     int32_t n_items;
+    const FwdShortItem* short_items;   // the pairs that go to the short-sequence kernel
+    int32_t n_short;
     void* out; float* lse; void* o_part; float* lse_part;
     int64_t T; int64_t part_rows;
     int32_t h; int32_t causal;
@@ -174,6 +192,9 @@ struct MergeParams {
     size_t bwd_dq_ds_smem_bytes##SUFFIX();                                                                            \
     cudaError_t launch_fwd##SUFFIX(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,               \
                                    const FwdParams& p, int grid, cudaStream_t stream);                                \
+    size_t fwd_short_smem_bytes##SUFFIX();                                                                            \
+    cudaError_t launch_fwd_short##SUFFIX(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv_sub,     \
+                                         const FwdParams& p, int grid, cudaStream_t stream);                          \
     cudaError_t launch_bwd_dq##SUFFIX(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,            \
                                       const CUtensorMap& mdo, const BwdParams& p, int grid, cudaStream_t stream);     \
     cudaError_t launch_bwd_dq_from_ds##SUFFIX(const CUtensorMap& mk, const BwdParams& p, int grid,                    \

@@ -13,15 +13,17 @@ import pytest
 import torch
 
 import hydra_workloads as hw
+from conftest import FWD_SHORT_LEN_DEFAULT
 from gpu_util import check, pairs_for, run_gpu, run_oracle
 
 pytestmark = pytest.mark.gpu
 
-CASES = {                       # name -> (kernel to stall, dS hand-off limit in bytes)
-    "forward": ("HYDRA_STALL_FWD", 4 << 30),
-    "backward_key_side": ("HYDRA_STALL_BWD_DKV", 4 << 30),
-    "backward_query_side_from_ds": ("HYDRA_STALL_BWD_DQ", 4 << 30),
-    "backward_query_side_recomputing": ("HYDRA_STALL_BWD_DQ", 0),
+CASES = {                       # name -> (kernel to stall, dS hand-off limit in bytes, forward's short-pair limit)
+    "forward_cta_pairs": ("HYDRA_STALL_FWD", 4 << 30, 0),
+    "forward_short_sequences": ("HYDRA_STALL_FWD", 4 << 30, 1 << 20),
+    "backward_key_side": ("HYDRA_STALL_BWD_DKV", 4 << 30, None),
+    "backward_query_side_from_ds": ("HYDRA_STALL_BWD_DQ", 4 << 30, None),
+    "backward_query_side_recomputing": ("HYDRA_STALL_BWD_DQ", 0, None),
 }
 
 
@@ -35,6 +37,8 @@ def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_correct(case):
     cu = w.cu()
     lib_pairs, rows, ora_pairs = pairs_for(cu, [0, 0, 0, 1])      # the 300-token sequence is cut and merged
     P.hydra_set_bwd_scratch_limit(CASES[case][1])
+    if CASES[case][2] is not None:
+        P.hydra_set_fwd_short_len(CASES[case][2])
     try:
         step = AttnStep(cu, w.n_heads, lib_pairs, rows)
         q, k, v, do = (bits_to_tensor(x[n]) for n in ("q", "k", "v", "do"))
@@ -62,3 +66,4 @@ def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_correct(case):
         check(got, ref, label=f"after a timed-out {case}: ")
     finally:
         P.hydra_set_bwd_scratch_limit(4 << 30)
+        P.hydra_set_fwd_short_len(FWD_SHORT_LEN_DEFAULT)

@@ -8,7 +8,7 @@ import hydra_workloads as hw
 import oracle
 from gpu_util import check, pairs_for
 
-pytestmark = pytest.mark.gpu
+pytestmark = [pytest.mark.gpu, pytest.mark.usefixtures("both_forward_kernels")]
 DQK, DV = hw.D_QK, hw.D_V
 
 

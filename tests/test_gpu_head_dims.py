@@ -10,7 +10,7 @@ import hydra_workloads as hw
 import oracle
 from gpu_util import check, guard, pairs_for
 
-pytestmark = pytest.mark.gpu
+pytestmark = [pytest.mark.gpu, pytest.mark.usefixtures("both_forward_kernels")]
 D = 128
 
 

@@ -10,7 +10,7 @@ import hydra_workloads as hw
 import oracle
 from gpu_util import TOL_LSE, TOL_REL, check, pairs_for, row_rel_err, run_gpu, run_oracle
 
-pytestmark = pytest.mark.gpu
+pytestmark = [pytest.mark.gpu, pytest.mark.usefixtures("both_forward_kernels")]
 DQK, DV = hw.D_QK, hw.D_V
 
 

@@ -14,7 +14,7 @@ import torch
 import hydra_workloads as hw
 from gpu_util import check, run_oracle
 
-pytestmark = pytest.mark.gpu
+pytestmark = [pytest.mark.gpu, pytest.mark.usefixtures("both_forward_kernels")]
 DQK, DV = hw.D_QK, hw.D_V
 
 
