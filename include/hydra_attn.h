@@ -504,7 +504,8 @@ int32_t hydra_poll_status(void* workspace, void* cuda_stream, int32_t* device_st
  * part of the method). The producer thread of thread block 0 of every tensor-core kernel reads the
  * cycle counter and the nanosecond timer when it starts and when it has issued its last load;
  * mhz_out[3] receives cycles / microsecond for the forward, the key-side backward and the query-side
- * backward kernel (0 for a kernel the call did not run). Synchronises the stream. On a power-capped
+ * backward kernel (0 for a kernel the call did not run; the forward's figure is the CTA-pair kernel's if the
+ * call used it, else the short-sequence kernel's). Synchronises the stream. On a power-capped
  * part this is the clock the kernel really ran at; the driver's clock query, sampled between
  * kernels, is not.
  */

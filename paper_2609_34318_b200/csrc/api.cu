@@ -2219,8 +2219,11 @@ int32_t hydra_poll_clocks(void* workspace, void* cuda_stream, double* mhz_out)
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return HYDRA_ERR_CUDA;
     StatusBlock sb;
     if (cudaMemcpy(&sb, workspace, sizeof sb, cudaMemcpyDeviceToHost) != cudaSuccess) return HYDRA_ERR_CUDA;
-    for (int i = 0; i < 3; ++i)
-        mhz_out[i] = sb.probe_ns[i] ? 1e3 * static_cast<double>(sb.probe_cycles[i]) / static_cast<double>(sb.probe_ns[i]) : 0.0;
+    for (int i = 0; i < 3; ++i) {
+        // the forward's figure comes from the CTA-pair kernel if the call used it, else from the short-sequence one
+        const int src = (i == QUEUE_FWD && !sb.probe_ns[i]) ? QUEUE_FWD_SHORT : i;
+        mhz_out[i] = sb.probe_ns[src] ? 1e3 * static_cast<double>(sb.probe_cycles[src]) / static_cast<double>(sb.probe_ns[src]) : 0.0;
+    }
     return HYDRA_OK;
 }
 
