@@ -593,11 +593,14 @@ void order_items(std::vector<Item>& items, const std::vector<int32_t>& block_of,
 // longest item of the even share, so when the longest item is under 5 % of that share the block order needs
 // no check; only otherwise (few, long, equal sequences: few items) is the queue simulated as above.
 struct GroupEntry { int32_t a, b, c, cost; };
-template <class Item, class Make>
-std::vector<Item> order_by_groups(std::vector<std::vector<GroupEntry>>& groups, int32_t h, int workers, Make make)
+// The groups longest first (their entries longest first inside), the number of items, and whether the block
+// order needs no check against the queue simulation.
+struct GroupOrder { std::vector<int32_t> order; int64_t n_items = 0; bool settled = true; };
+GroupOrder order_groups(std::vector<std::vector<GroupEntry>>& groups, int32_t h, int workers)
 {
+    GroupOrder go;
     std::vector<int64_t> group_cost(groups.size(), 0);
-    int64_t total = 0, n_items = 0;
+    int64_t total = 0;
     int32_t longest = 0;
     for (size_t g = 0; g < groups.size(); ++g) {
         std::stable_sort(groups[g].begin(), groups[g].end(),
@@ -607,28 +610,34 @@ std::vector<Item> order_by_groups(std::vector<std::vector<GroupEntry>>& groups, 
             total += static_cast<int64_t>(e.cost + kItemOverhead) * h;
             longest = std::max(longest, e.cost);
         }
-        n_items += static_cast<int64_t>(groups[g].size()) * h;
+        go.n_items += static_cast<int64_t>(groups[g].size()) * h;
     }
-    std::vector<int32_t> order(groups.size());
-    for (size_t g = 0; g < groups.size(); ++g) order[g] = static_cast<int32_t>(g);
-    std::sort(order.begin(), order.end(), [&](int32_t x, int32_t y) {
+    go.order.resize(groups.size());
+    for (size_t g = 0; g < groups.size(); ++g) go.order[g] = static_cast<int32_t>(g);
+    std::sort(go.order.begin(), go.order.end(), [&](int32_t x, int32_t y) {
         return group_cost[x] != group_cost[y] ? group_cost[x] > group_cost[y] : x < y;
     });
-    std::vector<Item> items;
-    items.reserve(static_cast<size_t>(n_items));
     const int64_t even = (total + workers - 1) / workers;
-    const bool settled = static_cast<int64_t>(longest + kItemOverhead) * 20 <= even;
+    go.settled = static_cast<int64_t>(longest + kItemOverhead) * 20 <= even;
+    return go;
+}
+template <class Item, class Make>
+std::vector<Item> order_by_groups(std::vector<std::vector<GroupEntry>>& groups, int32_t h, int workers, Make make)
+{
+    const GroupOrder go = order_groups(groups, h, workers);
+    std::vector<Item> items;
+    items.reserve(static_cast<size_t>(go.n_items));
     std::vector<int32_t> block_of, cost;
-    for (int32_t g : order)
+    for (int32_t g : go.order)
         for (int32_t a = 0; a < h; ++a)
             for (const GroupEntry& e : groups[g]) {
                 items.push_back(make(g, a, e));
-                if (!settled) {
+                if (!go.settled) {
                     block_of.push_back(g * h + a);
                     cost.push_back(e.cost);
                 }
             }
-    if (!settled) order_items(items, block_of, cost, workers);
+    if (!go.settled) order_items(items, block_of, cost, workers);
     return items;
 }
 
@@ -693,18 +702,51 @@ void build_fwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& 
         groups, pb.h, plan_workers(2),
         [](int32_t g, int32_t a, const GroupEntry& e) { return FwdItem{g, a, e.a, e.b, e.c, {0, 0, 0}}; });
     const std::vector<PairDev> dev_pairs = device_pairs(pb);
-    // the short kernel's items carry what they need of their pair (its slots start an item from this alone)
-    const std::vector<FwdShortItem> short_items = order_by_groups<FwdShortItem>(
-        groups_short, pb.h, 2 * plan_workers(1), [&](int32_t g, int32_t a, const GroupEntry& e) {
-            const PairDev& d = dev_pairs[g];
-            return FwdShortItem{d.q_tok0 + e.a, e.c, d.k_tok0, d.k_len, e.a + d.off, e.b, a, d.out_row0 + e.a,
-                                d.to_part, {0, 0, 0}};
-        });
     plan.off_pairs = append(blob, dev_pairs);
     plan.off_items = append(blob, items);
     plan.n_items = static_cast<int32_t>(items.size());
-    plan.off_items2 = append(blob, short_items);
-    plan.n_items2 = static_cast<int32_t>(short_items.size());
+    // The short kernel's items carry what they need of their pair (its slots start an item from this alone). A
+    // micro-batch of short sequences has tens of thousands of them and a new one arrives with every step, so in
+    // the common case (many items, none long: the block order is final) they are written straight into the
+    // table, a group's entries once and then one copy per head with the head number set.
+    auto make_short = [&](int32_t g, int32_t a, const GroupEntry& e) {
+        const PairDev& d = dev_pairs[g];
+        FwdShortItem it{};
+        it.q_tok0 = d.q_tok0 + e.a;
+        it.k_tok0 = d.k_tok0;
+        it.k_len = d.k_len;
+        it.off = e.a + d.off;
+        it.out_row0 = d.out_row0 + e.a;
+        it.head = static_cast<uint16_t>(a);
+        it.n_kv = static_cast<uint16_t>(e.b);
+        it.rows = static_cast<uint8_t>(e.c);
+        it.to_part = static_cast<uint8_t>(d.to_part);
+        return it;
+    };
+    const int short_workers = 2 * plan_workers(1);
+    const GroupOrder go = order_groups(groups_short, pb.h, short_workers);
+    if (go.settled) {
+        const size_t off = align_up(blob.size(), 16);
+        blob.resize(off + static_cast<size_t>(go.n_items) * sizeof(FwdShortItem));
+        FwdShortItem* dst = reinterpret_cast<FwdShortItem*>(blob.data() + off);
+        std::vector<FwdShortItem> block;
+        for (int32_t g : go.order) {
+            block.clear();
+            for (const GroupEntry& e : groups_short[g]) block.push_back(make_short(g, 0, e));
+            for (int32_t a = 0; a < pb.h; ++a) {
+                std::memcpy(dst, block.data(), block.size() * sizeof(FwdShortItem));
+                for (size_t i = 0; i < block.size(); ++i) dst[i].head = static_cast<uint16_t>(a);
+                dst += block.size();
+            }
+        }
+        plan.off_items2 = off;
+        plan.n_items2 = static_cast<int32_t>(go.n_items);
+    } else {
+        const std::vector<FwdShortItem> short_items =
+            order_by_groups<FwdShortItem>(groups_short, pb.h, short_workers, make_short);
+        plan.off_items2 = append(blob, short_items);
+        plan.n_items2 = static_cast<int32_t>(short_items.size());
+    }
 }
 
 void build_merge(const Problem& pb, Plan& plan, std::vector<uint8_t>& blob)
@@ -1091,7 +1133,8 @@ void hydra_set_plan_arena_bytes(uint64_t bytes) { g_arena_bytes.store(bytes); }
 
 void hydra_set_plan_prefetch(int32_t on) { g_plan_prefetch.store(on != 0); }
 
-void hydra_set_fwd_short_len(int32_t len) { g_fwd_short_len.store(len > 0 ? len : 0); }
+// (a work item counts its 64-key steps in 16 bits)
+void hydra_set_fwd_short_len(int32_t len) { g_fwd_short_len.store(len > 0 ? std::min(len, 1 << 21) : 0); }
 
 double hydra_plan_build_seconds(int32_t which, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
                                 const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal)

@@ -69,18 +69,20 @@ struct FwdItem {
 
 // Work item of the short-sequence forward kernel: one 128-row q tile of one pair and head, self-contained
 // (a slot of that kernel reads nothing else to start it).
-struct FwdShortItem {
+struct alignas(16) FwdShortItem {
     int32_t q_tok0;    // token index of the tile's first q row
-    int32_t rows;      // q rows of the tile that exist (1..128)
     int32_t k_tok0;    // token index of the pair's first kv row
     int32_t k_len;
     int32_t off;       // key j is visible to row r of the tile iff j <= r + off (causal)
-    int32_t n_kv;      // steps of FWD_SHORT_KEYS keys the tile visits; 0: its rows see no key
-    int32_t head;
     int32_t out_row0;  // output row of the tile's first q row (partial buffers or out / lse)
-    int32_t to_part;   // 1: partial buffers, 0: out / lse
-    int32_t pad[3];
+    uint16_t head;
+    uint16_t n_kv;     // steps of FWD_SHORT_KEYS keys the tile visits; 0: its rows see no key
+    uint8_t rows;      // q rows of the tile that exist (1..128)
+    uint8_t to_part;   // 1: partial buffers, 0: out / lse
+    uint16_t pad;
+    int32_t pad2;
 };
+static_assert(sizeof(FwdShortItem) == 32, "two 16-byte loads per work item");
 
 // Backward work item: one tile of one chunk and head, visiting every pair that shares the chunk.
 struct GroupItem {
