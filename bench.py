@@ -780,8 +780,8 @@ NCU_DRAM_BYTES_PER_LAUNCH = {
     # with the dS hand-off: 1.76 GB of the key-side kernel's writes and of the query-side kernel's reads are dS
     ("bwd_dkv", "packed32k"): (2804310000, ("bwd_kernels.cu",) + _TENSOR_DEPS, "593bb7d3d1d3", "2026-11-25"),
     ("bwd_dq", "packed32k"): (2069075000, ("bwd_kernels.cu",) + _TENSOR_DEPS, "593bb7d3d1d3", "2026-11-25"),
-    ("merge", "short64k_split"): (769407400, ("aux_kernels.cu", "hydra_internal.h"), "bd79e74a8912", "2026-11-25"),
-    ("bwd_prep", "short64k_split"): (1082133344, ("aux_kernels.cu", "hydra_internal.h"), "bd79e74a8912", "2026-11-25"),
+    ("merge", "short64k_split"): (769407400, ("aux_kernels.cu", "hydra_internal.h", "sm100_ptx.cuh"), "bd79e74a8912", "2026-11-25"),
+    ("bwd_prep", "short64k_split"): (1082133344, ("aux_kernels.cu", "hydra_internal.h", "sm100_ptx.cuh"), "bd79e74a8912", "2026-11-25"),
 }
 
 

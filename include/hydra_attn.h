@@ -563,9 +563,10 @@ void hydra_set_plan_prefetch(int32_t on);
  * regime of Section 2.2, where most sequences are short and a tile's chain of dependent steps, not the tensor
  * core, sets the pace), all others to the CTA-pair kernel; if the short pairs carry less than a quarter of a
  * call's work, that call uses the CTA-pair kernel alone. Both compute the same function to the same tolerance
- * (not bit for bit: their summation orders differ). len = 0 switches the short-sequence kernel off; the
- * default is 1536 (where the two kernels take equal time on sequences of one length). Takes effect with the next
- * call.
+ * (not bit for bit: their summation orders differ). len = 0 switches the short-sequence kernel off; a negative
+ * len (the default) lets the library choose: 2048 for heads of 192 with a K / V head per query head, 4608 with
+ * shared K / V heads or heads of 128 (where the kernels were measured to take equal time on sequences of one
+ * length). Takes effect with the next call.
  */
 void hydra_set_fwd_short_len(int32_t len);
 /*

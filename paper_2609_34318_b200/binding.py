@@ -292,7 +292,8 @@ def hydra_set_plan_prefetch(on: bool) -> None:
 
 
 def hydra_set_fwd_short_len(length: int) -> None:
-    """Pairs with q and kv ranges of at most `length` tokens use the short-sequence forward kernel (0: off)."""
+    """Pairs with q and kv ranges of at most `length` tokens use the short-sequence forward kernel (0: off;
+    negative, the default: 2048, or 4608 with shared K / V heads or heads of 128)."""
     _lib.hydra_set_fwd_short_len(int(length))
 
 

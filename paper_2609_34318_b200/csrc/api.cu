@@ -71,6 +71,7 @@ struct Problem {
     int32_t n_seqs = 0, h = 0;
     int64_t T = 0;
     int32_t dqk = D_QK;     // q / k head dimension of the call: 192 or 128 (the value dimension is 128)
+    int32_t kv_group = 1;   // query heads per K / V head (the forward's routing looks at it)
     // Local layouts (a rank of a ring holds only its own q chunks and the visiting kv chunks): where the
     // chunks of the sequences sit in the q-side tensors (q, out, lse, dout, dq) and in the kv-side tensors
     // (k, v, dk, dv). Empty tables = the packed layout, row = cu[seq] + position, Tq = Tk = T.
@@ -418,8 +419,18 @@ void arena_note_use(const Plan& plan, int device, cudaStream_t stream)
 }
 
 // Pairs whose q range and kv range are both at most this long go to the short-sequence forward kernel
-// (0: none do). See build_fwd.
-std::atomic<int32_t> g_fwd_short_len{1536};
+// (0: none do; negative: chosen by the library from the head layout). See build_fwd.
+std::atomic<int32_t> g_fwd_short_len{-1};
+// Where the two forward kernels take equal time on sequences of one length (32K tokens, 16 heads, two GPUs of
+// the pool): with a K / V head per query head at d_qk = 192 between 2048 and 3072 tokens; with shared K / V
+// heads, or at d_qk = 128 (where a slot of the short-sequence kernel has room for a second V stage), between
+// 4096 and 8192, and the 32K packed workload (sequences up to 4441 tokens) runs 11-15 % faster on it.
+int32_t fwd_short_len_for(const Problem& pb)
+{
+    const int32_t set = g_fwd_short_len.load();
+    if (set >= 0) return set;
+    return (pb.dqk == D_QK && pb.kv_group == 1) ? 2048 : 4608;
+}
 static_assert(FWD_SHORT_KEYS == SUB, "the short forward kernel reads K through the 64-row map of the CTA-pair kernel");
 
 std::vector<uint8_t> make_key(int kind, int device, const Problem& pb, int causal)
@@ -430,7 +441,7 @@ std::vector<uint8_t> make_key(int kind, int device, const Problem& pb, int causa
         key.insert(key.end(), b, b + n);
     };
     // the forward's tables depend on which pairs go to the short-sequence kernel
-    const int32_t head[6] = {kind, device, pb.h, causal, pb.n_seqs, kind == HYDRA_WS_FWD ? g_fwd_short_len.load() : 0};
+    const int32_t head[6] = {kind, device, pb.h, causal, pb.n_seqs, kind == HYDRA_WS_FWD ? fwd_short_len_for(pb) : 0};
     put(head, sizeof head);
     put(pb.cu.data(), pb.cu.size() * sizeof(int32_t));
     put(pb.pairs.data(), pb.pairs.size() * sizeof(hydra_pair_t));
@@ -656,7 +667,7 @@ void build_fwd(const Problem& pb, int causal, Plan& plan, std::vector<uint8_t>& 
     // bound by the length of a tile's chain of steps, and more, shorter chains per SM win; on long pairs its
     // operand sharing and its 256-row tiles do. A second launch has a price of its own (its start and its
     // tail), so the short kernel is used only if the short pairs carry at least a quarter of the call's work.
-    const int32_t short_len = g_fwd_short_len.load();
+    const int32_t short_len = fwd_short_len_for(pb);
     std::vector<uint8_t> is_short(pb.pairs.size(), 0);
     {
         double work_short = 0, work_all = 0;
@@ -765,6 +776,7 @@ void build_merge(const Problem& pb, Plan& plan, std::vector<uint8_t>& blob)
             g.rows = p.q_len;
             g.list_off = static_cast<int32_t>(lists.size());
             g.n_parts = static_cast<int32_t>(j - i);
+            plan.n_items2 = std::max(plan.n_items2, g.n_parts);     // (of a merge plan: the most partials of a chunk)
             for (size_t t = i; t < j; ++t) lists.push_back(pb.pairs[t].part_row);
             for (int32_t r = 0; r < g.rows; r += MERGE_ROWS)
                 items.push_back(MergeItem{static_cast<int32_t>(groups.size()), r});
@@ -1134,7 +1146,7 @@ void hydra_set_plan_arena_bytes(uint64_t bytes) { g_arena_bytes.store(bytes); }
 void hydra_set_plan_prefetch(int32_t on) { g_plan_prefetch.store(on != 0); }
 
 // (a work item counts its 64-key steps in 16 bits)
-void hydra_set_fwd_short_len(int32_t len) { g_fwd_short_len.store(len > 0 ? std::min(len, 1 << 21) : 0); }
+void hydra_set_fwd_short_len(int32_t len) { g_fwd_short_len.store(std::min(len, 1 << 21)); }
 
 double hydra_plan_build_seconds(int32_t which, const int32_t* cu, int32_t n_seqs, int32_t n_heads,
                                 const hydra_pair_t* pairs, int32_t n_pairs, int32_t causal)
@@ -1365,6 +1377,7 @@ int32_t fwd_core(Problem& pb, const void* q, const void* k, const void* v, int32
     const int32_t n_heads = pb.h;
     const KernelSet* ks = kernel_set(pb.dqk, D_V);
     if (n_kv_heads < 1 || n_heads % n_kv_heads) return HYDRA_ERR_INVALID_ARG;
+    pb.kv_group = n_heads / n_kv_heads;
     if (!(softmax_scale > 0.f) || !std::isfinite(softmax_scale)) return HYDRA_ERR_INVALID_ARG;
     if (!workspace || !aligned16(workspace)) return HYDRA_ERR_INVALID_ARG;
     if (workspace_bytes < kStatusBytes) return HYDRA_ERR_WORKSPACE_TOO_SMALL;
@@ -1489,6 +1502,7 @@ int32_t merge_core(const Problem& pb, const void* o_part, const float* lse_part,
     mp.o_part = o_part; mp.lse_part = lse_part; mp.out = out; mp.lse = lse;
     mp.T = pb.Tq; mp.part_rows = part_rows; mp.h = n_heads;
     mp.accumulate = accumulate;
+    mp.max_parts = plan->n_items2;
     if (launch_merge_counted(mp, stream) != cudaSuccess) return HYDRA_ERR_CUDA;
     return HYDRA_OK;
 }

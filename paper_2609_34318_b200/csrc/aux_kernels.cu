@@ -11,6 +11,7 @@
 #include <utility>
 
 #include "hydra_internal.h"
+#include "sm100_ptx.cuh"
 
 namespace hydra {
 
@@ -60,8 +61,19 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v)
 
 // One block = MERGE_ROWS consecutive rows of one chunk, all heads.  For (row, head):
 //   M = max_p LSE_p;  Z = sum_p exp(LSE_p - M);  LSE = M + ln Z;  O = sum_p (exp(LSE_p - M) / Z) O_p
-template <bool kAccumulate>
-__global__ void __launch_bounds__(kThreads, 6)
+// An earlier form (two partials requested up front, the rest one round trip each, the running sums corrected
+// per partial) kept the issue slots 71-73 % busy at 4.4-5.0 TB/s, so the inner loop is kept short: the partials of a (row, head) are taken four at a time,
+// all four loads and their LSEs requested before anything is computed (most chunks have two to four partials:
+// one round trip); the weights exp(LSE_p - M) are formed once per group of four, so the running sums are
+// corrected at most once per group instead of once per partial and the final 1 / Z is folded into one
+// multiply per element; the products are packed two-element FMAs; (row, head) advance without a division.
+// kBatch = partials requested together: 4 (four blocks per SM, 64 registers) when some chunk has more than two
+// partials, else 2 (six blocks per SM: with two partials per chunk, as in a sequence cut in two, occupancy is
+// worth more than loads in flight per thread). Measured, L2 flushed: 256K ring workload 4.93 -> 5.72 TB/s (89 % of
+// the measured copy bandwidth), many-short split workload 4.74 -> 4.97 TB/s; with four at a time for every chunk
+// the latter fell to 4.1, with five or six blocks per SM for kBatch = 4 (spills) the former to 5.69 / 5.26.
+template <bool kAccumulate, int kBatch>
+__global__ void __launch_bounds__(kThreads, kBatch == 2 ? 6 : 4)
 hydra_lse_merge_kernel(const MergeParams p)
 {
     const MergeItem item = p.items[blockIdx.x];
@@ -69,78 +81,97 @@ hydra_lse_merge_kernel(const MergeParams p)
     const int32_t* part_row = p.lists + g.list_off;
     const int rows = min(MERGE_ROWS, g.rows - item.row0);
     const int lane = threadIdx.x & (kLanesPerUnit - 1);
-    const int unit0 = threadIdx.x / kLanesPerUnit;
     const uint4* o_part = static_cast<const uint4*>(p.o_part);
     uint4* out = static_cast<uint4*>(p.out);
     constexpr int kVecPerRow = D_V / 8;           // uint4 per (row, head)
+    constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+    const int n_units = rows * p.h;
+    // (row, head) of this lane group's first unit; later units are kUnitsPerPass further on
+    int u = threadIdx.x / kLanesPerUnit;
+    int r = u / p.h, a = u - r * p.h;
+    const int step_r = kUnitsPerPass / p.h, step_a = kUnitsPerPass - step_r * p.h;
 
-    for (int u = unit0; u < rows * p.h; u += kUnitsPerPass) {
-        const int r = item.row0 + u / p.h, a = u % p.h;
-        const float* lse_row = p.lse_part + static_cast<int64_t>(a) * p.part_rows + r;
-        // The first two partials (every merged chunk has at least two) are requested before anything
-        // else, together with their LSEs: one round trip to memory instead of two (all LSEs for the
-        // maximum, then O) for most chunks. The running maximum is corrected on the fly for the
-        // partials that follow.
-        const int64_t prow0 = static_cast<int64_t>(part_row[0]) + r;
-        const int64_t prow1 = static_cast<int64_t>(part_row[g.n_parts > 1 ? 1 : 0]) + r;
-        const uint4 v0 = ld_stream(o_part + (prow0 * p.h + a) * kVecPerRow + lane);
-        const uint4 v1 = ld_stream(o_part + (prow1 * p.h + a) * kVecPerRow + lane);
-        const float l0 = __ldg(lse_row + part_row[0]);
-        const float l1 = g.n_parts > 1 ? __ldg(lse_row + part_row[1]) : neg_inf();
-        // streaming form (one ring step at a time): what out / lse hold so far is one more input
-        const int64_t tok = static_cast<int64_t>(g.out_tok0) + r;
-        uint4 v_cur = make_uint4(0u, 0u, 0u, 0u);
-        float l_cur = neg_inf();
-        if (kAccumulate) {
-            v_cur = out[(tok * p.h + a) * kVecPerRow + lane];
-            l_cur = p.lse[static_cast<int64_t>(a) * p.T + tok];
-        }
-        float m = neg_inf();
+    for (; u < n_units; u += kUnitsPerPass) {
+        const int row = item.row0 + r;
+        const float* lse_row = p.lse_part + static_cast<int64_t>(a) * p.part_rows + row;
+        const uint4* o_row = o_part + (static_cast<int64_t>(row) * p.h + a) * kVecPerRow + lane;
+        const int64_t part_stride = static_cast<int64_t>(p.h) * kVecPerRow;     // uint4 per partial row
+        const int64_t tok = static_cast<int64_t>(g.out_tok0) + row;
+        uint4* out_v = out + (tok * p.h + a) * kVecPerRow + lane;
+        float* lse_out = p.lse + static_cast<int64_t>(a) * p.T + tok;
+        // everything relative to m (in log2 units): acc = sum_p 2^(l_p - m) O_p, z = sum_p 2^(l_p - m)
+        float m = neg_inf(), z = 0.f;
         float acc[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-        float z = 0.f;
-        auto add = [&](const uint4& v, float l) {          // online update: acc, z are relative to m
-            if (l == neg_inf()) return;                      // a partial that saw no key
-            if (l > m) {
-                const float c = __expf(m - l);               // 0 when m = -inf
+        // streaming form (one ring step at a time): what out / lse hold so far is one more input
+        uint4 v_cur = make_uint4(0u, 0u, 0u, 0u);
+        float l_cur = neg_inf();
+        if (kAccumulate) {
+            l_cur = *lse_out * kLog2e;
+            if (l_cur != neg_inf()) v_cur = *out_v;
+        }
+        for (int q0 = 0; q0 < g.n_parts; q0 += kBatch) {
+            uint4 v[kBatch];
+            float l[kBatch];
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                const bool have = q0 + i < g.n_parts;
+                const int32_t pr = part_row[have ? q0 + i : q0];
+                l[i] = have ? __ldg(lse_row + pr) * kLog2e : neg_inf();
+                v[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (have) v[i] = ld_stream(o_row + pr * part_stride);
+            }
+            // a partial that saw no key (LSE = -inf) counts for nothing, whatever its O rows hold
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i)
+                if (l[i] == neg_inf()) v[i] = make_uint4(0u, 0u, 0u, 0u);
+            float m_new = fmaxf(l[0], l[1]);
+            if (kBatch == 4) m_new = fmaxf(m_new, fmaxf(l[kBatch - 2], l[kBatch - 1]));
+            if (kAccumulate && q0 == 0) m_new = fmaxf(m_new, l_cur);
+            if (m_new > m) {                             // (never for m_new = -inf)
+                const float c = ex2_approx(m - m_new);   // 0 when m = -inf
                 z *= c;
 #pragma unroll
                 for (int e = 0; e < 8; ++e) acc[e] *= c;
-                m = l;
+                m = m_new;
             }
-            const float w = __expf(l - m);
-            z += w;
-            float f[8];
-            unpack8(v, f);
+            if (m == neg_inf()) continue;                // nothing visible so far: every weight is 0
+            if (kAccumulate && q0 == 0) {
+                const float w = ex2_approx(l_cur - m);
+                z += w;
+                float f[8];
+                unpack8(v_cur, f);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = fmaf(w, f[e], acc[e]);
-        };
-        if (kAccumulate) add(v_cur, l_cur);
-        add(v0, l0);
-        add(v1, l1);
-        for (int q = 2; q < g.n_parts; ++q) {
-            const int64_t prow = static_cast<int64_t>(part_row[q]) + r;
-            add(ld_stream(o_part + (prow * p.h + a) * kVecPerRow + lane), __ldg(lse_row + part_row[q]));
-        }
-        if (z > 0.f) {
-            const float inv = 1.f / z;
+                for (int e = 0; e < 8; e += 2) ffma2(acc[e], acc[e + 1], f[e], f[e + 1], w, w, acc[e], acc[e + 1]);
+            }
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] *= inv;
-        } else {
-            m = neg_inf();
+            for (int i = 0; i < kBatch; ++i) {
+                if (q0 + i >= g.n_parts) break;          // (the same for every thread of the block)
+                const float w = ex2_approx(l[i] - m);    // 0 for a partial that saw no key
+                z += w;
+                float f[8];
+                unpack8(v[i], f);
+#pragma unroll
+                for (int e = 0; e < 8; e += 2) ffma2(acc[e], acc[e + 1], f[e], f[e + 1], w, w, acc[e], acc[e + 1]);
+            }
         }
-        out[(tok * p.h + a) * kVecPerRow + lane] = pack8(acc);
-        if (lane == 0)
-            p.lse[static_cast<int64_t>(a) * p.T + tok] = (m == neg_inf()) ? neg_inf() : m + __logf(z);
+        const float inv = z > 0.f ? 1.f / z : 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] *= inv;
+        *out_v = pack8(acc);
+        if (lane == 0) *lse_out = z > 0.f ? (m + __log2f(z)) * kLn2 : neg_inf();
+        a += step_a;
+        r += step_r;
+        if (a >= p.h) { a -= p.h; ++r; }
     }
 }
 // (Measured and not kept, all on the 256K ring workload and the many-short split workload, L2 flushed, against
-// this kernel's 4.4-5.0 TB/s depending on the GPU of the pool: persistent blocks with the tables in shared
+// the earlier form's 4.4-5.0 TB/s depending on the GPU of the pool: persistent blocks with the tables in shared
 // memory and four partial loads per lane group in flight, 4.3-4.5 TB/s; two (row, head) vectors per lane group
 // at two blocks per SM, 3.5 TB/s; partials staged through shared memory by bulk asynchronous copies, three
-// 64 KB stages and sixteen consumer warps per SM, 3.1-3.8 TB/s. What carries this kernel is its occupancy:
-// six short-lived blocks per SM in different phases keep more loads in flight than any of those.)
+// 64 KB stages and sixteen consumer warps per SM, 3.1-3.8 TB/s. Short-lived blocks in different phases keep
+// more loads in flight than any of those.)
 
 // D[a, t] = sum_e dO[t, a, e] * O[t, a, e]
 __global__ void __launch_bounds__(kThreads)
@@ -257,8 +288,14 @@ cudaError_t launch_ulysses(bool pack, const void* src, void* dst, int64_t n_toke
 cudaError_t launch_merge(const MergeParams& p, cudaStream_t stream)
 {
     if (p.n_items == 0) return cudaSuccess;
-    if (p.accumulate) hydra_lse_merge_kernel<true><<<p.n_items, kThreads, 0, stream>>>(p);
-    else hydra_lse_merge_kernel<false><<<p.n_items, kThreads, 0, stream>>>(p);
+    const bool wide = p.max_parts > 2;
+    if (p.accumulate) {
+        if (wide) hydra_lse_merge_kernel<true, 4><<<p.n_items, kThreads, 0, stream>>>(p);
+        else hydra_lse_merge_kernel<true, 2><<<p.n_items, kThreads, 0, stream>>>(p);
+    } else {
+        if (wide) hydra_lse_merge_kernel<false, 4><<<p.n_items, kThreads, 0, stream>>>(p);
+        else hydra_lse_merge_kernel<false, 2><<<p.n_items, kThreads, 0, stream>>>(p);
+    }
     return cudaGetLastError();
 }
 
@@ -347,6 +384,7 @@ extern "C" int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_
     static MergeItem items[kNoAllocMaxItems];
     static std::pair<int64_t, int64_t> part_iv[kNoAllocMaxParts], out_iv[kNoAllocMaxGroups];   // [first, end) rows
     int n_groups = 0, n_parts = 0, n_items = 0;
+    int32_t max_parts = 0;
     for (int i = 0; i < n_pairs;) {
         int j = i;
         while (j < n_pairs && pairs[j].group == pairs[i].group) ++j;
@@ -376,6 +414,7 @@ extern "C" int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_
                 items[n_items++] = MergeItem{n_groups, r};
             }
             out_iv[n_groups] = {g.out_tok0, int64_t{g.out_tok0} + g.rows};
+            max_parts = std::max(max_parts, g.n_parts);
             groups[n_groups++] = g;
         } else {
             for (int t = i; t < j; ++t)
@@ -418,6 +457,7 @@ extern "C" int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_
     mp.lists = reinterpret_cast<const int32_t*>(tables + kNoAllocGroupsBytes);
     mp.items = reinterpret_cast<const MergeItem*>(tables + kNoAllocGroupsBytes + kNoAllocPartsBytes);
     mp.n_items = n_items;
+    mp.max_parts = max_parts;
     mp.o_part = o_part; mp.lse_part = lse_part; mp.out = out; mp.lse = lse;
     mp.T = cu[n_seqs]; mp.part_rows = part_rows; mp.h = n_heads;
     // counted and timed like every other merge launch (hydra_launch_count, hydra_profile_collect)

@@ -182,6 +182,7 @@ struct MergeParams {
     int64_t T; int64_t part_rows;
     int32_t h;
     int32_t accumulate;         // 1: the current (out, lse) rows are one more input of their merge
+    int32_t max_parts;          // most partials any chunk has (chooses how many are requested together)
 };
 
 // The tensor-core kernels exist once per supported q / k head dimension (the kernel files are compiled

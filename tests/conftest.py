@@ -27,7 +27,7 @@ def pytest_collection_modifyitems(config, items):
             item.add_marker(skip)
 
 
-FWD_SHORT_LEN_DEFAULT = 1536
+FWD_SHORT_LEN_DEFAULT = -1        # the library chooses by head layout
 
 
 @pytest.fixture(params=["cta_pair_forward", "short_sequence_forward"])

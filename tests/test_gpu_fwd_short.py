@@ -45,7 +45,7 @@ def default_routing():
     [1, 1, 1, 2],                 # work items of a single row and a single key
     [63, 65, 64],                 # one key more and one key less than a step
     [129, 257, 64, 500, 127],     # one row more than a tile, one more than two
-    [1536],                       # the longest sequence the default routing sends here: 12 tiles, up to 24 steps
+    [2048],                       # the longest sequence the default routing sends here: 16 tiles, up to 32 steps
     [200] * 40,                   # more work items than the two slots of every SM hold at once
 ])
 def test_short_sequences_against_the_oracle(lengths):
@@ -67,7 +67,7 @@ def test_random_length_mixes_and_both_kernels_agree():
         x = rand_inputs(100 + trial, int(cu[-1]), h)
         ref = run_oracle(x, cu, backward=False)
         res = {}
-        for name, limit in (("short", FWD_SHORT_LEN_DEFAULT), ("pair", 0)):
+        for name, limit in (("short", 1 << 20), ("pair", 0)):
             P.hydra_set_fwd_short_len(limit)
             res[name] = run_gpu(x, cu, h, backward=False)
             check(res[name], ref, names=("out", "lse"), label=f"trial {trial} {name} ")
@@ -82,7 +82,7 @@ def test_one_call_uses_both_kernels_when_short_pairs_carry_enough_work():
     import paper_2609_34318_b200 as P
     from paper_2609_34318_b200.runner import AttnStep, bits_to_tensor
     h = 2
-    for lengths, launches in (([2000] + [300] * 30, 2), ([2000, 300, 300], 1), ([300] * 8, 1)):
+    for lengths, launches in (([3000] + [300] * 60, 2), ([3000, 300, 300], 1), ([300] * 8, 1)):
         cu = hw.cu_seqlens(lengths)
         x = rand_inputs(len(lengths), int(cu[-1]), h)
         step = AttnStep(cu, h)
