@@ -125,3 +125,31 @@ def row_rel_err(got, ref):
     nr = np.linalg.norm(r, axis=1)
     ok = nr > 0
     return float((np.linalg.norm(g - r, axis=1)[ok] / nr[ok]).max()) if ok.any() else 0.0
+
+
+def oracle_merge_of_partials(cu, pairs, o_part, lse_part, T, h, out_cur=None, lse_cur=None):
+    """fp64 merge (the oracle's) of partial buffers as they stand on the GPU, per merged q chunk; NaN elsewhere.
+    With out_cur / lse_cur (numpy, [T,h,dv] / [h,T]) the current rows are one more input (streaming form)."""
+    o_np = o_part.float().cpu().numpy().astype(np.float64)
+    l_np = lse_part.cpu().numpy().astype(np.float64)
+    out = np.full((T, h, hw.D_V), np.nan)
+    lse = np.full((h, T), np.nan)
+    i = 0
+    while i < len(pairs):
+        j = i
+        while j < len(pairs) and pairs[j]["group"] == pairs[i]["group"]:
+            j += 1
+        p = pairs[i]
+        if p["part_row"] >= 0 and p["q_len"] > 0:
+            n = int(p["q_len"])
+            os_ = [o_np[int(pairs[t]["part_row"]):int(pairs[t]["part_row"]) + n] for t in range(i, j)]
+            ls_ = [l_np[:, int(pairs[t]["part_row"]):int(pairs[t]["part_row"]) + n] for t in range(i, j)]
+            t0 = int(cu[p["seq"]]) + int(p["q_start"])
+            if out_cur is not None:
+                os_ = [out_cur[t0:t0 + n]] + os_
+                ls_ = [lse_cur[:, t0:t0 + n]] + ls_
+            mo, ml = oracle.lse_merge(os_, ls_)
+            out[t0:t0 + n] = mo
+            lse[:, t0:t0 + n] = ml
+        i = j
+    return out, lse

@@ -16,7 +16,7 @@ import torch
 
 import hydra_workloads as hw
 import oracle
-from gpu_util import TOL_LSE, TOL_REL
+from gpu_util import TOL_LSE, TOL_REL, oracle_merge_of_partials
 
 pytestmark = pytest.mark.gpu
 
@@ -36,30 +36,6 @@ def _partials(lengths, h, cp_r, seed):
                      part_rows, step.workspace)
     torch.cuda.synchronize()
     return P, cu, pairs, part_rows, step
-
-
-def _oracle_merge(cu, pairs, o_part, lse_part, T, h):
-    """fp64 merge (the oracle's) of the GPU's own partials, per merged q chunk; NaN elsewhere."""
-    o_np = o_part.float().cpu().numpy().astype(np.float64)
-    l_np = lse_part.cpu().numpy().astype(np.float64)
-    out = np.full((T, h, hw.D_V), np.nan)
-    lse = np.full((h, T), np.nan)
-    i = 0
-    while i < len(pairs):
-        j = i
-        while j < len(pairs) and pairs[j]["group"] == pairs[i]["group"]:
-            j += 1
-        p = pairs[i]
-        if p["part_row"] >= 0 and p["q_len"] > 0:
-            n = int(p["q_len"])
-            os_ = [o_np[int(pairs[t]["part_row"]):int(pairs[t]["part_row"]) + n] for t in range(i, j)]
-            ls_ = [l_np[:, int(pairs[t]["part_row"]):int(pairs[t]["part_row"]) + n] for t in range(i, j)]
-            mo, ml = oracle.lse_merge(os_, ls_)
-            t0 = int(cu[p["seq"]]) + int(p["q_start"])
-            out[t0:t0 + n] = mo
-            lse[:, t0:t0 + n] = ml
-        i = j
-    return out, lse
 
 
 def _merge_both_ways(lengths, h, cp_r, seed, memory_must_stay_flat):
@@ -92,7 +68,7 @@ def _merge_both_ways(lengths, h, cp_r, seed, memory_must_stay_flat):
     assert np.abs(a - b).max() <= TOL_REL * np.abs(a).max()
     assert np.abs(la - lb).max() <= TOL_LSE
     # against the oracle's merge of the same partials, element by element
-    ref_o, ref_l = _oracle_merge(cu, pairs, step.o_part, step.lse_part, T, h)
+    ref_o, ref_l = oracle_merge_of_partials(cu, pairs, step.o_part, step.lse_part, T, h)
     rows = np.nonzero(merged)[0]
     got_o = out_b.float().cpu().numpy().astype(np.float64)[rows]
     got_l = lse_b.cpu().numpy().astype(np.float64)[:, rows]
