@@ -540,30 +540,23 @@ HYDRA_K(hydra_bwd_dq_kernel)(const __grid_constant__ CUtensorMap map_q, const __
                 const int cmax = jmax - ti.t * TILE - g * 64;      // columns 0..cmax of this half are visible
                 uint32_t ds[32];
                 float lse2_h = lse2_t;
-                // interior tiles (every column visible to every row of the warp) skip the masking
-                const bool masked = __any_sync(0xffffffffu, cmax < 63);
+                // Interior tiles (every column visible to every row of the warp) skip the masking; elsewhere the
+                // masked scores become -inf, whose probability exp2(-inf) is 0 by itself: one arithmetic path.
+                if (__any_sync(0xffffffffu, cmax < 63)) {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c)
+                        if (c > cmax) s[c] = __float_as_uint(neg_inf());
+                }
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
-                    if (masked) {
 #pragma unroll
-                        for (int c = half * 32; c < half * 32 + 32; c += 2) {
-                            float p0 = ex2_approx(fmaf(__uint_as_float(s[c]), p.scale_log2, -lse2_h));
-                            float p1 = ex2_approx(fmaf(__uint_as_float(s[c + 1]), p.scale_log2, -lse2_h));
-                            if (c > cmax) p0 = 0.f;
-                            if (c + 1 > cmax) p1 = 0.f;
-                            ds[c >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c]) - dsum),
-                                                     p1 * (__uint_as_float(dp[c + 1]) - dsum));
-                        }
-                    } else {
-#pragma unroll
-                        for (int c = half * 32; c < half * 32 + 32; c += 2) {
-                            float x0, x1, d0, d1;
-                            ffma2(x0, x1, __uint_as_float(s[c]), __uint_as_float(s[c + 1]), p.scale_log2, p.scale_log2,
-                                  -lse2_h, -lse2_h);
-                            fadd2(d0, d1, __uint_as_float(dp[c]), __uint_as_float(dp[c + 1]), -dsum, -dsum);
-                            fmul2(d0, d1, d0, d1, ex2_approx(x0), ex2_approx(x1));
-                            ds[c >> 1] = pack_bf16x2(d0, d1);
-                        }
+                    for (int c = half * 32; c < half * 32 + 32; c += 2) {
+                        float x0, x1, d0, d1;
+                        ffma2(x0, x1, __uint_as_float(s[c]), __uint_as_float(s[c + 1]), p.scale_log2, p.scale_log2,
+                              -lse2_h, -lse2_h);
+                        fadd2(d0, d1, __uint_as_float(dp[c]), __uint_as_float(dp[c + 1]), -dsum, -dsum);
+                        fmul2(d0, d1, d0, d1, ex2_approx(x0), ex2_approx(x1));
+                        ds[c >> 1] = pack_bf16x2(d0, d1);
                     }
                     if (half == 0 && c_ds > 0) {           // the previous dQ update has read dS
                         ok = wait(B_DSFREE, c_ds - 1u);
@@ -950,39 +943,27 @@ HYDRA_K(hydra_bwd_dkv_kernel)(const __grid_constant__ CUtensorMap map_q, const _
                 const float4* nlse4 = reinterpret_cast<const float4*>(&s_lse2[st][g * 32]);
                 const float4* ndsum4 = reinterpret_cast<const float4*>(&s_dsum[st][g * 32]);
                 uint32_t pk[16], ds[16];
-                // interior sub-tiles (every q row visible from every kv row of the warp) skip the masking
+                // Interior sub-tiles (every q row visible from every kv row of the warp) skip the masking; elsewhere
+                // the masked scores become -inf, whose probability exp2(-inf) is 0 by itself: one arithmetic path.
                 if (__any_sync(0xffffffffu, c_lo > 0 || c_hi < 32)) {
 #pragma unroll
-                    for (int c = 0; c < 32; c += 4) {
-                        const float4 nl = nlse4[c >> 2], nd = ndsum4[c >> 2];
-                        const float nlv[4] = {nl.x, nl.y, nl.z, nl.w}, ndv[4] = {nd.x, nd.y, nd.z, nd.w};
+                    for (int c = 0; c < 32; ++c)
+                        if (c < c_lo || c >= c_hi) s[c] = __float_as_uint(neg_inf());
+                }
 #pragma unroll
-                        for (int e = 0; e < 4; e += 2) {
-                            float p0 = ex2_approx(fmaf(__uint_as_float(s[c + e]), p.scale_log2, nlv[e]));
-                            float p1 = ex2_approx(fmaf(__uint_as_float(s[c + e + 1]), p.scale_log2, nlv[e + 1]));
-                            if (c + e < c_lo || c + e >= c_hi) p0 = 0.f;
-                            if (c + e + 1 < c_lo || c + e + 1 >= c_hi) p1 = 0.f;
-                            pk[(c + e) >> 1] = pack_bf16x2(p0, p1);
-                            ds[(c + e) >> 1] = pack_bf16x2(p0 * (__uint_as_float(dp[c + e]) + ndv[e]),
-                                                           p1 * (__uint_as_float(dp[c + e + 1]) + ndv[e + 1]));
-                        }
-                    }
-                } else {
+                for (int c = 0; c < 32; c += 4) {
+                    const float4 nl = nlse4[c >> 2], nd = ndsum4[c >> 2];
+                    const float nlv[4] = {nl.x, nl.y, nl.z, nl.w}, ndv[4] = {nd.x, nd.y, nd.z, nd.w};
 #pragma unroll
-                    for (int c = 0; c < 32; c += 4) {
-                        const float4 nl = nlse4[c >> 2], nd = ndsum4[c >> 2];
-                        const float nlv[4] = {nl.x, nl.y, nl.z, nl.w}, ndv[4] = {nd.x, nd.y, nd.z, nd.w};
-#pragma unroll
-                        for (int e = 0; e < 4; e += 2) {
-                            float x0, x1, d0, d1;
-                            ffma2(x0, x1, __uint_as_float(s[c + e]), __uint_as_float(s[c + e + 1]), p.scale_log2,
-                                  p.scale_log2, nlv[e], nlv[e + 1]);
-                            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
-                            fadd2(d0, d1, __uint_as_float(dp[c + e]), __uint_as_float(dp[c + e + 1]), ndv[e], ndv[e + 1]);
-                            fmul2(d0, d1, d0, d1, p0, p1);
-                            pk[(c + e) >> 1] = pack_bf16x2(p0, p1);
-                            ds[(c + e) >> 1] = pack_bf16x2(d0, d1);
-                        }
+                    for (int e = 0; e < 4; e += 2) {
+                        float x0, x1, d0, d1;
+                        ffma2(x0, x1, __uint_as_float(s[c + e]), __uint_as_float(s[c + e + 1]), p.scale_log2,
+                              p.scale_log2, nlv[e], nlv[e + 1]);
+                        const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                        fadd2(d0, d1, __uint_as_float(dp[c + e]), __uint_as_float(dp[c + e + 1]), ndv[e], ndv[e + 1]);
+                        fmul2(d0, d1, d0, d1, p0, p1);
+                        pk[(c + e) >> 1] = pack_bf16x2(p0, p1);
+                        ds[(c + e) >> 1] = pack_bf16x2(d0, d1);
                     }
                 }
                 if (c_pds > 0) {                       // the previous dV / dK updates have read P and dS
