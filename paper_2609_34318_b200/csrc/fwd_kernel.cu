@@ -453,6 +453,7 @@ HYDRA_K(hydra_fwd_kernel)(const __grid_constant__ CUtensorMap map_q, const __gri
             if (!ok) break;
             tc_fence_after_sync();
             const float inv_l = (l_run > 0.f) ? 1.f / l_run : 0.f;
+            const bool wide = (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;
 #pragma unroll
             for (int c0 = 0; c0 < D_V; c0 += 32) {
                 uint32_t o[32];
@@ -463,14 +464,21 @@ HYDRA_K(hydra_fwd_kernel)(const __grid_constant__ CUtensorMap map_q, const __gri
                     mbar_arrive_warp_leader(bar(B_OFREE + t));
                 }
                 if (row_valid) {
+                    // 32 bytes per store where the address allows it (the interface asks for 16): a thread's row
+                    // is 4 KB from its neighbour's, every store of a warp touches 32 lines, whole sectors halve
+                    // the number of such instructions
 #pragma unroll
-                    for (int e = 0; e < 32; e += 8) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(o[e + 0]) * inv_l, __uint_as_float(o[e + 1]) * inv_l);
-                        w.y = pack_bf16x2(__uint_as_float(o[e + 2]) * inv_l, __uint_as_float(o[e + 3]) * inv_l);
-                        w.z = pack_bf16x2(__uint_as_float(o[e + 4]) * inv_l, __uint_as_float(o[e + 5]) * inv_l);
-                        w.w = pack_bf16x2(__uint_as_float(o[e + 6]) * inv_l, __uint_as_float(o[e + 7]) * inv_l);
-                        dst[(c0 + e) >> 3] = w;
+                    for (int e = 0; e < 32; e += 16) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            w[i] = pack_bf16x2(__uint_as_float(o[e + 2 * i]) * inv_l, __uint_as_float(o[e + 2 * i + 1]) * inv_l);
+                        if (wide) {
+                            st_global_v8(dst + ((c0 + e) >> 3), w);
+                        } else {
+                            dst[(c0 + e) >> 3] = make_uint4(w[0], w[1], w[2], w[3]);
+                            dst[((c0 + e) >> 3) + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+                        }
                     }
                 }
             }

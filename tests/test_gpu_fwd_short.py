@@ -112,10 +112,12 @@ def test_non_causal_short_pairs():
     check(got, run_oracle(x, cu, causal=False), label="non-causal short ")
 
 
-def test_output_that_is_16_but_not_32_byte_aligned():
-    """The interface asks for 16-byte alignment; the short-sequence kernel stores 32 bytes at a time only
-    when the address allows it."""
+@pytest.mark.parametrize("short_len", [FWD_SHORT_LEN_DEFAULT, 0])
+def test_output_that_is_16_but_not_32_byte_aligned(short_len):
+    """The interface asks for 16-byte alignment; both forward kernels store 32 bytes at a time only when the
+    address allows it."""
     import paper_2609_34318_b200 as P
+    P.hydra_set_fwd_short_len(short_len)
     from paper_2609_34318_b200.runner import AttnStep, bits_to_tensor
     h = 2
     lengths = [70, 300]
