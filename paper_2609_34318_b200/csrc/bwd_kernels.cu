@@ -53,17 +53,25 @@ constexpr int kSched = 4;                  // depth of the in-CTA ring of work-i
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
 __device__ __forceinline__ float pos_inf() { return __int_as_float(0x7f800000); }
 
+// n (a multiple of 16) values of a thread's own row. Rows of neighbouring threads are kilobytes apart, so every
+// store of the warp touches 32 lines: 32-byte stores (one sector per thread) where the address allows it (the
+// interface asks for 16-byte alignment only) halve the number of such instructions.
 __device__ __forceinline__ void store_row_bf16(__nv_bfloat16* dst, const uint32_t* v, int n, float mul)
 {
     uint4* d4 = reinterpret_cast<uint4*>(dst);
+    const bool wide = (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;
 #pragma unroll
-    for (int e = 0; e < n; e += 8) {
-        uint4 w;
-        w.x = pack_bf16x2(__uint_as_float(v[e + 0]) * mul, __uint_as_float(v[e + 1]) * mul);
-        w.y = pack_bf16x2(__uint_as_float(v[e + 2]) * mul, __uint_as_float(v[e + 3]) * mul);
-        w.z = pack_bf16x2(__uint_as_float(v[e + 4]) * mul, __uint_as_float(v[e + 5]) * mul);
-        w.w = pack_bf16x2(__uint_as_float(v[e + 6]) * mul, __uint_as_float(v[e + 7]) * mul);
-        d4[e >> 3] = w;
+    for (int e = 0; e < n; e += 16) {
+        uint32_t w[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            w[i] = pack_bf16x2(__uint_as_float(v[e + 2 * i]) * mul, __uint_as_float(v[e + 2 * i + 1]) * mul);
+        if (wide) {
+            st_global_v8(d4 + (e >> 3), w);
+        } else {
+            d4[e >> 3] = make_uint4(w[0], w[1], w[2], w[3]);
+            d4[(e >> 3) + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+        }
     }
 }
 
