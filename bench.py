@@ -776,10 +776,10 @@ def merge_groups(pairs):
 _TENSOR_DEPS = ("sm100_ptx.cuh", "hydra_internal.h")
 NCU_DRAM_BYTES_PER_LAUNCH = {
     # (kernel, workload): (bytes per launch, source files, their hash at capture time, capture date)
-    ("fwd", "packed32k"): (692078000, ("fwd_kernel.cu",) + _TENSOR_DEPS, "d4a1c338aeea", "2026-11-25"),
+    ("fwd", "packed32k"): (693289000, ("fwd_kernel.cu",) + _TENSOR_DEPS, "05986dad8ea8", "2026-11-25"),
     # with the dS hand-off: 1.76 GB of the key-side kernel's writes and of the query-side kernel's reads are dS
-    ("bwd_dkv", "packed32k"): (2801232000, ("bwd_kernels.cu",) + _TENSOR_DEPS, "4da3210eca3e", "2026-11-25"),
-    ("bwd_dq", "packed32k"): (2068946000, ("bwd_kernels.cu",) + _TENSOR_DEPS, "4da3210eca3e", "2026-11-25"),
+    ("bwd_dkv", "packed32k"): (2831744000, ("bwd_kernels.cu",) + _TENSOR_DEPS, "1fb384b3f8f2", "2026-11-25"),
+    ("bwd_dq", "packed32k"): (2068468000, ("bwd_kernels.cu",) + _TENSOR_DEPS, "1fb384b3f8f2", "2026-11-25"),
     ("merge", "short64k_split"): (765167000, ("aux_kernels.cu", "hydra_internal.h", "sm100_ptx.cuh"), "233647b9053e", "2026-11-25"),
     ("bwd_prep", "short64k_split"): (1082033000, ("aux_kernels.cu", "hydra_internal.h", "sm100_ptx.cuh"), "233647b9053e", "2026-11-25"),
 }
