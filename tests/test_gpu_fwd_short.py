@@ -136,3 +136,43 @@ def test_output_that_is_16_but_not_32_byte_aligned(short_len):
     got = out.float().cpu().numpy().astype(np.float64)
     assert np.abs(got - ref["out"]).max() <= TOL_REL * np.abs(ref["out"]).max()
     assert bool((raw[:off] == 0).all()) and bool((raw[off + T * h * DV * 2:] == 0).all())
+
+
+@pytest.mark.parametrize("short_len", [1 << 20, 0])
+@pytest.mark.parametrize("q_start,q_len,k_start,k_len", [
+    (0, 300, 200, 100),       # the first 200 q rows come before every key: a whole tile without keys, one with some
+    (10, 140, 149, 60),       # only the last q row sees a key (its own position)
+    (0, 130, 200, 90),        # no q row sees any key
+    (50, 200, 0, 0),          # an empty kv range
+    (255, 5, 0, 260),         # five rows at the end of a long kv range
+])
+def test_partials_of_hand_made_pairs_with_rows_that_see_no_key(short_len, q_start, q_len, k_start, k_len):
+    """Rows of a pair that see no key get O = 0 and LSE = -inf (their weight in a merge is then 0): on both
+    forward kernels, for whole tiles without keys, for single rows, and for pairs with no visible key at all."""
+    import oracle
+    import paper_2609_34318_b200 as P
+    from paper_2609_34318_b200.runner import AttnStep, bits_to_tensor
+    P.hydra_set_fwd_short_len(short_len)
+    lengths, h = [31, 300, 64], 2
+    cu = hw.cu_seqlens(lengths)
+    T = int(cu[-1])
+    x = rand_inputs(q_start + k_len, T, h)
+    pair = dict(seq=1, q_start=q_start, q_len=q_len, k_start=k_start, k_len=k_len, part_row=3, group=0)
+    step = AttnStep(cu, h, [pair], q_len + 5)
+    step.o_part.fill_(float("nan"))
+    step.lse_part.fill_(float("nan"))
+    q, k, v = (bits_to_tensor(x[n]) for n in ("q", "k", "v"))
+    P.hydra_attn_fwd(q, k, v, cu, h, step.pairs, True, step.scale, step.out, step.lse, step.o_part, step.lse_part,
+                     q_len + 5, step.workspace)
+    assert step.poll()[0] == 0
+    ref_o, ref_l = oracle.attn_partial(x["q"], x["k"], x["v"], cu, pair, True, np.float32(step.scale))
+    got_o = step.o_part.float().cpu().numpy().astype(np.float64)
+    got_l = step.lse_part.cpu().numpy().astype(np.float64)
+    assert np.isnan(got_l[:, :3]).all() and np.isnan(got_l[:, 3 + q_len:]).all(), "rows outside the pair were written"
+    o, l = got_o[3:3 + q_len], got_l[:, 3:3 + q_len]
+    assert np.array_equal(np.isneginf(l), np.isneginf(ref_l)), "which rows see no key"
+    fin = np.isfinite(ref_l)
+    if fin.any():
+        assert np.abs(l[fin] - ref_l[fin]).max() <= TOL_LSE
+    assert np.abs(o - ref_o).max() <= TOL_REL * max(np.abs(ref_o).max(), 1e-30) + 0.0
+    assert (o[np.isneginf(ref_l).T] == 0).all()
