@@ -23,6 +23,15 @@
 // UMMA issuers (one thread each; warp 10 also allocates the tensor memory).
 // K is staged as [64 keys x d_qk] (K-major B operand of S = Q K^T, N = 64), V as [64 keys x 128] in two
 // 64-column boxes (MN-major B operand of O += P V), both straight from their token-major TMA tiles.
+//
+// What bounds a slot in steady state at d_qk = 192 is its single V stage (V(j + 1) can only be asked for when
+// P V(j) has completed and arrives about 1600 cycles later), which is about what the softmax of 64 columns takes
+// with its fixed latencies; on a workload of 300-token sequences the kernel as a whole is bound by HBM (it moves
+// 5.3 TB/s). Measured and not kept: four more warps that read O out and store it while the softmax warps start
+// the next item (512 threads, registers divided with setmaxnreg, row sums handed over in shared memory: 34 %
+// slower on short sequences, 9 % on 4096-token ones, although the same kernel with the extra warps idle ran as
+// fast as without them); handing P over at the start of the next step, after the next scores have been asked
+// for from tensor memory (2 % slower: the step is bound by V, not by that load).
 #include <cuda_bf16.h>
 
 #include "hydra_internal.h"
