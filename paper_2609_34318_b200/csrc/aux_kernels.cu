@@ -86,19 +86,29 @@ hydra_lse_merge_kernel(const MergeParams p)
     constexpr int kVecPerRow = D_V / 8;           // uint4 per (row, head)
     constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
     const int n_units = rows * p.h;
-    // (row, head) of this lane group's first unit; later units are kUnitsPerPass further on
+    // Unit u of the block is (row r, head a) = (u / h, u % h). The O vectors of consecutive units are
+    // consecutive in memory ((row * h + a) * 256 bytes = (row0 * h + u) * 256 bytes), in the partial buffers and in
+    // out alike, so their addresses advance by a constant; only the LSE addresses ([h, rows] layouts) need r and
+    // a, which advance without a division. The offsets of the first batch of partials do not depend on the
+    // unit at all and are formed once per block.
     int u = threadIdx.x / kLanesPerUnit;
     int r = u / p.h, a = u - r * p.h;
     const int step_r = kUnitsPerPass / p.h, step_a = kUnitsPerPass - step_r * p.h;
+    const int64_t part_stride = static_cast<int64_t>(p.h) * kVecPerRow;         // uint4 per partial row
+    const uint4* o_row = o_part + (static_cast<int64_t>(item.row0) * p.h + u) * kVecPerRow + lane;
+    uint4* out_v = out + ((static_cast<int64_t>(g.out_tok0) + item.row0) * p.h + u) * kVecPerRow + lane;
+    int32_t pr0[kBatch];
+    int64_t off0[kBatch];
+#pragma unroll
+    for (int i = 0; i < kBatch; ++i) {
+        pr0[i] = part_row[i < g.n_parts ? i : 0];
+        off0[i] = pr0[i] * part_stride;
+    }
 
-    for (; u < n_units; u += kUnitsPerPass) {
+    for (; u < n_units; u += kUnitsPerPass, o_row += kUnitsPerPass * kVecPerRow, out_v += kUnitsPerPass * kVecPerRow) {
         const int row = item.row0 + r;
         const float* lse_row = p.lse_part + static_cast<int64_t>(a) * p.part_rows + row;
-        const uint4* o_row = o_part + (static_cast<int64_t>(row) * p.h + a) * kVecPerRow + lane;
-        const int64_t part_stride = static_cast<int64_t>(p.h) * kVecPerRow;     // uint4 per partial row
-        const int64_t tok = static_cast<int64_t>(g.out_tok0) + row;
-        uint4* out_v = out + (tok * p.h + a) * kVecPerRow + lane;
-        float* lse_out = p.lse + static_cast<int64_t>(a) * p.T + tok;
+        float* lse_out = p.lse + static_cast<int64_t>(a) * p.T + g.out_tok0 + row;
         // everything relative to m (in log2 units): acc = sum_p 2^(l_p - m) O_p, z = sum_p 2^(l_p - m)
         float m = neg_inf(), z = 0.f;
         float acc[8];
@@ -117,10 +127,11 @@ hydra_lse_merge_kernel(const MergeParams p)
 #pragma unroll
             for (int i = 0; i < kBatch; ++i) {
                 const bool have = q0 + i < g.n_parts;
-                const int32_t pr = part_row[have ? q0 + i : q0];
+                const int32_t pr = q0 == 0 ? pr0[i] : part_row[have ? q0 + i : q0];
+                const int64_t off = q0 == 0 ? off0[i] : pr * part_stride;
                 l[i] = have ? __ldg(lse_row + pr) * kLog2e : neg_inf();
                 v[i] = make_uint4(0u, 0u, 0u, 0u);
-                if (have) v[i] = ld_stream(o_row + pr * part_stride);
+                if (have) v[i] = ld_stream(o_row + off);
             }
             // a partial that saw no key (LSE = -inf) counts for nothing, whatever its O rows hold
 #pragma unroll
@@ -156,7 +167,7 @@ hydra_lse_merge_kernel(const MergeParams p)
                 for (int e = 0; e < 8; e += 2) ffma2(acc[e], acc[e + 1], f[e], f[e + 1], w, w, acc[e], acc[e + 1]);
             }
         }
-        const float inv = z > 0.f ? 1.f / z : 0.f;
+        const float inv = z > 0.f ? __frcp_rn(z) : 0.f;
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[e] *= inv;
         *out_v = pack8(acc);
