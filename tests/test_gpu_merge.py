@@ -90,3 +90,31 @@ def test_streaming_merge_takes_the_current_rows_as_one_more_input(cp_r):
                                                 out_cur=out0.float().cpu().numpy().astype(np.float64),
                                                 lse_cur=lse0.cpu().numpy().astype(np.float64))
     _compare(out, lse, ref_out, ref_lse, f"streaming cp_r {cp_r}")
+
+
+def test_buffers_that_are_16_but_not_32_byte_aligned_take_the_16_byte_kernel():
+    """The interface asks for 16-byte alignment; the merge moves 32 bytes per lane only when both the partial
+    buffer and out allow it."""
+    import paper_2609_34318_b200 as P
+    rng = np.random.default_rng(3)
+    lengths, h, cp_r = [333, 70], 2, 2
+    cu = hw.cu_seqlens(lengths)
+    T = int(cu[-1])
+    pairs, part_rows, _, _ = P.hydra_zigzag_pairs(cu, cp_r)
+    o_al, lse_part, _ = _fill(rng, part_rows, h, 0.2, 4.0)
+
+    def shifted(t):                                          # the same values at an address that is 16 modulo 32
+        raw = torch.zeros(t.numel() * t.element_size() + 64, dtype=torch.uint8, device="cuda")
+        off = (16 - raw.data_ptr() % 32) % 32
+        view = raw[off:off + t.numel() * t.element_size()].view(t.dtype).view(t.shape)
+        view.copy_(t)
+        assert view.data_ptr() % 32 == 16
+        return view
+    o_part = shifted(o_al)
+    out = shifted(torch.full((T, h, DV), float("nan"), dtype=torch.bfloat16, device="cuda"))
+    lse = torch.full((h, T), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(4096, dtype=torch.uint8, device="cuda")
+    P.hydra_lse_merge(o_part, lse_part, part_rows, cu, h, pairs, out, lse, ws)
+    torch.cuda.synchronize()
+    ref_out, ref_lse = oracle_merge_of_partials(cu, pairs, o_part, lse_part, T, h)
+    _compare(out, lse, ref_out, ref_lse, "16-byte aligned buffers")
