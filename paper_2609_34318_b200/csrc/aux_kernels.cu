@@ -338,6 +338,33 @@ hydra_bwd_prep_kernel(const uint4* __restrict__ dout, const uint4* __restrict__ 
     }
 }
 
+// The same with 32 bytes per lane (8 lanes per (row, head), 256-bit loads), for 32-byte aligned buffers.
+__global__ void __launch_bounds__(kThreads)
+hydra_bwd_prep_wide_kernel(const V8* __restrict__ dout, const V8* __restrict__ out, float* __restrict__ dsum,
+                           int64_t T, int32_t h)
+{
+    constexpr int kLanes = 8, kUnits = kThreads / kLanes, kVecPerRow = D_V / 16;
+    const int lane = threadIdx.x & (kLanes - 1);
+    const int64_t units = T * h;
+    for (int64_t u = static_cast<int64_t>(blockIdx.x) * kUnits + threadIdx.x / kLanes; u < units;
+         u += static_cast<int64_t>(gridDim.x) * kUnits) {
+        float a[16], b[16];
+        unpack16(ld_stream32(dout + u * kVecPerRow + lane), a);
+        unpack16(ld_stream32(out + u * kVecPerRow + lane), b);
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+        for (int e = 0; e < 16; e += 2) ffma2(s0, s1, a[e], a[e + 1], b[e], b[e + 1], s0, s1);
+        float s = s0 + s1;
+#pragma unroll
+        for (int o = kLanes / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) {
+            const int64_t t = u / h;
+            const int a_head = static_cast<int>(u - t * h);
+            dsum[static_cast<int64_t>(a_head) * T + t] = s;
+        }
+    }
+}
+
 // grad (bf16) = acc (fp32), eight elements per thread: two 16-byte loads, one 16-byte store.
 __global__ void __launch_bounds__(kThreads)
 hydra_grad_cast_kernel(const float4* acc, uint4* grad, int64_t n8, int64_t n, const float* acc_tail,
@@ -359,9 +386,41 @@ hydra_grad_cast_kernel(const float4* acc, uint4* grad, int64_t n8, int64_t n, co
     }
 }
 
+// Sixteen elements per thread (two 32-byte loads, one 32-byte store), for 32-byte aligned buffers; the
+// elements past the last multiple of sixteen go one per thread.
+__global__ void __launch_bounds__(kThreads)
+hydra_grad_cast_wide_kernel(const V8* acc, V8* grad, int64_t n16, int64_t n, const float* acc_tail,
+                            __nv_bfloat16* grad_tail)
+{
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kThreads;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x; i < n16; i += stride) {
+        const V8 a = ld_stream32(acc + 2 * i), b = ld_stream32(acc + 2 * i + 1);
+        uint32_t w[8];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            w[e] = pack_bf16x2(__uint_as_float(a.w[2 * e]), __uint_as_float(a.w[2 * e + 1]));
+            w[4 + e] = pack_bf16x2(__uint_as_float(b.w[2 * e]), __uint_as_float(b.w[2 * e + 1]));
+        }
+        st_global_v8(grad + i, w);
+    }
+    if (blockIdx.x == 0) {
+        const int64_t t = n16 * 16 + threadIdx.x;
+        if (t < n) grad_tail[t] = __float2bfloat16_rn(acc_tail[t]);
+    }
+}
+
 cudaError_t launch_grad_cast(const float* acc, void* grad, int64_t n, cudaStream_t stream)
 {
     if (n <= 0) return cudaSuccess;
+    if (((reinterpret_cast<uintptr_t>(acc) | reinterpret_cast<uintptr_t>(grad)) & 31u) == 0) {
+        const int64_t n16 = n / 16;
+        const int64_t blocks = (n16 + kThreads - 1) / kThreads;
+        const int grid = static_cast<int>(blocks < 1 ? 1 : (blocks < 148 * 16 ? blocks : 148 * 16));
+        hydra_grad_cast_wide_kernel<<<grid, kThreads, 0, stream>>>(reinterpret_cast<const V8*>(acc),
+                                                               static_cast<V8*>(grad), n16, n, acc,
+                                                               static_cast<__nv_bfloat16*>(grad));
+        return cudaGetLastError();
+    }
     const int64_t n8 = n / 8;
     const int64_t blocks = (n8 + kThreads - 1) / kThreads;
     const int grid = static_cast<int>(blocks < 1 ? 1 : (blocks < 148 * 16 ? blocks : 148 * 16));
@@ -453,6 +512,13 @@ cudaError_t launch_bwd_prep(const void* dout, const void* out, float* dsum, int6
     if (T * h == 0) return cudaSuccess;
     const int64_t passes = (T * h + kUnitsPerPass - 1) / kUnitsPerPass;
     const int grid = static_cast<int>(passes < 148 * 16 ? passes : 148 * 16);
+    if (((reinterpret_cast<uintptr_t>(dout) | reinterpret_cast<uintptr_t>(out)) & 31u) == 0) {
+        const int64_t wide_passes = (T * h + 2 * kUnitsPerPass - 1) / (2 * kUnitsPerPass);
+        const int wide_grid = static_cast<int>(wide_passes < 148 * 16 ? wide_passes : 148 * 16);
+        hydra_bwd_prep_wide_kernel<<<wide_grid, kThreads, 0, stream>>>(static_cast<const V8*>(dout),
+                                                                   static_cast<const V8*>(out), dsum, T, h);
+        return cudaGetLastError();
+    }
     hydra_bwd_prep_kernel<<<grid, kThreads, 0, stream>>>(static_cast<const uint4*>(dout),
                                                          static_cast<const uint4*>(out), dsum, T, h);
     return cudaGetLastError();
