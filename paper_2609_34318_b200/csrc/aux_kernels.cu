@@ -3,7 +3,8 @@
 //   hydra_bwd_prep_kernel   D = rowsum(dO * O)
 //   hydra_grad_cast_kernel  fp32 gradient accumulators -> bf16 (after a backward run step by step)
 //   hydra_ulysses_kernel    the local permutation before / after the head <-> sequence all-to-all
-// Both move every byte once with 16-byte accesses: 16 lanes own one (row, head) vector of 128 bf16.
+// All move every byte once: 8 lanes with 32-byte accesses own one (row, head) vector of 128 bf16 (16 lanes with
+// 16-byte accesses where a buffer is only 16-byte aligned).
 #include <cuda_bf16.h>
 
 #include <algorithm>
