@@ -123,3 +123,43 @@ def test_bad_arguments_are_refused():
     assert P.hydra_gate_apply(z, z, 12, z, check=False) == P.HYDRA_ERR_INVALID_ARG
     assert P.hydra_mla_kv_assemble(z, z, z, 4, 2, 128, 63, 128, THETA, z, z, check=False) == P.HYDRA_ERR_INVALID_ARG
     assert P.hydra_launch_count() == n0
+
+
+@pytest.mark.parametrize("in_place", [False, True])
+def test_dimensions_that_are_not_multiples_of_eight_take_the_four_byte_kernels(in_place):
+    """The kernels move 16 bytes per access where every dimension is a multiple of 8 elements; other (even)
+    dimensions fall back to one rotary pair per access. Heads of 20 with rotary columns [4, 16); an up-projection of
+    12 + 10 columns with a rotary key of 4."""
+    import paper_2609_34318_b200 as P
+    rng = np.random.default_rng(54)
+    lengths, h = [9, 70], 3
+    pos = positions_for(lengths)
+    T = len(pos)
+    pd = torch.from_numpy(pos).cuda()
+    xb = bits(rng, (T, h, 20))
+    x = hw.bf16_bits_to_f64(xb)
+    ref = M.rope(x, pos, 4, 12, THETA)
+    xd = dev(xb)
+    yd = xd if in_place else torch.full_like(xd, float("nan"))
+    P.hydra_mla_rope(xd, pd, T, h, 20, 4, 12, THETA, False, yd)
+    torch.cuda.synchronize()
+    got = f64(yd)
+    assert np.array_equal(got[..., :4], x[..., :4]) and np.array_equal(got[..., 16:], x[..., 16:])
+    close(got[..., 4:16], ref[..., 4:16], np.abs(x).max(), "rope, odd dimensions")
+    up_b, pe_b = bits(rng, (T, h, 22)), bits(rng, (T, 4))
+    k_ref, v_ref = M.kv_assemble(hw.bf16_bits_to_f64(up_b), hw.bf16_bits_to_f64(pe_b), pos, 12, 4, 10, THETA)
+    k = torch.full((T, h, 16), float("nan"), dtype=torch.bfloat16, device="cuda")
+    v = torch.full((T, h, 10), float("nan"), dtype=torch.bfloat16, device="cuda")
+    P.hydra_mla_kv_assemble(dev(up_b), dev(pe_b), pd, T, h, 12, 4, 10, THETA, k, v)
+    torch.cuda.synchronize()
+    gk, gv = f64(k), f64(v)
+    assert np.array_equal(gk[..., :12], k_ref[..., :12]) and np.array_equal(gv, v_ref)
+    close(gk[..., 12:], k_ref[..., 12:], np.abs(hw.bf16_bits_to_f64(pe_b)).max(), "assembled key, odd dimensions")
+    dk_b, dv_b = bits(rng, (T, h, 16)), bits(rng, (T, h, 10))
+    up_ref, pe_ref = M.kv_assemble_bwd(hw.bf16_bits_to_f64(dk_b), hw.bf16_bits_to_f64(dv_b), pos, 12, 4, 10, THETA)
+    dup = torch.full((T, h, 22), float("nan"), dtype=torch.bfloat16, device="cuda")
+    dpe = torch.full((T, 4), float("nan"), dtype=torch.bfloat16, device="cuda")
+    P.hydra_mla_kv_assemble_bwd(dev(dk_b), dev(dv_b), pd, T, h, 12, 4, 10, THETA, dup, dpe)
+    torch.cuda.synchronize()
+    assert np.array_equal(f64(dup), up_ref)
+    close(f64(dpe), pe_ref, np.abs(pe_ref).max(), "rotary key gradient, odd dimensions")
