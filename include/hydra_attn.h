@@ -480,7 +480,8 @@ int32_t hydra_gate_apply_bwd(const void* dy, const void* out, const void* gate, 
 /*
  * Per-kernel timing (measurement aid, not part of the method). While enabled, every kernel launch
  * is bracketed by CUDA events on its stream. hydra_profile_collect waits for the recorded events,
- * adds their durations into ms_out[8] and their counts into launches_out[8] (index: 0 forward,
+ * adds their durations into ms_out[8] and their counts into launches_out[8] (index: 0 forward, both of its
+ * kernels when a call uses both,
  * 1 merge, 2 backward prep, 3 backward dK/dV, 4 backward dQ, 5 gradient cast, 6 Ulysses pack / unpack,
  * 7 the elementwise steps of the gated MLA block)
  * and forgets them.
@@ -530,7 +531,7 @@ void hydra_set_wait_limit_ns(uint64_t ns);
  * block in `detail` and returns by itself (no trap, no endless loop, nothing in flight). Outputs of such
  * a launch are not written. ns = 0 (the default) switches the hook off; it costs one predicate per launch.
  */
-#define HYDRA_STALL_FWD 0
+#define HYDRA_STALL_FWD 0       /* either forward kernel */
 #define HYDRA_STALL_BWD_DKV 1
 #define HYDRA_STALL_BWD_DQ 2    /* either form of the query-side kernel */
 void hydra_debug_stall(int32_t kernel, uint64_t ns);
