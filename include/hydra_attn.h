@@ -314,8 +314,10 @@ int32_t hydra_attn_bwd_accumulate_gqa(const void* q, const void* k, const void* 
 /*
  * The whole step (forward of every pair, merge, backward; Sections 3.5 and 5.2 as above) with HOST
  * buffers: copies q, k, v, dout to the device, runs hydra_attn_fwd, hydra_lse_merge (if any pair has
- * partial rows) and hydra_attn_bwd, and copies out, lse, dq, dk, dv back. Heads are independent,
- * so with 4 or more heads the step is pipelined over groups of 2 or 4 heads: the kernels run on
+ * partial rows) and hydra_attn_bwd, and copies out, lse, dq, dk, dv back. Sequences and heads are
+ * independent, so the step is pipelined over groups: runs of whole sequences with all heads
+ * (contiguous on the host) when every sequence is small against the step, else groups of 2 or 4
+ * heads over all sequences (with 4 or more heads). The kernels run on
  * `cuda_stream`, the copies in and out on two internal streams (created once per device, on the
  * first call), so that both directions of the host link are busy at once. Work enqueued on
  * `cuda_stream` before the call precedes all of it, and `cuda_stream` completes only when the last

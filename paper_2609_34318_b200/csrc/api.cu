@@ -1093,6 +1093,40 @@ HostPipe* host_pipe()
     if (!ok) return nullptr;
     return &pipes.emplace(dev, p).first->second;
 }
+
+// Groups of the host-buffer step. The out-copy of a group cannot start before its in-copy has ended, so a step
+// takes the copies of one direction plus those of its largest group, and every copy costs some 15 us beyond its
+// bytes. When the copies bound the step and every sequence fits a group of 1/24 of the (token, head) pairs (not
+// under 1 MB of inputs: the launches of a group cost about as much as that copy), a group is a run of whole
+// sequences with all heads, contiguous on the host. Otherwise it is a range of heads over all sequences, strided on
+// the host: two heads when the copies bound the step, four (which keep the kernels efficient) when the arithmetic
+// does; narrower rows slow the link down, and so did groups of both kinds mixed in one step (copies of a few MB).
+struct HostGroup { int32_t s0, s1, h0, hn; int64_t t0, tn; };
+std::vector<HostGroup> host_groups(const Problem& pb, bool copy_bound)
+{
+    std::vector<HostGroup> g;
+    const int32_t h = pb.h;
+    if (copy_bound) {
+        int64_t target = std::max<int64_t>(pb.T * h / 24, (int64_t{1} << 20) / ((2 * D_QK + 2 * D_V) * 2));
+        for (bool fits = true; fits; target *= 2) {
+            g.clear();
+            for (int32_t s = 0; s < pb.n_seqs && fits;) {
+                int32_t e = s;
+                int64_t tok = 0;
+                while (e < pb.n_seqs && (tok + pb.cu[e + 1] - pb.cu[e]) * h <= target) tok += pb.cu[e + 1] - pb.cu[e], ++e;
+                fits = e > s;
+                if (tok > 0) g.push_back({s, e, 0, h, pb.cu[s], tok});
+                s = e;
+            }
+            if (fits && g.size() <= static_cast<size_t>(HostPipe::kMaxGroups)) return g;
+        }
+        g.clear();
+    }
+    int32_t hg = h < 4 ? h : (copy_bound ? 2 : 4);
+    hg = std::max(hg, (h + HostPipe::kMaxGroups - 1) / HostPipe::kMaxGroups);
+    for (int32_t h0 = 0; h0 < h; h0 += hg) g.push_back({0, pb.n_seqs, h0, std::min(hg, h - h0), 0, pb.T});
+    return g;
+}
 }  // namespace
 
 extern "C" {
@@ -2043,19 +2077,13 @@ int32_t hydra_attn_fwd_bwd_host(const void* q_host, const void* k_host, const vo
     float* lse_part = static_cast<float*>(carve(static_cast<size_t>(std::max<int64_t>(part_rows, 1)) * n_heads * 4));
     void* ws = carve(kStatusBytes + align_up(th * 4, 256));
     const size_t ws_bytes = kStatusBytes + align_up(th * 4, 256);
-    const bool any_part = part_rows > 0;
 
-    // Heads are independent, so the step is pipelined over groups of heads: while group g computes,
-    // group g+1 is on its way in and group g-1 on its way out, on two internal copy streams; the PCIe
-    // link then carries both directions at once instead of one after the other. On the device a
-    // group is a compact [T, heads_of_group, d] tensor (the g-th slice of each arena tensor); on the
-    // host it is a strided view of [T, n_heads, d], moved by 2-D copies.
+    // Sequences and heads are independent, so the step is pipelined over groups (a range of whole sequences
+    // times a range of heads): while group g computes, group g+1 is on its way in and group g-1 on its way
+    // out, on two internal copy streams; the host link then carries both directions at once. On the device a
+    // group is a compact [tokens, heads_of_group, d] tensor inside its token range of each arena tensor.
     HostPipe* pipe = host_pipe();
     if (!pipe) return HYDRA_ERR_CUDA;
-    // Group size: when the copies dominate (short sequences: bytes grow with T, arithmetic with the
-    // pair count), small groups shorten the fill and the drain of the pipeline and the kernels,
-    // though less efficient on few heads, still hide under the copies; when the arithmetic
-    // dominates, larger groups keep the kernels efficient. Rough rates: 50 GB/s, 700 TFLOP/s.
     double pair_count = 0.0;
     for (const auto& p : pb.pairs) {
         const double full = static_cast<double>(p.q_len) * p.k_len;
@@ -2063,65 +2091,87 @@ int32_t hydra_attn_fwd_bwd_host(const void* q_host, const void* k_host, const vo
                                                   static_cast<double>(p.q_len) * std::max(0, p.q_start - p.k_start))
                              : full;
     }
+    // rough rates: 50 GB/s per direction, 700 TFLOP/s
     const double copy_s = static_cast<double>(pb.T) * (2 * D_QK + 2 * D_V) * 2 / 50e9;   // per head, one direction
     const double math_s = pair_count * 3.5 * 2 * (D_QK + D_V) / 700e12;                  // per head
-    int32_t hg = n_heads < 4 ? n_heads : (math_s < 0.5 * copy_s ? 2 : 4);
-    hg = std::max(hg, (n_heads + HostPipe::kMaxGroups - 1) / HostPipe::kMaxGroups);   // at most kMaxGroups groups
-    const int32_t n_groups = (n_heads + hg - 1) / hg;
-    size_t lse_off[HostPipe::kMaxGroups + 1] = {0};         // LSE slices start on 256-byte boundaries
-    for (int32_t g = 0; g < n_groups; ++g)
-        lse_off[g + 1] = align_up(lse_off[g] + static_cast<size_t>(pb.T) * std::min(hg, n_heads - g * hg) * 4, 256);
-    const size_t T = static_cast<size_t>(pb.T);
-    auto copy2d = [&](void* dst, size_t dpitch, const void* src, size_t spitch, size_t width, cudaMemcpyKind kind,
-                      cudaStream_t st) { return cudaMemcpy2DAsync(dst, dpitch, src, spitch, width, T, kind, st); };
+    const std::vector<HostGroup> groups = host_groups(pb, math_s < 0.5 * copy_s);
+    const int32_t n_groups = static_cast<int32_t>(groups.size());
+    const size_t H = static_cast<size_t>(n_heads);
+    struct Slice { size_t oqk, ov, lse; };                  // byte offsets of a group's tensors in the arena tensors
+    std::vector<Slice> slice(n_groups);
+    size_t lse_off = 0;
+    for (int32_t g = 0; g < n_groups; ++g) {
+        const HostGroup& G = groups[g];
+        const size_t th0 = static_cast<size_t>(G.t0) * H + static_cast<size_t>(G.tn) * G.h0;   // (token, head) pairs before it
+        slice[g] = {th0 * D_QK * 2, th0 * D_V * 2, lse_off};
+        lse_off = align_up(lse_off + static_cast<size_t>(G.tn) * G.hn * 4, 256);
+    }
+    // one tensor of a group between the host's [T, n_heads, d] layout and the group's compact one
+    auto move = [&](const HostGroup& G, uint8_t* dev, const uint8_t* host_base, size_t row_bytes, bool to_device,
+                    cudaStream_t st) {
+        uint8_t* host = const_cast<uint8_t*>(host_base) + (static_cast<size_t>(G.t0) * H + G.h0) * row_bytes;
+        const cudaMemcpyKind kind = to_device ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost;
+        const size_t width = static_cast<size_t>(G.hn) * row_bytes, rows = static_cast<size_t>(G.tn);
+        if (G.hn == n_heads)
+            return to_device ? cudaMemcpyAsync(dev, host, width * rows, kind, st) : cudaMemcpyAsync(host, dev, width * rows, kind, st);
+        return to_device ? cudaMemcpy2DAsync(dev, width, host, H * row_bytes, width, rows, kind, st)
+                         : cudaMemcpy2DAsync(host, H * row_bytes, dev, width, width, rows, kind, st);
+    };
     if (cudaEventRecord(pipe->start, stream) || cudaStreamWaitEvent(pipe->in, pipe->start, 0) ||
         cudaStreamWaitEvent(pipe->out, pipe->start, 0))
         return HYDRA_ERR_CUDA;
     for (int32_t g = 0; g < n_groups; ++g) {
-        const int32_t h0 = g * hg, hn = std::min(hg, n_heads - h0);
-        const size_t oqk = T * h0 * D_QK * 2, ov = T * h0 * D_V * 2;          // the group's slice of the arena tensors
-        const size_t wqk = static_cast<size_t>(hn) * D_QK * 2, wv = static_cast<size_t>(hn) * D_V * 2;
-        const size_t pqk = static_cast<size_t>(n_heads) * D_QK * 2, pv = static_cast<size_t>(n_heads) * D_V * 2;
-        const uint8_t* qh = static_cast<const uint8_t*>(q_host) + static_cast<size_t>(h0) * D_QK * 2;
-        const uint8_t* kh = static_cast<const uint8_t*>(k_host) + static_cast<size_t>(h0) * D_QK * 2;
-        const uint8_t* vh = static_cast<const uint8_t*>(v_host) + static_cast<size_t>(h0) * D_V * 2;
-        const uint8_t* doh = static_cast<const uint8_t*>(dout_host) + static_cast<size_t>(h0) * D_V * 2;
-        if (copy2d(q + oqk, wqk, qh, pqk, wqk, cudaMemcpyHostToDevice, pipe->in) ||
-            copy2d(k + oqk, wqk, kh, pqk, wqk, cudaMemcpyHostToDevice, pipe->in) ||
-            copy2d(v + ov, wv, vh, pv, wv, cudaMemcpyHostToDevice, pipe->in) ||
-            copy2d(dout + ov, wv, doh, pv, wv, cudaMemcpyHostToDevice, pipe->in) ||
+        const HostGroup& G = groups[g];
+        if (move(G, q + slice[g].oqk, static_cast<const uint8_t*>(q_host), D_QK * 2, true, pipe->in) ||
+            move(G, k + slice[g].oqk, static_cast<const uint8_t*>(k_host), D_QK * 2, true, pipe->in) ||
+            move(G, v + slice[g].ov, static_cast<const uint8_t*>(v_host), D_V * 2, true, pipe->in) ||
+            move(G, dout + slice[g].ov, static_cast<const uint8_t*>(dout_host), D_V * 2, true, pipe->in) ||
             cudaEventRecord(pipe->in_done[g], pipe->in))
             return HYDRA_ERR_CUDA;
     }
+    std::vector<int32_t> cu_g;
+    std::vector<hydra_pair_t> pairs_g;
     for (int32_t g = 0; g < n_groups; ++g) {
-        const int32_t h0 = g * hg, hn = std::min(hg, n_heads - h0);
-        const size_t oqk = T * h0 * D_QK * 2, ov = T * h0 * D_V * 2;
-        const size_t wqk = static_cast<size_t>(hn) * D_QK * 2, wv = static_cast<size_t>(hn) * D_V * 2;
-        const size_t pqk = static_cast<size_t>(n_heads) * D_QK * 2, pv = static_cast<size_t>(n_heads) * D_V * 2;
-        float* lse_g = reinterpret_cast<float*>(lse + lse_off[g]);
+        const HostGroup& G = groups[g];
+        const size_t oqk = slice[g].oqk, ov = slice[g].ov;
+        float* lse_g = reinterpret_cast<float*>(lse + slice[g].lse);
+        if (g == 0 || G.s0 != groups[g - 1].s0) {            // the sequences of this group, and their pairs, renumbered
+            cu_g.assign(cu + G.s0, cu + G.s1 + 1);
+            for (int32_t& c : cu_g) c -= cu[G.s0];
+            pairs_g.clear();
+            for (int32_t i = 0; i < n_pairs; ++i)
+                if (pairs[i].seq >= G.s0 && pairs[i].seq < G.s1) {
+                    pairs_g.push_back(pairs[i]);
+                    pairs_g.back().seq -= G.s0;
+                }
+        }
+        const int32_t ns = G.s1 - G.s0, np = static_cast<int32_t>(pairs_g.size());
+        const hydra_pair_t* pg = np ? pairs_g.data() : nullptr;
+        bool part = false;
+        for (const hydra_pair_t& p : pairs_g) part = part || p.part_row >= 0;
         if (cudaStreamWaitEvent(stream, pipe->in_done[g], 0)) return HYDRA_ERR_CUDA;
-        if (int32_t s = hydra_attn_fwd(q + oqk, k + oqk, v + ov, cu, n_seqs, hn, pairs, n_pairs, causal, softmax_scale,
-                                       out + ov, lse_g, any_part ? o_part : nullptr, any_part ? lse_part : nullptr,
-                                       part_rows, ws, ws_bytes, cuda_stream))
-            return s;
-        if (any_part)
-            if (int32_t s = hydra_lse_merge(o_part, lse_part, part_rows, cu, n_seqs, hn, pairs, n_pairs, out + ov,
-                                            lse_g, ws, ws_bytes, cuda_stream))
+        if (n_pairs == 0 || np > 0) {                        // sequences without any pair of the caller's list: nothing to compute
+            if (int32_t s = hydra_attn_fwd(q + oqk, k + oqk, v + ov, cu_g.data(), ns, G.hn, pg, np, causal, softmax_scale,
+                                           out + ov, lse_g, part ? o_part : nullptr, part ? lse_part : nullptr,
+                                           part ? part_rows : 0, ws, ws_bytes, cuda_stream))
                 return s;
-        if (int32_t s = hydra_attn_bwd(q + oqk, k + oqk, v + ov, out + ov, lse_g, dout + ov, cu, n_seqs, hn, pairs,
-                                       n_pairs, causal, softmax_scale, dq_ + oqk, dk_ + oqk, dv_ + ov, ws, ws_bytes,
-                                       cuda_stream))
-            return s;
-        uint8_t* outh = static_cast<uint8_t*>(out_host) + static_cast<size_t>(h0) * D_V * 2;
-        uint8_t* dqh = static_cast<uint8_t*>(dq_host) + static_cast<size_t>(h0) * D_QK * 2;
-        uint8_t* dkh = static_cast<uint8_t*>(dk_host) + static_cast<size_t>(h0) * D_QK * 2;
-        uint8_t* dvh = static_cast<uint8_t*>(dv_host) + static_cast<size_t>(h0) * D_V * 2;
+            if (part)
+                if (int32_t s = hydra_lse_merge(o_part, lse_part, part_rows, cu_g.data(), ns, G.hn, pg, np, out + ov,
+                                                lse_g, ws, ws_bytes, cuda_stream))
+                    return s;
+            if (int32_t s = hydra_attn_bwd(q + oqk, k + oqk, v + ov, out + ov, lse_g, dout + ov, cu_g.data(), ns, G.hn,
+                                           pg, np, causal, softmax_scale, dq_ + oqk, dk_ + oqk, dv_ + ov, ws, ws_bytes,
+                                           cuda_stream))
+                return s;
+        }
         if (cudaEventRecord(pipe->comp_done[g], stream) || cudaStreamWaitEvent(pipe->out, pipe->comp_done[g], 0) ||
-            copy2d(outh, pv, out + ov, wv, wv, cudaMemcpyDeviceToHost, pipe->out) ||
-            cudaMemcpyAsync(lse_host + T * h0, lse_g, T * hn * 4, cudaMemcpyDeviceToHost, pipe->out) ||
-            copy2d(dqh, pqk, dq_ + oqk, wqk, wqk, cudaMemcpyDeviceToHost, pipe->out) ||
-            copy2d(dkh, pqk, dk_ + oqk, wqk, wqk, cudaMemcpyDeviceToHost, pipe->out) ||
-            copy2d(dvh, pv, dv_ + ov, wv, wv, cudaMemcpyDeviceToHost, pipe->out))
+            move(G, out + ov, static_cast<const uint8_t*>(out_host), D_V * 2, false, pipe->out) ||
+            cudaMemcpy2DAsync(lse_host + static_cast<size_t>(G.h0) * pb.T + G.t0, static_cast<size_t>(pb.T) * 4, lse_g,
+                              static_cast<size_t>(G.tn) * 4, static_cast<size_t>(G.tn) * 4, G.hn, cudaMemcpyDeviceToHost,
+                              pipe->out) ||
+            move(G, dq_ + oqk, static_cast<const uint8_t*>(dq_host), D_QK * 2, false, pipe->out) ||
+            move(G, dk_ + oqk, static_cast<const uint8_t*>(dk_host), D_QK * 2, false, pipe->out) ||
+            move(G, dv_ + ov, static_cast<const uint8_t*>(dv_host), D_V * 2, false, pipe->out))
             return HYDRA_ERR_CUDA;
     }
     // the caller's stream completes when the last copy out has completed

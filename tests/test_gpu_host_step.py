@@ -1,8 +1,10 @@
 """The whole step through the C ABI with HOST buffers (`hydra_attn_fwd_bwd_host`) against the oracle.
 
-The entry point pipelines groups of heads over two internal copy streams; the cases cover a head count
-that splits into full groups plus a remainder, a single group, chunked pairs through the merge, and
-two calls in a row on the same arena (the internal streams and events are reused).
+The entry point pipelines groups over two internal copy streams: runs of whole sequences when every sequence is
+small against the step, ranges of heads over all sequences otherwise. The cases cover a head count that splits
+into full groups plus a remainder, a single group, a step of many short sequences (groups of sequences, one of
+them empty), chunked pairs through the merge in both forms, and two calls in a row on the same arena (the
+internal streams and events are reused).
 """
 import numpy as np
 import pytest
@@ -48,6 +50,19 @@ def test_host_step_matches_the_oracle(h, cp_r):
     got = host_step(x, cu, h, lib_pairs)
     ref = run_oracle(x, cu, True, pairs=ora_pairs)
     check(got, ref, label=f"host step h={h} cp_r={cp_r}: ")
+
+
+@pytest.mark.parametrize("h,cp_r", [(8, 0), (6, 1), (5, 0)])
+def test_host_step_in_groups_of_sequences(h, cp_r):
+    """Many short sequences, none over a group's share of the step: runs of sequences travel as contiguous token
+    ranges with all heads (about 16 groups here); a sequence without tokens sits inside one of them."""
+    lengths = [5] * 60 + [0] + [17, 40, 3] * 12 + [90] * 6
+    cu = hw.cu_seqlens(lengths)
+    x = rand_inputs(np.random.default_rng(300 + h), int(cu[-1]), h)
+    lib_pairs, _, ora_pairs = pairs_for(cu, cp_r) if cp_r else (None, 0, None)
+    got = host_step(x, cu, h, lib_pairs)
+    ref = run_oracle(x, cu, True, pairs=ora_pairs)
+    check(got, ref, label=f"host step in groups of sequences h={h} cp_r={cp_r}: ")
 
 
 def test_two_host_steps_in_a_row_give_the_same_bits():
