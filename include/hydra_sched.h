@@ -70,8 +70,8 @@ int32_t hydra_sched_cp(int64_t s, int64_t s_max, int32_t C, int64_t B);
  *   - if there is none, the micro-batch is closed and the document opens the next one;
  *   - the micro-batch is also closed when the next document's degree is smaller than the one just
  *     used, no rank is free, and the least-loaded group carries at least 3/4 of the per-rank load
- *     of the most loaded one ("k has shrunk and MB balanced": the paper does not define the test;
- *     this is the reading taken here);
+ *     of the most loaded one (the early-close test at the end of Algorithm 1's inner loop, which the
+ *     paper names without defining it: this is the reading taken here);
  *   - idle ranks of a closed micro-batch are backfilled by doubling the smallest group (the more
  *     loaded one among equals) while it is no larger than the number of idle ranks;
  *   - groups then take consecutive rank blocks in order of decreasing size, so that every group

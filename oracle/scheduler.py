@@ -20,7 +20,7 @@ ceil2(x) is the smallest power of two that is at least x.
 Readings where the paper only sketches (the library takes the same ones; they are listed in the design
 notes):
   R1  Ties after (size, load) go to the group opened first; equal lengths keep their input order.
-  R2  "k has shrunk and MB balanced": after a placement, if the next document's degree is smaller than
+  R2  the early-close test at the end of Algorithm 1's inner loop (degree shrunk, micro-batch balanced): after a placement, if the next document's degree is smaller than
       the degree just used, every rank is busy, and the least-loaded group carries at least 3/4 of the
       per-rank load of the most loaded one, the micro-batch is closed.
   R3  Backfill: while the smallest open group (ties: higher per-rank load first, then opened first) is
