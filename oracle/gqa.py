@@ -3,8 +3,8 @@ for the GQA model of Section 6, which shares eight KV heads).
 
 TEST INFRASTRUCTURE ONLY. Nothing in the product path imports this module.
 
-Definition used (the paper names the head counts only; this is the usual grouping, stated as a reading in
-the design notes): with g = h / h_kv, query head a attends to KV head a // g. So the forward is the
+Definition used (the paper names the head counts only; this is the usual grouping, taken as a reading):
+with g = h / h_kv, query head a attends to KV head a // g. So the forward is the
 per-head attention of the plain oracle on K, V with every KV head written out g times, and the gradient of
 a KV head is the SUM of the per-head gradients of the g query heads that read it. The two steps are written
 exactly like that: expand, call the plain oracle, sum.

@@ -17,11 +17,10 @@ What follows the paper literally
   are backfilled; next micro-batch.
 ceil2(x) is the smallest power of two that is at least x.
 
-Readings where the paper only sketches (the library takes the same ones; they are listed in the design
-notes):
+Readings where the paper only sketches (the library takes the same ones):
   R1  Ties after (size, load) go to the group opened first; equal lengths keep their input order.
-  R2  the early-close test at the end of Algorithm 1's inner loop (degree shrunk, micro-batch balanced): after a placement, if the next document's degree is smaller than
-      the degree just used, every rank is busy, and the least-loaded group carries at least 3/4 of the
+  R2  The early-close test at the end of Algorithm 1's inner loop (degree shrunk, micro-batch balanced): after a
+      placement, if the next document's degree is smaller than the degree just used, every rank is busy, and the least-loaded group carries at least 3/4 of the
       per-rank load of the most loaded one, the micro-batch is closed.
   R3  Backfill: while the smallest open group (ties: higher per-rank load first, then opened first) is
       no larger than the number of idle ranks, it is doubled (its documents run at twice the degree).
