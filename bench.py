@@ -699,6 +699,46 @@ def run_report(args, w):
         report["d128_gqa_8_to_1"] = {"kv_heads": h_kv, "ms": dms, "tflops": tf(flops128, sum(dms.values())),
                                      "flop_convention": "2 * pairs * h * (128 + 128) forward, backward 2.5 x"}
         del q8, k8, v8, do8, out8, dq8, dk8, dv8, ws8
+    # The elementwise steps of a gated MLA block around the kernel (Section 5.2.2) on this workload's tokens and
+    # heads: RoPE on the rotary slice of q (out of place), assembly of k / v from the up-projection and its
+    # backward, the output gate and its backward; L2 flushed before each, rates over the algorithmic bytes.
+    n, hh = w.total, w.n_heads
+    d_nope, d_rope = hw.D_QK - 64, 64
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(hw.SEED + 7)
+    rnd = lambda *shape: torch.randn(shape, generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    pos = (torch.arange(n, device="cuda", dtype=torch.int32) % 4096).contiguous()
+    q_rot = torch.empty_like(t["q"])
+    kv_up, k_pe = rnd(n, hh, d_nope + hw.D_V), rnd(n, d_rope)
+    k_as, v_as = torch.empty_like(t["k"]), torch.empty_like(t["v"])
+    dkv_up, dk_pe = torch.empty_like(kv_up), torch.empty_like(k_pe)
+    gate, y = rnd(n, hh, hw.D_V), torch.empty_like(t["v"])
+    d_out, d_gate = torch.empty_like(y), torch.empty_like(y)
+    kv_bytes = (kv_up.numel() + k_pe.numel() + k_as.numel() + v_as.numel()) * 2.0
+    ops = {
+        "rope_q": (lambda: P.hydra_mla_rope(t["q"], pos, n, hh, hw.D_QK, d_nope, d_rope, 10000.0, False, q_rot),
+                   t["q"].numel() * 4.0),
+        "kv_assemble": (lambda: P.hydra_mla_kv_assemble(kv_up, k_pe, pos, n, hh, d_nope, d_rope, hw.D_V, 10000.0,
+                                                        k_as, v_as), kv_bytes),
+        "kv_assemble_bwd": (lambda: P.hydra_mla_kv_assemble_bwd(k_as, v_as, pos, n, hh, d_nope, d_rope, hw.D_V,
+                                                                10000.0, dkv_up, dk_pe), kv_bytes),
+        "gate": (lambda: P.hydra_gate_apply(t["v"], gate, y.numel(), y), y.numel() * 6.0),
+        "gate_bwd": (lambda: P.hydra_gate_apply_bwd(y, t["v"], gate, y.numel(), d_out, d_gate), y.numel() * 10.0),
+    }
+    report["mla_elementwise"] = {}
+    for name, (fn, nbytes) in ops.items():
+        times = []
+        for _ in range(5):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        ms = statistics.median(times)
+        report["mla_elementwise"][name] = {"ms": ms, "bytes": nbytes, "gbs": gbs(nbytes, ms)}
+    del q_rot, kv_up, k_pe, k_as, v_as, dkv_up, dk_pe, gate, y, d_out, d_gate
     if args.per_sequence:
         # every sequence alone, same kernels: its share of the time next to its share of sum(L^2)
         shares = []
