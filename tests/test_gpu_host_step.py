@@ -65,6 +65,30 @@ def test_host_step_in_groups_of_sequences(h, cp_r):
     check(got, ref, label=f"host step in groups of sequences h={h} cp_r={cp_r}: ")
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_random_host_steps(seed):
+    """Seeded mixes: many short sequences (groups of sequences), short ones around a long one and a few long ones
+    (groups of heads), 1 to 12 heads, some sequences cut into zigzag chunks."""
+    rng = np.random.default_rng(5000 + seed)
+    style = ["many_short", "mixed", "few"][seed % 3]
+    if style == "many_short":
+        lengths = [int(v) for v in rng.integers(0, 120, size=int(rng.integers(20, 120)))]
+    elif style == "mixed":
+        lengths = [int(v) for v in rng.integers(1, 200, size=int(rng.integers(5, 40)))] + [int(rng.integers(300, 1500))]
+        lengths = [lengths[i] for i in rng.permutation(len(lengths))]
+    else:
+        lengths = [int(v) for v in rng.integers(1, 900, size=int(rng.integers(1, 4)))]
+    if sum(lengths) == 0:
+        lengths.append(3)
+    h = int(rng.integers(1, 13))
+    cp_r = [int(v) for v in rng.choice([0, 0, 0, 1, 2], size=len(lengths))]
+    cu = hw.cu_seqlens(lengths)
+    x = rand_inputs(rng, int(cu[-1]), h)
+    lib_pairs, _, ora_pairs = pairs_for(cu, cp_r) if any(cp_r) else (None, 0, None)
+    got = host_step(x, cu, h, lib_pairs)
+    check(got, run_oracle(x, cu, True, pairs=ora_pairs), label=f"host step seed {seed} ({style}, h={h}): ")
+
+
 def test_two_host_steps_in_a_row_give_the_same_bits():
     cu = hw.cu_seqlens([200, 513])
     x = rand_inputs(np.random.default_rng(7), int(cu[-1]), 12)
