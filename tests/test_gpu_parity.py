@@ -179,6 +179,36 @@ def bf16_operand_backward(x, L, scale, out_given):
     return dict(dq=scale * ds @ k, dk=scale * ds.T @ q, dv=bf16_round(p).T @ g)
 
 
+@pytest.mark.parametrize("L", [2, 3, 4])
+def test_a_sequence_of_two_to_four_tokens_alone(L):
+    """With two to four keys the probabilities are of order one and dS = P (dP - D) is a difference of near-equal
+    numbers, so the rounding of the stored bf16 O inside D = <dO, O> (about 2^-9 |dO| |O| sqrt(128), the same at every
+    length) is no longer small against dQ, whose largest entry is small when only one or two rows have a gradient
+    at all: the oracle's own dQ moves by up to 4 % of its maximum when its O is rounded to bf16
+    (tests/test_oracle_pins.py::test_rounding_the_stored_output_moves_dq_of_tiny_sequences). Same protocol as the
+    monotone-score case: the GPU must match, within the contract's 2e-2, the fp64 model evaluated from what the
+    kernel was given (its own stored O); against the oracle the bound is set from that model's distance to it.
+    O and LSE are held to the contract against the oracle."""
+    h = 1
+    scale = float(np.float32(1.0 / np.sqrt(np.float32(DQK))))
+    worst = {n: 0.0 for n in ("dq", "dk", "dv")}
+    for seed in range(24):
+        x = rand_inputs(np.random.default_rng(9100 + 31 * L + seed), L, h)
+        cu = hw.cu_seqlens([L])
+        got = run_gpu(x, cu, h)
+        ref = run_oracle(x, cu)
+        check(got, ref, names=("out", "lse"), label=f"L={L} seed {seed} ")
+        model = bf16_operand_backward(x, L, scale, got["out"][:, 0])
+        for n in ("dq", "dk", "dv"):
+            g, m, r = got[n][:, 0], model[n], ref[n][:, 0]
+            top = np.abs(r).max()
+            err_model, err_oracle, model_oracle = (np.abs(a - b).max() / top for a, b in ((g, m), (g, r), (m, r)))
+            worst[n] = max(worst[n], err_oracle)
+            assert err_model <= TOL_REL, (n, seed, err_model)
+            assert err_oracle <= TOL_REL + 1.5 * model_oracle, (n, seed, err_oracle, model_oracle)
+    print(f"L={L}: largest gpu-oracle distance over 24 seeds, relative to max|ref|: {worst}")
+
+
 def test_large_scores():
     rng = np.random.default_rng(8)
     L, h = 520, 2
