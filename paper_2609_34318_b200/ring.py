@@ -175,7 +175,9 @@ class RingRank:
         self.dq_acc = new((rows, h, dqk), f32)
         self.dkv_acc = [(new((cap, h_kv, dqk), f32), new((cap, h_kv, dv), f32)) for _ in range(2)]
         ws = compute.workspace_bytes(sched, rank) if hasattr(compute, "workspace_bytes") else 4096
-        self.workspace = torch.empty(ws, dtype=torch.uint8, device=self.device)
+        # zeroed: a rank whose steps hold no pair (sequences shorter than the number of chunks) launches nothing,
+        # and its status block must still read as OK
+        self.workspace = torch.zeros(ws, dtype=torch.uint8, device=self.device)
         self.log: List[Tuple[str, int, int]] = []          # (phase, step, source): what ran, for the schedule tests
 
     def forward(self, q, k, v):
