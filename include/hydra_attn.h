@@ -498,6 +498,8 @@ const char* hydra_status_string(int32_t status);
  * Synchronises `cuda_stream` and reports what the kernels of the last call that used `workspace`
  * left in its status word: *device_status is HYDRA_OK or HYDRA_ERR_DEVICE_TIMEOUT, *detail the
  * index of the work item that gave up (or -1). Returns HYDRA_ERR_CUDA if the stream is in error.
+ * A workspace that no call has launched kernels with (none yet, or only calls without any token or pair, which
+ * launch nothing) holds whatever the caller put there: zero it at allocation if it may be polled in that state.
  */
 int32_t hydra_poll_status(void* workspace, void* cuda_stream, int32_t* device_status,
                           int64_t* detail);

@@ -45,7 +45,7 @@ class AttnStep:
         self.dv = torch.empty((T, h, B.D_V), dtype=bf, device=dev)
         ws = max(B.hydra_workspace_bytes(w, self.cu, h, self.pairs)
                  for w in (B.HYDRA_WS_FWD, B.HYDRA_WS_MERGE, B.HYDRA_WS_BWD))
-        self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)
+        self.workspace = torch.zeros(ws, dtype=torch.uint8, device=dev)    # status reads OK before the first launch
         self.has_partials = self.pairs is not None and bool((self.pairs["part_row"] >= 0).any())
 
     def forward(self, q, k, v, stream=None):
