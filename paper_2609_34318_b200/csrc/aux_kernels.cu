@@ -600,10 +600,7 @@ extern "C" int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_
                                            void* cuda_stream)
 {
     using namespace hydra;
-    if (n_seqs < 1 || !cu || n_heads < 1 || !pairs || n_pairs < 1 || part_rows < 1) return HYDRA_ERR_INVALID_ARG;
-    const void* ptrs[] = {o_part, lse_part, out, lse};
-    for (const void* p : ptrs)
-        if (!p || (reinterpret_cast<uintptr_t>(p) & 15u)) return HYDRA_ERR_INVALID_ARG;
+    if (n_seqs < 1 || !cu || n_heads < 1 || !pairs || n_pairs < 1 || part_rows < 0) return HYDRA_ERR_INVALID_ARG;
     if (cu[0] != 0) return HYDRA_ERR_INVALID_ARG;
     for (int b = 0; b < n_seqs; ++b)
         if (cu[b + 1] < cu[b]) return HYDRA_ERR_INVALID_ARG;
@@ -655,7 +652,10 @@ extern "C" int32_t hydra_lse_merge_noalloc(const void* o_part, const float* lse_
         }
         i = j;
     }
-    if (n_items == 0) return HYDRA_OK;
+    if (n_items == 0) return HYDRA_OK;                 // no chunk has partials: nothing to merge, as in hydra_lse_merge
+    const void* ptrs[] = {o_part, lse_part, out, lse};
+    for (const void* p : ptrs)
+        if (!p || (reinterpret_cast<uintptr_t>(p) & 15u)) return HYDRA_ERR_INVALID_ARG;
     // as in hydra_lse_merge: the partials may not share rows of the partial buffers, and two merged q
     // chunks may not write the same rows of out / lse (std::sort works in place: no heap)
     std::sort(part_iv, part_iv + n_parts);

@@ -35,7 +35,8 @@ def _compare(out, lse, ref_out, ref_lse, label):
     assert rows.any()
     assert np.array_equal(np.isneginf(got_l[rows]), np.isneginf(ref_lse[rows])), f"{label}: -inf pattern of LSE"
     fin = rows & np.isfinite(ref_lse)
-    assert np.abs(got_l[fin] - ref_lse[fin]).max() <= TOL_LSE, label
+    if fin.any():
+        assert np.abs(got_l[fin] - ref_lse[fin]).max() <= TOL_LSE, label
     sel = rows.T                                             # [T, h]
     assert np.isfinite(got_o[sel]).all(), f"{label}: a partial without keys leaked into O"
     # one rounding of the fp32 result to bf16, plus the approximate exponentials of the weights

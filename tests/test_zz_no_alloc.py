@@ -112,3 +112,23 @@ def test_no_alloc_merge_rejects_overlapping_rows_like_the_ordinary_merge():
         s = fn(dummy, dummy, part_rows, cu, 1, bad, dummy, dummy, *extra, check=False)
         assert s == P.HYDRA_ERR_INVALID_ARG, (fn.__name__, s)
     assert P.hydra_launch_count() == n0
+
+
+@pytest.mark.parametrize("lengths,cp_r", [([1], 3), ([1, 1, 1], 2)])
+def test_no_alloc_merge_with_nothing_to_merge_is_a_no_op_like_the_ordinary_merge(lengths, cp_r):
+    """One-token sequences: every q chunk that exists has a single pair, which wrote out / lse itself. Both
+    entry points return OK without a launch and without touching anything, whatever the partial buffers are."""
+    import paper_2609_34318_b200 as P
+    cu = hw.cu_seqlens(lengths)
+    T = int(cu[-1])
+    pairs, part_rows, _, _ = P.hydra_zigzag_pairs(cu, cp_r)
+    assert part_rows == 0 and (pairs["part_row"] < 0).all()
+    out = torch.full((T, 2, hw.D_V), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((2, T), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    n0 = P.hydra_launch_count()
+    assert P.hydra_lse_merge(None, None, 0, cu, 2, pairs, out, lse, ws, check=False) == P.HYDRA_OK
+    assert P.hydra_lse_merge_noalloc(None, None, 0, cu, 2, pairs, out, lse, check=False) == P.HYDRA_OK
+    torch.cuda.synchronize()
+    assert P.hydra_launch_count() == n0
+    assert torch.isnan(out.float()).all() and torch.isnan(lse).all()
