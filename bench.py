@@ -820,8 +820,8 @@ NCU_DRAM_BYTES_PER_LAUNCH = {
     # with the dS hand-off: 1.76 GB of the key-side kernel's writes and of the query-side kernel's reads are dS
     ("bwd_dkv", "packed32k"): (2831744000, ("bwd_kernels.cu",) + _TENSOR_DEPS, "1fb384b3f8f2", "2026-11-25"),
     ("bwd_dq", "packed32k"): (2068468000, ("bwd_kernels.cu",) + _TENSOR_DEPS, "1fb384b3f8f2", "2026-11-25"),
-    ("merge", "short64k_split"): (790308000, ("aux_kernels.cu", "hydra_internal.h", "sm100_ptx.cuh"), "86b27c5f119c", "2026-11-25"),
-    ("bwd_prep", "short64k_split"): (1085302000, ("aux_kernels.cu", "hydra_internal.h", "sm100_ptx.cuh"), "86b27c5f119c", "2026-11-25"),
+    ("merge", "short64k_split"): (789849000, ("aux_kernels.cu", "hydra_internal.h", "sm100_ptx.cuh"), "a9b796e47f1c", "2026-11-25"),
+    ("bwd_prep", "short64k_split"): (1086315000, ("aux_kernels.cu", "hydra_internal.h", "sm100_ptx.cuh"), "a9b796e47f1c", "2026-11-25"),
 }
 
 
