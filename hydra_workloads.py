@@ -160,6 +160,10 @@ def workload(name: str) -> Workload:
     if name == "ring256k":
         return Workload("ring256k", [262144], 16, cp_r=4,
                         note="one 256K sequence, outer ring of 4: 8 zigzag chunks, 36 pairs, merged")
+    if name == "ring64k":
+        return Workload("ring64k", [65536], 16, cp_r=1,
+                        note="a slice of the 256K configuration for profiling: one 64K sequence in two of its "
+                             "32K-token chunks, 2 diagonal pairs and 1 full pair, merged")
     if name == "skewed128k":
         return Workload("skewed128k", lengths_skewed(), 16,
                         note="one 96K sequence + Pareto(1.2) tail filling 32K")
@@ -172,5 +176,5 @@ def workload(name: str) -> Workload:
     raise KeyError(name)
 
 
-WORKLOADS = ("tiny", "tiny_split", "packed32k", "ring256k", "skewed128k", "short64k",
+WORKLOADS = ("tiny", "tiny_split", "packed32k", "ring256k", "ring64k", "skewed128k", "short64k",
              "short64k_split")
